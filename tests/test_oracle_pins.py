@@ -1,0 +1,461 @@
+"""Pins of the CPU oracle against what the paper and the mathematics fix (no GPU, no CUDA code).
+
+Each test names the passage of the LOCKS paper it rests on.  A plausible mistake in the oracle
+(dropped term, wrong sign, wrong index, transposed operand, wrong normalisation set) fails at
+least one of them.
+"""
+import itertools
+import math
+
+import numpy as np
+import pytest
+
+import oracle
+from common import read_golden
+
+SM = 1.0 / math.sqrt(128.0)
+rng = np.random.default_rng(1234)
+
+
+def low_rank_page(rank, B=16, d=128, noise=0.0, seed=0):
+    g = np.random.default_rng(seed)
+    mu = g.standard_normal(d)
+    dirs = g.standard_normal((rank, d))
+    a = g.standard_normal((B, rank)) * 3.0
+    return mu + a @ dirs + noise * g.standard_normal((B, d))
+
+
+# ------------------------------------------------------------------ eigensolver (library cross-check)
+
+@pytest.mark.parametrize("n", [2, 5, 16])
+def test_jacobi_matches_numpy_eigh(n):
+    A = rng.standard_normal((n, n))
+    A = A @ A.T
+    lam, U = oracle.eigh_jacobi(A)
+    ref = np.linalg.eigvalsh(A)[::-1]
+    assert np.allclose(lam, ref, rtol=1e-12, atol=1e-12 * abs(ref).max())
+    assert np.allclose(U.T @ U, np.eye(n), atol=1e-12)
+    assert np.allclose(U @ np.diag(lam) @ U.T, A, atol=1e-10 * abs(A).max())
+    w, Q = np.linalg.eigh(A)
+    for l in range(n):  # projectors onto each (simple) eigenvector agree
+        pr = np.outer(U[:, l], U[:, l])
+        qr = np.outer(Q[:, n - 1 - l], Q[:, n - 1 - l])
+        assert np.abs(pr - qr).max() < 1e-9
+
+
+def test_jacobi_degenerate_and_zero():
+    lam, U = oracle.eigh_jacobi(np.zeros((4, 4)))
+    assert np.all(lam == 0) and np.allclose(U, np.eye(4))
+    lam, U = oracle.eigh_jacobi(np.diag([1.0, 3.0, 3.0, 2.0]))
+    assert np.allclose(lam, [3, 3, 2, 1])
+
+
+# ------------------------------------------------------------------ build invariants (Sec. 4 Build; Cor. 2)
+
+@pytest.mark.parametrize("r", [1, 2, 4, 8, 15])
+def test_build_invariants(r):
+    keys = low_rank_page(6, noise=0.1, seed=r)
+    mu, V, C, lam, r_eff = oracle.build_page(keys, r)
+    D = keys - keys.mean(0)
+    assert r_eff == r
+    assert np.allclose(mu, keys.mean(0), atol=1e-13)
+    assert np.allclose(V @ V.T, np.eye(r), atol=1e-9)               # orthonormal basis
+    assert np.allclose(C.sum(0), 0, atol=1e-9)                      # centred coefficients
+    assert np.allclose(C.T @ C, np.diag(lam[:r]), atol=1e-8 * lam[0])   # C^T C = Sigma_r^2
+    assert np.allclose(C, D @ V.T, atol=1e-9 * np.sqrt(lam[0]))         # c_i = V^T delta_i
+    assert np.isclose(lam.sum(), (D * D).sum(), rtol=1e-12)             # trace
+    resid = ((D - C @ V) ** 2).sum()
+    assert np.isclose(resid, lam[r:].sum(), rtol=1e-8, atol=1e-9 * lam[0])  # Eckart-Young tail
+    sv = np.linalg.svd(D, compute_uv=False)
+    assert np.allclose(np.sqrt(np.maximum(lam[:15], 0)), sv[:15], rtol=1e-9, atol=1e-9 * sv[0])
+    for l in range(r):  # sign convention
+        assert V[l, np.argmax(np.abs(V[l]))] > 0
+
+
+def test_build_drops_zero_modes():
+    keys = low_rank_page(3, noise=0.0, seed=5)                      # rank(D) = 3
+    mu, V, C, lam, r_eff = oracle.build_page(keys, 8)
+    assert r_eff == 3
+    assert np.all(V[3:] == 0) and np.all(C[:, 3:] == 0)
+    # a centred page never has more than B-1 modes
+    keys = np.random.default_rng(0).standard_normal((16, 128))
+    _, V, C, lam, r_eff = oracle.build_page(keys, 16)
+    assert r_eff == 15 and np.all(V[15] == 0) and np.all(C[:, 15] == 0)
+    # all keys identical: D = 0, nothing kept
+    _, V, C, lam, r_eff = oracle.build_page(np.tile(keys[:1], (16, 1)), 8)
+    assert r_eff == 0 and np.all(V == 0) and np.all(C == 0)
+
+
+# ------------------------------------------------------------------ Eq. (1) against the exact log-mass
+
+def test_full_rank_summary_is_exact():
+    """Prop. 3 / Sec. 4: r >= rank(D_j) reproduces the exact page log-mass."""
+    g = np.random.default_rng(7)
+    keys = g.standard_normal((16, 128)) * 2.0
+    q = g.standard_normal(128) * 1.5
+    mu, V, C, lam, _ = oracle.build_page(keys, 16)
+    assert abs(oracle.score(mu, V, C, q, SM) - oracle.exact_lse(keys, q, SM)) < 1e-10
+    keys = low_rank_page(5, noise=0.0, seed=3)                      # planted rank 5 <= r = 8
+    mu, V, C, lam, _ = oracle.build_page(keys, 8)
+    assert abs(oracle.score(mu, V, C, q, SM) - oracle.exact_lse(keys, q, SM)) < 1e-10
+    mu, V, C, lam, _ = oracle.build_page(keys, 4)                   # r < rank: no longer exact
+    assert abs(oracle.score(mu, V, C, q, SM) - oracle.exact_lse(keys, q, SM)) > 1e-4
+
+
+def test_exact_lse_matches_definition():
+    g = np.random.default_rng(8)
+    keys, q = g.standard_normal((16, 128)), g.standard_normal(128)
+    ref = np.log(np.exp(keys @ q * SM).sum())
+    assert abs(oracle.exact_lse(keys, q, SM) - ref) < 1e-12
+    assert abs(oracle.exact_lse(keys[:5], q, SM) - np.log(np.exp(keys[:5] @ q * SM).sum())) < 1e-12
+
+
+def test_score_error_bounds():
+    """Prop. 3: |s^ - s| <= max_i |q_perp . delta_perp_i|/sqrt(d) <= |q_perp| sigma_{r+1}/sqrt(d)
+    <= |q_perp| sqrt(tau_r)/sqrt(d), on every page and query tried."""
+    g = np.random.default_rng(9)
+    for trial in range(40):
+        r = [2, 4, 8][trial % 3]
+        keys = low_rank_page(6, noise=0.3, seed=100 + trial)
+        q = g.standard_normal(128) * (1 + trial % 4)
+        mu, V, C, lam, _ = oracle.build_page(keys, r)
+        err = abs(oracle.score(mu, V, C, q, SM) - oracle.exact_lse(keys, q, SM))
+        D = keys - mu
+        dperp = D - C @ V
+        qperp = q - V.T @ (V @ q)
+        b1 = np.abs(dperp @ qperp).max() * SM
+        b2 = np.linalg.norm(qperp) * math.sqrt(lam[r]) * SM
+        b3 = np.linalg.norm(qperp) * math.sqrt(lam[r:].sum()) * SM
+        assert err <= b1 * (1 + 1e-9) + 1e-12
+        assert b1 <= b2 * (1 + 1e-9) and b2 <= b3 * (1 + 1e-9)
+        assert err > 0  # the bound is not vacuous: truncation does perturb the score
+
+
+def test_score_closed_forms():
+    g = np.random.default_rng(10)
+    q = g.standard_normal(128)
+    key = g.standard_normal(128)
+    # identical keys: s^ = q.mu/sqrt(d) + log B
+    mu, V, C, _, _ = oracle.build_page(np.tile(key, (16, 1)), 8)
+    assert abs(oracle.score(mu, V, C, q, SM) - (SM * q @ key + math.log(16))) < 1e-12
+    # rank-1 deviations: r = 1 is exact
+    keys = key + np.outer(g.standard_normal(16), g.standard_normal(128))
+    mu, V, C, _, _ = oracle.build_page(keys, 1)
+    assert abs(oracle.score(mu, V, C, q, SM) - oracle.exact_lse(keys, q, SM)) < 1e-10
+    # a single rank-r score by hand: mu = 0, V = e_0, c_i = i  ->  log sum_i exp(q_0 i / sqrt d)
+    V = np.zeros((1, 128)); V[0, 0] = 1.0
+    C = np.arange(16, dtype=float).reshape(16, 1)
+    ref = np.log(np.exp(q[0] * np.arange(16) * SM).sum())
+    assert abs(oracle.score(np.zeros(128), V, C, q, SM) - ref) < 1e-12
+    # the centroid term enters once, inside the scale
+    assert abs(oracle.score(key, V, C, q, SM) - (ref + SM * q @ key)) < 1e-12
+
+
+def test_score_symmetries():
+    """Token permutation and a common rotation of keys and query leave s^ unchanged."""
+    g = np.random.default_rng(11)
+    keys = low_rank_page(6, noise=0.2, seed=21)
+    q = g.standard_normal(128)
+    mu, V, C, _, _ = oracle.build_page(keys, 4)
+    s0 = oracle.score(mu, V, C, q, SM)
+    perm = g.permutation(16)
+    mu, V, C, _, _ = oracle.build_page(keys[perm], 4)
+    assert abs(oracle.score(mu, V, C, q, SM) - s0) < 1e-10
+    Q, _ = np.linalg.qr(g.standard_normal((128, 128)))
+    mu, V, C, _, _ = oracle.build_page(keys @ Q, 4)
+    assert abs(oracle.score(mu, V, C, q @ Q, SM) - s0) < 1e-9
+
+
+# ------------------------------------------------------------------ isotropic null (paper-printed numbers)
+
+def test_isotropic_null_matches_paper():
+    med, mean, std = read_golden("isotropic_null.txt")[0]
+    g = np.random.default_rng(2024)
+    frac = np.empty(20000)
+    for i in range(20000):
+        keys = g.standard_normal((16, 128))
+        D = keys - keys.mean(0)
+        lam, _ = oracle.eigh_jacobi(D @ D.T)
+        frac[i] = lam[:8].sum() / lam.sum()
+    assert abs(np.median(frac) - med) < 0.002
+    assert abs(frac.mean() - mean) < 0.002
+    assert abs(frac.std() - std) < 0.001
+
+
+# ------------------------------------------------------------------ storage formats
+
+def test_payload_bytes_match_paper_table():
+    for r, stored, alpha, ceil_, red, share in read_golden("payload_table.txt"):
+        r = int(r)
+        nbytes = oracle.summary_payload_bytes(oracle.FMT_I4, r)
+        assert nbytes == int(stored)
+        assert round(nbytes / 8192, 3) == alpha
+        assert round(8192 / nbytes) == int(ceil_)
+        N, b = 1 << 20, 2048
+        dense = N * 512
+        ours = (N // 16) * nbytes + b * 512
+        assert round(dense / ours, 1) == red
+        assert round(100 * (N // 16) * nbytes / ours) == int(share)
+        assert oracle.summary_stride_bytes(oracle.FMT_I4, r) % 16 == 0
+        assert 0 <= oracle.summary_stride_bytes(oracle.FMT_I4, r) - nbytes < 16
+    for B, pct in read_golden("pagesize_payload.txt"):
+        B = int(B)
+        logical = 128 * 8 // 2 + B * 8 + 128
+        assert round(100 * logical / (B * 512), 1) == pct
+    assert oracle.summary_payload_bytes(oracle.FMT_F32, 8) == 5120
+
+
+def test_half_conversion_matches_numpy():
+    g = np.random.default_rng(3)
+    xs = np.concatenate([g.standard_normal(2000) * 10.0 ** g.integers(-9, 5, 2000),
+                         [0.0, 1.0, 65504.0, 65519.9, 65520.0, 1e-8, 5.96e-8, 2.98e-8, 2.99e-8, 6.1e-5]])
+    for x in xs:
+        bits = oracle.double_to_half(float(x))
+        ref = np.float16(x)
+        assert bits == int(ref.view(np.uint16)), (x, bits, ref)
+        if np.isfinite(ref):
+            assert oracle.half_to_double(bits) == float(ref)
+
+
+@pytest.mark.parametrize("r", [2, 4, 8])
+def test_i4_pack_roundtrip_and_quantiser(r):
+    keys = low_rank_page(6, noise=0.2, seed=40 + r) + 3.0
+    mu, V, C, _, _ = oracle.build_page(keys, r)
+    blob = oracle.pack(oracle.FMT_I4, mu, V, C)
+    assert blob.size == oracle.summary_stride_bytes(oracle.FMT_I4, r)
+    assert np.all(blob[oracle.summary_payload_bytes(oracle.FMT_I4, r):] == 0)
+    cV, cC, cMu, sV, sC, sMu = oracle.unpack_codes(r, blob)
+    mu2, V2, C2 = oracle.unpack(oracle.FMT_I4, r, blob)
+    assert np.abs(cV).max() <= 7 and np.abs(cC).max() <= 127 and np.abs(cMu).max() <= 127
+    for l in range(r):   # one fp16 scale per basis column, abs-max symmetric, round-half-even codes
+        assert sV[l] == float(np.float16(np.abs(V[l]).max() / 7))
+        assert np.array_equal(cV[l], np.clip(np.rint(V[l] / sV[l]), -7, 7))
+        assert np.allclose(V2[l], cV[l] * sV[l], rtol=0, atol=0)
+        assert np.abs(V2[l] - V[l]).max() <= 0.5 * sV[l] * (1 + 1e-3) + 1e-12
+    for i in range(16):  # one scale per coefficient row
+        assert sC[i] == float(np.float16(np.abs(C[i]).max() / 127))
+        assert np.array_equal(cC[i], np.clip(np.rint(C[i] / sC[i]), -127, 127))
+        assert np.array_equal(C2[i], cC[i] * sC[i])
+    assert sMu == float(np.float16(np.abs(mu).max() / 127))
+    assert np.array_equal(cMu, np.clip(np.rint(mu / sMu), -127, 127))
+    assert np.array_equal(mu2, cMu * sMu)
+
+
+@pytest.mark.parametrize("r", [2, 4, 8])
+def test_i4_layout_is_a_bijection(r):
+    """Every payload byte/nibble is owned by exactly one entry: flipping one entry changes exactly
+    one nibble (basis) or one byte (coefficients, centroid) and nothing else."""
+    V = np.zeros((r, 128)); C = np.zeros((16, r)); mu = np.zeros(128)
+    V[:, 0] = 7.0; C[:, 0] = 127.0; mu[0] = 127.0       # fixes every scale at 1.0
+    base = oracle.pack(oracle.FMT_I4, mu, V, C)
+    seen = set()
+    for l in range(r):
+        for c in range(1, 128):
+            V2 = V.copy(); V2[l, c] = 3.0
+            diff = np.nonzero(oracle.pack(oracle.FMT_I4, mu, V2, C) != base)[0]
+            assert diff.size == 1
+            b = oracle.pack(oracle.FMT_I4, mu, V2, C)[diff[0]] ^ base[diff[0]]
+            key = (int(diff[0]), "lo" if b < 16 else "hi")
+            assert key not in seen
+            seen.add(key)
+    for i in range(16):
+        for l in range(1, r):
+            C2 = C.copy(); C2[i, l] = 5.0
+            diff = np.nonzero(oracle.pack(oracle.FMT_I4, mu, V, C2) != base)[0]
+            assert diff.size == 1 and ("c", int(diff[0])) not in seen
+            seen.add(("c", int(diff[0])))
+    for c in range(1, 128):
+        mu2 = mu.copy(); mu2[c] = 9.0
+        diff = np.nonzero(oracle.pack(oracle.FMT_I4, mu2, V, C) != base)[0]
+        assert diff.size == 1 and ("m", int(diff[0])) not in seen
+        seen.add(("m", int(diff[0])))
+
+
+def test_zero_scale_gives_zero_codes():
+    blob = oracle.pack(oracle.FMT_I4, np.zeros(128), np.zeros((8, 128)), np.zeros((16, 8)))
+    mu, V, C = oracle.unpack(oracle.FMT_I4, 8, blob)
+    assert not mu.any() and not V.any() and not C.any()
+    assert abs(oracle.score(mu, V, C, np.ones(128), SM) - math.log(16)) < 1e-12
+
+
+def test_f32_format_roundtrip():
+    keys = low_rank_page(6, noise=0.2, seed=77)
+    mu, V, C, _, _ = oracle.build_page(keys, 8)
+    mu2, V2, C2 = oracle.unpack(oracle.FMT_F32, 8, oracle.pack(oracle.FMT_F32, mu, V, C))
+    assert np.array_equal(mu2, mu.astype(np.float32)) and np.array_equal(V2, V.astype(np.float32))
+    assert np.array_equal(C2, C.astype(np.float32))
+
+
+# ------------------------------------------------------------------ combine + selection (Cor. 4, Thm. 1)
+
+def shares(s):
+    e = np.exp(s - s.max(axis=1, keepdims=True))
+    return e / e.sum(axis=1, keepdims=True)
+
+
+def test_select_brute_force_maximises_group_coverage():
+    """Cor. 4: among k-sets containing sink and most recent page, the selected set maximises the
+    group-mean coverage sum_{j in S} m_bar_j (shares normalised over the candidates)."""
+    g = np.random.default_rng(12)
+    for trial in range(30):
+        P = int(g.integers(4, 12)); G = int(g.integers(1, 5)); k = int(g.integers(2, min(6, P)))
+        s = g.standard_normal((G, P)) * 3
+        ids, cnt, logm = oracle.select_one(s, P, k)
+        assert cnt == k and ids[0] == 0 and ids[k - 1] == P - 1 and np.all(np.diff(ids[:k]) > 0)
+        mbar = shares(s[:, 1:P - 1]).mean(0)                       # candidate pages 1..P-2
+        assert np.allclose(np.exp(logm[1:P - 1]), mbar, rtol=1e-12)
+        best = max(sum(mbar[j - 1] for j in comb)
+                   for comb in itertools.combinations(range(1, P - 1), k - 2))
+        got = sum(mbar[j - 1] for j in ids[1:k - 1])
+        assert abs(got - best) < 1e-13
+
+
+def test_select_edge_cases_and_ties():
+    s = np.zeros((2, 10))
+    ids, cnt, _ = oracle.select_one(s, 10, 4)                      # all tied: lower indices win
+    assert cnt == 4 and ids.tolist() == [0, 1, 2, 9]
+    ids, cnt, _ = oracle.select_one(s, 3, 4)                       # P <= k: every page
+    assert cnt == 3 and ids.tolist() == [0, 1, 2, -1]
+    ids, cnt, _ = oracle.select_one(s, 1, 4)
+    assert cnt == 1 and ids.tolist() == [0, -1, -1, -1]
+    ids, cnt, _ = oracle.select_one(s, 10, 2)                      # k = 2: sink + recent only
+    assert cnt == 2 and ids.tolist() == [0, 9]
+    # a head-wise constant shift changes no share and no set (Eq. 2 factorisation remark)
+    g = np.random.default_rng(13)
+    s = g.standard_normal((4, 40)) * 2
+    a, _, la = oracle.select_one(s, 40, 8)
+    b, _, lb = oracle.select_one(s + g.standard_normal((4, 1)) * 50, 40, 8)
+    assert np.array_equal(a, b) and np.allclose(la[1:39], lb[1:39], atol=1e-10)
+    # the sink and last page's own scores are never read
+    s2 = s.copy(); s2[:, 0] = 1e9; s2[:, 39] = -1e9
+    c, _, _ = oracle.select_one(s2, 40, 8)
+    assert np.array_equal(a, c)
+
+
+def test_share_sandwich_and_retention():
+    """Thm. 1 steps 2-3: |log m^bar - log m_bar| <= 2 eta and the estimated-share set keeps at least
+    e^{-4 eta} of the candidate coverage of the exact-share set."""
+    g = np.random.default_rng(14)
+    for trial in range(20):
+        G, P, k = 4, 60, 10
+        s = g.standard_normal((G, P)) * 4
+        eta = 0.05 * (1 + trial % 5)
+        shat = s + g.uniform(-eta, eta, size=s.shape)
+        ia, _, la = oracle.select_one(s, P, k)
+        ib, _, lb = oracle.select_one(shat, P, k)
+        assert np.abs(la[1:P - 1] - lb[1:P - 1]).max() <= 2 * eta + 1e-12
+        m = np.exp(la)
+        cov_exact = m[ia[1:k - 1]].sum()
+        cov_est = m[ib[1:k - 1]].sum()
+        assert cov_est >= math.exp(-4 * eta) * cov_exact - 1e-12
+
+
+# ------------------------------------------------------------------ attention (Sec. 3, Lemma 1)
+
+def tiny_cache(T=70, Hq=4, Hkv=2, B=16, d=128, seed=0, nb_extra=3):
+    g = np.random.default_rng(seed)
+    P = -(-T // B)
+    nb = P + nb_extra
+    k = g.standard_normal((nb, Hkv, B, d)).astype(np.float32)
+    v = g.standard_normal((nb, Hkv, B, d)).astype(np.float32)
+    bt = g.permutation(nb)[:P].astype(np.int32).reshape(1, P)
+    return oracle.Cache(k, v, bt, np.array([T], np.int32), Hq), g
+
+
+def dense_reference(cache, q, pages):
+    """Textbook softmax attention over the tokens of the given pages, straight from numpy."""
+    B, d, G = cache.B, cache.d, cache.Hq // cache.Hkv
+    T = int(cache.seq_lens[0])
+    out = np.zeros((cache.Hq, d)); lse = np.zeros(cache.Hq)
+    for gq in range(cache.Hq):
+        h = gq // G
+        ks, vs = [], []
+        for p in pages:
+            blk = cache.block_table[0, p]
+            n = min(B, T - p * B)
+            ks.append(cache.k[blk, h, :n]); vs.append(cache.v[blk, h, :n])
+        ks, vs = np.concatenate(ks).astype(np.float64), np.concatenate(vs).astype(np.float64)
+        x = ks @ q[0, gq].astype(np.float64) / math.sqrt(d)
+        w = np.exp(x - x.max())
+        out[gq] = (w / w.sum()) @ vs
+        lse[gq] = x.max() + math.log(w.sum())
+    return out, lse
+
+
+def test_attend_matches_textbook_softmax():
+    cache, g = tiny_cache(T=70)
+    q = g.standard_normal((1, 4, 128)).astype(np.float32)
+    out, lse = oracle.attend(cache, q, SM)                          # dense: all 5 pages, 70 tokens
+    ref, rl = dense_reference(cache, q, range(5))
+    assert np.allclose(out[0], ref, atol=1e-12) and np.allclose(lse[0], rl, atol=1e-12)
+    ids = np.array([[[0, 2, 4, -1], [1, 4, -1, -1]]], np.int32)
+    cnt = np.array([[3, 2]], np.int32)
+    out, lse = oracle.attend(cache, q, SM, ids, cnt)
+    for h, pages in enumerate([[0, 2, 4], [1, 4]]):
+        ref, rl = dense_reference(cache, q, pages)
+        assert np.allclose(out[0, 2 * h:2 * h + 2], ref[2 * h:2 * h + 2], atol=1e-12)
+        assert np.allclose(lse[0, 2 * h:2 * h + 2], rl[2 * h:2 * h + 2], atol=1e-12)
+
+
+def test_attend_special_cases():
+    # a single token: the output is that token's value
+    cache, g = tiny_cache(T=1)
+    q = g.standard_normal((1, 4, 128)).astype(np.float32)
+    out, lse = oracle.attend(cache, q, SM)
+    blk = cache.block_table[0, 0]
+    for gq in range(4):
+        assert np.allclose(out[0, gq], cache.v[blk, gq // 2, 0], atol=1e-12)
+        assert abs(lse[0, gq] - SM * float(cache.k[blk, gq // 2, 0].astype(np.float64) @ q[0, gq])) < 1e-9
+    # zero query: uniform weights, output is the mean value, lse = log T
+    cache, g = tiny_cache(T=37)
+    out, lse = oracle.attend(cache, np.zeros((1, 4, 128), np.float32), SM)
+    ref, _ = dense_reference(cache, np.zeros((1, 4, 128), np.float32), range(3))
+    assert np.allclose(out[0], ref, atol=1e-12) and np.allclose(lse, math.log(37), atol=1e-12)
+
+
+def test_coverage_identity_and_bound():
+    """Lemma 1(i): o - o_S = eps (vbar_Sc - vbar_S) exactly, and |o - o_S| <= 2R(1 - gamma_S)."""
+    cache, g = tiny_cache(T=160, Hq=2, Hkv=2)
+    q = g.standard_normal((1, 2, 128)).astype(np.float32) * 3
+    P = 10
+    full, lse_full = oracle.attend(cache, q, SM)
+    for trial in range(5):
+        S = sorted(g.choice(P, size=4, replace=False).tolist())
+        Sc = [p for p in range(P) if p not in S]
+        ids = np.array([[S, S]], np.int32); cnt = np.array([[4, 4]], np.int32)
+        oS, lS = oracle.attend(cache, q, SM, ids, cnt)
+        idc = np.array([[Sc, Sc]], np.int32); cnc = np.array([[6, 6]], np.int32)
+        oC, lC = oracle.attend(cache, q, SM, idc, cnc)
+        gamma = np.exp(lS - lse_full)                               # coverage of S
+        assert np.allclose(np.exp(lS - lse_full) + np.exp(lC - lse_full), 1, atol=1e-12)
+        eps = 1 - gamma
+        assert np.allclose(full - oS, eps[..., None] * (oC - oS), atol=1e-12)
+        R = np.linalg.norm(cache.v.astype(np.float64), axis=-1).max()
+        assert np.all(np.linalg.norm(full - oS, axis=-1) <= 2 * R * eps + 1e-12)
+
+
+def test_full_budget_equals_dense_and_pipeline_runs():
+    """Budget >= all pages selects everything, so the sparse output is the dense one; with a small
+    budget the pipeline returns sink + recent + top pages."""
+    import torch
+    import locks_synth
+    from common import oracle_cache, fmt_code
+    w = locks_synth.config0().with_(seq_lens=[300], budget=4096, carriers=2)
+    case = locks_synth.make_case(w)
+    cache = oracle_cache(case)
+    q = case.q.numpy()
+    summ = oracle.build_summaries(cache, w.rank, fmt_code(w))
+    ids, cnt, out, lse = oracle.decode_step(cache, q, w.rank, fmt_code(w), summ, SM, w.k)
+    P = 19
+    assert cnt[0, 0] == P and ids[0, 0, :P].tolist() == list(range(P))
+    dense, dl = oracle.attend(cache, q, SM)
+    assert np.allclose(out, dense, atol=1e-13) and np.allclose(lse, dl, atol=1e-13)
+    ids, cnt, out, lse = oracle.decode_step(cache, q, w.rank, fmt_code(w), summ, SM, 6)
+    assert cnt[0, 0] == 6 and ids[0, 0, 0] == 0 and ids[0, 0, 5] == P - 1
+    for cp in case.carrier_pages[0]:                                # planted carriers are found
+        assert cp in ids[0, 0].tolist()
+    # the estimated masses follow the exact ones within the proven bound on this data
+    shat = oracle.page_logmass(cache, q, w.rank, fmt_code(w), summ, SM)
+    sex = oracle.page_logmass(cache, q, w.rank, fmt_code(w), None, SM, exact=True)
+    assert np.nanmax(np.abs(shat - sex)[:, :, :P - 1]) < 0.5
+    assert np.all(np.isnan(shat[:, :, P - 1:]))
