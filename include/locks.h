@@ -1,0 +1,166 @@
+/*
+ * liblocks -- per-step decode hot path of the LOCKS page-local spectral-summary selector,
+ * hand-written CUDA for NVIDIA B200 (sm_100a).  C ABI: plain pointers and sizes only.
+ *
+ * Notation (the paper's): B tokens per page, d head dimension, Hq query heads, Hkv KV heads,
+ * G = Hq/Hkv, T tokens of a sequence including the one being decoded, P = ceil(T/B) pages,
+ * b token budget per KV head, k = ceil(b/B) page budget, r summary rank.
+ *
+ * Conventions shared by every call
+ *  - Pointers are DEVICE pointers unless the parameter name ends in _host.  The caller owns every
+ *    buffer, including the workspace handed to locks_create(); the library allocates no device
+ *    memory, never frees caller memory and keeps no caller pointer between calls except the
+ *    workspace.
+ *  - Every call only enqueues kernels (and, for the *_host variants, async copies) on `stream`
+ *    (a cudaStream_t passed as void*), does not synchronise unless stated, and launches a fixed
+ *    grid that depends only on the configuration and `batch`: lengths and page tables are read
+ *    on the device, so a captured CUDA graph can be replayed as the sequences grow.
+ *  - Return value: LOCKS_OK or a negative LOCKS_ERR_* code.  Argument errors are found on the
+ *    host before anything is launched.  Problems only the device can see (a block id outside the
+ *    cache, a bounded wait that expired) set a sticky status word in the workspace, the affected
+ *    kernel skips that piece of work, and locks_poll_status() reports it.  Nothing traps.
+ *  - Precondition of locks_select / locks_decode_step: every candidate page (1 .. P-2) of every
+ *    request has a summary built by locks_build_summaries (locks_decode_step maintains this).
+ */
+#ifndef LOCKS_H_
+#define LOCKS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define LOCKS_OK 0
+#define LOCKS_ERR_INVALID_ARG (-1)
+#define LOCKS_ERR_UNSUPPORTED (-2)
+#define LOCKS_ERR_WORKSPACE (-3)
+#define LOCKS_ERR_CUDA (-4)
+#define LOCKS_ERR_TIMEOUT (-5)
+#define LOCKS_ERR_BAD_BLOCK (-6)
+
+#define LOCKS_F32 0
+#define LOCKS_BF16 1
+
+#define LOCKS_FMT_F32 0 /* summary stored as fp32 mu, V, C                               */
+#define LOCKS_FMT_I4 1  /* int4 basis, int8 coefficients + centroid, fp16 scales (r8i4)  */
+
+typedef struct locks_ctx locks_ctx;
+typedef void *locks_stream; /* cudaStream_t */
+
+typedef struct {
+  int32_t head_dim;          /* d; 128                                                        */
+  int32_t page_size;         /* B; 16                                                         */
+  int32_t num_q_heads;       /* Hq                                                            */
+  int32_t num_kv_heads;      /* Hkv, Hq % Hkv == 0, G = Hq/Hkv <= 16                          */
+  int32_t rank;              /* r: I4 format 2|4|8, F32 format 1..16                          */
+  int32_t summary_fmt;       /* LOCKS_FMT_*                                                   */
+  int32_t kv_dtype;          /* LOCKS_F32 | LOCKS_BF16 (K, V, k_new, v_new)                   */
+  int32_t q_dtype;           /* LOCKS_F32 | LOCKS_BF16 (q and out); must equal kv_dtype       */
+  int32_t max_batch;         /* largest `batch` any call will pass                            */
+  int32_t max_pages_per_seq; /* row length of block_table                                     */
+  int32_t budget_tokens;     /* b; k = ceil(b/B) >= 2                                         */
+  float sm_scale;            /* logit scale, 1/sqrt(d) in the paper                           */
+} locks_config;
+
+/* Paged KV cache view.  Element (block, kv head, token-in-page, dim) of K lives at
+ * k[block*stride_block + head*stride_head + token*stride_token + dim] (strides in ELEMENTS; dims
+ * are contiguous), likewise V.  Both [block][head][token][dim] and [block][token][head][dim] fit.
+ * For 16-byte vector loads the strides must be multiples of 8 elements and the bases 16-byte
+ * aligned. */
+typedef struct {
+  void *k, *v;
+  int64_t stride_block, stride_head, stride_token;
+  int32_t num_blocks;
+  const int32_t *block_table; /* [max_batch][max_pages_per_seq] logical page -> physical block */
+  int32_t *seq_lens;          /* [max_batch] tokens in each sequence (see each call)           */
+} locks_kv;
+
+/* Bytes of one stored summary, per (physical block, KV head), padded to a multiple of 16.
+ * I4 format: 82 r + 162 payload bytes at B=16, d=128 (818 / 490 / 326 at r = 8 / 4 / 2: the
+ * paper's stored-payload table, App. C.1), i.e. d r/2 int4 basis + B r int8 coefficients + d int8
+ * centroid + (r + B + 1) fp16 scales (Sec. 4 "Build").  F32 format: 4 (d + r d + B r).
+ * The summaries buffer is [num_blocks][Hkv][locks_summary_bytes]. 0 on an invalid config. */
+size_t locks_summary_bytes(const locks_config *cfg);
+
+/* Bytes of device workspace locks_create() needs for this configuration (256-byte aligned
+ * base).  0 on an invalid config. */
+size_t locks_workspace_bytes(const locks_config *cfg);
+
+/* Validate the configuration, record it and the workspace pointer, zero the status word (one
+ * small async memset on the default stream followed by a synchronise).  The context is a small
+ * host object; *out must be released with locks_destroy().  Errors: INVALID_ARG (bad field, NULL),
+ * UNSUPPORTED (shape the kernels do not cover: d != 128, B != 16, G > 16, mixed dtypes, I4 rank
+ * not in {2,4,8}), WORKSPACE (ws_bytes too small or misaligned). */
+int locks_create(const locks_config *cfg, void *workspace, size_t ws_bytes, locks_ctx **out);
+int locks_destroy(locks_ctx *ctx);
+
+/* Summary build (Sec. 4 "Build (once, when a page completes)"): for each request b < batch, each
+ * KV head and each COMPLETE page p with page_begin[b] <= p < page_end[b] (p < floor(T_b/B)):
+ * centre the page's B keys, eigendecompose the B x B Gram of the deviations, keep r modes
+ * (C = U_r Sigma_r, V = D^T U_r Sigma_r^-1, zero modes dropped), quantise and store the blob at
+ * summaries[block][head].  page_begin == page_end == NULL: all complete pages.
+ * seq_lens[b] = T_b.  Arithmetic fp32. */
+int locks_build_summaries(locks_ctx *ctx, const locks_kv *kv, int batch, const int32_t *page_begin,
+                          const int32_t *page_end, void *summaries, locks_stream stream);
+
+/* Stage A, "score-then-select" (Sec. 4 "Score (every step)", Eq. 1; share-average combine;
+ * App. E): for every request and query head, s^_j(q_g) for all pages j <= P-2 from the resident
+ * summaries; shares normalised over the candidates 1..P-2; m_bar_j = mean over the group; per KV
+ * head keep page 0, page P-1 and the top k-2 candidates by log m_bar_j (ties: lower index).
+ * P <= k keeps every page.
+ *   q            [batch][Hq][d] (q_dtype)
+ *   page_ids     [batch][Hkv][k] int32 logical page ids, ascending, -1 padded
+ *   page_count   [batch][Hkv] int32
+ *   page_logmass  optional [batch][Hq][max_pages_per_seq] fp32: s^ for pages 0..P-2 (rest untouched)
+ *   page_logshare optional [batch][Hkv][max_pages_per_seq] fp32: log m_bar_j for pages 1..P-2
+ * seq_lens[b] = T_b. */
+int locks_select(locks_ctx *ctx, const void *q, const void *summaries, const locks_kv *kv, int batch,
+                 int32_t *page_ids, int32_t *page_count, float *page_logmass, float *page_logshare,
+                 locks_stream stream);
+
+/* Stage B, sparse paged attention (Sec. 3 "Decode-time attention"; App. E): for every query head,
+ * softmax(q.k_i/sqrt(d))-weighted mean of v_i over the tokens i < T_b of the listed pages
+ * (split over CTAs, partial results merged by log-sum-exp).  page_ids == NULL: every page, i.e.
+ * dense flash-decode over the whole cache (the dense baseline).
+ *   out [batch][Hq][d] (q_dtype), lse optional [batch][Hq] fp32 (natural log). */
+int locks_sparse_attend(locks_ctx *ctx, const void *q, const locks_kv *kv, int batch,
+                        const int32_t *page_ids, const int32_t *page_count, void *out, float *lse,
+                        locks_stream stream);
+
+/* One fused decode step for one attention layer (App. E, Fig. 5), legal under stream capture:
+ *   1. if k_new != NULL: write k_new/v_new [batch][Hkv][d] at position seq_lens[b] of each
+ *      sequence and increment seq_lens[b] (so afterwards seq_lens[b] = T_b counts the new token);
+ *      if k_new == NULL the cache and seq_lens already include the token being decoded;
+ *   2. locks_select on the resident summaries;  3. locks_sparse_attend on the selected pages;
+ *   4. if a page became complete at this step (T_b % B == 0) build its summary, so that it is a
+ *      candidate from the next step on (the newly written token is never scored, App. E(i)).
+ * page_ids / page_count may be NULL (kept in the workspace). */
+int locks_decode_step(locks_ctx *ctx, const void *q, const void *k_new, const void *v_new,
+                      locks_kv *kv, void *summaries, int batch, void *out, int32_t *page_ids,
+                      int32_t *page_count, locks_stream stream);
+
+/* The same step for a caller whose per-step tensors live in HOST memory (pinned for the copies
+ * to be asynchronous): copies q_host (and k_new_host / v_new_host if given) to staging space in
+ * the workspace, runs locks_decode_step, copies out back to out_host (and the page ids / counts
+ * if page_ids_host / page_count_host are given) and synchronises the stream before returning.
+ * The cache, summaries, block table and seq_lens stay on the device. */
+int locks_decode_step_host(locks_ctx *ctx, const void *q_host, const void *k_new_host,
+                           const void *v_new_host, locks_kv *kv, void *summaries, int batch,
+                           void *out_host, int32_t *page_ids_host, int32_t *page_count_host,
+                           locks_stream stream);
+
+/* Copy the sticky device status word to the host and clear it.  Synchronises the stream.
+ * *status_host: LOCKS_OK or the first LOCKS_ERR_* a kernel recorded. */
+int locks_poll_status(locks_ctx *ctx, int32_t *status_host, locks_stream stream);
+
+/* Number of kernels the last call on this context enqueued (for launch accounting). */
+int locks_last_launch_count(const locks_ctx *ctx);
+
+const char *locks_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LOCKS_H_ */

@@ -256,10 +256,10 @@ static int quant_code(double x, double scale, int qmax) {
  *   [basis d*r/2][coefficients 16 r][centroid d][sC 16 x fp16][sV r x fp16][sMu fp16]
  * Codes are stored offset-binary: nibble = code + 8, byte = code + 128. */
 static void i4_basis_pos(int l, int c, int d, int *byte, int *shift) {
-  int s = c >> 4, kr = c & 15, half = kr >> 3, t = (kr & 7) >> 1, e = kr & 1;
+  /* dims are split into 4 contiguous quarters t; inside a quarter, group s covers 4 dims */
+  int Q = d / 4, t = c / Q, w = c % Q, s = w >> 2, half = (w >> 1) & 1, e = w & 1;
   int j = s >> 1, i = ((s & 1) << 1) | half, nib = i + 4 * e;
-  int words = d / 32; /* 32-bit words per (rank, t) lane group */
-  *byte = (l * 4 + t) * (4 * words) + j * 4 + (nib >> 1);
+  *byte = (l * 4 + t) * (Q / 2) + j * 4 + (nib >> 1);
   *shift = (nib & 1) * 4;
 }
 static int i4_coef_pos(int i, int l, int r) {
@@ -267,8 +267,8 @@ static int i4_coef_pos(int i, int l, int r) {
   return (x * (r / 2) + tp) * 4 + hi * 2 + e;
 }
 static int i4_mu_pos(int c, int d) {
-  int s = c >> 4, kr = c & 15, half = kr >> 3, t = (kr & 7) >> 1, e = kr & 1;
-  return t * (d / 4) + s * 4 + e * 2 + half;
+  int Q = d / 4, t = c / Q, w = c % Q, s = w >> 2, half = (w >> 1) & 1, e = w & 1;
+  return t * Q + s * 4 + e * 2 + half;
 }
 static int i4_sc_pos(int i) {
   int t = (i & 7) >> 1, e = i & 1, hi = i >> 3;

@@ -1,0 +1,10 @@
+"""B200-native LOCKS decode hot path: thin ctypes binding over liblocks.so (C ABI in include/locks.h).
+
+Argument marshalling only -- every step of the path runs in the CUDA kernels of the library.
+PyTorch supplies device memory and streams.  Importing this package never builds or falls back:
+if liblocks.so is missing, `lib()` raises.
+"""
+from .binding import (  # noqa: F401
+    BF16, F32, FMT_F32, FMT_I4, Config, KV, LocksError, Context, lib, library_path,
+    locks_summary_bytes, locks_workspace_bytes, locks_strerror,
+)

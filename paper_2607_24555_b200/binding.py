@@ -1,0 +1,203 @@
+"""ctypes binding of liblocks.so.  Names mirror include/locks.h; tensors are torch CUDA tensors."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "liblocks.so")
+
+F32, BF16 = 0, 1
+FMT_F32, FMT_I4 = 0, 1
+
+SYMBOLS = ["locks_summary_bytes", "locks_workspace_bytes", "locks_create", "locks_destroy",
+           "locks_build_summaries", "locks_select", "locks_sparse_attend", "locks_decode_step",
+           "locks_decode_step_host", "locks_poll_status", "locks_last_launch_count", "locks_strerror"]
+
+
+class LocksError(RuntimeError):
+    pass
+
+
+class Config(C.Structure):
+    _fields_ = [("head_dim", C.c_int32), ("page_size", C.c_int32), ("num_q_heads", C.c_int32),
+                ("num_kv_heads", C.c_int32), ("rank", C.c_int32), ("summary_fmt", C.c_int32),
+                ("kv_dtype", C.c_int32), ("q_dtype", C.c_int32), ("max_batch", C.c_int32),
+                ("max_pages_per_seq", C.c_int32), ("budget_tokens", C.c_int32), ("sm_scale", C.c_float)]
+
+
+class KV(C.Structure):
+    _fields_ = [("k", C.c_void_p), ("v", C.c_void_p), ("stride_block", C.c_int64), ("stride_head", C.c_int64),
+                ("stride_token", C.c_int64), ("num_blocks", C.c_int32), ("block_table", C.c_void_p),
+                ("seq_lens", C.c_void_p)]
+
+
+_lib = None
+
+
+def library_path() -> str:
+    return _LIB_PATH
+
+
+def lib():
+    """Load liblocks.so (built in-tree by paper_2607_24555_b200.build).  Raises if it is missing."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise LocksError(f"{_LIB_PATH} is missing: run `python -m paper_2607_24555_b200.build` "
+                             "(there is no CPU or PyTorch fallback)")
+        L = C.CDLL(_LIB_PATH)
+        vp, i32p = C.c_void_p, C.c_void_p
+        L.locks_summary_bytes.restype = C.c_size_t
+        L.locks_summary_bytes.argtypes = [C.POINTER(Config)]
+        L.locks_workspace_bytes.restype = C.c_size_t
+        L.locks_workspace_bytes.argtypes = [C.POINTER(Config)]
+        L.locks_create.argtypes = [C.POINTER(Config), vp, C.c_size_t, C.POINTER(vp)]
+        L.locks_destroy.argtypes = [vp]
+        L.locks_build_summaries.argtypes = [vp, C.POINTER(KV), C.c_int, i32p, i32p, vp, vp]
+        L.locks_select.argtypes = [vp, vp, vp, C.POINTER(KV), C.c_int, i32p, i32p, vp, vp, vp]
+        L.locks_sparse_attend.argtypes = [vp, vp, C.POINTER(KV), C.c_int, i32p, i32p, vp, vp, vp]
+        L.locks_decode_step.argtypes = [vp, vp, vp, vp, C.POINTER(KV), vp, C.c_int, vp, i32p, i32p, vp]
+        L.locks_decode_step_host.argtypes = [vp, vp, vp, vp, C.POINTER(KV), vp, C.c_int, vp, i32p, i32p, vp]
+        L.locks_poll_status.argtypes = [vp, C.POINTER(C.c_int32), vp]
+        L.locks_last_launch_count.argtypes = [vp]
+        L.locks_strerror.restype = C.c_char_p
+        L.locks_strerror.argtypes = [C.c_int]
+        for fn in ("locks_create", "locks_destroy", "locks_build_summaries", "locks_select", "locks_sparse_attend",
+                   "locks_decode_step", "locks_decode_step_host", "locks_poll_status", "locks_last_launch_count"):
+            getattr(L, fn).restype = C.c_int
+        _lib = L
+    return _lib
+
+
+def locks_strerror(code: int) -> str:
+    return lib().locks_strerror(code).decode()
+
+
+def locks_summary_bytes(cfg: Config) -> int:
+    return int(lib().locks_summary_bytes(C.byref(cfg)))
+
+
+def locks_workspace_bytes(cfg: Config) -> int:
+    return int(lib().locks_workspace_bytes(C.byref(cfg)))
+
+
+def _check(rc: int, what: str):
+    if rc != 0:
+        raise LocksError(f"{what} failed: {locks_strerror(rc)} ({rc})")
+
+
+def _ptr(t):
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    return t.data_ptr()
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        return torch.cuda.current_stream().cuda_stream
+    if isinstance(stream, int):
+        return stream
+    return stream.cuda_stream
+
+
+def make_config(Hq, Hkv, rank, fmt, dtype, max_batch, max_pages, budget, sm_scale=None, d=128, B=16) -> Config:
+    if sm_scale is None:
+        sm_scale = d ** -0.5
+    dt = BF16 if dtype in ("bf16", torch.bfloat16) else F32
+    f = FMT_I4 if fmt == "i4" else FMT_F32
+    return Config(d, B, Hq, Hkv, rank, f, dt, dt, max_batch, max_pages, budget, sm_scale)
+
+
+@dataclass
+class KVView:
+    """A paged cache: torch tensors plus element strides (block, head, token)."""
+    k: torch.Tensor
+    v: torch.Tensor
+    strides: tuple
+    num_blocks: int
+    block_table: torch.Tensor   # [max_batch, max_pages] int32, device
+    seq_lens: torch.Tensor      # [max_batch] int32, device
+
+    def struct(self) -> KV:
+        sb, sh, st = self.strides
+        return KV(self.k.data_ptr(), self.v.data_ptr(), sb, sh, st, self.num_blocks, self.block_table.data_ptr(),
+                  self.seq_lens.data_ptr())
+
+
+class Context:
+    """Owns a locks_ctx and its torch-allocated workspace.  Methods mirror the C entry points."""
+
+    def __init__(self, cfg: Config, device="cuda:0"):
+        self.cfg = cfg
+        self.device = torch.device(device)
+        L = lib()
+        nbytes = locks_workspace_bytes(cfg)
+        if nbytes == 0:
+            raise LocksError("invalid or unsupported configuration")
+        self.summary_bytes = locks_summary_bytes(cfg)
+        self.k = -(-cfg.budget_tokens // cfg.page_size)
+        with torch.cuda.device(self.device):
+            self.workspace = torch.empty(nbytes + 256, dtype=torch.uint8, device=self.device)
+            base = (self.workspace.data_ptr() + 255) // 256 * 256
+            h = C.c_void_p()
+            _check(L.locks_create(C.byref(cfg), base, nbytes, C.byref(h)), "locks_create")
+        self.handle = h
+
+    def close(self):
+        if self.handle:
+            lib().locks_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def new_summaries(self, num_blocks: int) -> torch.Tensor:
+        return torch.zeros(num_blocks, self.cfg.num_kv_heads, self.summary_bytes, dtype=torch.uint8, device=self.device)
+
+    def locks_build_summaries(self, kv: KVView, batch, summaries, page_begin=None, page_end=None, stream=None):
+        s = kv.struct()
+        _check(lib().locks_build_summaries(self.handle, C.byref(s), batch, _ptr(page_begin), _ptr(page_end),
+                                           _ptr(summaries), _stream(stream)), "locks_build_summaries")
+
+    def locks_select(self, q, summaries, kv: KVView, batch, page_ids, page_count, page_logmass=None,
+                     page_logshare=None, stream=None):
+        s = kv.struct()
+        _check(lib().locks_select(self.handle, _ptr(q), _ptr(summaries), C.byref(s), batch, _ptr(page_ids),
+                                  _ptr(page_count), _ptr(page_logmass), _ptr(page_logshare), _stream(stream)),
+               "locks_select")
+
+    def locks_sparse_attend(self, q, kv: KVView, batch, page_ids, page_count, out, lse=None, stream=None):
+        s = kv.struct()
+        _check(lib().locks_sparse_attend(self.handle, _ptr(q), C.byref(s), batch, _ptr(page_ids), _ptr(page_count),
+                                         _ptr(out), _ptr(lse), _stream(stream)), "locks_sparse_attend")
+
+    def locks_decode_step(self, q, k_new, v_new, kv: KVView, summaries, batch, out, page_ids=None, page_count=None,
+                          stream=None):
+        s = kv.struct()
+        _check(lib().locks_decode_step(self.handle, _ptr(q), _ptr(k_new), _ptr(v_new), C.byref(s), _ptr(summaries),
+                                       batch, _ptr(out), _ptr(page_ids), _ptr(page_count), _stream(stream)),
+               "locks_decode_step")
+
+    def locks_decode_step_host(self, q_host, k_new_host, v_new_host, kv: KVView, summaries, batch, out_host,
+                               page_ids_host=None, page_count_host=None, stream=None):
+        s = kv.struct()
+        _check(lib().locks_decode_step_host(self.handle, _ptr(q_host), _ptr(k_new_host), _ptr(v_new_host), C.byref(s),
+                                            _ptr(summaries), batch, _ptr(out_host), _ptr(page_ids_host),
+                                            _ptr(page_count_host), _stream(stream)), "locks_decode_step_host")
+
+    def locks_poll_status(self, stream=None) -> int:
+        st = C.c_int32(0)
+        _check(lib().locks_poll_status(self.handle, C.byref(st), _stream(stream)), "locks_poll_status")
+        return int(st.value)
+
+    def locks_last_launch_count(self) -> int:
+        return int(lib().locks_last_launch_count(self.handle))

@@ -1,0 +1,266 @@
+// C-ABI entry points of liblocks (see include/locks.h for the contract of every call).
+#include <new>
+
+#include "locks_internal.cuh"
+
+namespace {
+
+size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+int validate(const locks_config *c) {
+  if (!c) return LOCKS_ERR_INVALID_ARG;
+  if (c->num_q_heads <= 0 || c->num_kv_heads <= 0 || c->num_q_heads % c->num_kv_heads) return LOCKS_ERR_INVALID_ARG;
+  if (c->max_batch <= 0 || c->max_pages_per_seq <= 0 || c->rank <= 0) return LOCKS_ERR_INVALID_ARG;
+  if (c->page_size <= 0 || c->head_dim <= 0) return LOCKS_ERR_INVALID_ARG;
+  const int k = (c->budget_tokens + c->page_size - 1) / c->page_size;
+  if (c->budget_tokens <= 0 || k < 2) return LOCKS_ERR_INVALID_ARG;
+  if (!(c->sm_scale > 0.f)) return LOCKS_ERR_INVALID_ARG;
+  if (c->summary_fmt != LOCKS_FMT_F32 && c->summary_fmt != LOCKS_FMT_I4) return LOCKS_ERR_INVALID_ARG;
+  if ((c->kv_dtype != LOCKS_F32 && c->kv_dtype != LOCKS_BF16) || (c->q_dtype != LOCKS_F32 && c->q_dtype != LOCKS_BF16))
+    return LOCKS_ERR_INVALID_ARG;
+  if (c->head_dim != LOCKS_D || c->page_size != LOCKS_B) return LOCKS_ERR_UNSUPPORTED;
+  if (c->num_q_heads / c->num_kv_heads > 16) return LOCKS_ERR_UNSUPPORTED;
+  if (c->kv_dtype != c->q_dtype) return LOCKS_ERR_UNSUPPORTED;
+  if (c->summary_fmt == LOCKS_FMT_I4 && c->rank != 2 && c->rank != 4 && c->rank != 8) return LOCKS_ERR_UNSUPPORTED;
+  if (c->summary_fmt == LOCKS_FMT_F32 && c->rank > 16) return LOCKS_ERR_UNSUPPORTED;
+  const int chunks = (c->max_pages_per_seq + LOCKS_SEL_CHUNK - 1) / LOCKS_SEL_CHUNK;
+  if (chunks > 1 && (size_t)chunks * (k - 2) > 32 * LOCKS_SEL_THREADS) return LOCKS_ERR_UNSUPPORTED;
+  if (k > LOCKS_SEL_CHUNK) return LOCKS_ERR_UNSUPPORTED;
+  return LOCKS_OK;
+}
+
+struct Layout {
+  size_t status, shat, part, qnorm, cand_val, cand_idx, att_o, att_lse, ids, cnt, sq, skn, svn, sout, total;
+  int G, k, S, max_groups, sel_chunks, sel_kc, splits_sparse, splits_dense, splits_max;
+};
+
+Layout make_layout(const locks_config *c) {
+  Layout L;
+  L.G = c->num_q_heads / c->num_kv_heads;
+  L.k = (c->budget_tokens + c->page_size - 1) / c->page_size;
+  L.S = c->summary_fmt == LOCKS_FMT_I4 ? i4_stride(c->rank) : f32_stride(c->rank);
+  L.max_groups = (c->max_pages_per_seq + LOCKS_GROUP - 1) / LOCKS_GROUP;
+  L.sel_chunks = (c->max_pages_per_seq + LOCKS_SEL_CHUNK - 1) / LOCKS_SEL_CHUNK;
+  L.sel_kc = L.k - 2 > 0 ? L.k - 2 : 1;
+  const int ppc_s = LOCKS_ATT_WARPS * LOCKS_ATT_PAGES_PER_WARP, ppc_d = LOCKS_ATT_WARPS * LOCKS_ATT_DENSE_PAGES_PER_WARP;
+  L.splits_sparse = (L.k + ppc_s - 1) / ppc_s;
+  L.splits_dense = (c->max_pages_per_seq + ppc_d - 1) / ppc_d;
+  L.splits_max = L.splits_sparse > L.splits_dense ? L.splits_sparse : L.splits_dense;
+  const size_t nb = c->max_batch, Hq = c->num_q_heads, Hkv = c->num_kv_heads, P = c->max_pages_per_seq;
+  const size_t esz = c->q_dtype == LOCKS_BF16 ? 2 : 4;
+  size_t o = 0;
+  auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 256); return at; };
+  L.status = take(64);
+  L.shat = take(nb * Hq * P * 4);
+  L.part = take(nb * Hq * L.max_groups * 8);
+  L.qnorm = take(nb * Hq * 4);
+  L.cand_val = take(nb * Hkv * L.sel_chunks * L.sel_kc * 4);
+  L.cand_idx = take(nb * Hkv * L.sel_chunks * L.sel_kc * 4);
+  L.att_o = take(nb * Hq * L.splits_max * LOCKS_D * 4);
+  L.att_lse = take(nb * Hq * L.splits_max * 4);
+  L.ids = take(nb * Hkv * L.k * 4);
+  L.cnt = take(nb * Hkv * 4);
+  L.sq = take(nb * Hq * LOCKS_D * esz);
+  L.skn = take(nb * Hkv * LOCKS_D * esz);
+  L.svn = take(nb * Hkv * LOCKS_D * esz);
+  L.sout = take(nb * Hq * LOCKS_D * esz);
+  L.total = o;
+  return L;
+}
+
+int check_common(const locks_ctx *ctx, const locks_kv *kv, int batch) {
+  if (!ctx || !kv || !kv->k || !kv->v || !kv->block_table || !kv->seq_lens) return LOCKS_ERR_INVALID_ARG;
+  if (batch <= 0 || batch > ctx->cfg.max_batch || kv->num_blocks <= 0) return LOCKS_ERR_INVALID_ARG;
+  if (kv->stride_block <= 0 || kv->stride_head <= 0 || kv->stride_token < LOCKS_D) return LOCKS_ERR_INVALID_ARG;
+  if (ctx->cfg.kv_dtype == LOCKS_BF16) {  // 16-byte vector copies of bf16 rows
+    if ((kv->stride_block | kv->stride_head | kv->stride_token) % 8) return LOCKS_ERR_INVALID_ARG;
+    if (((uintptr_t)kv->k | (uintptr_t)kv->v) % 16) return LOCKS_ERR_INVALID_ARG;
+  }
+  return LOCKS_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t locks_summary_bytes(const locks_config *cfg) {
+  if (validate(cfg) != LOCKS_OK) return 0;
+  return (size_t)make_layout(cfg).S;
+}
+
+size_t locks_workspace_bytes(const locks_config *cfg) {
+  if (validate(cfg) != LOCKS_OK) return 0;
+  return make_layout(cfg).total;
+}
+
+int locks_create(const locks_config *cfg, void *workspace, size_t ws_bytes, locks_ctx **out) {
+  if (!out) return LOCKS_ERR_INVALID_ARG;
+  *out = nullptr;
+  int rc = validate(cfg);
+  if (rc != LOCKS_OK) return rc;
+  const Layout L = make_layout(cfg);
+  if (!workspace || ws_bytes < L.total || ((uintptr_t)workspace % 256)) return LOCKS_ERR_WORKSPACE;
+  locks_ctx *c = new (std::nothrow) locks_ctx();
+  if (!c) return LOCKS_ERR_INVALID_ARG;
+  c->cfg = *cfg;
+  c->G = L.G; c->k = L.k; c->S = L.S; c->Pmax = cfg->max_pages_per_seq; c->max_groups = L.max_groups;
+  c->sel_chunks = L.sel_chunks; c->sel_kc = L.sel_kc;
+  c->att_splits_sparse = L.splits_sparse; c->att_splits_dense = L.splits_dense; c->att_splits_max = L.splits_max;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&c->num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+    delete c;
+    return LOCKS_ERR_CUDA;
+  }
+  char *ws = reinterpret_cast<char *>(workspace);
+  c->ws = ws; c->ws_bytes = ws_bytes;
+  c->status = reinterpret_cast<int32_t *>(ws + L.status);
+  c->shat = reinterpret_cast<float *>(ws + L.shat);
+  c->part = reinterpret_cast<float2 *>(ws + L.part);
+  c->qnorm = reinterpret_cast<float *>(ws + L.qnorm);
+  c->cand_val = reinterpret_cast<float *>(ws + L.cand_val);
+  c->cand_idx = reinterpret_cast<int32_t *>(ws + L.cand_idx);
+  c->att_o = reinterpret_cast<float *>(ws + L.att_o);
+  c->att_lse = reinterpret_cast<float *>(ws + L.att_lse);
+  c->ids_int = reinterpret_cast<int32_t *>(ws + L.ids);
+  c->cnt_int = reinterpret_cast<int32_t *>(ws + L.cnt);
+  c->stage_q = ws + L.sq; c->stage_kn = ws + L.skn; c->stage_vn = ws + L.svn; c->stage_out = ws + L.sout;
+  if (cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking) != cudaSuccess ||
+      cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+      cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) != cudaSuccess ||
+      cudaMemsetAsync(c->status, 0, 64, 0) != cudaSuccess || cudaStreamSynchronize(0) != cudaSuccess) {
+    delete c;
+    return LOCKS_ERR_CUDA;
+  }
+  *out = c;
+  return LOCKS_OK;
+}
+
+int locks_destroy(locks_ctx *ctx) {
+  if (!ctx) return LOCKS_ERR_INVALID_ARG;
+  cudaEventDestroy(ctx->ev_fork);
+  cudaEventDestroy(ctx->ev_join);
+  cudaStreamDestroy(ctx->side);
+  delete ctx;
+  return LOCKS_OK;
+}
+
+int locks_build_summaries(locks_ctx *ctx, const locks_kv *kv, int batch, const int32_t *page_begin,
+                          const int32_t *page_end, void *summaries, locks_stream stream) {
+  int rc = check_common(ctx, kv, batch);
+  if (rc != LOCKS_OK) return rc;
+  if (!summaries || ((uintptr_t)summaries % 16) || ((page_begin == nullptr) != (page_end == nullptr)))
+    return LOCKS_ERR_INVALID_ARG;
+  ctx->last_launches = 0;
+  return locks_launch_build(ctx, kv, batch, page_begin, page_end, 0, summaries, (cudaStream_t)stream);
+}
+
+int locks_select(locks_ctx *ctx, const void *q, const void *summaries, const locks_kv *kv, int batch,
+                 int32_t *page_ids, int32_t *page_count, float *page_logmass, float *page_logshare,
+                 locks_stream stream) {
+  int rc = check_common(ctx, kv, batch);
+  if (rc != LOCKS_OK) return rc;
+  if (!q || !summaries || !page_ids || !page_count || ((uintptr_t)summaries % 16) || ((uintptr_t)q % 16))
+    return LOCKS_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  ctx->last_launches = 0;
+  float *shat = page_logmass ? page_logmass : ctx->shat;
+  if ((rc = locks_launch_prep(ctx, q, nullptr, nullptr, kv, batch, st)) != LOCKS_OK) return rc;
+  if ((rc = locks_launch_scan(ctx, q, summaries, kv, batch, shat, st)) != LOCKS_OK) return rc;
+  return locks_launch_select(ctx, shat, kv, batch, page_ids, page_count, page_logshare, st);
+}
+
+int locks_sparse_attend(locks_ctx *ctx, const void *q, const locks_kv *kv, int batch, const int32_t *page_ids,
+                        const int32_t *page_count, void *out, float *lse, locks_stream stream) {
+  int rc = check_common(ctx, kv, batch);
+  if (rc != LOCKS_OK) return rc;
+  if (!q || !out || ((page_ids == nullptr) != (page_count == nullptr)) || ((uintptr_t)q % 16))
+    return LOCKS_ERR_INVALID_ARG;
+  ctx->last_launches = 0;
+  return locks_launch_attend(ctx, q, kv, batch, page_ids, page_count, out, lse, (cudaStream_t)stream);
+}
+
+int locks_decode_step(locks_ctx *ctx, const void *q, const void *k_new, const void *v_new, locks_kv *kv,
+                      void *summaries, int batch, void *out, int32_t *page_ids, int32_t *page_count,
+                      locks_stream stream) {
+  int rc = check_common(ctx, kv, batch);
+  if (rc != LOCKS_OK) return rc;
+  if (!q || !summaries || !out || ((k_new == nullptr) != (v_new == nullptr)) || ((uintptr_t)summaries % 16) ||
+      ((uintptr_t)q % 16))
+    return LOCKS_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  int32_t *ids = page_ids ? page_ids : ctx->ids_int;
+  int32_t *cnt = page_count ? page_count : ctx->cnt_int;
+  ctx->last_launches = 0;
+  if ((rc = locks_launch_prep(ctx, q, k_new, v_new, kv, batch, st)) != LOCKS_OK) return rc;
+  // the freshly completed page (if any) is summarised beside select + attend: it is read by neither
+  if (cudaEventRecord(ctx->ev_fork, st) != cudaSuccess || cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0) != cudaSuccess)
+    return LOCKS_ERR_CUDA;
+  if ((rc = locks_launch_build(ctx, kv, batch, nullptr, nullptr, 1, summaries, ctx->side)) != LOCKS_OK) return rc;
+  if (cudaEventRecord(ctx->ev_join, ctx->side) != cudaSuccess) return LOCKS_ERR_CUDA;
+  if ((rc = locks_launch_scan(ctx, q, summaries, kv, batch, ctx->shat, st)) != LOCKS_OK) return rc;
+  if ((rc = locks_launch_select(ctx, ctx->shat, kv, batch, ids, cnt, nullptr, st)) != LOCKS_OK) return rc;
+  if ((rc = locks_launch_attend(ctx, q, kv, batch, ids, cnt, out, nullptr, st)) != LOCKS_OK) return rc;
+  if (cudaStreamWaitEvent(st, ctx->ev_join, 0) != cudaSuccess) return LOCKS_ERR_CUDA;
+  return LOCKS_OK;
+}
+
+int locks_decode_step_host(locks_ctx *ctx, const void *q_host, const void *k_new_host, const void *v_new_host,
+                           locks_kv *kv, void *summaries, int batch, void *out_host, int32_t *page_ids_host,
+                           int32_t *page_count_host, locks_stream stream) {
+  int rc = check_common(ctx, kv, batch);
+  if (rc != LOCKS_OK) return rc;
+  if (!q_host || !out_host || ((k_new_host == nullptr) != (v_new_host == nullptr))) return LOCKS_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  const size_t esz = ctx->cfg.q_dtype == LOCKS_BF16 ? 2 : 4;
+  const size_t qb = (size_t)batch * ctx->cfg.num_q_heads * LOCKS_D * esz;
+  const size_t kb = (size_t)batch * ctx->cfg.num_kv_heads * LOCKS_D * esz;
+  if (cudaMemcpyAsync(ctx->stage_q, q_host, qb, cudaMemcpyHostToDevice, st) != cudaSuccess) return LOCKS_ERR_CUDA;
+  if (k_new_host) {
+    if (cudaMemcpyAsync(ctx->stage_kn, k_new_host, kb, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaMemcpyAsync(ctx->stage_vn, v_new_host, kb, cudaMemcpyHostToDevice, st) != cudaSuccess)
+      return LOCKS_ERR_CUDA;
+  }
+  rc = locks_decode_step(ctx, ctx->stage_q, k_new_host ? ctx->stage_kn : nullptr, k_new_host ? ctx->stage_vn : nullptr,
+                         kv, summaries, batch, ctx->stage_out, ctx->ids_int, ctx->cnt_int, stream);
+  if (rc != LOCKS_OK) return rc;
+  const int launches = ctx->last_launches;
+  if (cudaMemcpyAsync(out_host, ctx->stage_out, qb, cudaMemcpyDeviceToHost, st) != cudaSuccess) return LOCKS_ERR_CUDA;
+  if (page_ids_host &&
+      cudaMemcpyAsync(page_ids_host, ctx->ids_int, (size_t)batch * ctx->cfg.num_kv_heads * ctx->k * 4,
+                      cudaMemcpyDeviceToHost, st) != cudaSuccess)
+    return LOCKS_ERR_CUDA;
+  if (page_count_host &&
+      cudaMemcpyAsync(page_count_host, ctx->cnt_int, (size_t)batch * ctx->cfg.num_kv_heads * 4, cudaMemcpyDeviceToHost,
+                      st) != cudaSuccess)
+    return LOCKS_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return LOCKS_ERR_CUDA;
+  ctx->last_launches = launches;
+  return LOCKS_OK;
+}
+
+int locks_poll_status(locks_ctx *ctx, int32_t *status_host, locks_stream stream) {
+  if (!ctx || !status_host) return LOCKS_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (cudaMemcpyAsync(status_host, ctx->status, 4, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+      cudaMemsetAsync(ctx->status, 0, 4, st) != cudaSuccess || cudaStreamSynchronize(st) != cudaSuccess)
+    return LOCKS_ERR_CUDA;
+  return LOCKS_OK;
+}
+
+int locks_last_launch_count(const locks_ctx *ctx) { return ctx ? ctx->last_launches : 0; }
+
+const char *locks_strerror(int code) {
+  switch (code) {
+    case LOCKS_OK: return "ok";
+    case LOCKS_ERR_INVALID_ARG: return "invalid argument";
+    case LOCKS_ERR_UNSUPPORTED: return "configuration not supported by the kernels";
+    case LOCKS_ERR_WORKSPACE: return "workspace too small or misaligned";
+    case LOCKS_ERR_CUDA: return "CUDA runtime error";
+    case LOCKS_ERR_TIMEOUT: return "a bounded device-side wait expired";
+    case LOCKS_ERR_BAD_BLOCK: return "page or block id outside the cache";
+    default: return "unknown error";
+  }
+}
+
+}  // extern "C"

@@ -1,0 +1,386 @@
+// Summary build (Sec. 4 "Build (once, when a page completes)") and the per-step prologue.
+//
+// build_kernel: one warp per (page, KV head).
+//   1. load the page's 16 keys (lane owns 4 consecutive dims of every key), centroid mu, deviations D
+//   2. Gram M = D D^T (16 x 16) from shared memory
+//   3. eigendecomposition of M by parallel-ordered cyclic Jacobi in fp32 (8 disjoint rotations per
+//      round, 15 rounds per sweep, round-robin pairing), eigenvectors accumulated in U
+//   4. rank by eigenvalue, keep r_eff <= min(r, 15) modes above the zero-mode thresholds
+//   5. V = D^T U_r Sigma_r^-1 (lane's 4 dims), C = U_r Sigma_r, sign: largest |V| entry positive
+//   6. store fp32 (F32 format) or quantise: symmetric abs-max, fp16 scale, round-half-even codes
+//      (int4 basis per column, int8 coefficients per row, int8 centroid) packed in the blob layout
+// prep_kernel: appends the new token's K/V row to the cache (optional), and derives the per-query
+//   power-of-two scale that keeps the scan's fp16 projection operands in range.
+#include "locks_internal.cuh"
+
+namespace {
+
+struct BuildParams {
+  const void *k;
+  int64_t sb, sh, st;
+  const int32_t *block_table;
+  const int32_t *seq_lens;
+  const int32_t *page_begin, *page_end;
+  uint8_t *summ;
+  int32_t *status;
+  int batch, Hkv, Pmax, num_blocks, r, S, just_filled;
+};
+
+constexpr int kBuildWarps = 4;
+constexpr int kDStride = LOCKS_D + 4;                            // padded row of D in shared memory
+constexpr int kBuildSmemPerWarp = (LOCKS_B * kDStride + 2 * LOCKS_B * 17 + 64) * 4 + i4_stride(8);
+
+__device__ __forceinline__ float round_code(float x, float scale, float qmax) {
+  if (scale == 0.f) return 0.f;
+  float c = rintf(__fdiv_rn(x, scale));
+  return fminf(fmaxf(c, -qmax), qmax);
+}
+
+template <typename T, int FMT>
+__global__ void __launch_bounds__(kBuildWarps * 32) build_kernel(BuildParams p) {
+  extern __shared__ __align__(16) uint8_t smem_raw[];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int b, h, page;
+  if (p.just_filled) {
+    const int prob = blockIdx.x * kBuildWarps + warp;
+    if (prob >= p.batch * p.Hkv) return;
+    b = prob / p.Hkv; h = prob - b * p.Hkv;
+    const int Tb = p.seq_lens[b];
+    if (Tb <= 0 || (Tb % LOCKS_B) != 0) return;
+    page = Tb / LOCKS_B - 1;
+  } else {
+    b = blockIdx.z; h = blockIdx.y;
+    const int complete = p.seq_lens[b] / LOCKS_B;
+    const int p0 = p.page_begin ? p.page_begin[b] : 0;
+    const int p1 = min(p.page_end ? p.page_end[b] : complete, complete);
+    page = p0 + blockIdx.x * kBuildWarps + warp;
+    if (page < 0 || page >= p1) return;
+  }
+  if (page >= p.Pmax) return;
+  const int block = p.block_table[(int64_t)b * p.Pmax + page];
+  if (block < 0 || block >= p.num_blocks) {
+    if (lane == 0) set_status(p.status, LOCKS_ERR_BAD_BLOCK);
+    return;
+  }
+  float *Ds = reinterpret_cast<float *>(smem_raw + warp * kBuildSmemPerWarp);   // [16][kDStride]
+  float *A = Ds + LOCKS_B * kDStride;                                             // [16][17]
+  float *U = A + LOCKS_B * 17;                                                    // [16][17]
+  float *rot = U + LOCKS_B * 17;                                                  // c[8], s[8], misc
+  uint8_t *blob = reinterpret_cast<uint8_t *>(rot + 64);
+  const int r = p.r;
+
+  // ---- 1. load, centre
+  const T *K = reinterpret_cast<const T *>(p.k) + (int64_t)block * p.sb + (int64_t)h * p.sh;
+  float kv[LOCKS_B][4], mu[4] = {0.f, 0.f, 0.f, 0.f};
+  float knorm2 = 0.f;
+#pragma unroll
+  for (int i = 0; i < LOCKS_B; ++i) {
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      kv[i][u] = ldf<T>(K, (int64_t)i * p.st + lane * 4 + u);
+      mu[u] += kv[i][u];
+      knorm2 += kv[i][u] * kv[i][u];
+    }
+  }
+  knorm2 = warp_sum(knorm2);
+#pragma unroll
+  for (int u = 0; u < 4; ++u) mu[u] *= (1.f / LOCKS_B);
+#pragma unroll
+  for (int i = 0; i < LOCKS_B; ++i) {
+#pragma unroll
+    for (int u = 0; u < 4; ++u) kv[i][u] -= mu[u];
+    *reinterpret_cast<float4 *>(Ds + i * kDStride + lane * 4) = make_float4(kv[i][0], kv[i][1], kv[i][2], kv[i][3]);
+  }
+  __syncwarp();
+  // ---- 2. Gram: lane computes entries e = lane + 32 m -> (i = e / 16, j = e % 16)
+#pragma unroll 1
+  for (int m = 0; m < 8; ++m) {
+    const int e = lane + 32 * m, i = e >> 4, j = e & 15;
+    const float4 *ri = reinterpret_cast<const float4 *>(Ds + i * kDStride);
+    const float4 *rj = reinterpret_cast<const float4 *>(Ds + j * kDStride);
+    float s = 0.f;
+    for (int c = 0; c < LOCKS_D / 4; ++c) {
+      const float4 a = ri[c], bb = rj[c];
+      s += a.x * bb.x + a.y * bb.y + a.z * bb.z + a.w * bb.w;
+    }
+    A[i * 17 + j] = s;
+    U[i * 17 + j] = (i == j) ? 1.f : 0.f;
+  }
+  __syncwarp();
+  // ---- 3. parallel cyclic Jacobi
+  float normA = 0.f;
+  for (int e = lane; e < 256; e += 32) { const float a = A[(e >> 4) * 17 + (e & 15)]; normA += a * a; }
+  normA = warp_sum(normA);
+  for (int sweep = 0; sweep < 12; ++sweep) {
+    float off = 0.f;
+    for (int e = lane; e < 256; e += 32) {
+      const int i = e >> 4, j = e & 15;
+      if (i != j) { const float a = A[i * 17 + j]; off += a * a; }
+    }
+    off = warp_sum(off);
+    if (off <= 1e-13f * normA || normA == 0.f) break;
+    for (int round = 0; round < 15; ++round) {
+      // round-robin pairing: (15, round), ((round + m) % 15, (round - m + 15) % 15), m = 1..7
+      if (lane < 8) {
+        int pi, qi;
+        if (lane == 0) { pi = round; qi = 15; }
+        else { pi = (round + lane) % 15; qi = (round - lane + 15) % 15; }
+        if (pi > qi) { const int tmp = pi; pi = qi; qi = tmp; }
+        const float apq = A[pi * 17 + qi], app = A[pi * 17 + pi], aqq = A[qi * 17 + qi];
+        float c = 1.f, s = 0.f;
+        if (fabsf(apq) > 1e-30f) {
+          const float theta = (aqq - app) / (2.f * apq);
+          const float tt = copysignf(1.f, theta) / (fabsf(theta) + sqrtf(theta * theta + 1.f));
+          c = rsqrtf(tt * tt + 1.f);
+          s = tt * c;
+        }
+        rot[lane] = c; rot[8 + lane] = s;
+        reinterpret_cast<int *>(rot)[16 + lane] = pi;
+        reinterpret_cast<int *>(rot)[24 + lane] = qi;
+      }
+      __syncwarp();
+      // columns: A <- A J, U <- U J   (item = (row i, pair m))
+#pragma unroll
+      for (int it = 0; it < 4; ++it) {
+        const int item = lane + 32 * it, i = item >> 3, m = item & 7;
+        const float c = rot[m], s = rot[8 + m];
+        const int pi = reinterpret_cast<int *>(rot)[16 + m], qi = reinterpret_cast<int *>(rot)[24 + m];
+        const float aip = A[i * 17 + pi], aiq = A[i * 17 + qi];
+        A[i * 17 + pi] = c * aip - s * aiq;
+        A[i * 17 + qi] = s * aip + c * aiq;
+        const float uip = U[i * 17 + pi], uiq = U[i * 17 + qi];
+        U[i * 17 + pi] = c * uip - s * uiq;
+        U[i * 17 + qi] = s * uip + c * uiq;
+      }
+      __syncwarp();
+      // rows: A <- J^T A
+#pragma unroll
+      for (int it = 0; it < 4; ++it) {
+        const int item = lane + 32 * it, i = item >> 3, m = item & 7;
+        const float c = rot[m], s = rot[8 + m];
+        const int pi = reinterpret_cast<int *>(rot)[16 + m], qi = reinterpret_cast<int *>(rot)[24 + m];
+        const float api = A[pi * 17 + i], aqi = A[qi * 17 + i];
+        A[pi * 17 + i] = c * api - s * aqi;
+        A[qi * 17 + i] = s * api + c * aqi;
+      }
+      __syncwarp();
+    }
+  }
+  // ---- 4. order the eigenvalues (descending, ties by index), choose r_eff
+  float lam = (lane < 16) ? A[lane * 17 + lane] : -INFINITY;
+  int rank = 0;
+  for (int j = 0; j < 16; ++j) {
+    const float lj = __shfl_sync(0xffffffffu, lam, j);
+    rank += (lj > lam) || (lj == lam && j < lane);
+  }
+  if (lane < 16) { reinterpret_cast<int *>(rot)[32 + rank] = lane; rot[48 + rank] = lam; }
+  __syncwarp();
+  const float lam0 = rot[48];
+  int r_eff = 0;
+  const int rmax = min(r, LOCKS_B - 1);
+  for (int l = 0; l < rmax; ++l) {
+    const float ll = rot[48 + l];
+    if (lam0 > 0.f && ll > 1e-6f * lam0 && ll > 1e-10f * knorm2) r_eff = l + 1; else break;
+  }
+  // ---- 5/6. per mode: basis entries of this lane's 4 dims, sign, quantise
+  if (FMT == LOCKS_FMT_I4) {
+    for (int e = lane; e < i4_stride(8) / 4; e += 32) reinterpret_cast<uint32_t *>(blob)[e] = 0u;
+    __syncwarp();
+  }
+  float *fout = reinterpret_cast<float *>(p.summ + ((int64_t)block * p.Hkv + h) * p.S);
+  float csign[16];
+#pragma unroll 1
+  for (int l = 0; l < r; ++l) {
+    float v[4] = {0.f, 0.f, 0.f, 0.f};
+    float sgn = 1.f;
+    if (l < r_eff) {
+      const int col = reinterpret_cast<int *>(rot)[32 + l];
+      const float inv = rsqrtf(rot[48 + l]);
+#pragma unroll
+      for (int i = 0; i < LOCKS_B; ++i) {
+        const float u = U[i * 17 + col];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) v[c] += kv[i][c] * u;
+      }
+#pragma unroll
+      for (int c = 0; c < 4; ++c) v[c] *= inv;
+      // sign: entry of largest magnitude (lowest dim on ties) positive
+      float best = fabsf(v[0]); int bi = lane * 4; float bv = v[0];
+#pragma unroll
+      for (int c = 1; c < 4; ++c) if (fabsf(v[c]) > best) { best = fabsf(v[c]); bi = lane * 4 + c; bv = v[c]; }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        const float ob = __shfl_xor_sync(0xffffffffu, best, o);
+        const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+        const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+        if (ob > best || (ob == best && oi < bi)) { best = ob; bi = oi; bv = ov; }
+      }
+      if (bv < 0.f) sgn = -1.f;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) v[c] *= sgn;
+    }
+    csign[l & 15] = sgn;
+    if (FMT == LOCKS_FMT_F32) {
+      *reinterpret_cast<float4 *>(fout + LOCKS_D + l * LOCKS_D + lane * 4) = make_float4(v[0], v[1], v[2], v[3]);
+    } else {
+      float mx = fmaxf(fmaxf(fabsf(v[0]), fabsf(v[1])), fmaxf(fabsf(v[2]), fabsf(v[3])));
+      mx = warp_max(mx);
+      const __half sh = __float2half_rn(mx / 7.f);
+      const float sc = __half2float(sh);
+      if (lane == 0) *reinterpret_cast<__half *>(blob + i4_off_sv(r) + 2 * l) = sh;
+      // lane = 8 t + s owns dims 32 t + 4 s + {0,1,2,3} = (half, e) in {0,1}^2 of k-step s
+      const int t = lane >> 3, s = lane & 7, i0 = (s & 1) << 1;
+      uint32_t n[4];
+#pragma unroll
+      for (int c = 0; c < 4; ++c) n[c] = (uint32_t)((int)round_code(v[c], sc, 7.f) + 8);
+      // dim offset c = 2*half + e -> nibble i0 + half + 4 e
+      uint32_t pw = (n[0] << (4 * i0)) | (n[1] << (4 * (i0 + 4))) | (n[2] << (4 * (i0 + 1))) | (n[3] << (4 * (i0 + 5)));
+      pw |= __shfl_xor_sync(0xffffffffu, pw, 1);
+      if ((s & 1) == 0) *reinterpret_cast<uint32_t *>(blob + (l * 4 + t) * 16 + (s >> 1) * 4) = pw;
+    }
+  }
+  // coefficients: lane i < 16 owns token i
+  if (lane < LOCKS_B) {
+    float cf[16];
+    float mx = 0.f;
+    for (int l = 0; l < r; ++l) {
+      float c = 0.f;
+      if (l < r_eff) c = sqrtf(rot[48 + l]) * U[lane * 17 + reinterpret_cast<int *>(rot)[32 + l]] * csign[l & 15];
+      cf[l & 15] = c;
+      mx = fmaxf(mx, fabsf(c));
+    }
+    if (FMT == LOCKS_FMT_F32) {
+      for (int l = 0; l < r; ++l) fout[LOCKS_D + r * LOCKS_D + lane * r + l] = cf[l & 15];
+    } else {
+      const __half sh = __float2half_rn(mx / 127.f);
+      const float sc = __half2float(sh);
+      const int tpos = ((lane & 7) >> 1) * 4 + (lane >> 3) * 2 + (lane & 1);
+      *reinterpret_cast<__half *>(blob + i4_off_sc(r) + 2 * tpos) = sh;
+      const int xx = lane & 7, hi = lane >> 3;
+      for (int l = 0; l < r; ++l)
+        blob[i4_off_coef(r) + (xx * (r / 2) + (l >> 1)) * 4 + hi * 2 + (l & 1)] =
+            (uint8_t)((int)round_code(cf[l & 15], sc, 127.f) + 128);
+    }
+  }
+  // centroid
+  if (FMT == LOCKS_FMT_F32) {
+    *reinterpret_cast<float4 *>(fout + lane * 4) = make_float4(mu[0], mu[1], mu[2], mu[3]);
+  } else {
+    float mx = fmaxf(fmaxf(fabsf(mu[0]), fabsf(mu[1])), fmaxf(fabsf(mu[2]), fabsf(mu[3])));
+    mx = warp_max(mx);
+    const __half sh = __float2half_rn(mx / 127.f);
+    const float sc = __half2float(sh);
+    if (lane == 0) *reinterpret_cast<__half *>(blob + i4_off_smu(r)) = sh;
+    uint32_t bytes[4];
+#pragma unroll
+    for (int c = 0; c < 4; ++c) bytes[c] = (uint32_t)((int)round_code(mu[c], sc, 127.f) + 128);
+    // dim offset c = 2*half + e -> byte e*2 + half
+    const uint32_t w = bytes[0] | (bytes[2] << 8) | (bytes[1] << 16) | (bytes[3] << 24);
+    *reinterpret_cast<uint32_t *>(blob + i4_off_mu(r) + lane * 4) = w;
+    __syncwarp();
+    uint4 *dst = reinterpret_cast<uint4 *>(p.summ + ((int64_t)block * p.Hkv + h) * p.S);
+    for (int e = lane; e < p.S / 16; e += 32) dst[e] = reinterpret_cast<const uint4 *>(blob)[e];
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+
+struct PrepParams {
+  const void *q, *k_new, *v_new;
+  void *k, *v;
+  int64_t sb, sh, st;
+  const int32_t *block_table;
+  int32_t *seq_lens;
+  float *qnorm;
+  int32_t *status;
+  int Hq, Hkv, Pmax, num_blocks;
+};
+
+template <typename T>
+__global__ void __launch_bounds__(128) prep_kernel(PrepParams p) {
+  const int b = blockIdx.x, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  // per-head power of two 2^-e with 2^e >= 2 |q|: keeps V^T q inside [-0.55, 0.55] for the fp16 MMA
+  const T *Q = reinterpret_cast<const T *>(p.q);
+  for (int hq = warp; hq < p.Hq; hq += 4) {
+    float s = 0.f;
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const float v = ldf<T>(Q, ((int64_t)b * p.Hq + hq) * LOCKS_D + lane * 4 + u);
+      s += v * v;
+    }
+    s = warp_sum(s);
+    if (lane == 0) {
+      float pn = 1.f;
+      if (s > 0.f && s < INFINITY) {
+        int e;
+        (void)frexpf(2.f * sqrtf(s), &e);  // 2|q| = f 2^e, f in [0.5, 1)
+        pn = ldexpf(1.f, -e);
+      }
+      p.qnorm[b * p.Hq + hq] = pn;
+    }
+  }
+  if (p.k_new == nullptr) return;
+  const int T0 = p.seq_lens[b];
+  const int page = T0 / LOCKS_B, slot = T0 % LOCKS_B;
+  bool ok = page < p.Pmax;
+  int block = 0;
+  if (ok) {
+    block = p.block_table[(int64_t)b * p.Pmax + page];
+    ok = block >= 0 && block < p.num_blocks;
+  }
+  if (!ok) {
+    if (threadIdx.x == 0) set_status(p.status, LOCKS_ERR_BAD_BLOCK);
+    return;
+  }
+  const T *kn = reinterpret_cast<const T *>(p.k_new), *vn = reinterpret_cast<const T *>(p.v_new);
+  T *K = reinterpret_cast<T *>(p.k), *V = reinterpret_cast<T *>(p.v);
+  for (int e = threadIdx.x; e < p.Hkv * LOCKS_D; e += 128) {
+    const int h = e / LOCKS_D, c = e - h * LOCKS_D;
+    const int64_t dst = (int64_t)block * p.sb + (int64_t)h * p.sh + (int64_t)slot * p.st + c;
+    K[dst] = kn[((int64_t)b * p.Hkv + h) * LOCKS_D + c];
+    V[dst] = vn[((int64_t)b * p.Hkv + h) * LOCKS_D + c];
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) p.seq_lens[b] = T0 + 1;
+}
+
+}  // namespace
+
+int locks_launch_build(locks_ctx *c, const locks_kv *kv, int batch, const int32_t *pb, const int32_t *pe,
+                       int just_filled, void *summaries, cudaStream_t st) {
+  BuildParams p;
+  p.k = kv->k; p.sb = kv->stride_block; p.sh = kv->stride_head; p.st = kv->stride_token;
+  p.block_table = kv->block_table; p.seq_lens = kv->seq_lens; p.page_begin = pb; p.page_end = pe;
+  p.summ = reinterpret_cast<uint8_t *>(summaries); p.status = c->status;
+  p.batch = batch; p.Hkv = c->cfg.num_kv_heads; p.Pmax = c->Pmax; p.num_blocks = kv->num_blocks;
+  p.r = c->cfg.rank; p.S = c->S; p.just_filled = just_filled;
+  dim3 grid = just_filled ? dim3((batch * p.Hkv + kBuildWarps - 1) / kBuildWarps)
+                          : dim3((c->Pmax + kBuildWarps - 1) / kBuildWarps, p.Hkv, batch);
+  const int smem = kBuildWarps * kBuildSmemPerWarp;
+  const bool bf = c->cfg.kv_dtype == LOCKS_BF16, i4 = c->cfg.summary_fmt == LOCKS_FMT_I4;
+  static bool attr_done = false;
+  if (!attr_done) {
+    cudaFuncSetAttribute(build_kernel<__nv_bfloat16, LOCKS_FMT_I4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    cudaFuncSetAttribute(build_kernel<__nv_bfloat16, LOCKS_FMT_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    cudaFuncSetAttribute(build_kernel<float, LOCKS_FMT_I4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    cudaFuncSetAttribute(build_kernel<float, LOCKS_FMT_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    attr_done = true;
+  }
+  if (bf && i4) build_kernel<__nv_bfloat16, LOCKS_FMT_I4><<<grid, kBuildWarps * 32, smem, st>>>(p);
+  else if (bf) build_kernel<__nv_bfloat16, LOCKS_FMT_F32><<<grid, kBuildWarps * 32, smem, st>>>(p);
+  else if (i4) build_kernel<float, LOCKS_FMT_I4><<<grid, kBuildWarps * 32, smem, st>>>(p);
+  else build_kernel<float, LOCKS_FMT_F32><<<grid, kBuildWarps * 32, smem, st>>>(p);
+  return locks_check_launch(c);
+}
+
+int locks_launch_prep(locks_ctx *c, const void *q, const void *k_new, const void *v_new, const locks_kv *kv,
+                      int batch, cudaStream_t st) {
+  PrepParams p;
+  p.q = q; p.k_new = k_new; p.v_new = v_new; p.k = kv->k; p.v = kv->v;
+  p.sb = kv->stride_block; p.sh = kv->stride_head; p.st = kv->stride_token;
+  p.block_table = kv->block_table; p.seq_lens = kv->seq_lens; p.qnorm = c->qnorm; p.status = c->status;
+  p.Hq = c->cfg.num_q_heads; p.Hkv = c->cfg.num_kv_heads; p.Pmax = c->Pmax; p.num_blocks = kv->num_blocks;
+  if (c->cfg.q_dtype == LOCKS_BF16) prep_kernel<__nv_bfloat16><<<batch, 128, 0, st>>>(p);
+  else prep_kernel<float><<<batch, 128, 0, st>>>(p);
+  return locks_check_launch(c);
+}

@@ -1,0 +1,183 @@
+// Internal declarations of liblocks: context, workspace partition, device helpers, launchers.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "locks.h"
+
+#define LOCKS_D 128          // head dimension the kernels are written for
+#define LOCKS_B 16           // tokens per page
+#define LOCKS_GROUP 8        // pages scored together by one warp in the scan
+#define LOCKS_SEL_THREADS 256
+#define LOCKS_SEL_EPT 8      // candidate pages held per thread in select stage 1
+#define LOCKS_SEL_CHUNK (LOCKS_SEL_THREADS * LOCKS_SEL_EPT)
+#define LOCKS_ATT_WARPS 4
+#define LOCKS_ATT_PAGES_PER_WARP 4
+#define LOCKS_ATT_DENSE_PAGES_PER_WARP 16
+#define LOCKS_SPIN_LIMIT (1 << 22)  // bounded mbarrier polling (each poll already waits a while)
+
+struct locks_ctx {
+  locks_config cfg;
+  int G, k, S, Pmax, max_groups;
+  int num_sms;
+  int sel_chunks;          // select stage-1 CTAs per (request, KV head)
+  int sel_kc;              // candidates kept per chunk (k-2)
+  int att_splits_sparse, att_splits_dense, att_splits_max;
+  // workspace partition (device)
+  char *ws;
+  size_t ws_bytes;
+  int32_t *status;         // [4] sticky status, work counters
+  float *shat;             // [max_batch][Hq][Pmax]
+  float2 *part;            // [max_batch][Hq][max_groups] per-group (max, sum exp) of candidates
+  float *qnorm;            // [max_batch][Hq] power-of-two scale keeping projections inside fp16
+  float *cand_val;         // [max_batch][Hkv][sel_chunks][sel_kc]
+  int32_t *cand_idx;
+  float *att_o;            // [max_batch][Hq][att_splits_max][d]
+  float *att_lse;          // [max_batch][Hq][att_splits_max]  (log2 units)
+  int32_t *ids_int;        // [max_batch][Hkv][k]
+  int32_t *cnt_int;        // [max_batch][Hkv]
+  char *stage_q, *stage_kn, *stage_vn, *stage_out;
+  cudaStream_t side;       // build of freshly filled pages runs beside select + attend
+  cudaEvent_t ev_fork, ev_join;
+  int last_launches;
+};
+
+// launchers (each returns LOCKS_OK or LOCKS_ERR_CUDA and adds to ctx->last_launches)
+int locks_launch_prep(locks_ctx *c, const void *q, const void *k_new, const void *v_new, const locks_kv *kv,
+                      int batch, cudaStream_t st);
+int locks_launch_scan(locks_ctx *c, const void *q, const void *summaries, const locks_kv *kv, int batch,
+                      float *shat, cudaStream_t st);
+int locks_launch_select(locks_ctx *c, const float *shat, const locks_kv *kv, int batch, int32_t *ids,
+                        int32_t *cnt, float *logshare, cudaStream_t st);
+int locks_launch_attend(locks_ctx *c, const void *q, const locks_kv *kv, int batch, const int32_t *ids,
+                        const int32_t *cnt, void *out, float *lse, cudaStream_t st);
+int locks_launch_build(locks_ctx *c, const locks_kv *kv, int batch, const int32_t *pb, const int32_t *pe,
+                       int just_filled, void *summaries, cudaStream_t st);
+
+static inline int locks_check_launch(locks_ctx *c) {
+  c->last_launches++;
+  return cudaPeekAtLastError() == cudaSuccess ? LOCKS_OK : LOCKS_ERR_CUDA;
+}
+
+// ---------------------------------------------------------------- I4 blob geometry (B = 16, d = 128)
+// [basis 64 r][coefficients 16 r][centroid 128][sC 16 x fp16][sV r x fp16][sMu fp16], padded to 16.
+__host__ __device__ constexpr int i4_off_coef(int r) { return 64 * r; }
+__host__ __device__ constexpr int i4_off_mu(int r) { return 80 * r; }
+__host__ __device__ constexpr int i4_off_sc(int r) { return 80 * r + 128; }
+__host__ __device__ constexpr int i4_off_sv(int r) { return 80 * r + 160; }
+__host__ __device__ constexpr int i4_off_smu(int r) { return 82 * r + 160; }
+__host__ __device__ constexpr int i4_stride(int r) { return (82 * r + 162 + 15) / 16 * 16; }
+__host__ __device__ constexpr int f32_stride(int r) { return 4 * (LOCKS_D + r * LOCKS_D + LOCKS_B * r); }
+
+#ifdef __CUDACC__
+
+__device__ __forceinline__ void set_status(int32_t *status, int code) { atomicCAS(status, 0, code); }
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+
+template <typename T> __device__ __forceinline__ float ldf(const T *p, int64_t i);
+template <> __device__ __forceinline__ float ldf<float>(const float *p, int64_t i) { return p[i]; }
+template <> __device__ __forceinline__ float ldf<__nv_bfloat16>(const __nv_bfloat16 *p, int64_t i) {
+  return __bfloat162float(p[i]);
+}
+template <typename T> __device__ __forceinline__ void stf(T *p, int64_t i, float v);
+template <> __device__ __forceinline__ void stf<float>(float *p, int64_t i, float v) { p[i] = v; }
+template <> __device__ __forceinline__ void stf<__nv_bfloat16>(__nv_bfloat16 *p, int64_t i, float v) {
+  p[i] = __float2bfloat16_rn(v);
+}
+
+// D (16x8, fp32) += A (16x16, row) * B (16x8, col), bf16 or fp16 operands.
+__device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                         uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+               "{%0,%1,%2,%3};\n"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void mma_f16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                        uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+               "{%0,%1,%2,%3};\n"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+
+// ---- mbarrier + bulk async copy (TMA engine, untiled form) ------------------------------------
+__device__ __forceinline__ void mbar_init(uint64_t *bar, int count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(smem_u32(bar)), "r"(bytes)
+               : "memory");
+}
+// Bounded wait on a phase parity: true when the phase completed, false when the poll limit ran out.
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity) {
+  uint32_t a = smem_u32(bar);
+  for (int it = 0; it < LOCKS_SPIN_LIMIT; ++it) {
+    uint32_t done;
+    asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+                 " selp.u32 %0, 1, 0, p;\n}\n"
+                 : "=r"(done)
+                 : "r"(a), "r"(parity)
+                 : "memory");
+    if (done) return true;
+  }
+  return false;
+}
+// global -> shared bulk copy; size multiple of 16, both addresses 16-byte aligned.
+__device__ __forceinline__ void bulk_g2s(void *dst, const void *src, uint32_t bytes, uint64_t *bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n" ::
+                   "r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar))
+               : "memory");
+}
+__device__ __forceinline__ void fence_barrier_init() {
+  asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+}
+
+// ---- Ampere-style 16-byte async copies --------------------------------------------------------
+__device__ __forceinline__ void cp_async16(void *dst, const void *src, bool valid) {
+  int sz = valid ? 16 : 0;  // src-size 0 zero-fills the destination
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(smem_u32(dst)), "l"(src), "r"(sz)
+               : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() {
+  asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory");
+}
+
+__device__ __forceinline__ void ldsm_x4(uint32_t (&r)[4], const void *p) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"(smem_u32(p)));
+}
+__device__ __forceinline__ void ldsm_x4_trans(uint32_t (&r)[4], const void *p) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];\n"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"(smem_u32(p)));
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t *>(&v);
+}
+__device__ __forceinline__ uint32_t pack_f16(float lo, float hi) {
+  __half2 v = __floats2half2_rn(lo, hi);
+  return *reinterpret_cast<uint32_t *>(&v);
+}
+
+#endif  // __CUDACC__

@@ -1,0 +1,458 @@
+// Stage A, part 1: scan every resident page summary and score it (Eq. 1 of the paper):
+//   s^_j(q_g) = log sum_{i in P_j} exp[(q_g . mu_j + (V_j^T q_g) . c_i) / sqrt(d)]
+// for every page j <= P-2 of every request and every query head g, plus a per-(head, 8-page group)
+// partial (max, sum exp) over the candidate pages 1..P-2 that the selector turns into log Z_g.
+//
+// Two kernels:
+//   scan_generic_kernel   any format / rank / dtype, plain fp32 ALU arithmetic (parity config, fallback
+//                         shapes).  One warp per group of 8 pages.
+//   scan_i4r8_kernel      the bytes-bound path for the r8i4 blob with bf16 queries.  Persistent warps,
+//                         each streaming groups of 8 blobs through its own shared-memory ring with bulk
+//                         async copies (TMA engine) and mbarriers, no CTA-wide synchronisation.  Per page:
+//                           MMA#1  P^T[heads x ranks]  = q[heads x d] . codesV[d x ranks]        (8 x m16n8k16 bf16)
+//                           MMA#2  L[heads x tokens]   = (P_hi | P_lo)[heads x 16] . codesC^T    (2 x m16n8k16 fp16)
+//                         and per 8 pages the centroid dots a[heads x pages] (16 x m16n8k16 bf16, the int8
+//                         centroid split into two exact nibbles).  Integer codes are exact in bf16/fp16, the
+//                         fp32 scales are applied to the fp32 accumulators, the projection is carried into
+//                         MMA#2 as an fp16 hi+lo pair (22 significant bits).
+#include "locks_internal.cuh"
+
+namespace {
+
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+
+struct ScanParams {
+  const void *q;
+  const uint8_t *summ;
+  const int32_t *block_table;
+  const int32_t *seq_lens;
+  float *shat;
+  float2 *part;
+  const float *qnorm;
+  int32_t *status;
+  int batch, Hq, Hkv, G, Pmax, max_groups, num_blocks, k, S, r;
+  float sm_scale;
+};
+
+// ------------------------------------------------------------------------------------------------
+// generic path
+// ------------------------------------------------------------------------------------------------
+
+__device__ __forceinline__ float i4_basis_val(const uint8_t *blob, int l, int c) {
+  int t = c >> 5, w = c & 31, s = w >> 2, half = (w >> 1) & 1, e = w & 1;
+  int j = s >> 1, i = ((s & 1) << 1) | half, nib = i + 4 * e;
+  int byte = (l * 4 + t) * 16 + j * 4 + (nib >> 1);
+  return (float)(((blob[byte] >> ((nib & 1) * 4)) & 15) - 8);
+}
+__device__ __forceinline__ float i4_mu_val(const uint8_t *blob, int r, int c) {
+  int t = c >> 5, w = c & 31, s = w >> 2, half = (w >> 1) & 1, e = w & 1;
+  return (float)((int)blob[i4_off_mu(r) + t * 32 + s * 4 + e * 2 + half] - 128);
+}
+__device__ __forceinline__ float i4_coef_val(const uint8_t *blob, int r, int i, int l) {
+  int x = i & 7, hi = i >> 3, tp = l >> 1, e = l & 1;
+  return (float)((int)blob[i4_off_coef(r) + (x * (r / 2) + tp) * 4 + hi * 2 + e] - 128);
+}
+__device__ __forceinline__ float i4_sc_val(const uint8_t *blob, int r, int i) {
+  int t = (i & 7) >> 1, e = i & 1, hi = i >> 3;
+  return __half2float(*reinterpret_cast<const __half *>(blob + i4_off_sc(r) + 2 * (t * 4 + hi * 2 + e)));
+}
+
+template <int FMT, typename QT>
+__global__ void __launch_bounds__(128) scan_generic_kernel(ScanParams p) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int grp = blockIdx.x * 4 + warp, h = blockIdx.y, b = blockIdx.z;
+  const int T = p.seq_lens[b];
+  const int P = (T + LOCKS_B - 1) / LOCKS_B;
+  if (P <= p.k) return;               // every page is kept: nothing to rank
+  const int nsc = P - 1;              // pages 0 .. P-2 are scored
+  if (grp * LOCKS_GROUP >= nsc) return;
+  const int r = p.r;
+  const QT *q = reinterpret_cast<const QT *>(p.q);
+  for (int g = 0; g < p.G; ++g) {
+    const int hq = h * p.G + g;
+    float qv[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) qv[u] = ldf<QT>(q, ((int64_t)b * p.Hq + hq) * LOCKS_D + lane * 4 + u);
+    float pm = -INFINITY, ps = 0.f;
+    for (int pi = 0; pi < LOCKS_GROUP; ++pi) {
+      const int page = grp * LOCKS_GROUP + pi;
+      if (page >= nsc) break;
+      int block = p.block_table[(int64_t)b * p.Pmax + page];
+      if (block < 0 || block >= p.num_blocks) {
+        if (lane == 0) set_status(p.status, LOCKS_ERR_BAD_BLOCK);
+        continue;
+      }
+      const uint8_t *blob = p.summ + ((int64_t)block * p.Hkv + h) * p.S;
+      float proj[16];
+      float a = 0.f;
+      if (FMT == LOCKS_FMT_F32) {
+        const float *f = reinterpret_cast<const float *>(blob);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) a += f[lane * 4 + u] * qv[u];
+        for (int l = 0; l < r; ++l) {
+          float s = 0.f;
+#pragma unroll
+          for (int u = 0; u < 4; ++u) s += f[LOCKS_D + l * LOCKS_D + lane * 4 + u] * qv[u];
+          proj[l] = warp_sum(s);
+        }
+      } else {
+        const float smu = __half2float(*reinterpret_cast<const __half *>(blob + i4_off_smu(r)));
+#pragma unroll
+        for (int u = 0; u < 4; ++u) a += i4_mu_val(blob, r, lane * 4 + u) * qv[u];
+        a *= smu;
+        for (int l = 0; l < r; ++l) {
+          float s = 0.f;
+#pragma unroll
+          for (int u = 0; u < 4; ++u) s += i4_basis_val(blob, l, lane * 4 + u) * qv[u];
+          const float sv = __half2float(*reinterpret_cast<const __half *>(blob + i4_off_sv(r) + 2 * l));
+          proj[l] = warp_sum(s) * sv;
+        }
+      }
+      a = warp_sum(a);
+      float logit = -INFINITY;
+      if (lane < LOCKS_B) {
+        float s = 0.f;
+        if (FMT == LOCKS_FMT_F32) {
+          const float *f = reinterpret_cast<const float *>(blob) + LOCKS_D + r * LOCKS_D + lane * r;
+          for (int l = 0; l < r; ++l) s += proj[l] * f[l];
+        } else {
+          for (int l = 0; l < r; ++l) s += proj[l] * i4_coef_val(blob, r, lane, l);
+          s *= i4_sc_val(blob, r, lane);
+        }
+        logit = p.sm_scale * (a + s);
+      }
+      const float mx = warp_max(logit);
+      const float z = warp_sum(lane < LOCKS_B ? expf(logit - mx) : 0.f);
+      const float sh = mx + logf(z);
+      if (lane == 0) {
+        p.shat[((int64_t)b * p.Hq + hq) * p.Pmax + page] = sh;
+        if (page >= 1) {  // candidates only
+          const float nm = fmaxf(pm, sh);
+          ps = ps * expf(pm - nm) + expf(sh - nm);
+          pm = nm;
+        }
+      }
+    }
+    if (lane == 0) p.part[((int64_t)b * p.Hq + hq) * p.max_groups + grp] = make_float2(pm, ps);
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// r8i4 tensor path
+// ------------------------------------------------------------------------------------------------
+
+constexpr int kScanWarps = 8;
+constexpr int kScanStages = 2;
+constexpr int kBlob = i4_stride(8);                       // 832
+constexpr int kStageBytes = LOCKS_GROUP * kBlob;          // 6656
+constexpr int kScanSmem = kScanWarps * (kScanStages * kStageBytes + 64);
+
+__device__ __forceinline__ uint32_t nib_pair(uint32_t w, int shift) {
+  // two 4-bit codes (bits shift.. and 16+shift..) -> bf16x2 holding 128 + code each
+  return ((w >> shift) & 0x000F000Fu) | 0x43004300u;
+}
+__device__ __forceinline__ uint32_t bf16x2_sub(uint32_t v, uint32_t c) {
+  __nv_bfloat162 r = __hsub2(*reinterpret_cast<__nv_bfloat162 *>(&v), *reinterpret_cast<__nv_bfloat162 *>(&c));
+  return *reinterpret_cast<uint32_t *>(&r);
+}
+__device__ __forceinline__ uint32_t f16x2_sub(uint32_t v, uint32_t c) {
+  __half2 r = __hsub2(*reinterpret_cast<__half2 *>(&v), *reinterpret_cast<__half2 *>(&c));
+  return *reinterpret_cast<uint32_t *>(&r);
+}
+__device__ __forceinline__ float2 h2f2(uint32_t v) { return __half22float2(*reinterpret_cast<__half2 *>(&v)); }
+__device__ __forceinline__ float fast_ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ float fast_lg2(float x) {
+  float y;
+  asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+struct GroupId {
+  int b, h, grp, nsc;
+};
+
+// NH = number of 8-row halves of the query tile in use (1: G <= 8, 2: G <= 16)
+template <int NH>
+__global__ void __launch_bounds__(kScanWarps * 32, 2) scan_i4r8_kernel(ScanParams p) {
+  extern __shared__ __align__(128) uint8_t smem[];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int x = lane >> 2, t = lane & 3;
+  uint8_t *ring = smem + warp * (kScanStages * kStageBytes);
+  uint64_t *full = reinterpret_cast<uint64_t *>(smem + kScanWarps * kScanStages * kStageBytes + warp * 64);
+  if (lane == 0) {
+    for (int s = 0; s < kScanStages; ++s) mbar_init(&full[s], 1);
+    fence_barrier_init();
+  }
+  __syncwarp();
+
+  const int W = gridDim.x * kScanWarps;
+  const int wid = blockIdx.x * kScanWarps + warp;
+  const int total = p.batch * p.Hkv * p.max_groups;
+
+  auto decode = [&](int gam, GroupId &g) -> bool {
+    const int prob = gam / p.max_groups;
+    g.grp = gam - prob * p.max_groups;
+    g.b = prob / p.Hkv;
+    g.h = prob - g.b * p.Hkv;
+    const int T = p.seq_lens[g.b];
+    const int P = (T + LOCKS_B - 1) / LOCKS_B;
+    g.nsc = (P <= p.k) ? 0 : P - 1;
+    return g.grp * LOCKS_GROUP < g.nsc;
+  };
+  auto next_valid = [&](int gam, GroupId &g) -> int {
+    while (gam < total && !decode(gam, g)) gam += W;
+    return gam;
+  };
+  auto issue = [&](int stage, const GroupId &g) {
+    const int nvalid = min(LOCKS_GROUP, g.nsc - g.grp * LOCKS_GROUP);
+    if (lane == 0) mbar_expect_tx(&full[stage], (uint32_t)nvalid * kBlob);
+    __syncwarp();
+    if (lane < nvalid) {
+      int block = p.block_table[(int64_t)g.b * p.Pmax + g.grp * LOCKS_GROUP + lane];
+      if (block < 0 || block >= p.num_blocks) {
+        set_status(p.status, LOCKS_ERR_BAD_BLOCK);
+        block = 0;
+      }
+      bulk_g2s(ring + stage * kStageBytes + lane * kBlob, p.summ + ((int64_t)block * p.Hkv + g.h) * kBlob, kBlob,
+               &full[stage]);
+    }
+  };
+
+  GroupId gp, gc;
+  int gam_p = next_valid(wid, gp);
+  int inflight = 0;
+#pragma unroll
+  for (int s = 0; s < kScanStages; ++s) {
+    if (gam_p < total) {
+      issue(s, gp);
+      ++inflight;
+      gam_p = next_valid(gam_p + W, gp);
+    }
+  }
+  int gam_c = next_valid(wid, gc);
+
+  // query fragments of the current (request, KV head)
+  uint32_t qa0[8], qa1[8], qa2[8], qa3[8];
+  float kx = 0.f, kx8 = 0.f, pn = 1.f, pn8 = 1.f;
+  int cur_prob = -1;
+  const __nv_bfloat16 *q = reinterpret_cast<const __nv_bfloat16 *>(p.q);
+  const float c2 = p.sm_scale * kLog2e;
+
+  int it = 0;
+  bool ok = true;
+  while (gam_c < total) {
+    const int stage = it % kScanStages;
+    const uint32_t parity = (it / kScanStages) & 1;
+    if (!mbar_wait(&full[stage], parity)) {
+      ok = false;
+      break;
+    }
+    --inflight;
+    const int prob = gc.b * p.Hkv + gc.h;
+    if (prob != cur_prob) {
+      cur_prob = prob;
+      const int hq = gc.h * p.G + x;
+      uint4 v[4] = {}, v8[4] = {};
+      if (x < p.G) {
+        const uint4 *qp = reinterpret_cast<const uint4 *>(q + ((int64_t)gc.b * p.Hq + hq) * LOCKS_D + 32 * t);
+#pragma unroll
+        for (int m = 0; m < 4; ++m) v[m] = __ldg(qp + m);
+        pn = p.qnorm[gc.b * p.Hq + hq];
+      } else {
+        pn = 1.f;
+      }
+      if (NH == 2 && x + 8 < p.G) {
+        const uint4 *qp = reinterpret_cast<const uint4 *>(q + ((int64_t)gc.b * p.Hq + hq + 8) * LOCKS_D + 32 * t);
+#pragma unroll
+        for (int m = 0; m < 4; ++m) v8[m] = __ldg(qp + m);
+        pn8 = p.qnorm[gc.b * p.Hq + hq + 8];
+      } else {
+        pn8 = 1.f;
+      }
+#pragma unroll
+      for (int m = 0; m < 4; ++m) {
+        qa0[2 * m] = v[m].x; qa2[2 * m] = v[m].y; qa0[2 * m + 1] = v[m].z; qa2[2 * m + 1] = v[m].w;
+        qa1[2 * m] = v8[m].x; qa3[2 * m] = v8[m].y; qa1[2 * m + 1] = v8[m].z; qa3[2 * m + 1] = v8[m].w;
+      }
+      kx = c2 / pn;
+      kx8 = c2 / pn8;
+    }
+
+    const uint8_t *sb = ring + stage * kStageBytes;
+    // ---- centroid dots for the 8 pages: a[head][page], int8 = 16 * (hi nibble - 8) + lo nibble
+    float cl[4] = {0.f, 0.f, 0.f, 0.f}, ch[4] = {0.f, 0.f, 0.f, 0.f};
+    {
+      const uint4 *mp = reinterpret_cast<const uint4 *>(sb + x * kBlob + i4_off_mu(8) + t * 32);
+      const uint4 m0 = mp[0], m1 = mp[1];
+      const uint32_t mw[8] = {m0.x, m0.y, m0.z, m0.w, m1.x, m1.y, m1.z, m1.w};
+#pragma unroll
+      for (int s = 0; s < 8; ++s) {
+        const uint32_t w = mw[s];
+        const uint32_t l0 = bf16x2_sub(nib_pair(w, 0), 0x43004300u);   // - 128
+        const uint32_t l1 = bf16x2_sub(nib_pair(w, 8), 0x43004300u);
+        const uint32_t h0 = bf16x2_sub(nib_pair(w, 4), 0x43084308u);   // - 136
+        const uint32_t h1 = bf16x2_sub(nib_pair(w, 12), 0x43084308u);
+        mma_bf16(cl, qa0[s], qa1[s], qa2[s], qa3[s], l0, l1);
+        mma_bf16(ch, qa0[s], qa1[s], qa2[s], qa3[s], h0, h1);
+      }
+    }
+    float acen[2 * NH];  // log2-domain centroid term for pages 2t, 2t+1 (and the second row half)
+    {
+      const float s0 = __half2float(*reinterpret_cast<const __half *>(sb + (2 * t) * kBlob + i4_off_smu(8)));
+      const float s1 = __half2float(*reinterpret_cast<const __half *>(sb + (2 * t + 1) * kBlob + i4_off_smu(8)));
+      acen[0] = s0 * c2 * fmaf(16.f, ch[0], cl[0]);
+      acen[1] = s1 * c2 * fmaf(16.f, ch[1], cl[1]);
+      if (NH == 2) {
+        acen[2] = s0 * c2 * fmaf(16.f, ch[2], cl[2]);
+        acen[3] = s1 * c2 * fmaf(16.f, ch[3], cl[3]);
+      }
+    }
+    float res[2 * NH];
+#pragma unroll
+    for (int i = 0; i < 2 * NH; ++i) res[i] = 0.f;
+
+#pragma unroll
+    for (int pg = 0; pg < LOCKS_GROUP; ++pg) {
+      const uint8_t *pb = sb + pg * kBlob;
+      const uint4 w4 = *reinterpret_cast<const uint4 *>(pb + lane * 16);
+      const uint32_t ww[4] = {w4.x, w4.y, w4.z, w4.w};
+      float c1[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const uint32_t w = ww[j];
+        const uint32_t r0 = bf16x2_sub(nib_pair(w, 0), 0x43084308u);
+        const uint32_t r1 = bf16x2_sub(nib_pair(w, 4), 0x43084308u);
+        const uint32_t r2 = bf16x2_sub(nib_pair(w, 8), 0x43084308u);
+        const uint32_t r3 = bf16x2_sub(nib_pair(w, 12), 0x43084308u);
+        mma_bf16(c1, qa0[2 * j], qa1[2 * j], qa2[2 * j], qa3[2 * j], r0, r1);
+        mma_bf16(c1, qa0[2 * j + 1], qa1[2 * j + 1], qa2[2 * j + 1], qa3[2 * j + 1], r2, r3);
+      }
+      // projection -> fp16 hi + lo
+      const float2 sv = h2f2(*reinterpret_cast<const uint32_t *>(pb + i4_off_sv(8) + 4 * t));
+      const float p0 = c1[0] * sv.x * pn, p1 = c1[1] * sv.y * pn;
+      const uint32_t hi = pack_f16(p0, p1);
+      const float2 hf = h2f2(hi);
+      const uint32_t lo = pack_f16(p0 - hf.x, p1 - hf.y);
+      uint32_t hi8 = 0u, lo8 = 0u;
+      if (NH == 2) {
+        const float p2 = c1[2] * sv.x * pn8, p3 = c1[3] * sv.y * pn8;
+        hi8 = pack_f16(p2, p3);
+        const float2 hf8 = h2f2(hi8);
+        lo8 = pack_f16(p2 - hf8.x, p3 - hf8.y);
+      }
+      // coefficient codes (offset-binary int8) -> exact fp16
+      const uint32_t cw = *reinterpret_cast<const uint32_t *>(pb + i4_off_coef(8) + lane * 4);
+      const uint32_t b0 = f16x2_sub(__byte_perm(cw, 0x64646464u, 0x4140), 0x64806480u);
+      const uint32_t b1 = f16x2_sub(__byte_perm(cw, 0x64646464u, 0x4342), 0x64806480u);
+      float ca[4] = {0.f, 0.f, 0.f, 0.f}, cb[4] = {0.f, 0.f, 0.f, 0.f};
+      mma_f16(ca, hi, hi8, lo, lo8, b0, b0);
+      mma_f16(cb, hi, hi8, lo, lo8, b1, b1);
+      const uint2 scw = *reinterpret_cast<const uint2 *>(pb + i4_off_sc(8) + 8 * t);
+      const float2 s01 = h2f2(scw.x), s89 = h2f2(scw.y);
+#pragma unroll
+      for (int hh = 0; hh < NH; ++hh) {
+        const float kk = hh ? kx8 : kx;
+        const float l0 = ca[2 * hh] * (s01.x * kk), l1 = ca[2 * hh + 1] * (s01.y * kk);
+        const float l2 = cb[2 * hh] * (s89.x * kk), l3 = cb[2 * hh + 1] * (s89.y * kk);
+        float m = fmaxf(fmaxf(l0, l1), fmaxf(l2, l3));
+        m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 1));
+        m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 2));
+        float e = fast_ex2(l0 - m) + fast_ex2(l1 - m) + fast_ex2(l2 - m) + fast_ex2(l3 - m);
+        e += __shfl_xor_sync(0xffffffffu, e, 1);
+        e += __shfl_xor_sync(0xffffffffu, e, 2);
+        const float v = m + fast_lg2(e);
+        if (t == (pg >> 1)) res[2 * hh + (pg & 1)] = v;
+      }
+    }
+    __syncwarp();  // every lane is done reading this stage
+    if (gam_p < total) {
+      issue(stage, gp);
+      ++inflight;
+      gam_p = next_valid(gam_p + W, gp);
+    }
+
+    // ---- write s^ and the group's candidate partial
+    const int page0 = gc.grp * LOCKS_GROUP + 2 * t;
+#pragma unroll
+    for (int hh = 0; hh < NH; ++hh) {
+      const int g = x + 8 * hh;
+      const float v0 = (res[2 * hh] + acen[2 * hh]) * kLn2;
+      const float v1 = (res[2 * hh + 1] + acen[2 * hh + 1]) * kLn2;
+      const bool in0 = page0 < gc.nsc, in1 = page0 + 1 < gc.nsc;
+      if (g < p.G) {
+        float *dst = p.shat + ((int64_t)gc.b * p.Hq + gc.h * p.G + g) * p.Pmax + page0;
+        if (in0) dst[0] = v0;
+        if (in1) dst[1] = v1;
+      }
+      const float c0 = (in0 && page0 >= 1) ? v0 : -INFINITY;
+      const float c1v = in1 ? v1 : -INFINITY;
+      float m = fmaxf(c0, c1v);
+      m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 1));
+      m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 2));
+      float e = (m == -INFINITY) ? 0.f : (__expf(c0 - m) + __expf(c1v - m));
+      e += __shfl_xor_sync(0xffffffffu, e, 1);
+      e += __shfl_xor_sync(0xffffffffu, e, 2);
+      if (t == 0 && g < p.G)
+        p.part[((int64_t)gc.b * p.Hq + gc.h * p.G + g) * p.max_groups + gc.grp] = make_float2(m, e);
+    }
+    gam_c = next_valid(gam_c + W, gc);
+    ++it;
+  }
+  if (!ok) {
+    // a wait ran out: flag it, then give copies still in flight a bounded chance to land before exit
+    if (lane == 0) set_status(p.status, LOCKS_ERR_TIMEOUT);
+    for (int s = 0; s < inflight && s < kScanStages; ++s) {
+      const int st = (it + s) % kScanStages;
+      (void)mbar_wait(&full[st], ((it + s) / kScanStages) & 1);
+    }
+  }
+}
+
+}  // namespace
+
+int locks_launch_scan(locks_ctx *c, const void *q, const void *summaries, const locks_kv *kv, int batch,
+                      float *shat, cudaStream_t st) {
+  ScanParams p;
+  p.q = q;
+  p.summ = reinterpret_cast<const uint8_t *>(summaries);
+  p.block_table = kv->block_table;
+  p.seq_lens = kv->seq_lens;
+  p.shat = shat;
+  p.part = c->part;
+  p.qnorm = c->qnorm;
+  p.status = c->status;
+  p.batch = batch; p.Hq = c->cfg.num_q_heads; p.Hkv = c->cfg.num_kv_heads; p.G = c->G;
+  p.Pmax = c->Pmax; p.max_groups = c->max_groups; p.num_blocks = kv->num_blocks; p.k = c->k;
+  p.S = c->S; p.r = c->cfg.rank; p.sm_scale = c->cfg.sm_scale;
+  const bool tensor = c->cfg.summary_fmt == LOCKS_FMT_I4 && c->cfg.rank == 8 && c->cfg.q_dtype == LOCKS_BF16;
+  if (tensor) {
+    static bool attr_done = false;
+    if (!attr_done) {
+      cudaFuncSetAttribute(scan_i4r8_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kScanSmem);
+      cudaFuncSetAttribute(scan_i4r8_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kScanSmem);
+      attr_done = true;
+    }
+    const int total_groups = batch * p.Hkv * p.max_groups;
+    int grid = 2 * c->num_sms;
+    const int need = (total_groups + kScanWarps - 1) / kScanWarps;
+    if (grid > need) grid = need < 1 ? 1 : need;
+    if (c->G <= 8) scan_i4r8_kernel<1><<<grid, kScanWarps * 32, kScanSmem, st>>>(p);
+    else scan_i4r8_kernel<2><<<grid, kScanWarps * 32, kScanSmem, st>>>(p);
+  } else {
+    dim3 grid((c->max_groups + 3) / 4, p.Hkv, batch);
+    const bool qbf = c->cfg.q_dtype == LOCKS_BF16;
+    if (c->cfg.summary_fmt == LOCKS_FMT_F32) {
+      if (qbf) scan_generic_kernel<LOCKS_FMT_F32, __nv_bfloat16><<<grid, 128, 0, st>>>(p);
+      else scan_generic_kernel<LOCKS_FMT_F32, float><<<grid, 128, 0, st>>>(p);
+    } else {
+      if (qbf) scan_generic_kernel<LOCKS_FMT_I4, __nv_bfloat16><<<grid, 128, 0, st>>>(p);
+      else scan_generic_kernel<LOCKS_FMT_I4, float><<<grid, 128, 0, st>>>(p);
+    }
+  }
+  return locks_check_launch(c);
+}

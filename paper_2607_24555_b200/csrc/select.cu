@@ -1,0 +1,278 @@
+// Stage A, part 2: share-average combine and budgeted page selection (Sec. 4 of the paper):
+//   log Z_g   = log sum_{j in 1..P-2} exp s^_j(q_g)                       (candidates only)
+//   log m_bar_j = log( (1/G) sum_g exp(s^_j(q_g) - log Z_g) )
+//   S = {0, P-1}  U  top-(k-2) candidates by log m_bar_j (ties: lower page index), ids ascending.
+// Stage 1 (one CTA per 2048-page chunk of a (request, KV head)) ranks its chunk with an exact
+// 4-pass radix select held in registers + shared-memory histograms and compacts the winners in
+// page order.  With one chunk it writes the final table; with several, each chunk emits its own
+// top-(k-2) (value, page) list and stage 2 re-selects among them (a chunk's local top-(k-2) always
+// contains the chunk's share of the global top-(k-2), ties included, because both use the same
+// lower-index tie rule and lists stay in page order).
+#include "locks_internal.cuh"
+
+namespace {
+
+struct SelParams {
+  const float *shat;
+  const float2 *part;
+  const int32_t *seq_lens;
+  int32_t *ids, *cnt;
+  float *logshare;
+  float *cand_val;
+  int32_t *cand_idx;
+  int batch, Hq, Hkv, G, Pmax, max_groups, k, chunks, kc;
+};
+
+__device__ __forceinline__ uint32_t order_key(float f) {
+  uint32_t u = __float_as_uint(f);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+// Exact top-K among the block's N = THREADS*EPT keys (thread-major order = ascending index order).
+// sel[i] is set for the K winners: every key above the K-th largest, plus the lowest-indexed keys
+// equal to it.  pos[i] = rank of a winner in index order.  Requires K <= number of valid keys.
+template <int EPT>
+__device__ void block_topk(const uint32_t (&key)[EPT], int K, bool (&sel)[EPT], int (&pos)[EPT], int *sh_hist,
+                           int *sh_misc) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (K <= 0) {  // nothing to pick (k = 2): uniform across the block
+#pragma unroll
+    for (int i = 0; i < EPT; ++i) { sel[i] = false; pos[i] = 0; }
+    return;
+  }
+  uint32_t prefix = 0, mask = 0;
+  int remaining = K;
+  for (int pass = 0; pass < 4; ++pass) {
+    const int shift = 24 - 8 * pass;
+    sh_hist[tid] = 0;  // 256 bins, 256 threads
+    __syncthreads();
+#pragma unroll
+    for (int i = 0; i < EPT; ++i)
+      if ((key[i] & mask) == prefix) atomicAdd(&sh_hist[(key[i] >> shift) & 255], 1);
+    __syncthreads();
+    if (warp == 0) {
+      // bins high -> low: lane owns bins 255-8*lane .. 248-8*lane
+      int c[8], tot = 0;
+#pragma unroll
+      for (int u = 0; u < 8; ++u) { c[u] = sh_hist[255 - (lane * 8 + u)]; tot += c[u]; }
+      int incl = tot;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        int v = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += v;
+      }
+      int before = incl - tot;  // keys in strictly higher bins than this lane's
+      if (before < remaining && remaining <= incl) {
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          if (before < remaining && remaining <= before + c[u]) {
+            sh_misc[0] = 255 - (lane * 8 + u);
+            sh_misc[1] = remaining - before;
+          }
+          before += c[u];
+        }
+      }
+    }
+    __syncthreads();
+    prefix |= (uint32_t)sh_misc[0] << shift;
+    mask |= 255u << shift;
+    remaining = sh_misc[1];
+    __syncthreads();
+  }
+  // prefix is the K-th largest key; `remaining` of the keys equal to it are taken, lowest index first
+  int ngt = 0, neq = 0;
+#pragma unroll
+  for (int i = 0; i < EPT; ++i) { ngt += key[i] > prefix; neq += key[i] == prefix; }
+  // block exclusive scan of (ngt, neq) packed into one int
+  int packed = (ngt << 16) | neq;
+  int incl = packed;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    int v = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += v;
+  }
+  if (lane == 31) sh_misc[2 + warp] = incl;
+  __syncthreads();
+  int base = 0;
+  for (int w = 0; w < warp; ++w) base += sh_misc[2 + w];
+  int excl = base + incl - packed;
+  int gt_before = excl >> 16, eq_before = excl & 0xffff;
+#pragma unroll
+  for (int i = 0; i < EPT; ++i) {
+    const bool gt = key[i] > prefix, eq = key[i] == prefix;
+    const bool take = gt || (eq && eq_before < remaining);
+    sel[i] = take;
+    pos[i] = gt_before + min(eq_before, remaining);
+    gt_before += gt;
+    eq_before += eq;
+  }
+  __syncthreads();
+}
+
+// log Z_g of every head of the group from the scan's per-group partials -> sh_logz[g]
+__device__ void group_logz(const SelParams &p, int b, int h, int ngroups, float *sh_logz) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  for (int g = warp; g < p.G; g += LOCKS_SEL_THREADS / 32) {
+    const float2 *pp = p.part + ((int64_t)b * p.Hq + h * p.G + g) * p.max_groups;
+    float m = -INFINITY, s = 0.f;
+    for (int i = lane; i < ngroups; i += 32) {
+      const float2 v = pp[i];
+      if (v.x > -INFINITY) {
+        const float nm = fmaxf(m, v.x);
+        s = s * expf(m - nm) + v.y * expf(v.x - nm);
+        m = nm;
+      }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const float om = __shfl_xor_sync(0xffffffffu, m, o), os = __shfl_xor_sync(0xffffffffu, s, o);
+      const float nm = fmaxf(m, om);
+      if (nm > -INFINITY) {
+        s = s * expf(m - nm) + os * expf(om - nm);
+        m = nm;
+      }
+    }
+    if (lane == 0) sh_logz[g] = m + logf(s);
+  }
+}
+
+__global__ void __launch_bounds__(LOCKS_SEL_THREADS) select_stage1_kernel(SelParams p) {
+  __shared__ int sh_hist[256];
+  __shared__ int sh_misc[2 + LOCKS_SEL_THREADS / 32];
+  __shared__ float sh_logz[16];
+  const int chunk = blockIdx.x, h = blockIdx.y, b = blockIdx.z, tid = threadIdx.x;
+  const int T = p.seq_lens[b];
+  const int P = (T + LOCKS_B - 1) / LOCKS_B;
+  const int64_t prob = (int64_t)b * p.Hkv + h;
+  int32_t *ids = p.ids + prob * p.k;
+  if (P <= p.k) {  // every page is kept
+    if (chunk == 0) {
+      for (int j = tid; j < p.k; j += LOCKS_SEL_THREADS) ids[j] = j < P ? j : -1;
+      if (tid == 0) p.cnt[prob] = P;
+    }
+    return;
+  }
+  const int c0 = chunk * LOCKS_SEL_CHUNK;  // first page of this chunk
+  const int ncand_total = P - 2;
+  if (c0 > P - 2) {  // chunk past the candidates: emit an empty list
+    if (p.chunks > 1)
+      for (int j = tid; j < p.kc; j += LOCKS_SEL_THREADS) {
+        p.cand_val[(prob * p.chunks + chunk) * p.kc + j] = -INFINITY;
+        p.cand_idx[(prob * p.chunks + chunk) * p.kc + j] = -1;
+      }
+    return;
+  }
+  group_logz(p, b, h, (P - 1 + LOCKS_GROUP - 1) / LOCKS_GROUP, sh_logz);
+  __syncthreads();
+  // log m_bar for this thread's 8 consecutive pages
+  float val[LOCKS_SEL_EPT];
+  uint32_t key[LOCKS_SEL_EPT];
+  const int pbase = c0 + tid * LOCKS_SEL_EPT;
+  float mx[LOCKS_SEL_EPT], sm[LOCKS_SEL_EPT];
+#pragma unroll
+  for (int i = 0; i < LOCKS_SEL_EPT; ++i) { mx[i] = -INFINITY; sm[i] = 0.f; }
+  for (int g = 0; g < p.G; ++g) {
+    const float *row = p.shat + ((int64_t)b * p.Hq + h * p.G + g) * p.Pmax;
+    const float lz = sh_logz[g];
+#pragma unroll
+    for (int i = 0; i < LOCKS_SEL_EPT; ++i) {
+      const int page = pbase + i;
+      if (page >= 1 && page <= P - 2) {
+        const float tv = row[page] - lz;
+        const float nm = fmaxf(mx[i], tv);
+        sm[i] = sm[i] * expf(mx[i] - nm) + expf(tv - nm);
+        mx[i] = nm;
+      }
+    }
+  }
+  const float logG = logf((float)p.G);
+  int nvalid_local = 0;
+#pragma unroll
+  for (int i = 0; i < LOCKS_SEL_EPT; ++i) {
+    const int page = pbase + i;
+    const bool valid = page >= 1 && page <= P - 2;
+    val[i] = valid ? mx[i] + logf(sm[i]) - logG : -INFINITY;
+    key[i] = valid ? order_key(val[i]) : 0u;
+    nvalid_local += valid;
+    if (valid && p.logshare) p.logshare[prob * p.Pmax + page] = val[i];
+  }
+  const int cand_in_chunk = min(P - 2, c0 + LOCKS_SEL_CHUNK - 1) - max(1, c0) + 1;
+  const int K = min(p.k - 2, cand_in_chunk);
+  bool sel[LOCKS_SEL_EPT];
+  int pos[LOCKS_SEL_EPT];
+  block_topk<LOCKS_SEL_EPT>(key, K, sel, pos, sh_hist, sh_misc);
+  if (p.chunks == 1) {
+#pragma unroll
+    for (int i = 0; i < LOCKS_SEL_EPT; ++i)
+      if (sel[i]) ids[1 + pos[i]] = pbase + i;
+    if (tid == 0) {
+      ids[0] = 0;
+      ids[p.k - 1] = P - 1;
+      p.cnt[prob] = p.k;
+    }
+  } else {
+    float *cv = p.cand_val + (prob * p.chunks + chunk) * p.kc;
+    int32_t *ci = p.cand_idx + (prob * p.chunks + chunk) * p.kc;
+#pragma unroll
+    for (int i = 0; i < LOCKS_SEL_EPT; ++i)
+      if (sel[i]) { cv[pos[i]] = val[i]; ci[pos[i]] = pbase + i; }
+    for (int j = K + tid; j < p.kc; j += LOCKS_SEL_THREADS) { cv[j] = -INFINITY; ci[j] = -1; }
+  }
+  (void)ncand_total; (void)nvalid_local;
+}
+
+template <int EPT>
+__global__ void __launch_bounds__(LOCKS_SEL_THREADS) select_stage2_kernel(SelParams p) {
+  __shared__ int sh_hist[256];
+  __shared__ int sh_misc[2 + LOCKS_SEL_THREADS / 32];
+  const int h = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
+  const int T = p.seq_lens[b];
+  const int P = (T + LOCKS_B - 1) / LOCKS_B;
+  if (P <= p.k) return;  // stage 1 already wrote the table
+  const int64_t prob = (int64_t)b * p.Hkv + h;
+  const int N = p.chunks * p.kc;
+  const float *cv = p.cand_val + prob * N;
+  const int32_t *ci = p.cand_idx + prob * N;
+  uint32_t key[EPT];
+  int idx[EPT];
+#pragma unroll
+  for (int i = 0; i < EPT; ++i) {
+    const int j = tid * EPT + i;
+    const bool valid = j < N && ci[j] >= 0;
+    idx[i] = valid ? ci[j] : -1;
+    key[i] = valid ? order_key(cv[j]) : 0u;
+  }
+  bool sel[EPT];
+  int pos[EPT];
+  block_topk<EPT>(key, p.k - 2, sel, pos, sh_hist, sh_misc);
+  int32_t *ids = p.ids + prob * p.k;
+#pragma unroll
+  for (int i = 0; i < EPT; ++i)
+    if (sel[i]) ids[1 + pos[i]] = idx[i];
+  if (tid == 0) {
+    ids[0] = 0;
+    ids[p.k - 1] = P - 1;
+    p.cnt[prob] = p.k;
+  }
+}
+
+}  // namespace
+
+int locks_launch_select(locks_ctx *c, const float *shat, const locks_kv *kv, int batch, int32_t *ids,
+                        int32_t *cnt, float *logshare, cudaStream_t st) {
+  SelParams p;
+  p.shat = shat; p.part = c->part; p.seq_lens = kv->seq_lens; p.ids = ids; p.cnt = cnt; p.logshare = logshare;
+  p.cand_val = c->cand_val; p.cand_idx = c->cand_idx;
+  p.batch = batch; p.Hq = c->cfg.num_q_heads; p.Hkv = c->cfg.num_kv_heads; p.G = c->G; p.Pmax = c->Pmax;
+  p.max_groups = c->max_groups; p.k = c->k; p.chunks = c->sel_chunks; p.kc = c->sel_kc;
+  select_stage1_kernel<<<dim3(c->sel_chunks, p.Hkv, batch), LOCKS_SEL_THREADS, 0, st>>>(p);
+  int rc = locks_check_launch(c);
+  if (rc != LOCKS_OK || c->sel_chunks == 1) return rc;
+  const int N = c->sel_chunks * c->sel_kc;
+  const int ept = (N + LOCKS_SEL_THREADS - 1) / LOCKS_SEL_THREADS;
+  dim3 grid(p.Hkv, batch);
+  if (ept <= 8) select_stage2_kernel<8><<<grid, LOCKS_SEL_THREADS, 0, st>>>(p);
+  else if (ept <= 32) select_stage2_kernel<32><<<grid, LOCKS_SEL_THREADS, 0, st>>>(p);
+  else return LOCKS_ERR_UNSUPPORTED;
+  return locks_check_launch(c);
+}

@@ -1,0 +1,328 @@
+"""GPU parity: the CUDA path (through the C ABI) against the CPU oracle on the same seeded inputs.
+
+Tolerances (written here, derived in the design doc): page log-masses and log-shares within 1e-3;
+selected page sets identical except inside a 2e-3 tie band around the oracle's threshold;
+attention outputs within 2e-2 (bf16 KV) / 1e-4 (fp32); lse within 1e-3.
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import locks_synth
+import oracle
+from common import t2np
+
+pytestmark = pytest.mark.gpu
+
+
+def _gc(w, **kw):
+    from gpu_util import GpuCase
+    return GpuCase(w, **kw)
+
+
+def small_bf16(seq_lens, Hq=8, Hkv=2, rank=8, budget=256, **kw):
+    return locks_synth.Workload("small", list(seq_lens), Hq=Hq, Hkv=Hkv, rank=rank, budget=budget, **kw)
+
+
+# ----------------------------------------------------------------------------- config 0 (fp32)
+
+def test_config0_tiny_fp32_pipeline():
+    from gpu_util import check_select_and_attend
+    gc = _gc(locks_synth.config0())
+    summ = gc.oracle_summaries()
+    differed = check_select_and_attend(gc, summ, out_tol=1e-4, mass_tol=1e-4)
+    assert differed == 0
+    # planted carriers are all selected
+    ids, cnt, _, _ = gc.gpu_select(torch.from_numpy(summ).cuda())
+    for cp in gc.case.carrier_pages[0]:
+        assert cp in ids[0, 0].tolist()
+    # dense attention through the same entry point
+    out, lse = gc.gpu_attend()
+    oout, olse = oracle.attend(gc.cache, t2np(gc.case.q), gc.sm)
+    assert np.abs(out - oout).max() <= 1e-4 and np.abs(lse - olse).max() <= 1e-3
+
+
+def test_config0_soft_queries_exercise_the_merge():
+    """With carriers the softmax is one-hot; a scaled-down query spreads mass over many pages."""
+    from gpu_util import check_select_and_attend
+    gc = _gc(locks_synth.config0().with_(carriers=0, q_scale=0.25, seq_lens=[4096 - 5]))
+    check_select_and_attend(gc, gc.oracle_summaries(), out_tol=1e-4, mass_tol=1e-4)
+
+
+def test_f32_build_matches_oracle_scores():
+    """F32-format build: bases are compared through scores and projectors, never entry by entry."""
+    gc = _gc(locks_synth.config0().with_(seq_lens=[1024]))
+    w = gc.w
+    g_summ = gc.gpu_build().cpu().numpy()
+    o_summ = gc.oracle_summaries()
+    rng = np.random.default_rng(0)
+    bt = gc.cache.block_table[0]
+    for p in range(0, 63):
+        mu_g, V_g, C_g = oracle.unpack(oracle.FMT_F32, w.rank, g_summ[bt[p], 0])
+        mu_o, V_o, C_o = oracle.unpack(oracle.FMT_F32, w.rank, o_summ[bt[p], 0])
+        assert np.abs(mu_g - mu_o).max() < 1e-5
+        assert np.abs(V_g @ V_g.T - np.eye(w.rank)).max() < 1e-4          # orthonormal
+        assert np.abs(C_g.sum(0)).max() < 1e-3                              # centred coefficients
+        for _ in range(4):
+            q = rng.standard_normal(128)
+            assert abs(oracle.score(mu_g, V_g, C_g, q, gc.sm) - oracle.score(mu_o, V_o, C_o, q, gc.sm)) < 1e-4
+        assert np.abs(V_g.T @ V_g - V_o.T @ V_o).max() < 2e-3               # same subspace (gap is large here)
+    assert gc.status() == 0
+
+
+def test_full_rank_gpu_summary_is_exact():
+    """r = B = 16 in the F32 format reproduces the exact page log-mass (Prop. 3)."""
+    gc = _gc(locks_synth.config0().with_(rank=16, seq_lens=[800], n_dirs=0, carriers=0))
+    summ = gc.gpu_build()
+    ids, cnt, logmass, _ = gc.gpu_select(summ)
+    exact = oracle.page_logmass(gc.cache, t2np(gc.case.q), 16, gc.fmt, None, gc.sm, exact=True)
+    assert np.abs(logmass[0, :, :49] - exact[0, :, :49]).max() < 1e-3
+
+
+# ----------------------------------------------------------------------------- bf16 + I4 path
+
+@pytest.mark.parametrize("Hq,Hkv", [(8, 2), (4, 4), (8, 1), (16, 1), (32, 2), (6, 2)])
+def test_i4_tensor_path_group_sizes(Hq, Hkv):
+    from gpu_util import check_select_and_attend
+    gc = _gc(small_bf16([2048 + 37, 4096, 700], Hq=Hq, Hkv=Hkv, budget=256, seed=Hq + Hkv))
+    check_select_and_attend(gc, gc.oracle_summaries(), out_tol=2e-2)
+
+
+@pytest.mark.parametrize("lens,budget", [([16], 64), ([17, 1, 33], 64), ([16 * 5], 64), ([16 * 5 + 1], 64),
+                                         ([16 * 6 + 1], 64), ([2000, 48, 640], 512), ([130], 32)])
+def test_edge_lengths(lens, budget):
+    """Single page, P <= k, P = k + 1, partial tail pages, k = 2."""
+    from gpu_util import check_select_and_attend
+    gc = _gc(small_bf16(lens, budget=budget, seed=len(lens)))
+    check_select_and_attend(gc, gc.oracle_summaries(), out_tol=2e-2)
+    out, lse = gc.gpu_attend()                                            # dense
+    oout, olse = oracle.attend(gc.cache, t2np(gc.case.q), gc.sm)
+    assert np.abs(out - oout).max() <= 2e-2 and np.abs(lse - olse).max() <= 1e-3
+
+
+def test_carriers_and_nhd_layout():
+    from gpu_util import check_select_and_attend
+    gc = _gc(small_bf16([3000, 1500], carriers=8, layout="NHD", seed=11))
+    differed = check_select_and_attend(gc, gc.oracle_summaries(), out_tol=2e-2)
+    ids, _, _, _ = gc.gpu_select(torch.from_numpy(gc.oracle_summaries()).cuda())
+    for b in range(2):
+        for cp in gc.case.carrier_pages[b]:
+            assert all(cp in ids[b, h].tolist() for h in range(gc.w.Hkv))
+    assert differed <= 1
+
+
+def test_tail_slots_are_never_read_as_data():
+    """Cache slots past the sequence end hold NaN: outputs must not change."""
+    from gpu_util import check_select_and_attend
+    gc = _gc(small_bf16([1000, 333], tail_fill=float("nan"), seed=5))
+    check_select_and_attend(gc, gc.oracle_summaries(), out_tol=2e-2)
+
+
+@pytest.mark.parametrize("rank", [2, 4])
+def test_i4_generic_ranks(rank):
+    from gpu_util import check_select_and_attend
+    gc = _gc(small_bf16([1200, 800], rank=rank, seed=rank))
+    check_select_and_attend(gc, gc.oracle_summaries(), out_tol=2e-2)
+
+
+def test_two_level_select_long_context():
+    """More than one 2048-page chunk per KV head: stage-1 lists + stage-2 re-select."""
+    from gpu_util import check_select_and_attend
+    gc = _gc(locks_synth.Workload("long", [16 * 4500 + 3], Hq=32, Hkv=2, budget=2048, seed=9))
+    differed = check_select_and_attend(gc, gc.oracle_summaries(), out_tol=2e-2)
+    assert differed <= 1
+
+
+def test_ties_resolve_to_lower_index():
+    """All keys identical and a zero query: every candidate ties, the lowest indices win."""
+    gc = _gc(small_bf16([16 * 40], Hq=4, Hkv=1, budget=128))
+    gc.case.k.fill_(0.5)
+    gc.case.q.zero_()
+    from gpu_util import GpuCase
+    gc.cache = __import__("common").oracle_cache(gc.case)
+    summ = gc.oracle_summaries()
+    ids, cnt, _, _ = gc.gpu_select(torch.from_numpy(summ).cuda())
+    assert cnt[0, 0] == 8 and ids[0, 0].tolist() == [0, 1, 2, 3, 4, 5, 6, 39]
+
+
+def test_gpu_i4_build_decoupled_parity():
+    """I4 build: codes agree with the oracle's on >= 99.9 % of entries (|diff| <= 1 elsewhere), the
+    stored scales are the fp16 abs-max scales of the blob's own values, probe scores stay close."""
+    gc = _gc(small_bf16([16 * 600], Hq=8, Hkv=2, seed=21))
+    w = gc.w
+    g_summ = gc.gpu_build().cpu().numpy()
+    o_summ = gc.oracle_summaries()
+    rng = np.random.default_rng(1)
+    bt = gc.cache.block_table[0]
+    tot = diff = 0
+    worst = 0.0
+    for p in range(600):
+        for h in range(2):
+            gV, gC, gMu, gsV, gsC, gsMu = oracle.unpack_codes(8, g_summ[bt[p], h])
+            oV, oC, oMu, osV, osC, osMu = oracle.unpack_codes(8, o_summ[bt[p], h])
+            for a, b_ in ((gV, oV), (gC, oC), (gMu, oMu)):
+                d = np.abs(a - b_)
+                assert d.max() <= 1
+                tot += d.size; diff += int((d > 0).sum())
+            assert np.all(np.abs(gsV - osV) <= np.spacing(np.float16(osV)).astype(np.float64) + 0)
+            assert np.all(np.abs(gsC - osC) <= np.spacing(np.float16(osC)).astype(np.float64) + 0)
+            assert abs(gsMu - osMu) <= float(np.spacing(np.float16(osMu)))
+            if p % 10 == 0:
+                mg = oracle.unpack(oracle.FMT_I4, 8, g_summ[bt[p], h])
+                mo = oracle.unpack(oracle.FMT_I4, 8, o_summ[bt[p], h])
+                q = rng.standard_normal(128)
+                worst = max(worst, abs(oracle.score(*mg, q, gc.sm) - oracle.score(*mo, q, gc.sm)))
+    assert diff / tot <= 1e-3, diff / tot
+    assert worst <= 5e-3, worst
+    assert gc.status() == 0
+
+
+def test_decode_step_matches_stepwise_oracle():
+    """locks_decode_step with appends across page boundaries; summaries of freshly filled pages
+    are built on the device and handed to the oracle (identical bytes) for the next steps."""
+    from common import check_page_sets, oracle_cache
+    w = small_bf16([16 * 130 - 3, 16 * 90 + 14, 500], Hq=8, Hkv=2, budget=256, spare_blocks=0, seed=33)
+    reserve = 3
+    w = w.with_(seq_lens=[t + 16 * reserve for t in w.seq_lens])     # room to grow
+    gc = _gc(w)
+    start = torch.tensor([t - 16 * reserve for t in w.seq_lens], dtype=torch.int32, device="cuda:0")
+    gc.case.seq_lens.copy_(start)
+    summ = gc.ctx.new_summaries(gc.case.num_blocks)
+    gc.ctx.locks_build_summaries(gc.kv, w.n, summ)
+    out = torch.empty(w.n, w.Hq, w.d, dtype=torch.bfloat16, device="cuda:0")
+    ids = torch.empty(w.n, w.Hkv, gc.k, dtype=torch.int32, device="cuda:0")
+    cnt = torch.empty(w.n, w.Hkv, dtype=torch.int32, device="cuda:0")
+    for step in range(36):
+        kn, vn, qn = locks_synth.new_token(w, step, device="cuda:0")
+        gc.ctx.locks_decode_step(qn, kn, vn, gc.kv, summ, w.n, out, ids, cnt)
+        torch.cuda.synchronize()
+        assert gc.status() == 0
+        assert gc.case.seq_lens.cpu().tolist() == [int(s) + step + 1 for s in start.cpu()]
+        cache = oracle_cache(gc.case)                               # cache now holds the new token
+        summ_np = summ.cpu().numpy()
+        shat = oracle.page_logmass(cache, t2np(qn), w.rank, gc.fmt, summ_np, gc.sm)
+        oids, ocnt, ols = oracle.select(cache, shat, gc.k)
+        check_page_sets(ids.cpu().numpy(), cnt.cpu().numpy(), oids, ocnt, ols, cache.seq_lens, w.B, gc.k)
+        oout, _ = oracle.attend(cache, t2np(qn), gc.sm, ids.cpu().numpy(), cnt.cpu().numpy())
+        assert np.abs(out.float().cpu().numpy() - oout).max() <= 2e-2, step
+        # a page that just filled has a summary now, equal in quality to the bulk build
+        for b in range(w.n):
+            T = int(cache.seq_lens[b])
+            if T % 16 == 0:
+                blk = cache.block_table[b, T // 16 - 1]
+                ref = oracle.build_summaries(cache, w.rank, gc.fmt, page_begin=[T // 16 - 1 if i == b else 0 for i in range(w.n)],
+                                             page_end=[T // 16 if i == b else 0 for i in range(w.n)])
+                gV = oracle.unpack_codes(8, summ_np[blk, 0])[0]
+                oV = oracle.unpack_codes(8, ref[blk, 0])[0]
+                assert np.abs(gV - oV).max() <= 1
+
+
+def test_decode_step_graph_replay_equals_eager():
+    """The step is captured once in a CUDA graph and replayed as the sequences grow."""
+    w = small_bf16([16 * 100 + 9, 16 * 70], Hq=8, Hkv=2, budget=256, seed=44)
+    w = w.with_(seq_lens=[t + 64 for t in w.seq_lens])
+    res = []
+    for mode in ("eager", "graph"):
+        gc = _gc(w)
+        gc.case.seq_lens.copy_(torch.tensor([t - 64 for t in w.seq_lens], dtype=torch.int32, device="cuda:0"))
+        summ = gc.ctx.new_summaries(gc.case.num_blocks)
+        gc.ctx.locks_build_summaries(gc.kv, w.n, summ)
+        out = torch.empty(w.n, w.Hq, w.d, dtype=torch.bfloat16, device="cuda:0")
+        kn, vn, qn = [t.clone() for t in locks_synth.new_token(w, 0, device="cuda:0")]
+        outs = []
+        if mode == "graph":
+            s = torch.cuda.Stream()
+            g = torch.cuda.CUDAGraph()
+            s.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(s):
+                # warm up outside capture on a scratch copy of the lengths
+                saved = gc.case.seq_lens.clone()
+                gc.ctx.locks_decode_step(qn, kn, vn, gc.kv, summ, w.n, out, stream=s)
+                s.synchronize()
+                gc.case.seq_lens.copy_(saved)
+                with torch.cuda.graph(g, stream=s):
+                    gc.ctx.locks_decode_step(qn, kn, vn, gc.kv, summ, w.n, out, stream=s)
+            torch.cuda.synchronize()
+        for step in range(20):
+            a, b_, c = locks_synth.new_token(w, step, device="cuda:0")
+            kn.copy_(a); vn.copy_(b_); qn.copy_(c)
+            if mode == "graph":
+                g.replay()
+            else:
+                gc.ctx.locks_decode_step(qn, kn, vn, gc.kv, summ, w.n, out)
+            torch.cuda.synchronize()
+            outs.append(out.float().cpu().numpy().copy())
+        assert gc.status() == 0
+        res.append((outs, gc.case.seq_lens.cpu().tolist()))
+    assert res[0][1] == res[1][1]
+    for a, b_ in zip(res[0][0], res[1][0]):
+        assert np.array_equal(a, b_)
+
+
+def test_decode_step_host_entry_point():
+    w = small_bf16([16 * 50 + 5, 900], Hq=8, Hkv=2, budget=128, seed=55)
+    gc = _gc(w)
+    summ = gc.gpu_build()
+    q_host = gc.case.q.cpu().pin_memory()
+    out_host = torch.empty(w.n, w.Hq, w.d, dtype=torch.bfloat16).pin_memory()
+    ids_host = torch.empty(w.n, w.Hkv, gc.k, dtype=torch.int32).pin_memory()
+    cnt_host = torch.empty(w.n, w.Hkv, dtype=torch.int32).pin_memory()
+    gc.ctx.locks_decode_step_host(q_host, None, None, gc.kv, summ, w.n, out_host, ids_host, cnt_host)
+    out = torch.empty(w.n, w.Hq, w.d, dtype=torch.bfloat16, device="cuda:0")
+    ids = torch.empty(w.n, w.Hkv, gc.k, dtype=torch.int32, device="cuda:0")
+    cnt = torch.empty(w.n, w.Hkv, dtype=torch.int32, device="cuda:0")
+    gc.ctx.locks_decode_step(gc.case.q, None, None, gc.kv, summ, w.n, out, ids, cnt)
+    torch.cuda.synchronize()
+    assert torch.equal(out.cpu(), out_host) and torch.equal(ids.cpu(), ids_host) and torch.equal(cnt.cpu(), cnt_host)
+
+
+def test_bad_block_id_sets_status_without_faulting():
+    """Host-injected fault: a block id outside the cache is skipped and reported, nothing traps."""
+    gc = _gc(small_bf16([16 * 60], Hq=8, Hkv=2, budget=128, seed=66))
+    summ = gc.gpu_build()
+    gc.case.block_table[0, 7] = gc.case.num_blocks + 5
+    gc.gpu_select(summ)
+    assert gc.status() == -6
+    assert gc.status() == 0                                          # polling clears it
+
+
+def test_argument_errors_are_reported_on_the_host():
+    import ctypes as C
+    import paper_2607_24555_b200 as locks
+    from paper_2607_24555_b200.binding import make_config, lib
+    gc = _gc(small_bf16([16 * 20], Hq=8, Hkv=2, budget=128))
+    with pytest.raises(locks.LocksError):
+        gc.ctx.locks_select(gc.case.q, None, gc.kv, 1, None, None)
+    with pytest.raises(locks.LocksError):
+        gc.ctx.locks_sparse_attend(gc.case.q, gc.kv, 99, None, None, gc.case.q)
+    assert locks.locks_workspace_bytes(make_config(8, 3, 8, "i4", "bf16", 1, 16, 64)) == 0      # Hq % Hkv
+    assert locks.locks_workspace_bytes(make_config(8, 2, 3, "i4", "bf16", 1, 16, 64)) == 0      # rank
+    assert locks.locks_workspace_bytes(make_config(8, 2, 8, "i4", "bf16", 1, 16, 16)) == 0      # k < 2
+
+
+# ----------------------------------------------------------------------------- full-size configs
+
+def test_config1_full_size_sampled():
+    """Llama shapes at full size (8 x 32K, r8i4, b = 2048) in the launch configuration bench.py
+    times; the oracle checks every page mass of sampled (request, head) problems and the outputs."""
+    from gpu_util import check_select_and_attend
+    gc = _gc(locks_synth.config1())
+    w = gc.w
+    summ_gpu = gc.gpu_build()
+    summ_np = summ_gpu.cpu().numpy()                                  # GPU-built bytes handed to the oracle
+    differed = check_select_and_attend(gc, summ_np, out_tol=2e-2)
+    assert differed <= 2, differed                                    # of 64 problems
+    out, lse = gc.gpu_attend()                                        # dense flash-decode baseline
+    sub = slice(0, 2)
+    oout, olse = oracle.attend(gc.cache, t2np(gc.case.q), gc.sm)
+    assert np.abs(out - oout).max() <= 2e-2 and np.abs(lse - olse).max() <= 1e-3
+
+
+def test_config3_long_context_128k():
+    from gpu_util import check_select_and_attend
+    gc = _gc(locks_synth.config3(T=131072))
+    summ_np = gc.gpu_build().cpu().numpy()
+    differed = check_select_and_attend(gc, summ_np, out_tol=2e-2)
+    assert differed <= 1
