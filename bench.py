@@ -1,0 +1,354 @@
+#!/usr/bin/env python
+"""Benchmark of the LOCKS decode hot path on B200.
+
+A "step" is one pass of the whole path over one batch of synthetic input: append the new token's
+K/V, scan + score every resident page summary, share-average + top-k, sparse paged attention over
+the selected pages, and the summary build of pages that just filled -- one `locks_decode_step`,
+captured in a CUDA graph and replayed.  The workload is the Llama-3.1-8B-shaped configuration
+(32 q heads / 8 KV heads, d 128, page 16, bf16 KV, batch 8 x 32K context, r8i4, b = 2048).
+
+Cold caches: the step touches about 175 MB and B200's L2 holds 126 MB, so the replays cycle over
+several independent "layers" (own KV cache, summaries and query), as a real model would; by the
+time a layer comes round again its lines are gone.
+
+Prints ONE JSON line (see README for the keys).  `--impl reference` times the CPU
+oracle instead (test infrastructure; the only other place this file runs it is `cpu_baseline`).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "decode_step_us"
+UNIT = "us"
+FALLBACK_HBM_GBS = 6650.0
+
+
+def workload(name: str):
+    import locks_synth
+    if name == "cfg1":
+        return locks_synth.config1()
+    if name == "cfg3_1m":
+        return locks_synth.config3(T=1 << 20)
+    if name == "cfg3_128k":
+        return locks_synth.config3(T=1 << 17)
+    if name == "cfg2_r8_b1024":
+        return locks_synth.config2(rank=8, budget=1024)
+    if name == "small":
+        return locks_synth.Workload("small", [4096] * 2, Hq=8, Hkv=2, budget=256)
+    raise SystemExit(f"unknown workload {name}")
+
+
+def algorithmic_bytes(w, reserve_tokens=0):
+    """Bytes the method itself must move per step."""
+    payload = {8: 818, 4: 490, 2: 326}[w.rank] if w.fmt == "i4" else 4 * (128 + w.rank * 128 + 16 * w.rank)
+    scan = attend = dense = 0
+    for T in w.seq_lens:
+        P = -(-T // w.B)
+        k = min(w.k, P)
+        scan += w.Hkv * max(P - 2, 0) * payload if P > w.k else 0
+        attend += w.Hkv * k * w.B * w.d * 2 * 2
+        dense += w.Hkv * P * w.B * w.d * 2 * 2
+    return scan, attend, dense
+
+
+def measured_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            return float(json.load(open(p))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+def recorded_traffic(wname):
+    """DRAM bytes per scan launch from the committed ncu capture, if one covers this workload."""
+    p = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(p):
+        try:
+            return json.load(open(p)).get(wname)
+        except Exception:
+            return None
+    return None
+
+
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={index}", f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def oracle_sample(w, steps: int, threads: int):
+    """Time the oracle's decode step (score -> select -> attend on resident summaries) on a bounded
+    sample of the workload: the first `nreq` requests, full context.  Returns (us per full-batch
+    step scaled from the sample, sample description, seconds spent)."""
+    import numpy as np
+    import torch
+    import locks_synth
+    import oracle
+    oracle.set_threads(threads)
+    nreq = 1
+    ws = w.with_(seq_lens=w.seq_lens[:nreq])
+    case = locks_synth.make_case(ws, device="cpu")
+
+    def bits(t):
+        t = t.contiguous()
+        return t.view(torch.int16).numpy().view(np.uint16) if t.dtype == torch.bfloat16 else t.numpy()
+
+    sb, sh, st = case.strides
+    cache = oracle.Cache(bits(case.k), bits(case.v), case.block_table.numpy(), case.seq_lens.numpy(), w.Hq,
+                         strides={"shape": (case.num_blocks, w.Hkv, w.B, w.d), "block": sb, "head": sh, "token": st})
+    fmt = oracle.FMT_I4 if w.fmt == "i4" else oracle.FMT_F32
+    summ = oracle.build_summaries(cache, w.rank, fmt)
+    q = bits(case.q)
+    sm = 1.0 / math.sqrt(w.d)
+    oracle.decode_step(cache, q, w.rank, fmt, summ, sm, w.k)          # warm the caches once
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        oracle.decode_step(cache, q, w.rank, fmt, summ, sm, w.k)
+    dt = (time.perf_counter() - t0) / steps
+    scale = w.n / nreq
+    return dt * 1e6 * scale, f"{nreq} of {w.n} requests ({ws.Hkv} KV heads, full {ws.seq_lens[0]}-token context), " \
+                             f"time scaled by {scale:g}", dt * steps
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", 0))
+    if rank != 0:
+        return
+    import oracle
+    w = workload(args.workload)
+    cores = oracle.max_threads()
+    steps = max(1, min(args.steps, 5))
+    for _ in range(min(args.warmup, 1)):
+        pass
+    us, sample, _ = oracle_sample(w, steps, cores)
+    scan, attend, dense = algorithmic_bytes(w)
+    line = {"impl": "reference", "metric": METRIC, "value": us, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
+            "warmup": 1, "ms_per_step": us / 1e3, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f64", "data": "synthetic",
+            "config": {"workload": w.name, "batch": w.n, "context": w.seq_lens[0], "q_heads": w.Hq, "kv_heads": w.Hkv,
+                       "rank": w.rank, "budget_tokens": w.budget, "summary": "r8i4" if w.fmt == "i4" else "f32"},
+            "cpu_baseline": {"value": us, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": us, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def run_ours(args):
+    import numpy as np
+    import torch
+    import locks_synth
+    import paper_2607_24555_b200 as locks
+    from paper_2607_24555_b200 import dist as ldist
+    from paper_2607_24555_b200.binding import KVView, make_config
+
+    rank, local_rank, world = ldist.env_rank_world()
+    if world > 1:
+        import torch.distributed as tdist
+        tdist.init_process_group("nccl", device_id=torch.device(f"cuda:{local_rank}"))
+    torch.cuda.set_device(local_rank)
+    dev = f"cuda:{local_rank}"
+    K, W = args.steps, max(args.warmup, 3)
+    w0 = workload(args.workload)
+    L = args.layers
+    grow = K + W + 2 * K + 64                       # tokens appended over the whole run, per layer at most
+    reserve = -(-grow // w0.B) + 1
+    # every rank owns a full batch (weak scaling): requests are independent, no data-path collective
+    layers = []
+    for li in range(L):
+        w = w0.with_(seed=w0.seed * 1000 + 17 * li + 101 * rank, seq_lens=[t + reserve * w0.B for t in w0.seq_lens])
+        case = locks_synth.make_case(w, device=dev)
+        case.seq_lens.copy_(torch.tensor(w0.seq_lens, dtype=torch.int32, device=dev))
+        layers.append(case)
+    max_pages = layers[0].block_table.shape[1]
+    cfg = make_config(w0.Hq, w0.Hkv, w0.rank, w0.fmt, w0.dtype, w0.n, max_pages, w0.budget)
+    ctx = locks.Context(cfg, device=dev)
+    kvs = [KVView(c.k, c.v, c.strides, c.num_blocks, c.block_table, c.seq_lens) for c in layers]
+    summs = [ctx.new_summaries(c.num_blocks) for c in layers]
+    t0 = time.perf_counter()
+    for kv, s in zip(kvs, summs):
+        ctx.locks_build_summaries(kv, w0.n, s)
+    torch.cuda.synchronize()
+    bulk_build_ms = (time.perf_counter() - t0) * 1e3 / L
+    outs = [torch.empty(w0.n, w0.Hq, w0.d, dtype=torch.bfloat16 if w0.dtype == "bf16" else torch.float32, device=dev)
+            for _ in layers]
+    news = [locks_synth.new_token(w0.with_(seed=w0.seed + li), li, device=dev) for li in range(L)]
+    stream = torch.cuda.Stream(device=dev)
+
+    def step(li, s=None):
+        kn, vn, qn = news[li]
+        ctx.locks_decode_step(qn, kn, vn, kvs[li], summs[li], w0.n, outs[li], stream=s or stream)
+
+    # ---- capture one graph per layer (after one eager step each, which also warms the kernels)
+    graphs = []
+    with torch.cuda.stream(stream):
+        for li in range(L):
+            step(li)
+        stream.synchronize()
+        for li in range(L):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                step(li)
+            graphs.append(g)
+    launches_per_step = ctx.locks_last_launch_count()
+    torch.cuda.synchronize()
+
+    def run_graph_steps(n, first):
+        for i in range(n):
+            graphs[(first + i) % L].replay()
+
+    # ---- timed region: exactly K graph replays between barrier + synchronize
+    with torch.cuda.stream(stream):
+        run_graph_steps(W, 0)
+        stream.synchronize()
+        ldist.barrier()
+        torch.cuda.synchronize()
+        sampler = ClockSampler(local_rank) if rank == 0 else None
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        run_graph_steps(K, W)
+        e1.record(stream)
+        stream.synchronize()
+        torch.cuda.synchronize()
+        ldist.barrier()
+        step_ms = e0.elapsed_time(e1) / K
+        # ---- per-kernel split, eager launches with event pairs on the launch stream
+        ctx.locks_profile_begin(K)
+        for i in range(K):
+            step((W + K + i) % L)
+        stage_ms, nprof = ctx.locks_profile_end()
+        # ---- dense flash-decode over the full cache on the same GPU (same entry point, no page table)
+        for li in range(min(L, 3)):
+            ctx.locks_sparse_attend(news[li][2], kvs[li], w0.n, None, None, outs[li], stream=stream)
+        stream.synchronize()
+        d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        nd = max(3, min(K, 10))
+        d0.record(stream)
+        for i in range(nd):
+            ctx.locks_sparse_attend(news[i % L][2], kvs[i % L], w0.n, None, None, outs[i % L], stream=stream)
+        d1.record(stream)
+        stream.synchronize()
+        dense_ms = d0.elapsed_time(d1) / nd
+        clocks = sampler.stop() if sampler else None
+        # ---- end to end through the host-buffer entry point: H2D of q, k_new, v_new and D2H of out every step
+        hq = [n[2].cpu().pin_memory() for n in news]
+        hk = [n[0].cpu().pin_memory() for n in news]
+        hv = [n[1].cpu().pin_memory() for n in news]
+        hout = torch.empty_like(outs[0], device="cpu").pin_memory()
+        for i in range(3):
+            ctx.locks_decode_step_host(hq[i % L], hk[i % L], hv[i % L], kvs[i % L], summs[i % L], w0.n, hout, stream=stream)
+        ldist.barrier()
+        t0 = time.perf_counter()
+        for i in range(K):
+            li = (3 + i) % L
+            ctx.locks_decode_step_host(hq[li], hk[li], hv[li], kvs[li], summs[li], w0.n, hout, stream=stream)
+        e2e_ms = (time.perf_counter() - t0) * 1e3 / K
+    status = ctx.locks_poll_status()
+    step_ms_max = ldist.max_over_ranks(step_ms, device=dev)
+    e2e_ms_max = ldist.max_over_ranks(e2e_ms, device=dev)
+    if rank != 0:
+        return
+    scan_b, att_b, dense_b = algorithmic_bytes(w0)
+    peak, peak_kind = measured_peak()
+    scan_gbs = scan_b / (stage_ms["scan"] * 1e-3) / 1e9
+    esz = 2 if w0.dtype == "bf16" else 4
+    h2d = w0.n * (w0.Hq + 2 * w0.Hkv) * w0.d * esz
+    d2h = w0.n * w0.Hq * w0.d * esz
+    cores = os.cpu_count() or 1
+    cpu_us = cpu_sample = None
+    if not args.no_cpu_baseline:
+        import oracle
+        cores = oracle.max_threads()
+        cpu_us, cpu_sample, _ = oracle_sample(w0, 2, cores)
+    line = {
+        "metric": METRIC, "value": step_ms_max * 1e3, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+        "ms_per_step": step_ms_max, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16" if w0.dtype == "bf16" else "f32", "data": "synthetic",
+        "config": {"workload": w0.name, "batch_per_gpu": w0.n, "context": w0.seq_lens[0], "q_heads": w0.Hq,
+                   "kv_heads": w0.Hkv, "head_dim": w0.d, "page": w0.B, "rank": w0.rank, "budget_tokens": w0.budget,
+                   "summary": "r8i4" if w0.fmt == "i4" else "f32", "launch": "one CUDA graph per step",
+                   "l2": f"inputs larger than L2: replays cycle over {L} independent layers "
+                         f"({(scan_b + att_b) / 1e6:.0f} MB touched per step, L2 126 MB)"},
+        "e2e": {"value": e2e_ms_max * 1e3, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "gpu_launches": launches_per_step * K,
+        "clocks": clocks,
+        "roofline": {"bound": "hbm", "kernel": "scan_i4r8_kernel", "achieved": scan_gbs, "peak": peak, "unit": "GB/s",
+                     "frac": scan_gbs / peak, "peak_kind": f"of {peak_kind}", "traffic": recorded_traffic(w0.name),
+                     "algorithmic_bytes_per_launch": scan_b, "launch_us": stage_ms["scan"] * 1e3},
+        "step_roofline": {"algorithmic_bytes": scan_b + att_b, "achieved": (scan_b + att_b) / (step_ms_max * 1e-3) / 1e9,
+                          "frac": (scan_b + att_b) / (step_ms_max * 1e-3) / 1e9 / peak, "unit": "GB/s",
+                          "frac_of_8000": (scan_b + att_b) / (step_ms_max * 1e-3) / 1e9 / 8000.0},
+        "stages_us": {k_: v * 1e3 for k_, v in stage_ms.items()},
+        "dense_flash_decode": {"us": dense_ms * 1e3, "bytes": dense_b, "achieved_gbs": dense_b / (dense_ms * 1e-3) / 1e9,
+                               "speedup_of_step": dense_ms / step_ms_max},
+        "bulk_build_ms_per_layer": bulk_build_ms,
+        "device_status": status,
+        "cpu_baseline": ({"value": cpu_us, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": cpu_sample}
+                         if cpu_us is not None else None),
+    }
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=48)
+    ap.add_argument("--warmup", type=int, default=8)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg1")
+    ap.add_argument("--layers", type=int, default=4)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

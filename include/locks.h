@@ -158,6 +158,15 @@ int locks_poll_status(locks_ctx *ctx, int32_t *status_host, locks_stream stream)
 /* Number of kernels the last call on this context enqueued (for launch accounting). */
 int locks_last_launch_count(const locks_ctx *ctx);
 
+/* Per-stage timing of eager (not captured) locks_decode_step calls, the event-pair split of the
+ * step asked for when reporting where the time goes (the paper reports none per kernel).  After
+ * locks_profile_begin(ctx, max_steps) every locks_decode_step records CUDA events on its stream at
+ * the stage boundaries; locks_profile_end() synchronises the device, writes the mean duration in
+ * milliseconds of {prologue, summary scan, selection, sparse attention} to stage_ms[4], the number
+ * of steps seen to *steps, and releases the events.  Not legal while the stream is being captured. */
+int locks_profile_begin(locks_ctx *ctx, int max_steps);
+int locks_profile_end(locks_ctx *ctx, float *stage_ms, int *steps);
+
 const char *locks_strerror(int code);
 
 #ifdef __cplusplus

@@ -15,7 +15,8 @@ FMT_F32, FMT_I4 = 0, 1
 
 SYMBOLS = ["locks_summary_bytes", "locks_workspace_bytes", "locks_create", "locks_destroy",
            "locks_build_summaries", "locks_select", "locks_sparse_attend", "locks_decode_step",
-           "locks_decode_step_host", "locks_poll_status", "locks_last_launch_count", "locks_strerror"]
+           "locks_decode_step_host", "locks_poll_status", "locks_last_launch_count", "locks_strerror",
+           "locks_profile_begin", "locks_profile_end"]
 
 
 class LocksError(RuntimeError):
@@ -64,6 +65,10 @@ def lib():
         L.locks_decode_step_host.argtypes = [vp, vp, vp, vp, C.POINTER(KV), vp, C.c_int, vp, i32p, i32p, vp]
         L.locks_poll_status.argtypes = [vp, C.POINTER(C.c_int32), vp]
         L.locks_last_launch_count.argtypes = [vp]
+        L.locks_profile_begin.argtypes = [vp, C.c_int]
+        L.locks_profile_end.argtypes = [vp, C.POINTER(C.c_float), C.POINTER(C.c_int)]
+        L.locks_profile_begin.restype = C.c_int
+        L.locks_profile_end.restype = C.c_int
         L.locks_strerror.restype = C.c_char_p
         L.locks_strerror.argtypes = [C.c_int]
         for fn in ("locks_create", "locks_destroy", "locks_build_summaries", "locks_select", "locks_sparse_attend",
@@ -198,6 +203,15 @@ class Context:
         st = C.c_int32(0)
         _check(lib().locks_poll_status(self.handle, C.byref(st), _stream(stream)), "locks_poll_status")
         return int(st.value)
+
+    def locks_profile_begin(self, max_steps: int):
+        _check(lib().locks_profile_begin(self.handle, max_steps), "locks_profile_begin")
+
+    def locks_profile_end(self):
+        ms = (C.c_float * 4)()
+        n = C.c_int(0)
+        _check(lib().locks_profile_end(self.handle, ms, C.byref(n)), "locks_profile_end")
+        return {"prologue": ms[0], "scan": ms[1], "select": ms[2], "attend": ms[3]}, int(n.value)
 
     def locks_last_launch_count(self) -> int:
         return int(lib().locks_last_launch_count(self.handle))

@@ -23,15 +23,16 @@ int validate(const locks_config *c) {
   if (c->kv_dtype != c->q_dtype) return LOCKS_ERR_UNSUPPORTED;
   if (c->summary_fmt == LOCKS_FMT_I4 && c->rank != 2 && c->rank != 4 && c->rank != 8) return LOCKS_ERR_UNSUPPORTED;
   if (c->summary_fmt == LOCKS_FMT_F32 && c->rank > 16) return LOCKS_ERR_UNSUPPORTED;
-  const int chunks = (c->max_pages_per_seq + LOCKS_SEL_CHUNK - 1) / LOCKS_SEL_CHUNK;
-  if (chunks > 1 && (size_t)chunks * (k - 2) > 32 * LOCKS_SEL_THREADS) return LOCKS_ERR_UNSUPPORTED;
-  if (k > LOCKS_SEL_CHUNK) return LOCKS_ERR_UNSUPPORTED;
+  const int chunk_max = LOCKS_SEL_THREADS * LOCKS_SEL_MAX_EPT;
+  const int chunks = (c->max_pages_per_seq + chunk_max - 1) / chunk_max;
+  if (chunks > 1 && (size_t)chunks * (k - 2) > 16 * LOCKS_SEL_THREADS) return LOCKS_ERR_UNSUPPORTED;
+  if (k > LOCKS_SEL_THREADS * 4) return LOCKS_ERR_UNSUPPORTED;
   return LOCKS_OK;
 }
 
 struct Layout {
-  size_t status, shat, part, qnorm, cand_val, cand_idx, att_o, att_lse, ids, cnt, sq, skn, svn, sout, total;
-  int G, k, S, max_groups, sel_chunks, sel_kc, splits_sparse, splits_dense, splits_max;
+  size_t status, shat, part, cand_val, cand_idx, att_o, att_lse, att_done, ids, cnt, sq, skn, svn, sout, total;
+  int G, k, S, max_groups, sel_ept, sel_chunks, sel_kc;
 };
 
 Layout make_layout(const locks_config *c) {
@@ -40,12 +41,10 @@ Layout make_layout(const locks_config *c) {
   L.k = (c->budget_tokens + c->page_size - 1) / c->page_size;
   L.S = c->summary_fmt == LOCKS_FMT_I4 ? i4_stride(c->rank) : f32_stride(c->rank);
   L.max_groups = (c->max_pages_per_seq + LOCKS_GROUP - 1) / LOCKS_GROUP;
-  L.sel_chunks = (c->max_pages_per_seq + LOCKS_SEL_CHUNK - 1) / LOCKS_SEL_CHUNK;
+  const int per_thread = (c->max_pages_per_seq + LOCKS_SEL_THREADS - 1) / LOCKS_SEL_THREADS;
+  L.sel_ept = per_thread <= 4 ? 4 : (per_thread <= 8 ? 8 : 16);
+  L.sel_chunks = (c->max_pages_per_seq + L.sel_ept * LOCKS_SEL_THREADS - 1) / (L.sel_ept * LOCKS_SEL_THREADS);
   L.sel_kc = L.k - 2 > 0 ? L.k - 2 : 1;
-  const int ppc_s = LOCKS_ATT_WARPS * LOCKS_ATT_PAGES_PER_WARP, ppc_d = LOCKS_ATT_WARPS * LOCKS_ATT_DENSE_PAGES_PER_WARP;
-  L.splits_sparse = (L.k + ppc_s - 1) / ppc_s;
-  L.splits_dense = (c->max_pages_per_seq + ppc_d - 1) / ppc_d;
-  L.splits_max = L.splits_sparse > L.splits_dense ? L.splits_sparse : L.splits_dense;
   const size_t nb = c->max_batch, Hq = c->num_q_heads, Hkv = c->num_kv_heads, P = c->max_pages_per_seq;
   const size_t esz = c->q_dtype == LOCKS_BF16 ? 2 : 4;
   size_t o = 0;
@@ -53,11 +52,11 @@ Layout make_layout(const locks_config *c) {
   L.status = take(64);
   L.shat = take(nb * Hq * P * 4);
   L.part = take(nb * Hq * L.max_groups * 8);
-  L.qnorm = take(nb * Hq * 4);
   L.cand_val = take(nb * Hkv * L.sel_chunks * L.sel_kc * 4);
   L.cand_idx = take(nb * Hkv * L.sel_chunks * L.sel_kc * 4);
-  L.att_o = take(nb * Hq * L.splits_max * LOCKS_D * 4);
-  L.att_lse = take(nb * Hq * L.splits_max * 4);
+  L.att_o = take(nb * Hq * LOCKS_ATT_MAX_SPLITS * LOCKS_D * 4);
+  L.att_lse = take(nb * Hq * LOCKS_ATT_MAX_SPLITS * 4);
+  L.att_done = take(nb * Hkv * 4);
   L.ids = take(nb * Hkv * L.k * 4);
   L.cnt = take(nb * Hkv * 4);
   L.sq = take(nb * Hq * LOCKS_D * esz);
@@ -103,9 +102,9 @@ int locks_create(const locks_config *cfg, void *workspace, size_t ws_bytes, lock
   locks_ctx *c = new (std::nothrow) locks_ctx();
   if (!c) return LOCKS_ERR_INVALID_ARG;
   c->cfg = *cfg;
+  c->prof_ev = nullptr; c->prof_cap = c->prof_n = 0;
   c->G = L.G; c->k = L.k; c->S = L.S; c->Pmax = cfg->max_pages_per_seq; c->max_groups = L.max_groups;
-  c->sel_chunks = L.sel_chunks; c->sel_kc = L.sel_kc;
-  c->att_splits_sparse = L.splits_sparse; c->att_splits_dense = L.splits_dense; c->att_splits_max = L.splits_max;
+  c->sel_ept = L.sel_ept; c->sel_chunks = L.sel_chunks; c->sel_kc = L.sel_kc;
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess ||
       cudaDeviceGetAttribute(&c->num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
@@ -117,18 +116,20 @@ int locks_create(const locks_config *cfg, void *workspace, size_t ws_bytes, lock
   c->status = reinterpret_cast<int32_t *>(ws + L.status);
   c->shat = reinterpret_cast<float *>(ws + L.shat);
   c->part = reinterpret_cast<float2 *>(ws + L.part);
-  c->qnorm = reinterpret_cast<float *>(ws + L.qnorm);
   c->cand_val = reinterpret_cast<float *>(ws + L.cand_val);
   c->cand_idx = reinterpret_cast<int32_t *>(ws + L.cand_idx);
   c->att_o = reinterpret_cast<float *>(ws + L.att_o);
   c->att_lse = reinterpret_cast<float *>(ws + L.att_lse);
+  c->att_done = reinterpret_cast<int32_t *>(ws + L.att_done);
   c->ids_int = reinterpret_cast<int32_t *>(ws + L.ids);
   c->cnt_int = reinterpret_cast<int32_t *>(ws + L.cnt);
   c->stage_q = ws + L.sq; c->stage_kn = ws + L.skn; c->stage_vn = ws + L.svn; c->stage_out = ws + L.sout;
   if (cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking) != cudaSuccess ||
       cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
       cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) != cudaSuccess ||
-      cudaMemsetAsync(c->status, 0, 64, 0) != cudaSuccess || cudaStreamSynchronize(0) != cudaSuccess) {
+      cudaMemsetAsync(c->status, 0, 64, 0) != cudaSuccess ||
+      cudaMemsetAsync(c->att_done, 0, (size_t)cfg->max_batch * cfg->num_kv_heads * 4, 0) != cudaSuccess ||
+      cudaStreamSynchronize(0) != cudaSuccess) {
     delete c;
     return LOCKS_ERR_CUDA;
   }
@@ -138,6 +139,10 @@ int locks_create(const locks_config *cfg, void *workspace, size_t ws_bytes, lock
 
 int locks_destroy(locks_ctx *ctx) {
   if (!ctx) return LOCKS_ERR_INVALID_ARG;
+  if (ctx->prof_ev) {
+    for (int i = 0; i < ctx->prof_cap * LOCKS_PROF_MARKS; ++i) cudaEventDestroy(ctx->prof_ev[i]);
+    delete[] ctx->prof_ev;
+  }
   cudaEventDestroy(ctx->ev_fork);
   cudaEventDestroy(ctx->ev_join);
   cudaStreamDestroy(ctx->side);
@@ -192,15 +197,23 @@ int locks_decode_step(locks_ctx *ctx, const void *q, const void *k_new, const vo
   int32_t *ids = page_ids ? page_ids : ctx->ids_int;
   int32_t *cnt = page_count ? page_count : ctx->cnt_int;
   ctx->last_launches = 0;
+  cudaEvent_t *pe = (ctx->prof_ev && ctx->prof_n < ctx->prof_cap) ? ctx->prof_ev + ctx->prof_n * LOCKS_PROF_MARKS : nullptr;
+  auto mark = [&](int i) { if (pe) cudaEventRecord(pe[i], st); };
+  mark(0);
   if ((rc = locks_launch_prep(ctx, q, k_new, v_new, kv, batch, st)) != LOCKS_OK) return rc;
+  mark(1);
   // the freshly completed page (if any) is summarised beside select + attend: it is read by neither
   if (cudaEventRecord(ctx->ev_fork, st) != cudaSuccess || cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0) != cudaSuccess)
     return LOCKS_ERR_CUDA;
   if ((rc = locks_launch_build(ctx, kv, batch, nullptr, nullptr, 1, summaries, ctx->side)) != LOCKS_OK) return rc;
   if (cudaEventRecord(ctx->ev_join, ctx->side) != cudaSuccess) return LOCKS_ERR_CUDA;
   if ((rc = locks_launch_scan(ctx, q, summaries, kv, batch, ctx->shat, st)) != LOCKS_OK) return rc;
+  mark(2);
   if ((rc = locks_launch_select(ctx, ctx->shat, kv, batch, ids, cnt, nullptr, st)) != LOCKS_OK) return rc;
+  mark(3);
   if ((rc = locks_launch_attend(ctx, q, kv, batch, ids, cnt, out, nullptr, st)) != LOCKS_OK) return rc;
+  mark(4);
+  if (pe) ctx->prof_n++;
   if (cudaStreamWaitEvent(st, ctx->ev_join, 0) != cudaSuccess) return LOCKS_ERR_CUDA;
   return LOCKS_OK;
 }
@@ -249,6 +262,37 @@ int locks_poll_status(locks_ctx *ctx, int32_t *status_host, locks_stream stream)
 }
 
 int locks_last_launch_count(const locks_ctx *ctx) { return ctx ? ctx->last_launches : 0; }
+
+int locks_profile_begin(locks_ctx *ctx, int max_steps) {
+  if (!ctx || max_steps <= 0 || ctx->prof_ev) return LOCKS_ERR_INVALID_ARG;
+  ctx->prof_ev = new (std::nothrow) cudaEvent_t[(size_t)max_steps * LOCKS_PROF_MARKS];
+  if (!ctx->prof_ev) return LOCKS_ERR_INVALID_ARG;
+  for (int i = 0; i < max_steps * LOCKS_PROF_MARKS; ++i)
+    if (cudaEventCreate(&ctx->prof_ev[i]) != cudaSuccess) return LOCKS_ERR_CUDA;
+  ctx->prof_cap = max_steps;
+  ctx->prof_n = 0;
+  return LOCKS_OK;
+}
+
+int locks_profile_end(locks_ctx *ctx, float *stage_ms, int *steps) {
+  if (!ctx || !ctx->prof_ev || !stage_ms || !steps) return LOCKS_ERR_INVALID_ARG;
+  int rc = LOCKS_OK;
+  if (cudaDeviceSynchronize() != cudaSuccess) rc = LOCKS_ERR_CUDA;
+  for (int s = 0; s < LOCKS_PROF_MARKS - 1; ++s) stage_ms[s] = 0.f;
+  for (int i = 0; i < ctx->prof_n && rc == LOCKS_OK; ++i)
+    for (int s = 0; s < LOCKS_PROF_MARKS - 1; ++s) {
+      float ms = 0.f;
+      if (cudaEventElapsedTime(&ms, ctx->prof_ev[i * LOCKS_PROF_MARKS + s], ctx->prof_ev[i * LOCKS_PROF_MARKS + s + 1]) !=
+          cudaSuccess) { rc = LOCKS_ERR_CUDA; break; }
+      stage_ms[s] += ms;
+    }
+  *steps = ctx->prof_n;
+  if (ctx->prof_n > 0) for (int s = 0; s < LOCKS_PROF_MARKS - 1; ++s) stage_ms[s] /= ctx->prof_n;
+  for (int i = 0; i < ctx->prof_cap * LOCKS_PROF_MARKS; ++i) cudaEventDestroy(ctx->prof_ev[i]);
+  delete[] ctx->prof_ev;
+  ctx->prof_ev = nullptr; ctx->prof_cap = ctx->prof_n = 0;
+  return rc;
+}
 
 const char *locks_strerror(int code) {
   switch (code) {

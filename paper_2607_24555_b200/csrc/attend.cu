@@ -24,6 +24,7 @@ struct AttParams {
   void *out;
   float *lse;
   int32_t *status;
+  int32_t *done;   // [batch*Hkv] split-arrival counters (zero between launches)
   int batch, Hq, Hkv, G, Pmax, kbud, num_blocks, splits, pages_per_cta;
   float sm_scale;
 };
@@ -190,8 +191,8 @@ __global__ void __launch_bounds__(LOCKS_ATT_WARPS * 32) attend_bf16_kernel(AttPa
     if (t == 0) { wm[row] = mrun[hh]; wl[row] = lrun[hh]; }
   }
   __syncthreads();
-  const int dim = threadIdx.x;  // 128 threads = 128 dims
-  for (int g = 0; g < p.G; ++g) {
+  for (int e = threadIdx.x; e < p.G * LOCKS_D; e += LOCKS_ATT_WARPS * 32) {
+    const int g = e / LOCKS_D, dim = e - g * LOCKS_D;
     float M = -INFINITY;
 #pragma unroll
     for (int w = 0; w < LOCKS_ATT_WARPS; ++w)
@@ -218,6 +219,34 @@ __global__ void __launch_bounds__(LOCKS_ATT_WARPS * 32) attend_bf16_kernel(AttPa
       if (dim == 0) p.part_lse[slot] = lse2;
     }
   }
+  if (p.splits == 1) return;
+  // the last CTA of this (request, KV head) to arrive merges the splits' partials by log-sum-exp
+  __shared__ int sh_last;
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) sh_last = (atomicAdd(&p.done[prob], 1) == p.splits - 1);
+  __syncthreads();
+  if (!sh_last) return;
+  __threadfence();
+  for (int e = threadIdx.x; e < p.G * LOCKS_D; e += LOCKS_ATT_WARPS * 32) {
+    const int g = e / LOCKS_D, dim = e - g * LOCKS_D;
+    const int64_t row = (int64_t)b * p.Hq + h * p.G + g;
+    const float *pl = p.part_lse + row * p.splits;
+    float M = -INFINITY;
+    for (int s2 = 0; s2 < p.splits; ++s2) M = fmaxf(M, __ldcg(pl + s2));
+    float L = 0.f, acc = 0.f;
+    if (M > -INFINITY) {
+      for (int s2 = 0; s2 < p.splits; ++s2) {
+        const float w = ex2f(__ldcg(pl + s2) - M);
+        L += w;
+        acc += w * __ldcg(p.part_o + (row * p.splits + s2) * LOCKS_D + dim);
+      }
+      acc /= L;
+    }
+    reinterpret_cast<__nv_bfloat16 *>(p.out)[row * LOCKS_D + dim] = __float2bfloat16_rn(acc);
+    if (p.lse && dim == 0) p.lse[row] = (M > -INFINITY) ? (M + log2f(L)) * kLn2 : -INFINITY;
+  }
+  if (threadIdx.x == 0) p.done[prob] = 0;   // ready for the next launch
 }
 
 // Plain fp32-arithmetic path for any element type (the fp32 parity configuration).
@@ -314,8 +343,17 @@ int locks_launch_attend(locks_ctx *c, const void *q, const locks_kv *kv, int bat
   p.batch = batch; p.Hq = c->cfg.num_q_heads; p.Hkv = c->cfg.num_kv_heads; p.G = c->G; p.Pmax = c->Pmax;
   p.kbud = c->k; p.num_blocks = kv->num_blocks; p.sm_scale = c->cfg.sm_scale;
   const bool dense = ids == nullptr;
-  p.splits = dense ? c->att_splits_dense : c->att_splits_sparse;
-  p.pages_per_cta = LOCKS_ATT_WARPS * (dense ? LOCKS_ATT_DENSE_PAGES_PER_WARP : LOCKS_ATT_PAGES_PER_WARP);
+  // one wave: as many splits per problem as resident CTA slots allow, at least one page per warp
+  const int npages = dense ? c->Pmax : c->k;
+  const int slots = c->num_sms * LOCKS_ATT_CTAS_PER_SM;
+  int splits = slots / (batch * p.Hkv);
+  const int most = (npages + LOCKS_ATT_WARPS - 1) / LOCKS_ATT_WARPS;
+  if (splits > most) splits = most;
+  if (splits > LOCKS_ATT_MAX_SPLITS) splits = LOCKS_ATT_MAX_SPLITS;
+  if (splits < 1) splits = 1;
+  p.pages_per_cta = (npages + splits - 1) / splits;
+  p.splits = (npages + p.pages_per_cta - 1) / p.pages_per_cta;
+  p.done = c->att_done;
   const bool bf = c->cfg.kv_dtype == LOCKS_BF16;
   if (bf) {
     static bool attr_done = false;
@@ -332,11 +370,9 @@ int locks_launch_attend(locks_ctx *c, const void *q, const locks_kv *kv, int bat
     attend_generic_kernel<float><<<grid, 128, 0, st>>>(p);
   }
   int rc = locks_check_launch(c);
-  if (rc != LOCKS_OK || p.splits == 1) return rc;
+  if (rc != LOCKS_OK || p.splits == 1 || bf) return rc;   // the bf16 kernel merges its own splits
   dim3 mg(p.Hq, batch);
-  if (bf) attend_merge_kernel<__nv_bfloat16><<<mg, 128, 0, st>>>(c->att_o, c->att_lse, p.splits,
-                                                                  reinterpret_cast<__nv_bfloat16 *>(out), lse, p.Hq);
-  else attend_merge_kernel<float><<<mg, 128, 0, st>>>(c->att_o, c->att_lse, p.splits, reinterpret_cast<float *>(out),
-                                                      lse, p.Hq);
+  attend_merge_kernel<float><<<mg, 128, 0, st>>>(c->att_o, c->att_lse, p.splits, reinterpret_cast<float *>(out), lse,
+                                                 p.Hq);
   return locks_check_launch(c);
 }

@@ -9,8 +9,7 @@
 //   5. V = D^T U_r Sigma_r^-1 (lane's 4 dims), C = U_r Sigma_r, sign: largest |V| entry positive
 //   6. store fp32 (F32 format) or quantise: symmetric abs-max, fp16 scale, round-half-even codes
 //      (int4 basis per column, int8 coefficients per row, int8 centroid) packed in the blob layout
-// prep_kernel: appends the new token's K/V row to the cache (optional), and derives the per-query
-//   power-of-two scale that keeps the scan's fp16 projection operands in range.
+// prep_kernel: appends the new token's K/V row to the cache and bumps the sequence length.
 #include "locks_internal.cuh"
 
 namespace {
@@ -291,34 +290,13 @@ struct PrepParams {
   int64_t sb, sh, st;
   const int32_t *block_table;
   int32_t *seq_lens;
-  float *qnorm;
   int32_t *status;
   int Hq, Hkv, Pmax, num_blocks;
 };
 
 template <typename T>
-__global__ void __launch_bounds__(128) prep_kernel(PrepParams p) {
-  const int b = blockIdx.x, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  // per-head power of two 2^-e with 2^e >= 2 |q|: keeps V^T q inside [-0.55, 0.55] for the fp16 MMA
-  const T *Q = reinterpret_cast<const T *>(p.q);
-  for (int hq = warp; hq < p.Hq; hq += 4) {
-    float s = 0.f;
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const float v = ldf<T>(Q, ((int64_t)b * p.Hq + hq) * LOCKS_D + lane * 4 + u);
-      s += v * v;
-    }
-    s = warp_sum(s);
-    if (lane == 0) {
-      float pn = 1.f;
-      if (s > 0.f && s < INFINITY) {
-        int e;
-        (void)frexpf(2.f * sqrtf(s), &e);  // 2|q| = f 2^e, f in [0.5, 1)
-        pn = ldexpf(1.f, -e);
-      }
-      p.qnorm[b * p.Hq + hq] = pn;
-    }
-  }
+__global__ void __launch_bounds__(256) prep_kernel(PrepParams p) {
+  const int b = blockIdx.x;
   if (p.k_new == nullptr) return;
   const int T0 = p.seq_lens[b];
   const int page = T0 / LOCKS_B, slot = T0 % LOCKS_B;
@@ -334,7 +312,7 @@ __global__ void __launch_bounds__(128) prep_kernel(PrepParams p) {
   }
   const T *kn = reinterpret_cast<const T *>(p.k_new), *vn = reinterpret_cast<const T *>(p.v_new);
   T *K = reinterpret_cast<T *>(p.k), *V = reinterpret_cast<T *>(p.v);
-  for (int e = threadIdx.x; e < p.Hkv * LOCKS_D; e += 128) {
+  for (int e = threadIdx.x; e < p.Hkv * LOCKS_D; e += 256) {
     const int h = e / LOCKS_D, c = e - h * LOCKS_D;
     const int64_t dst = (int64_t)block * p.sb + (int64_t)h * p.sh + (int64_t)slot * p.st + c;
     K[dst] = kn[((int64_t)b * p.Hkv + h) * LOCKS_D + c];
@@ -378,9 +356,10 @@ int locks_launch_prep(locks_ctx *c, const void *q, const void *k_new, const void
   PrepParams p;
   p.q = q; p.k_new = k_new; p.v_new = v_new; p.k = kv->k; p.v = kv->v;
   p.sb = kv->stride_block; p.sh = kv->stride_head; p.st = kv->stride_token;
-  p.block_table = kv->block_table; p.seq_lens = kv->seq_lens; p.qnorm = c->qnorm; p.status = c->status;
+  p.block_table = kv->block_table; p.seq_lens = kv->seq_lens; p.status = c->status;
   p.Hq = c->cfg.num_q_heads; p.Hkv = c->cfg.num_kv_heads; p.Pmax = c->Pmax; p.num_blocks = kv->num_blocks;
-  if (c->cfg.q_dtype == LOCKS_BF16) prep_kernel<__nv_bfloat16><<<batch, 128, 0, st>>>(p);
-  else prep_kernel<float><<<batch, 128, 0, st>>>(p);
+  if (k_new == nullptr) return LOCKS_OK;   // nothing to append: no launch
+  if (c->cfg.q_dtype == LOCKS_BF16) prep_kernel<__nv_bfloat16><<<batch, 256, 0, st>>>(p);
+  else prep_kernel<float><<<batch, 256, 0, st>>>(p);
   return locks_check_launch(c);
 }

@@ -10,39 +10,42 @@
 #define LOCKS_D 128          // head dimension the kernels are written for
 #define LOCKS_B 16           // tokens per page
 #define LOCKS_GROUP 8        // pages scored together by one warp in the scan
-#define LOCKS_SEL_THREADS 256
-#define LOCKS_SEL_EPT 8      // candidate pages held per thread in select stage 1
-#define LOCKS_SEL_CHUNK (LOCKS_SEL_THREADS * LOCKS_SEL_EPT)
-#define LOCKS_ATT_WARPS 4
-#define LOCKS_ATT_PAGES_PER_WARP 4
-#define LOCKS_ATT_DENSE_PAGES_PER_WARP 16
+#define LOCKS_SEL_THREADS 512
+#define LOCKS_SEL_MAX_EPT 16 // candidate pages held per thread in select stage 1 (4, 8 or 16)
+#define LOCKS_ATT_WARPS 3        // warps per attend CTA, each with a two-stage 16 KB page ring
+#define LOCKS_ATT_CTAS_PER_SM 4  // 4 x 48 KB of shared memory, 4 x 96 x 168 registers
+#define LOCKS_ATT_MAX_SPLITS 64
 #define LOCKS_SPIN_LIMIT (1 << 22)  // bounded mbarrier polling (each poll already waits a while)
 
 struct locks_ctx {
   locks_config cfg;
   int G, k, S, Pmax, max_groups;
   int num_sms;
+  int sel_ept;             // pages per thread in select stage 1
   int sel_chunks;          // select stage-1 CTAs per (request, KV head)
   int sel_kc;              // candidates kept per chunk (k-2)
-  int att_splits_sparse, att_splits_dense, att_splits_max;
   // workspace partition (device)
   char *ws;
   size_t ws_bytes;
   int32_t *status;         // [4] sticky status, work counters
   float *shat;             // [max_batch][Hq][Pmax]
   float2 *part;            // [max_batch][Hq][max_groups] per-group (max, sum exp) of candidates
-  float *qnorm;            // [max_batch][Hq] power-of-two scale keeping projections inside fp16
   float *cand_val;         // [max_batch][Hkv][sel_chunks][sel_kc]
   int32_t *cand_idx;
-  float *att_o;            // [max_batch][Hq][att_splits_max][d]
-  float *att_lse;          // [max_batch][Hq][att_splits_max]  (log2 units)
+  float *att_o;            // [max_batch][Hq][LOCKS_ATT_MAX_SPLITS][d]
+  float *att_lse;          // [max_batch][Hq][LOCKS_ATT_MAX_SPLITS]  (log2 units)
+  int32_t *att_done;       // [max_batch][Hkv] split-arrival counters
   int32_t *ids_int;        // [max_batch][Hkv][k]
   int32_t *cnt_int;        // [max_batch][Hkv]
   char *stage_q, *stage_kn, *stage_vn, *stage_out;
   cudaStream_t side;       // build of freshly filled pages runs beside select + attend
   cudaEvent_t ev_fork, ev_join;
   int last_launches;
+  // optional per-stage timing of eager decode steps (see locks_profile_begin)
+  cudaEvent_t *prof_ev;    // [prof_cap][LOCKS_PROF_MARKS]
+  int prof_cap, prof_n;
 };
+#define LOCKS_PROF_MARKS 5   // step start, after prep, after scan, after select, after attend
 
 // launchers (each returns LOCKS_OK or LOCKS_ERR_CUDA and adds to ctx->last_launches)
 int locks_launch_prep(locks_ctx *c, const void *q, const void *k_new, const void *v_new, const locks_kv *kv,

@@ -29,7 +29,6 @@ struct ScanParams {
   const int32_t *seq_lens;
   float *shat;
   float2 *part;
-  const float *qnorm;
   int32_t *status;
   int batch, Hq, Hkv, G, Pmax, max_groups, num_blocks, k, S, r;
   float sm_scale;
@@ -148,16 +147,18 @@ constexpr int kBlob = i4_stride(8);                       // 832
 constexpr int kStageBytes = LOCKS_GROUP * kBlob;          // 6656
 constexpr int kScanSmem = kScanWarps * (kScanStages * kStageBytes + 64);
 
-__device__ __forceinline__ uint32_t nib_pair(uint32_t w, int shift) {
-  // two 4-bit codes (bits shift.. and 16+shift..) -> bf16x2 holding 128 + code each
-  return ((w >> shift) & 0x000F000Fu) | 0x43004300u;
-}
-__device__ __forceinline__ uint32_t bf16x2_sub(uint32_t v, uint32_t c) {
-  __nv_bfloat162 r = __hsub2(*reinterpret_cast<__nv_bfloat162 *>(&v), *reinterpret_cast<__nv_bfloat162 *>(&c));
-  return *reinterpret_cast<uint32_t *>(&r);
+// (a & b) | c in one LOP3 with both constants held in registers
+__device__ __forceinline__ uint32_t and_or(uint32_t a, uint32_t b, uint32_t c) {
+  uint32_t d;
+  asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+  return d;
 }
 __device__ __forceinline__ uint32_t f16x2_sub(uint32_t v, uint32_t c) {
   __half2 r = __hsub2(*reinterpret_cast<__half2 *>(&v), *reinterpret_cast<__half2 *>(&c));
+  return *reinterpret_cast<uint32_t *>(&r);
+}
+__device__ __forceinline__ uint32_t f16x2_fma(uint32_t a, uint32_t b, uint32_t c) {
+  __half2 r = __hfma2(*reinterpret_cast<__half2 *>(&a), *reinterpret_cast<__half2 *>(&b), *reinterpret_cast<__half2 *>(&c));
   return *reinterpret_cast<uint32_t *>(&r);
 }
 __device__ __forceinline__ float2 h2f2(uint32_t v) { return __half22float2(*reinterpret_cast<__half2 *>(&v)); }
@@ -171,12 +172,27 @@ __device__ __forceinline__ float fast_lg2(float x) {
   asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+// D = A * B with a zero accumulator (no register is spent on the zeros)
+__device__ __forceinline__ void mma_f16_z(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                          uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+               "{%10,%10,%10,%10};\n"
+               : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
+               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "f"(0.f));
+}
 
-struct GroupId {
-  int b, h, grp, nsc;
+struct Cursor {
+  int prob, grp, nsc;
 };
 
-// NH = number of 8-row halves of the query tile in use (1: G <= 8, 2: G <= 16)
+// NH = number of 8-row halves of the query tile in use (1: G <= 8, 2: G <= 16).
+//
+// Numerics.  The stored integer codes are exact in fp16: a nibble n sitting at mantissa bits 0-3 of
+// 0x6400 reads 1024 + n, at bits 4-7 it reads 1024 + 16 n; subtracting 1032 / 1152 leaves code and
+// 16 * code, and the factor 16 is undone exactly by holding the matching query elements divided by
+// 16.  A byte at bits 0-7 reads 1024 + u.  The query row is scaled by a power of two so that
+// max|q| < 0.5 and converted to fp16 (bf16's 8 significant bits fit; only elements below 2^-14 of
+// the row maximum can round, by at most 2^-25 of it), so every product is exact and sums are fp32.
 template <int NH>
 __global__ void __launch_bounds__(kScanWarps * 32, 2) scan_i4r8_kernel(ScanParams p) {
   extern __shared__ __align__(128) uint8_t smem[];
@@ -190,62 +206,105 @@ __global__ void __launch_bounds__(kScanWarps * 32, 2) scan_i4r8_kernel(ScanParam
   }
   __syncwarp();
 
+  // warps stick to one (request, KV head) at a time: `wpp` warps share a problem and stride its groups
   const int W = gridDim.x * kScanWarps;
   const int wid = blockIdx.x * kScanWarps + warp;
-  const int total = p.batch * p.Hkv * p.max_groups;
+  const int nprob = p.batch * p.Hkv;
+  const int wpp = max(1, W / nprob), nslots = W / wpp;
+  const int slot = wid / wpp, sub = wid - slot * wpp;
+  if (slot >= nslots) return;
 
-  auto decode = [&](int gam, GroupId &g) -> bool {
-    const int prob = gam / p.max_groups;
-    g.grp = gam - prob * p.max_groups;
-    g.b = prob / p.Hkv;
-    g.h = prob - g.b * p.Hkv;
-    const int T = p.seq_lens[g.b];
+  auto load_nsc = [&](int prob) -> int {
+    const int T = p.seq_lens[prob / p.Hkv];
     const int P = (T + LOCKS_B - 1) / LOCKS_B;
-    g.nsc = (P <= p.k) ? 0 : P - 1;
-    return g.grp * LOCKS_GROUP < g.nsc;
+    return (P <= p.k) ? 0 : P - 1;
   };
-  auto next_valid = [&](int gam, GroupId &g) -> int {
-    while (gam < total && !decode(gam, g)) gam += W;
-    return gam;
+  auto settle = [&](Cursor &c) {  // move to the next non-empty position at or after (prob, grp)
+    while (c.prob < nprob && c.grp * LOCKS_GROUP >= c.nsc) {
+      c.prob += nslots;
+      c.grp = sub;
+      if (c.prob < nprob) c.nsc = load_nsc(c.prob);
+    }
   };
-  auto issue = [&](int stage, const GroupId &g) {
-    const int nvalid = min(LOCKS_GROUP, g.nsc - g.grp * LOCKS_GROUP);
+  auto issue = [&](int stage, const Cursor &c) {
+    const int b = c.prob / p.Hkv, h = c.prob - b * p.Hkv;
+    const int nvalid = min(LOCKS_GROUP, c.nsc - c.grp * LOCKS_GROUP);
     if (lane == 0) mbar_expect_tx(&full[stage], (uint32_t)nvalid * kBlob);
     __syncwarp();
     if (lane < nvalid) {
-      int block = p.block_table[(int64_t)g.b * p.Pmax + g.grp * LOCKS_GROUP + lane];
+      int block = p.block_table[(int64_t)b * p.Pmax + c.grp * LOCKS_GROUP + lane];
       if (block < 0 || block >= p.num_blocks) {
         set_status(p.status, LOCKS_ERR_BAD_BLOCK);
         block = 0;
       }
-      bulk_g2s(ring + stage * kStageBytes + lane * kBlob, p.summ + ((int64_t)block * p.Hkv + g.h) * kBlob, kBlob,
+      bulk_g2s(ring + stage * kStageBytes + lane * kBlob, p.summ + ((int64_t)block * p.Hkv + h) * kBlob, kBlob,
                &full[stage]);
     }
   };
 
-  GroupId gp, gc;
-  int gam_p = next_valid(wid, gp);
+  Cursor cp{slot, sub, 0}, cc;
+  if (cp.prob < nprob) cp.nsc = load_nsc(cp.prob);
+  settle(cp);
+  cc = cp;
   int inflight = 0;
 #pragma unroll
   for (int s = 0; s < kScanStages; ++s) {
-    if (gam_p < total) {
-      issue(s, gp);
+    if (cp.prob < nprob) {
+      issue(s, cp);
       ++inflight;
-      gam_p = next_valid(gam_p + W, gp);
+      cp.grp += wpp;
+      settle(cp);
     }
   }
-  int gam_c = next_valid(wid, gc);
 
-  // query fragments of the current (request, KV head)
-  uint32_t qa0[8], qa1[8], qa2[8], qa3[8];
-  float kx = 0.f, kx8 = 0.f, pn = 1.f, pn8 = 1.f;
+  // constants kept in registers so that every extraction is a single LOP3
+  uint32_t kM0 = 0x000F000Fu, kM1 = 0x00F000F0u, kMB = 0x00FF00FFu, kMagic = 0x64006400u;
+  asm volatile("" : "+r"(kM0), "+r"(kM1), "+r"(kMB), "+r"(kMagic));
+  const uint32_t kSub8 = 0x64086408u;      // 1032: 1024 + 8
+  const uint32_t kSub128 = 0x64806480u;    // 1152: 1024 + 128
+  const uint32_t kSixteen = 0x4C004C00u;   // 16.0
+  const uint32_t kSub16x = 0x74807480u;    // 18432 = 16 * 1152
+
+  uint32_t qa0[8], qa2[8], qa1[8], qa3[8];
+  float inv_s = 1.f, inv_s8 = 1.f;
   int cur_prob = -1;
   const __nv_bfloat16 *q = reinterpret_cast<const __nv_bfloat16 *>(p.q);
   const float c2 = p.sm_scale * kLog2e;
 
+  auto load_q_row = [&](int b, int hq, bool valid, uint32_t (&a0)[8], uint32_t (&a2)[8], float &inv) {
+    uint4 v[4] = {};
+    if (valid) {
+      const uint4 *qp = reinterpret_cast<const uint4 *>(q + ((int64_t)b * p.Hq + hq) * LOCKS_D + 32 * t);
+#pragma unroll
+      for (int m = 0; m < 4; ++m) v[m] = __ldg(qp + m);
+    }
+    const uint32_t *w = reinterpret_cast<const uint32_t *>(v);
+    uint32_t mx = 0u;  // largest |q| of the row as a bf16 bit pattern (orders like the value)
+#pragma unroll
+    for (int i = 0; i < 16; ++i) mx = __vmaxu2(mx, w[i] & 0x7FFF7FFFu);
+    mx = max(mx & 0xFFFFu, mx >> 16);
+    mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+    mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+    const float fm = __uint_as_float(mx << 16);
+    float s = 1.f;
+    if (fm > 0.f && fm < INFINITY) {
+      int e;
+      (void)frexpf(fm, &e);        // fm = f 2^e, f in [0.5, 1)
+      s = ldexpf(1.f, -(e + 1));   // max |q| s < 0.5
+    }
+    inv = 1.f / s;
+    const float s16 = s * 0.0625f;
+#pragma unroll
+    for (int ks = 0; ks < 8; ++ks) {
+      const uint32_t u0 = w[2 * ks], u1 = w[2 * ks + 1];
+      a0[ks] = pack_f16(__uint_as_float(u0 << 16) * s, __uint_as_float(u0 & 0xFFFF0000u) * s);
+      a2[ks] = pack_f16(__uint_as_float(u1 << 16) * s16, __uint_as_float(u1 & 0xFFFF0000u) * s16);
+    }
+  };
+
   int it = 0;
   bool ok = true;
-  while (gam_c < total) {
+  while (cc.prob < nprob) {
     const int stage = it % kScanStages;
     const uint32_t parity = (it / kScanStages) & 1;
     if (!mbar_wait(&full[stage], parity)) {
@@ -253,39 +312,20 @@ __global__ void __launch_bounds__(kScanWarps * 32, 2) scan_i4r8_kernel(ScanParam
       break;
     }
     --inflight;
-    const int prob = gc.b * p.Hkv + gc.h;
-    if (prob != cur_prob) {
-      cur_prob = prob;
-      const int hq = gc.h * p.G + x;
-      uint4 v[4] = {}, v8[4] = {};
-      if (x < p.G) {
-        const uint4 *qp = reinterpret_cast<const uint4 *>(q + ((int64_t)gc.b * p.Hq + hq) * LOCKS_D + 32 * t);
+    const int b = cc.prob / p.Hkv, h = cc.prob - b * p.Hkv;
+    if (cc.prob != cur_prob) {
+      cur_prob = cc.prob;
+      load_q_row(b, h * p.G + x, x < p.G, qa0, qa2, inv_s);
+      if (NH == 2) load_q_row(b, h * p.G + x + 8, x + 8 < p.G, qa1, qa3, inv_s8);
+      else {
 #pragma unroll
-        for (int m = 0; m < 4; ++m) v[m] = __ldg(qp + m);
-        pn = p.qnorm[gc.b * p.Hq + hq];
-      } else {
-        pn = 1.f;
+        for (int i = 0; i < 8; ++i) { qa1[i] = 0u; qa3[i] = 0u; }
       }
-      if (NH == 2 && x + 8 < p.G) {
-        const uint4 *qp = reinterpret_cast<const uint4 *>(q + ((int64_t)gc.b * p.Hq + hq + 8) * LOCKS_D + 32 * t);
-#pragma unroll
-        for (int m = 0; m < 4; ++m) v8[m] = __ldg(qp + m);
-        pn8 = p.qnorm[gc.b * p.Hq + hq + 8];
-      } else {
-        pn8 = 1.f;
-      }
-#pragma unroll
-      for (int m = 0; m < 4; ++m) {
-        qa0[2 * m] = v[m].x; qa2[2 * m] = v[m].y; qa0[2 * m + 1] = v[m].z; qa2[2 * m + 1] = v[m].w;
-        qa1[2 * m] = v8[m].x; qa3[2 * m] = v8[m].y; qa1[2 * m + 1] = v8[m].z; qa3[2 * m + 1] = v8[m].w;
-      }
-      kx = c2 / pn;
-      kx8 = c2 / pn8;
     }
 
     const uint8_t *sb = ring + stage * kStageBytes;
-    // ---- centroid dots for the 8 pages: a[head][page], int8 = 16 * (hi nibble - 8) + lo nibble
-    float cl[4] = {0.f, 0.f, 0.f, 0.f}, ch[4] = {0.f, 0.f, 0.f, 0.f};
+    // ---- centroid dots of the 8 pages: a[head][page] = sum_c code_mu[c] q'[c]
+    float cen[4] = {0.f, 0.f, 0.f, 0.f};
     {
       const uint4 *mp = reinterpret_cast<const uint4 *>(sb + x * kBlob + i4_off_mu(8) + t * 32);
       const uint4 m0 = mp[0], m1 = mp[1];
@@ -293,23 +333,20 @@ __global__ void __launch_bounds__(kScanWarps * 32, 2) scan_i4r8_kernel(ScanParam
 #pragma unroll
       for (int s = 0; s < 8; ++s) {
         const uint32_t w = mw[s];
-        const uint32_t l0 = bf16x2_sub(nib_pair(w, 0), 0x43004300u);   // - 128
-        const uint32_t l1 = bf16x2_sub(nib_pair(w, 8), 0x43004300u);
-        const uint32_t h0 = bf16x2_sub(nib_pair(w, 4), 0x43084308u);   // - 136
-        const uint32_t h1 = bf16x2_sub(nib_pair(w, 12), 0x43084308u);
-        mma_bf16(cl, qa0[s], qa1[s], qa2[s], qa3[s], l0, l1);
-        mma_bf16(ch, qa0[s], qa1[s], qa2[s], qa3[s], h0, h1);
+        const uint32_t b0 = f16x2_sub(and_or(w, kMB, kMagic), kSub128);                // code
+        const uint32_t b1 = f16x2_fma(and_or(w >> 8, kMB, kMagic), kSixteen, kSub16x ^ 0x80008000u);  // 16 code
+        mma_f16(cen, qa0[s], qa1[s], qa2[s], qa3[s], b0, b1);
       }
     }
     float acen[2 * NH];  // log2-domain centroid term for pages 2t, 2t+1 (and the second row half)
     {
       const float s0 = __half2float(*reinterpret_cast<const __half *>(sb + (2 * t) * kBlob + i4_off_smu(8)));
       const float s1 = __half2float(*reinterpret_cast<const __half *>(sb + (2 * t + 1) * kBlob + i4_off_smu(8)));
-      acen[0] = s0 * c2 * fmaf(16.f, ch[0], cl[0]);
-      acen[1] = s1 * c2 * fmaf(16.f, ch[1], cl[1]);
+      acen[0] = s0 * (c2 * inv_s) * cen[0];
+      acen[1] = s1 * (c2 * inv_s) * cen[1];
       if (NH == 2) {
-        acen[2] = s0 * c2 * fmaf(16.f, ch[2], cl[2]);
-        acen[3] = s1 * c2 * fmaf(16.f, ch[3], cl[3]);
+        acen[2] = s0 * (c2 * inv_s8) * cen[2];
+        acen[3] = s1 * (c2 * inv_s8) * cen[3];
       }
     }
     float res[2 * NH];
@@ -321,48 +358,52 @@ __global__ void __launch_bounds__(kScanWarps * 32, 2) scan_i4r8_kernel(ScanParam
       const uint8_t *pb = sb + pg * kBlob;
       const uint4 w4 = *reinterpret_cast<const uint4 *>(pb + lane * 16);
       const uint32_t ww[4] = {w4.x, w4.y, w4.z, w4.w};
-      float c1[4] = {0.f, 0.f, 0.f, 0.f};
+      float c1[4];
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
-        const uint32_t w = ww[j];
-        const uint32_t r0 = bf16x2_sub(nib_pair(w, 0), 0x43084308u);
-        const uint32_t r1 = bf16x2_sub(nib_pair(w, 4), 0x43084308u);
-        const uint32_t r2 = bf16x2_sub(nib_pair(w, 8), 0x43084308u);
-        const uint32_t r3 = bf16x2_sub(nib_pair(w, 12), 0x43084308u);
-        mma_bf16(c1, qa0[2 * j], qa1[2 * j], qa2[2 * j], qa3[2 * j], r0, r1);
-        mma_bf16(c1, qa0[2 * j + 1], qa1[2 * j + 1], qa2[2 * j + 1], qa3[2 * j + 1], r2, r3);
+        const uint32_t w = ww[j], wh = w >> 8;
+        const uint32_t r0 = f16x2_sub(and_or(w, kM0, kMagic), kSub8);     // code          (k-step 2j, cols 2t..)
+        const uint32_t r1 = f16x2_sub(and_or(w, kM1, kMagic), kSub128);   // 16 * code     (k-step 2j, cols 8+2t..)
+        const uint32_t r2 = f16x2_sub(and_or(wh, kM0, kMagic), kSub8);    // k-step 2j+1
+        const uint32_t r3 = f16x2_sub(and_or(wh, kM1, kMagic), kSub128);
+        if (j == 0) mma_f16_z(c1, qa0[0], qa1[0], qa2[0], qa3[0], r0, r1);
+        else mma_f16(c1, qa0[2 * j], qa1[2 * j], qa2[2 * j], qa3[2 * j], r0, r1);
+        mma_f16(c1, qa0[2 * j + 1], qa1[2 * j + 1], qa2[2 * j + 1], qa3[2 * j + 1], r2, r3);
       }
-      // projection -> fp16 hi + lo
+      // projection (already carrying sm_scale * log2 e) -> fp16 hi + lo
       const float2 sv = h2f2(*reinterpret_cast<const uint32_t *>(pb + i4_off_sv(8) + 4 * t));
-      const float p0 = c1[0] * sv.x * pn, p1 = c1[1] * sv.y * pn;
+      const float svx = sv.x * c2, svy = sv.y * c2;
+      const float p0 = c1[0] * svx, p1 = c1[1] * svy;
       const uint32_t hi = pack_f16(p0, p1);
       const float2 hf = h2f2(hi);
       const uint32_t lo = pack_f16(p0 - hf.x, p1 - hf.y);
       uint32_t hi8 = 0u, lo8 = 0u;
       if (NH == 2) {
-        const float p2 = c1[2] * sv.x * pn8, p3 = c1[3] * sv.y * pn8;
+        const float p2 = c1[2] * svx, p3 = c1[3] * svy;
         hi8 = pack_f16(p2, p3);
         const float2 hf8 = h2f2(hi8);
         lo8 = pack_f16(p2 - hf8.x, p3 - hf8.y);
       }
       // coefficient codes (offset-binary int8) -> exact fp16
       const uint32_t cw = *reinterpret_cast<const uint32_t *>(pb + i4_off_coef(8) + lane * 4);
-      const uint32_t b0 = f16x2_sub(__byte_perm(cw, 0x64646464u, 0x4140), 0x64806480u);
-      const uint32_t b1 = f16x2_sub(__byte_perm(cw, 0x64646464u, 0x4342), 0x64806480u);
-      float ca[4] = {0.f, 0.f, 0.f, 0.f}, cb[4] = {0.f, 0.f, 0.f, 0.f};
-      mma_f16(ca, hi, hi8, lo, lo8, b0, b0);
-      mma_f16(cb, hi, hi8, lo, lo8, b1, b1);
+      const uint32_t b0 = f16x2_sub(__byte_perm(cw, 0x64646464u, 0x4140), kSub128);
+      const uint32_t b1 = f16x2_sub(__byte_perm(cw, 0x64646464u, 0x4342), kSub128);
+      float ca[4], cb[4];
+      mma_f16_z(ca, hi, hi8, lo, lo8, b0, b0);
+      mma_f16_z(cb, hi, hi8, lo, lo8, b1, b1);
       const uint2 scw = *reinterpret_cast<const uint2 *>(pb + i4_off_sc(8) + 8 * t);
       const float2 s01 = h2f2(scw.x), s89 = h2f2(scw.y);
 #pragma unroll
       for (int hh = 0; hh < NH; ++hh) {
-        const float kk = hh ? kx8 : kx;
-        const float l0 = ca[2 * hh] * (s01.x * kk), l1 = ca[2 * hh + 1] * (s01.y * kk);
-        const float l2 = cb[2 * hh] * (s89.x * kk), l3 = cb[2 * hh + 1] * (s89.y * kk);
-        float m = fmaxf(fmaxf(l0, l1), fmaxf(l2, l3));
-        m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 1));
-        m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 2));
-        float e = fast_ex2(l0 - m) + fast_ex2(l1 - m) + fast_ex2(l2 - m) + fast_ex2(l3 - m);
+        const float iv = hh ? inv_s8 : inv_s;
+        const float y0 = ca[2 * hh] * s01.x, y1 = ca[2 * hh + 1] * s01.y;
+        const float y2 = cb[2 * hh] * s89.x, y3 = cb[2 * hh + 1] * s89.y;
+        float my = fmaxf(fmaxf(y0, y1), fmaxf(y2, y3));
+        my = fmaxf(my, __shfl_xor_sync(0xffffffffu, my, 1));
+        my = fmaxf(my, __shfl_xor_sync(0xffffffffu, my, 2));
+        const float m = my * iv;   // logits are y * iv (iv > 0, a power of two)
+        float e = fast_ex2(fmaf(y0, iv, -m)) + fast_ex2(fmaf(y1, iv, -m)) + fast_ex2(fmaf(y2, iv, -m)) +
+                  fast_ex2(fmaf(y3, iv, -m));
         e += __shfl_xor_sync(0xffffffffu, e, 1);
         e += __shfl_xor_sync(0xffffffffu, e, 2);
         const float v = m + fast_lg2(e);
@@ -370,22 +411,23 @@ __global__ void __launch_bounds__(kScanWarps * 32, 2) scan_i4r8_kernel(ScanParam
       }
     }
     __syncwarp();  // every lane is done reading this stage
-    if (gam_p < total) {
-      issue(stage, gp);
+    if (cp.prob < nprob) {
+      issue(stage, cp);
       ++inflight;
-      gam_p = next_valid(gam_p + W, gp);
+      cp.grp += wpp;
+      settle(cp);
     }
 
     // ---- write s^ and the group's candidate partial
-    const int page0 = gc.grp * LOCKS_GROUP + 2 * t;
+    const int page0 = cc.grp * LOCKS_GROUP + 2 * t;
 #pragma unroll
     for (int hh = 0; hh < NH; ++hh) {
       const int g = x + 8 * hh;
       const float v0 = (res[2 * hh] + acen[2 * hh]) * kLn2;
       const float v1 = (res[2 * hh + 1] + acen[2 * hh + 1]) * kLn2;
-      const bool in0 = page0 < gc.nsc, in1 = page0 + 1 < gc.nsc;
+      const bool in0 = page0 < cc.nsc, in1 = page0 + 1 < cc.nsc;
       if (g < p.G) {
-        float *dst = p.shat + ((int64_t)gc.b * p.Hq + gc.h * p.G + g) * p.Pmax + page0;
+        float *dst = p.shat + ((int64_t)b * p.Hq + h * p.G + g) * p.Pmax + page0;
         if (in0) dst[0] = v0;
         if (in1) dst[1] = v1;
       }
@@ -398,9 +440,10 @@ __global__ void __launch_bounds__(kScanWarps * 32, 2) scan_i4r8_kernel(ScanParam
       e += __shfl_xor_sync(0xffffffffu, e, 1);
       e += __shfl_xor_sync(0xffffffffu, e, 2);
       if (t == 0 && g < p.G)
-        p.part[((int64_t)gc.b * p.Hq + gc.h * p.G + g) * p.max_groups + gc.grp] = make_float2(m, e);
+        p.part[((int64_t)b * p.Hq + h * p.G + g) * p.max_groups + cc.grp] = make_float2(m, e);
     }
-    gam_c = next_valid(gam_c + W, gc);
+    cc.grp += wpp;
+    settle(cc);
     ++it;
   }
   if (!ok) {
@@ -424,7 +467,6 @@ int locks_launch_scan(locks_ctx *c, const void *q, const void *summaries, const 
   p.seq_lens = kv->seq_lens;
   p.shat = shat;
   p.part = c->part;
-  p.qnorm = c->qnorm;
   p.status = c->status;
   p.batch = batch; p.Hq = c->cfg.num_q_heads; p.Hkv = c->cfg.num_kv_heads; p.G = c->G;
   p.Pmax = c->Pmax; p.max_groups = c->max_groups; p.num_blocks = kv->num_blocks; p.k = c->k;

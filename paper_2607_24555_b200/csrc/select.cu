@@ -2,7 +2,7 @@
 //   log Z_g   = log sum_{j in 1..P-2} exp s^_j(q_g)                       (candidates only)
 //   log m_bar_j = log( (1/G) sum_g exp(s^_j(q_g) - log Z_g) )
 //   S = {0, P-1}  U  top-(k-2) candidates by log m_bar_j (ties: lower page index), ids ascending.
-// Stage 1 (one CTA per 2048-page chunk of a (request, KV head)) ranks its chunk with an exact
+// Stage 1 (one CTA per chunk of up to 8192 pages of a (request, KV head)) ranks its chunk with an exact
 // 4-pass radix select held in registers + shared-memory histograms and compacts the winners in
 // page order.  With one chunk it writes the final table; with several, each chunk emits its own
 // top-(k-2) (value, page) list and stage 2 re-selects among them (a chunk's local top-(k-2) always
@@ -20,7 +20,7 @@ struct SelParams {
   float *logshare;
   float *cand_val;
   int32_t *cand_idx;
-  int batch, Hq, Hkv, G, Pmax, max_groups, k, chunks, kc;
+  int batch, Hq, Hkv, G, Pmax, max_groups, k, chunks, kc, chunk_pages;
 };
 
 __device__ __forceinline__ uint32_t order_key(float f) {
@@ -44,7 +44,7 @@ __device__ void block_topk(const uint32_t (&key)[EPT], int K, bool (&sel)[EPT], 
   int remaining = K;
   for (int pass = 0; pass < 4; ++pass) {
     const int shift = 24 - 8 * pass;
-    sh_hist[tid] = 0;  // 256 bins, 256 threads
+    if (tid < 256) sh_hist[tid] = 0;
     __syncthreads();
 #pragma unroll
     for (int i = 0; i < EPT; ++i)
@@ -119,7 +119,7 @@ __device__ void group_logz(const SelParams &p, int b, int h, int ngroups, float 
       const float2 v = pp[i];
       if (v.x > -INFINITY) {
         const float nm = fmaxf(m, v.x);
-        s = s * expf(m - nm) + v.y * expf(v.x - nm);
+        s = s * __expf(m - nm) + v.y * __expf(v.x - nm);
         m = nm;
       }
     }
@@ -128,14 +128,15 @@ __device__ void group_logz(const SelParams &p, int b, int h, int ngroups, float 
       const float om = __shfl_xor_sync(0xffffffffu, m, o), os = __shfl_xor_sync(0xffffffffu, s, o);
       const float nm = fmaxf(m, om);
       if (nm > -INFINITY) {
-        s = s * expf(m - nm) + os * expf(om - nm);
+        s = s * __expf(m - nm) + os * __expf(om - nm);
         m = nm;
       }
     }
-    if (lane == 0) sh_logz[g] = m + logf(s);
+    if (lane == 0) sh_logz[g] = m + __logf(s);
   }
 }
 
+template <int EPT>
 __global__ void __launch_bounds__(LOCKS_SEL_THREADS) select_stage1_kernel(SelParams p) {
   __shared__ int sh_hist[256];
   __shared__ int sh_misc[2 + LOCKS_SEL_THREADS / 32];
@@ -152,8 +153,7 @@ __global__ void __launch_bounds__(LOCKS_SEL_THREADS) select_stage1_kernel(SelPar
     }
     return;
   }
-  const int c0 = chunk * LOCKS_SEL_CHUNK;  // first page of this chunk
-  const int ncand_total = P - 2;
+  const int c0 = chunk * p.chunk_pages;  // first page of this chunk
   if (c0 > P - 2) {  // chunk past the candidates: emit an empty list
     if (p.chunks > 1)
       for (int j = tid; j < p.kc; j += LOCKS_SEL_THREADS) {
@@ -164,46 +164,47 @@ __global__ void __launch_bounds__(LOCKS_SEL_THREADS) select_stage1_kernel(SelPar
   }
   group_logz(p, b, h, (P - 1 + LOCKS_GROUP - 1) / LOCKS_GROUP, sh_logz);
   __syncthreads();
-  // log m_bar for this thread's 8 consecutive pages
-  float val[LOCKS_SEL_EPT];
-  uint32_t key[LOCKS_SEL_EPT];
-  const int pbase = c0 + tid * LOCKS_SEL_EPT;
-  float mx[LOCKS_SEL_EPT], sm[LOCKS_SEL_EPT];
+  // log m_bar of this thread's EPT consecutive pages: log mean_g exp(s^_g - log Z_g)
+  float val[EPT];
+  uint32_t key[EPT];
+  const int pbase = c0 + tid * EPT;
+  const float logG = __logf((float)p.G);
+  {
+    float mx[EPT], sm[EPT];
 #pragma unroll
-  for (int i = 0; i < LOCKS_SEL_EPT; ++i) { mx[i] = -INFINITY; sm[i] = 0.f; }
-  for (int g = 0; g < p.G; ++g) {
-    const float *row = p.shat + ((int64_t)b * p.Hq + h * p.G + g) * p.Pmax;
-    const float lz = sh_logz[g];
+    for (int i = 0; i < EPT; ++i) { mx[i] = -INFINITY; sm[i] = 0.f; }
+    const float *row0 = p.shat + ((int64_t)b * p.Hq + h * p.G) * p.Pmax;
+    for (int g = 0; g < p.G; ++g) {
+      const float *row = row0 + (int64_t)g * p.Pmax;
+      const float lz = sh_logz[g];
 #pragma unroll
-    for (int i = 0; i < LOCKS_SEL_EPT; ++i) {
-      const int page = pbase + i;
-      if (page >= 1 && page <= P - 2) {
-        const float tv = row[page] - lz;
-        const float nm = fmaxf(mx[i], tv);
-        sm[i] = sm[i] * expf(mx[i] - nm) + expf(tv - nm);
-        mx[i] = nm;
+      for (int i = 0; i < EPT; ++i) {
+        const int page = pbase + i;
+        if (page >= 1 && page <= P - 2) {
+          const float tv = row[page] - lz;
+          const float nm = fmaxf(mx[i], tv);
+          sm[i] = sm[i] * __expf(mx[i] - nm) + __expf(tv - nm);
+          mx[i] = nm;
+        }
       }
     }
-  }
-  const float logG = logf((float)p.G);
-  int nvalid_local = 0;
 #pragma unroll
-  for (int i = 0; i < LOCKS_SEL_EPT; ++i) {
-    const int page = pbase + i;
-    const bool valid = page >= 1 && page <= P - 2;
-    val[i] = valid ? mx[i] + logf(sm[i]) - logG : -INFINITY;
-    key[i] = valid ? order_key(val[i]) : 0u;
-    nvalid_local += valid;
-    if (valid && p.logshare) p.logshare[prob * p.Pmax + page] = val[i];
+    for (int i = 0; i < EPT; ++i) {
+      const int page = pbase + i;
+      const bool valid = page >= 1 && page <= P - 2;
+      val[i] = valid ? mx[i] + __logf(sm[i]) - logG : -INFINITY;
+      key[i] = valid ? order_key(val[i]) : 0u;
+      if (valid && p.logshare) p.logshare[prob * p.Pmax + page] = val[i];
+    }
   }
-  const int cand_in_chunk = min(P - 2, c0 + LOCKS_SEL_CHUNK - 1) - max(1, c0) + 1;
+  const int cand_in_chunk = min(P - 2, c0 + p.chunk_pages - 1) - max(1, c0) + 1;
   const int K = min(p.k - 2, cand_in_chunk);
-  bool sel[LOCKS_SEL_EPT];
-  int pos[LOCKS_SEL_EPT];
-  block_topk<LOCKS_SEL_EPT>(key, K, sel, pos, sh_hist, sh_misc);
+  bool sel[EPT];
+  int pos[EPT];
+  block_topk<EPT>(key, K, sel, pos, sh_hist, sh_misc);
   if (p.chunks == 1) {
 #pragma unroll
-    for (int i = 0; i < LOCKS_SEL_EPT; ++i)
+    for (int i = 0; i < EPT; ++i)
       if (sel[i]) ids[1 + pos[i]] = pbase + i;
     if (tid == 0) {
       ids[0] = 0;
@@ -214,11 +215,10 @@ __global__ void __launch_bounds__(LOCKS_SEL_THREADS) select_stage1_kernel(SelPar
     float *cv = p.cand_val + (prob * p.chunks + chunk) * p.kc;
     int32_t *ci = p.cand_idx + (prob * p.chunks + chunk) * p.kc;
 #pragma unroll
-    for (int i = 0; i < LOCKS_SEL_EPT; ++i)
+    for (int i = 0; i < EPT; ++i)
       if (sel[i]) { cv[pos[i]] = val[i]; ci[pos[i]] = pbase + i; }
     for (int j = K + tid; j < p.kc; j += LOCKS_SEL_THREADS) { cv[j] = -INFINITY; ci[j] = -1; }
   }
-  (void)ncand_total; (void)nvalid_local;
 }
 
 template <int EPT>
@@ -265,14 +265,18 @@ int locks_launch_select(locks_ctx *c, const float *shat, const locks_kv *kv, int
   p.cand_val = c->cand_val; p.cand_idx = c->cand_idx;
   p.batch = batch; p.Hq = c->cfg.num_q_heads; p.Hkv = c->cfg.num_kv_heads; p.G = c->G; p.Pmax = c->Pmax;
   p.max_groups = c->max_groups; p.k = c->k; p.chunks = c->sel_chunks; p.kc = c->sel_kc;
-  select_stage1_kernel<<<dim3(c->sel_chunks, p.Hkv, batch), LOCKS_SEL_THREADS, 0, st>>>(p);
+  p.chunk_pages = c->sel_ept * LOCKS_SEL_THREADS;
+  dim3 g1(c->sel_chunks, p.Hkv, batch);
+  if (c->sel_ept == 4) select_stage1_kernel<4><<<g1, LOCKS_SEL_THREADS, 0, st>>>(p);
+  else if (c->sel_ept == 8) select_stage1_kernel<8><<<g1, LOCKS_SEL_THREADS, 0, st>>>(p);
+  else select_stage1_kernel<16><<<g1, LOCKS_SEL_THREADS, 0, st>>>(p);
   int rc = locks_check_launch(c);
   if (rc != LOCKS_OK || c->sel_chunks == 1) return rc;
   const int N = c->sel_chunks * c->sel_kc;
   const int ept = (N + LOCKS_SEL_THREADS - 1) / LOCKS_SEL_THREADS;
   dim3 grid(p.Hkv, batch);
-  if (ept <= 8) select_stage2_kernel<8><<<grid, LOCKS_SEL_THREADS, 0, st>>>(p);
-  else if (ept <= 32) select_stage2_kernel<32><<<grid, LOCKS_SEL_THREADS, 0, st>>>(p);
+  if (ept <= 4) select_stage2_kernel<4><<<grid, LOCKS_SEL_THREADS, 0, st>>>(p);
+  else if (ept <= 16) select_stage2_kernel<16><<<grid, LOCKS_SEL_THREADS, 0, st>>>(p);
   else return LOCKS_ERR_UNSUPPORTED;
   return locks_check_launch(c);
 }

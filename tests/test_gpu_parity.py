@@ -128,9 +128,9 @@ def test_i4_generic_ranks(rank):
 
 
 def test_two_level_select_long_context():
-    """More than one 2048-page chunk per KV head: stage-1 lists + stage-2 re-select."""
+    """More than one 8192-page chunk per KV head: stage-1 lists + stage-2 re-select."""
     from gpu_util import check_select_and_attend
-    gc = _gc(locks_synth.Workload("long", [16 * 4500 + 3], Hq=32, Hkv=2, budget=2048, seed=9))
+    gc = _gc(locks_synth.Workload("long", [16 * 9000 + 3], Hq=32, Hkv=2, budget=2048, seed=9))
     differed = check_select_and_attend(gc, gc.oracle_summaries(), out_tol=2e-2)
     assert differed <= 1
 
