@@ -50,7 +50,18 @@ __device__ __forceinline__ bool resolve_page(const AttParams &p, int b, int64_t 
   return ntok > 0;
 }
 
-template <int NH>
+__device__ __forceinline__ uint32_t movm_trans_b16(uint32_t v) {
+  uint32_t d;
+  asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(v));
+  return d;
+}
+
+// Orientation: tokens are the MMA rows.  Per page (16 tokens):
+//   S^T[16 tokens x 8 heads]  = K[16 x 128] . q^T[128 x 8]          (8 k-steps, A = K via ldmatrix)
+//   O^T[128 dims x 8 heads]  += V^T[128 x 16] . P^T[16 x 8]          (8 row tiles, A = V via ldmatrix.trans,
+//                                                                   B = P^T after an 8x8 movmatrix transpose)
+// so both products use all 16 rows of the tile and the accumulator is 32 registers per 8 heads.
+template <int NH, bool CONTIG>
 __global__ void __launch_bounds__(LOCKS_ATT_WARPS * 32) attend_bf16_kernel(AttParams p) {
   extern __shared__ __align__(128) uint8_t smem[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -63,111 +74,156 @@ __global__ void __launch_bounds__(LOCKS_ATT_WARPS * 32) attend_bf16_kernel(AttPa
   const int lo = split * p.pages_per_cta;
   const int hi = min(lo + p.pages_per_cta, npages);
   uint8_t *ring = smem + warp * 2 * kAttStage;
-  const __nv_bfloat16 *K = reinterpret_cast<const __nv_bfloat16 *>(p.k);
-  const __nv_bfloat16 *V = reinterpret_cast<const __nv_bfloat16 *>(p.v);
+  const uint8_t *Kb = reinterpret_cast<const uint8_t *>(p.k);
+  const uint8_t *Vb = reinterpret_cast<const uint8_t *>(p.v);
 
-  // query fragments: rows = heads of the group
-  uint32_t qa[8][4];
+  // query as the B operand: lane (x, t) holds head x (+8), dims 16 s + 2t.. and 16 s + 8 + 2t..
+  uint32_t qb[NH][8][2];
   {
     const __nv_bfloat16 *q = reinterpret_cast<const __nv_bfloat16 *>(p.q);
-    const uint32_t *q0 = reinterpret_cast<const uint32_t *>(q + ((int64_t)b * p.Hq + h * p.G + x) * LOCKS_D);
-    const uint32_t *q8 = reinterpret_cast<const uint32_t *>(q + ((int64_t)b * p.Hq + h * p.G + x + 8) * LOCKS_D);
 #pragma unroll
-    for (int s = 0; s < 8; ++s) {
-      qa[s][0] = (x < p.G) ? __ldg(q0 + 8 * s + t) : 0u;
-      qa[s][2] = (x < p.G) ? __ldg(q0 + 8 * s + 4 + t) : 0u;
-      qa[s][1] = (NH == 2 && x + 8 < p.G) ? __ldg(q8 + 8 * s + t) : 0u;
-      qa[s][3] = (NH == 2 && x + 8 < p.G) ? __ldg(q8 + 8 * s + 4 + t) : 0u;
+    for (int hh = 0; hh < NH; ++hh) {
+      const int g = x + 8 * hh;
+      const uint32_t *qr = reinterpret_cast<const uint32_t *>(q + ((int64_t)b * p.Hq + h * p.G + g) * LOCKS_D);
+#pragma unroll
+      for (int s = 0; s < 8; ++s) {
+        qb[hh][s][0] = (g < p.G) ? __ldg(qr + 8 * s + t) : 0u;
+        qb[hh][s][1] = (g < p.G) ? __ldg(qr + 8 * s + 4 + t) : 0u;
+      }
     }
   }
   const float c2 = p.sm_scale * kLog2e;
 
-  float oacc[16][4];
+  float oacc[8][NH][4];
 #pragma unroll
-  for (int i = 0; i < 16; ++i) { oacc[i][0] = oacc[i][1] = oacc[i][2] = oacc[i][3] = 0.f; }
-  float mrun[2] = {-INFINITY, -INFINITY}, lrun[2] = {0.f, 0.f};
+  for (int i = 0; i < 8; ++i)
+#pragma unroll
+    for (int hh = 0; hh < NH; ++hh) oacc[i][hh][0] = oacc[i][hh][1] = oacc[i][hh][2] = oacc[i][hh][3] = 0.f;
+  float mrun[NH][2], lrun[NH][2];   // per head column 2t, 2t+1 (+8): running max, this lane's partial sum
+#pragma unroll
+  for (int hh = 0; hh < NH; ++hh) { mrun[hh][0] = mrun[hh][1] = -INFINITY; lrun[hh][0] = lrun[hh][1] = 0.f; }
 
-  auto issue = [&](int idx, int stage) -> int {  // returns valid tokens (0: nothing loaded)
-    int block = 0, ntok = 0;
-    const bool okp = resolve_page(p, b, prob, idx, T, block, ntok);
-    if (!okp) ntok = 0;
+  // per-lane constants of the 16-byte copies: copy i moves chunk (lane & 15) of token (lane >> 4) + 2 i
+  const int tok0 = lane >> 4, ch0 = lane & 15;
+  const int64_t goff0 = ((int64_t)tok0 * p.st + ch0 * 8) * 2;       // bytes
+  const int64_t gstep = p.st * 4;                                    // two token rows, bytes
+  uint32_t sw[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) sw[i] = (uint32_t)(tok0 * 256 + (((ch0 ^ tok0) ^ ((2 * i) & 7)) << 4));
+
+  // page ids and physical blocks of this warp's pages are resolved 32 at a time, one lane each, so the
+  // two dependent global loads are paid once per batch instead of once per page
+  const int first = lo + warp;
+  auto resolve_batch = [&](int jb, int &blk, int &nt) {
+    const int idx = first + (jb + lane) * LOCKS_ATT_WARPS;
+    blk = 0;
+    nt = 0;
+    if (idx < hi && !resolve_page(p, b, prob, idx, T, blk, nt)) nt = 0;
+  };
+  int blk_cur, nt_cur, blk_nxt = 0, nt_nxt = 0;
+  resolve_batch(0, blk_cur, nt_cur);
+
+  auto issue = [&](int j, int stage) -> int {  // j-th page of this warp; returns its valid tokens
+    const int block = __shfl_sync(0xffffffffu, blk_cur, j & 31);
+    const int ntok = __shfl_sync(0xffffffffu, nt_cur, j & 31);
     uint8_t *kt = ring + stage * kAttStage, *vt = kt + kTile;
-    const int64_t base = (int64_t)block * p.sb + (int64_t)h * p.sh;
+    const int64_t base = ((int64_t)block * p.sb + (int64_t)h * p.sh) * 2 + goff0;
+    const uint8_t *kp = Kb + base, *vp = Vb + base;
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
-      const int c = lane + 32 * i, tok = c >> 4, ch = c & 15;
-      const int64_t off = base + (int64_t)tok * p.st + ch * 8;
-      const int so = tok * 256 + ((ch ^ (tok & 7)) << 4);
-      cp_async16(kt + so, K + off, tok < ntok);   // rows past the sequence end are zero-filled
-      cp_async16(vt + so, V + off, tok < ntok);
+      const uint32_t so = sw[i & 3] + 512 * i;
+      const bool valid = tok0 + 2 * i < ntok;   // rows past the sequence end are zero-filled
+      if (CONTIG) {   // token rows are 256 bytes apart: immediate offsets
+        cp_async16(kt + so, kp + i * 512, valid);
+        cp_async16(vt + so, vp + i * 512, valid);
+      } else {
+        cp_async16(kt + so, kp + i * gstep, valid);
+        cp_async16(vt + so, vp + i * gstep, valid);
+      }
     }
     cp_async_commit();
     return ntok;
   };
 
-  const int first = lo + warp;
   int ntok_cur = 0, ntok_next = 0;
-  if (first < hi) ntok_cur = issue(first, 0);
+  if (first < hi) ntok_cur = issue(0, 0);
   int j = 0;
   for (int idx = first; idx < hi; idx += LOCKS_ATT_WARPS, ++j) {
     const int stage = j & 1;
     const bool more = idx + LOCKS_ATT_WARPS < hi;
-    if (more) ntok_next = issue(idx + LOCKS_ATT_WARPS, stage ^ 1);
+    if ((j & 31) == 15) resolve_batch((j & ~31) + 32, blk_nxt, nt_nxt);   // next batch, half a batch early
+    if (more) {
+      if (((j + 1) & 31) == 0) { blk_cur = blk_nxt; nt_cur = nt_nxt; }
+      ntok_next = issue(j + 1, stage ^ 1);
+    }
     if (more) cp_async_wait<1>(); else cp_async_wait<0>();
     __syncwarp();
     const uint8_t *kt = ring + stage * kAttStage, *vt = kt + kTile;
     const int ntok = ntok_cur;
-    // ---- S = q K^T  (16 heads x 16 tokens)
-    float sacc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+    const int m = lane >> 3, rr = lane & 7;
+    // ---- S^T = K q^T
+    float sacc[NH][4];
+#pragma unroll
+    for (int hh = 0; hh < NH; ++hh) sacc[hh][0] = sacc[hh][1] = sacc[hh][2] = sacc[hh][3] = 0.f;
     {
-      const int m = lane >> 3, rr = lane & 7;
-#pragma unroll
-      for (int s2 = 0; s2 < 4; ++s2) {
-#pragma unroll
-        for (int nt = 0; nt < 2; ++nt) {
-          const int tok = nt * 8 + rr, ch = 4 * s2 + m;
-          uint32_t r[4];
-          ldsm_x4(r, kt + tok * 256 + ((ch ^ (tok & 7)) << 4));
-          mma_bf16(sacc[nt], qa[2 * s2][0], qa[2 * s2][1], qa[2 * s2][2], qa[2 * s2][3], r[0], r[1]);
-          mma_bf16(sacc[nt], qa[2 * s2 + 1][0], qa[2 * s2 + 1][1], qa[2 * s2 + 1][2], qa[2 * s2 + 1][3], r[2], r[3]);
-        }
-      }
-    }
-    // ---- online softmax per head row
-    uint32_t pa[4] = {0u, 0u, 0u, 0u};
-#pragma unroll
-    for (int hh = 0; hh < NH; ++hh) {
-      float v0 = sacc[0][2 * hh] * c2, v1 = sacc[0][2 * hh + 1] * c2;
-      float v2 = sacc[1][2 * hh] * c2, v3 = sacc[1][2 * hh + 1] * c2;
-      if (2 * t >= ntok) v0 = -INFINITY;
-      if (2 * t + 1 >= ntok) v1 = -INFINITY;
-      if (8 + 2 * t >= ntok) v2 = -INFINITY;
-      if (9 + 2 * t >= ntok) v3 = -INFINITY;
-      float m = fmaxf(fmaxf(v0, v1), fmaxf(v2, v3));
-      m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 1));
-      m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 2));
-      const float mnew = fmaxf(mrun[hh], m);
-      const float msafe = (mnew == -INFINITY) ? 0.f : mnew;
-      const float alpha = ex2f(mrun[hh] - msafe);
-      const float p0 = ex2f(v0 - msafe), p1 = ex2f(v1 - msafe), p2 = ex2f(v2 - msafe), p3 = ex2f(v3 - msafe);
-      lrun[hh] = lrun[hh] * alpha + (p0 + p1) + (p2 + p3);
-      mrun[hh] = mnew;
-#pragma unroll
-      for (int i = 0; i < 16; ++i) { oacc[i][2 * hh] *= alpha; oacc[i][2 * hh + 1] *= alpha; }
-      pa[hh] = pack_bf16(p0, p1);
-      pa[2 + hh] = pack_bf16(p2, p3);
-    }
-    // ---- O += P V
-    {
-      const int m = lane >> 3, rr = lane & 7;
       const int tok = (m & 1) * 8 + rr;
 #pragma unroll
-      for (int ntp = 0; ntp < 8; ++ntp) {
-        const int ch = 2 * ntp + (m >> 1);
+      for (int s = 0; s < 8; ++s) {
+        const int ch = 2 * s + (m >> 1);
+        uint32_t r[4];
+        ldsm_x4(r, kt + tok * 256 + ((ch ^ (tok & 7)) << 4));
+#pragma unroll
+        for (int hh = 0; hh < NH; ++hh) mma_bf16(sacc[hh], r[0], r[1], r[2], r[3], qb[hh][s][0], qb[hh][s][1]);
+      }
+    }
+    // ---- online softmax down the token rows; this lane: tokens x, x + 8, heads 2t, 2t+1 (+8)
+    uint32_t pb0[NH], pb1[NH];
+    const bool v0ok = x < ntok, v1ok = x + 8 < ntok;
+#pragma unroll
+    for (int hh = 0; hh < NH; ++hh) {
+      float sv[4];
+      sv[0] = v0ok ? sacc[hh][0] * c2 : -INFINITY;
+      sv[1] = v0ok ? sacc[hh][1] * c2 : -INFINITY;
+      sv[2] = v1ok ? sacc[hh][2] * c2 : -INFINITY;
+      sv[3] = v1ok ? sacc[hh][3] * c2 : -INFINITY;
+      float cm0 = fmaxf(sv[0], sv[2]), cm1 = fmaxf(sv[1], sv[3]);
+#pragma unroll
+      for (int o = 4; o < 32; o <<= 1) {
+        cm0 = fmaxf(cm0, __shfl_xor_sync(0xffffffffu, cm0, o));
+        cm1 = fmaxf(cm1, __shfl_xor_sync(0xffffffffu, cm1, o));
+      }
+      const float mn0 = fmaxf(mrun[hh][0], cm0), mn1 = fmaxf(mrun[hh][1], cm1);
+      const float ms0 = (mn0 == -INFINITY) ? 0.f : mn0, ms1 = (mn1 == -INFINITY) ? 0.f : mn1;
+      const bool moved = (mn0 != mrun[hh][0]) || (mn1 != mrun[hh][1]);
+      if (__any_sync(0xffffffffu, moved)) {   // rescale only when some running max rose
+        const float a0 = ex2f(mrun[hh][0] - ms0), a1 = ex2f(mrun[hh][1] - ms1);
+        lrun[hh][0] *= a0;
+        lrun[hh][1] *= a1;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          oacc[i][hh][0] *= a0; oacc[i][hh][2] *= a0;
+          oacc[i][hh][1] *= a1; oacc[i][hh][3] *= a1;
+        }
+      }
+      mrun[hh][0] = mn0;
+      mrun[hh][1] = mn1;
+      const float p00 = ex2f(sv[0] - ms0), p01 = ex2f(sv[1] - ms1), p10 = ex2f(sv[2] - ms0), p11 = ex2f(sv[3] - ms1);
+      lrun[hh][0] += p00 + p10;
+      lrun[hh][1] += p01 + p11;
+      // P^T rows (tokens) -> B fragment (k = tokens 2t, 2t+1 | 8 + 2t.., n = head x)
+      pb0[hh] = movm_trans_b16(pack_bf16(p00, p01));
+      pb1[hh] = movm_trans_b16(pack_bf16(p10, p11));
+    }
+    // ---- O^T += V^T P^T
+    {
+      const int tok = (m >> 1) * 8 + rr;
+#pragma unroll
+      for (int mt = 0; mt < 8; ++mt) {
+        const int ch = 2 * mt + (m & 1);
         uint32_t r[4];
         ldsm_x4_trans(r, vt + tok * 256 + ((ch ^ (tok & 7)) << 4));
-        mma_bf16(oacc[2 * ntp], pa[0], pa[1], pa[2], pa[3], r[0], r[1]);
-        mma_bf16(oacc[2 * ntp + 1], pa[0], pa[1], pa[2], pa[3], r[2], r[3]);
+#pragma unroll
+        for (int hh = 0; hh < NH; ++hh) mma_bf16(oacc[mt][hh], r[0], r[1], r[2], r[3], pb0[hh], pb1[hh]);
       }
     }
     __syncwarp();
@@ -175,20 +231,26 @@ __global__ void __launch_bounds__(LOCKS_ATT_WARPS * 32) attend_bf16_kernel(AttPa
   }
   cp_async_wait<0>();
 #pragma unroll
-  for (int hh = 0; hh < NH; ++hh) {
-    lrun[hh] += __shfl_xor_sync(0xffffffffu, lrun[hh], 1);
-    lrun[hh] += __shfl_xor_sync(0xffffffffu, lrun[hh], 2);
-  }
+  for (int hh = 0; hh < NH; ++hh)
+#pragma unroll
+    for (int c = 0; c < 2; ++c)
+#pragma unroll
+      for (int o = 4; o < 32; o <<= 1) lrun[hh][c] += __shfl_xor_sync(0xffffffffu, lrun[hh][c], o);
   __syncthreads();  // every warp is done with its ring: reuse it for the merge
-  float *wo = reinterpret_cast<float *>(ring);          // [16][128] fp32
+  float *wo = reinterpret_cast<float *>(ring);          // [16 heads][128] fp32
   float *wm = wo + 16 * LOCKS_D, *wl = wm + 16;          // [16], [16]
 #pragma unroll
   for (int hh = 0; hh < NH; ++hh) {
-    const int row = x + 8 * hh;
 #pragma unroll
-    for (int nt = 0; nt < 16; ++nt)
-      *reinterpret_cast<float2 *>(wo + row * LOCKS_D + nt * 8 + 2 * t) = make_float2(oacc[nt][2 * hh], oacc[nt][2 * hh + 1]);
-    if (t == 0) { wm[row] = mrun[hh]; wl[row] = lrun[hh]; }
+    for (int c = 0; c < 2; ++c) {
+      const int row = 8 * hh + 2 * t + c;
+#pragma unroll
+      for (int mt = 0; mt < 8; ++mt) {
+        wo[row * LOCKS_D + 16 * mt + x] = oacc[mt][hh][c];
+        wo[row * LOCKS_D + 16 * mt + 8 + x] = oacc[mt][hh][2 + c];
+      }
+      if (x == 0) { wm[row] = mrun[hh][c]; wl[row] = lrun[hh][c]; }
+    }
   }
   __syncthreads();
   for (int e = threadIdx.x; e < p.G * LOCKS_D; e += LOCKS_ATT_WARPS * 32) {
@@ -358,13 +420,21 @@ int locks_launch_attend(locks_ctx *c, const void *q, const locks_kv *kv, int bat
   if (bf) {
     static bool attr_done = false;
     if (!attr_done) {
-      cudaFuncSetAttribute(attend_bf16_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttSmem);
-      cudaFuncSetAttribute(attend_bf16_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttSmem);
+      cudaFuncSetAttribute(attend_bf16_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttSmem);
+      cudaFuncSetAttribute(attend_bf16_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttSmem);
+      cudaFuncSetAttribute(attend_bf16_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttSmem);
+      cudaFuncSetAttribute(attend_bf16_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttSmem);
       attr_done = true;
     }
     dim3 grid(p.splits, p.Hkv, batch);
-    if (c->G <= 8) attend_bf16_kernel<1><<<grid, LOCKS_ATT_WARPS * 32, kAttSmem, st>>>(p);
-    else attend_bf16_kernel<2><<<grid, LOCKS_ATT_WARPS * 32, kAttSmem, st>>>(p);
+    const bool contig = kv->stride_token == LOCKS_D;
+    if (c->G <= 8) {
+      if (contig) attend_bf16_kernel<1, true><<<grid, LOCKS_ATT_WARPS * 32, kAttSmem, st>>>(p);
+      else attend_bf16_kernel<1, false><<<grid, LOCKS_ATT_WARPS * 32, kAttSmem, st>>>(p);
+    } else {
+      if (contig) attend_bf16_kernel<2, true><<<grid, LOCKS_ATT_WARPS * 32, kAttSmem, st>>>(p);
+      else attend_bf16_kernel<2, false><<<grid, LOCKS_ATT_WARPS * 32, kAttSmem, st>>>(p);
+    }
   } else {
     dim3 grid(p.splits, p.Hq, batch);
     attend_generic_kernel<float><<<grid, 128, 0, st>>>(p);

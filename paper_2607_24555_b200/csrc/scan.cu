@@ -8,13 +8,11 @@
 //                         shapes).  One warp per group of 8 pages.
 //   scan_i4r8_kernel      the bytes-bound path for the r8i4 blob with bf16 queries.  Persistent warps,
 //                         each streaming groups of 8 blobs through its own shared-memory ring with bulk
-//                         async copies (TMA engine) and mbarriers, no CTA-wide synchronisation.  Per page:
-//                           MMA#1  P^T[heads x ranks]  = q[heads x d] . codesV[d x ranks]        (8 x m16n8k16 bf16)
-//                           MMA#2  L[heads x tokens]   = (P_hi | P_lo)[heads x 16] . codesC^T    (2 x m16n8k16 fp16)
-//                         and per 8 pages the centroid dots a[heads x pages] (16 x m16n8k16 bf16, the int8
-//                         centroid split into two exact nibbles).  Integer codes are exact in bf16/fp16, the
-//                         fp32 scales are applied to the fp32 accumulators, the projection is carried into
-//                         MMA#2 as an fp16 hi+lo pair (22 significant bits).
+//                         async copies (TMA engine) and mbarriers, no CTA-wide synchronisation.  Per page pair:
+//                           MMA#1  P[2 pages x 8 ranks, heads] = codesV[16 x d] . q^T[d x heads]   (8 x m16n8k16 fp16)
+//                         per page, after an 8x8 movmatrix transpose of the fp16 hi/lo projection:
+//                           MMA#2  L[heads, tokens] = (P_hi | P_lo)[heads x 16] . codesC^T          (2 x m16n8k16 fp16)
+//                         and per 8 pages the centroid dots a[heads, pages] (8 x m16n8k16 fp16).
 #include "locks_internal.cuh"
 
 namespace {
@@ -175,8 +173,8 @@ __device__ __forceinline__ float fast_lg2(float x) {
 // D = A * B with a zero accumulator (no register is spent on the zeros)
 __device__ __forceinline__ void mma_f16_z(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                           uint32_t b0, uint32_t b1) {
-  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
-               "{%10,%10,%10,%10};\n"
+  asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+      "{%10,%10,%10,%10};\n"
                : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
                : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "f"(0.f));
 }
@@ -185,14 +183,26 @@ struct Cursor {
   int prob, grp, nsc;
 };
 
-// NH = number of 8-row halves of the query tile in use (1: G <= 8, 2: G <= 16).
+__device__ __forceinline__ uint32_t movm_trans(uint32_t v) {
+  uint32_t d;
+  asm("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(v));
+  return d;
+}
+
+// NH = number of 8-head column tiles of the query in use (1: G <= 8, 2: G <= 16).
 //
-// Numerics.  The stored integer codes are exact in fp16: a nibble n sitting at mantissa bits 0-3 of
-// 0x6400 reads 1024 + n, at bits 4-7 it reads 1024 + 16 n; subtracting 1032 / 1152 leaves code and
-// 16 * code, and the factor 16 is undone exactly by holding the matching query elements divided by
-// 16.  A byte at bits 0-7 reads 1024 + u.  The query row is scaled by a power of two so that
-// max|q| < 0.5 and converted to fp16 (bf16's 8 significant bits fit; only elements below 2^-14 of
-// the row maximum can round, by at most 2^-25 of it), so every product is exact and sums are fp32.
+// Numerics.  Every stored code enters the tensor core exactly.
+//  * A basis nibble n = code + 8 masked in place is an fp16 SUBNORMAL: at bits 0-3 it reads
+//    n 2^-24, at bits 4-7 it reads 16 n 2^-24 (both below 1024, so the encoding is linear); the
+//    factor 16 is undone exactly by holding the matching query elements divided by 16, the common
+//    2^-24 by an exact power-of-two multiply of the fp32 accumulator, and the +8 offset by
+//    subtracting 8 sum_c q'[c] (one fp32 constant per head).
+//  * Coefficient and centroid bytes u = code + 128 are placed in the mantissa of 0x6400 (1024 + u)
+//    and the 1152 is subtracted in fp16, which is exact.
+//  * The query row is scaled by a power of two so that max|q| < 0.5 and converted to fp16 (bf16's
+//    8 significant bits fit; only elements below 2^-14 of the row maximum can round, by at most
+//    2^-25 of it).  Products are exact, sums are fp32; the projection is carried into the second
+//    MMA as an fp16 hi + lo pair (22 significant bits).
 template <int NH>
 __global__ void __launch_bounds__(kScanWarps * 32, 2) scan_i4r8_kernel(ScanParams p) {
   extern __shared__ __align__(128) uint8_t smem[];
@@ -226,13 +236,19 @@ __global__ void __launch_bounds__(kScanWarps * 32, 2) scan_i4r8_kernel(ScanParam
       if (c.prob < nprob) c.nsc = load_nsc(c.prob);
     }
   };
-  auto issue = [&](int stage, const Cursor &c) {
-    const int b = c.prob / p.Hkv, h = c.prob - b * p.Hkv;
+  // the physical block of page (grp*8 + lane) of the producer cursor, fetched one group ahead of use
+  auto fetch_block = [&](const Cursor &c) -> int {
+    if (c.prob >= nprob) return 0;
+    const int page = c.grp * LOCKS_GROUP + lane;
+    if (lane >= LOCKS_GROUP || page >= c.nsc) return 0;
+    return p.block_table[(int64_t)(c.prob / p.Hkv) * p.Pmax + page];
+  };
+  auto issue = [&](int stage, const Cursor &c, int block) {
+    const int h = c.prob % p.Hkv;
     const int nvalid = min(LOCKS_GROUP, c.nsc - c.grp * LOCKS_GROUP);
     if (lane == 0) mbar_expect_tx(&full[stage], (uint32_t)nvalid * kBlob);
     __syncwarp();
     if (lane < nvalid) {
-      int block = p.block_table[(int64_t)b * p.Pmax + c.grp * LOCKS_GROUP + lane];
       if (block < 0 || block >= p.num_blocks) {
         set_status(p.status, LOCKS_ERR_BAD_BLOCK);
         block = 0;
@@ -247,31 +263,33 @@ __global__ void __launch_bounds__(kScanWarps * 32, 2) scan_i4r8_kernel(ScanParam
   settle(cp);
   cc = cp;
   int inflight = 0;
+  int next_block = fetch_block(cp);
 #pragma unroll
   for (int s = 0; s < kScanStages; ++s) {
     if (cp.prob < nprob) {
-      issue(s, cp);
+      issue(s, cp, next_block);
       ++inflight;
       cp.grp += wpp;
       settle(cp);
+      next_block = fetch_block(cp);
     }
   }
 
-  // constants kept in registers so that every extraction is a single LOP3
-  uint32_t kM0 = 0x000F000Fu, kM1 = 0x00F000F0u, kMB = 0x00FF00FFu, kMagic = 0x64006400u;
-  asm volatile("" : "+r"(kM0), "+r"(kM1), "+r"(kMB), "+r"(kMagic));
-  const uint32_t kSub8 = 0x64086408u;      // 1032: 1024 + 8
-  const uint32_t kSub128 = 0x64806480u;    // 1152: 1024 + 128
+  const uint32_t kM0 = 0x000F000Fu, kM1 = 0x00F000F0u;
+  uint32_t kMB = 0x00FF00FFu, kMagic = 0x64006400u;
+  asm volatile("" : "+r"(kMB), "+r"(kMagic));
+  const uint32_t kSub128 = 0x64806480u;    // 1152 = 1024 + 128
   const uint32_t kSixteen = 0x4C004C00u;   // 16.0
-  const uint32_t kSub16x = 0x74807480u;    // 18432 = 16 * 1152
+  const uint32_t kNeg16x = 0xF480F480u;    // -18432 = -16 * 1152
 
-  uint32_t qa0[8], qa2[8], qa1[8], qa3[8];
-  float inv_s = 1.f, inv_s8 = 1.f;
+  // query of the current problem: qb0/qb2 = this lane's dims of head x (tile 0) / head x + 8 (tile 1)
+  uint32_t qb0[NH][8], qb2[NH][8];
+  float inv_s[NH], ksum[2 * NH];   // 1/scale of head x (+8); 8 * sum_c q'[c] of heads 2t, 2t+1 (+8)
   int cur_prob = -1;
   const __nv_bfloat16 *q = reinterpret_cast<const __nv_bfloat16 *>(p.q);
   const float c2 = p.sm_scale * kLog2e;
 
-  auto load_q_row = [&](int b, int hq, bool valid, uint32_t (&a0)[8], uint32_t (&a2)[8], float &inv) {
+  auto load_q_row = [&](int b, int hq, bool valid, uint32_t (&a0)[8], uint32_t (&a2)[8], float &inv, float &sum8) {
     uint4 v[4] = {};
     if (valid) {
       const uint4 *qp = reinterpret_cast<const uint4 *>(q + ((int64_t)b * p.Hq + hq) * LOCKS_D + 32 * t);
@@ -294,12 +312,21 @@ __global__ void __launch_bounds__(kScanWarps * 32, 2) scan_i4r8_kernel(ScanParam
     }
     inv = 1.f / s;
     const float s16 = s * 0.0625f;
+    float acc = 0.f;
 #pragma unroll
     for (int ks = 0; ks < 8; ++ks) {
       const uint32_t u0 = w[2 * ks], u1 = w[2 * ks + 1];
-      a0[ks] = pack_f16(__uint_as_float(u0 << 16) * s, __uint_as_float(u0 & 0xFFFF0000u) * s);
-      a2[ks] = pack_f16(__uint_as_float(u1 << 16) * s16, __uint_as_float(u1 & 0xFFFF0000u) * s16);
+      const uint32_t h0 = pack_f16(__uint_as_float(u0 << 16) * s, __uint_as_float(u0 & 0xFFFF0000u) * s);
+      const uint32_t h1 = pack_f16(__uint_as_float(u1 << 16) * s, __uint_as_float(u1 & 0xFFFF0000u) * s);
+      const float2 f0 = h2f2(h0), f1 = h2f2(h1);
+      acc += (f0.x + f0.y) + (f1.x + f1.y);     // sum of the fp16 values actually multiplied
+      a0[ks] = h0;
+      a2[ks] = pack_f16(f1.x * 0.0625f, f1.y * 0.0625f);
     }
+    (void)s16;
+    acc += __shfl_xor_sync(0xffffffffu, acc, 1);
+    acc += __shfl_xor_sync(0xffffffffu, acc, 2);
+    sum8 = 8.f * acc;
   };
 
   int it = 0;
@@ -315,16 +342,18 @@ __global__ void __launch_bounds__(kScanWarps * 32, 2) scan_i4r8_kernel(ScanParam
     const int b = cc.prob / p.Hkv, h = cc.prob - b * p.Hkv;
     if (cc.prob != cur_prob) {
       cur_prob = cc.prob;
-      load_q_row(b, h * p.G + x, x < p.G, qa0, qa2, inv_s);
-      if (NH == 2) load_q_row(b, h * p.G + x + 8, x + 8 < p.G, qa1, qa3, inv_s8);
-      else {
 #pragma unroll
-        for (int i = 0; i < 8; ++i) { qa1[i] = 0u; qa3[i] = 0u; }
+      for (int hh = 0; hh < NH; ++hh) {
+        float s8;
+        load_q_row(b, h * p.G + x + 8 * hh, x + 8 * hh < p.G, qb0[hh], qb2[hh], inv_s[hh], s8);
+        // lane (x, t) owns head x; the column fragment needs heads 2t, 2t+1
+        ksum[2 * hh] = __shfl_sync(0xffffffffu, s8, (2 * t) * 4);
+        ksum[2 * hh + 1] = __shfl_sync(0xffffffffu, s8, (2 * t + 1) * 4);
       }
     }
 
     const uint8_t *sb = ring + stage * kStageBytes;
-    // ---- centroid dots of the 8 pages: a[head][page] = sum_c code_mu[c] q'[c]
+    // ---- centroid dots of the 8 pages: cen[head x (+8)][pages 2t, 2t+1] = sum_c code_mu[c] q'[c]
     float cen[4] = {0.f, 0.f, 0.f, 0.f};
     {
       const uint4 *mp = reinterpret_cast<const uint4 *>(sb + x * kBlob + i4_off_mu(8) + t * 32);
@@ -333,20 +362,19 @@ __global__ void __launch_bounds__(kScanWarps * 32, 2) scan_i4r8_kernel(ScanParam
 #pragma unroll
       for (int s = 0; s < 8; ++s) {
         const uint32_t w = mw[s];
-        const uint32_t b0 = f16x2_sub(and_or(w, kMB, kMagic), kSub128);                // code
-        const uint32_t b1 = f16x2_fma(and_or(w >> 8, kMB, kMagic), kSixteen, kSub16x ^ 0x80008000u);  // 16 code
-        mma_f16(cen, qa0[s], qa1[s], qa2[s], qa3[s], b0, b1);
+        const uint32_t b0 = f16x2_sub(and_or(w, kMB, kMagic), kSub128);              // code
+        const uint32_t b1 = f16x2_fma(and_or(w >> 8, kMB, kMagic), kSixteen, kNeg16x);  // 16 * code
+        mma_f16(cen, qb0[0][s], NH == 2 ? qb0[NH - 1][s] : 0u, qb2[0][s], NH == 2 ? qb2[NH - 1][s] : 0u, b0, b1);
       }
     }
-    float acen[2 * NH];  // log2-domain centroid term for pages 2t, 2t+1 (and the second row half)
+    float acen[2 * NH];  // log2-domain centroid term of pages 2t, 2t+1 for head x (and x + 8)
     {
       const float s0 = __half2float(*reinterpret_cast<const __half *>(sb + (2 * t) * kBlob + i4_off_smu(8)));
       const float s1 = __half2float(*reinterpret_cast<const __half *>(sb + (2 * t + 1) * kBlob + i4_off_smu(8)));
-      acen[0] = s0 * (c2 * inv_s) * cen[0];
-      acen[1] = s1 * (c2 * inv_s) * cen[1];
-      if (NH == 2) {
-        acen[2] = s0 * (c2 * inv_s8) * cen[2];
-        acen[3] = s1 * (c2 * inv_s8) * cen[3];
+#pragma unroll
+      for (int hh = 0; hh < NH; ++hh) {
+        acen[2 * hh] = s0 * (c2 * inv_s[hh]) * cen[2 * hh];
+        acen[2 * hh + 1] = s1 * (c2 * inv_s[hh]) * cen[2 * hh + 1];
       }
     }
     float res[2 * NH];
@@ -354,68 +382,74 @@ __global__ void __launch_bounds__(kScanWarps * 32, 2) scan_i4r8_kernel(ScanParam
     for (int i = 0; i < 2 * NH; ++i) res[i] = 0.f;
 
 #pragma unroll
-    for (int pg = 0; pg < LOCKS_GROUP; ++pg) {
-      const uint8_t *pb = sb + pg * kBlob;
-      const uint4 w4 = *reinterpret_cast<const uint4 *>(pb + lane * 16);
-      const uint32_t ww[4] = {w4.x, w4.y, w4.z, w4.w};
-      float c1[4];
+    for (int pp = 0; pp < LOCKS_GROUP / 2; ++pp) {
+      const uint8_t *pbA = sb + (2 * pp) * kBlob, *pbB = pbA + kBlob;
+      // ---- MMA #1: rows = (page A ranks 0-7, page B ranks 0-7), cols = heads, k = this lane quarter's dims
+      const uint4 wa4 = *reinterpret_cast<const uint4 *>(pbA + lane * 16);
+      const uint4 wb4 = *reinterpret_cast<const uint4 *>(pbB + lane * 16);
+      const uint32_t wa[4] = {wa4.x, wa4.y, wa4.z, wa4.w}, wb[4] = {wb4.x, wb4.y, wb4.z, wb4.w};
+      float c1[NH][4];
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
-        const uint32_t w = ww[j], wh = w >> 8;
-        const uint32_t r0 = f16x2_sub(and_or(w, kM0, kMagic), kSub8);     // code          (k-step 2j, cols 2t..)
-        const uint32_t r1 = f16x2_sub(and_or(w, kM1, kMagic), kSub128);   // 16 * code     (k-step 2j, cols 8+2t..)
-        const uint32_t r2 = f16x2_sub(and_or(wh, kM0, kMagic), kSub8);    // k-step 2j+1
-        const uint32_t r3 = f16x2_sub(and_or(wh, kM1, kMagic), kSub128);
-        if (j == 0) mma_f16_z(c1, qa0[0], qa1[0], qa2[0], qa3[0], r0, r1);
-        else mma_f16(c1, qa0[2 * j], qa1[2 * j], qa2[2 * j], qa3[2 * j], r0, r1);
-        mma_f16(c1, qa0[2 * j + 1], qa1[2 * j + 1], qa2[2 * j + 1], qa3[2 * j + 1], r2, r3);
-      }
-      // projection (already carrying sm_scale * log2 e) -> fp16 hi + lo
-      const float2 sv = h2f2(*reinterpret_cast<const uint32_t *>(pb + i4_off_sv(8) + 4 * t));
-      const float svx = sv.x * c2, svy = sv.y * c2;
-      const float p0 = c1[0] * svx, p1 = c1[1] * svy;
-      const uint32_t hi = pack_f16(p0, p1);
-      const float2 hf = h2f2(hi);
-      const uint32_t lo = pack_f16(p0 - hf.x, p1 - hf.y);
-      uint32_t hi8 = 0u, lo8 = 0u;
-      if (NH == 2) {
-        const float p2 = c1[2] * svx, p3 = c1[3] * svy;
-        hi8 = pack_f16(p2, p3);
-        const float2 hf8 = h2f2(hi8);
-        lo8 = pack_f16(p2 - hf8.x, p3 - hf8.y);
-      }
-      // coefficient codes (offset-binary int8) -> exact fp16
-      const uint32_t cw = *reinterpret_cast<const uint32_t *>(pb + i4_off_coef(8) + lane * 4);
-      const uint32_t b0 = f16x2_sub(__byte_perm(cw, 0x64646464u, 0x4140), kSub128);
-      const uint32_t b1 = f16x2_sub(__byte_perm(cw, 0x64646464u, 0x4342), kSub128);
-      float ca[4], cb[4];
-      mma_f16_z(ca, hi, hi8, lo, lo8, b0, b0);
-      mma_f16_z(cb, hi, hi8, lo, lo8, b1, b1);
-      const uint2 scw = *reinterpret_cast<const uint2 *>(pb + i4_off_sc(8) + 8 * t);
-      const float2 s01 = h2f2(scw.x), s89 = h2f2(scw.y);
+        const uint32_t ua = wa[j], ub = wb[j], ua8 = ua >> 8, ub8 = ub >> 8;
 #pragma unroll
-      for (int hh = 0; hh < NH; ++hh) {
-        const float iv = hh ? inv_s8 : inv_s;
-        const float y0 = ca[2 * hh] * s01.x, y1 = ca[2 * hh + 1] * s01.y;
-        const float y2 = cb[2 * hh] * s89.x, y3 = cb[2 * hh + 1] * s89.y;
-        float my = fmaxf(fmaxf(y0, y1), fmaxf(y2, y3));
-        my = fmaxf(my, __shfl_xor_sync(0xffffffffu, my, 1));
-        my = fmaxf(my, __shfl_xor_sync(0xffffffffu, my, 2));
-        const float m = my * iv;   // logits are y * iv (iv > 0, a power of two)
-        float e = fast_ex2(fmaf(y0, iv, -m)) + fast_ex2(fmaf(y1, iv, -m)) + fast_ex2(fmaf(y2, iv, -m)) +
-                  fast_ex2(fmaf(y3, iv, -m));
-        e += __shfl_xor_sync(0xffffffffu, e, 1);
-        e += __shfl_xor_sync(0xffffffffu, e, 2);
-        const float v = m + fast_lg2(e);
-        if (t == (pg >> 1)) res[2 * hh + (pg & 1)] = v;
+        for (int hh = 0; hh < NH; ++hh) {
+          if (j == 0) mma_f16_z(c1[hh], ua & kM0, ub & kM0, ua & kM1, ub & kM1, qb0[hh][0], qb2[hh][0]);
+          else mma_f16(c1[hh], ua & kM0, ub & kM0, ua & kM1, ub & kM1, qb0[hh][2 * j], qb2[hh][2 * j]);
+          mma_f16(c1[hh], ua8 & kM0, ub8 & kM0, ua8 & kM1, ub8 & kM1, qb0[hh][2 * j + 1], qb2[hh][2 * j + 1]);
+        }
+      }
+#pragma unroll
+      for (int pq = 0; pq < 2; ++pq) {
+        const int pg = 2 * pp + pq;
+        const uint8_t *pb = pq ? pbB : pbA;
+        // projection of rank x for heads 2t, 2t+1: undo 2^-24, remove the +8 offset, apply the column scale
+        const float sv = __half2float(*reinterpret_cast<const __half *>(pb + i4_off_sv(8) + 2 * x));
+        uint32_t hiT[NH], loT[NH];
+#pragma unroll
+        for (int hh = 0; hh < NH; ++hh) {
+          const float p0 = fmaf(c1[hh][2 * pq], 16777216.f, -ksum[2 * hh]) * sv;
+          const float p1 = fmaf(c1[hh][2 * pq + 1], 16777216.f, -ksum[2 * hh + 1]) * sv;
+          const uint32_t hi = pack_f16(p0, p1);
+          const float2 hf = h2f2(hi);
+          const uint32_t lo = pack_f16(p0 - hf.x, p1 - hf.y);
+          hiT[hh] = movm_trans(hi);   // -> lane (x = head, t): ranks 2t, 2t+1
+          loT[hh] = movm_trans(lo);
+        }
+        // ---- MMA #2: rows = heads, k = ranks (hi | lo), cols = tokens
+        const uint32_t cw = *reinterpret_cast<const uint32_t *>(pb + i4_off_coef(8) + lane * 4);
+        const uint32_t b0 = f16x2_sub(__byte_perm(cw, 0x64646464u, 0x4140), kSub128);
+        const uint32_t b1 = f16x2_sub(__byte_perm(cw, 0x64646464u, 0x4342), kSub128);
+        float ca[4], cb[4];
+        mma_f16_z(ca, hiT[0], NH == 2 ? hiT[NH - 1] : 0u, loT[0], NH == 2 ? loT[NH - 1] : 0u, b0, b0);
+        mma_f16_z(cb, hiT[0], NH == 2 ? hiT[NH - 1] : 0u, loT[0], NH == 2 ? loT[NH - 1] : 0u, b1, b1);
+        const uint2 scw = *reinterpret_cast<const uint2 *>(pb + i4_off_sc(8) + 8 * t);
+        const float2 s01 = h2f2(scw.x), s89 = h2f2(scw.y);
+#pragma unroll
+        for (int hh = 0; hh < NH; ++hh) {
+          const float iv = inv_s[hh] * c2;   // logits (log2 domain) are y * iv, iv > 0
+          const float y0 = ca[2 * hh] * s01.x, y1 = ca[2 * hh + 1] * s01.y;
+          const float y2 = cb[2 * hh] * s89.x, y3 = cb[2 * hh + 1] * s89.y;
+          float my = fmaxf(fmaxf(y0, y1), fmaxf(y2, y3));
+          my = fmaxf(my, __shfl_xor_sync(0xffffffffu, my, 1));
+          my = fmaxf(my, __shfl_xor_sync(0xffffffffu, my, 2));
+          const float m = my * iv;
+          float e = fast_ex2(fmaf(y0, iv, -m)) + fast_ex2(fmaf(y1, iv, -m)) + fast_ex2(fmaf(y2, iv, -m)) +
+                    fast_ex2(fmaf(y3, iv, -m));
+          e += __shfl_xor_sync(0xffffffffu, e, 1);
+          e += __shfl_xor_sync(0xffffffffu, e, 2);
+          const float v = m + fast_lg2(e);
+          if (t == (pg >> 1)) res[2 * hh + (pg & 1)] = v;
+        }
       }
     }
     __syncwarp();  // every lane is done reading this stage
     if (cp.prob < nprob) {
-      issue(stage, cp);
+      issue(stage, cp, next_block);
       ++inflight;
       cp.grp += wpp;
       settle(cp);
+      next_block = fetch_block(cp);
     }
 
     // ---- write s^ and the group's candidate partial

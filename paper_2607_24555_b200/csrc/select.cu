@@ -31,9 +31,14 @@ __device__ __forceinline__ uint32_t order_key(float f) {
 // Exact top-K among the block's N = THREADS*EPT keys (thread-major order = ascending index order).
 // sel[i] is set for the K winners: every key above the K-th largest, plus the lowest-indexed keys
 // equal to it.  pos[i] = rank of a winner in index order.  Requires K <= number of valid keys.
+// Four 8-bit radix passes.  Every warp counts into its own 256-bin histogram (page masses share their
+// leading bits, so a shared histogram would serialise all warps on one or two counters); bin b of
+// the block is then summed and suffix-scanned by thread b.
+// sh_hist: warps x 256 ints (zero on entry and on exit), sh_misc: 12 ints.
 template <int EPT>
 __device__ void block_topk(const uint32_t (&key)[EPT], int K, bool (&sel)[EPT], int (&pos)[EPT], int *sh_hist,
                            int *sh_misc) {
+  constexpr int NW = LOCKS_SEL_THREADS / 32;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   if (K <= 0) {  // nothing to pick (k = 2): uniform across the block
 #pragma unroll
@@ -44,40 +49,37 @@ __device__ void block_topk(const uint32_t (&key)[EPT], int K, bool (&sel)[EPT], 
   int remaining = K;
   for (int pass = 0; pass < 4; ++pass) {
     const int shift = 24 - 8 * pass;
-    if (tid < 256) sh_hist[tid] = 0;
-    __syncthreads();
+    int *mine = sh_hist + warp * 256;
 #pragma unroll
     for (int i = 0; i < EPT; ++i)
-      if ((key[i] & mask) == prefix) atomicAdd(&sh_hist[(key[i] >> shift) & 255], 1);
+      if ((key[i] & mask) == prefix) atomicAdd(&mine[(key[i] >> shift) & 255], 1);
     __syncthreads();
-    if (warp == 0) {
-      // bins high -> low: lane owns bins 255-8*lane .. 248-8*lane
-      int c[8], tot = 0;
+    int c = 0, incl = 0;
+    if (tid < 256) {   // thread b owns bin 255 - b: bins are scanned from the largest digit down
+      const int bin = 255 - tid;
 #pragma unroll
-      for (int u = 0; u < 8; ++u) { c[u] = sh_hist[255 - (lane * 8 + u)]; tot += c[u]; }
-      int incl = tot;
+      for (int w = 0; w < NW; ++w) { c += sh_hist[w * 256 + bin]; sh_hist[w * 256 + bin] = 0; }
+      incl = c;
 #pragma unroll
       for (int o = 1; o < 32; o <<= 1) {
         int v = __shfl_up_sync(0xffffffffu, incl, o);
         if (lane >= o) incl += v;
       }
-      int before = incl - tot;  // keys in strictly higher bins than this lane's
-      if (before < remaining && remaining <= incl) {
-#pragma unroll
-        for (int u = 0; u < 8; ++u) {
-          if (before < remaining && remaining <= before + c[u]) {
-            sh_misc[0] = 255 - (lane * 8 + u);
-            sh_misc[1] = remaining - before;
-          }
-          before += c[u];
-        }
+      if (lane == 31) sh_misc[4 + warp] = incl;
+    }
+    __syncthreads();
+    if (tid < 256) {
+      int before = incl - c;
+      for (int w = 0; w < warp; ++w) before += sh_misc[4 + w];
+      if (before < remaining && remaining <= before + c) {
+        sh_misc[(pass & 1) * 2] = 255 - tid;
+        sh_misc[(pass & 1) * 2 + 1] = remaining - before;
       }
     }
     __syncthreads();
-    prefix |= (uint32_t)sh_misc[0] << shift;
+    prefix |= (uint32_t)sh_misc[(pass & 1) * 2] << shift;
     mask |= 255u << shift;
-    remaining = sh_misc[1];
-    __syncthreads();
+    remaining = sh_misc[(pass & 1) * 2 + 1];
   }
   // prefix is the K-th largest key; `remaining` of the keys equal to it are taken, lowest index first
   int ngt = 0, neq = 0;
@@ -91,10 +93,11 @@ __device__ void block_topk(const uint32_t (&key)[EPT], int K, bool (&sel)[EPT], 
     int v = __shfl_up_sync(0xffffffffu, incl, o);
     if (lane >= o) incl += v;
   }
-  if (lane == 31) sh_misc[2 + warp] = incl;
+  __syncthreads();   // the last pass's readers of sh_misc[4..] are done
+  if (lane == 31) sh_misc[12 + warp] = incl;
   __syncthreads();
   int base = 0;
-  for (int w = 0; w < warp; ++w) base += sh_misc[2 + w];
+  for (int w = 0; w < warp; ++w) base += sh_misc[12 + w];
   int excl = base + incl - packed;
   int gt_before = excl >> 16, eq_before = excl & 0xffff;
 #pragma unroll
@@ -106,7 +109,6 @@ __device__ void block_topk(const uint32_t (&key)[EPT], int K, bool (&sel)[EPT], 
     gt_before += gt;
     eq_before += eq;
   }
-  __syncthreads();
 }
 
 // log Z_g of every head of the group from the scan's per-group partials -> sh_logz[g]
@@ -138,9 +140,10 @@ __device__ void group_logz(const SelParams &p, int b, int h, int ngroups, float 
 
 template <int EPT>
 __global__ void __launch_bounds__(LOCKS_SEL_THREADS) select_stage1_kernel(SelParams p) {
-  __shared__ int sh_hist[256];
-  __shared__ int sh_misc[2 + LOCKS_SEL_THREADS / 32];
+  __shared__ int sh_hist[(LOCKS_SEL_THREADS / 32) * 256];
+  __shared__ int sh_misc[12 + LOCKS_SEL_THREADS / 32];
   __shared__ float sh_logz[16];
+  for (int e = threadIdx.x; e < (LOCKS_SEL_THREADS / 32) * 256; e += LOCKS_SEL_THREADS) sh_hist[e] = 0;
   const int chunk = blockIdx.x, h = blockIdx.y, b = blockIdx.z, tid = threadIdx.x;
   const int T = p.seq_lens[b];
   const int P = (T + LOCKS_B - 1) / LOCKS_B;
@@ -162,19 +165,45 @@ __global__ void __launch_bounds__(LOCKS_SEL_THREADS) select_stage1_kernel(SelPar
       }
     return;
   }
+  // scores of the first heads are fetched before the log Z reduction so that the two latencies overlap
+  constexpr int PRE = EPT <= 8 ? 4 : 1;
+  const int pbase = c0 + tid * EPT;
+  const float *row0 = p.shat + ((int64_t)b * p.Hq + h * p.G) * p.Pmax;
+  float raw[PRE][EPT];
+#pragma unroll
+  for (int g = 0; g < PRE; ++g)
+#pragma unroll
+    for (int i = 0; i < EPT; ++i) {
+      const int page = pbase + i;
+      raw[g][i] = (g < p.G && page >= 1 && page <= P - 2) ? row0[(int64_t)g * p.Pmax + page] : 0.f;
+    }
   group_logz(p, b, h, (P - 1 + LOCKS_GROUP - 1) / LOCKS_GROUP, sh_logz);
   __syncthreads();
   // log m_bar of this thread's EPT consecutive pages: log mean_g exp(s^_g - log Z_g)
   float val[EPT];
   uint32_t key[EPT];
-  const int pbase = c0 + tid * EPT;
   const float logG = __logf((float)p.G);
   {
     float mx[EPT], sm[EPT];
 #pragma unroll
     for (int i = 0; i < EPT; ++i) { mx[i] = -INFINITY; sm[i] = 0.f; }
-    const float *row0 = p.shat + ((int64_t)b * p.Hq + h * p.G) * p.Pmax;
-    for (int g = 0; g < p.G; ++g) {
+#pragma unroll
+    for (int g = 0; g < PRE; ++g) {
+      if (g < p.G) {
+        const float lz = sh_logz[g];
+#pragma unroll
+        for (int i = 0; i < EPT; ++i) {
+          const int page = pbase + i;
+          if (page >= 1 && page <= P - 2) {
+            const float tv = raw[g][i] - lz;
+            const float nm = fmaxf(mx[i], tv);
+            sm[i] = sm[i] * __expf(mx[i] - nm) + __expf(tv - nm);
+            mx[i] = nm;
+          }
+        }
+      }
+    }
+    for (int g = PRE; g < p.G; ++g) {
       const float *row = row0 + (int64_t)g * p.Pmax;
       const float lz = sh_logz[g];
 #pragma unroll
@@ -223,9 +252,11 @@ __global__ void __launch_bounds__(LOCKS_SEL_THREADS) select_stage1_kernel(SelPar
 
 template <int EPT>
 __global__ void __launch_bounds__(LOCKS_SEL_THREADS) select_stage2_kernel(SelParams p) {
-  __shared__ int sh_hist[256];
-  __shared__ int sh_misc[2 + LOCKS_SEL_THREADS / 32];
+  __shared__ int sh_hist[(LOCKS_SEL_THREADS / 32) * 256];
+  __shared__ int sh_misc[12 + LOCKS_SEL_THREADS / 32];
   const int h = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
+  for (int e = tid; e < (LOCKS_SEL_THREADS / 32) * 256; e += LOCKS_SEL_THREADS) sh_hist[e] = 0;
+  __syncthreads();
   const int T = p.seq_lens[b];
   const int P = (T + LOCKS_B - 1) / LOCKS_B;
   if (P <= p.k) return;  // stage 1 already wrote the table
