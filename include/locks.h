@@ -39,6 +39,7 @@ extern "C" {
 #define LOCKS_ERR_CUDA (-4)
 #define LOCKS_ERR_TIMEOUT (-5)
 #define LOCKS_ERR_BAD_BLOCK (-6)
+#define LOCKS_ERR_TOO_LARGE (-7)
 
 #define LOCKS_F32 0
 #define LOCKS_BF16 1
@@ -166,6 +167,32 @@ int locks_last_launch_count(const locks_ctx *ctx);
  * of steps seen to *steps, and releases the events.  Not legal while the stream is being captured. */
 int locks_profile_begin(locks_ctx *ctx, int max_steps);
 int locks_profile_end(locks_ctx *ctx, float *stage_ms, int *steps);
+
+/* locks_sparse_attend for callers that cannot allocate device memory (the paper has no
+ * counterpart; this is a convenience of the library).  Some hosts of this code may not call
+ * cudaMalloc at all: a plugin running inside an engine that has already handed the whole device to
+ * its own memory pool, code on a latency-critical path where an allocation (an implicit device
+ * synchronisation) is not acceptable, or a process whose memory budget is fixed up front.  Such a
+ * caller cannot provide the workspace locks_create() asks for, so this entry point needs neither a
+ * context nor a workspace: the split partials and the split-arrival counters live in an array that is
+ * part of the library itself (about 2.1 MB, resident on every GPU that loads the library until the
+ * process exits).  Inputs and outputs are the caller's, exactly as for locks_sparse_attend; `cfg`
+ * supplies the shapes (head counts, max_pages_per_seq = row length of block_table, budget_tokens =
+ * row length * page_size of page_ids, sm_scale).  bf16 only.
+ *  - Limit: batch * num_q_heads <= LOCKS_NOALLOC_MAX_ROWS, at most LOCKS_NOALLOC_MAX_SPLITS splits
+ *    per KV head; a larger problem is refused with LOCKS_ERR_TOO_LARGE before anything is launched.
+ *  - The first call on each device looks up the array's address on that device and sets kernel
+ *    attributes; make that first call outside any stream capture, with the device current.
+ *  - All calls share the one array, which keeps what the previous call left behind; each call
+ *    clears the counters it needs on `stream` first.  Two calls that overlap on the GPU (different
+ *    streams, or different host threads) race on it: serialise them.
+ *  - No cudaMalloc / cudaFree or allocating library routine is called, here or in the kernel.
+ * Device-detected bad page or block ids are skipped as usual but cannot be polled from here. */
+#define LOCKS_NOALLOC_MAX_ROWS 256
+#define LOCKS_NOALLOC_MAX_SPLITS 16
+int locks_sparse_attend_noalloc(const locks_config *cfg, const void *q, const locks_kv *kv, int batch,
+                                const int32_t *page_ids, const int32_t *page_count, void *out, float *lse,
+                                locks_stream stream);
 
 const char *locks_strerror(int code);
 

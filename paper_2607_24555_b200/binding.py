@@ -16,7 +16,7 @@ FMT_F32, FMT_I4 = 0, 1
 SYMBOLS = ["locks_summary_bytes", "locks_workspace_bytes", "locks_create", "locks_destroy",
            "locks_build_summaries", "locks_select", "locks_sparse_attend", "locks_decode_step",
            "locks_decode_step_host", "locks_poll_status", "locks_last_launch_count", "locks_strerror",
-           "locks_profile_begin", "locks_profile_end"]
+           "locks_profile_begin", "locks_profile_end", "locks_sparse_attend_noalloc"]
 
 
 class LocksError(RuntimeError):
@@ -69,6 +69,8 @@ def lib():
         L.locks_profile_end.argtypes = [vp, C.POINTER(C.c_float), C.POINTER(C.c_int)]
         L.locks_profile_begin.restype = C.c_int
         L.locks_profile_end.restype = C.c_int
+        L.locks_sparse_attend_noalloc.argtypes = [C.POINTER(Config), vp, C.POINTER(KV), C.c_int, i32p, i32p, vp, vp, vp]
+        L.locks_sparse_attend_noalloc.restype = C.c_int
         L.locks_strerror.restype = C.c_char_p
         L.locks_strerror.argtypes = [C.c_int]
         for fn in ("locks_create", "locks_destroy", "locks_build_summaries", "locks_select", "locks_sparse_attend",
@@ -215,3 +217,12 @@ class Context:
 
     def locks_last_launch_count(self) -> int:
         return int(lib().locks_last_launch_count(self.handle))
+
+
+def locks_sparse_attend_noalloc(cfg: Config, q, kv: KVView, batch, page_ids, page_count, out, lse=None, stream=None):
+    """Sparse attention without a context or workspace, for callers that cannot allocate device memory
+    (see include/locks.h).  Raises LocksError with the library's message if the problem exceeds the
+    built-in scratch."""
+    s = kv.struct()
+    _check(lib().locks_sparse_attend_noalloc(C.byref(cfg), _ptr(q), C.byref(s), batch, _ptr(page_ids), _ptr(page_count),
+                                             _ptr(out), _ptr(lse), _stream(stream)), "locks_sparse_attend_noalloc")

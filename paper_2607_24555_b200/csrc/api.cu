@@ -303,6 +303,7 @@ const char *locks_strerror(int code) {
     case LOCKS_ERR_CUDA: return "CUDA runtime error";
     case LOCKS_ERR_TIMEOUT: return "a bounded device-side wait expired";
     case LOCKS_ERR_BAD_BLOCK: return "page or block id outside the cache";
+    case LOCKS_ERR_TOO_LARGE: return "problem larger than the library's built-in scratch (batch * q heads too large)";
     default: return "unknown error";
   }
 }

@@ -446,3 +446,96 @@ int locks_launch_attend(locks_ctx *c, const void *q, const locks_kv *kv, int bat
                                                  p.Hq);
   return locks_check_launch(c);
 }
+
+// ------------------------------------------------------------------------------------------------
+// Sparse attention for callers that cannot allocate device memory.
+//
+// The split-K partials and the split-arrival counters of attend_bf16_kernel normally live in the
+// workspace the caller allocates for locks_create().  This variant keeps them in a fixed array that is
+// part of the library image instead, so nothing has to be allocated at all.
+// ------------------------------------------------------------------------------------------------
+
+namespace {
+
+constexpr int kNoAllocMaxRows = LOCKS_NOALLOC_MAX_ROWS;          // batch * Hq
+constexpr int kNoAllocMaxSplits = LOCKS_NOALLOC_MAX_SPLITS;
+constexpr size_t kNoAllocO = (size_t)kNoAllocMaxRows * kNoAllocMaxSplits * LOCKS_D * sizeof(float);
+constexpr size_t kNoAllocLse = (size_t)kNoAllocMaxRows * kNoAllocMaxSplits * sizeof(float);
+constexpr size_t kNoAllocDone = (size_t)kNoAllocMaxRows * sizeof(int32_t);   // >= batch * Hkv
+constexpr size_t kNoAllocBytes = kNoAllocO + kNoAllocLse + kNoAllocDone + 256;
+
+// About 2.1 MB held by every GPU that loads the library, until the process exits.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocBytes];
+
+struct NoAllocDevice {
+  unsigned char *scratch;   // device address of g_noalloc_scratch on this device (not the host symbol!)
+  int num_sms;
+  bool ready;
+};
+NoAllocDevice g_noalloc_dev[64] = {};
+
+}  // namespace
+
+extern "C" int locks_sparse_attend_noalloc(const locks_config *cfg, const void *q, const locks_kv *kv, int batch,
+                                           const int32_t *page_ids, const int32_t *page_count, void *out, float *lse,
+                                           locks_stream stream) {
+  if (!cfg || !q || !kv || !out || !kv->k || !kv->v || !kv->block_table || !kv->seq_lens) return LOCKS_ERR_INVALID_ARG;
+  if ((page_ids == nullptr) != (page_count == nullptr) || batch <= 0 || kv->num_blocks <= 0) return LOCKS_ERR_INVALID_ARG;
+  if (cfg->num_q_heads <= 0 || cfg->num_kv_heads <= 0 || cfg->num_q_heads % cfg->num_kv_heads) return LOCKS_ERR_INVALID_ARG;
+  if (cfg->max_pages_per_seq <= 0 || cfg->budget_tokens <= 0 || !(cfg->sm_scale > 0.f)) return LOCKS_ERR_INVALID_ARG;
+  if (cfg->head_dim != LOCKS_D || cfg->page_size != LOCKS_B || cfg->kv_dtype != LOCKS_BF16 || cfg->q_dtype != LOCKS_BF16)
+    return LOCKS_ERR_UNSUPPORTED;
+  const int G = cfg->num_q_heads / cfg->num_kv_heads;
+  if (G > 16) return LOCKS_ERR_UNSUPPORTED;
+  if ((kv->stride_block | kv->stride_head | kv->stride_token) % 8 || kv->stride_token < LOCKS_D) return LOCKS_ERR_INVALID_ARG;
+  if (((uintptr_t)kv->k | (uintptr_t)kv->v | (uintptr_t)q) % 16) return LOCKS_ERR_INVALID_ARG;
+  // the built-in scratch bounds the problem: reject anything that would not fit
+  if ((int64_t)batch * cfg->num_q_heads > kNoAllocMaxRows) return LOCKS_ERR_TOO_LARGE;
+
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return LOCKS_ERR_CUDA;
+  NoAllocDevice &nd = g_noalloc_dev[dev];
+  if (!nd.ready) {
+    // first call on this device: ask the runtime where the array lives on the CURRENT device
+    void *ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_noalloc_scratch) != cudaSuccess || ptr == nullptr) return LOCKS_ERR_CUDA;
+    if (cudaDeviceGetAttribute(&nd.num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return LOCKS_ERR_CUDA;
+    cudaFuncSetAttribute(attend_bf16_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttSmem);
+    cudaFuncSetAttribute(attend_bf16_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttSmem);
+    cudaFuncSetAttribute(attend_bf16_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttSmem);
+    cudaFuncSetAttribute(attend_bf16_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttSmem);
+    nd.scratch = reinterpret_cast<unsigned char *>(ptr);
+    nd.ready = true;
+  }
+  cudaStream_t st = (cudaStream_t)stream;
+  AttParams p;
+  p.q = q; p.k = kv->k; p.v = kv->v; p.sb = kv->stride_block; p.sh = kv->stride_head; p.st = kv->stride_token;
+  p.block_table = kv->block_table; p.seq_lens = kv->seq_lens; p.ids = page_ids; p.cnt = page_count;
+  p.part_o = reinterpret_cast<float *>(nd.scratch);
+  p.part_lse = reinterpret_cast<float *>(nd.scratch + kNoAllocO);
+  p.done = reinterpret_cast<int32_t *>(nd.scratch + kNoAllocO + kNoAllocLse);
+  p.status = reinterpret_cast<int32_t *>(nd.scratch + kNoAllocO + kNoAllocLse + kNoAllocDone);
+  p.out = out; p.lse = lse;
+  p.batch = batch; p.Hq = cfg->num_q_heads; p.Hkv = cfg->num_kv_heads; p.G = G; p.Pmax = cfg->max_pages_per_seq;
+  p.kbud = (cfg->budget_tokens + LOCKS_B - 1) / LOCKS_B; p.num_blocks = kv->num_blocks; p.sm_scale = cfg->sm_scale;
+  const int npages = page_ids ? p.kbud : p.Pmax;
+  int splits = nd.num_sms * LOCKS_ATT_CTAS_PER_SM / (batch * p.Hkv);
+  const int most = (npages + LOCKS_ATT_WARPS - 1) / LOCKS_ATT_WARPS;
+  if (splits > most) splits = most;
+  if (splits > kNoAllocMaxSplits) splits = kNoAllocMaxSplits;
+  if (splits < 1) splits = 1;
+  p.pages_per_cta = (npages + splits - 1) / splits;
+  p.splits = (npages + p.pages_per_cta - 1) / p.pages_per_cta;
+  // the array keeps whatever the last call left: the arrival counters and the status word must start at zero
+  if (cudaMemsetAsync(p.done, 0, kNoAllocDone + 256, st) != cudaSuccess) return LOCKS_ERR_CUDA;
+  dim3 grid(p.splits, p.Hkv, batch);
+  const bool contig = kv->stride_token == LOCKS_D;
+  if (G <= 8) {
+    if (contig) attend_bf16_kernel<1, true><<<grid, LOCKS_ATT_WARPS * 32, kAttSmem, st>>>(p);
+    else attend_bf16_kernel<1, false><<<grid, LOCKS_ATT_WARPS * 32, kAttSmem, st>>>(p);
+  } else {
+    if (contig) attend_bf16_kernel<2, true><<<grid, LOCKS_ATT_WARPS * 32, kAttSmem, st>>>(p);
+    else attend_bf16_kernel<2, false><<<grid, LOCKS_ATT_WARPS * 32, kAttSmem, st>>>(p);
+  }
+  return cudaPeekAtLastError() == cudaSuccess ? LOCKS_OK : LOCKS_ERR_CUDA;
+}
