@@ -41,8 +41,13 @@ def workload(name: str):
         return locks_synth.config3(T=1 << 20)
     if name == "cfg3_128k":
         return locks_synth.config3(T=1 << 17)
-    if name == "cfg2_r8_b1024":
-        return locks_synth.config2(rank=8, budget=1024)
+    if name.startswith("cfg2_"):          # cfg2_r8_b1024, cfg2_r2_b256, ...
+        _, r, b = name.split("_")
+        return locks_synth.config2(rank=int(r[1:]), budget=int(b[1:]))
+    if name == "cfg3_512k":
+        return locks_synth.config3(T=1 << 19)
+    if name.startswith("cfg4_b"):
+        return locks_synth.config4(batch=int(name[6:]))
     if name == "small":
         return locks_synth.Workload("small", [4096] * 2, Hq=8, Hkv=2, budget=256)
     raise SystemExit(f"unknown workload {name}")
@@ -201,7 +206,8 @@ def run_ours(args):
     # every rank owns a full batch (weak scaling): requests are independent, no data-path collective
     layers = []
     for li in range(L):
-        w = w0.with_(seed=w0.seed * 1000 + 17 * li + 101 * rank, seq_lens=[t + reserve * w0.B for t in w0.seq_lens])
+        w = w0.with_(seed=w0.seed * 1000 + 17 * li + 101 * rank, seq_lens=[t + reserve * w0.B for t in w0.seq_lens],
+                     permute_blocks=not args.identity_blocks)
         case = locks_synth.make_case(w, device=dev)
         case.seq_lens.copy_(torch.tensor(w0.seq_lens, dtype=torch.int32, device=dev))
         layers.append(case)
@@ -312,6 +318,7 @@ def run_ours(args):
         "config": {"workload": w0.name, "batch_per_gpu": w0.n, "context": w0.seq_lens[0], "q_heads": w0.Hq,
                    "kv_heads": w0.Hkv, "head_dim": w0.d, "page": w0.B, "rank": w0.rank, "budget_tokens": w0.budget,
                    "summary": "r8i4" if w0.fmt == "i4" else "f32", "launch": "one CUDA graph per step",
+                   "block_mapping": "identity" if args.identity_blocks else "seeded random permutation",
                    "l2": f"inputs larger than L2: replays cycle over {L} independent layers "
                          f"({(scan_b + att_b) / 1e6:.0f} MB touched per step, L2 126 MB)"},
         "e2e": {"value": e2e_ms_max * 1e3, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
@@ -343,6 +350,8 @@ def main():
     ap.add_argument("--workload", default="cfg1")
     ap.add_argument("--layers", type=int, default=4)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--identity-blocks", action="store_true",
+                    help="logical page i of a request sits in consecutive physical blocks (default: seeded permutation)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

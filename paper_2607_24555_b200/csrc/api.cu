@@ -31,7 +31,7 @@ int validate(const locks_config *c) {
 }
 
 struct Layout {
-  size_t status, shat, part, cand_val, cand_idx, att_o, att_lse, att_done, ids, cnt, sq, skn, svn, sout, total;
+  size_t status, shat, part, logz, cand_val, cand_idx, att_o, att_lse, att_done, ids, cnt, sq, skn, svn, sout, total;
   int G, k, S, max_groups, sel_ept, sel_chunks, sel_kc;
 };
 
@@ -41,8 +41,13 @@ Layout make_layout(const locks_config *c) {
   L.k = (c->budget_tokens + c->page_size - 1) / c->page_size;
   L.S = c->summary_fmt == LOCKS_FMT_I4 ? i4_stride(c->rank) : f32_stride(c->rank);
   L.max_groups = (c->max_pages_per_seq + LOCKS_GROUP - 1) / LOCKS_GROUP;
-  const int per_thread = (c->max_pages_per_seq + LOCKS_SEL_THREADS - 1) / LOCKS_SEL_THREADS;
-  L.sel_ept = per_thread <= 4 ? 4 : (per_thread <= 8 ? 8 : 16);
+  // pages per thread in stage 1: the smallest of 4 / 8 / 16 whose per-chunk candidate lists still fit
+  // stage 2 (16 candidates per thread), so that long contexts are ranked by many CTAs
+  L.sel_ept = 16;
+  for (int ept = 4; ept <= 16; ept *= 2) {
+    const int chunks = (c->max_pages_per_seq + ept * LOCKS_SEL_THREADS - 1) / (ept * LOCKS_SEL_THREADS);
+    if (chunks == 1 || (size_t)chunks * (L.k - 2 > 0 ? L.k - 2 : 1) <= 16 * LOCKS_SEL_THREADS) { L.sel_ept = ept; break; }
+  }
   L.sel_chunks = (c->max_pages_per_seq + L.sel_ept * LOCKS_SEL_THREADS - 1) / (L.sel_ept * LOCKS_SEL_THREADS);
   L.sel_kc = L.k - 2 > 0 ? L.k - 2 : 1;
   const size_t nb = c->max_batch, Hq = c->num_q_heads, Hkv = c->num_kv_heads, P = c->max_pages_per_seq;
@@ -52,10 +57,13 @@ Layout make_layout(const locks_config *c) {
   L.status = take(64);
   L.shat = take(nb * Hq * P * 4);
   L.part = take(nb * Hq * L.max_groups * 8);
+  L.logz = take(nb * Hq * 4);
   L.cand_val = take(nb * Hkv * L.sel_chunks * L.sel_kc * 4);
   L.cand_idx = take(nb * Hkv * L.sel_chunks * L.sel_kc * 4);
-  L.att_o = take(nb * Hq * LOCKS_ATT_MAX_SPLITS * LOCKS_D * 4);
-  L.att_lse = take(nb * Hq * LOCKS_ATT_MAX_SPLITS * 4);
+  // split-K partial rows: batch * Hq * splits with splits <= slots / (batch * Hkv) (+1 rounding) and <= 128
+  const size_t att_rows = (size_t)L.G * LOCKS_ATT_SLOT_BOUND + 2 * nb * Hq;
+  L.att_o = take(att_rows * LOCKS_D * 4);
+  L.att_lse = take(att_rows * 4);
   L.att_done = take(nb * Hkv * 4);
   L.ids = take(nb * Hkv * L.k * 4);
   L.cnt = take(nb * Hkv * 4);
@@ -116,6 +124,7 @@ int locks_create(const locks_config *cfg, void *workspace, size_t ws_bytes, lock
   c->status = reinterpret_cast<int32_t *>(ws + L.status);
   c->shat = reinterpret_cast<float *>(ws + L.shat);
   c->part = reinterpret_cast<float2 *>(ws + L.part);
+  c->logz = reinterpret_cast<float *>(ws + L.logz);
   c->cand_val = reinterpret_cast<float *>(ws + L.cand_val);
   c->cand_idx = reinterpret_cast<int32_t *>(ws + L.cand_idx);
   c->att_o = reinterpret_cast<float *>(ws + L.att_o);
@@ -202,12 +211,13 @@ int locks_decode_step(locks_ctx *ctx, const void *q, const void *k_new, const vo
   mark(0);
   if ((rc = locks_launch_prep(ctx, q, k_new, v_new, kv, batch, st)) != LOCKS_OK) return rc;
   mark(1);
-  // the freshly completed page (if any) is summarised beside select + attend: it is read by neither
+  if ((rc = locks_launch_scan(ctx, q, summaries, kv, batch, ctx->shat, st)) != LOCKS_OK) return rc;
+  // the freshly completed page (if any) is summarised beside select + attend, which read neither it nor its
+  // summary.  The fork sits after the scan launch so that prologue -> scan stays a programmatic edge.
   if (cudaEventRecord(ctx->ev_fork, st) != cudaSuccess || cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0) != cudaSuccess)
     return LOCKS_ERR_CUDA;
   if ((rc = locks_launch_build(ctx, kv, batch, nullptr, nullptr, 1, summaries, ctx->side)) != LOCKS_OK) return rc;
   if (cudaEventRecord(ctx->ev_join, ctx->side) != cudaSuccess) return LOCKS_ERR_CUDA;
-  if ((rc = locks_launch_scan(ctx, q, summaries, kv, batch, ctx->shat, st)) != LOCKS_OK) return rc;
   mark(2);
   if ((rc = locks_launch_select(ctx, ctx->shat, kv, batch, ids, cnt, nullptr, st)) != LOCKS_OK) return rc;
   mark(3);

@@ -37,7 +37,8 @@ __device__ __forceinline__ float ex2f(float x) {
 
 constexpr int kTile = LOCKS_B * LOCKS_D * 2;                 // 4096 B: one K or V page tile in bf16
 constexpr int kAttStage = 2 * kTile;                         // K + V
-constexpr int kAttSmem = LOCKS_ATT_WARPS * 2 * kAttStage;    // two stages per warp
+constexpr int kAttStages = LOCKS_ATT_STAGES;                  // ring depth per warp
+constexpr int kAttSmem = LOCKS_ATT_WARPS * kAttStages * kAttStage;
 
 // Resolve the idx-th page of this problem's list: logical page, physical block, valid tokens.
 __device__ __forceinline__ bool resolve_page(const AttParams &p, int b, int64_t prob, int idx, int T, int &block,
@@ -68,14 +69,10 @@ __global__ void __launch_bounds__(LOCKS_ATT_WARPS * 32) attend_bf16_kernel(AttPa
   const int x = lane >> 2, t = lane & 3;
   const int split = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
   const int64_t prob = (int64_t)b * p.Hkv + h;
-  const int T = p.seq_lens[b];
-  const int P = (T + LOCKS_B - 1) / LOCKS_B;
-  const int npages = p.ids ? p.cnt[prob] : P;
-  const int lo = split * p.pages_per_cta;
-  const int hi = min(lo + p.pages_per_cta, npages);
-  uint8_t *ring = smem + warp * 2 * kAttStage;
+  uint8_t *ring = smem + warp * kAttStages * kAttStage;
   const uint8_t *Kb = reinterpret_cast<const uint8_t *>(p.k);
   const uint8_t *Vb = reinterpret_cast<const uint8_t *>(p.v);
+  pdl_trigger();
 
   // query as the B operand: lane (x, t) holds head x (+8), dims 16 s + 2t.. and 16 s + 8 + 2t..
   uint32_t qb[NH][8][2];
@@ -93,6 +90,12 @@ __global__ void __launch_bounds__(LOCKS_ATT_WARPS * 32) attend_bf16_kernel(AttPa
     }
   }
   const float c2 = p.sm_scale * kLog2e;
+  pdl_wait();   // page table from the selector, appended K/V rows, sequence lengths
+  const int T = p.seq_lens[b];
+  const int P = (T + LOCKS_B - 1) / LOCKS_B;
+  const int npages = p.ids ? p.cnt[prob] : P;
+  const int lo = split * p.pages_per_cta;
+  const int hi = min(lo + p.pages_per_cta, npages);
 
   float oacc[8][NH][4];
 #pragma unroll
@@ -145,18 +148,30 @@ __global__ void __launch_bounds__(LOCKS_ATT_WARPS * 32) attend_bf16_kernel(AttPa
     return ntok;
   };
 
-  int ntok_cur = 0, ntok_next = 0;
-  if (first < hi) ntok_cur = issue(0, 0);
-  int j = 0;
-  for (int idx = first; idx < hi; idx += LOCKS_ATT_WARPS, ++j) {
-    const int stage = j & 1;
-    const bool more = idx + LOCKS_ATT_WARPS < hi;
+  // ring of kAttStages pages per warp: pages j+1 .. j+kAttStages-1 are in flight while page j is used
+  const int npg = (hi > first) ? (hi - first + LOCKS_ATT_WARPS - 1) / LOCKS_ATT_WARPS : 0;   // this warp's pages
+  int ntok_ring[kAttStages];
+#pragma unroll
+  for (int s2 = 0; s2 < kAttStages - 1; ++s2) {
+    ntok_ring[s2] = 0;
+    if (s2 < npg) ntok_ring[s2] = issue(s2, s2); else cp_async_commit();
+  }
+  ntok_ring[kAttStages - 1] = 0;
+  for (int j = 0; j < npg; ++j) {
+    const int stage = j % kAttStages;
     if ((j & 31) == 15) resolve_batch((j & ~31) + 32, blk_nxt, nt_nxt);   // next batch, half a batch early
-    if (more) {
-      if (((j + 1) & 31) == 0) { blk_cur = blk_nxt; nt_cur = nt_nxt; }
-      ntok_next = issue(j + 1, stage ^ 1);
+    {
+      const int jn = j + kAttStages - 1;   // refill the slot freed by page j-1
+      if (((jn) & 31) == 0 && jn > 0) { blk_cur = blk_nxt; nt_cur = nt_nxt; }
+      int nt_new = 0;
+      if (jn < npg) nt_new = issue(jn, jn % kAttStages); else cp_async_commit();
+#pragma unroll
+      for (int s2 = 0; s2 < kAttStages; ++s2) if (s2 == jn % kAttStages) ntok_ring[s2] = nt_new;
     }
-    if (more) cp_async_wait<1>(); else cp_async_wait<0>();
+    cp_async_wait<kAttStages - 1>();
+    int ntok_cur = 0;
+#pragma unroll
+    for (int s2 = 0; s2 < kAttStages; ++s2) if (s2 == stage) ntok_cur = ntok_ring[s2];
     __syncwarp();
     const uint8_t *kt = ring + stage * kAttStage, *vt = kt + kTile;
     const int ntok = ntok_cur;
@@ -227,7 +242,6 @@ __global__ void __launch_bounds__(LOCKS_ATT_WARPS * 32) attend_bf16_kernel(AttPa
       }
     }
     __syncwarp();
-    ntok_cur = ntok_next;
   }
   cp_async_wait<0>();
 #pragma unroll
@@ -258,12 +272,12 @@ __global__ void __launch_bounds__(LOCKS_ATT_WARPS * 32) attend_bf16_kernel(AttPa
     float M = -INFINITY;
 #pragma unroll
     for (int w = 0; w < LOCKS_ATT_WARPS; ++w)
-      M = fmaxf(M, reinterpret_cast<const float *>(smem + w * 2 * kAttStage)[16 * LOCKS_D + g]);
+      M = fmaxf(M, reinterpret_cast<const float *>(smem + w * kAttStages * kAttStage)[16 * LOCKS_D + g]);
     float L = 0.f, o = 0.f;
     if (M > -INFINITY) {
 #pragma unroll
       for (int w = 0; w < LOCKS_ATT_WARPS; ++w) {
-        const float *ww = reinterpret_cast<const float *>(smem + w * 2 * kAttStage);
+        const float *ww = reinterpret_cast<const float *>(smem + w * kAttStages * kAttStage);
         const float sc = ex2f(ww[16 * LOCKS_D + g] - M);
         L += ww[16 * LOCKS_D + 16 + g] * sc;
         o += ww[g * LOCKS_D + dim] * sc;
@@ -290,23 +304,45 @@ __global__ void __launch_bounds__(LOCKS_ATT_WARPS * 32) attend_bf16_kernel(AttPa
   __syncthreads();
   if (!sh_last) return;
   __threadfence();
-  for (int e = threadIdx.x; e < p.G * LOCKS_D; e += LOCKS_ATT_WARPS * 32) {
-    const int g = e / LOCKS_D, dim = e - g * LOCKS_D;
-    const int64_t row = (int64_t)b * p.Hq + h * p.G + g;
-    const float *pl = p.part_lse + row * p.splits;
+  // weights of the splits: sh_w[g][s] = 2^(lse_s - max), then normalised by their sum
+  float *sh_w = reinterpret_cast<float *>(smem);   // [G][splits] <= 16 x 64 floats, the rings are idle now
+  constexpr int NT = LOCKS_ATT_WARPS * 32;
+  for (int e = threadIdx.x; e < p.G * p.splits; e += NT) {
+    const int g = e / p.splits, s2 = e - g * p.splits;
+    sh_w[e] = __ldcg(p.part_lse + ((int64_t)b * p.Hq + h * p.G + g) * p.splits + s2);
+  }
+  __syncthreads();
+  if (threadIdx.x < p.G) {
+    float *w = sh_w + threadIdx.x * p.splits;
     float M = -INFINITY;
-    for (int s2 = 0; s2 < p.splits; ++s2) M = fmaxf(M, __ldcg(pl + s2));
-    float L = 0.f, acc = 0.f;
-    if (M > -INFINITY) {
-      for (int s2 = 0; s2 < p.splits; ++s2) {
-        const float w = ex2f(__ldcg(pl + s2) - M);
-        L += w;
-        acc += w * __ldcg(p.part_o + (row * p.splits + s2) * LOCKS_D + dim);
+    for (int s2 = 0; s2 < p.splits; ++s2) M = fmaxf(M, w[s2]);
+    float L = 0.f;
+    for (int s2 = 0; s2 < p.splits; ++s2) { const float v = (M > -INFINITY) ? ex2f(w[s2] - M) : 0.f; w[s2] = v; L += v; }
+    const float inv = L > 0.f ? 1.f / L : 0.f;
+    for (int s2 = 0; s2 < p.splits; ++s2) w[s2] *= inv;
+    if (p.lse) p.lse[(int64_t)b * p.Hq + h * p.G + threadIdx.x] = (M > -INFINITY) ? (M + log2f(L)) * kLn2 : -INFINITY;
+  }
+  __syncthreads();
+  for (int e = threadIdx.x; e < p.G * (LOCKS_D / 4); e += NT) {   // four dims per thread, loads batched by 4 splits
+    const int g = e / (LOCKS_D / 4), d4 = e - g * (LOCKS_D / 4);
+    const int64_t row = (int64_t)b * p.Hq + h * p.G + g;
+    const float4 *po = reinterpret_cast<const float4 *>(p.part_o + row * p.splits * LOCKS_D) + d4;
+    const float *w = sh_w + g * p.splits;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int s0 = 0; s0 < p.splits; s0 += 4) {
+      float4 v[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        v[u] = (s0 + u < p.splits) ? __ldcg(po + (int64_t)(s0 + u) * (LOCKS_D / 4)) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const float ww = (s0 + u < p.splits) ? w[s0 + u] : 0.f;
+        acc.x += ww * v[u].x; acc.y += ww * v[u].y; acc.z += ww * v[u].z; acc.w += ww * v[u].w;
       }
-      acc /= L;
     }
-    reinterpret_cast<__nv_bfloat16 *>(p.out)[row * LOCKS_D + dim] = __float2bfloat16_rn(acc);
-    if (p.lse && dim == 0) p.lse[row] = (M > -INFINITY) ? (M + log2f(L)) * kLn2 : -INFINITY;
+    __nv_bfloat162 *dst = reinterpret_cast<__nv_bfloat162 *>(reinterpret_cast<__nv_bfloat16 *>(p.out) + row * LOCKS_D + 4 * d4);
+    dst[0] = __floats2bfloat162_rn(acc.x, acc.y);
+    dst[1] = __floats2bfloat162_rn(acc.z, acc.w);
   }
   if (threadIdx.x == 0) p.done[prob] = 0;   // ready for the next launch
 }
@@ -319,6 +355,7 @@ __global__ void __launch_bounds__(128) attend_generic_kernel(AttParams p) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int split = blockIdx.x, hq = blockIdx.y, b = blockIdx.z;
   const int h = hq / p.G;
+  pdl_wait();
   const int64_t prob = (int64_t)b * p.Hkv + h;
   const int Tn = p.seq_lens[b];
   const int P = (Tn + LOCKS_B - 1) / LOCKS_B;
@@ -377,6 +414,7 @@ template <typename T>
 __global__ void __launch_bounds__(128) attend_merge_kernel(const float *part_o, const float *part_lse, int splits,
                                                            T *out, float *lse, int Hq) {
   const int hq = blockIdx.x, b = blockIdx.y, dim = threadIdx.x;
+  pdl_wait();
   const int64_t row = (int64_t)b * Hq + hq;
   const float *pl = part_lse + row * splits;
   float M = -INFINITY;
@@ -407,7 +445,8 @@ int locks_launch_attend(locks_ctx *c, const void *q, const locks_kv *kv, int bat
   const bool dense = ids == nullptr;
   // one wave: as many splits per problem as resident CTA slots allow, at least one page per warp
   const int npages = dense ? c->Pmax : c->k;
-  const int slots = c->num_sms * LOCKS_ATT_CTAS_PER_SM;
+  int slots = c->num_sms * LOCKS_ATT_CTAS_PER_SM;
+  if (slots > LOCKS_ATT_SLOT_BOUND) slots = LOCKS_ATT_SLOT_BOUND;
   int splits = slots / (batch * p.Hkv);
   const int most = (npages + LOCKS_ATT_WARPS - 1) / LOCKS_ATT_WARPS;
   if (splits > most) splits = most;
@@ -428,22 +467,23 @@ int locks_launch_attend(locks_ctx *c, const void *q, const locks_kv *kv, int bat
     }
     dim3 grid(p.splits, p.Hkv, batch);
     const bool contig = kv->stride_token == LOCKS_D;
+    const dim3 blk(LOCKS_ATT_WARPS * 32);
     if (c->G <= 8) {
-      if (contig) attend_bf16_kernel<1, true><<<grid, LOCKS_ATT_WARPS * 32, kAttSmem, st>>>(p);
-      else attend_bf16_kernel<1, false><<<grid, LOCKS_ATT_WARPS * 32, kAttSmem, st>>>(p);
+      if (contig) locks_launch_pdl(attend_bf16_kernel<1, true>, grid, blk, kAttSmem, st, p);
+      else locks_launch_pdl(attend_bf16_kernel<1, false>, grid, blk, kAttSmem, st, p);
     } else {
-      if (contig) attend_bf16_kernel<2, true><<<grid, LOCKS_ATT_WARPS * 32, kAttSmem, st>>>(p);
-      else attend_bf16_kernel<2, false><<<grid, LOCKS_ATT_WARPS * 32, kAttSmem, st>>>(p);
+      if (contig) locks_launch_pdl(attend_bf16_kernel<2, true>, grid, blk, kAttSmem, st, p);
+      else locks_launch_pdl(attend_bf16_kernel<2, false>, grid, blk, kAttSmem, st, p);
     }
   } else {
     dim3 grid(p.splits, p.Hq, batch);
-    attend_generic_kernel<float><<<grid, 128, 0, st>>>(p);
+    locks_launch_pdl(attend_generic_kernel<float>, grid, dim3(128), 0, st, p);
   }
   int rc = locks_check_launch(c);
   if (rc != LOCKS_OK || p.splits == 1 || bf) return rc;   // the bf16 kernel merges its own splits
   dim3 mg(p.Hq, batch);
-  attend_merge_kernel<float><<<mg, 128, 0, st>>>(c->att_o, c->att_lse, p.splits, reinterpret_cast<float *>(out), lse,
-                                                 p.Hq);
+  locks_launch_pdl(attend_merge_kernel<float>, mg, dim3(128), 0, st, (const float *)c->att_o, (const float *)c->att_lse,
+                   p.splits, reinterpret_cast<float *>(out), lse, p.Hq);
   return locks_check_launch(c);
 }
 

@@ -298,6 +298,8 @@ template <typename T>
 __global__ void __launch_bounds__(256) prep_kernel(PrepParams p) {
   const int b = blockIdx.x;
   if (p.k_new == nullptr) return;
+  pdl_trigger();
+  pdl_wait();   // the previous step's readers of the cache and of seq_lens are done
   const int T0 = p.seq_lens[b];
   const int page = T0 / LOCKS_B, slot = T0 % LOCKS_B;
   bool ok = page < p.Pmax;
@@ -359,7 +361,7 @@ int locks_launch_prep(locks_ctx *c, const void *q, const void *k_new, const void
   p.block_table = kv->block_table; p.seq_lens = kv->seq_lens; p.status = c->status;
   p.Hq = c->cfg.num_q_heads; p.Hkv = c->cfg.num_kv_heads; p.Pmax = c->Pmax; p.num_blocks = kv->num_blocks;
   if (k_new == nullptr) return LOCKS_OK;   // nothing to append: no launch
-  if (c->cfg.q_dtype == LOCKS_BF16) prep_kernel<__nv_bfloat16><<<batch, 256, 0, st>>>(p);
-  else prep_kernel<float><<<batch, 256, 0, st>>>(p);
+  if (c->cfg.q_dtype == LOCKS_BF16) locks_launch_pdl(prep_kernel<__nv_bfloat16>, dim3(batch), dim3(256), 0, st, p);
+  else locks_launch_pdl(prep_kernel<float>, dim3(batch), dim3(256), 0, st, p);
   return locks_check_launch(c);
 }

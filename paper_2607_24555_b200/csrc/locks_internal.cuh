@@ -9,12 +9,17 @@
 
 #define LOCKS_D 128          // head dimension the kernels are written for
 #define LOCKS_B 16           // tokens per page
-#define LOCKS_GROUP 8        // pages scored together by one warp in the scan
+#define LOCKS_GROUP 8        // pages scored together by one warp in the scan (one ring stage, one partial)
 #define LOCKS_SEL_THREADS 512
 #define LOCKS_SEL_MAX_EPT 16 // candidate pages held per thread in select stage 1 (4, 8 or 16)
-#define LOCKS_ATT_WARPS 3        // warps per attend CTA, each with a two-stage 16 KB page ring
-#define LOCKS_ATT_CTAS_PER_SM 4  // 4 x 48 KB of shared memory, 4 x 96 x 168 registers
-#define LOCKS_ATT_MAX_SPLITS 64
+#define LOCKS_ATT_WARPS 3        // warps per attend CTA
+#define LOCKS_ATT_STAGES 2       // pages (4 KB of K + 4 KB of V each) in each warp's ring
+#define LOCKS_ATT_CTAS_PER_SM 4  // 4 x 48 KB of shared memory
+#define LOCKS_ATT_MAX_SPLITS 128
+#define LOCKS_ATT_SLOT_BOUND 1024 // upper bound on resident attend CTAs of any supported GPU (148 SMs x 4 on B200)
+#ifndef LOCKS_SCAN_BULK
+#define LOCKS_SCAN_BULK 1      // staging of summary blobs in the scan: 1 = cp.async.bulk (TMA) + mbarrier, 0 = 16-byte cp.async
+#endif
 #define LOCKS_SPIN_LIMIT (1 << 22)  // bounded mbarrier polling (each poll already waits a while)
 
 struct locks_ctx {
@@ -30,10 +35,11 @@ struct locks_ctx {
   int32_t *status;         // [4] sticky status, work counters
   float *shat;             // [max_batch][Hq][Pmax]
   float2 *part;            // [max_batch][Hq][max_groups] per-group (max, sum exp) of candidates
+  float *logz;             // [max_batch][Hq] log Z_g (chunked selection only)
   float *cand_val;         // [max_batch][Hkv][sel_chunks][sel_kc]
   int32_t *cand_idx;
-  float *att_o;            // [max_batch][Hq][LOCKS_ATT_MAX_SPLITS][d]
-  float *att_lse;          // [max_batch][Hq][LOCKS_ATT_MAX_SPLITS]  (log2 units)
+  float *att_o;            // [rows][d], rows = batch * Hq * splits <= att_rows
+  float *att_lse;          // [rows]  (log2 units)
   int32_t *att_done;       // [max_batch][Hkv] split-arrival counters
   int32_t *ids_int;        // [max_batch][Hkv][k]
   int32_t *cnt_int;        // [max_batch][Hkv]
@@ -59,6 +65,25 @@ int locks_launch_attend(locks_ctx *c, const void *q, const locks_kv *kv, int bat
 int locks_launch_build(locks_ctx *c, const locks_kv *kv, int batch, const int32_t *pb, const int32_t *pe,
                        int just_filled, void *summaries, cudaStream_t st);
 
+// Launch with programmatic dependent launch allowed: the kernel may be scheduled while its stream
+// predecessor is still draining; it must execute pdl_wait() before touching anything the predecessor
+// writes (the wait returns once the predecessor grid has completed and its writes are visible).
+template <typename... KArgs, typename... Args>
+static inline void locks_launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                    Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = 1;
+  (void)cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+
 static inline int locks_check_launch(locks_ctx *c) {
   c->last_launches++;
   return cudaPeekAtLastError() == cudaSuccess ? LOCKS_OK : LOCKS_ERR_CUDA;
@@ -77,6 +102,10 @@ __host__ __device__ constexpr int f32_stride(int r) { return 4 * (LOCKS_D + r * 
 #ifdef __CUDACC__
 
 __device__ __forceinline__ void set_status(int32_t *status, int code) { atomicCAS(status, 0, code); }
+
+// programmatic dependent launch: wait for the stream predecessor / let the successor be scheduled
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll

@@ -59,6 +59,7 @@ template <int FMT, typename QT>
 __global__ void __launch_bounds__(128) scan_generic_kernel(ScanParams p) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int grp = blockIdx.x * 4 + warp, h = blockIdx.y, b = blockIdx.z;
+  pdl_wait();
   const int T = p.seq_lens[b];
   const int P = (T + LOCKS_B - 1) / LOCKS_B;
   if (P <= p.k) return;               // every page is kept: nothing to rank
@@ -141,9 +142,11 @@ __global__ void __launch_bounds__(128) scan_generic_kernel(ScanParams p) {
 
 constexpr int kScanWarps = 8;
 constexpr int kScanStages = 2;
+constexpr int kScanCtasPerSm = 2;
 constexpr int kBlob = i4_stride(8);                       // 832
 constexpr int kStageBytes = LOCKS_GROUP * kBlob;          // 6656
 constexpr int kScanSmem = kScanWarps * (kScanStages * kStageBytes + 64);
+constexpr bool kScanBulk = LOCKS_SCAN_BULK;             // true: cp.async.bulk + mbarrier, false: 16-byte cp.async
 
 // (a & b) | c in one LOP3 with both constants held in registers
 __device__ __forceinline__ uint32_t and_or(uint32_t a, uint32_t b, uint32_t c) {
@@ -180,7 +183,7 @@ __device__ __forceinline__ void mma_f16_z(float (&d)[4], uint32_t a0, uint32_t a
 }
 
 struct Cursor {
-  int prob, grp, nsc;
+  int prob, grp, nsc, b, h;   // (request, KV head) of prob are refreshed only when prob changes
 };
 
 __device__ __forceinline__ uint32_t movm_trans(uint32_t v) {
@@ -203,8 +206,11 @@ __device__ __forceinline__ uint32_t movm_trans(uint32_t v) {
 //    8 significant bits fit; only elements below 2^-14 of the row maximum can round, by at most
 //    2^-25 of it).  Products are exact, sums are fp32; the projection is carried into the second
 //    MMA as an fp16 hi + lo pair (22 significant bits).
-template <int NH>
-__global__ void __launch_bounds__(kScanWarps * 32, 2) scan_i4r8_kernel(ScanParams p) {
+// PK (G <= 4 only): the 8 head columns hold the group twice, so that after MMA#1 the projection, MMA#2 and
+// the log-sum-exp handle two pages at once (rows 0-3 = page A's heads, rows 4-7 = page B's heads, the two
+// pages separated along K) instead of leaving half of the lanes idle.
+template <int NH, bool PK>
+__global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4r8_kernel(ScanParams p) {
   extern __shared__ __align__(128) uint8_t smem[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int x = lane >> 2, t = lane & 3;
@@ -215,6 +221,8 @@ __global__ void __launch_bounds__(kScanWarps * 32, 2) scan_i4r8_kernel(ScanParam
     fence_barrier_init();
   }
   __syncwarp();
+  pdl_trigger();   // single-wave kernel: the selector may be scheduled as SMs drain
+  pdl_wait();      // sequence lengths (append) and the previous consumers of the workspace are done
 
   // warps stick to one (request, KV head) at a time: `wpp` warps share a problem and stride its groups
   const int W = gridDim.x * kScanWarps;
@@ -224,16 +232,18 @@ __global__ void __launch_bounds__(kScanWarps * 32, 2) scan_i4r8_kernel(ScanParam
   const int slot = wid / wpp, sub = wid - slot * wpp;
   if (slot >= nslots) return;
 
-  auto load_nsc = [&](int prob) -> int {
-    const int T = p.seq_lens[prob / p.Hkv];
+  auto enter = [&](Cursor &c) {   // refresh the per-problem fields of the cursor
+    c.b = c.prob / p.Hkv;
+    c.h = c.prob - c.b * p.Hkv;
+    const int T = p.seq_lens[c.b];
     const int P = (T + LOCKS_B - 1) / LOCKS_B;
-    return (P <= p.k) ? 0 : P - 1;
+    c.nsc = (P <= p.k) ? 0 : P - 1;
   };
   auto settle = [&](Cursor &c) {  // move to the next non-empty position at or after (prob, grp)
     while (c.prob < nprob && c.grp * LOCKS_GROUP >= c.nsc) {
       c.prob += nslots;
       c.grp = sub;
-      if (c.prob < nprob) c.nsc = load_nsc(c.prob);
+      if (c.prob < nprob) enter(c);
     }
   };
   // the physical block of page (grp*8 + lane) of the producer cursor, fetched one group ahead of use
@@ -241,25 +251,40 @@ __global__ void __launch_bounds__(kScanWarps * 32, 2) scan_i4r8_kernel(ScanParam
     if (c.prob >= nprob) return 0;
     const int page = c.grp * LOCKS_GROUP + lane;
     if (lane >= LOCKS_GROUP || page >= c.nsc) return 0;
-    return p.block_table[(int64_t)(c.prob / p.Hkv) * p.Pmax + page];
+    return p.block_table[(int64_t)c.b * p.Pmax + page];
   };
   auto issue = [&](int stage, const Cursor &c, int block) {
-    const int h = c.prob % p.Hkv;
+    const int h = c.h;
     const int nvalid = min(LOCKS_GROUP, c.nsc - c.grp * LOCKS_GROUP);
-    if (lane == 0) mbar_expect_tx(&full[stage], (uint32_t)nvalid * kBlob);
-    __syncwarp();
-    if (lane < nvalid) {
-      if (block < 0 || block >= p.num_blocks) {
-        set_status(p.status, LOCKS_ERR_BAD_BLOCK);
-        block = 0;
+    if (lane < nvalid && (block < 0 || block >= p.num_blocks)) {
+      set_status(p.status, LOCKS_ERR_BAD_BLOCK);
+      block = 0;
+    }
+    if (kScanBulk) {
+      if (lane == 0) mbar_expect_tx(&full[stage], (uint32_t)nvalid * kBlob);
+      __syncwarp();
+      if (lane < nvalid)
+        bulk_g2s(ring + stage * kStageBytes + lane * kBlob, p.summ + ((int64_t)block * p.Hkv + h) * kBlob, kBlob,
+                 &full[stage]);
+    } else {
+      // 52 16-byte chunks per blob: lanes 0-25 copy chunks lane and lane + 26 of every page of the group
+      uint8_t *dst = ring + stage * kStageBytes + lane * 16;
+#pragma unroll
+      for (int pg = 0; pg < LOCKS_GROUP; ++pg) {
+        const int blk = __shfl_sync(0xffffffffu, block, pg);
+        const uint8_t *src = p.summ + ((int64_t)blk * p.Hkv + h) * kBlob + lane * 16;
+        const bool on = lane < 26 && pg < nvalid;
+        if (on) {
+          cp_async16(dst + pg * kBlob, src, true);
+          cp_async16(dst + pg * kBlob + 416, src + 416, true);
+        }
       }
-      bulk_g2s(ring + stage * kStageBytes + lane * kBlob, p.summ + ((int64_t)block * p.Hkv + h) * kBlob, kBlob,
-               &full[stage]);
+      cp_async_commit();
     }
   };
 
-  Cursor cp{slot, sub, 0}, cc;
-  if (cp.prob < nprob) cp.nsc = load_nsc(cp.prob);
+  Cursor cp{slot, sub, 0, 0, 0}, cc;
+  if (cp.prob < nprob) enter(cp);
   settle(cp);
   cc = cp;
   int inflight = 0;
@@ -334,19 +359,26 @@ __global__ void __launch_bounds__(kScanWarps * 32, 2) scan_i4r8_kernel(ScanParam
   while (cc.prob < nprob) {
     const int stage = it % kScanStages;
     const uint32_t parity = (it / kScanStages) & 1;
-    if (!mbar_wait(&full[stage], parity)) {
-      ok = false;
-      break;
+    if (kScanBulk) {
+      if (!mbar_wait(&full[stage], parity)) {
+        ok = false;
+        break;
+      }
+    } else {
+      // groups complete in order: all but the newest (kScanStages - 1) committed groups must have landed
+      if (inflight >= kScanStages) cp_async_wait<kScanStages - 1>(); else cp_async_wait<0>();
+      __syncwarp();
     }
     --inflight;
-    const int b = cc.prob / p.Hkv, h = cc.prob - b * p.Hkv;
+    const int b = cc.b, h = cc.h;
     if (cc.prob != cur_prob) {
       cur_prob = cc.prob;
 #pragma unroll
       for (int hh = 0; hh < NH; ++hh) {
         float s8;
-        load_q_row(b, h * p.G + x + 8 * hh, x + 8 * hh < p.G, qb0[hh], qb2[hh], inv_s[hh], s8);
-        // lane (x, t) owns head x; the column fragment needs heads 2t, 2t+1
+        const int gx = PK ? (x & 3) : x + 8 * hh;   // head held by this lane's column
+        load_q_row(b, h * p.G + gx, gx < p.G, qb0[hh], qb2[hh], inv_s[hh], s8);
+        // lane (x, t) owns head gx; the column fragment needs the heads of columns 2t, 2t+1
         ksum[2 * hh] = __shfl_sync(0xffffffffu, s8, (2 * t) * 4);
         ksum[2 * hh + 1] = __shfl_sync(0xffffffffu, s8, (2 * t + 1) * 4);
       }
@@ -356,7 +388,7 @@ __global__ void __launch_bounds__(kScanWarps * 32, 2) scan_i4r8_kernel(ScanParam
     // ---- centroid dots of the 8 pages: cen[head x (+8)][pages 2t, 2t+1] = sum_c code_mu[c] q'[c]
     float cen[4] = {0.f, 0.f, 0.f, 0.f};
     {
-      const uint4 *mp = reinterpret_cast<const uint4 *>(sb + x * kBlob + i4_off_mu(8) + t * 32);
+      const uint4 *mp = reinterpret_cast<const uint4 *>(sb + (x & (LOCKS_GROUP - 1)) * kBlob + i4_off_mu(8) + t * 32);
       const uint4 m0 = mp[0], m1 = mp[1];
       const uint32_t mw[8] = {m0.x, m0.y, m0.z, m0.w, m1.x, m1.y, m1.z, m1.w};
 #pragma unroll
@@ -369,8 +401,9 @@ __global__ void __launch_bounds__(kScanWarps * 32, 2) scan_i4r8_kernel(ScanParam
     }
     float acen[2 * NH];  // log2-domain centroid term of pages 2t, 2t+1 for head x (and x + 8)
     {
-      const float s0 = __half2float(*reinterpret_cast<const __half *>(sb + (2 * t) * kBlob + i4_off_smu(8)));
-      const float s1 = __half2float(*reinterpret_cast<const __half *>(sb + (2 * t + 1) * kBlob + i4_off_smu(8)));
+      const int pg0 = (2 * t) & (LOCKS_GROUP - 1);   // lanes t >= LOCKS_GROUP / 2 hold nothing useful
+      const float s0 = __half2float(*reinterpret_cast<const __half *>(sb + pg0 * kBlob + i4_off_smu(8)));
+      const float s1 = __half2float(*reinterpret_cast<const __half *>(sb + (pg0 + 1) * kBlob + i4_off_smu(8)));
 #pragma unroll
       for (int hh = 0; hh < NH; ++hh) {
         acen[2 * hh] = s0 * (c2 * inv_s[hh]) * cen[2 * hh];
@@ -399,6 +432,46 @@ __global__ void __launch_bounds__(kScanWarps * 32, 2) scan_i4r8_kernel(ScanParam
           mma_f16(c1[hh], ua8 & kM0, ub8 & kM0, ua8 & kM1, ub8 & kM1, qb0[hh][2 * j + 1], qb2[hh][2 * j + 1]);
         }
       }
+      if (PK) {
+        // lanes t < 2 carry page A (columns 0-3), lanes t >= 2 page B (columns 4-7)
+        const bool pa = t < 2;
+        const uint8_t *pbs = pa ? pbA : pbB;
+        const float sv = __half2float(*reinterpret_cast<const __half *>(pbs + i4_off_sv(8) + 2 * x));
+        const float p0 = fmaf(pa ? c1[0][0] : c1[0][2], 16777216.f, -ksum[0]) * sv;
+        const float p1 = fmaf(pa ? c1[0][1] : c1[0][3], 16777216.f, -ksum[1]) * sv;
+        const uint32_t hi = pack_f16(p0, p1);
+        const float2 hf = h2f2(hi);
+        const uint32_t lo = pack_f16(p0 - hf.x, p1 - hf.y);
+        const uint32_t hiT = movm_trans(hi), loT = movm_trans(lo);   // lane (x, t): row x, ranks 2t, 2t+1
+        const bool ra = x < 4;                                        // row x: page A head x | page B head x - 4
+        const uint32_t hA = ra ? hiT : 0u, hB = ra ? 0u : hiT, lA = ra ? loT : 0u, lB = ra ? 0u : loT;
+        const uint32_t cwa = *reinterpret_cast<const uint32_t *>(pbA + i4_off_coef(8) + lane * 4);
+        const uint32_t cwb = *reinterpret_cast<const uint32_t *>(pbB + i4_off_coef(8) + lane * 4);
+        const uint32_t a0 = f16x2_sub(__byte_perm(cwa, 0x64646464u, 0x4140), kSub128);
+        const uint32_t a1 = f16x2_sub(__byte_perm(cwa, 0x64646464u, 0x4342), kSub128);
+        const uint32_t b0 = f16x2_sub(__byte_perm(cwb, 0x64646464u, 0x4140), kSub128);
+        const uint32_t b1 = f16x2_sub(__byte_perm(cwb, 0x64646464u, 0x4342), kSub128);
+        // k 0-7 = page A's ranks, k 8-15 = page B's ranks; hi and lo parts accumulate into the same tile
+        float ca[4], cb[4];
+        mma_f16_z(ca, hA, 0u, hB, 0u, a0, b0);
+        mma_f16(ca, lA, 0u, lB, 0u, a0, b0);
+        mma_f16_z(cb, hA, 0u, hB, 0u, a1, b1);
+        mma_f16(cb, lA, 0u, lB, 0u, a1, b1);
+        const uint2 scw = *reinterpret_cast<const uint2 *>((ra ? pbA : pbB) + i4_off_sc(8) + 8 * t);
+        const float2 s01 = h2f2(scw.x), s89 = h2f2(scw.y);
+        const float iv = inv_s[0] * c2;
+        const float y0 = ca[0] * s01.x, y1 = ca[1] * s01.y, y2 = cb[0] * s89.x, y3 = cb[1] * s89.y;
+        float my = fmaxf(fmaxf(y0, y1), fmaxf(y2, y3));
+        my = fmaxf(my, __shfl_xor_sync(0xffffffffu, my, 1));
+        my = fmaxf(my, __shfl_xor_sync(0xffffffffu, my, 2));
+        const float m = my * iv;
+        float e = fast_ex2(fmaf(y0, iv, -m)) + fast_ex2(fmaf(y1, iv, -m)) + fast_ex2(fmaf(y2, iv, -m)) +
+                  fast_ex2(fmaf(y3, iv, -m));
+        e += __shfl_xor_sync(0xffffffffu, e, 1);
+        e += __shfl_xor_sync(0xffffffffu, e, 2);
+        // lane (x, t = pp) keeps the result of page 2 pp + (x >> 2), head x & 3
+        if (t == pp) res[0] = m + fast_lg2(e) + (ra ? acen[0] : acen[1]);
+      } else {
 #pragma unroll
       for (int pq = 0; pq < 2; ++pq) {
         const int pg = 2 * pp + pq;
@@ -443,6 +516,7 @@ __global__ void __launch_bounds__(kScanWarps * 32, 2) scan_i4r8_kernel(ScanParam
         }
       }
     }
+      }
     __syncwarp();  // every lane is done reading this stage
     if (cp.prob < nprob) {
       issue(stage, cp, next_block);
@@ -453,13 +527,30 @@ __global__ void __launch_bounds__(kScanWarps * 32, 2) scan_i4r8_kernel(ScanParam
     }
 
     // ---- write s^ and the group's candidate partial
+    if (PK) {
+      const int g = x & 3, page = cc.grp * LOCKS_GROUP + 2 * t + (x >> 2);
+      const float v = res[0] * kLn2;
+      const bool in = t < LOCKS_GROUP / 2 && page < cc.nsc;
+      if (g < p.G && in) p.shat[((int64_t)b * p.Hq + h * p.G + g) * p.Pmax + page] = v;
+      const float c0 = (in && page >= 1) ? v : -INFINITY;
+      float m = c0;
+      m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 1));
+      m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 2));
+      m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 16));
+      float e = (m == -INFINITY) ? 0.f : __expf(c0 - m);
+      e += __shfl_xor_sync(0xffffffffu, e, 1);
+      e += __shfl_xor_sync(0xffffffffu, e, 2);
+      e += __shfl_xor_sync(0xffffffffu, e, 16);
+      if (t == 0 && x < 4 && g < p.G)
+        p.part[((int64_t)b * p.Hq + h * p.G + g) * p.max_groups + cc.grp] = make_float2(m, e);
+    } else {
     const int page0 = cc.grp * LOCKS_GROUP + 2 * t;
 #pragma unroll
     for (int hh = 0; hh < NH; ++hh) {
       const int g = x + 8 * hh;
       const float v0 = (res[2 * hh] + acen[2 * hh]) * kLn2;
       const float v1 = (res[2 * hh + 1] + acen[2 * hh + 1]) * kLn2;
-      const bool in0 = page0 < cc.nsc, in1 = page0 + 1 < cc.nsc;
+      const bool in0 = t < LOCKS_GROUP / 2 && page0 < cc.nsc, in1 = t < LOCKS_GROUP / 2 && page0 + 1 < cc.nsc;
       if (g < p.G) {
         float *dst = p.shat + ((int64_t)b * p.Hq + h * p.G + g) * p.Pmax + page0;
         if (in0) dst[0] = v0;
@@ -475,6 +566,7 @@ __global__ void __launch_bounds__(kScanWarps * 32, 2) scan_i4r8_kernel(ScanParam
       e += __shfl_xor_sync(0xffffffffu, e, 2);
       if (t == 0 && g < p.G)
         p.part[((int64_t)b * p.Hq + h * p.G + g) * p.max_groups + cc.grp] = make_float2(m, e);
+    }
     }
     cc.grp += wpp;
     settle(cc);
@@ -509,25 +601,27 @@ int locks_launch_scan(locks_ctx *c, const void *q, const void *summaries, const 
   if (tensor) {
     static bool attr_done = false;
     if (!attr_done) {
-      cudaFuncSetAttribute(scan_i4r8_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kScanSmem);
-      cudaFuncSetAttribute(scan_i4r8_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kScanSmem);
+      cudaFuncSetAttribute(scan_i4r8_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kScanSmem);
+      cudaFuncSetAttribute(scan_i4r8_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kScanSmem);
+      cudaFuncSetAttribute(scan_i4r8_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kScanSmem);
       attr_done = true;
     }
     const int total_groups = batch * p.Hkv * p.max_groups;
-    int grid = 2 * c->num_sms;
+    int grid = kScanCtasPerSm * c->num_sms;
     const int need = (total_groups + kScanWarps - 1) / kScanWarps;
     if (grid > need) grid = need < 1 ? 1 : need;
-    if (c->G <= 8) scan_i4r8_kernel<1><<<grid, kScanWarps * 32, kScanSmem, st>>>(p);
-    else scan_i4r8_kernel<2><<<grid, kScanWarps * 32, kScanSmem, st>>>(p);
+    if (c->G <= 4) locks_launch_pdl(scan_i4r8_kernel<1, true>, dim3(grid), dim3(kScanWarps * 32), kScanSmem, st, p);
+    else if (c->G <= 8) locks_launch_pdl(scan_i4r8_kernel<1, false>, dim3(grid), dim3(kScanWarps * 32), kScanSmem, st, p);
+    else locks_launch_pdl(scan_i4r8_kernel<2, false>, dim3(grid), dim3(kScanWarps * 32), kScanSmem, st, p);
   } else {
     dim3 grid((c->max_groups + 3) / 4, p.Hkv, batch);
     const bool qbf = c->cfg.q_dtype == LOCKS_BF16;
     if (c->cfg.summary_fmt == LOCKS_FMT_F32) {
-      if (qbf) scan_generic_kernel<LOCKS_FMT_F32, __nv_bfloat16><<<grid, 128, 0, st>>>(p);
-      else scan_generic_kernel<LOCKS_FMT_F32, float><<<grid, 128, 0, st>>>(p);
+      if (qbf) locks_launch_pdl(scan_generic_kernel<LOCKS_FMT_F32, __nv_bfloat16>, grid, dim3(128), 0, st, p);
+      else locks_launch_pdl(scan_generic_kernel<LOCKS_FMT_F32, float>, grid, dim3(128), 0, st, p);
     } else {
-      if (qbf) scan_generic_kernel<LOCKS_FMT_I4, __nv_bfloat16><<<grid, 128, 0, st>>>(p);
-      else scan_generic_kernel<LOCKS_FMT_I4, float><<<grid, 128, 0, st>>>(p);
+      if (qbf) locks_launch_pdl(scan_generic_kernel<LOCKS_FMT_I4, __nv_bfloat16>, grid, dim3(128), 0, st, p);
+      else locks_launch_pdl(scan_generic_kernel<LOCKS_FMT_I4, float>, grid, dim3(128), 0, st, p);
     }
   }
   return locks_check_launch(c);

@@ -20,6 +20,7 @@ struct SelParams {
   float *logshare;
   float *cand_val;
   int32_t *cand_idx;
+  float *logz;      // [batch][Hq] log Z_g, written by logz_kernel when a problem spans several chunks
   int batch, Hq, Hkv, G, Pmax, max_groups, k, chunks, kc, chunk_pages;
 };
 
@@ -138,12 +139,52 @@ __device__ void group_logz(const SelParams &p, int b, int h, int ngroups, float 
   }
 }
 
+// log Z_g of one query head from the scan's per-group partials (used when a problem is ranked in chunks)
+__global__ void __launch_bounds__(256) logz_kernel(SelParams p) {
+  __shared__ float sm_m[8], sm_s[8];
+  const int hq = blockIdx.x, b = blockIdx.y, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  pdl_trigger();
+  pdl_wait();
+  const int T = p.seq_lens[b];
+  const int P = (T + LOCKS_B - 1) / LOCKS_B;
+  if (P <= p.k) return;
+  const int ngroups = (P - 1 + LOCKS_GROUP - 1) / LOCKS_GROUP;
+  const float2 *pp = p.part + ((int64_t)b * p.Hq + hq) * p.max_groups;
+  float m = -INFINITY, s = 0.f;
+  for (int i = threadIdx.x; i < ngroups; i += 256) {
+    const float2 v = pp[i];
+    if (v.x > -INFINITY) {
+      const float nm = fmaxf(m, v.x);
+      s = s * __expf(m - nm) + v.y * __expf(v.x - nm);
+      m = nm;
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const float om = __shfl_xor_sync(0xffffffffu, m, o), os = __shfl_xor_sync(0xffffffffu, s, o);
+    const float nm = fmaxf(m, om);
+    if (nm > -INFINITY) { s = s * __expf(m - nm) + os * __expf(om - nm); m = nm; }
+  }
+  if (lane == 0) { sm_m[warp] = m; sm_s[warp] = s; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float M = -INFINITY, S = 0.f;
+    for (int w = 0; w < 8; ++w) {
+      const float nm = fmaxf(M, sm_m[w]);
+      if (nm > -INFINITY) { S = S * __expf(M - nm) + sm_s[w] * __expf(sm_m[w] - nm); M = nm; }
+    }
+    p.logz[b * p.Hq + hq] = M + __logf(S);
+  }
+}
+
 template <int EPT>
 __global__ void __launch_bounds__(LOCKS_SEL_THREADS) select_stage1_kernel(SelParams p) {
   __shared__ int sh_hist[(LOCKS_SEL_THREADS / 32) * 256];
   __shared__ int sh_misc[12 + LOCKS_SEL_THREADS / 32];
   __shared__ float sh_logz[16];
   for (int e = threadIdx.x; e < (LOCKS_SEL_THREADS / 32) * 256; e += LOCKS_SEL_THREADS) sh_hist[e] = 0;
+  pdl_trigger();
+  pdl_wait();   // the scan's scores and partials
   const int chunk = blockIdx.x, h = blockIdx.y, b = blockIdx.z, tid = threadIdx.x;
   const int T = p.seq_lens[b];
   const int P = (T + LOCKS_B - 1) / LOCKS_B;
@@ -177,7 +218,8 @@ __global__ void __launch_bounds__(LOCKS_SEL_THREADS) select_stage1_kernel(SelPar
       const int page = pbase + i;
       raw[g][i] = (g < p.G && page >= 1 && page <= P - 2) ? row0[(int64_t)g * p.Pmax + page] : 0.f;
     }
-  group_logz(p, b, h, (P - 1 + LOCKS_GROUP - 1) / LOCKS_GROUP, sh_logz);
+  if (p.chunks == 1) group_logz(p, b, h, (P - 1 + LOCKS_GROUP - 1) / LOCKS_GROUP, sh_logz);
+  else if (tid < p.G) sh_logz[tid] = p.logz[b * p.Hq + h * p.G + tid];
   __syncthreads();
   // log m_bar of this thread's EPT consecutive pages: log mean_g exp(s^_g - log Z_g)
   float val[EPT];
@@ -256,6 +298,8 @@ __global__ void __launch_bounds__(LOCKS_SEL_THREADS) select_stage2_kernel(SelPar
   __shared__ int sh_misc[12 + LOCKS_SEL_THREADS / 32];
   const int h = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
   for (int e = tid; e < (LOCKS_SEL_THREADS / 32) * 256; e += LOCKS_SEL_THREADS) sh_hist[e] = 0;
+  pdl_trigger();
+  pdl_wait();   // stage 1's candidate lists
   __syncthreads();
   const int T = p.seq_lens[b];
   const int P = (T + LOCKS_B - 1) / LOCKS_B;
@@ -297,17 +341,23 @@ int locks_launch_select(locks_ctx *c, const float *shat, const locks_kv *kv, int
   p.batch = batch; p.Hq = c->cfg.num_q_heads; p.Hkv = c->cfg.num_kv_heads; p.G = c->G; p.Pmax = c->Pmax;
   p.max_groups = c->max_groups; p.k = c->k; p.chunks = c->sel_chunks; p.kc = c->sel_kc;
   p.chunk_pages = c->sel_ept * LOCKS_SEL_THREADS;
+  p.logz = c->logz;
+  if (c->sel_chunks > 1) {
+    locks_launch_pdl(logz_kernel, dim3(p.Hq, batch), dim3(256), 0, st, p);
+    int rc0 = locks_check_launch(c);
+    if (rc0 != LOCKS_OK) return rc0;
+  }
   dim3 g1(c->sel_chunks, p.Hkv, batch);
-  if (c->sel_ept == 4) select_stage1_kernel<4><<<g1, LOCKS_SEL_THREADS, 0, st>>>(p);
-  else if (c->sel_ept == 8) select_stage1_kernel<8><<<g1, LOCKS_SEL_THREADS, 0, st>>>(p);
-  else select_stage1_kernel<16><<<g1, LOCKS_SEL_THREADS, 0, st>>>(p);
+  if (c->sel_ept == 4) locks_launch_pdl(select_stage1_kernel<4>, g1, dim3(LOCKS_SEL_THREADS), 0, st, p);
+  else if (c->sel_ept == 8) locks_launch_pdl(select_stage1_kernel<8>, g1, dim3(LOCKS_SEL_THREADS), 0, st, p);
+  else locks_launch_pdl(select_stage1_kernel<16>, g1, dim3(LOCKS_SEL_THREADS), 0, st, p);
   int rc = locks_check_launch(c);
   if (rc != LOCKS_OK || c->sel_chunks == 1) return rc;
   const int N = c->sel_chunks * c->sel_kc;
   const int ept = (N + LOCKS_SEL_THREADS - 1) / LOCKS_SEL_THREADS;
   dim3 grid(p.Hkv, batch);
-  if (ept <= 4) select_stage2_kernel<4><<<grid, LOCKS_SEL_THREADS, 0, st>>>(p);
-  else if (ept <= 16) select_stage2_kernel<16><<<grid, LOCKS_SEL_THREADS, 0, st>>>(p);
+  if (ept <= 4) locks_launch_pdl(select_stage2_kernel<4>, grid, dim3(LOCKS_SEL_THREADS), 0, st, p);
+  else if (ept <= 16) locks_launch_pdl(select_stage2_kernel<16>, grid, dim3(LOCKS_SEL_THREADS), 0, st, p);
   else return LOCKS_ERR_UNSUPPORTED;
   return locks_check_launch(c);
 }
