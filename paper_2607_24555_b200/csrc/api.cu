@@ -41,12 +41,19 @@ Layout make_layout(const locks_config *c) {
   L.k = (c->budget_tokens + c->page_size - 1) / c->page_size;
   L.S = c->summary_fmt == LOCKS_FMT_I4 ? i4_stride(c->rank) : f32_stride(c->rank);
   L.max_groups = (c->max_pages_per_seq + LOCKS_GROUP - 1) / LOCKS_GROUP;
-  // pages per thread in stage 1: the smallest of 4 / 8 / 16 whose per-chunk candidate lists still fit
-  // stage 2 (16 candidates per thread), so that long contexts are ranked by many CTAs
+  // pages per thread in stage 1 (4 / 8 / 16).  With many (request, KV head) problems one CTA per problem
+  // already fills the GPU, so a context of up to 8192 pages is ranked in one chunk; with few problems
+  // the smallest chunk whose candidate lists still fit stage 2 is taken, so that many CTAs share the work.
+  const int per_thread = (c->max_pages_per_seq + LOCKS_SEL_THREADS - 1) / LOCKS_SEL_THREADS;
+  const bool many_problems = (int64_t)c->max_batch * c->num_kv_heads >= 32;
   L.sel_ept = 16;
-  for (int ept = 4; ept <= 16; ept *= 2) {
-    const int chunks = (c->max_pages_per_seq + ept * LOCKS_SEL_THREADS - 1) / (ept * LOCKS_SEL_THREADS);
-    if (chunks == 1 || (size_t)chunks * (L.k - 2 > 0 ? L.k - 2 : 1) <= 16 * LOCKS_SEL_THREADS) { L.sel_ept = ept; break; }
+  if (many_problems && per_thread <= 16) {
+    L.sel_ept = per_thread <= 4 ? 4 : (per_thread <= 8 ? 8 : 16);
+  } else {
+    for (int ept = 4; ept <= 16; ept *= 2) {
+      const int chunks = (c->max_pages_per_seq + ept * LOCKS_SEL_THREADS - 1) / (ept * LOCKS_SEL_THREADS);
+      if (chunks == 1 || (size_t)chunks * (L.k - 2 > 0 ? L.k - 2 : 1) <= 16 * LOCKS_SEL_THREADS) { L.sel_ept = ept; break; }
+    }
   }
   L.sel_chunks = (c->max_pages_per_seq + L.sel_ept * LOCKS_SEL_THREADS - 1) / (L.sel_ept * LOCKS_SEL_THREADS);
   L.sel_kc = L.k - 2 > 0 ? L.k - 2 : 1;
@@ -111,6 +118,7 @@ int locks_create(const locks_config *cfg, void *workspace, size_t ws_bytes, lock
   if (!c) return LOCKS_ERR_INVALID_ARG;
   c->cfg = *cfg;
   c->prof_ev = nullptr; c->prof_cap = c->prof_n = 0;
+  c->part_slots = L.max_groups;
   c->G = L.G; c->k = L.k; c->S = L.S; c->Pmax = cfg->max_pages_per_seq; c->max_groups = L.max_groups;
   c->sel_ept = L.sel_ept; c->sel_chunks = L.sel_chunks; c->sel_kc = L.sel_kc;
   int dev = 0;

@@ -26,6 +26,7 @@ struct AttParams {
   int32_t *status;
   int32_t *done;   // [batch*Hkv] split-arrival counters (zero between launches)
   int batch, Hq, Hkv, G, Pmax, kbud, num_blocks, splits, pages_per_cta;
+  int fused_merge;   // 1: the last CTA of a problem merges its splits; 0: a separate merge kernel follows
   float sm_scale;
 };
 
@@ -295,7 +296,7 @@ __global__ void __launch_bounds__(LOCKS_ATT_WARPS * 32) attend_bf16_kernel(AttPa
       if (dim == 0) p.part_lse[slot] = lse2;
     }
   }
-  if (p.splits == 1) return;
+  if (p.splits == 1 || !p.fused_merge) return;
   // the last CTA of this (request, KV head) to arrive merges the splits' partials by log-sum-exp
   __shared__ int sh_last;
   __threadfence();
@@ -410,26 +411,54 @@ __global__ void __launch_bounds__(128) attend_generic_kernel(AttParams p) {
   }
 }
 
+// Merge of the split-K partials of one query head: 128 threads = 4 split slices x 32 four-dim columns.
 template <typename T>
 __global__ void __launch_bounds__(128) attend_merge_kernel(const float *part_o, const float *part_lse, int splits,
                                                            T *out, float *lse, int Hq) {
-  const int hq = blockIdx.x, b = blockIdx.y, dim = threadIdx.x;
+  __shared__ float sw[LOCKS_ATT_MAX_SPLITS];
+  __shared__ float4 sacc[4][32];
+  const int hq = blockIdx.x, b = blockIdx.y, tid = threadIdx.x, lane = tid & 31;
   pdl_wait();
   const int64_t row = (int64_t)b * Hq + hq;
-  const float *pl = part_lse + row * splits;
-  float M = -INFINITY;
-  for (int s = 0; s < splits; ++s) M = fmaxf(M, pl[s]);
-  float L = 0.f, acc = 0.f;
-  if (M > -INFINITY) {
-    for (int s = 0; s < splits; ++s) {
-      const float w = exp2f(pl[s] - M);
-      L += w;
-      acc += w * part_o[(row * splits + s) * LOCKS_D + dim];
-    }
-    acc /= L;
+  for (int s = tid; s < splits; s += 128) sw[s] = part_lse[row * splits + s];
+  __syncthreads();
+  if (tid < 32) {
+    float M = -INFINITY;
+    for (int s = lane; s < splits; s += 32) M = fmaxf(M, sw[s]);
+    M = warp_max(M);
+    float L = 0.f;
+    for (int s = lane; s < splits; s += 32) { const float w = (M > -INFINITY) ? exp2f(sw[s] - M) : 0.f; sw[s] = w; L += w; }
+    L = warp_sum(L);
+    const float inv = L > 0.f ? 1.f / L : 0.f;
+    __syncwarp();
+    for (int s = lane; s < splits; s += 32) sw[s] *= inv;
+    if (lse && lane == 0) lse[row] = (M > -INFINITY) ? (M + log2f(L)) * kLn2 : -INFINITY;
   }
-  stf<T>(out, row * LOCKS_D + dim, acc);
-  if (lse && dim == 0) lse[row] = (M > -INFINITY) ? (M + log2f(L)) * kLn2 : -INFINITY;
+  __syncthreads();
+  const int sl = tid >> 5;
+  const float4 *po = reinterpret_cast<const float4 *>(part_o + row * splits * LOCKS_D) + lane;
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int s0 = sl; s0 < splits; s0 += 16) {
+    float4 v[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+      v[u] = (s0 + 4 * u < splits) ? __ldcg(po + (int64_t)(s0 + 4 * u) * (LOCKS_D / 4)) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const float w = (s0 + 4 * u < splits) ? sw[s0 + 4 * u] : 0.f;
+      acc.x += w * v[u].x; acc.y += w * v[u].y; acc.z += w * v[u].z; acc.w += w * v[u].w;
+    }
+  }
+  sacc[sl][lane] = acc;
+  __syncthreads();
+  if (sl == 0) {
+    const float4 a1 = sacc[1][lane], a2 = sacc[2][lane], a3 = sacc[3][lane];
+    acc.x += a1.x + a2.x + a3.x; acc.y += a1.y + a2.y + a3.y; acc.z += a1.z + a2.z + a3.z; acc.w += a1.w + a2.w + a3.w;
+    stf<T>(out, row * LOCKS_D + 4 * lane + 0, acc.x);
+    stf<T>(out, row * LOCKS_D + 4 * lane + 1, acc.y);
+    stf<T>(out, row * LOCKS_D + 4 * lane + 2, acc.z);
+    stf<T>(out, row * LOCKS_D + 4 * lane + 3, acc.w);
+  }
 }
 
 }  // namespace
@@ -455,6 +484,9 @@ int locks_launch_attend(locks_ctx *c, const void *q, const locks_kv *kv, int bat
   p.pages_per_cta = (npages + splits - 1) / splits;
   p.splits = (npages + p.pages_per_cta - 1) / p.pages_per_cta;
   p.done = c->att_done;
+  // a single CTA merging many splits of many heads is a serial tail: beyond 64 (head, split) pairs use the
+  // parallel merge kernel instead
+  p.fused_merge = (c->G * p.splits <= 64) ? 1 : 0;
   const bool bf = c->cfg.kv_dtype == LOCKS_BF16;
   if (bf) {
     static bool attr_done = false;
@@ -480,10 +512,12 @@ int locks_launch_attend(locks_ctx *c, const void *q, const locks_kv *kv, int bat
     locks_launch_pdl(attend_generic_kernel<float>, grid, dim3(128), 0, st, p);
   }
   int rc = locks_check_launch(c);
-  if (rc != LOCKS_OK || p.splits == 1 || bf) return rc;   // the bf16 kernel merges its own splits
+  if (rc != LOCKS_OK || p.splits == 1 || (bf && p.fused_merge)) return rc;
   dim3 mg(p.Hq, batch);
-  locks_launch_pdl(attend_merge_kernel<float>, mg, dim3(128), 0, st, (const float *)c->att_o, (const float *)c->att_lse,
-                   p.splits, reinterpret_cast<float *>(out), lse, p.Hq);
+  if (bf) locks_launch_pdl(attend_merge_kernel<__nv_bfloat16>, mg, dim3(128), 0, st, (const float *)c->att_o,
+                           (const float *)c->att_lse, p.splits, reinterpret_cast<__nv_bfloat16 *>(out), lse, p.Hq);
+  else locks_launch_pdl(attend_merge_kernel<float>, mg, dim3(128), 0, st, (const float *)c->att_o,
+                        (const float *)c->att_lse, p.splits, reinterpret_cast<float *>(out), lse, p.Hq);
   return locks_check_launch(c);
 }
 
@@ -566,6 +600,7 @@ extern "C" int locks_sparse_attend_noalloc(const locks_config *cfg, const void *
   if (splits < 1) splits = 1;
   p.pages_per_cta = (npages + splits - 1) / splits;
   p.splits = (npages + p.pages_per_cta - 1) / p.pages_per_cta;
+  p.fused_merge = 1;
   // the array keeps whatever the last call left: the arrival counters and the status word must start at zero
   if (cudaMemsetAsync(p.done, 0, kNoAllocDone + 256, st) != cudaSuccess) return LOCKS_ERR_CUDA;
   dim3 grid(p.splits, p.Hkv, batch);

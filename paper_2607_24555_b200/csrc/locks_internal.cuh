@@ -26,6 +26,7 @@ struct locks_ctx {
   locks_config cfg;
   int G, k, S, Pmax, max_groups;
   int num_sms;
+  int part_slots;          // partial slots per (request, head) the last scan launch may have filled
   int sel_ept;             // pages per thread in select stage 1
   int sel_chunks;          // select stage-1 CTAs per (request, KV head)
   int sel_kc;              // candidates kept per chunk (k-2)
@@ -34,7 +35,7 @@ struct locks_ctx {
   size_t ws_bytes;
   int32_t *status;         // [4] sticky status, work counters
   float *shat;             // [max_batch][Hq][Pmax]
-  float2 *part;            // [max_batch][Hq][max_groups] per-group (max, sum exp) of candidates
+  float2 *part;            // [max_batch][Hq][max_groups] partial (max, sum exp) over candidate pages
   float *logz;             // [max_batch][Hq] log Z_g (chunked selection only)
   float *cand_val;         // [max_batch][Hkv][sel_chunks][sel_kc]
   int32_t *cand_idx;

@@ -354,6 +354,37 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4r8_ker
     sum8 = 8.f * acc;
   };
 
+  // candidate partial (max, sum exp) of the current problem, kept per lane and reduced across the warp
+  // only when the warp moves on: one (head, warp) partial per problem instead of one per group
+  float pm[NH], ps[NH];
+#pragma unroll
+  for (int hh = 0; hh < NH; ++hh) { pm[hh] = -INFINITY; ps[hh] = 0.f; }
+  int cur_b = 0, cur_h = 0;
+  auto accumulate = [&](float &m, float &sacc, float v) {   // online log-sum-exp, one exp per value
+    if (v > -INFINITY) {
+      const float d = v - m, e = __expf(-fabsf(d));
+      if (d > 0.f) { sacc = sacc * e + 1.f; m = v; } else sacc += e;
+    }
+  };
+  auto flush = [&]() {
+#pragma unroll
+    for (int hh = 0; hh < NH; ++hh) {
+      float m = pm[hh], sacc = ps[hh];
+#pragma unroll
+      for (int o = 1; o <= 16; o <<= 1) {
+        if (o == 4 || o == 8 || (o == 16 && !PK)) continue;   // lanes sharing a head: t (1, 2) and, packed, x bit 2
+        const float om = __shfl_xor_sync(0xffffffffu, m, o), os = __shfl_xor_sync(0xffffffffu, sacc, o);
+        const float nm = fmaxf(m, om);
+        if (nm > -INFINITY) { sacc = sacc * __expf(m - nm) + os * __expf(om - nm); m = nm; }
+      }
+      const int g = PK ? (x & 3) : x + 8 * hh;
+      if (t == 0 && (!PK || x < 4) && g < p.G)
+        p.part[((int64_t)cur_b * p.Hq + cur_h * p.G + g) * p.max_groups + sub] = make_float2(m, sacc);
+      pm[hh] = -INFINITY;
+      ps[hh] = 0.f;
+    }
+  };
+
   int it = 0;
   bool ok = true;
   while (cc.prob < nprob) {
@@ -372,7 +403,10 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4r8_ker
     --inflight;
     const int b = cc.b, h = cc.h;
     if (cc.prob != cur_prob) {
+      if (cur_prob >= 0) flush();
       cur_prob = cc.prob;
+      cur_b = b;
+      cur_h = h;
 #pragma unroll
       for (int hh = 0; hh < NH; ++hh) {
         float s8;
@@ -532,17 +566,7 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4r8_ker
       const float v = res[0] * kLn2;
       const bool in = t < LOCKS_GROUP / 2 && page < cc.nsc;
       if (g < p.G && in) p.shat[((int64_t)b * p.Hq + h * p.G + g) * p.Pmax + page] = v;
-      const float c0 = (in && page >= 1) ? v : -INFINITY;
-      float m = c0;
-      m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 1));
-      m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 2));
-      m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 16));
-      float e = (m == -INFINITY) ? 0.f : __expf(c0 - m);
-      e += __shfl_xor_sync(0xffffffffu, e, 1);
-      e += __shfl_xor_sync(0xffffffffu, e, 2);
-      e += __shfl_xor_sync(0xffffffffu, e, 16);
-      if (t == 0 && x < 4 && g < p.G)
-        p.part[((int64_t)b * p.Hq + h * p.G + g) * p.max_groups + cc.grp] = make_float2(m, e);
+      accumulate(pm[0], ps[0], (in && page >= 1) ? v : -INFINITY);
     } else {
     const int page0 = cc.grp * LOCKS_GROUP + 2 * t;
 #pragma unroll
@@ -556,22 +580,15 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4r8_ker
         if (in0) dst[0] = v0;
         if (in1) dst[1] = v1;
       }
-      const float c0 = (in0 && page0 >= 1) ? v0 : -INFINITY;
-      const float c1v = in1 ? v1 : -INFINITY;
-      float m = fmaxf(c0, c1v);
-      m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 1));
-      m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 2));
-      float e = (m == -INFINITY) ? 0.f : (__expf(c0 - m) + __expf(c1v - m));
-      e += __shfl_xor_sync(0xffffffffu, e, 1);
-      e += __shfl_xor_sync(0xffffffffu, e, 2);
-      if (t == 0 && g < p.G)
-        p.part[((int64_t)b * p.Hq + h * p.G + g) * p.max_groups + cc.grp] = make_float2(m, e);
+      accumulate(pm[hh], ps[hh], (in0 && page0 >= 1) ? v0 : -INFINITY);
+      accumulate(pm[hh], ps[hh], in1 ? v1 : -INFINITY);
     }
     }
     cc.grp += wpp;
     settle(cc);
     ++it;
   }
+  if (ok && cur_prob >= 0) flush();
   if (!ok) {
     // a wait ran out: flag it, then give copies still in flight a bounded chance to land before exit
     if (lane == 0) set_status(p.status, LOCKS_ERR_TIMEOUT);
@@ -598,6 +615,7 @@ int locks_launch_scan(locks_ctx *c, const void *q, const void *summaries, const 
   p.Pmax = c->Pmax; p.max_groups = c->max_groups; p.num_blocks = kv->num_blocks; p.k = c->k;
   p.S = c->S; p.r = c->cfg.rank; p.sm_scale = c->cfg.sm_scale;
   const bool tensor = c->cfg.summary_fmt == LOCKS_FMT_I4 && c->cfg.rank == 8 && c->cfg.q_dtype == LOCKS_BF16;
+  c->part_slots = c->max_groups;   // generic kernel: one partial per 8-page group
   if (tensor) {
     static bool attr_done = false;
     if (!attr_done) {
@@ -610,6 +628,10 @@ int locks_launch_scan(locks_ctx *c, const void *q, const void *summaries, const 
     int grid = kScanCtasPerSm * c->num_sms;
     const int need = (total_groups + kScanWarps - 1) / kScanWarps;
     if (grid > need) grid = need < 1 ? 1 : need;
+    {   // tensor kernel: one partial per (problem, warp); mirrors the kernel's own partition
+      const int W = grid * kScanWarps, nprob = batch * p.Hkv;
+      c->part_slots = W / nprob > 1 ? W / nprob : 1;
+    }
     if (c->G <= 4) locks_launch_pdl(scan_i4r8_kernel<1, true>, dim3(grid), dim3(kScanWarps * 32), kScanSmem, st, p);
     else if (c->G <= 8) locks_launch_pdl(scan_i4r8_kernel<1, false>, dim3(grid), dim3(kScanWarps * 32), kScanSmem, st, p);
     else locks_launch_pdl(scan_i4r8_kernel<2, false>, dim3(grid), dim3(kScanWarps * 32), kScanSmem, st, p);

@@ -2,15 +2,19 @@
 //   log Z_g   = log sum_{j in 1..P-2} exp s^_j(q_g)                       (candidates only)
 //   log m_bar_j = log( (1/G) sum_g exp(s^_j(q_g) - log Z_g) )
 //   S = {0, P-1}  U  top-(k-2) candidates by log m_bar_j (ties: lower page index), ids ascending.
-// Stage 1 (one CTA per chunk of up to 8192 pages of a (request, KV head)) ranks its chunk with an exact
-// 4-pass radix select held in registers + shared-memory histograms and compacts the winners in
-// page order.  With one chunk it writes the final table; with several, each chunk emits its own
-// top-(k-2) (value, page) list and stage 2 re-selects among them (a chunk's local top-(k-2) always
-// contains the chunk's share of the global top-(k-2), ties included, because both use the same
-// lower-index tie rule and lists stay in page order).
+// Stage 1 (one 512-thread CTA per chunk of 2048 / 4096 / 8192 pages of a (request, KV head)) ranks its
+// chunk with an exact 4-pass radix select over keys held in registers and compacts the winners in
+// page order.  With one chunk it writes the final table; with several, log Z comes from a small
+// reduction kernel, each chunk emits its own top-(k-2) (value, page) list and stage 2 re-selects
+// among them (a chunk's local top-(k-2) always contains the chunk's share of the global top-(k-2),
+// ties included, because both use the same lower-index tie rule and lists stay in page order).
+// Pages are dealt to threads round-robin (element i of thread t is page i*512 + t), so loads are
+// coalesced and every thread is busy whatever the context length.
 #include "locks_internal.cuh"
 
 namespace {
+
+constexpr int kNW = LOCKS_SEL_THREADS / 32;
 
 struct SelParams {
   const float *shat;
@@ -21,7 +25,15 @@ struct SelParams {
   float *cand_val;
   int32_t *cand_idx;
   float *logz;      // [batch][Hq] log Z_g, written by logz_kernel when a problem spans several chunks
-  int batch, Hq, Hkv, G, Pmax, max_groups, k, chunks, kc, chunk_pages;
+  int batch, Hq, Hkv, G, Pmax, max_groups, k, chunks, kc, chunk_pages, part_slots;
+};
+
+struct SelShared {
+  int hist[kNW * 256];   // one 256-bin histogram per warp
+  int misc[16];          // per-pass result (double-buffered)
+  int wsum[8];
+  int cnt[16 * kNW];     // per (slab, warp) winner counts for the ordered compaction
+  float logz[16];
 };
 
 __device__ __forceinline__ uint32_t order_key(float f) {
@@ -29,17 +41,14 @@ __device__ __forceinline__ uint32_t order_key(float f) {
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
-// Exact top-K among the block's N = THREADS*EPT keys (thread-major order = ascending index order).
+// Exact top-K among the block's N = 512*EPT keys; element i of thread t has index i*512 + t.
 // sel[i] is set for the K winners: every key above the K-th largest, plus the lowest-indexed keys
 // equal to it.  pos[i] = rank of a winner in index order.  Requires K <= number of valid keys.
-// Four 8-bit radix passes.  Every warp counts into its own 256-bin histogram (page masses share their
+// Four 8-bit radix passes.  Every warp counts into its own histogram (page masses share their
 // leading bits, so a shared histogram would serialise all warps on one or two counters); bin b of
-// the block is then summed and suffix-scanned by thread b.
-// sh_hist: warps x 256 ints (zero on entry and on exit), sh_misc: 12 ints.
+// the block is then summed and suffix-scanned by thread 255 - b.  sh.hist must be zero on entry.
 template <int EPT>
-__device__ void block_topk(const uint32_t (&key)[EPT], int K, bool (&sel)[EPT], int (&pos)[EPT], int *sh_hist,
-                           int *sh_misc) {
-  constexpr int NW = LOCKS_SEL_THREADS / 32;
+__device__ void block_topk(const uint32_t (&key)[EPT], int K, bool (&sel)[EPT], int (&pos)[EPT], SelShared &sh) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   if (K <= 0) {  // nothing to pick (k = 2): uniform across the block
 #pragma unroll
@@ -50,91 +59,95 @@ __device__ void block_topk(const uint32_t (&key)[EPT], int K, bool (&sel)[EPT], 
   int remaining = K;
   for (int pass = 0; pass < 4; ++pass) {
     const int shift = 24 - 8 * pass;
-    int *mine = sh_hist + warp * 256;
+    int *mine = sh.hist + warp * 256;
 #pragma unroll
     for (int i = 0; i < EPT; ++i)
       if ((key[i] & mask) == prefix) atomicAdd(&mine[(key[i] >> shift) & 255], 1);
     __syncthreads();
     int c = 0, incl = 0;
-    if (tid < 256) {   // thread b owns bin 255 - b: bins are scanned from the largest digit down
+    if (tid < 256) {   // thread t owns bin 255 - t: bins are scanned from the largest digit down
       const int bin = 255 - tid;
 #pragma unroll
-      for (int w = 0; w < NW; ++w) { c += sh_hist[w * 256 + bin]; sh_hist[w * 256 + bin] = 0; }
+      for (int w = 0; w < kNW; ++w) { c += sh.hist[w * 256 + bin]; sh.hist[w * 256 + bin] = 0; }
       incl = c;
 #pragma unroll
       for (int o = 1; o < 32; o <<= 1) {
         int v = __shfl_up_sync(0xffffffffu, incl, o);
         if (lane >= o) incl += v;
       }
-      if (lane == 31) sh_misc[4 + warp] = incl;
+      if (lane == 31) sh.wsum[warp] = incl;
     }
     __syncthreads();
     if (tid < 256) {
       int before = incl - c;
-      for (int w = 0; w < warp; ++w) before += sh_misc[4 + w];
+      for (int w = 0; w < warp; ++w) before += sh.wsum[w];
       if (before < remaining && remaining <= before + c) {
-        sh_misc[(pass & 1) * 2] = 255 - tid;
-        sh_misc[(pass & 1) * 2 + 1] = remaining - before;
+        sh.misc[(pass & 1) * 2] = 255 - tid;
+        sh.misc[(pass & 1) * 2 + 1] = remaining - before;
       }
     }
     __syncthreads();
-    prefix |= (uint32_t)sh_misc[(pass & 1) * 2] << shift;
+    prefix |= (uint32_t)sh.misc[(pass & 1) * 2] << shift;
     mask |= 255u << shift;
-    remaining = sh_misc[(pass & 1) * 2 + 1];
+    remaining = sh.misc[(pass & 1) * 2 + 1];
   }
-  // prefix is the K-th largest key; `remaining` of the keys equal to it are taken, lowest index first
-  int ngt = 0, neq = 0;
-#pragma unroll
-  for (int i = 0; i < EPT; ++i) { ngt += key[i] > prefix; neq += key[i] == prefix; }
-  // block exclusive scan of (ngt, neq) packed into one int
-  int packed = (ngt << 16) | neq;
-  int incl = packed;
-#pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    int v = __shfl_up_sync(0xffffffffu, incl, o);
-    if (lane >= o) incl += v;
-  }
-  __syncthreads();   // the last pass's readers of sh_misc[4..] are done
-  if (lane == 31) sh_misc[12 + warp] = incl;
-  __syncthreads();
-  int base = 0;
-  for (int w = 0; w < warp; ++w) base += sh_misc[12 + w];
-  int excl = base + incl - packed;
-  int gt_before = excl >> 16, eq_before = excl & 0xffff;
+  // prefix is the K-th largest key; `remaining` of the keys equal to it are taken, lowest index first.
+  // Ordered compaction: slab i holds indices i*512 .. i*512+511, one per thread.
+  uint32_t bg[EPT], be[EPT];
 #pragma unroll
   for (int i = 0; i < EPT; ++i) {
+    bg[i] = __ballot_sync(0xffffffffu, key[i] > prefix);
+    be[i] = __ballot_sync(0xffffffffu, key[i] == prefix);
+    if (lane == 0) sh.cnt[i * kNW + warp] = (__popc(bg[i]) << 16) | __popc(be[i]);
+  }
+  __syncthreads();
+  if (warp == 0) {   // exclusive scan of the EPT*kNW counts in (slab, warp) order
+    constexpr int N = EPT * kNW, PER = (N + 31) / 32;
+    int v[PER], tot = 0;
+#pragma unroll
+    for (int u = 0; u < PER; ++u) { const int e = lane * PER + u; v[u] = e < N ? sh.cnt[e] : 0; tot += v[u]; }
+    int incl = tot;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      int x = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += x;
+    }
+    int run = incl - tot;
+#pragma unroll
+    for (int u = 0; u < PER; ++u) { const int e = lane * PER + u; if (e < N) sh.cnt[e] = run; run += v[u]; }
+  }
+  __syncthreads();
+  const uint32_t lt = (1u << lane) - 1u;
+#pragma unroll
+  for (int i = 0; i < EPT; ++i) {
+    const int base = sh.cnt[i * kNW + warp];
+    const int gt_before = (base >> 16) + __popc(bg[i] & lt), eq_before = (base & 0xffff) + __popc(be[i] & lt);
     const bool gt = key[i] > prefix, eq = key[i] == prefix;
-    const bool take = gt || (eq && eq_before < remaining);
-    sel[i] = take;
+    sel[i] = gt || (eq && eq_before < remaining);
     pos[i] = gt_before + min(eq_before, remaining);
-    gt_before += gt;
-    eq_before += eq;
+  }
+}
+
+__device__ __forceinline__ void lse_merge(float &m, float &s, float om, float os) {
+  const float nm = fmaxf(m, om);
+  if (nm > -INFINITY) {
+    s = s * __expf(m - nm) + os * __expf(om - nm);
+    m = nm;
   }
 }
 
 // log Z_g of every head of the group from the scan's per-group partials -> sh_logz[g]
 __device__ void group_logz(const SelParams &p, int b, int h, int ngroups, float *sh_logz) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  for (int g = warp; g < p.G; g += LOCKS_SEL_THREADS / 32) {
+  for (int g = warp; g < p.G; g += kNW) {
     const float2 *pp = p.part + ((int64_t)b * p.Hq + h * p.G + g) * p.max_groups;
     float m = -INFINITY, s = 0.f;
     for (int i = lane; i < ngroups; i += 32) {
       const float2 v = pp[i];
-      if (v.x > -INFINITY) {
-        const float nm = fmaxf(m, v.x);
-        s = s * __expf(m - nm) + v.y * __expf(v.x - nm);
-        m = nm;
-      }
+      if (v.x > -INFINITY) lse_merge(m, s, v.x, v.y);
     }
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      const float om = __shfl_xor_sync(0xffffffffu, m, o), os = __shfl_xor_sync(0xffffffffu, s, o);
-      const float nm = fmaxf(m, om);
-      if (nm > -INFINITY) {
-        s = s * __expf(m - nm) + os * __expf(om - nm);
-        m = nm;
-      }
-    }
+    for (int o = 16; o > 0; o >>= 1) lse_merge(m, s, __shfl_xor_sync(0xffffffffu, m, o), __shfl_xor_sync(0xffffffffu, s, o));
     if (lane == 0) sh_logz[g] = m + __logf(s);
   }
 }
@@ -148,44 +161,35 @@ __global__ void __launch_bounds__(256) logz_kernel(SelParams p) {
   const int T = p.seq_lens[b];
   const int P = (T + LOCKS_B - 1) / LOCKS_B;
   if (P <= p.k) return;
-  const int ngroups = (P - 1 + LOCKS_GROUP - 1) / LOCKS_GROUP;
+  const int nparts = min(p.part_slots, (P - 1 + LOCKS_GROUP - 1) / LOCKS_GROUP);
   const float2 *pp = p.part + ((int64_t)b * p.Hq + hq) * p.max_groups;
   float m = -INFINITY, s = 0.f;
-  for (int i = threadIdx.x; i < ngroups; i += 256) {
-    const float2 v = pp[i];
-    if (v.x > -INFINITY) {
-      const float nm = fmaxf(m, v.x);
-      s = s * __expf(m - nm) + v.y * __expf(v.x - nm);
-      m = nm;
-    }
+  for (int i0 = threadIdx.x; i0 < nparts; i0 += 256 * 4) {   // four loads in flight per thread
+    float2 v[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) v[u] = (i0 + 256 * u < nparts) ? pp[i0 + 256 * u] : make_float2(-INFINITY, 0.f);
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+      if (v[u].x > -INFINITY) lse_merge(m, s, v[u].x, v[u].y);
   }
 #pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-    const float om = __shfl_xor_sync(0xffffffffu, m, o), os = __shfl_xor_sync(0xffffffffu, s, o);
-    const float nm = fmaxf(m, om);
-    if (nm > -INFINITY) { s = s * __expf(m - nm) + os * __expf(om - nm); m = nm; }
-  }
+  for (int o = 16; o > 0; o >>= 1) lse_merge(m, s, __shfl_xor_sync(0xffffffffu, m, o), __shfl_xor_sync(0xffffffffu, s, o));
   if (lane == 0) { sm_m[warp] = m; sm_s[warp] = s; }
   __syncthreads();
   if (threadIdx.x == 0) {
     float M = -INFINITY, S = 0.f;
-    for (int w = 0; w < 8; ++w) {
-      const float nm = fmaxf(M, sm_m[w]);
-      if (nm > -INFINITY) { S = S * __expf(M - nm) + sm_s[w] * __expf(sm_m[w] - nm); M = nm; }
-    }
+    for (int w = 0; w < 8; ++w) lse_merge(M, S, sm_m[w], sm_s[w]);
     p.logz[b * p.Hq + hq] = M + __logf(S);
   }
 }
 
 template <int EPT>
 __global__ void __launch_bounds__(LOCKS_SEL_THREADS) select_stage1_kernel(SelParams p) {
-  __shared__ int sh_hist[(LOCKS_SEL_THREADS / 32) * 256];
-  __shared__ int sh_misc[12 + LOCKS_SEL_THREADS / 32];
-  __shared__ float sh_logz[16];
-  for (int e = threadIdx.x; e < (LOCKS_SEL_THREADS / 32) * 256; e += LOCKS_SEL_THREADS) sh_hist[e] = 0;
+  __shared__ SelShared sh;
+  const int chunk = blockIdx.x, h = blockIdx.y, b = blockIdx.z, tid = threadIdx.x;
+  for (int e = tid; e < kNW * 256; e += LOCKS_SEL_THREADS) sh.hist[e] = 0;
   pdl_trigger();
   pdl_wait();   // the scan's scores and partials
-  const int chunk = blockIdx.x, h = blockIdx.y, b = blockIdx.z, tid = threadIdx.x;
   const int T = p.seq_lens[b];
   const int P = (T + LOCKS_B - 1) / LOCKS_B;
   const int64_t prob = (int64_t)b * p.Hkv + h;
@@ -207,21 +211,24 @@ __global__ void __launch_bounds__(LOCKS_SEL_THREADS) select_stage1_kernel(SelPar
     return;
   }
   // scores of the first heads are fetched before the log Z reduction so that the two latencies overlap
-  constexpr int PRE = EPT <= 8 ? 4 : 1;
-  const int pbase = c0 + tid * EPT;
+  constexpr int PRE = EPT <= 8 ? 4 : 2;
   const float *row0 = p.shat + ((int64_t)b * p.Hq + h * p.G) * p.Pmax;
+  bool valid[EPT];
   float raw[PRE][EPT];
+#pragma unroll
+  for (int i = 0; i < EPT; ++i) {
+    const int page = c0 + i * LOCKS_SEL_THREADS + tid;
+    valid[i] = page >= 1 && page <= P - 2;
+  }
 #pragma unroll
   for (int g = 0; g < PRE; ++g)
 #pragma unroll
-    for (int i = 0; i < EPT; ++i) {
-      const int page = pbase + i;
-      raw[g][i] = (g < p.G && page >= 1 && page <= P - 2) ? row0[(int64_t)g * p.Pmax + page] : 0.f;
-    }
-  if (p.chunks == 1) group_logz(p, b, h, (P - 1 + LOCKS_GROUP - 1) / LOCKS_GROUP, sh_logz);
-  else if (tid < p.G) sh_logz[tid] = p.logz[b * p.Hq + h * p.G + tid];
+    for (int i = 0; i < EPT; ++i)
+      raw[g][i] = (g < p.G && valid[i]) ? row0[(int64_t)g * p.Pmax + c0 + i * LOCKS_SEL_THREADS + tid] : 0.f;
+  if (p.chunks == 1) group_logz(p, b, h, min(p.part_slots, (P - 1 + LOCKS_GROUP - 1) / LOCKS_GROUP), sh.logz);
+  else if (tid < p.G) sh.logz[tid] = p.logz[b * p.Hq + h * p.G + tid];
   __syncthreads();
-  // log m_bar of this thread's EPT consecutive pages: log mean_g exp(s^_g - log Z_g)
+  // log m_bar of this thread's pages: log mean_g exp(s^_g - log Z_g)
   float val[EPT];
   uint32_t key[EPT];
   const float logG = __logf((float)p.G);
@@ -232,51 +239,38 @@ __global__ void __launch_bounds__(LOCKS_SEL_THREADS) select_stage1_kernel(SelPar
 #pragma unroll
     for (int g = 0; g < PRE; ++g) {
       if (g < p.G) {
-        const float lz = sh_logz[g];
+        const float lz = sh.logz[g];
 #pragma unroll
-        for (int i = 0; i < EPT; ++i) {
-          const int page = pbase + i;
-          if (page >= 1 && page <= P - 2) {
-            const float tv = raw[g][i] - lz;
-            const float nm = fmaxf(mx[i], tv);
-            sm[i] = sm[i] * __expf(mx[i] - nm) + __expf(tv - nm);
-            mx[i] = nm;
-          }
-        }
+        for (int i = 0; i < EPT; ++i)
+          if (valid[i]) lse_merge(mx[i], sm[i], raw[g][i] - lz, 1.f);
       }
     }
     for (int g = PRE; g < p.G; ++g) {
-      const float *row = row0 + (int64_t)g * p.Pmax;
-      const float lz = sh_logz[g];
+      const float *row = row0 + (int64_t)g * p.Pmax + c0 + tid;
+      const float lz = sh.logz[g];
+      float tv[EPT];
 #pragma unroll
-      for (int i = 0; i < EPT; ++i) {
-        const int page = pbase + i;
-        if (page >= 1 && page <= P - 2) {
-          const float tv = row[page] - lz;
-          const float nm = fmaxf(mx[i], tv);
-          sm[i] = sm[i] * __expf(mx[i] - nm) + __expf(tv - nm);
-          mx[i] = nm;
-        }
-      }
+      for (int i = 0; i < EPT; ++i) tv[i] = valid[i] ? row[i * LOCKS_SEL_THREADS] : 0.f;
+#pragma unroll
+      for (int i = 0; i < EPT; ++i)
+        if (valid[i]) lse_merge(mx[i], sm[i], tv[i] - lz, 1.f);
     }
 #pragma unroll
     for (int i = 0; i < EPT; ++i) {
-      const int page = pbase + i;
-      const bool valid = page >= 1 && page <= P - 2;
-      val[i] = valid ? mx[i] + __logf(sm[i]) - logG : -INFINITY;
-      key[i] = valid ? order_key(val[i]) : 0u;
-      if (valid && p.logshare) p.logshare[prob * p.Pmax + page] = val[i];
+      val[i] = valid[i] ? mx[i] + __logf(sm[i]) - logG : -INFINITY;
+      key[i] = valid[i] ? order_key(val[i]) : 0u;
+      if (valid[i] && p.logshare) p.logshare[prob * p.Pmax + c0 + i * LOCKS_SEL_THREADS + tid] = val[i];
     }
   }
   const int cand_in_chunk = min(P - 2, c0 + p.chunk_pages - 1) - max(1, c0) + 1;
   const int K = min(p.k - 2, cand_in_chunk);
   bool sel[EPT];
   int pos[EPT];
-  block_topk<EPT>(key, K, sel, pos, sh_hist, sh_misc);
+  block_topk<EPT>(key, K, sel, pos, sh);
   if (p.chunks == 1) {
 #pragma unroll
     for (int i = 0; i < EPT; ++i)
-      if (sel[i]) ids[1 + pos[i]] = pbase + i;
+      if (sel[i]) ids[1 + pos[i]] = c0 + i * LOCKS_SEL_THREADS + tid;
     if (tid == 0) {
       ids[0] = 0;
       ids[p.k - 1] = P - 1;
@@ -287,17 +281,16 @@ __global__ void __launch_bounds__(LOCKS_SEL_THREADS) select_stage1_kernel(SelPar
     int32_t *ci = p.cand_idx + (prob * p.chunks + chunk) * p.kc;
 #pragma unroll
     for (int i = 0; i < EPT; ++i)
-      if (sel[i]) { cv[pos[i]] = val[i]; ci[pos[i]] = pbase + i; }
+      if (sel[i]) { cv[pos[i]] = val[i]; ci[pos[i]] = c0 + i * LOCKS_SEL_THREADS + tid; }
     for (int j = K + tid; j < p.kc; j += LOCKS_SEL_THREADS) { cv[j] = -INFINITY; ci[j] = -1; }
   }
 }
 
 template <int EPT>
 __global__ void __launch_bounds__(LOCKS_SEL_THREADS) select_stage2_kernel(SelParams p) {
-  __shared__ int sh_hist[(LOCKS_SEL_THREADS / 32) * 256];
-  __shared__ int sh_misc[12 + LOCKS_SEL_THREADS / 32];
+  __shared__ SelShared sh;
   const int h = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
-  for (int e = tid; e < (LOCKS_SEL_THREADS / 32) * 256; e += LOCKS_SEL_THREADS) sh_hist[e] = 0;
+  for (int e = tid; e < kNW * 256; e += LOCKS_SEL_THREADS) sh.hist[e] = 0;
   pdl_trigger();
   pdl_wait();   // stage 1's candidate lists
   __syncthreads();
@@ -312,14 +305,14 @@ __global__ void __launch_bounds__(LOCKS_SEL_THREADS) select_stage2_kernel(SelPar
   int idx[EPT];
 #pragma unroll
   for (int i = 0; i < EPT; ++i) {
-    const int j = tid * EPT + i;
-    const bool valid = j < N && ci[j] >= 0;
-    idx[i] = valid ? ci[j] : -1;
-    key[i] = valid ? order_key(cv[j]) : 0u;
+    const int j = i * LOCKS_SEL_THREADS + tid;   // list position = ascending page order
+    const bool ok = j < N && ci[j] >= 0;
+    idx[i] = ok ? ci[j] : -1;
+    key[i] = ok ? order_key(cv[j]) : 0u;
   }
   bool sel[EPT];
   int pos[EPT];
-  block_topk<EPT>(key, p.k - 2, sel, pos, sh_hist, sh_misc);
+  block_topk<EPT>(key, p.k - 2, sel, pos, sh);
   int32_t *ids = p.ids + prob * p.k;
 #pragma unroll
   for (int i = 0; i < EPT; ++i)
@@ -342,6 +335,7 @@ int locks_launch_select(locks_ctx *c, const float *shat, const locks_kv *kv, int
   p.max_groups = c->max_groups; p.k = c->k; p.chunks = c->sel_chunks; p.kc = c->sel_kc;
   p.chunk_pages = c->sel_ept * LOCKS_SEL_THREADS;
   p.logz = c->logz;
+  p.part_slots = c->part_slots;
   if (c->sel_chunks > 1) {
     locks_launch_pdl(logz_kernel, dim3(p.Hq, batch), dim3(256), 0, st, p);
     int rc0 = locks_check_launch(c);
