@@ -164,9 +164,13 @@ int locks_last_launch_count(const locks_ctx *ctx);
  * locks_profile_begin(ctx, max_steps) every locks_decode_step records CUDA events on its stream at
  * the stage boundaries; locks_profile_end() synchronises the device, writes the mean duration in
  * milliseconds of {prologue, summary scan, selection, sparse attention} to stage_ms[4], the number
- * of steps seen to *steps, and releases the events.  Not legal while the stream is being captured. */
+ * of steps seen to *steps, and releases the events. */
 int locks_profile_begin(locks_ctx *ctx, int max_steps);
 int locks_profile_end(locks_ctx *ctx, float *stage_ms, int *steps);
+/* A locks_decode_step CAPTURED while profiling is on records the same stage boundaries as event
+ * nodes of the graph (always into the first slot).  After a replay, locks_profile_read()
+ * synchronises `stream` and writes that replay's four stage durations (ms) to stage_ms[4]. */
+int locks_profile_read(locks_ctx *ctx, float *stage_ms, locks_stream stream);
 
 /* locks_sparse_attend for callers that cannot allocate device memory (the paper has no
  * counterpart; this is a convenience of the library).  Some hosts of this code may not call

@@ -16,7 +16,7 @@ FMT_F32, FMT_I4 = 0, 1
 SYMBOLS = ["locks_summary_bytes", "locks_workspace_bytes", "locks_create", "locks_destroy",
            "locks_build_summaries", "locks_select", "locks_sparse_attend", "locks_decode_step",
            "locks_decode_step_host", "locks_poll_status", "locks_last_launch_count", "locks_strerror",
-           "locks_profile_begin", "locks_profile_end", "locks_sparse_attend_noalloc"]
+           "locks_profile_begin", "locks_profile_end", "locks_profile_read", "locks_sparse_attend_noalloc"]
 
 
 class LocksError(RuntimeError):
@@ -67,6 +67,8 @@ def lib():
         L.locks_last_launch_count.argtypes = [vp]
         L.locks_profile_begin.argtypes = [vp, C.c_int]
         L.locks_profile_end.argtypes = [vp, C.POINTER(C.c_float), C.POINTER(C.c_int)]
+        L.locks_profile_read.argtypes = [vp, C.POINTER(C.c_float), vp]
+        L.locks_profile_read.restype = C.c_int
         L.locks_profile_begin.restype = C.c_int
         L.locks_profile_end.restype = C.c_int
         L.locks_sparse_attend_noalloc.argtypes = [C.POINTER(Config), vp, C.POINTER(KV), C.c_int, i32p, i32p, vp, vp, vp]
@@ -214,6 +216,11 @@ class Context:
         n = C.c_int(0)
         _check(lib().locks_profile_end(self.handle, ms, C.byref(n)), "locks_profile_end")
         return {"prologue": ms[0], "scan": ms[1], "select": ms[2], "attend": ms[3]}, int(n.value)
+
+    def locks_profile_read(self, stream=None):
+        ms = (C.c_float * 4)()
+        _check(lib().locks_profile_read(self.handle, ms, _stream(stream)), "locks_profile_read")
+        return {"prologue": ms[0], "scan": ms[1], "select": ms[2], "attend": ms[3]}
 
     def locks_last_launch_count(self) -> int:
         return int(lib().locks_last_launch_count(self.handle))

@@ -215,7 +215,15 @@ int locks_decode_step(locks_ctx *ctx, const void *q, const void *k_new, const vo
   int32_t *cnt = page_count ? page_count : ctx->cnt_int;
   ctx->last_launches = 0;
   cudaEvent_t *pe = (ctx->prof_ev && ctx->prof_n < ctx->prof_cap) ? ctx->prof_ev + ctx->prof_n * LOCKS_PROF_MARKS : nullptr;
-  auto mark = [&](int i) { if (pe) cudaEventRecord(pe[i], st); };
+  cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+  if (pe) cudaStreamIsCapturing(st, &cap);
+  const bool capturing = cap == cudaStreamCaptureStatusActive;
+  if (pe && capturing) pe = ctx->prof_ev;   // a captured step always reports through slot 0
+  auto mark = [&](int i) {
+    if (!pe) return;
+    if (capturing) cudaEventRecordWithFlags(pe[i], st, cudaEventRecordExternal);   // becomes an event-record node
+    else cudaEventRecord(pe[i], st);
+  };
   mark(0);
   if ((rc = locks_launch_prep(ctx, q, k_new, v_new, kv, batch, st)) != LOCKS_OK) return rc;
   mark(1);
@@ -231,7 +239,7 @@ int locks_decode_step(locks_ctx *ctx, const void *q, const void *k_new, const vo
   mark(3);
   if ((rc = locks_launch_attend(ctx, q, kv, batch, ids, cnt, out, nullptr, st)) != LOCKS_OK) return rc;
   mark(4);
-  if (pe) ctx->prof_n++;
+  if (pe && !capturing) ctx->prof_n++;
   if (cudaStreamWaitEvent(st, ctx->ev_join, 0) != cudaSuccess) return LOCKS_ERR_CUDA;
   return LOCKS_OK;
 }
@@ -289,6 +297,14 @@ int locks_profile_begin(locks_ctx *ctx, int max_steps) {
     if (cudaEventCreate(&ctx->prof_ev[i]) != cudaSuccess) return LOCKS_ERR_CUDA;
   ctx->prof_cap = max_steps;
   ctx->prof_n = 0;
+  return LOCKS_OK;
+}
+
+int locks_profile_read(locks_ctx *ctx, float *stage_ms, locks_stream stream) {
+  if (!ctx || !ctx->prof_ev || !stage_ms) return LOCKS_ERR_INVALID_ARG;
+  if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return LOCKS_ERR_CUDA;
+  for (int s = 0; s < LOCKS_PROF_MARKS - 1; ++s)
+    if (cudaEventElapsedTime(&stage_ms[s], ctx->prof_ev[s], ctx->prof_ev[s + 1]) != cudaSuccess) return LOCKS_ERR_CUDA;
   return LOCKS_OK;
 }
 

@@ -48,7 +48,8 @@ __device__ __forceinline__ uint32_t order_key(float f) {
 // leading bits, so a shared histogram would serialise all warps on one or two counters); bin b of
 // the block is then summed and suffix-scanned by thread 255 - b.  sh.hist must be zero on entry.
 template <int EPT>
-__device__ void block_topk(const uint32_t (&key)[EPT], int K, bool (&sel)[EPT], int (&pos)[EPT], SelShared &sh) {
+__device__ void block_topk(const uint32_t (&key)[EPT], int K, bool (&sel)[EPT], int (&pos)[EPT], SelShared &sh,
+                           int nslab = EPT) {   // slabs >= nslab hold no valid key (uniform across the block)
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   if (K <= 0) {  // nothing to pick (k = 2): uniform across the block
 #pragma unroll
@@ -62,7 +63,7 @@ __device__ void block_topk(const uint32_t (&key)[EPT], int K, bool (&sel)[EPT], 
     int *mine = sh.hist + warp * 256;
 #pragma unroll
     for (int i = 0; i < EPT; ++i)
-      if ((key[i] & mask) == prefix) atomicAdd(&mine[(key[i] >> shift) & 255], 1);
+      if (i < nslab && (key[i] & mask) == prefix) atomicAdd(&mine[(key[i] >> shift) & 255], 1);
     __syncthreads();
     int c = 0, incl = 0;
     if (tid < 256) {   // thread t owns bin 255 - t: bins are scanned from the largest digit down
@@ -96,8 +97,11 @@ __device__ void block_topk(const uint32_t (&key)[EPT], int K, bool (&sel)[EPT], 
   uint32_t bg[EPT], be[EPT];
 #pragma unroll
   for (int i = 0; i < EPT; ++i) {
-    bg[i] = __ballot_sync(0xffffffffu, key[i] > prefix);
-    be[i] = __ballot_sync(0xffffffffu, key[i] == prefix);
+    bg[i] = be[i] = 0u;
+    if (i < nslab) {
+      bg[i] = __ballot_sync(0xffffffffu, key[i] > prefix);
+      be[i] = __ballot_sync(0xffffffffu, key[i] == prefix);
+    }
     if (lane == 0) sh.cnt[i * kNW + warp] = (__popc(bg[i]) << 16) | __popc(be[i]);
   }
   __syncthreads();
@@ -215,10 +219,13 @@ __global__ void __launch_bounds__(LOCKS_SEL_THREADS) select_stage1_kernel(SelPar
   const float *row0 = p.shat + ((int64_t)b * p.Hq + h * p.G) * p.Pmax;
   bool valid[EPT];
   float raw[PRE][EPT];
+  // slabs of 512 pages that hold at least one candidate of this chunk (the configured maximum context
+  // is usually longer than the sequence)
+  const int nslab = min(EPT, (min(P - 1, c0 + p.chunk_pages) - c0 + LOCKS_SEL_THREADS - 1) / LOCKS_SEL_THREADS);
 #pragma unroll
   for (int i = 0; i < EPT; ++i) {
     const int page = c0 + i * LOCKS_SEL_THREADS + tid;
-    valid[i] = page >= 1 && page <= P - 2;
+    valid[i] = i < nslab && page >= 1 && page <= P - 2;
   }
 #pragma unroll
   for (int g = 0; g < PRE; ++g)
@@ -250,7 +257,7 @@ __global__ void __launch_bounds__(LOCKS_SEL_THREADS) select_stage1_kernel(SelPar
       const float lz = sh.logz[g];
       float tv[EPT];
 #pragma unroll
-      for (int i = 0; i < EPT; ++i) tv[i] = valid[i] ? row[i * LOCKS_SEL_THREADS] : 0.f;
+      for (int i = 0; i < EPT; ++i) tv[i] = (i < nslab && valid[i]) ? row[i * LOCKS_SEL_THREADS] : 0.f;
 #pragma unroll
       for (int i = 0; i < EPT; ++i)
         if (valid[i]) lse_merge(mx[i], sm[i], tv[i] - lz, 1.f);
@@ -266,7 +273,7 @@ __global__ void __launch_bounds__(LOCKS_SEL_THREADS) select_stage1_kernel(SelPar
   const int K = min(p.k - 2, cand_in_chunk);
   bool sel[EPT];
   int pos[EPT];
-  block_topk<EPT>(key, K, sel, pos, sh);
+  block_topk<EPT>(key, K, sel, pos, sh, nslab);
   if (p.chunks == 1) {
 #pragma unroll
     for (int i = 0; i < EPT; ++i)
