@@ -281,7 +281,7 @@ def run_ours(args):
             with torch.cuda.graph(g, stream=stream):
                 step(li)
             pgraphs.append(g)
-        stage_ms = {"prologue": 0.0, "scan": 0.0, "select": 0.0, "attend": 0.0}
+        stage_ms = {"scan": 0.0, "select": 0.0, "attend": 0.0}
         for i in range(K + 2):
             pgraphs[(W + K + i) % L].replay()
             one = ctx.locks_profile_read(stream=stream)

@@ -137,6 +137,11 @@ int locks_sparse_attend(locks_ctx *ctx, const void *q, const locks_kv *kv, int b
  *   2. locks_select on the resident summaries;  3. locks_sparse_attend on the selected pages;
  *   4. if a page became complete at this step (T_b % B == 0) build its summary, so that it is a
  *      candidate from the next step on (the newly written token is never scored, App. E(i)).
+ * These are the results; inside, the token is counted from the first kernel on, its rows are written by
+ * the selector's kernel (no page summary depends on them) and seq_lens is stored back there, so the
+ * append costs no launch of its own.  k_new / v_new: device, 16-byte aligned.  A sequence whose
+ * block-table row is full keeps its length, nothing is written for it and LOCKS_ERR_BAD_BLOCK is
+ * recorded in the status word.
  * page_ids / page_count may be NULL (kept in the workspace). */
 int locks_decode_step(locks_ctx *ctx, const void *q, const void *k_new, const void *v_new,
                       locks_kv *kv, void *summaries, int batch, void *out, int32_t *page_ids,
@@ -163,13 +168,13 @@ int locks_last_launch_count(const locks_ctx *ctx);
  * step asked for when reporting where the time goes (the paper reports none per kernel).  After
  * locks_profile_begin(ctx, max_steps) every locks_decode_step records CUDA events on its stream at
  * the stage boundaries; locks_profile_end() synchronises the device, writes the mean duration in
- * milliseconds of {prologue, summary scan, selection, sparse attention} to stage_ms[4], the number
- * of steps seen to *steps, and releases the events. */
+ * milliseconds of {summary scan, selection (with the append), sparse attention} to stage_ms[3], the
+ * number of steps seen to *steps, and releases the events. */
 int locks_profile_begin(locks_ctx *ctx, int max_steps);
 int locks_profile_end(locks_ctx *ctx, float *stage_ms, int *steps);
 /* A locks_decode_step CAPTURED while profiling is on records the same stage boundaries as event
  * nodes of the graph (always into the first slot).  After a replay, locks_profile_read()
- * synchronises `stream` and writes that replay's four stage durations (ms) to stage_ms[4]. */
+ * synchronises `stream` and writes that replay's three stage durations (ms) to stage_ms[3]. */
 int locks_profile_read(locks_ctx *ctx, float *stage_ms, locks_stream stream);
 
 /* locks_sparse_attend for callers that cannot allocate device memory (the paper has no

@@ -212,15 +212,15 @@ class Context:
         _check(lib().locks_profile_begin(self.handle, max_steps), "locks_profile_begin")
 
     def locks_profile_end(self):
-        ms = (C.c_float * 4)()
+        ms = (C.c_float * 3)()
         n = C.c_int(0)
         _check(lib().locks_profile_end(self.handle, ms, C.byref(n)), "locks_profile_end")
-        return {"prologue": ms[0], "scan": ms[1], "select": ms[2], "attend": ms[3]}, int(n.value)
+        return {"scan": ms[0], "select": ms[1], "attend": ms[2]}, int(n.value)
 
     def locks_profile_read(self, stream=None):
-        ms = (C.c_float * 4)()
+        ms = (C.c_float * 3)()
         _check(lib().locks_profile_read(self.handle, ms, _stream(stream)), "locks_profile_read")
-        return {"prologue": ms[0], "scan": ms[1], "select": ms[2], "attend": ms[3]}
+        return {"scan": ms[0], "select": ms[1], "attend": ms[2]}
 
     def locks_last_launch_count(self) -> int:
         return int(lib().locks_last_launch_count(self.handle))

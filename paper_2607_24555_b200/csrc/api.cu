@@ -31,7 +31,7 @@ int validate(const locks_config *c) {
 }
 
 struct Layout {
-  size_t status, shat, part, logz, cand_val, cand_idx, att_o, att_lse, att_done, ids, cnt, sq, skn, svn, sout, total;
+  size_t status, shat, part, logz, cand_val, cand_idx, att_o, att_lse, att_done, ids, cnt, sq, skn, svn, sout, seq_eff, total;
   int G, k, S, max_groups, sel_ept, sel_chunks, sel_kc;
 };
 
@@ -78,6 +78,7 @@ Layout make_layout(const locks_config *c) {
   L.skn = take(nb * Hkv * LOCKS_D * esz);
   L.svn = take(nb * Hkv * LOCKS_D * esz);
   L.sout = take(nb * Hq * LOCKS_D * esz);
+  L.seq_eff = take(2 * nb * 4);
   L.total = o;
   return L;
 }
@@ -86,10 +87,10 @@ int check_common(const locks_ctx *ctx, const locks_kv *kv, int batch) {
   if (!ctx || !kv || !kv->k || !kv->v || !kv->block_table || !kv->seq_lens) return LOCKS_ERR_INVALID_ARG;
   if (batch <= 0 || batch > ctx->cfg.max_batch || kv->num_blocks <= 0) return LOCKS_ERR_INVALID_ARG;
   if (kv->stride_block <= 0 || kv->stride_head <= 0 || kv->stride_token < LOCKS_D) return LOCKS_ERR_INVALID_ARG;
-  if (ctx->cfg.kv_dtype == LOCKS_BF16) {  // 16-byte vector copies of bf16 rows
-    if ((kv->stride_block | kv->stride_head | kv->stride_token) % 8) return LOCKS_ERR_INVALID_ARG;
-    if (((uintptr_t)kv->k | (uintptr_t)kv->v) % 16) return LOCKS_ERR_INVALID_ARG;
-  }
+  // 16-byte vector copies of cache rows
+  if ((kv->stride_block | kv->stride_head | kv->stride_token) % (ctx->cfg.kv_dtype == LOCKS_BF16 ? 8 : 4))
+    return LOCKS_ERR_INVALID_ARG;
+  if (((uintptr_t)kv->k | (uintptr_t)kv->v) % 16) return LOCKS_ERR_INVALID_ARG;
   return LOCKS_OK;
 }
 
@@ -140,6 +141,7 @@ int locks_create(const locks_config *cfg, void *workspace, size_t ws_bytes, lock
   c->att_done = reinterpret_cast<int32_t *>(ws + L.att_done);
   c->ids_int = reinterpret_cast<int32_t *>(ws + L.ids);
   c->cnt_int = reinterpret_cast<int32_t *>(ws + L.cnt);
+  c->seq_eff = reinterpret_cast<int32_t *>(ws + L.seq_eff);
   c->stage_q = ws + L.sq; c->stage_kn = ws + L.skn; c->stage_vn = ws + L.svn; c->stage_out = ws + L.sout;
   if (cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking) != cudaSuccess ||
       cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
@@ -187,9 +189,8 @@ int locks_select(locks_ctx *ctx, const void *q, const void *summaries, const loc
   cudaStream_t st = (cudaStream_t)stream;
   ctx->last_launches = 0;
   float *shat = page_logmass ? page_logmass : ctx->shat;
-  if ((rc = locks_launch_prep(ctx, q, nullptr, nullptr, kv, batch, st)) != LOCKS_OK) return rc;
-  if ((rc = locks_launch_scan(ctx, q, summaries, kv, batch, shat, st)) != LOCKS_OK) return rc;
-  return locks_launch_select(ctx, shat, kv, batch, page_ids, page_count, page_logshare, st);
+  if ((rc = locks_launch_scan(ctx, q, summaries, kv, batch, shat, 0, st)) != LOCKS_OK) return rc;
+  return locks_launch_select(ctx, shat, kv, batch, page_ids, page_count, page_logshare, nullptr, st);
 }
 
 int locks_sparse_attend(locks_ctx *ctx, const void *q, const locks_kv *kv, int batch, const int32_t *page_ids,
@@ -208,7 +209,7 @@ int locks_decode_step(locks_ctx *ctx, const void *q, const void *k_new, const vo
   int rc = check_common(ctx, kv, batch);
   if (rc != LOCKS_OK) return rc;
   if (!q || !summaries || !out || ((k_new == nullptr) != (v_new == nullptr)) || ((uintptr_t)summaries % 16) ||
-      ((uintptr_t)q % 16))
+      ((uintptr_t)q % 16) || ((uintptr_t)k_new % 16) || ((uintptr_t)v_new % 16))
     return LOCKS_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)stream;
   int32_t *ids = page_ids ? page_ids : ctx->ids_int;
@@ -224,21 +225,31 @@ int locks_decode_step(locks_ctx *ctx, const void *q, const void *k_new, const vo
     if (capturing) cudaEventRecordWithFlags(pe[i], st, cudaEventRecordExternal);   // becomes an event-record node
     else cudaEventRecord(pe[i], st);
   };
+  // The new token is counted from the scan on (lengths one longer, published in the workspace); its K/V
+  // rows are written by the selector's kernel, beside the ranking, which is early enough for the two
+  // readers of the last page (attention, and the summary build when the token completes a page).
+  locks_append app;
+  locks_kv kv_step = *kv;
+  if (k_new) {
+    app.k_new = k_new; app.v_new = v_new; app.k = kv->k; app.v = kv->v;
+    app.sb = kv->stride_block; app.sh = kv->stride_head; app.st = kv->stride_token;
+    app.block_table = kv->block_table; app.seq_eff = ctx->seq_eff; app.seq_commit = kv->seq_lens;
+    app.num_blocks = kv->num_blocks; app.esz = ctx->cfg.kv_dtype == LOCKS_BF16 ? 2 : 4;
+    kv_step.seq_lens = ctx->seq_eff;
+  }
   mark(0);
-  if ((rc = locks_launch_prep(ctx, q, k_new, v_new, kv, batch, st)) != LOCKS_OK) return rc;
+  if ((rc = locks_launch_scan(ctx, q, summaries, kv, batch, ctx->shat, k_new ? 1 : 0, st)) != LOCKS_OK) return rc;
   mark(1);
-  if ((rc = locks_launch_scan(ctx, q, summaries, kv, batch, ctx->shat, st)) != LOCKS_OK) return rc;
-  // the freshly completed page (if any) is summarised beside select + attend, which read neither it nor its
-  // summary.  The fork sits after the scan launch so that prologue -> scan stays a programmatic edge.
+  if ((rc = locks_launch_select(ctx, ctx->shat, &kv_step, batch, ids, cnt, nullptr, k_new ? &app : nullptr, st)) != LOCKS_OK)
+    return rc;
+  // the freshly completed page (if any) is summarised beside attention, which does not read its summary
   if (cudaEventRecord(ctx->ev_fork, st) != cudaSuccess || cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0) != cudaSuccess)
     return LOCKS_ERR_CUDA;
-  if ((rc = locks_launch_build(ctx, kv, batch, nullptr, nullptr, 1, summaries, ctx->side)) != LOCKS_OK) return rc;
+  if ((rc = locks_launch_build(ctx, &kv_step, batch, nullptr, nullptr, 1, summaries, ctx->side)) != LOCKS_OK) return rc;
   if (cudaEventRecord(ctx->ev_join, ctx->side) != cudaSuccess) return LOCKS_ERR_CUDA;
   mark(2);
-  if ((rc = locks_launch_select(ctx, ctx->shat, kv, batch, ids, cnt, nullptr, st)) != LOCKS_OK) return rc;
+  if ((rc = locks_launch_attend(ctx, q, &kv_step, batch, ids, cnt, out, nullptr, st)) != LOCKS_OK) return rc;
   mark(3);
-  if ((rc = locks_launch_attend(ctx, q, kv, batch, ids, cnt, out, nullptr, st)) != LOCKS_OK) return rc;
-  mark(4);
   if (pe && !capturing) ctx->prof_n++;
   if (cudaStreamWaitEvent(st, ctx->ev_join, 0) != cudaSuccess) return LOCKS_ERR_CUDA;
   return LOCKS_OK;

@@ -1,4 +1,4 @@
-// Summary build (Sec. 4 "Build (once, when a page completes)") and the per-step prologue.
+// Summary build (Sec. 4 "Build (once, when a page completes)").
 //
 // build_kernel: one warp per (page, KV head).
 //   1. load the page's 16 keys (lane owns 4 consecutive dims of every key), centroid mu, deviations D
@@ -9,7 +9,6 @@
 //   5. V = D^T U_r Sigma_r^-1 (lane's 4 dims), C = U_r Sigma_r, sign: largest |V| entry positive
 //   6. store fp32 (F32 format) or quantise: symmetric abs-max, fp16 scale, round-half-even codes
 //      (int4 basis per column, int8 coefficients per row, int8 centroid) packed in the blob layout
-// prep_kernel: appends the new token's K/V row to the cache and bumps the sequence length.
 #include "locks_internal.cuh"
 
 namespace {
@@ -282,48 +281,6 @@ __global__ void __launch_bounds__(kBuildWarps * 32) build_kernel(BuildParams p) 
   }
 }
 
-// ------------------------------------------------------------------------------------------------
-
-struct PrepParams {
-  const void *q, *k_new, *v_new;
-  void *k, *v;
-  int64_t sb, sh, st;
-  const int32_t *block_table;
-  int32_t *seq_lens;
-  int32_t *status;
-  int Hq, Hkv, Pmax, num_blocks;
-};
-
-template <typename T>
-__global__ void __launch_bounds__(256) prep_kernel(PrepParams p) {
-  const int b = blockIdx.x;
-  if (p.k_new == nullptr) return;
-  pdl_trigger();
-  pdl_wait();   // the previous step's readers of the cache and of seq_lens are done
-  const int T0 = p.seq_lens[b];
-  const int page = T0 / LOCKS_B, slot = T0 % LOCKS_B;
-  bool ok = page < p.Pmax;
-  int block = 0;
-  if (ok) {
-    block = p.block_table[(int64_t)b * p.Pmax + page];
-    ok = block >= 0 && block < p.num_blocks;
-  }
-  if (!ok) {
-    if (threadIdx.x == 0) set_status(p.status, LOCKS_ERR_BAD_BLOCK);
-    return;
-  }
-  const T *kn = reinterpret_cast<const T *>(p.k_new), *vn = reinterpret_cast<const T *>(p.v_new);
-  T *K = reinterpret_cast<T *>(p.k), *V = reinterpret_cast<T *>(p.v);
-  for (int e = threadIdx.x; e < p.Hkv * LOCKS_D; e += 256) {
-    const int h = e / LOCKS_D, c = e - h * LOCKS_D;
-    const int64_t dst = (int64_t)block * p.sb + (int64_t)h * p.sh + (int64_t)slot * p.st + c;
-    K[dst] = kn[((int64_t)b * p.Hkv + h) * LOCKS_D + c];
-    V[dst] = vn[((int64_t)b * p.Hkv + h) * LOCKS_D + c];
-  }
-  __syncthreads();
-  if (threadIdx.x == 0) p.seq_lens[b] = T0 + 1;
-}
-
 }  // namespace
 
 int locks_launch_build(locks_ctx *c, const locks_kv *kv, int batch, const int32_t *pb, const int32_t *pe,
@@ -350,18 +307,5 @@ int locks_launch_build(locks_ctx *c, const locks_kv *kv, int batch, const int32_
   else if (bf) build_kernel<__nv_bfloat16, LOCKS_FMT_F32><<<grid, kBuildWarps * 32, smem, st>>>(p);
   else if (i4) build_kernel<float, LOCKS_FMT_I4><<<grid, kBuildWarps * 32, smem, st>>>(p);
   else build_kernel<float, LOCKS_FMT_F32><<<grid, kBuildWarps * 32, smem, st>>>(p);
-  return locks_check_launch(c);
-}
-
-int locks_launch_prep(locks_ctx *c, const void *q, const void *k_new, const void *v_new, const locks_kv *kv,
-                      int batch, cudaStream_t st) {
-  PrepParams p;
-  p.q = q; p.k_new = k_new; p.v_new = v_new; p.k = kv->k; p.v = kv->v;
-  p.sb = kv->stride_block; p.sh = kv->stride_head; p.st = kv->stride_token;
-  p.block_table = kv->block_table; p.seq_lens = kv->seq_lens; p.status = c->status;
-  p.Hq = c->cfg.num_q_heads; p.Hkv = c->cfg.num_kv_heads; p.Pmax = c->Pmax; p.num_blocks = kv->num_blocks;
-  if (k_new == nullptr) return LOCKS_OK;   // nothing to append: no launch
-  if (c->cfg.q_dtype == LOCKS_BF16) locks_launch_pdl(prep_kernel<__nv_bfloat16>, dim3(batch), dim3(256), 0, st, p);
-  else locks_launch_pdl(prep_kernel<float>, dim3(batch), dim3(256), 0, st, p);
   return locks_check_launch(c);
 }

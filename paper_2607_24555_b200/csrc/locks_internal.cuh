@@ -45,22 +45,33 @@ struct locks_ctx {
   int32_t *ids_int;        // [max_batch][Hkv][k]
   int32_t *cnt_int;        // [max_batch][Hkv]
   char *stage_q, *stage_kn, *stage_vn, *stage_out;
-  cudaStream_t side;       // build of freshly filled pages runs beside select + attend
+  int32_t *seq_eff;        // [2][max_batch] decode step in flight: effective lengths, append positions
+  cudaStream_t side;       // build of freshly filled pages runs beside attend
   cudaEvent_t ev_fork, ev_join;
   int last_launches;
   // optional per-stage timing of eager decode steps (see locks_profile_begin)
   cudaEvent_t *prof_ev;    // [prof_cap][LOCKS_PROF_MARKS]
   int prof_cap, prof_n;
 };
-#define LOCKS_PROF_MARKS 5   // step start, after prep, after scan, after select, after attend
+#define LOCKS_PROF_MARKS 4   // step start, after scan, after select, after attend
+
+// The new token of a decode step, handed to the selector's first kernel, which writes it into the cache.
+struct locks_append {
+  const void *k_new, *v_new;   // [batch][Hkv][d]; k_new == nullptr: nothing to append
+  void *k, *v;
+  int64_t sb, sh, st;          // cache strides in elements
+  const int32_t *block_table;
+  const int32_t *seq_eff;      // published by the scan: [batch] lengths, [batch] append positions
+  int32_t *seq_commit;         // the caller's sequence lengths
+  int num_blocks, esz;
+};
 
 // launchers (each returns LOCKS_OK or LOCKS_ERR_CUDA and adds to ctx->last_launches)
-int locks_launch_prep(locks_ctx *c, const void *q, const void *k_new, const void *v_new, const locks_kv *kv,
-                      int batch, cudaStream_t st);
+// seq_inc = 1: lengths are taken one token longer than kv->seq_lens says and published in ctx->seq_eff
 int locks_launch_scan(locks_ctx *c, const void *q, const void *summaries, const locks_kv *kv, int batch,
-                      float *shat, cudaStream_t st);
+                      float *shat, int seq_inc, cudaStream_t st);
 int locks_launch_select(locks_ctx *c, const float *shat, const locks_kv *kv, int batch, int32_t *ids,
-                        int32_t *cnt, float *logshare, cudaStream_t st);
+                        int32_t *cnt, float *logshare, const locks_append *app, cudaStream_t st);
 int locks_launch_attend(locks_ctx *c, const void *q, const locks_kv *kv, int batch, const int32_t *ids,
                         const int32_t *cnt, void *out, float *lse, cudaStream_t st);
 int locks_launch_build(locks_ctx *c, const locks_kv *kv, int batch, const int32_t *pb, const int32_t *pe,

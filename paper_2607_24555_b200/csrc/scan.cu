@@ -30,7 +30,27 @@ struct ScanParams {
   int32_t *status;
   int batch, Hq, Hkv, G, Pmax, max_groups, num_blocks, k, S, r;
   float sm_scale;
+  // decode step with an appended token: lengths count the token that the selector's kernel is about to
+  // write (seq_inc = 1); the first CTA publishes them, and the append position, for the step's later kernels
+  int seq_inc;
+  int32_t *seq_eff;   // [2][max_batch]: effective length, append position (-1: none) -- or nullptr
 };
+
+// Length of request b as this step sees it.  A sequence that has no room for the token keeps its length.
+__device__ __forceinline__ int step_len(const ScanParams &p, int b) {
+  return min(p.seq_lens[b] + p.seq_inc, p.Pmax * LOCKS_B);
+}
+
+__device__ __forceinline__ void publish_lengths(const ScanParams &p, bool first_cta, int tid, int nthreads) {
+  if (!first_cta || !p.seq_eff) return;
+  for (int b = tid; b < p.batch; b += nthreads) {
+    const int T0 = p.seq_lens[b], T1 = T0 + p.seq_inc;
+    const bool room = T1 <= p.Pmax * LOCKS_B;
+    if (!room) set_status(p.status, LOCKS_ERR_BAD_BLOCK);
+    p.seq_eff[b] = room ? T1 : T0;
+    p.seq_eff[p.batch + b] = (room && p.seq_inc) ? T0 : -1;
+  }
+}
 
 // ------------------------------------------------------------------------------------------------
 // generic path
@@ -60,7 +80,8 @@ __global__ void __launch_bounds__(128) scan_generic_kernel(ScanParams p) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int grp = blockIdx.x * 4 + warp, h = blockIdx.y, b = blockIdx.z;
   pdl_wait();
-  const int T = p.seq_lens[b];
+  publish_lengths(p, (blockIdx.x | blockIdx.y | blockIdx.z) == 0, threadIdx.x, 128);
+  const int T = step_len(p, b);
   const int P = (T + LOCKS_B - 1) / LOCKS_B;
   if (P <= p.k) return;               // every page is kept: nothing to rank
   const int nsc = P - 1;              // pages 0 .. P-2 are scored
@@ -222,7 +243,8 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4r8_ker
   }
   __syncwarp();
   pdl_trigger();   // single-wave kernel: the selector may be scheduled as SMs drain
-  pdl_wait();      // sequence lengths (append) and the previous consumers of the workspace are done
+  pdl_wait();      // sequence lengths and the previous consumers of the workspace are done
+  publish_lengths(p, blockIdx.x == 0, threadIdx.x, kScanWarps * 32);
 
   // warps stick to one (request, KV head) at a time: `wpp` warps share a problem and stride its groups
   const int W = gridDim.x * kScanWarps;
@@ -235,7 +257,7 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4r8_ker
   auto enter = [&](Cursor &c) {   // refresh the per-problem fields of the cursor
     c.b = c.prob / p.Hkv;
     c.h = c.prob - c.b * p.Hkv;
-    const int T = p.seq_lens[c.b];
+    const int T = step_len(p, c.b);
     const int P = (T + LOCKS_B - 1) / LOCKS_B;
     c.nsc = (P <= p.k) ? 0 : P - 1;
   };
@@ -602,8 +624,10 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4r8_ker
 }  // namespace
 
 int locks_launch_scan(locks_ctx *c, const void *q, const void *summaries, const locks_kv *kv, int batch,
-                      float *shat, cudaStream_t st) {
+                      float *shat, int seq_inc, cudaStream_t st) {
   ScanParams p;
+  p.seq_inc = seq_inc;
+  p.seq_eff = seq_inc ? c->seq_eff : nullptr;
   p.q = q;
   p.summ = reinterpret_cast<const uint8_t *>(summaries);
   p.block_table = kv->block_table;

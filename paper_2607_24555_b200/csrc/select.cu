@@ -25,8 +25,41 @@ struct SelParams {
   float *cand_val;
   int32_t *cand_idx;
   float *logz;      // [batch][Hq] log Z_g, written by logz_kernel when a problem spans several chunks
+  int32_t *status;
   int batch, Hq, Hkv, G, Pmax, max_groups, k, chunks, kc, chunk_pages, part_slots;
+  locks_append app;  // decode step only: the new token's K/V rows, written here beside the ranking
 };
+
+// Decode step: the CTA of (request b, KV head h) writes the new token's K and V rows of that head into the
+// cache (one warp, a few independent loads and stores beside the ranking's own loads), and the CTA of
+// head 0 stores the step's length back to the caller's array.  Nothing reads the caller's array between
+// the scan (complete before this kernel passes its wait) and the end of the step: the step's other
+// kernels take lengths from the published copy.
+__device__ __forceinline__ void append_token(const locks_append &a, int batch, int Hkv, int Pmax, int b, int h,
+                                             int lane, int T, int32_t *status) {
+  if (h == 0 && lane == 0) a.seq_commit[b] = T;
+  const int at = a.seq_eff[batch + b];
+  if (at < 0) return;
+  const int page = at / LOCKS_B, slot = at % LOCKS_B;
+  const int block = a.block_table[(int64_t)b * Pmax + page];
+  if (block < 0 || block >= a.num_blocks) {
+    if (lane == 0) set_status(status, LOCKS_ERR_BAD_BLOCK);
+    return;
+  }
+  const int64_t dst = (int64_t)block * a.sb + (int64_t)h * a.sh + (int64_t)slot * a.st;
+  const int64_t src = ((int64_t)b * Hkv + h) * LOCKS_D;
+  if (a.esz == 2) {
+    const uint2 kk = reinterpret_cast<const uint2 *>(reinterpret_cast<const uint16_t *>(a.k_new) + src)[lane];
+    const uint2 vv = reinterpret_cast<const uint2 *>(reinterpret_cast<const uint16_t *>(a.v_new) + src)[lane];
+    reinterpret_cast<uint2 *>(reinterpret_cast<uint16_t *>(a.k) + dst)[lane] = kk;
+    reinterpret_cast<uint2 *>(reinterpret_cast<uint16_t *>(a.v) + dst)[lane] = vv;
+  } else {
+    const uint4 kk = reinterpret_cast<const uint4 *>(reinterpret_cast<const uint32_t *>(a.k_new) + src)[lane];
+    const uint4 vv = reinterpret_cast<const uint4 *>(reinterpret_cast<const uint32_t *>(a.v_new) + src)[lane];
+    reinterpret_cast<uint4 *>(reinterpret_cast<uint32_t *>(a.k) + dst)[lane] = kk;
+    reinterpret_cast<uint4 *>(reinterpret_cast<uint32_t *>(a.v) + dst)[lane] = vv;
+  }
+}
 
 struct SelShared {
   int hist[kNW * 256];   // one 256-bin histogram per warp
@@ -195,6 +228,8 @@ __global__ void __launch_bounds__(LOCKS_SEL_THREADS) select_stage1_kernel(SelPar
   pdl_trigger();
   pdl_wait();   // the scan's scores and partials
   const int T = p.seq_lens[b];
+  if (p.app.k_new && chunk == 0 && tid >= LOCKS_SEL_THREADS - 32)
+    append_token(p.app, p.batch, p.Hkv, p.Pmax, b, h, tid & 31, T, p.status);
   const int P = (T + LOCKS_B - 1) / LOCKS_B;
   const int64_t prob = (int64_t)b * p.Hkv + h;
   int32_t *ids = p.ids + prob * p.k;
@@ -334,8 +369,11 @@ __global__ void __launch_bounds__(LOCKS_SEL_THREADS) select_stage2_kernel(SelPar
 }  // namespace
 
 int locks_launch_select(locks_ctx *c, const float *shat, const locks_kv *kv, int batch, int32_t *ids,
-                        int32_t *cnt, float *logshare, cudaStream_t st) {
+                        int32_t *cnt, float *logshare, const locks_append *app, cudaStream_t st) {
   SelParams p;
+  if (app) p.app = *app;
+  else p.app.k_new = nullptr;
+  p.status = c->status;
   p.shat = shat; p.part = c->part; p.seq_lens = kv->seq_lens; p.ids = ids; p.cnt = cnt; p.logshare = logshare;
   p.cand_val = c->cand_val; p.cand_idx = c->cand_idx;
   p.batch = batch; p.Hq = c->cfg.num_q_heads; p.Hkv = c->cfg.num_kv_heads; p.G = c->G; p.Pmax = c->Pmax;
