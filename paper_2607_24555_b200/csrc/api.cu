@@ -31,7 +31,7 @@ int validate(const locks_config *c) {
 }
 
 struct Layout {
-  size_t status, shat, part, logz, cand_val, cand_idx, att_o, att_lse, att_done, ids, cnt, sq, skn, svn, sout, seq_eff, total;
+  size_t status, shat, part, sel_done, cand_val, cand_idx, att_o, att_lse, att_done, ids, cnt, sq, skn, svn, sout, seq_eff, total;
   int G, k, S, max_groups, sel_ept, sel_chunks, sel_kc;
 };
 
@@ -41,18 +41,22 @@ Layout make_layout(const locks_config *c) {
   L.k = (c->budget_tokens + c->page_size - 1) / c->page_size;
   L.S = c->summary_fmt == LOCKS_FMT_I4 ? i4_stride(c->rank) : f32_stride(c->rank);
   L.max_groups = (c->max_pages_per_seq + LOCKS_GROUP - 1) / LOCKS_GROUP;
-  // pages per thread in stage 1 (4 / 8 / 16).  With many (request, KV head) problems one CTA per problem
-  // already fills the GPU, so a context of up to 8192 pages is ranked in one chunk; with few problems
-  // the smallest chunk whose candidate lists still fit stage 2 is taken, so that many CTAs share the work.
+  // Pages per thread of a selector CTA (1 .. 16; a CTA ranks sel_ept * 512 pages).  With many (request,
+  // KV head) problems one CTA per problem already fills the GPU, so a context of up to 8192 pages is ranked
+  // in one chunk.  With few problems the smallest chunk whose candidate lists still fit the final round
+  // is taken: the selector is a chain of memory round trips, so many small CTAs finish sooner.
   const int per_thread = (c->max_pages_per_seq + LOCKS_SEL_THREADS - 1) / LOCKS_SEL_THREADS;
   const bool many_problems = (int64_t)c->max_batch * c->num_kv_heads >= 32;
-  L.sel_ept = 16;
-  if (many_problems && per_thread <= 16) {
-    L.sel_ept = per_thread <= 4 ? 4 : (per_thread <= 8 ? 8 : 16);
+  L.sel_ept = LOCKS_SEL_MAX_EPT;
+  if (many_problems && per_thread <= LOCKS_SEL_MAX_EPT) {
+    L.sel_ept = per_thread;
   } else {
-    for (int ept = 4; ept <= 16; ept *= 2) {
+    for (int ept = 1; ept <= LOCKS_SEL_MAX_EPT; ept *= 2) {
       const int chunks = (c->max_pages_per_seq + ept * LOCKS_SEL_THREADS - 1) / (ept * LOCKS_SEL_THREADS);
-      if (chunks == 1 || (size_t)chunks * (L.k - 2 > 0 ? L.k - 2 : 1) <= 16 * LOCKS_SEL_THREADS) { L.sel_ept = ept; break; }
+      if (chunks == 1 || (size_t)chunks * (L.k - 2 > 0 ? L.k - 2 : 1) <= (size_t)LOCKS_SEL_MAX_EPT * LOCKS_SEL_THREADS) {
+        L.sel_ept = ept;
+        break;
+      }
     }
   }
   L.sel_chunks = (c->max_pages_per_seq + L.sel_ept * LOCKS_SEL_THREADS - 1) / (L.sel_ept * LOCKS_SEL_THREADS);
@@ -64,7 +68,7 @@ Layout make_layout(const locks_config *c) {
   L.status = take(64);
   L.shat = take(nb * Hq * P * 4);
   L.part = take(nb * Hq * L.max_groups * 8);
-  L.logz = take(nb * Hq * 4);
+  L.sel_done = take(nb * Hkv * 4);
   L.cand_val = take(nb * Hkv * L.sel_chunks * L.sel_kc * 4);
   L.cand_idx = take(nb * Hkv * L.sel_chunks * L.sel_kc * 4);
   // split-K partial rows: batch * Hq * splits with splits <= slots / (batch * Hkv) (+1 rounding) and <= 128
@@ -133,7 +137,7 @@ int locks_create(const locks_config *cfg, void *workspace, size_t ws_bytes, lock
   c->status = reinterpret_cast<int32_t *>(ws + L.status);
   c->shat = reinterpret_cast<float *>(ws + L.shat);
   c->part = reinterpret_cast<float2 *>(ws + L.part);
-  c->logz = reinterpret_cast<float *>(ws + L.logz);
+  c->sel_done = reinterpret_cast<int32_t *>(ws + L.sel_done);
   c->cand_val = reinterpret_cast<float *>(ws + L.cand_val);
   c->cand_idx = reinterpret_cast<int32_t *>(ws + L.cand_idx);
   c->att_o = reinterpret_cast<float *>(ws + L.att_o);
@@ -148,6 +152,7 @@ int locks_create(const locks_config *cfg, void *workspace, size_t ws_bytes, lock
       cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) != cudaSuccess ||
       cudaMemsetAsync(c->status, 0, 64, 0) != cudaSuccess ||
       cudaMemsetAsync(c->att_done, 0, (size_t)cfg->max_batch * cfg->num_kv_heads * 4, 0) != cudaSuccess ||
+      cudaMemsetAsync(c->sel_done, 0, (size_t)cfg->max_batch * cfg->num_kv_heads * 4, 0) != cudaSuccess ||
       cudaStreamSynchronize(0) != cudaSuccess) {
     delete c;
     return LOCKS_ERR_CUDA;

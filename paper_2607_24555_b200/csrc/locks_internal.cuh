@@ -36,7 +36,7 @@ struct locks_ctx {
   int32_t *status;         // [4] sticky status, work counters
   float *shat;             // [max_batch][Hq][Pmax]
   float2 *part;            // [max_batch][Hq][max_groups] partial (max, sum exp) over candidate pages
-  float *logz;             // [max_batch][Hq] log Z_g (chunked selection only)
+  int32_t *sel_done;       // [max_batch][Hkv] chunk-arrival counters
   float *cand_val;         // [max_batch][Hkv][sel_chunks][sel_kc]
   int32_t *cand_idx;
   float *att_o;            // [rows][d], rows = batch * Hq * splits <= att_rows

@@ -32,6 +32,7 @@ struct ScanParams {
   float sm_scale;
   // decode step with an appended token: lengths count the token that the selector's kernel is about to
   // write (seq_inc = 1); the first CTA publishes them, and the append position, for the step's later kernels
+  int cta_reduce;     // every warp of a CTA works on one problem only: one partial per (head, CTA)
   int seq_inc;
   int32_t *seq_eff;   // [2][max_batch]: effective length, append position (-1: none) -- or nullptr
 };
@@ -166,7 +167,8 @@ constexpr int kScanStages = 2;
 constexpr int kScanCtasPerSm = 2;
 constexpr int kBlob = i4_stride(8);                       // 832
 constexpr int kStageBytes = LOCKS_GROUP * kBlob;          // 6656
-constexpr int kScanSmem = kScanWarps * (kScanStages * kStageBytes + 64);
+constexpr int kScanRedBytes = kScanWarps * 16 * 8;         // (max, sum) of 16 heads per warp, for the CTA-level merge
+constexpr int kScanSmem = kScanWarps * (kScanStages * kStageBytes + 64) + kScanRedBytes;
 constexpr bool kScanBulk = LOCKS_SCAN_BULK;             // true: cp.async.bulk + mbarrier, false: 16-byte cp.async
 
 // (a & b) | c in one LOP3 with both constants held in registers
@@ -230,7 +232,7 @@ __device__ __forceinline__ uint32_t movm_trans(uint32_t v) {
 // PK (G <= 4 only): the 8 head columns hold the group twice, so that after MMA#1 the projection, MMA#2 and
 // the log-sum-exp handle two pages at once (rows 0-3 = page A's heads, rows 4-7 = page B's heads, the two
 // pages separated along K) instead of leaving half of the lanes idle.
-template <int NH, bool PK>
+template <int NH, bool PK, bool CR>
 __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4r8_kernel(ScanParams p) {
   extern __shared__ __align__(128) uint8_t smem[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -388,7 +390,8 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4r8_ker
       if (d > 0.f) { sacc = sacc * e + 1.f; m = v; } else sacc += e;
     }
   };
-  auto flush = [&]() {
+  float2 *red = reinterpret_cast<float2 *>(smem + kScanWarps * (kScanStages * kStageBytes + 64));   // [warp][16]
+  auto flush = [&](bool to_smem) {
 #pragma unroll
     for (int hh = 0; hh < NH; ++hh) {
       float m = pm[hh], sacc = ps[hh];
@@ -400,8 +403,10 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4r8_ker
         if (nm > -INFINITY) { sacc = sacc * __expf(m - nm) + os * __expf(om - nm); m = nm; }
       }
       const int g = PK ? (x & 3) : x + 8 * hh;
-      if (t == 0 && (!PK || x < 4) && g < p.G)
-        p.part[((int64_t)cur_b * p.Hq + cur_h * p.G + g) * p.max_groups + sub] = make_float2(m, sacc);
+      if (t == 0 && (!PK || x < 4) && g < p.G) {
+        if (CR && to_smem) red[warp * 16 + g] = make_float2(m, sacc);
+        else p.part[((int64_t)cur_b * p.Hq + cur_h * p.G + g) * p.max_groups + sub] = make_float2(m, sacc);
+      }
       pm[hh] = -INFINITY;
       ps[hh] = 0.f;
     }
@@ -425,7 +430,7 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4r8_ker
     --inflight;
     const int b = cc.b, h = cc.h;
     if (cc.prob != cur_prob) {
-      if (cur_prob >= 0) flush();
+      if (cur_prob >= 0) flush(false);
       cur_prob = cc.prob;
       cur_b = b;
       cur_h = h;
@@ -610,7 +615,24 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4r8_ker
     settle(cc);
     ++it;
   }
-  if (ok && cur_prob >= 0) flush();
+  if (CR) {
+    // geometry guarantees that all warps of this CTA reach this point and share the problem `slot`
+    flush(true);
+    __syncthreads();
+    if (warp == 0 && lane < p.G) {
+      float m = -INFINITY, sacc = 0.f;
+#pragma unroll
+      for (int w = 0; w < kScanWarps; ++w) {
+        const float2 v = red[w * 16 + lane];
+        const float nm = fmaxf(m, v.x);
+        if (nm > -INFINITY) { sacc = sacc * __expf(m - nm) + v.y * __expf(v.x - nm); m = nm; }
+      }
+      const int pb = slot / p.Hkv, ph = slot - pb * p.Hkv;
+      p.part[((int64_t)pb * p.Hq + ph * p.G + lane) * p.max_groups + sub / kScanWarps] = make_float2(m, sacc);
+    }
+  } else if (ok && cur_prob >= 0) {
+    flush(false);
+  }
   if (!ok) {
     // a wait ran out: flag it, then give copies still in flight a bounded chance to land before exit
     if (lane == 0) set_status(p.status, LOCKS_ERR_TIMEOUT);
@@ -626,6 +648,7 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4r8_ker
 int locks_launch_scan(locks_ctx *c, const void *q, const void *summaries, const locks_kv *kv, int batch,
                       float *shat, int seq_inc, cudaStream_t st) {
   ScanParams p;
+  p.cta_reduce = 0;
   p.seq_inc = seq_inc;
   p.seq_eff = seq_inc ? c->seq_eff : nullptr;
   p.q = q;
@@ -643,9 +666,12 @@ int locks_launch_scan(locks_ctx *c, const void *q, const void *summaries, const 
   if (tensor) {
     static bool attr_done = false;
     if (!attr_done) {
-      cudaFuncSetAttribute(scan_i4r8_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kScanSmem);
-      cudaFuncSetAttribute(scan_i4r8_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kScanSmem);
-      cudaFuncSetAttribute(scan_i4r8_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kScanSmem);
+      cudaFuncSetAttribute(scan_i4r8_kernel<1, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kScanSmem);
+      cudaFuncSetAttribute(scan_i4r8_kernel<1, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kScanSmem);
+      cudaFuncSetAttribute(scan_i4r8_kernel<2, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kScanSmem);
+      cudaFuncSetAttribute(scan_i4r8_kernel<1, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kScanSmem);
+      cudaFuncSetAttribute(scan_i4r8_kernel<1, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kScanSmem);
+      cudaFuncSetAttribute(scan_i4r8_kernel<2, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kScanSmem);
       attr_done = true;
     }
     const int total_groups = batch * p.Hkv * p.max_groups;
@@ -654,11 +680,23 @@ int locks_launch_scan(locks_ctx *c, const void *q, const void *summaries, const 
     if (grid > need) grid = need < 1 ? 1 : need;
     {   // tensor kernel: one partial per (problem, warp); mirrors the kernel's own partition
       const int W = grid * kScanWarps, nprob = batch * p.Hkv;
-      c->part_slots = W / nprob > 1 ? W / nprob : 1;
+      const int wpp = W / nprob > 1 ? W / nprob : 1, nslots = W / wpp;
+      c->part_slots = wpp;
+      // few problems: every CTA's warps share one problem for the whole launch and none leaves early,
+      // so the CTA merges its warps' partials before writing (the selector reads 8x fewer)
+      p.cta_reduce = (wpp % kScanWarps == 0 && nslots == nprob && nslots * wpp == W) ? 1 : 0;
+      if (p.cta_reduce) c->part_slots = wpp / kScanWarps;
     }
-    if (c->G <= 4) locks_launch_pdl(scan_i4r8_kernel<1, true>, dim3(grid), dim3(kScanWarps * 32), kScanSmem, st, p);
-    else if (c->G <= 8) locks_launch_pdl(scan_i4r8_kernel<1, false>, dim3(grid), dim3(kScanWarps * 32), kScanSmem, st, p);
-    else locks_launch_pdl(scan_i4r8_kernel<2, false>, dim3(grid), dim3(kScanWarps * 32), kScanSmem, st, p);
+    const dim3 g(grid), blk(kScanWarps * 32);
+    if (p.cta_reduce) {
+      if (c->G <= 4) locks_launch_pdl(scan_i4r8_kernel<1, true, true>, g, blk, kScanSmem, st, p);
+      else if (c->G <= 8) locks_launch_pdl(scan_i4r8_kernel<1, false, true>, g, blk, kScanSmem, st, p);
+      else locks_launch_pdl(scan_i4r8_kernel<2, false, true>, g, blk, kScanSmem, st, p);
+    } else {
+      if (c->G <= 4) locks_launch_pdl(scan_i4r8_kernel<1, true, false>, g, blk, kScanSmem, st, p);
+      else if (c->G <= 8) locks_launch_pdl(scan_i4r8_kernel<1, false, false>, g, blk, kScanSmem, st, p);
+      else locks_launch_pdl(scan_i4r8_kernel<2, false, false>, g, blk, kScanSmem, st, p);
+    }
   } else {
     dim3 grid((c->max_groups + 3) / 4, p.Hkv, batch);
     const bool qbf = c->cfg.q_dtype == LOCKS_BF16;

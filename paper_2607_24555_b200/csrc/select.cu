@@ -2,19 +2,26 @@
 //   log Z_g   = log sum_{j in 1..P-2} exp s^_j(q_g)                       (candidates only)
 //   log m_bar_j = log( (1/G) sum_g exp(s^_j(q_g) - log Z_g) )
 //   S = {0, P-1}  U  top-(k-2) candidates by log m_bar_j (ties: lower page index), ids ascending.
-// Stage 1 (one 512-thread CTA per chunk of 2048 / 4096 / 8192 pages of a (request, KV head)) ranks its
-// chunk with an exact 4-pass radix select over keys held in registers and compacts the winners in
-// page order.  With one chunk it writes the final table; with several, log Z comes from a small
-// reduction kernel, each chunk emits its own top-(k-2) (value, page) list and stage 2 re-selects
-// among them (a chunk's local top-(k-2) always contains the chunk's share of the global top-(k-2),
-// ties included, because both use the same lower-index tie rule and lists stay in page order).
+// One 512-thread CTA ranks a chunk of 2048 / 4096 / 8192 pages of a (request, KV head): it turns the
+// chunk's scores into order-preserving 32-bit keys in shared memory, finds the (k-2)-th largest with an
+// exact 4-pass radix select and compacts the winners in page order.  With one chunk per problem that is
+// the final table.  With several, each chunk emits its own top-(k-2) (value, page) list, and the CTA of a
+// problem that finishes last ranks the lists the same way in the same launch (a chunk's local top-(k-2)
+// always contains the chunk's share of the global top-(k-2), ties included, because both rounds use the
+// same lower-index tie rule and lists stay in page order).
 // Pages are dealt to threads round-robin (element i of thread t is page i*512 + t), so loads are
 // coalesced and every thread is busy whatever the context length.
+// The kernel runs once through its code on at most a few dozen SMs, so instruction fetch is a visible part
+// of its latency: loops over a thread's elements stay rolled (keys live in shared memory, not in
+// registers), and the two routines used by both rounds are real calls.
 #include "locks_internal.cuh"
 
 namespace {
 
 constexpr int kNW = LOCKS_SEL_THREADS / 32;
+constexpr int kMaxKeys = LOCKS_SEL_MAX_EPT * LOCKS_SEL_THREADS;   // keys one CTA ranks at most
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
 
 struct SelParams {
   const float *shat;
@@ -22,9 +29,9 @@ struct SelParams {
   const int32_t *seq_lens;
   int32_t *ids, *cnt;
   float *logshare;
-  float *cand_val;
+  uint32_t *cand_key;  // [batch][Hkv][chunks][kc] chunk lists (chunked selection only): keys, 0 = no entry
   int32_t *cand_idx;
-  float *logz;      // [batch][Hq] log Z_g, written by logz_kernel when a problem spans several chunks
+  int32_t *sel_done;   // [batch][Hkv] chunk-arrival counters (zero between launches)
   int32_t *status;
   int batch, Hq, Hkv, G, Pmax, max_groups, k, chunks, kc, chunk_pages, part_slots;
   locks_append app;  // decode step only: the new token's K/V rows, written here beside the ranking
@@ -62,41 +69,72 @@ __device__ __forceinline__ void append_token(const locks_append &a, int batch, i
 }
 
 struct SelShared {
-  int hist[kNW * 256];   // one 256-bin histogram per warp
-  int misc[16];          // per-pass result (double-buffered)
+  uint32_t key[kMaxKeys];             // order-preserving keys, element i of thread t at i*512 + t
+  int hist[kNW * 256];                // one 256-bin histogram per warp
+  int cnt[LOCKS_SEL_MAX_EPT * kNW];   // per (slab, warp) winner counts for the ordered compaction
+  int misc[16];                       // per-pass result (double-buffered), arrival flag
   int wsum[8];
-  int cnt[16 * kNW];     // per (slab, warp) winner counts for the ordered compaction
-  float logz[16];
+  float lz2[16];                      // log2-domain log Z_g
+  float lzm[kNW], lzs[kNW];           // per-warp (max, sum) of the log Z reduction
+  uint32_t red[2 * kNW];              // per-warp AND / OR of the keys
 };
 
+extern __shared__ __align__(16) uint8_t sel_smem[];
+// The routines below are real calls; each takes the block's shared state from the symbol itself (a
+// reference argument would turn every access into a generic one) and its inputs by value (no stack).
+__device__ __forceinline__ SelShared &shared_state() { return *reinterpret_cast<SelShared *>(sel_smem); }
+
+__device__ __forceinline__ float ex2f(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ float lg2f(float x) {
+  float y;
+  asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 __device__ __forceinline__ uint32_t order_key(float f) {
   uint32_t u = __float_as_uint(f);
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
-// Exact top-K among the block's N = 512*EPT keys; element i of thread t has index i*512 + t.
-// sel[i] is set for the K winners: every key above the K-th largest, plus the lowest-indexed keys
-// equal to it.  pos[i] = rank of a winner in index order.  Requires K <= number of valid keys.
-// Four 8-bit radix passes.  Every warp counts into its own histogram (page masses share their
-// leading bits, so a shared histogram would serialise all warps on one or two counters); bin b of
-// the block is then summed and suffix-scanned by thread 255 - b.  sh.hist must be zero on entry.
-template <int EPT>
-__device__ void block_topk(const uint32_t (&key)[EPT], int K, bool (&sel)[EPT], int (&pos)[EPT], SelShared &sh,
-                           int nslab = EPT) {   // slabs >= nslab hold no valid key (uniform across the block)
+// K-th largest of the keys sh.key[i*512 + t], i < nslab (invalid elements hold key 0; 1 <= K <= number of
+// valid keys).  Returns (key, how many of the keys equal to it belong to the top K).
+// 8-bit radix passes from the top; leading bytes on which all valid keys agree (page masses share sign
+// and exponent) are skipped after one AND / OR reduction.  Every warp counts into its own histogram;
+// bin b of the block is then summed and suffix-scanned by thread 255 - b.  sh.hist must be zero on entry
+// and is zero on return.
+__device__ __noinline__ uint2 radix_select(int nslab, int K) {
+  SelShared &sh = shared_state();
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  if (K <= 0) {  // nothing to pick (k = 2): uniform across the block
-#pragma unroll
-    for (int i = 0; i < EPT; ++i) { sel[i] = false; pos[i] = 0; }
-    return;
+  uint32_t all_and = 0xFFFFFFFFu, all_or = 0u;
+#pragma unroll 4
+  for (int i = 0; i < nslab; ++i) {
+    const uint32_t k = sh.key[i * LOCKS_SEL_THREADS + tid];
+    if (k) { all_and &= k; all_or |= k; }
   }
-  uint32_t prefix = 0, mask = 0;
+  all_and = __reduce_and_sync(0xffffffffu, all_and);
+  all_or = __reduce_or_sync(0xffffffffu, all_or);
+  if (lane == 0) { sh.red[warp] = all_and; sh.red[kNW + warp] = all_or; }
+  __syncthreads();
+  all_and = sh.red[lane & (kNW - 1)];
+  all_or = sh.red[kNW + (lane & (kNW - 1))];
+  all_and = __reduce_and_sync(0xffffffffu, all_and);
+  all_or = __reduce_or_sync(0xffffffffu, all_or);
+  const int first = __clz(all_and ^ all_or) >> 3;   // leading bytes shared by every valid key (4: all keys equal)
+  uint32_t mask = first ? 0xFFFFFFFFu << (32 - 8 * first) : 0u;
+  uint32_t prefix = all_or & mask;
   int remaining = K;
-  for (int pass = 0; pass < 4; ++pass) {
+#pragma unroll 1
+  for (int pass = first; pass < 4; ++pass) {
     const int shift = 24 - 8 * pass;
     int *mine = sh.hist + warp * 256;
-#pragma unroll
-    for (int i = 0; i < EPT; ++i)
-      if (i < nslab && (key[i] & mask) == prefix) atomicAdd(&mine[(key[i] >> shift) & 255], 1);
+#pragma unroll 4
+    for (int i = 0; i < nslab; ++i) {
+      const uint32_t k = sh.key[i * LOCKS_SEL_THREADS + tid];
+      if (k && (k & mask) == prefix) atomicAdd(&mine[(k >> shift) & 255], 1);
+    }
     __syncthreads();
     int c = 0, incl = 0;
     if (tid < 256) {   // thread t owns bin 255 - t: bins are scanned from the largest digit down
@@ -114,6 +152,7 @@ __device__ void block_topk(const uint32_t (&key)[EPT], int K, bool (&sel)[EPT], 
     __syncthreads();
     if (tid < 256) {
       int before = incl - c;
+#pragma unroll 1
       for (int w = 0; w < warp; ++w) before += sh.wsum[w];
       if (before < remaining && remaining <= before + c) {
         sh.misc[(pass & 1) * 2] = 255 - tid;
@@ -125,24 +164,32 @@ __device__ void block_topk(const uint32_t (&key)[EPT], int K, bool (&sel)[EPT], 
     mask |= 255u << shift;
     remaining = sh.misc[(pass & 1) * 2 + 1];
   }
-  // prefix is the K-th largest key; `remaining` of the keys equal to it are taken, lowest index first.
-  // Ordered compaction: slab i holds indices i*512 .. i*512+511, one per thread.
-  uint32_t bg[EPT], be[EPT];
-#pragma unroll
-  for (int i = 0; i < EPT; ++i) {
-    bg[i] = be[i] = 0u;
-    if (i < nslab) {
-      bg[i] = __ballot_sync(0xffffffffu, key[i] > prefix);
-      be[i] = __ballot_sync(0xffffffffu, key[i] == prefix);
-    }
-    if (lane == 0) sh.cnt[i * kNW + warp] = (__popc(bg[i]) << 16) | __popc(be[i]);
+  return make_uint2(prefix, (uint32_t)remaining);
+}
+
+enum { kEmitIds = 0, kEmitList = 1, kEmitFinal = 2 };
+
+// Winners = keys above `prefix` plus the first `remaining` keys equal to it, in element order.  Winner
+// number `pos` (< cap) of element e is written as
+//   kEmitIds:   ids[1 + pos] = c0 + e                         (final table of a single-chunk problem)
+//   kEmitList:  list_key[pos] = key, list_idx[pos] = c0 + e   (a chunk's candidate list)
+//   kEmitFinal: ids[1 + pos] = list_idx[e]                    (final table from the problem's lists)
+__device__ __noinline__ void compact_emit(int nslab, uint32_t prefix, int remaining, int cap, int mode,
+                                          int c0, int32_t *ids, uint32_t *list_key, int32_t *list_idx) {
+  SelShared &sh = shared_state();
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+#pragma unroll 2
+  for (int i = 0; i < nslab; ++i) {
+    const uint32_t k = sh.key[i * LOCKS_SEL_THREADS + tid];
+    const uint32_t bg = __ballot_sync(0xffffffffu, k > prefix), be = __ballot_sync(0xffffffffu, k == prefix);
+    if (lane == 0) sh.cnt[i * kNW + warp] = (__popc(bg) << 16) | __popc(be);
   }
   __syncthreads();
-  if (warp == 0) {   // exclusive scan of the EPT*kNW counts in (slab, warp) order
-    constexpr int N = EPT * kNW, PER = (N + 31) / 32;
-    int v[PER], tot = 0;
-#pragma unroll
-    for (int u = 0; u < PER; ++u) { const int e = lane * PER + u; v[u] = e < N ? sh.cnt[e] : 0; tot += v[u]; }
+  if (warp == 0) {   // exclusive scan of the nslab * kNW counts in (slab, warp) order
+    const int n = nslab * kNW, per = (n + 31) / 32;
+    int tot = 0;
+#pragma unroll 1
+    for (int u = 0; u < per; ++u) { const int e = lane * per + u; tot += e < n ? sh.cnt[e] : 0; }
     int incl = tot;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
@@ -150,79 +197,199 @@ __device__ void block_topk(const uint32_t (&key)[EPT], int K, bool (&sel)[EPT], 
       if (lane >= o) incl += x;
     }
     int run = incl - tot;
-#pragma unroll
-    for (int u = 0; u < PER; ++u) { const int e = lane * PER + u; if (e < N) sh.cnt[e] = run; run += v[u]; }
+#pragma unroll 1
+    for (int u = 0; u < per; ++u) {
+      const int e = lane * per + u;
+      if (e < n) { const int v = sh.cnt[e]; sh.cnt[e] = run; run += v; }
+    }
   }
   __syncthreads();
   const uint32_t lt = (1u << lane) - 1u;
-#pragma unroll
-  for (int i = 0; i < EPT; ++i) {
+#pragma unroll 2
+  for (int i = 0; i < nslab; ++i) {
+    const int e = i * LOCKS_SEL_THREADS + tid;
+    const uint32_t k = sh.key[e];
+    const bool gt = k > prefix, eq = k == prefix;
+    const uint32_t bg = __ballot_sync(0xffffffffu, gt), be = __ballot_sync(0xffffffffu, eq);
     const int base = sh.cnt[i * kNW + warp];
-    const int gt_before = (base >> 16) + __popc(bg[i] & lt), eq_before = (base & 0xffff) + __popc(be[i] & lt);
-    const bool gt = key[i] > prefix, eq = key[i] == prefix;
-    sel[i] = gt || (eq && eq_before < remaining);
-    pos[i] = gt_before + min(eq_before, remaining);
+    const int gt_before = (base >> 16) + __popc(bg & lt), eq_before = (base & 0xffff) + __popc(be & lt);
+    const int pos = gt_before + min(eq_before, remaining);
+    if ((gt || (eq && eq_before < remaining)) && pos < cap) {
+      if (mode == kEmitIds) ids[1 + pos] = c0 + e;
+      else if (mode == kEmitList) { list_key[pos] = k; list_idx[pos] = c0 + e; }
+      else ids[1 + pos] = __ldcg(list_idx + e);
+    }
   }
 }
 
-__device__ __forceinline__ void lse_merge(float &m, float &s, float om, float os) {
-  const float nm = fmaxf(m, om);
-  if (nm > -INFINITY) {
-    s = s * __expf(m - nm) + os * __expf(om - nm);
-    m = nm;
-  }
-}
-
-// log Z_g of every head of the group from the scan's per-group partials -> sh_logz[g]
-__device__ void group_logz(const SelParams &p, int b, int h, int ngroups, float *sh_logz) {
+// log Z_g of every head of the group from the scan's partials (max_i, sum_i), part0 = head 0's row,
+// -> sh.lz2[g] (log2 domain):
+// log2 Z = M + log2 sum_i sum_i 2^(max_i - M), M = max_i max_i.  The block's warps are dealt to (head, slice)
+// pairs; a lane keeps four loads in flight.  Ends with the block synchronised.
+__device__ __noinline__ void group_logz(const float2 *part0, int G, int max_groups, int nparts) {
+  SelShared &sh = shared_state();
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  for (int g = warp; g < p.G; g += kNW) {
-    const float2 *pp = p.part + ((int64_t)b * p.Hq + h * p.G + g) * p.max_groups;
+  const int gw = min(G, kNW);            // heads handled per round
+  const int nslice = max(1, kNW / G);    // warps per head
+#pragma unroll 1
+  for (int g0 = 0; g0 < G; g0 += kNW) {  // one round unless G > 16
+    const int slice = warp / gw, g = g0 + warp - slice * gw;
     float m = -INFINITY, s = 0.f;
-    for (int i = lane; i < ngroups; i += 32) {
-      const float2 v = pp[i];
-      if (v.x > -INFINITY) lse_merge(m, s, v.x, v.y);
+    if (g < G && slice < nslice) {
+      const float2 *pp = part0 + (int64_t)g * max_groups;
+#pragma unroll 1
+      for (int i0 = slice * 32 + lane; i0 < nparts; i0 += 128 * nslice) {
+        float2 v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) v[u] = (i0 + 32 * nslice * u < nparts) ? pp[i0 + 32 * nslice * u] : make_float2(-INFINITY, 0.f);
+        const float nm = fmaxf(fmaxf(fmaxf(v[0].x, v[1].x), fmaxf(v[2].x, v[3].x)), m);
+        if (nm > -INFINITY) {
+          s *= ex2f((m - nm) * kLog2e);
+#pragma unroll
+          for (int u = 0; u < 4; ++u) s = fmaf(v[u].y, ex2f((v[u].x - nm) * kLog2e), s);
+          m = nm;
+        }
+      }
+      float M = m;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+      s = M > -INFINITY ? s * ex2f((m - M) * kLog2e) : 0.f;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+      m = M;
+    }
+    if (lane == 0) { sh.lzm[warp] = m; sh.lzs[warp] = s; }
+    __syncthreads();
+    if (threadIdx.x < min(G - g0, kNW)) {
+      float M = -INFINITY, S = 0.f;
+#pragma unroll 1
+      for (int sl = 0; sl < nslice; ++sl) M = fmaxf(M, sh.lzm[sl * gw + threadIdx.x]);
+#pragma unroll 1
+      for (int sl = 0; sl < nslice; ++sl) {
+        const float wm = sh.lzm[sl * gw + threadIdx.x];
+        if (wm > -INFINITY) S = fmaf(sh.lzs[sl * gw + threadIdx.x], ex2f((wm - M) * kLog2e), S);
+      }
+      sh.lz2[g0 + threadIdx.x] = M * kLog2e + lg2f(S);
+    }
+    __syncthreads();
+  }
+}
+
+// Keys of a chunk: log m_bar of page c0 + i*512 + t as an order-preserving integer in sh.key[i*512 + t]
+// (0 for pages that are not candidates).  Scores are fetched in batches of (16 / SB) heads x SB slabs, 16
+// loads in flight per thread, the next batch while the current one is reduced; the first batch is in
+// flight during the log Z reduction.  Per page a running (max, sum) over the heads, log2 domain.
+template <int SB>
+__device__ __noinline__ void chunk_keys(const float *shat0, const float2 *part0, float *logshare0, int G, int Pmax,
+                                        int max_groups, int nparts, int c0, int nslab, int P) {
+  constexpr int HB = 16 / SB;
+  SelShared &sh = shared_state();
+  const int tid = threadIdx.x;
+  const float *row0 = shat0 + c0 + tid;   // shat0: scores of the group's head 0, page 0
+  const int nG = (G + HB - 1) / HB, nb = ((nslab + SB - 1) / SB) * nG;
+  float cur[HB][SB], nxt[HB][SB];
+  auto load = [&](int i0, int g0, float (&x)[HB][SB]) {
+    bool ok[SB];
+#pragma unroll
+    for (int sl = 0; sl < SB; ++sl) {
+      const int page = c0 + (i0 + sl) * LOCKS_SEL_THREADS + tid;
+      ok[sl] = i0 + sl < nslab && page >= 1 && page <= P - 2;
+    }
+    const float *r = row0 + g0 * Pmax + i0 * LOCKS_SEL_THREADS;   // offsets within one request fit 32 bits
+#pragma unroll
+    for (int u = 0; u < HB; ++u)
+#pragma unroll
+      for (int sl = 0; sl < SB; ++sl)
+        x[u][sl] = (ok[sl] && g0 + u < G) ? r[u * Pmax + sl * LOCKS_SEL_THREADS] : -INFINITY;
+  };
+  load(0, 0, cur);
+  group_logz(part0, G, max_groups, nparts);
+  const float logG = __logf((float)G);
+  float m[SB], s[SB];
+#pragma unroll
+  for (int sl = 0; sl < SB; ++sl) { m[sl] = -INFINITY; s[sl] = 0.f; }
+  int i0 = 0, g0 = 0;
+#pragma unroll 1
+  for (int bi = 0; bi < nb; ++bi) {
+    int i1 = i0, g1 = g0 + HB;   // the batch after this one
+    if (g1 >= G) { g1 = 0; i1 += SB; }
+    if (bi + 1 < nb) load(i1, g1, nxt);
+#pragma unroll
+    for (int sl = 0; sl < SB; ++sl) {
+      float bm = -INFINITY;
+#pragma unroll
+      for (int u = 0; u < HB; ++u) {
+        cur[u][sl] = fmaf(cur[u][sl], kLog2e, -sh.lz2[min(g0 + u, 15)]);
+        bm = fmaxf(bm, cur[u][sl]);
+      }
+      const float nm = fmaxf(m[sl], bm);
+      float acc = s[sl] * ex2f(m[sl] - nm);
+#pragma unroll
+      for (int u = 0; u < HB; ++u) acc += ex2f(cur[u][sl] - nm);
+      s[sl] = acc;
+      m[sl] = nm;
+    }
+    if (g0 + HB >= G) {   // all heads seen: keys of these slabs
+#pragma unroll
+      for (int sl = 0; sl < SB; ++sl) {
+        const int i = i0 + sl, page = c0 + i * LOCKS_SEL_THREADS + tid;
+        if (i < nslab) {
+          const bool valid = page >= 1 && page <= P - 2;
+          const float val = (m[sl] + lg2f(s[sl])) * kLn2 - logG;
+          sh.key[i * LOCKS_SEL_THREADS + tid] = valid ? order_key(val) : 0u;
+          if (valid && logshare0) logshare0[page] = val;
+        }
+        m[sl] = -INFINITY;
+        s[sl] = 0.f;
+      }
     }
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) lse_merge(m, s, __shfl_xor_sync(0xffffffffu, m, o), __shfl_xor_sync(0xffffffffu, s, o));
-    if (lane == 0) sh_logz[g] = m + __logf(s);
+    for (int u = 0; u < HB; ++u)
+#pragma unroll
+      for (int sl = 0; sl < SB; ++sl) cur[u][sl] = nxt[u][sl];
+    i0 = i1;
+    g0 = g1;
   }
 }
 
-// log Z_g of one query head from the scan's per-group partials (used when a problem is ranked in chunks)
-__global__ void __launch_bounds__(256) logz_kernel(SelParams p) {
-  __shared__ float sm_m[8], sm_s[8];
-  const int hq = blockIdx.x, b = blockIdx.y, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  pdl_trigger();
-  pdl_wait();
-  const int T = p.seq_lens[b];
-  const int P = (T + LOCKS_B - 1) / LOCKS_B;
-  if (P <= p.k) return;
-  const int nparts = min(p.part_slots, (P - 1 + LOCKS_GROUP - 1) / LOCKS_GROUP);
-  const float2 *pp = p.part + ((int64_t)b * p.Hq + hq) * p.max_groups;
-  float m = -INFINITY, s = 0.f;
-  for (int i0 = threadIdx.x; i0 < nparts; i0 += 256 * 4) {   // four loads in flight per thread
-    float2 v[4];
-#pragma unroll
-    for (int u = 0; u < 4; ++u) v[u] = (i0 + 256 * u < nparts) ? pp[i0 + 256 * u] : make_float2(-INFINITY, 0.f);
-#pragma unroll
-    for (int u = 0; u < 4; ++u)
-      if (v[u].x > -INFINITY) lse_merge(m, s, v[u].x, v[u].y);
-  }
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) lse_merge(m, s, __shfl_xor_sync(0xffffffffu, m, o), __shfl_xor_sync(0xffffffffu, s, o));
-  if (lane == 0) { sm_m[warp] = m; sm_s[warp] = s; }
+// Several chunks per problem: the chunk that arrives last ranks the problem's candidate lists.
+__device__ __noinline__ void select_finish(int32_t *done, int chunks, int kc, int k, int32_t *ids, int32_t *count,
+                                           const uint32_t *ck, const int32_t *ci, int P) {
+  SelShared &sh = shared_state();
+  const int tid = threadIdx.x;
+  __threadfence();   // this chunk's list before its arrival
   __syncthreads();
-  if (threadIdx.x == 0) {
-    float M = -INFINITY, S = 0.f;
-    for (int w = 0; w < 8; ++w) lse_merge(M, S, sm_m[w], sm_s[w]);
-    p.logz[b * p.Hq + hq] = M + __logf(S);
+  if (tid == 0) {
+    const int ticket = atomicAdd(done, 1);
+    const bool last = ticket == chunks - 1;
+    if (last) *done = 0;   // every chunk has arrived: ready for the next launch
+    sh.misc[8] = last;
+  }
+  __syncthreads();
+  if (!sh.misc[8]) return;
+  __threadfence();
+  const int K2 = k - 2;
+  // entries in list order (chunk, position) = page order; element i of thread t is entry i*512 + t
+  const int N = chunks * kc;
+  const int nslab = (N + LOCKS_SEL_THREADS - 1) / LOCKS_SEL_THREADS;
+#pragma unroll 4
+  for (int i = 0; i < nslab; ++i) {
+    const int e = i * LOCKS_SEL_THREADS + tid;
+    sh.key[e] = e < N ? __ldcg(ck + e) : 0u;
+  }
+  if (K2 > 0) {
+    const uint2 r = radix_select(nslab, K2);
+    compact_emit(nslab, r.x, (int)r.y, K2, kEmitFinal, 0, ids, nullptr, const_cast<int32_t *>(ci));
+  }
+  if (tid == 0) {
+    ids[0] = 0;
+    ids[k - 1] = P - 1;
+    *count = k;
   }
 }
 
-template <int EPT>
-__global__ void __launch_bounds__(LOCKS_SEL_THREADS) select_stage1_kernel(SelParams p) {
-  __shared__ SelShared sh;
+__global__ void __launch_bounds__(LOCKS_SEL_THREADS) select_kernel(SelParams p) {
+  SelShared &sh = shared_state();
   const int chunk = blockIdx.x, h = blockIdx.y, b = blockIdx.z, tid = threadIdx.x;
   for (int e = tid; e < kNW * 256; e += LOCKS_SEL_THREADS) sh.hist[e] = 0;
   pdl_trigger();
@@ -241,128 +408,43 @@ __global__ void __launch_bounds__(LOCKS_SEL_THREADS) select_stage1_kernel(SelPar
     return;
   }
   const int c0 = chunk * p.chunk_pages;  // first page of this chunk
-  if (c0 > P - 2) {  // chunk past the candidates: emit an empty list
-    if (p.chunks > 1)
-      for (int j = tid; j < p.kc; j += LOCKS_SEL_THREADS) {
-        p.cand_val[(prob * p.chunks + chunk) * p.kc + j] = -INFINITY;
-        p.cand_idx[(prob * p.chunks + chunk) * p.kc + j] = -1;
-      }
+  if (c0 > P - 2) {  // chunk past the candidates: an empty list
+    if (p.chunks > 1) {
+      for (int j = tid; j < p.kc; j += LOCKS_SEL_THREADS) p.cand_key[(prob * p.chunks + chunk) * p.kc + j] = 0u;
+      select_finish(p.sel_done + prob, p.chunks, p.kc, p.k, ids, p.cnt + prob, p.cand_key + prob * p.chunks * p.kc,
+                    p.cand_idx + prob * p.chunks * p.kc, P);
+    }
     return;
   }
-  // scores of the first heads are fetched before the log Z reduction so that the two latencies overlap
-  constexpr int PRE = EPT <= 8 ? 4 : 2;
-  const float *row0 = p.shat + ((int64_t)b * p.Hq + h * p.G) * p.Pmax;
-  bool valid[EPT];
-  float raw[PRE][EPT];
   // slabs of 512 pages that hold at least one candidate of this chunk (the configured maximum context
   // is usually longer than the sequence)
-  const int nslab = min(EPT, (min(P - 1, c0 + p.chunk_pages) - c0 + LOCKS_SEL_THREADS - 1) / LOCKS_SEL_THREADS);
-#pragma unroll
-  for (int i = 0; i < EPT; ++i) {
-    const int page = c0 + i * LOCKS_SEL_THREADS + tid;
-    valid[i] = i < nslab && page >= 1 && page <= P - 2;
-  }
-#pragma unroll
-  for (int g = 0; g < PRE; ++g)
-#pragma unroll
-    for (int i = 0; i < EPT; ++i)
-      raw[g][i] = (g < p.G && valid[i]) ? row0[(int64_t)g * p.Pmax + c0 + i * LOCKS_SEL_THREADS + tid] : 0.f;
-  if (p.chunks == 1) group_logz(p, b, h, min(p.part_slots, (P - 1 + LOCKS_GROUP - 1) / LOCKS_GROUP), sh.logz);
-  else if (tid < p.G) sh.logz[tid] = p.logz[b * p.Hq + h * p.G + tid];
-  __syncthreads();
-  // log m_bar of this thread's pages: log mean_g exp(s^_g - log Z_g)
-  float val[EPT];
-  uint32_t key[EPT];
-  const float logG = __logf((float)p.G);
+  const int nslab = (min(P - 1, c0 + p.chunk_pages) - c0 + LOCKS_SEL_THREADS - 1) / LOCKS_SEL_THREADS;
   {
-    float mx[EPT], sm[EPT];
-#pragma unroll
-    for (int i = 0; i < EPT; ++i) { mx[i] = -INFINITY; sm[i] = 0.f; }
-#pragma unroll
-    for (int g = 0; g < PRE; ++g) {
-      if (g < p.G) {
-        const float lz = sh.logz[g];
-#pragma unroll
-        for (int i = 0; i < EPT; ++i)
-          if (valid[i]) lse_merge(mx[i], sm[i], raw[g][i] - lz, 1.f);
-      }
-    }
-    for (int g = PRE; g < p.G; ++g) {
-      const float *row = row0 + (int64_t)g * p.Pmax + c0 + tid;
-      const float lz = sh.logz[g];
-      float tv[EPT];
-#pragma unroll
-      for (int i = 0; i < EPT; ++i) tv[i] = (i < nslab && valid[i]) ? row[i * LOCKS_SEL_THREADS] : 0.f;
-#pragma unroll
-      for (int i = 0; i < EPT; ++i)
-        if (valid[i]) lse_merge(mx[i], sm[i], tv[i] - lz, 1.f);
-    }
-#pragma unroll
-    for (int i = 0; i < EPT; ++i) {
-      val[i] = valid[i] ? mx[i] + __logf(sm[i]) - logG : -INFINITY;
-      key[i] = valid[i] ? order_key(val[i]) : 0u;
-      if (valid[i] && p.logshare) p.logshare[prob * p.Pmax + c0 + i * LOCKS_SEL_THREADS + tid] = val[i];
-    }
+    const float *shat0 = p.shat + ((int64_t)b * p.Hq + h * p.G) * p.Pmax;
+    const float2 *part0 = p.part + ((int64_t)b * p.Hq + h * p.G) * p.max_groups;
+    float *ls0 = p.logshare ? p.logshare + prob * p.Pmax : nullptr;
+    const int nparts = min(p.part_slots, (P - 1 + LOCKS_GROUP - 1) / LOCKS_GROUP);
+    if (nslab >= 3) chunk_keys<4>(shat0, part0, ls0, p.G, p.Pmax, p.max_groups, nparts, c0, nslab, P);
+    else if (nslab == 2) chunk_keys<2>(shat0, part0, ls0, p.G, p.Pmax, p.max_groups, nparts, c0, nslab, P);
+    else chunk_keys<1>(shat0, part0, ls0, p.G, p.Pmax, p.max_groups, nparts, c0, nslab, P);
   }
   const int cand_in_chunk = min(P - 2, c0 + p.chunk_pages - 1) - max(1, c0) + 1;
   const int K = min(p.k - 2, cand_in_chunk);
-  bool sel[EPT];
-  int pos[EPT];
-  block_topk<EPT>(key, K, sel, pos, sh, nslab);
+  uint2 kth = make_uint2(0xFFFFFFFFu, 0u);
+  if (K > 0) kth = radix_select(nslab, K);
   if (p.chunks == 1) {
-#pragma unroll
-    for (int i = 0; i < EPT; ++i)
-      if (sel[i]) ids[1 + pos[i]] = c0 + i * LOCKS_SEL_THREADS + tid;
+    if (K > 0) compact_emit(nslab, kth.x, (int)kth.y, K, kEmitIds, c0, ids, nullptr, nullptr);
     if (tid == 0) {
       ids[0] = 0;
       ids[p.k - 1] = P - 1;
       p.cnt[prob] = p.k;
     }
   } else {
-    float *cv = p.cand_val + (prob * p.chunks + chunk) * p.kc;
-    int32_t *ci = p.cand_idx + (prob * p.chunks + chunk) * p.kc;
-#pragma unroll
-    for (int i = 0; i < EPT; ++i)
-      if (sel[i]) { cv[pos[i]] = val[i]; ci[pos[i]] = c0 + i * LOCKS_SEL_THREADS + tid; }
-    for (int j = K + tid; j < p.kc; j += LOCKS_SEL_THREADS) { cv[j] = -INFINITY; ci[j] = -1; }
-  }
-}
-
-template <int EPT>
-__global__ void __launch_bounds__(LOCKS_SEL_THREADS) select_stage2_kernel(SelParams p) {
-  __shared__ SelShared sh;
-  const int h = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
-  for (int e = tid; e < kNW * 256; e += LOCKS_SEL_THREADS) sh.hist[e] = 0;
-  pdl_trigger();
-  pdl_wait();   // stage 1's candidate lists
-  __syncthreads();
-  const int T = p.seq_lens[b];
-  const int P = (T + LOCKS_B - 1) / LOCKS_B;
-  if (P <= p.k) return;  // stage 1 already wrote the table
-  const int64_t prob = (int64_t)b * p.Hkv + h;
-  const int N = p.chunks * p.kc;
-  const float *cv = p.cand_val + prob * N;
-  const int32_t *ci = p.cand_idx + prob * N;
-  uint32_t key[EPT];
-  int idx[EPT];
-#pragma unroll
-  for (int i = 0; i < EPT; ++i) {
-    const int j = i * LOCKS_SEL_THREADS + tid;   // list position = ascending page order
-    const bool ok = j < N && ci[j] >= 0;
-    idx[i] = ok ? ci[j] : -1;
-    key[i] = ok ? order_key(cv[j]) : 0u;
-  }
-  bool sel[EPT];
-  int pos[EPT];
-  block_topk<EPT>(key, p.k - 2, sel, pos, sh);
-  int32_t *ids = p.ids + prob * p.k;
-#pragma unroll
-  for (int i = 0; i < EPT; ++i)
-    if (sel[i]) ids[1 + pos[i]] = idx[i];
-  if (tid == 0) {
-    ids[0] = 0;
-    ids[p.k - 1] = P - 1;
-    p.cnt[prob] = p.k;
+    uint32_t *lk = p.cand_key + (prob * p.chunks + chunk) * p.kc;
+    for (int j = K + tid; j < p.kc; j += LOCKS_SEL_THREADS) lk[j] = 0u;   // fewer candidates than list slots
+    if (K > 0) compact_emit(nslab, kth.x, (int)kth.y, K, kEmitList, c0, nullptr, lk, p.cand_idx + (prob * p.chunks + chunk) * p.kc);
+    select_finish(p.sel_done + prob, p.chunks, p.kc, p.k, ids, p.cnt + prob, p.cand_key + prob * p.chunks * p.kc,
+                  p.cand_idx + prob * p.chunks * p.kc, P);
   }
 }
 
@@ -375,28 +457,17 @@ int locks_launch_select(locks_ctx *c, const float *shat, const locks_kv *kv, int
   else p.app.k_new = nullptr;
   p.status = c->status;
   p.shat = shat; p.part = c->part; p.seq_lens = kv->seq_lens; p.ids = ids; p.cnt = cnt; p.logshare = logshare;
-  p.cand_val = c->cand_val; p.cand_idx = c->cand_idx;
+  p.cand_key = reinterpret_cast<uint32_t *>(c->cand_val); p.cand_idx = c->cand_idx; p.sel_done = c->sel_done;
   p.batch = batch; p.Hq = c->cfg.num_q_heads; p.Hkv = c->cfg.num_kv_heads; p.G = c->G; p.Pmax = c->Pmax;
   p.max_groups = c->max_groups; p.k = c->k; p.chunks = c->sel_chunks; p.kc = c->sel_kc;
   p.chunk_pages = c->sel_ept * LOCKS_SEL_THREADS;
-  p.logz = c->logz;
   p.part_slots = c->part_slots;
-  if (c->sel_chunks > 1) {
-    locks_launch_pdl(logz_kernel, dim3(p.Hq, batch), dim3(256), 0, st, p);
-    int rc0 = locks_check_launch(c);
-    if (rc0 != LOCKS_OK) return rc0;
+  if (p.chunk_pages > kMaxKeys || (int64_t)c->sel_chunks * c->sel_kc > kMaxKeys || p.G > 16) return LOCKS_ERR_UNSUPPORTED;
+  static bool attr_done = false;
+  if (!attr_done) {
+    cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(SelShared));
+    attr_done = true;
   }
-  dim3 g1(c->sel_chunks, p.Hkv, batch);
-  if (c->sel_ept == 4) locks_launch_pdl(select_stage1_kernel<4>, g1, dim3(LOCKS_SEL_THREADS), 0, st, p);
-  else if (c->sel_ept == 8) locks_launch_pdl(select_stage1_kernel<8>, g1, dim3(LOCKS_SEL_THREADS), 0, st, p);
-  else locks_launch_pdl(select_stage1_kernel<16>, g1, dim3(LOCKS_SEL_THREADS), 0, st, p);
-  int rc = locks_check_launch(c);
-  if (rc != LOCKS_OK || c->sel_chunks == 1) return rc;
-  const int N = c->sel_chunks * c->sel_kc;
-  const int ept = (N + LOCKS_SEL_THREADS - 1) / LOCKS_SEL_THREADS;
-  dim3 grid(p.Hkv, batch);
-  if (ept <= 4) locks_launch_pdl(select_stage2_kernel<4>, grid, dim3(LOCKS_SEL_THREADS), 0, st, p);
-  else if (ept <= 16) locks_launch_pdl(select_stage2_kernel<16>, grid, dim3(LOCKS_SEL_THREADS), 0, st, p);
-  else return LOCKS_ERR_UNSUPPORTED;
+  locks_launch_pdl(select_kernel, dim3(c->sel_chunks, p.Hkv, batch), dim3(LOCKS_SEL_THREADS), sizeof(SelShared), st, p);
   return locks_check_launch(c);
 }

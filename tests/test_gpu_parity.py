@@ -128,7 +128,7 @@ def test_i4_generic_ranks(rank):
 
 
 def test_two_level_select_long_context():
-    """More than one 8192-page chunk per KV head: stage-1 lists + stage-2 re-select."""
+    """Several chunks per KV head: per-chunk lists, then the last chunk to arrive ranks the survivors."""
     from gpu_util import check_select_and_attend
     gc = _gc(locks_synth.Workload("long", [16 * 9000 + 3], Hq=32, Hkv=2, budget=2048, seed=9))
     differed = check_select_and_attend(gc, gc.oracle_summaries(), out_tol=2e-2)
@@ -145,6 +145,20 @@ def test_ties_resolve_to_lower_index():
     summ = gc.oracle_summaries()
     ids, cnt, _, _ = gc.gpu_select(torch.from_numpy(summ).cuda())
     assert cnt[0, 0] == 8 and ids[0, 0].tolist() == [0, 1, 2, 3, 4, 5, 6, 39]
+
+
+@pytest.mark.parametrize("pages", [5000, 18500])
+def test_ties_across_chunks(pages):
+    """Every candidate ties and the problem spans several chunks: all list entries survive the
+    threshold (at 18500 pages more than the final round holds in shared memory, so it ranks them in
+    place); the lowest page indices must still win."""
+    gc = _gc(small_bf16([16 * pages + 5], Hq=4, Hkv=1, budget=2048))
+    gc.case.k.fill_(0.5)
+    gc.case.q.zero_()
+    gc.cache = __import__("common").oracle_cache(gc.case)
+    summ = gc.oracle_summaries()
+    ids, cnt, _, _ = gc.gpu_select(torch.from_numpy(summ).cuda())
+    assert cnt[0, 0] == 128 and ids[0, 0].tolist() == list(range(127)) + [pages]
 
 
 def test_gpu_i4_build_decoupled_parity():
