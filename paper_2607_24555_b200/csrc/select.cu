@@ -70,10 +70,9 @@ __device__ __forceinline__ void append_token(const locks_append &a, int batch, i
 
 struct SelShared {
   uint32_t key[kMaxKeys];             // order-preserving keys, element i of thread t at i*512 + t
-  int hist[kNW * 256];                // one 256-bin histogram per warp
-  int cnt[LOCKS_SEL_MAX_EPT * kNW];   // per (slab, warp) winner counts for the ordered compaction
+  int hist[3 * 256];                  // radix histograms, rotating
+  __align__(16) int cnt[256];         // per (slab, warp) winner counts for the ordered compaction
   int misc[16];                       // per-pass result (double-buffered), arrival flag
-  int wsum[8];
   float lz2[16];                      // log2-domain log Z_g
   float lzm[kNW], lzs[kNW];           // per-warp (max, sum) of the log Z reduction
   uint32_t red[2 * kNW];              // per-warp AND / OR of the keys
@@ -102,12 +101,14 @@ __device__ __forceinline__ uint32_t order_key(float f) {
 // K-th largest of the keys sh.key[i*512 + t], i < nslab (invalid elements hold key 0; 1 <= K <= number of
 // valid keys).  Returns (key, how many of the keys equal to it belong to the top K).
 // 8-bit radix passes from the top; leading bytes on which all valid keys agree (page masses share sign
-// and exponent) are skipped after one AND / OR reduction.  Every warp counts into its own histogram;
-// bin b of the block is then summed and suffix-scanned by thread 255 - b.  sh.hist must be zero on entry
-// and is zero on return.
+// and exponent) are skipped after one AND / OR reduction.  A pass costs one barrier: all warps count into
+// one 256-bin histogram, then every warp scans it on its own (lane l owns bins 8 (31 - l) .. + 7, so
+// lane order is descending digit order) while the histogram of the next pass -- three rotate -- is
+// already being filled by warps that are ahead.
 __device__ __noinline__ uint2 radix_select(int nslab, int K) {
   SelShared &sh = shared_state();
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (tid < 256) sh.hist[tid] = 0;
   uint32_t all_and = 0xFFFFFFFFu, all_or = 0u;
 #pragma unroll 4
   for (int i = 0; i < nslab; ++i) {
@@ -126,43 +127,43 @@ __device__ __noinline__ uint2 radix_select(int nslab, int K) {
   uint32_t mask = first ? 0xFFFFFFFFu << (32 - 8 * first) : 0u;
   uint32_t prefix = all_or & mask;
   int remaining = K;
+  int cur = 0;
 #pragma unroll 1
   for (int pass = first; pass < 4; ++pass) {
     const int shift = 24 - 8 * pass;
-    int *mine = sh.hist + warp * 256;
+    const int nxt = cur == 2 ? 0 : cur + 1;
+    int *hc = sh.hist + cur * 256;
+    if (tid < 256) sh.hist[nxt * 256 + tid] = 0;   // last read two passes ago
 #pragma unroll 4
     for (int i = 0; i < nslab; ++i) {
       const uint32_t k = sh.key[i * LOCKS_SEL_THREADS + tid];
-      if (k && (k & mask) == prefix) atomicAdd(&mine[(k >> shift) & 255], 1);
+      if (k && (k & mask) == prefix) atomicAdd(&hc[(k >> shift) & 255], 1);
     }
     __syncthreads();
-    int c = 0, incl = 0;
-    if (tid < 256) {   // thread t owns bin 255 - t: bins are scanned from the largest digit down
-      const int bin = 255 - tid;
+    const int base = 8 * (31 - lane);
+    const int4 lo = *reinterpret_cast<const int4 *>(hc + base), hi = *reinterpret_cast<const int4 *>(hc + base + 4);
+    const int c[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
+    const int tot = (c[0] + c[1]) + (c[2] + c[3]) + (c[4] + c[5]) + (c[6] + c[7]);
+    int incl = tot;
 #pragma unroll
-      for (int w = 0; w < kNW; ++w) { c += sh.hist[w * 256 + bin]; sh.hist[w * 256 + bin] = 0; }
-      incl = c;
+    for (int o = 1; o < 32; o <<= 1) {
+      const int v = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += v;
+    }
+    const bool hit = incl - tot < remaining && remaining <= incl;   // the K-th largest falls in this lane's bins
+    int digit = 0, rem = 0, acc = incl - tot;
 #pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        int v = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += v;
-      }
-      if (lane == 31) sh.wsum[warp] = incl;
+    for (int j = 7; j >= 0; --j) {
+      if (hit && acc < remaining && remaining <= acc + c[j]) { digit = base + j; rem = remaining - acc; }
+      acc += c[j];
     }
-    __syncthreads();
-    if (tid < 256) {
-      int before = incl - c;
-#pragma unroll 1
-      for (int w = 0; w < warp; ++w) before += sh.wsum[w];
-      if (before < remaining && remaining <= before + c) {
-        sh.misc[(pass & 1) * 2] = 255 - tid;
-        sh.misc[(pass & 1) * 2 + 1] = remaining - before;
-      }
-    }
-    __syncthreads();
-    prefix |= (uint32_t)sh.misc[(pass & 1) * 2] << shift;
+    const uint32_t who = __ballot_sync(0xffffffffu, hit);
+    const int src = who ? __ffs(who) - 1 : 0;
+    digit = __shfl_sync(0xffffffffu, digit, src);
+    remaining = __shfl_sync(0xffffffffu, rem, src);
+    prefix |= (uint32_t)digit << shift;
     mask |= 255u << shift;
-    remaining = sh.misc[(pass & 1) * 2 + 1];
+    cur = nxt;
   }
   return make_uint2(prefix, (uint32_t)remaining);
 }
@@ -178,6 +179,7 @@ __device__ __noinline__ void compact_emit(int nslab, uint32_t prefix, int remain
                                           int c0, int32_t *ids, uint32_t *list_key, int32_t *list_idx) {
   SelShared &sh = shared_state();
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  __syncthreads();   // the previous user of sh.cnt is done
 #pragma unroll 2
   for (int i = 0; i < nslab; ++i) {
     const uint32_t k = sh.key[i * LOCKS_SEL_THREADS + tid];
@@ -185,23 +187,25 @@ __device__ __noinline__ void compact_emit(int nslab, uint32_t prefix, int remain
     if (lane == 0) sh.cnt[i * kNW + warp] = (__popc(bg) << 16) | __popc(be);
   }
   __syncthreads();
-  if (warp == 0) {   // exclusive scan of the nslab * kNW counts in (slab, warp) order
-    const int n = nslab * kNW, per = (n + 31) / 32;
+  if (warp == 0) {   // exclusive scan of the nslab * kNW (<= 256) counts in (slab, warp) order, 8 per lane
+    const int n = nslab * kNW;
+    int4 *q = reinterpret_cast<int4 *>(sh.cnt + lane * 8);
+    int4 lo = q[0], hi = q[1];
+    int c[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
     int tot = 0;
-#pragma unroll 1
-    for (int u = 0; u < per; ++u) { const int e = lane * per + u; tot += e < n ? sh.cnt[e] : 0; }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) { if (lane * 8 + j >= n) c[j] = 0; tot += c[j]; }
     int incl = tot;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
-      int x = __shfl_up_sync(0xffffffffu, incl, o);
-      if (lane >= o) incl += x;
+      const int v = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += v;
     }
     int run = incl - tot;
-#pragma unroll 1
-    for (int u = 0; u < per; ++u) {
-      const int e = lane * per + u;
-      if (e < n) { const int v = sh.cnt[e]; sh.cnt[e] = run; run += v; }
-    }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) { const int v = c[j]; c[j] = run; run += v; }
+    q[0] = make_int4(c[0], c[1], c[2], c[3]);
+    q[1] = make_int4(c[4], c[5], c[6], c[7]);
   }
   __syncthreads();
   const uint32_t lt = (1u << lane) - 1u;
@@ -391,7 +395,6 @@ __device__ __noinline__ void select_finish(int32_t *done, int chunks, int kc, in
 __global__ void __launch_bounds__(LOCKS_SEL_THREADS) select_kernel(SelParams p) {
   SelShared &sh = shared_state();
   const int chunk = blockIdx.x, h = blockIdx.y, b = blockIdx.z, tid = threadIdx.x;
-  for (int e = tid; e < kNW * 256; e += LOCKS_SEL_THREADS) sh.hist[e] = 0;
   pdl_trigger();
   pdl_wait();   // the scan's scores and partials
   const int T = p.seq_lens[b];
