@@ -340,7 +340,7 @@ def run_ours(args):
         "e2e": {"value": e2e_ms_max * 1e3, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": launches_per_step * K,
         "clocks": clocks,
-        "roofline": {"bound": "hbm", "kernel": "scan_i4r8_kernel", "achieved": scan_gbs, "peak": peak, "unit": "GB/s",
+        "roofline": {"bound": "hbm", "kernel": "scan_i4_kernel", "achieved": scan_gbs, "peak": peak, "unit": "GB/s",
                      "frac": scan_gbs / peak, "peak_kind": f"of {peak_kind}", "traffic": recorded_traffic(w0.name),
                      "algorithmic_bytes_per_launch": scan_b, "launch_us": stage_ms["scan"] * 1e3},
         "step_roofline": {"algorithmic_bytes": scan_b + att_b, "achieved": (scan_b + att_b) / (step_ms_max * 1e-3) / 1e9,

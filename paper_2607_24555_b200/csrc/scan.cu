@@ -6,7 +6,8 @@
 // Two kernels:
 //   scan_generic_kernel   any format / rank / dtype, plain fp32 ALU arithmetic (parity config, fallback
 //                         shapes).  One warp per group of 8 pages.
-//   scan_i4r8_kernel      the bytes-bound path for the r8i4 blob with bf16 queries.  Persistent warps,
+//   scan_i4_kernel<R>     the bytes-bound path for int4/int8 blobs of rank R = 2, 4, 8 with bf16 queries (ranks
+//                         below 8 run the rank-8 tile with the missing ranks fed as zeros).  Persistent warps,
 //                         each streaming groups of 8 blobs through its own shared-memory ring with bulk
 //                         async copies (TMA engine) and mbarriers, no CTA-wide synchronisation.  Per page pair:
 //                           MMA#1  P[2 pages x 8 ranks, heads] = codesV[16 x d] . q^T[d x heads]   (8 x m16n8k16 fp16)
@@ -165,8 +166,7 @@ __global__ void __launch_bounds__(128) scan_generic_kernel(ScanParams p) {
 constexpr int kScanWarps = 8;
 constexpr int kScanStages = 2;
 constexpr int kScanCtasPerSm = 2;
-constexpr int kBlob = i4_stride(8);                       // 832
-constexpr int kStageBytes = LOCKS_GROUP * kBlob;          // 6656
+constexpr int kStageBytes = LOCKS_GROUP * i4_stride(8);   // 6656: a stage holds 8 summaries of any rank
 constexpr int kScanRedBytes = kScanWarps * 16 * 8;         // (max, sum) of 16 heads per warp, for the CTA-level merge
 constexpr int kScanSmem = kScanWarps * (kScanStages * kStageBytes + 64) + kScanRedBytes;
 constexpr bool kScanBulk = LOCKS_SCAN_BULK;             // true: cp.async.bulk + mbarrier, false: 16-byte cp.async
@@ -232,8 +232,9 @@ __device__ __forceinline__ uint32_t movm_trans(uint32_t v) {
 // PK (G <= 4 only): the 8 head columns hold the group twice, so that after MMA#1 the projection, MMA#2 and
 // the log-sum-exp handle two pages at once (rows 0-3 = page A's heads, rows 4-7 = page B's heads, the two
 // pages separated along K) instead of leaving half of the lanes idle.
-template <int NH, bool PK, bool CR>
-__global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4r8_kernel(ScanParams p) {
+template <int R, int NH, bool PK, bool CR>
+__global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4_kernel(ScanParams p) {
+  constexpr int kBlob = i4_stride(R);   // stored bytes of one summary; a stage keeps room for rank-8 blobs
   extern __shared__ __align__(128) uint8_t smem[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int x = lane >> 2, t = lane & 3;
@@ -291,17 +292,14 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4r8_ker
         bulk_g2s(ring + stage * kStageBytes + lane * kBlob, p.summ + ((int64_t)block * p.Hkv + h) * kBlob, kBlob,
                  &full[stage]);
     } else {
-      // 52 16-byte chunks per blob: lanes 0-25 copy chunks lane and lane + 26 of every page of the group
-      uint8_t *dst = ring + stage * kStageBytes + lane * 16;
+      // 16-byte chunks of a blob are dealt to the lanes
+      uint8_t *dst = ring + stage * kStageBytes;
 #pragma unroll
       for (int pg = 0; pg < LOCKS_GROUP; ++pg) {
         const int blk = __shfl_sync(0xffffffffu, block, pg);
-        const uint8_t *src = p.summ + ((int64_t)blk * p.Hkv + h) * kBlob + lane * 16;
-        const bool on = lane < 26 && pg < nvalid;
-        if (on) {
-          cp_async16(dst + pg * kBlob, src, true);
-          cp_async16(dst + pg * kBlob + 416, src + 416, true);
-        }
+        const uint8_t *src = p.summ + ((int64_t)blk * p.Hkv + h) * kBlob;
+        if (pg < nvalid)
+          for (int c = lane; c < kBlob / 16; c += 32) cp_async16(dst + pg * kBlob + c * 16, src + c * 16, true);
       }
       cp_async_commit();
     }
@@ -449,7 +447,7 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4r8_ker
     // ---- centroid dots of the 8 pages: cen[head x (+8)][pages 2t, 2t+1] = sum_c code_mu[c] q'[c]
     float cen[4] = {0.f, 0.f, 0.f, 0.f};
     {
-      const uint4 *mp = reinterpret_cast<const uint4 *>(sb + (x & (LOCKS_GROUP - 1)) * kBlob + i4_off_mu(8) + t * 32);
+      const uint4 *mp = reinterpret_cast<const uint4 *>(sb + (x & (LOCKS_GROUP - 1)) * kBlob + i4_off_mu(R) + t * 32);
       const uint4 m0 = mp[0], m1 = mp[1];
       const uint32_t mw[8] = {m0.x, m0.y, m0.z, m0.w, m1.x, m1.y, m1.z, m1.w};
 #pragma unroll
@@ -463,8 +461,8 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4r8_ker
     float acen[2 * NH];  // log2-domain centroid term of pages 2t, 2t+1 for head x (and x + 8)
     {
       const int pg0 = (2 * t) & (LOCKS_GROUP - 1);   // lanes t >= LOCKS_GROUP / 2 hold nothing useful
-      const float s0 = __half2float(*reinterpret_cast<const __half *>(sb + pg0 * kBlob + i4_off_smu(8)));
-      const float s1 = __half2float(*reinterpret_cast<const __half *>(sb + (pg0 + 1) * kBlob + i4_off_smu(8)));
+      const float s0 = __half2float(*reinterpret_cast<const __half *>(sb + pg0 * kBlob + i4_off_smu(R)));
+      const float s1 = __half2float(*reinterpret_cast<const __half *>(sb + (pg0 + 1) * kBlob + i4_off_smu(R)));
 #pragma unroll
       for (int hh = 0; hh < NH; ++hh) {
         acen[2 * hh] = s0 * (c2 * inv_s[hh]) * cen[2 * hh];
@@ -479,8 +477,9 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4r8_ker
     for (int pp = 0; pp < LOCKS_GROUP / 2; ++pp) {
       const uint8_t *pbA = sb + (2 * pp) * kBlob, *pbB = pbA + kBlob;
       // ---- MMA #1: rows = (page A ranks 0-7, page B ranks 0-7), cols = heads, k = this lane quarter's dims
-      const uint4 wa4 = *reinterpret_cast<const uint4 *>(pbA + lane * 16);
-      const uint4 wb4 = *reinterpret_cast<const uint4 *>(pbB + lane * 16);
+      // lane (x, t) holds rank x, dim quarter t; ranks >= R do not exist (their column scale reads as 0 below)
+      const uint4 wa4 = (R == 8 || x < R) ? *reinterpret_cast<const uint4 *>(pbA + lane * 16) : make_uint4(0u, 0u, 0u, 0u);
+      const uint4 wb4 = (R == 8 || x < R) ? *reinterpret_cast<const uint4 *>(pbB + lane * 16) : make_uint4(0u, 0u, 0u, 0u);
       const uint32_t wa[4] = {wa4.x, wa4.y, wa4.z, wa4.w}, wb[4] = {wb4.x, wb4.y, wb4.z, wb4.w};
       float c1[NH][4];
 #pragma unroll
@@ -497,7 +496,7 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4r8_ker
         // lanes t < 2 carry page A (columns 0-3), lanes t >= 2 page B (columns 4-7)
         const bool pa = t < 2;
         const uint8_t *pbs = pa ? pbA : pbB;
-        const float sv = __half2float(*reinterpret_cast<const __half *>(pbs + i4_off_sv(8) + 2 * x));
+        const float sv = (R == 8 || x < R) ? __half2float(*reinterpret_cast<const __half *>(pbs + i4_off_sv(R) + 2 * x)) : 0.f;
         const float p0 = fmaf(pa ? c1[0][0] : c1[0][2], 16777216.f, -ksum[0]) * sv;
         const float p1 = fmaf(pa ? c1[0][1] : c1[0][3], 16777216.f, -ksum[1]) * sv;
         const uint32_t hi = pack_f16(p0, p1);
@@ -506,8 +505,9 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4r8_ker
         const uint32_t hiT = movm_trans(hi), loT = movm_trans(lo);   // lane (x, t): row x, ranks 2t, 2t+1
         const bool ra = x < 4;                                        // row x: page A head x | page B head x - 4
         const uint32_t hA = ra ? hiT : 0u, hB = ra ? 0u : hiT, lA = ra ? loT : 0u, lB = ra ? 0u : loT;
-        const uint32_t cwa = *reinterpret_cast<const uint32_t *>(pbA + i4_off_coef(8) + lane * 4);
-        const uint32_t cwb = *reinterpret_cast<const uint32_t *>(pbB + i4_off_coef(8) + lane * 4);
+        // lane (x, t): tokens x and x + 8, ranks 2t and 2t + 1; missing rank pairs read as code 0
+        const uint32_t cwa = (t < R / 2) ? *reinterpret_cast<const uint32_t *>(pbA + i4_off_coef(R) + (x * (R / 2) + t) * 4) : 0x80808080u;
+        const uint32_t cwb = (t < R / 2) ? *reinterpret_cast<const uint32_t *>(pbB + i4_off_coef(R) + (x * (R / 2) + t) * 4) : 0x80808080u;
         const uint32_t a0 = f16x2_sub(__byte_perm(cwa, 0x64646464u, 0x4140), kSub128);
         const uint32_t a1 = f16x2_sub(__byte_perm(cwa, 0x64646464u, 0x4342), kSub128);
         const uint32_t b0 = f16x2_sub(__byte_perm(cwb, 0x64646464u, 0x4140), kSub128);
@@ -518,7 +518,7 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4r8_ker
         mma_f16(ca, lA, 0u, lB, 0u, a0, b0);
         mma_f16_z(cb, hA, 0u, hB, 0u, a1, b1);
         mma_f16(cb, lA, 0u, lB, 0u, a1, b1);
-        const uint2 scw = *reinterpret_cast<const uint2 *>((ra ? pbA : pbB) + i4_off_sc(8) + 8 * t);
+        const uint2 scw = *reinterpret_cast<const uint2 *>((ra ? pbA : pbB) + i4_off_sc(R) + 8 * t);
         const float2 s01 = h2f2(scw.x), s89 = h2f2(scw.y);
         const float iv = inv_s[0] * c2;
         const float y0 = ca[0] * s01.x, y1 = ca[1] * s01.y, y2 = cb[0] * s89.x, y3 = cb[1] * s89.y;
@@ -538,7 +538,7 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4r8_ker
         const int pg = 2 * pp + pq;
         const uint8_t *pb = pq ? pbB : pbA;
         // projection of rank x for heads 2t, 2t+1: undo 2^-24, remove the +8 offset, apply the column scale
-        const float sv = __half2float(*reinterpret_cast<const __half *>(pb + i4_off_sv(8) + 2 * x));
+        const float sv = (R == 8 || x < R) ? __half2float(*reinterpret_cast<const __half *>(pb + i4_off_sv(R) + 2 * x)) : 0.f;
         uint32_t hiT[NH], loT[NH];
 #pragma unroll
         for (int hh = 0; hh < NH; ++hh) {
@@ -551,13 +551,13 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4r8_ker
           loT[hh] = movm_trans(lo);
         }
         // ---- MMA #2: rows = heads, k = ranks (hi | lo), cols = tokens
-        const uint32_t cw = *reinterpret_cast<const uint32_t *>(pb + i4_off_coef(8) + lane * 4);
+        const uint32_t cw = (t < R / 2) ? *reinterpret_cast<const uint32_t *>(pb + i4_off_coef(R) + (x * (R / 2) + t) * 4) : 0x80808080u;
         const uint32_t b0 = f16x2_sub(__byte_perm(cw, 0x64646464u, 0x4140), kSub128);
         const uint32_t b1 = f16x2_sub(__byte_perm(cw, 0x64646464u, 0x4342), kSub128);
         float ca[4], cb[4];
         mma_f16_z(ca, hiT[0], NH == 2 ? hiT[NH - 1] : 0u, loT[0], NH == 2 ? loT[NH - 1] : 0u, b0, b0);
         mma_f16_z(cb, hiT[0], NH == 2 ? hiT[NH - 1] : 0u, loT[0], NH == 2 ? loT[NH - 1] : 0u, b1, b1);
-        const uint2 scw = *reinterpret_cast<const uint2 *>(pb + i4_off_sc(8) + 8 * t);
+        const uint2 scw = *reinterpret_cast<const uint2 *>(pb + i4_off_sc(R) + 8 * t);
         const float2 s01 = h2f2(scw.x), s89 = h2f2(scw.y);
 #pragma unroll
         for (int hh = 0; hh < NH; ++hh) {
@@ -661,19 +661,9 @@ int locks_launch_scan(locks_ctx *c, const void *q, const void *summaries, const 
   p.batch = batch; p.Hq = c->cfg.num_q_heads; p.Hkv = c->cfg.num_kv_heads; p.G = c->G;
   p.Pmax = c->Pmax; p.max_groups = c->max_groups; p.num_blocks = kv->num_blocks; p.k = c->k;
   p.S = c->S; p.r = c->cfg.rank; p.sm_scale = c->cfg.sm_scale;
-  const bool tensor = c->cfg.summary_fmt == LOCKS_FMT_I4 && c->cfg.rank == 8 && c->cfg.q_dtype == LOCKS_BF16;
+  const bool tensor = c->cfg.summary_fmt == LOCKS_FMT_I4 && c->cfg.q_dtype == LOCKS_BF16;   // ranks 2, 4, 8
   c->part_slots = c->max_groups;   // generic kernel: one partial per 8-page group
   if (tensor) {
-    static bool attr_done = false;
-    if (!attr_done) {
-      cudaFuncSetAttribute(scan_i4r8_kernel<1, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kScanSmem);
-      cudaFuncSetAttribute(scan_i4r8_kernel<1, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kScanSmem);
-      cudaFuncSetAttribute(scan_i4r8_kernel<2, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kScanSmem);
-      cudaFuncSetAttribute(scan_i4r8_kernel<1, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kScanSmem);
-      cudaFuncSetAttribute(scan_i4r8_kernel<1, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kScanSmem);
-      cudaFuncSetAttribute(scan_i4r8_kernel<2, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kScanSmem);
-      attr_done = true;
-    }
     const int total_groups = batch * p.Hkv * p.max_groups;
     int grid = kScanCtasPerSm * c->num_sms;
     const int need = (total_groups + kScanWarps - 1) / kScanWarps;
@@ -684,19 +674,29 @@ int locks_launch_scan(locks_ctx *c, const void *q, const void *summaries, const 
       c->part_slots = wpp;
       // few problems: every CTA's warps share one problem for the whole launch and none leaves early,
       // so the CTA merges its warps' partials before writing (the selector reads 8x fewer)
-      p.cta_reduce = (wpp % kScanWarps == 0 && nslots == nprob && nslots * wpp == W) ? 1 : 0;
+      p.cta_reduce = (c->cfg.rank == 8 && wpp % kScanWarps == 0 && nslots == nprob && nslots * wpp == W) ? 1 : 0;
       if (p.cta_reduce) c->part_slots = wpp / kScanWarps;
     }
     const dim3 g(grid), blk(kScanWarps * 32);
-    if (p.cta_reduce) {
-      if (c->G <= 4) locks_launch_pdl(scan_i4r8_kernel<1, true, true>, g, blk, kScanSmem, st, p);
-      else if (c->G <= 8) locks_launch_pdl(scan_i4r8_kernel<1, false, true>, g, blk, kScanSmem, st, p);
-      else locks_launch_pdl(scan_i4r8_kernel<2, false, true>, g, blk, kScanSmem, st, p);
-    } else {
-      if (c->G <= 4) locks_launch_pdl(scan_i4r8_kernel<1, true, false>, g, blk, kScanSmem, st, p);
-      else if (c->G <= 8) locks_launch_pdl(scan_i4r8_kernel<1, false, false>, g, blk, kScanSmem, st, p);
-      else locks_launch_pdl(scan_i4r8_kernel<2, false, false>, g, blk, kScanSmem, st, p);
-    }
+    const int gsel = c->G <= 4 ? 0 : (c->G <= 8 ? 1 : 2);
+#define LOCKS_SCAN_LAUNCH(R_, CR_)                                                                                     \
+  do {                                                                                                                 \
+    static bool attr_done = false;                                                                                     \
+    if (!attr_done) {                                                                                                  \
+      cudaFuncSetAttribute(scan_i4_kernel<R_, 1, true, CR_>, cudaFuncAttributeMaxDynamicSharedMemorySize, kScanSmem);  \
+      cudaFuncSetAttribute(scan_i4_kernel<R_, 1, false, CR_>, cudaFuncAttributeMaxDynamicSharedMemorySize, kScanSmem); \
+      cudaFuncSetAttribute(scan_i4_kernel<R_, 2, false, CR_>, cudaFuncAttributeMaxDynamicSharedMemorySize, kScanSmem); \
+      attr_done = true;                                                                                                \
+    }                                                                                                                  \
+    if (gsel == 0) locks_launch_pdl(scan_i4_kernel<R_, 1, true, CR_>, g, blk, kScanSmem, st, p);                       \
+    else if (gsel == 1) locks_launch_pdl(scan_i4_kernel<R_, 1, false, CR_>, g, blk, kScanSmem, st, p);                 \
+    else locks_launch_pdl(scan_i4_kernel<R_, 2, false, CR_>, g, blk, kScanSmem, st, p);                                \
+  } while (0)
+    if (c->cfg.rank == 8 && p.cta_reduce) LOCKS_SCAN_LAUNCH(8, true);
+    else if (c->cfg.rank == 8) LOCKS_SCAN_LAUNCH(8, false);
+    else if (c->cfg.rank == 4) LOCKS_SCAN_LAUNCH(4, false);
+    else LOCKS_SCAN_LAUNCH(2, false);
+#undef LOCKS_SCAN_LAUNCH
   } else {
     dim3 grid((c->max_groups + 3) / 4, p.Hkv, batch);
     const bool qbf = c->cfg.q_dtype == LOCKS_BF16;

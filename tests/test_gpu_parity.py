@@ -127,6 +127,22 @@ def test_i4_generic_ranks(rank):
     check_select_and_attend(gc, gc.oracle_summaries(), out_tol=2e-2)
 
 
+@pytest.mark.parametrize("rank", [2, 8])
+def test_i4_summaries_with_fp32_queries(rank):
+    """Quantised summaries with fp32 K, V and q: the plain fp32-arithmetic scan and attention paths."""
+    from gpu_util import check_select_and_attend
+    gc = _gc(small_bf16([1000, 700], rank=rank, seed=40 + rank, dtype="f32"))
+    check_select_and_attend(gc, gc.oracle_summaries(), out_tol=1e-4)
+
+
+@pytest.mark.parametrize("Hq,Hkv", [(12, 2), (32, 2)])
+def test_i4_rank2_group_sizes(Hq, Hkv):
+    """Rank-2 summaries through the tensor-core scan at group sizes 6 and 16."""
+    from gpu_util import check_select_and_attend
+    gc = _gc(small_bf16([1500, 900], Hq=Hq, Hkv=Hkv, rank=2, seed=50 + Hq))
+    check_select_and_attend(gc, gc.oracle_summaries(), out_tol=2e-2)
+
+
 def test_two_level_select_long_context():
     """Several chunks per KV head: per-chunk lists, then the last chunk to arrive ranks the survivors."""
     from gpu_util import check_select_and_attend
