@@ -20,6 +20,7 @@ namespace {
 
 constexpr int kNW = LOCKS_SEL_THREADS / 32;
 constexpr int kMaxKeys = LOCKS_SEL_MAX_EPT * LOCKS_SEL_THREADS;   // keys one CTA ranks at most
+constexpr int kMaxWin = 4 * LOCKS_SEL_THREADS;                    // k - 2 at most (checked on the host)
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 
@@ -76,6 +77,7 @@ struct SelShared {
   float lz2[16];                      // log2-domain log Z_g
   float lzm[kNW], lzs[kNW];           // per-warp (max, sum) of the log Z reduction
   uint32_t red[2 * kNW];              // per-warp AND / OR of the keys
+  int win[kMaxWin];                   // final round: entry index of winner number pos
 };
 
 extern __shared__ __align__(16) uint8_t sel_smem[];
@@ -179,6 +181,8 @@ __device__ __noinline__ void compact_emit(int nslab, uint32_t prefix, int remain
                                           int c0, int32_t *ids, uint32_t *list_key, int32_t *list_idx) {
   SelShared &sh = shared_state();
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (mode == kEmitFinal)
+    for (int j = tid; j < cap; j += LOCKS_SEL_THREADS) sh.win[j] = 0;   // a slot no winner fills still names a real entry
   __syncthreads();   // the previous user of sh.cnt is done
 #pragma unroll 2
   for (int i = 0; i < nslab; ++i) {
@@ -221,7 +225,17 @@ __device__ __noinline__ void compact_emit(int nslab, uint32_t prefix, int remain
     if ((gt || (eq && eq_before < remaining)) && pos < cap) {
       if (mode == kEmitIds) ids[1 + pos] = c0 + e;
       else if (mode == kEmitList) { list_key[pos] = k; list_idx[pos] = c0 + e; }
-      else ids[1 + pos] = __ldcg(list_idx + e);
+      else sh.win[pos] = e;   // the page of entry e is fetched below, all winners at once
+    }
+  }
+  if (mode == kEmitFinal) {
+    __syncthreads();
+    for (int j0 = tid; j0 < cap; j0 += 4 * LOCKS_SEL_THREADS) {
+      int v[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) { const int j = j0 + u * LOCKS_SEL_THREADS; v[u] = j < cap ? __ldcg(list_idx + sh.win[j]) : 0; }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) { const int j = j0 + u * LOCKS_SEL_THREADS; if (j < cap) ids[1 + j] = v[u]; }
     }
   }
 }
@@ -323,7 +337,7 @@ __device__ __noinline__ void chunk_keys(const float *shat0, const float2 *part0,
       float bm = -INFINITY;
 #pragma unroll
       for (int u = 0; u < HB; ++u) {
-        cur[u][sl] = fmaf(cur[u][sl], kLog2e, -sh.lz2[min(g0 + u, 15)]);
+        cur[u][sl] = fmaf(cur[u][sl], kLog2e, g0 + u < G ? -sh.lz2[g0 + u] : 0.f);   // heads past the group stay -inf
         bm = fmaxf(bm, cur[u][sl]);
       }
       const float nm = fmaxf(m[sl], bm);
