@@ -123,6 +123,7 @@ int locks_create(const locks_config *cfg, void *workspace, size_t ws_bytes, lock
   if (!c) return LOCKS_ERR_INVALID_ARG;
   c->cfg = *cfg;
   c->prof_ev = nullptr; c->prof_cap = c->prof_n = 0;
+  c->att_cluster_max = -1;
   c->part_slots = L.max_groups;
   c->G = L.G; c->k = L.k; c->S = L.S; c->Pmax = cfg->max_pages_per_seq; c->max_groups = L.max_groups;
   c->sel_ept = L.sel_ept; c->sel_chunks = L.sel_chunks; c->sel_kc = L.sel_kc;

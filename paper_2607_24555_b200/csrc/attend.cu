@@ -6,6 +6,7 @@
 // KV head are the M rows), keeps a running (max, sum, O) per head, and the CTA merges its warps by
 // log-sum-exp.  Partial (o, lse) per split are merged by a second small kernel.
 // A NULL page table means "all pages": the same kernel is the dense flash-decode baseline.
+#include <cooperative_groups.h>
 #include "locks_internal.cuh"
 
 namespace {
@@ -27,6 +28,7 @@ struct AttParams {
   int32_t *done;   // [batch*Hkv] split-arrival counters (zero between launches)
   int batch, Hq, Hkv, G, Pmax, kbud, num_blocks, splits, pages_per_cta;
   int fused_merge;   // 1: the last CTA of a problem merges its splits; 0: a separate merge kernel follows
+  int cluster;       // 1: the splits of a problem form one thread-block cluster and merge through its shared memory
   float sm_scale;
 };
 
@@ -268,6 +270,72 @@ __global__ void __launch_bounds__(LOCKS_ATT_WARPS * 32) attend_bf16_kernel(AttPa
     }
   }
   __syncthreads();
+  if (p.cluster) {
+    // The splits of this (request, KV head) are the CTAs of one cluster.  Each CTA first folds its warps into
+    // one unnormalised partial in its own shared memory; after a cluster barrier CTA r produces a slice of the
+    // problem's G x 128 outputs by reading every CTA's partial through distributed shared memory; a second
+    // barrier keeps every CTA's memory alive until its peers are done.  No partial leaves the SMs.
+    namespace cg = cooperative_groups;
+    cg::cluster_group cluster = cg::this_cluster();
+    constexpr int NT = LOCKS_ATT_WARPS * 32;
+    // the CTA's partial replaces warp 0's in place (element e is read and written by one thread only); its
+    // (max, sum) go to the idle tail of warp 1's ring, because other threads still read warp 0's
+    float *co = reinterpret_cast<float *>(smem);
+    float *cm = reinterpret_cast<float *>(smem + kAttStages * kAttStage) + 16 * LOCKS_D + 32, *cl = cm + 16;
+    for (int e = threadIdx.x; e < p.G * LOCKS_D; e += NT) {
+      const int g = e / LOCKS_D, dim = e - g * LOCKS_D;
+      float M = -INFINITY;
+#pragma unroll
+      for (int w = 0; w < LOCKS_ATT_WARPS; ++w)
+        M = fmaxf(M, reinterpret_cast<const float *>(smem + w * kAttStages * kAttStage)[16 * LOCKS_D + g]);
+      float L = 0.f, o = 0.f;
+      if (M > -INFINITY) {
+#pragma unroll
+        for (int w = 0; w < LOCKS_ATT_WARPS; ++w) {
+          const float *ww = reinterpret_cast<const float *>(smem + w * kAttStages * kAttStage);
+          const float sc = ex2f(ww[16 * LOCKS_D + g] - M);
+          L += ww[16 * LOCKS_D + 16 + g] * sc;
+          o += ww[g * LOCKS_D + dim] * sc;
+        }
+      }
+      co[e] = o;
+      if (dim == 0) { cm[g] = M; cl[g] = L; }
+    }
+    cluster.sync();
+    const int nout = p.G * LOCKS_D, per = (nout + p.splits - 1) / p.splits;
+    const int e1 = min(nout, (split + 1) * per);
+    for (int e = split * per + threadIdx.x; e < e1; e += NT) {
+      const int g = e / LOCKS_D;
+      float mv[16], lv[16], ov[16];
+#pragma unroll
+      for (int c = 0; c < 16; ++c) {
+        mv[c] = -INFINITY; lv[c] = 0.f; ov[c] = 0.f;
+        if (c < p.splits) {
+          mv[c] = cluster.map_shared_rank(cm, c)[g];
+          lv[c] = cluster.map_shared_rank(cl, c)[g];
+          ov[c] = cluster.map_shared_rank(co, c)[e];
+        }
+      }
+      float M = -INFINITY;
+#pragma unroll
+      for (int c = 0; c < 16; ++c) M = fmaxf(M, mv[c]);
+      float L = 0.f, o = 0.f;
+      if (M > -INFINITY) {
+#pragma unroll
+        for (int c = 0; c < 16; ++c) {
+          const float sc = ex2f(mv[c] - M);
+          L = fmaf(lv[c], sc, L);
+          o = fmaf(ov[c], sc, o);
+        }
+        o /= L;
+      }
+      const int64_t row = (int64_t)b * p.Hq + h * p.G + g;
+      reinterpret_cast<__nv_bfloat16 *>(p.out)[row * LOCKS_D + (e - g * LOCKS_D)] = __float2bfloat16_rn(o);
+      if (p.lse && e == g * LOCKS_D) p.lse[row] = (M > -INFINITY) ? (M + log2f(L)) * kLn2 : -INFINITY;
+    }
+    cluster.sync();
+    return;
+  }
   for (int e = threadIdx.x; e < p.G * LOCKS_D; e += LOCKS_ATT_WARPS * 32) {
     const int g = e / LOCKS_D, dim = e - g * LOCKS_D;
     float M = -INFINITY;
@@ -487,6 +555,40 @@ int locks_launch_attend(locks_ctx *c, const void *q, const locks_kv *kv, int bat
   // a single CTA merging many splits of many heads is a serial tail: beyond 64 (head, split) pairs use the
   // parallel merge kernel instead
   p.fused_merge = (c->G * p.splits <= 64) ? 1 : 0;
+  // Preferred: the splits of a problem as one thread-block cluster (2, 4, 8 or 16 CTAs) that merges through
+  // distributed shared memory, as long as a CTA then has at most 8 pages per warp to stream.
+  p.cluster = 0;
+  if (c->att_cluster_max < 0) {   // largest cluster of this kernel the device can place (probed once)
+    c->att_cluster_max = 0;
+    cudaFuncSetAttribute(attend_bf16_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttSmem);
+    cudaFuncSetAttribute(attend_bf16_kernel<1, true>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+    for (int cs = 16; cs >= 2 && c->att_cluster_max == 0; cs /= 2) {
+      cudaLaunchConfig_t lc = {};
+      lc.gridDim = dim3(cs, 1, 1);
+      lc.blockDim = dim3(LOCKS_ATT_WARPS * 32);
+      lc.dynamicSmemBytes = kAttSmem;
+      cudaLaunchAttribute at[1];
+      at[0].id = cudaLaunchAttributeClusterDimension;
+      at[0].val.clusterDim.x = cs; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+      lc.attrs = at;
+      lc.numAttrs = 1;
+      int nclusters = 0;
+      if (cudaOccupancyMaxActiveClusters(&nclusters, attend_bf16_kernel<1, true>, &lc) == cudaSuccess && nclusters > 0)
+        c->att_cluster_max = cs;
+    }
+    (void)cudaGetLastError();   // a refused probe is not an error of this call
+  }
+  if (c->cfg.kv_dtype == LOCKS_BF16 && splits >= 2 && c->att_cluster_max >= 2) {
+    int cs = 2;
+    while (cs * 2 <= splits && cs * 2 <= c->att_cluster_max) cs *= 2;
+    const int ppc = (npages + cs - 1) / cs;
+    if (ppc <= 8 * LOCKS_ATT_WARPS && (npages + ppc - 1) / ppc == cs) {
+      p.cluster = 1;
+      p.pages_per_cta = ppc;
+      p.splits = cs;
+      p.fused_merge = 1;   // no merge launch follows
+    }
+  }
   const bool bf = c->cfg.kv_dtype == LOCKS_BF16;
   if (bf) {
     static bool attr_done = false;
@@ -495,12 +597,24 @@ int locks_launch_attend(locks_ctx *c, const void *q, const locks_kv *kv, int bat
       cudaFuncSetAttribute(attend_bf16_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttSmem);
       cudaFuncSetAttribute(attend_bf16_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttSmem);
       cudaFuncSetAttribute(attend_bf16_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttSmem);
+      cudaFuncSetAttribute(attend_bf16_kernel<1, true>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+      cudaFuncSetAttribute(attend_bf16_kernel<2, true>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+      cudaFuncSetAttribute(attend_bf16_kernel<1, false>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+      cudaFuncSetAttribute(attend_bf16_kernel<2, false>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
       attr_done = true;
     }
     dim3 grid(p.splits, p.Hkv, batch);
     const bool contig = kv->stride_token == LOCKS_D;
     const dim3 blk(LOCKS_ATT_WARPS * 32);
-    if (c->G <= 8) {
+    if (p.cluster) {
+      if (c->G <= 8) {
+        if (contig) locks_launch_pdl_cluster(attend_bf16_kernel<1, true>, grid, blk, kAttSmem, p.splits, st, p);
+        else locks_launch_pdl_cluster(attend_bf16_kernel<1, false>, grid, blk, kAttSmem, p.splits, st, p);
+      } else {
+        if (contig) locks_launch_pdl_cluster(attend_bf16_kernel<2, true>, grid, blk, kAttSmem, p.splits, st, p);
+        else locks_launch_pdl_cluster(attend_bf16_kernel<2, false>, grid, blk, kAttSmem, p.splits, st, p);
+      }
+    } else if (c->G <= 8) {
       if (contig) locks_launch_pdl(attend_bf16_kernel<1, true>, grid, blk, kAttSmem, st, p);
       else locks_launch_pdl(attend_bf16_kernel<1, false>, grid, blk, kAttSmem, st, p);
     } else {
@@ -601,6 +715,7 @@ extern "C" int locks_sparse_attend_noalloc(const locks_config *cfg, const void *
   p.pages_per_cta = (npages + splits - 1) / splits;
   p.splits = (npages + p.pages_per_cta - 1) / p.pages_per_cta;
   p.fused_merge = 1;
+  p.cluster = 0;
   // the array keeps whatever the last call left: the arrival counters and the status word must start at zero
   if (cudaMemsetAsync(p.done, 0, kNoAllocDone + 256, st) != cudaSuccess) return LOCKS_ERR_CUDA;
   dim3 grid(p.splits, p.Hkv, batch);

@@ -49,6 +49,7 @@ struct locks_ctx {
   cudaStream_t side;       // build of freshly filled pages runs beside attend
   cudaEvent_t ev_fork, ev_join;
   int last_launches;
+  int att_cluster_max;     // largest thread-block cluster the attention kernel may use (-1: not probed yet)
   // optional per-stage timing of eager decode steps (see locks_profile_begin)
   cudaEvent_t *prof_ev;    // [prof_cap][LOCKS_PROF_MARKS]
   int prof_cap, prof_n;
@@ -93,6 +94,28 @@ static inline void locks_launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 bl
   at[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = at;
   cfg.numAttrs = 1;
+  (void)cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+
+// The same, with the grid's x dimension grouped into thread-block clusters of `cluster_x` CTAs
+// (distributed shared memory between the CTAs of a cluster).
+template <typename... KArgs, typename... Args>
+static inline void locks_launch_pdl_cluster(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, int cluster_x,
+                                            cudaStream_t st, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute at[2];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  at[1].id = cudaLaunchAttributeClusterDimension;
+  at[1].val.clusterDim.x = cluster_x;
+  at[1].val.clusterDim.y = 1;
+  at[1].val.clusterDim.z = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = 2;
   (void)cudaLaunchKernelEx(&cfg, kernel, args...);
 }
 
