@@ -332,6 +332,7 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4_kerne
   // query of the current problem: qb0/qb2 = this lane's dims of head x (tile 0) / head x + 8 (tile 1)
   uint32_t qb0[NH][8], qb2[NH][8];
   float inv_s[NH], ksum[2 * NH];   // 1/scale of head x (+8); 8 * sum_c q'[c] of heads 2t, 2t+1 (+8)
+  float inv2[2 * NH];              // 1/scale of heads 2t, 2t+1 (+8)
   int cur_prob = -1;
   const __nv_bfloat16 *q = reinterpret_cast<const __nv_bfloat16 *>(p.q);
   const float c2 = p.sm_scale * kLog2e;
@@ -440,12 +441,17 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4_kerne
         // lane (x, t) owns head gx; the column fragment needs the heads of columns 2t, 2t+1
         ksum[2 * hh] = __shfl_sync(0xffffffffu, s8, (2 * t) * 4);
         ksum[2 * hh + 1] = __shfl_sync(0xffffffffu, s8, (2 * t + 1) * 4);
+        inv2[2 * hh] = __shfl_sync(0xffffffffu, inv_s[hh], (2 * t) * 4);
+        inv2[2 * hh + 1] = __shfl_sync(0xffffffffu, inv_s[hh], (2 * t + 1) * 4);
       }
     }
 
     const uint8_t *sb = ring + stage * kStageBytes;
-    // ---- centroid dots of the 8 pages: cen[head x (+8)][pages 2t, 2t+1] = sum_c code_mu[c] q'[c]
-    float cen[4] = {0.f, 0.f, 0.f, 0.f};
+    // ---- centroid dots of the 8 pages.  Pages are the MMA rows (rows 8-15 idle) and the query is the B operand,
+    // the same register pairs MMA #1 uses: cenT[hh][0..1] = sum_c code_mu[page x][c] q'[head 2t, 2t+1 (+8 hh)][c]
+    float cenT[NH][4];
+#pragma unroll
+    for (int hh = 0; hh < NH; ++hh) cenT[hh][0] = cenT[hh][1] = cenT[hh][2] = cenT[hh][3] = 0.f;
     {
       const uint4 *mp = reinterpret_cast<const uint4 *>(sb + (x & (LOCKS_GROUP - 1)) * kBlob + i4_off_mu(R) + t * 32);
       const uint4 m0 = mp[0], m1 = mp[1];
@@ -455,18 +461,29 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4_kerne
         const uint32_t w = mw[s];
         const uint32_t b0 = f16x2_sub(and_or(w, kMB, kMagic), kSub128);              // code
         const uint32_t b1 = f16x2_fma(and_or(w >> 8, kMB, kMagic), kSixteen, kNeg16x);  // 16 * code
-        mma_f16(cen, qb0[0][s], NH == 2 ? qb0[NH - 1][s] : 0u, qb2[0][s], NH == 2 ? qb2[NH - 1][s] : 0u, b0, b1);
+#pragma unroll
+        for (int hh = 0; hh < NH; ++hh) mma_f16(cenT[hh], b0, 0u, b1, 0u, qb0[hh][s], qb2[hh][s]);
       }
     }
-    float acen[2 * NH];  // log2-domain centroid term of pages 2t, 2t+1 for head x (and x + 8)
+    // scaled at the lane that holds them (page x, heads 2t, 2t+1), then moved to the lanes that finish the pages
+    float acen[2 * NH];  // log2-domain centroid term: packed, of this lane's (page, head); else of pages 2t, 2t+1 for head x (+8)
     {
-      const int pg0 = (2 * t) & (LOCKS_GROUP - 1);   // lanes t >= LOCKS_GROUP / 2 hold nothing useful
-      const float s0 = __half2float(*reinterpret_cast<const __half *>(sb + pg0 * kBlob + i4_off_smu(R)));
-      const float s1 = __half2float(*reinterpret_cast<const __half *>(sb + (pg0 + 1) * kBlob + i4_off_smu(R)));
+      const float smu = __half2float(*reinterpret_cast<const __half *>(sb + (x & (LOCKS_GROUP - 1)) * kBlob + i4_off_smu(R)));
 #pragma unroll
       for (int hh = 0; hh < NH; ++hh) {
-        acen[2 * hh] = s0 * (c2 * inv_s[hh]) * cen[2 * hh];
-        acen[2 * hh + 1] = s1 * (c2 * inv_s[hh]) * cen[2 * hh + 1];
+        const float v0 = smu * (c2 * inv2[2 * hh]) * cenT[hh][0], v1 = smu * (c2 * inv2[2 * hh + 1]) * cenT[hh][1];
+        if (PK) {   // lane (x, t) finishes page 2t + (x >> 2), head x & 3: held by lane (that page, (x & 3) >> 1)
+          const int src = (2 * t + (x >> 2)) * 4 + ((x & 3) >> 1);
+          const float a0 = __shfl_sync(0xffffffffu, v0, src), a1 = __shfl_sync(0xffffffffu, v1, src);
+          acen[0] = (x & 1) ? a1 : a0;
+          acen[1] = 0.f;
+        } else {    // lane (x, t) finishes pages 2t, 2t + 1 for head x (+8 hh): held by lanes (page, x >> 1)
+          const int srcA = (2 * t) * 4 + (x >> 1), srcB = srcA + 4;
+          const float a0 = __shfl_sync(0xffffffffu, v0, srcA), a1 = __shfl_sync(0xffffffffu, v1, srcA);
+          const float b0 = __shfl_sync(0xffffffffu, v0, srcB), b1 = __shfl_sync(0xffffffffu, v1, srcB);
+          acen[2 * hh] = (x & 1) ? a1 : a0;
+          acen[2 * hh + 1] = (x & 1) ? b1 : b0;
+        }
       }
     }
     float res[2 * NH];
@@ -531,7 +548,7 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4_kerne
         e += __shfl_xor_sync(0xffffffffu, e, 1);
         e += __shfl_xor_sync(0xffffffffu, e, 2);
         // lane (x, t = pp) keeps the result of page 2 pp + (x >> 2), head x & 3
-        if (t == pp) res[0] = m + fast_lg2(e) + (ra ? acen[0] : acen[1]);
+        if (t == pp) res[0] = m + fast_lg2(e) + acen[0];
       } else {
 #pragma unroll
       for (int pq = 0; pq < 2; ++pq) {
