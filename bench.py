@@ -11,7 +11,10 @@ Cold caches: the step touches about 175 MB and B200's L2 holds 126 MB, so the re
 several independent "layers" (own KV cache, summaries and query), as a real model would; by the
 time a layer comes round again its lines are gone.
 
-Prints ONE JSON line (see README for the keys).  `--impl reference` times the CPU
+Prints ONE JSON line: metric / value / unit, the step time, `e2e` (the same step through the host-buffer entry
+point, copies included), `roofline` (scan kernel: algorithmic bytes / measured kernel time against the measured
+copy bandwidth, plus the kernel's DRAM traffic from the committed ncu capture), `cpu_baseline` (the oracle on the
+host cores), per-stage times, the dense flash-decode time on the same inputs, clocks and launch count.  `--impl reference` times the CPU
 oracle instead (test infrastructure; the only other place this file runs it is `cpu_baseline`).
 """
 from __future__ import annotations
@@ -54,7 +57,8 @@ def workload(name: str):
 
 
 def algorithmic_bytes(w, reserve_tokens=0):
-    """Bytes the method itself must move per step."""
+    """Bytes the method itself must move per step: 818 B (r8i4 payload) per scored (page, KV head) for the scan,
+    8192 B per selected (page, KV head) for attention."""
     payload = {8: 818, 4: 490, 2: 326}[w.rank] if w.fmt == "i4" else 4 * (128 + w.rank * 128 + 16 * w.rank)
     scan = attend = dense = 0
     for T in w.seq_lens:

@@ -1,6 +1,8 @@
 """GPU parity: the CUDA path (through the C ABI) against the CPU oracle on the same seeded inputs.
 
-Tolerances (written here, derived in the design doc): page log-masses and log-shares within 1e-3;
+Tolerances: page log-masses and log-shares within 1e-3 (fp32 accumulation of exactly represented integer
+codes: observed ~1e-5); outputs 2e-2 for bf16 KV because the probabilities enter the PV product as bf16 (8
+bits: <= 2^-9 |v|max ~ 1e-2 per output) and the output itself is rounded to bf16 (4e-3);
 selected page sets identical except inside a 2e-3 tie band around the oracle's threshold;
 attention outputs within 2e-2 (bf16 KV) / 1e-4 (fp32); lse within 1e-3.
 """
