@@ -311,12 +311,12 @@ def run_ours(args):
         hk = [n[0].cpu().pin_memory() for n in news]
         hv = [n[1].cpu().pin_memory() for n in news]
         hout = torch.empty_like(outs[0], device="cpu").pin_memory()
-        for i in range(3):
+        for i in range(3 * L):   # every layer's arguments seen often enough for the library to cache its launch
             ctx.locks_decode_step_host(hq[i % L], hk[i % L], hv[i % L], kvs[i % L], summs[i % L], w0.n, hout, stream=stream)
         ldist.barrier()
         t0 = time.perf_counter()
         for i in range(K):
-            li = (3 + i) % L
+            li = (3 * L + i) % L
             ctx.locks_decode_step_host(hq[li], hk[li], hv[li], kvs[li], summs[li], w0.n, hout, stream=stream)
         e2e_ms = (time.perf_counter() - t0) * 1e3 / K
     status = ctx.locks_poll_status()

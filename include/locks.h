@@ -151,7 +151,11 @@ int locks_decode_step(locks_ctx *ctx, const void *q, const void *k_new, const vo
  * to be asynchronous): copies q_host (and k_new_host / v_new_host if given) to staging space in
  * the workspace, runs locks_decode_step, copies out back to out_host (and the page ids / counts
  * if page_ids_host / page_count_host are given) and synchronises the stream before returning.
- * The cache, summaries, block table and seq_lens stay on the device. */
+ * The cache, summaries, block table and seq_lens stay on the device.
+ * Repeated calls with the same arguments (a serving loop calls once per layer and step with fixed
+ * buffers) are cached: from the third call on, the copies and the step are one CUDA-graph launch.
+ * The cache holds 8 argument sets per context, needs page-locked host buffers and a stream that is
+ * not being captured, and is released by locks_destroy(); other calls take the plain path. */
 int locks_decode_step_host(locks_ctx *ctx, const void *q_host, const void *k_new_host,
                            const void *v_new_host, locks_kv *kv, void *summaries, int batch,
                            void *out_host, int32_t *page_ids_host, int32_t *page_count_host,

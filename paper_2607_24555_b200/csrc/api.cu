@@ -124,6 +124,8 @@ int locks_create(const locks_config *cfg, void *workspace, size_t ws_bytes, lock
   c->cfg = *cfg;
   c->prof_ev = nullptr; c->prof_cap = c->prof_n = 0;
   c->att_cluster_max = -1;
+  for (int i = 0; i < LOCKS_HOST_GRAPHS; ++i) c->hg[i] = locks_host_graph{};
+  c->hg_next = 0;
   c->part_slots = L.max_groups;
   c->G = L.G; c->k = L.k; c->S = L.S; c->Pmax = cfg->max_pages_per_seq; c->max_groups = L.max_groups;
   c->sel_ept = L.sel_ept; c->sel_chunks = L.sel_chunks; c->sel_kc = L.sel_kc;
@@ -168,6 +170,8 @@ int locks_destroy(locks_ctx *ctx) {
     for (int i = 0; i < ctx->prof_cap * LOCKS_PROF_MARKS; ++i) cudaEventDestroy(ctx->prof_ev[i]);
     delete[] ctx->prof_ev;
   }
+  for (int i = 0; i < LOCKS_HOST_GRAPHS; ++i)
+    if (ctx->hg[i].exec) cudaGraphExecDestroy(ctx->hg[i].exec);
   cudaEventDestroy(ctx->ev_fork);
   cudaEventDestroy(ctx->ev_join);
   cudaStreamDestroy(ctx->side);
@@ -261,13 +265,12 @@ int locks_decode_step(locks_ctx *ctx, const void *q, const void *k_new, const vo
   return LOCKS_OK;
 }
 
-int locks_decode_step_host(locks_ctx *ctx, const void *q_host, const void *k_new_host, const void *v_new_host,
-                           locks_kv *kv, void *summaries, int batch, void *out_host, int32_t *page_ids_host,
-                           int32_t *page_count_host, locks_stream stream) {
-  int rc = check_common(ctx, kv, batch);
-  if (rc != LOCKS_OK) return rc;
-  if (!q_host || !out_host || ((k_new_host == nullptr) != (v_new_host == nullptr))) return LOCKS_ERR_INVALID_ARG;
-  cudaStream_t st = (cudaStream_t)stream;
+namespace {
+
+// copies in, the step, copies out -- enqueued on `st` (eagerly, or under capture)
+int enqueue_host_step(locks_ctx *ctx, const void *q_host, const void *k_new_host, const void *v_new_host, locks_kv *kv,
+                      void *summaries, int batch, void *out_host, int32_t *page_ids_host, int32_t *page_count_host,
+                      cudaStream_t st) {
   const size_t esz = ctx->cfg.q_dtype == LOCKS_BF16 ? 2 : 4;
   const size_t qb = (size_t)batch * ctx->cfg.num_q_heads * LOCKS_D * esz;
   const size_t kb = (size_t)batch * ctx->cfg.num_kv_heads * LOCKS_D * esz;
@@ -277,10 +280,9 @@ int locks_decode_step_host(locks_ctx *ctx, const void *q_host, const void *k_new
         cudaMemcpyAsync(ctx->stage_vn, v_new_host, kb, cudaMemcpyHostToDevice, st) != cudaSuccess)
       return LOCKS_ERR_CUDA;
   }
-  rc = locks_decode_step(ctx, ctx->stage_q, k_new_host ? ctx->stage_kn : nullptr, k_new_host ? ctx->stage_vn : nullptr,
-                         kv, summaries, batch, ctx->stage_out, ctx->ids_int, ctx->cnt_int, stream);
+  int rc = locks_decode_step(ctx, ctx->stage_q, k_new_host ? ctx->stage_kn : nullptr, k_new_host ? ctx->stage_vn : nullptr,
+                             kv, summaries, batch, ctx->stage_out, ctx->ids_int, ctx->cnt_int, (locks_stream)st);
   if (rc != LOCKS_OK) return rc;
-  const int launches = ctx->last_launches;
   if (cudaMemcpyAsync(out_host, ctx->stage_out, qb, cudaMemcpyDeviceToHost, st) != cudaSuccess) return LOCKS_ERR_CUDA;
   if (page_ids_host &&
       cudaMemcpyAsync(page_ids_host, ctx->ids_int, (size_t)batch * ctx->cfg.num_kv_heads * ctx->k * 4,
@@ -290,6 +292,75 @@ int locks_decode_step_host(locks_ctx *ctx, const void *q_host, const void *k_new
       cudaMemcpyAsync(page_count_host, ctx->cnt_int, (size_t)batch * ctx->cfg.num_kv_heads * 4, cudaMemcpyDeviceToHost,
                       st) != cudaSuccess)
     return LOCKS_ERR_CUDA;
+  return LOCKS_OK;
+}
+
+bool is_pinned(const void *p) {   // page-locked host memory (or nothing to copy)
+  if (!p) return true;
+  cudaPointerAttributes a;
+  if (cudaPointerGetAttributes(&a, p) != cudaSuccess) { (void)cudaGetLastError(); return false; }
+  return a.type == cudaMemoryTypeHost;
+}
+
+}  // namespace
+
+int locks_decode_step_host(locks_ctx *ctx, const void *q_host, const void *k_new_host, const void *v_new_host,
+                           locks_kv *kv, void *summaries, int batch, void *out_host, int32_t *page_ids_host,
+                           int32_t *page_count_host, locks_stream stream) {
+  int rc = check_common(ctx, kv, batch);
+  if (rc != LOCKS_OK) return rc;
+  if (!q_host || !out_host || ((k_new_host == nullptr) != (v_new_host == nullptr))) return LOCKS_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  // A caller that repeats the same arguments (one set per layer, every decode step) gets the whole call as
+  // one graph launch from the second repetition on: the copies and the four launches cost one submission.
+  // Needs page-locked host buffers, a stream that is not being captured, and per-stage timing switched off.
+  cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+  const bool graph_ok = cudaStreamIsCapturing(st, &cap) == cudaSuccess && cap == cudaStreamCaptureStatusNone &&
+                        !ctx->prof_ev && is_pinned(q_host) && is_pinned(k_new_host) && is_pinned(v_new_host) &&
+                        is_pinned(out_host) && is_pinned(page_ids_host) && is_pinned(page_count_host);
+  locks_host_graph *g = nullptr;
+  if (graph_ok) {
+    for (int i = 0; i < LOCKS_HOST_GRAPHS && !g; ++i) {
+      locks_host_graph &e = ctx->hg[i];
+      if (e.seen > 0 && e.q == q_host && e.kn == k_new_host && e.vn == v_new_host && e.out == out_host &&
+          e.summ == summaries && e.ids == page_ids_host && e.cnt == page_count_host && e.batch == batch && e.st == st &&
+          e.kv.k == kv->k && e.kv.v == kv->v && e.kv.stride_block == kv->stride_block &&
+          e.kv.stride_head == kv->stride_head && e.kv.stride_token == kv->stride_token &&
+          e.kv.num_blocks == kv->num_blocks && e.kv.block_table == kv->block_table && e.kv.seq_lens == kv->seq_lens)
+        g = &e;
+    }
+    if (!g) {   // new arguments: take the next slot
+      g = &ctx->hg[ctx->hg_next];
+      ctx->hg_next = (ctx->hg_next + 1) % LOCKS_HOST_GRAPHS;
+      if (g->exec) cudaGraphExecDestroy(g->exec);
+      *g = locks_host_graph{q_host, k_new_host, v_new_host, out_host, summaries, page_ids_host, page_count_host, *kv,
+                            batch, st, 0, 0, nullptr};
+    }
+    if (!g->exec && g->seen >= 1) {   // second call with these arguments: capture
+      cudaGraph_t graph = nullptr;
+      if (cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal) == cudaSuccess) {
+        rc = enqueue_host_step(ctx, q_host, k_new_host, v_new_host, kv, summaries, batch, out_host, page_ids_host,
+                               page_count_host, st);
+        g->launches = ctx->last_launches;
+        const cudaError_t ce = cudaStreamEndCapture(st, &graph);
+        if (rc == LOCKS_OK && ce == cudaSuccess && graph) {
+          if (cudaGraphInstantiate(&g->exec, graph, 0) != cudaSuccess) g->exec = nullptr;
+        }
+        if (graph) cudaGraphDestroy(graph);
+      }
+      (void)cudaGetLastError();   // a failed capture falls back to the eager path below
+    }
+    if (g->exec) {
+      if (cudaGraphLaunch(g->exec, st) != cudaSuccess || cudaStreamSynchronize(st) != cudaSuccess) return LOCKS_ERR_CUDA;
+      ctx->last_launches = g->launches;
+      return LOCKS_OK;
+    }
+    g->seen++;
+  }
+  rc = enqueue_host_step(ctx, q_host, k_new_host, v_new_host, kv, summaries, batch, out_host, page_ids_host,
+                         page_count_host, st);
+  if (rc != LOCKS_OK) return rc;
+  const int launches = ctx->last_launches;
   if (cudaStreamSynchronize(st) != cudaSuccess) return LOCKS_ERR_CUDA;
   ctx->last_launches = launches;
   return LOCKS_OK;

@@ -22,6 +22,20 @@
 #endif
 #define LOCKS_SPIN_LIMIT (1 << 22)  // bounded mbarrier polling (each poll already waits a while)
 
+// One cached CUDA graph of the host-buffer decode step (copies in, step, copies out) for one set of arguments.
+struct locks_host_graph {
+  const void *q, *kn, *vn;
+  void *out, *summ;
+  int32_t *ids, *cnt;
+  locks_kv kv;
+  int batch;
+  cudaStream_t st;
+  int seen;                 // eager calls made with these arguments
+  int launches;
+  cudaGraphExec_t exec;     // nullptr until the arguments have been seen twice
+};
+#define LOCKS_HOST_GRAPHS 8
+
 struct locks_ctx {
   locks_config cfg;
   int G, k, S, Pmax, max_groups;
@@ -49,6 +63,8 @@ struct locks_ctx {
   cudaStream_t side;       // build of freshly filled pages runs beside attend
   cudaEvent_t ev_fork, ev_join;
   int last_launches;
+  locks_host_graph hg[LOCKS_HOST_GRAPHS];
+  int hg_next;
   int att_cluster_max;     // largest thread-block cluster the attention kernel may use (-1: not probed yet)
   // optional per-stage timing of eager decode steps (see locks_profile_begin)
   cudaEvent_t *prof_ev;    // [prof_cap][LOCKS_PROF_MARKS]
