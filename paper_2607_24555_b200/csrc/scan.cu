@@ -490,6 +490,70 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4_kerne
 #pragma unroll
     for (int i = 0; i < 2 * NH; ++i) res[i] = 0.f;
 
+    if constexpr (R == 2 && PK) {
+      // ---- rank 2, G <= 4: one MMA #1 chain covers the whole group.  Rows = (page x >> 1, rank x & 1) for pages
+      // 0-3 and, in rows 8-15, pages 4-7; lane (x, t) loads the quarter-t words of that (page, rank).
+      const int pr = x >> 1, lr = x & 1;
+      const uint4 wa4 = *reinterpret_cast<const uint4 *>(sb + pr * kBlob + (lr * 4 + t) * 16);
+      const uint4 wb4 = *reinterpret_cast<const uint4 *>(sb + (4 + pr) * kBlob + (lr * 4 + t) * 16);
+      const uint32_t wa[4] = {wa4.x, wa4.y, wa4.z, wa4.w}, wb[4] = {wb4.x, wb4.y, wb4.z, wb4.w};
+      float c1[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const uint32_t ua = wa[j], ub = wb[j], ua8 = ua >> 8, ub8 = ub >> 8;
+        if (j == 0) mma_f16_z(c1, ua & kM0, ub & kM0, ua & kM1, ub & kM1, qb0[0][0], qb2[0][0]);
+        else mma_f16(c1, ua & kM0, ub & kM0, ua & kM1, ub & kM1, qb0[0][2 * j], qb2[0][2 * j]);
+        mma_f16(c1, ua8 & kM0, ub8 & kM0, ua8 & kM1, ub8 & kM1, qb0[0][2 * j + 1], qb2[0][2 * j + 1]);
+      }
+      // projections of (page, rank) for heads 2t, 2t+1: prj[half][e]
+      const float svA = __half2float(*reinterpret_cast<const __half *>(sb + pr * kBlob + i4_off_sv(R) + 2 * lr));
+      const float svB = __half2float(*reinterpret_cast<const __half *>(sb + (4 + pr) * kBlob + i4_off_sv(R) + 2 * lr));
+      const float prj[2][2] = {{fmaf(c1[0], 16777216.f, -ksum[0]) * svA, fmaf(c1[1], 16777216.f, -ksum[1]) * svA},
+                               {fmaf(c1[2], 16777216.f, -ksum[0]) * svB, fmaf(c1[3], 16777216.f, -ksum[1]) * svB}};
+      // ---- MMA #2, four pages at a time: rows = (page a, head g) = a * 4 + g, k = part * 8 + a * 2 + rank with
+      // part 0 = fp16 hi, part 1 = fp16 lo of the projection (block diagonal: a row meets its own page only),
+      // columns = tokens.  Lane (x, t) feeds page t of the four, head x & 3, if its row x (t < 2) or x + 8
+      // (t >= 2) belongs to that page; both ranks come from the lanes that hold them after MMA #1.
+      const bool mine = (x >> 2) == (t & 1);
+      const int src0 = (2 * t) * 4 + ((x & 3) >> 1), src1 = src0 + 4;   // lanes (rank 0 | rank 1 of page t, head pair)
+      const float iv = inv_s[0] * c2;
+#pragma unroll
+      for (int k4 = 0; k4 < 2; ++k4) {   // pages 4 k4 .. 4 k4 + 3
+        const float r00 = __shfl_sync(0xffffffffu, prj[k4][0], src0), r01 = __shfl_sync(0xffffffffu, prj[k4][1], src0);
+        const float r10 = __shfl_sync(0xffffffffu, prj[k4][0], src1), r11 = __shfl_sync(0xffffffffu, prj[k4][1], src1);
+        const float p0 = (x & 1) ? r01 : r00, p1 = (x & 1) ? r11 : r10;   // ranks 0, 1 of (page t, head x & 3)
+        uint32_t hi = pack_f16(p0, p1);
+        const float2 hf = h2f2(hi);
+        uint32_t lo = pack_f16(p0 - hf.x, p1 - hf.y);
+        if (!mine) { hi = 0u; lo = 0u; }
+        const uint32_t a0 = t < 2 ? hi : 0u, a1 = t < 2 ? 0u : hi, a2 = t < 2 ? lo : 0u, a3 = t < 2 ? 0u : lo;
+        // coefficients of page t, token x (and x + 8), ranks 0 and 1; the lo part meets the same values
+        const uint32_t cw = *reinterpret_cast<const uint32_t *>(sb + (4 * k4 + t) * kBlob + i4_off_coef(R) + x * 4);
+        const uint32_t bt0 = f16x2_sub(__byte_perm(cw, 0x64646464u, 0x4140), kSub128);
+        const uint32_t bt8 = f16x2_sub(__byte_perm(cw, 0x64646464u, 0x4342), kSub128);
+        float ca[4], cb[4];   // ca: tokens 2t, 2t+1; cb: tokens 2t+8, 2t+9; [0..1] row x, [2..3] row x + 8
+        mma_f16_z(ca, a0, a1, a2, a3, bt0, bt0);
+        mma_f16_z(cb, a0, a1, a2, a3, bt8, bt8);
+#pragma unroll
+        for (int hrow = 0; hrow < 2; ++hrow) {   // row x -> page 4 k4 + (x >> 2), row x + 8 -> two pages further
+          const int pg = 4 * k4 + 2 * hrow + (x >> 2);
+          const uint2 scw = *reinterpret_cast<const uint2 *>(sb + pg * kBlob + i4_off_sc(R) + 8 * t);
+          const float2 s01 = h2f2(scw.x), s89 = h2f2(scw.y);
+          const float y0 = ca[2 * hrow] * s01.x, y1 = ca[2 * hrow + 1] * s01.y;
+          const float y2 = cb[2 * hrow] * s89.x, y3 = cb[2 * hrow + 1] * s89.y;
+          float my = fmaxf(fmaxf(y0, y1), fmaxf(y2, y3));
+          my = fmaxf(my, __shfl_xor_sync(0xffffffffu, my, 1));
+          my = fmaxf(my, __shfl_xor_sync(0xffffffffu, my, 2));
+          const float m = my * iv;
+          float e = fast_ex2(fmaf(y0, iv, -m)) + fast_ex2(fmaf(y1, iv, -m)) + fast_ex2(fmaf(y2, iv, -m)) +
+                    fast_ex2(fmaf(y3, iv, -m));
+          e += __shfl_xor_sync(0xffffffffu, e, 1);
+          e += __shfl_xor_sync(0xffffffffu, e, 2);
+          // lane (x, t) keeps the result of page 2t + (x >> 2), head x & 3
+          if (t == 2 * k4 + hrow) res[0] = m + fast_lg2(e) + acen[0];
+        }
+      }
+    } else {
 #pragma unroll
     for (int pp = 0; pp < LOCKS_GROUP / 2; ++pp) {
       const uint8_t *pbA = sb + (2 * pp) * kBlob, *pbB = pbA + kBlob;
@@ -595,6 +659,7 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4_kerne
       }
     }
       }
+    }
     __syncwarp();  // every lane is done reading this stage
     if (cp.prob < nprob) {
       issue(stage, cp, next_block);
