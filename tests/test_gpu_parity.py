@@ -251,6 +251,33 @@ def test_decode_step_matches_stepwise_oracle():
                 assert np.abs(gV - oV).max() <= 1
 
 
+def test_decode_step_long_context_few_problems():
+    """Decode steps on one long request (several selector chunks per KV head, cluster-merged attention,
+    G = 16): the token is appended by the selector's first chunk, and a page fills on the way."""
+    from common import check_page_sets, oracle_cache
+    T0 = 16 * 4000 + 14
+    w = locks_synth.Workload("long-step", [T0 + 16], Hq=32, Hkv=2, budget=1024, seed=61)
+    gc = _gc(w)
+    gc.case.seq_lens.fill_(T0)
+    summ = gc.ctx.new_summaries(gc.case.num_blocks)
+    gc.ctx.locks_build_summaries(gc.kv, w.n, summ)
+    out = torch.empty(w.n, w.Hq, w.d, dtype=torch.bfloat16, device="cuda:0")
+    ids = torch.empty(w.n, w.Hkv, gc.k, dtype=torch.int32, device="cuda:0")
+    cnt = torch.empty(w.n, w.Hkv, dtype=torch.int32, device="cuda:0")
+    for step in range(3):
+        kn, vn, qn = locks_synth.new_token(w, step, device="cuda:0")
+        gc.ctx.locks_decode_step(qn, kn, vn, gc.kv, summ, w.n, out, ids, cnt)
+        torch.cuda.synchronize()
+        assert gc.status() == 0
+        assert gc.case.seq_lens.cpu().tolist() == [T0 + step + 1]
+        cache = oracle_cache(gc.case)
+        shat = oracle.page_logmass(cache, t2np(qn), w.rank, gc.fmt, summ.cpu().numpy(), gc.sm)
+        oids, ocnt, ols = oracle.select(cache, shat, gc.k)
+        check_page_sets(ids.cpu().numpy(), cnt.cpu().numpy(), oids, ocnt, ols, cache.seq_lens, w.B, gc.k)
+        oout, _ = oracle.attend(cache, t2np(qn), gc.sm, ids.cpu().numpy(), cnt.cpu().numpy())
+        assert np.abs(out.float().cpu().numpy() - oout).max() <= 2e-2, step
+
+
 def test_decode_step_graph_replay_equals_eager():
     """The step is captured once in a CUDA graph and replayed as the sequences grow."""
     w = small_bf16([16 * 100 + 9, 16 * 70], Hq=8, Hkv=2, budget=256, seed=44)
