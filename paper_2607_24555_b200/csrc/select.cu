@@ -102,8 +102,8 @@ __device__ __forceinline__ uint32_t order_key(float f) {
 
 // K-th largest of the keys sh.key[i*512 + t], i < nslab (invalid elements hold key 0; 1 <= K <= number of
 // valid keys).  Returns (key, how many of the keys equal to it belong to the top K).
-// 8-bit radix passes from the top; leading bytes on which all valid keys agree (page masses share sign
-// and exponent) are skipped after one AND / OR reduction.  A pass costs one barrier: all warps count into
+// Radix passes of up to 8 bits from the top; leading bits on which all valid keys agree (page masses share
+// sign and most of the exponent) are skipped after one AND / OR reduction.  A pass costs one barrier: all warps count into
 // one 256-bin histogram, then every warp scans it on its own (lane l owns bins 8 (31 - l) .. + 7, so
 // lane order is descending digit order) while the histogram of the next pass -- three rotate -- is
 // already being filled by warps that are ahead.
@@ -125,21 +125,27 @@ __device__ __noinline__ uint2 radix_select(int nslab, int K) {
   all_or = sh.red[kNW + (lane & (kNW - 1))];
   all_and = __reduce_and_sync(0xffffffffu, all_and);
   all_or = __reduce_or_sync(0xffffffffu, all_or);
-  const int first = __clz(all_and ^ all_or) >> 3;   // leading bytes shared by every valid key (4: all keys equal)
-  uint32_t mask = first ? 0xFFFFFFFFu << (32 - 8 * first) : 0u;
+  // Leading bits shared by every valid key (sign, most of the exponent) are skipped, bit by bit: the first
+  // pass then works on the eight most significant bits in which the keys really differ, which spreads them
+  // over the bins (hundreds of atomics on two or three counters would serialise), and the later passes see
+  // only the few keys of the threshold bin.
+  const int common = __clz(all_and ^ all_or);   // 32: all valid keys are equal
+  uint32_t mask = common ? 0xFFFFFFFFu << (32 - common) : 0u;
   uint32_t prefix = all_or & mask;
   int remaining = K;
   int cur = 0;
 #pragma unroll 1
-  for (int pass = first; pass < 4; ++pass) {
-    const int shift = 24 - 8 * pass;
+  for (int left = 32 - common; left > 0;) {   // bits not yet decided
+    const int width = min(8, left), shift = left - width;
+    const uint32_t dmask = (1u << width) - 1u;
+    left = shift;
     const int nxt = cur == 2 ? 0 : cur + 1;
     int *hc = sh.hist + cur * 256;
     if (tid < 256) sh.hist[nxt * 256 + tid] = 0;   // last read two passes ago
 #pragma unroll 4
     for (int i = 0; i < nslab; ++i) {
       const uint32_t k = sh.key[i * LOCKS_SEL_THREADS + tid];
-      if (k && (k & mask) == prefix) atomicAdd(&hc[(k >> shift) & 255], 1);
+      if (k && (k & mask) == prefix) atomicAdd(&hc[(k >> shift) & dmask], 1);
     }
     __syncthreads();
     const int base = 8 * (31 - lane);
@@ -164,7 +170,7 @@ __device__ __noinline__ uint2 radix_select(int nslab, int K) {
     digit = __shfl_sync(0xffffffffu, digit, src);
     remaining = __shfl_sync(0xffffffffu, rem, src);
     prefix |= (uint32_t)digit << shift;
-    mask |= 255u << shift;
+    mask |= dmask << shift;
     cur = nxt;
   }
   return make_uint2(prefix, (uint32_t)remaining);
