@@ -337,6 +337,43 @@ def test_decode_step_host_entry_point():
     assert torch.equal(out.cpu(), out_host) and torch.equal(ids.cpu(), ids_host) and torch.equal(cnt.cpu(), cnt_host)
 
 
+def test_decode_step_host_repeated_calls_match_device_steps():
+    """Repeated host-buffer steps with fixed buffers (from the second repetition on the library replays a
+    cached graph): each call appends its token and returns what the device entry point returns on a twin."""
+    w = small_bf16([16 * 60 + 13, 700], Hq=8, Hkv=2, budget=128, seed=57)
+    reserve = 2
+    w = w.with_(seq_lens=[t + 16 * reserve for t in w.seq_lens])
+    gc_h, gc_d = _gc(w), _gc(w)
+    start = torch.tensor([t - 16 * reserve for t in w.seq_lens], dtype=torch.int32, device="cuda:0")
+    outs = []
+    for gc in (gc_h, gc_d):
+        gc.case.seq_lens.copy_(start)
+    summ_h = gc_h.ctx.new_summaries(gc_h.case.num_blocks)
+    summ_d = gc_d.ctx.new_summaries(gc_d.case.num_blocks)
+    gc_h.ctx.locks_build_summaries(gc_h.kv, w.n, summ_h)
+    gc_d.ctx.locks_build_summaries(gc_d.kv, w.n, summ_d)
+    qh = torch.empty(w.n, w.Hq, w.d, dtype=torch.bfloat16).pin_memory()
+    kh = torch.empty(w.n, w.Hkv, w.d, dtype=torch.bfloat16).pin_memory()
+    vh = torch.empty(w.n, w.Hkv, w.d, dtype=torch.bfloat16).pin_memory()
+    out_host = torch.empty(w.n, w.Hq, w.d, dtype=torch.bfloat16).pin_memory()
+    ids_host = torch.empty(w.n, w.Hkv, gc_h.k, dtype=torch.int32).pin_memory()
+    cnt_host = torch.empty(w.n, w.Hkv, dtype=torch.int32).pin_memory()
+    out = torch.empty(w.n, w.Hq, w.d, dtype=torch.bfloat16, device="cuda:0")
+    ids = torch.empty(w.n, w.Hkv, gc_d.k, dtype=torch.int32, device="cuda:0")
+    cnt = torch.empty(w.n, w.Hkv, dtype=torch.int32, device="cuda:0")
+    for step in range(20):   # crosses a page boundary of both requests
+        kn, vn, qn = locks_synth.new_token(w, step, device="cuda:0")
+        qh.copy_(qn.cpu()); kh.copy_(kn.cpu()); vh.copy_(vn.cpu())
+        gc_h.ctx.locks_decode_step_host(qh, kh, vh, gc_h.kv, summ_h, w.n, out_host, ids_host, cnt_host)
+        gc_d.ctx.locks_decode_step(qn, kn, vn, gc_d.kv, summ_d, w.n, out, ids, cnt)
+        torch.cuda.synchronize()
+        assert torch.equal(gc_h.case.seq_lens, gc_d.case.seq_lens)
+        assert torch.equal(ids.cpu(), ids_host) and torch.equal(cnt.cpu(), cnt_host), step
+        assert torch.equal(out.cpu(), out_host), step
+    assert torch.equal(summ_h, summ_d)
+    assert gc_h.status() == 0 and gc_d.status() == 0
+
+
 def test_bad_block_id_sets_status_without_faulting():
     """Host-injected fault: a block id outside the cache is skipped and reported, nothing traps."""
     gc = _gc(small_bf16([16 * 60], Hq=8, Hkv=2, budget=128, seed=66))
