@@ -74,7 +74,7 @@ def config_dict(w, layers, identity):
     scan_b, att_b, _ = algorithmic_bytes(w)
     return {"workload": w.name, "batch_per_gpu": w.n, "context": w.seq_lens[0], "q_heads": w.Hq, "kv_heads": w.Hkv,
             "head_dim": w.d, "page": w.B, "rank": w.rank, "budget_tokens": w.budget,
-            "summary": "r8i4" if w.fmt == "i4" else "f32", "launch": "one CUDA graph per step",
+            "summary": f"r{w.rank}i4" if w.fmt == "i4" else f"r{w.rank}f32", "launch": "one CUDA graph per step",
             "block_mapping": "identity" if identity else "seeded random permutation",
             "l2": f"inputs larger than L2: replays cycle over {layers} independent layers "
                   f"({(scan_b + att_b) / 1e6:.0f} MB touched per step, L2 126 MB)"}
