@@ -184,8 +184,6 @@ def run_reference(args):
     w = workload(args.workload)
     cores = oracle.max_threads()
     steps = max(1, min(args.steps, 5))
-    for _ in range(min(args.warmup, 1)):
-        pass
     us, sample, _ = oracle_sample(w, steps, cores)
     scan, attend, dense = algorithmic_bytes(w)
     line = {"impl": "reference", "metric": METRIC, "value": us, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,

@@ -11,7 +11,7 @@
 #define LOCKS_B 16           // tokens per page
 #define LOCKS_GROUP 8        // pages scored together by one warp in the scan (one ring stage, one partial)
 #define LOCKS_SEL_THREADS 512
-#define LOCKS_SEL_MAX_EPT 16 // candidate pages held per thread in select stage 1 (4, 8 or 16)
+#define LOCKS_SEL_MAX_EPT 16 // pages per thread a selector CTA ranks at most (512 threads: 8192 pages or list entries)
 #define LOCKS_ATT_WARPS 3        // warps per attend CTA
 #define LOCKS_ATT_STAGES 2       // pages (4 KB of K + 4 KB of V each) in each warp's ring
 #define LOCKS_ATT_CTAS_PER_SM 4  // 4 x 48 KB of shared memory
@@ -41,8 +41,8 @@ struct locks_ctx {
   int G, k, S, Pmax, max_groups;
   int num_sms;
   int part_slots;          // partial slots per (request, head) the last scan launch may have filled
-  int sel_ept;             // pages per thread in select stage 1
-  int sel_chunks;          // select stage-1 CTAs per (request, KV head)
+  int sel_ept;             // pages per thread of a selector CTA (chunk = sel_ept * 512 pages)
+  int sel_chunks;          // selector CTAs (chunks) per (request, KV head)
   int sel_kc;              // candidates kept per chunk (k-2)
   // workspace partition (device)
   char *ws;
@@ -51,7 +51,7 @@ struct locks_ctx {
   float *shat;             // [max_batch][Hq][Pmax]
   float2 *part;            // [max_batch][Hq][max_groups] partial (max, sum exp) over candidate pages
   int32_t *sel_done;       // [max_batch][Hkv] chunk-arrival counters
-  float *cand_val;         // [max_batch][Hkv][sel_chunks][sel_kc]
+  float *cand_val;         // [max_batch][Hkv][sel_chunks][sel_kc] chunk lists: 32-bit keys (0 = no entry)
   int32_t *cand_idx;
   float *att_o;            // [rows][d], rows = batch * Hq * splits <= att_rows
   float *att_lse;          // [rows]  (log2 units)
