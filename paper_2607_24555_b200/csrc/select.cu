@@ -249,7 +249,7 @@ __device__ __noinline__ void compact_emit(int nslab, uint32_t prefix, int remain
 // log Z_g of every head of the group from the scan's partials (max_i, sum_i), part0 = head 0's row,
 // -> sh.lz2[g] (log2 domain):
 // log2 Z = M + log2 sum_i sum_i 2^(max_i - M), M = max_i max_i.  The block's warps are dealt to (head, slice)
-// pairs; a lane keeps four loads in flight.  Ends with the block synchronised.
+// pairs; a lane keeps eight loads in flight.  Ends with the block synchronised.
 __device__ __noinline__ void group_logz(const float2 *part0, int G, int max_groups, int nparts) {
   SelShared &sh = shared_state();
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -262,15 +262,17 @@ __device__ __noinline__ void group_logz(const float2 *part0, int G, int max_grou
     if (g < G && slice < nslice) {
       const float2 *pp = part0 + (int64_t)g * max_groups;
 #pragma unroll 1
-      for (int i0 = slice * 32 + lane; i0 < nparts; i0 += 128 * nslice) {
-        float2 v[4];
+      for (int i0 = slice * 32 + lane; i0 < nparts; i0 += 256 * nslice) {
+        float2 v[8];   // eight loads in flight: up to 256 partials of a head in one round trip
 #pragma unroll
-        for (int u = 0; u < 4; ++u) v[u] = (i0 + 32 * nslice * u < nparts) ? pp[i0 + 32 * nslice * u] : make_float2(-INFINITY, 0.f);
-        const float nm = fmaxf(fmaxf(fmaxf(v[0].x, v[1].x), fmaxf(v[2].x, v[3].x)), m);
+        for (int u = 0; u < 8; ++u) v[u] = (i0 + 32 * nslice * u < nparts) ? pp[i0 + 32 * nslice * u] : make_float2(-INFINITY, 0.f);
+        float nm = m;
+#pragma unroll
+        for (int u = 0; u < 8; ++u) nm = fmaxf(nm, v[u].x);
         if (nm > -INFINITY) {
           s *= ex2f((m - nm) * kLog2e);
 #pragma unroll
-          for (int u = 0; u < 4; ++u) s = fmaf(v[u].y, ex2f((v[u].x - nm) * kLog2e), s);
+          for (int u = 0; u < 8; ++u) s = fmaf(v[u].y, ex2f((v[u].x - nm) * kLog2e), s);
           m = nm;
         }
       }
