@@ -145,6 +145,33 @@ def test_i4_rank2_group_sizes(Hq, Hkv):
     check_select_and_attend(gc, gc.oracle_summaries(), out_tol=2e-2)
 
 
+@pytest.mark.parametrize("trial", range(24))
+def test_randomized_shapes(trial):
+    """Seeded random shapes: group size, rank, budget, request count, lengths (with ragged tails and requests
+    shorter than the budget), block layout, carriers.  Twice per case: the second call must reproduce the
+    first (no state left behind in the workspace)."""
+    from gpu_util import check_select_and_attend
+    rng = np.random.default_rng(1000 + trial)
+    Hkv = int(rng.choice([1, 2, 4]))
+    G = int(rng.choice([1, 2, 3, 4, 5, 7, 8, 12, 16]))
+    rank = int(rng.choice([2, 4, 8]))
+    budget = int(rng.choice([32, 64, 256, 512, 1024]))
+    n = int(rng.integers(1, 4))
+    lens = [int(rng.integers(1, 6000)) for _ in range(n)]
+    if trial % 3 == 0:
+        lens[0] = int(rng.integers(9000, 30000))      # one long request
+    w = small_bf16(lens, Hq=G * Hkv, Hkv=Hkv, rank=rank, budget=budget, seed=2000 + trial,
+                   layout="NHD" if trial % 4 == 1 else "HND", carriers=int(rng.choice([0, 0, 4])),
+                   q_scale=float(rng.choice([1.0, 0.25])))
+    gc = _gc(w)
+    summ = gc.oracle_summaries()
+    check_select_and_attend(gc, summ, out_tol=2e-2)
+    ids1, cnt1, lm1, ls1 = gc.gpu_select(torch.from_numpy(summ).cuda())
+    ids2, cnt2, lm2, ls2 = gc.gpu_select(torch.from_numpy(summ).cuda())
+    assert np.array_equal(ids1, ids2) and np.array_equal(cnt1, cnt2)
+    assert gc.status() == 0
+
+
 def test_two_level_select_long_context():
     """Several chunks per KV head: per-chunk lists, then the last chunk to arrive ranks the survivors."""
     from gpu_util import check_select_and_attend
