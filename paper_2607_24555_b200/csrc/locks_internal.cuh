@@ -17,6 +17,9 @@
 #define LOCKS_ATT_CTAS_PER_SM 4  // 4 x 48 KB of shared memory
 #define LOCKS_ATT_MAX_SPLITS 128
 #define LOCKS_ATT_SLOT_BOUND 1024 // upper bound on resident attend CTAs of any supported GPU (148 SMs x 4 on B200)
+#ifndef LOCKS_SCAN_GATHER
+#define LOCKS_SCAN_GATHER 1    // rank-8 scan: stage summaries four at a time with tensor-map gathers
+#endif
 #ifndef LOCKS_SCAN_BULK
 #define LOCKS_SCAN_BULK 1      // staging of summary blobs in the scan: 1 = cp.async.bulk (TMA) + mbarrier, 0 = 16-byte cp.async
 #endif

@@ -14,6 +14,9 @@
 //                         per page, after an 8x8 movmatrix transpose of the fp16 hi/lo projection:
 //                           MMA#2  L[heads, tokens] = (P_hi | P_lo)[heads x 16] . codesC^T          (2 x m16n8k16 fp16)
 //                         and per 8 pages the centroid dots a[heads, pages] (8 x m16n8k16 fp16).
+#include <cstring>
+#include <cuda.h>            // CUtensorMap (types only; the encoder is fetched from the driver at run time)
+#include <cudaTypedefs.h>
 #include "locks_internal.cuh"
 
 namespace {
@@ -34,6 +37,7 @@ struct ScanParams {
   // decode step with an appended token: lengths count the token that the selector's kernel is about to
   // write (seq_inc = 1); the first CTA publishes them, and the append position, for the step's later kernels
   int cta_reduce;     // every warp of a CTA works on one problem only: one partial per (head, CTA)
+  int use_gather;     // rank 8: stage four summaries per tensor-map gather instead of one bulk copy each
   int seq_inc;
   int32_t *seq_eff;   // [2][max_batch]: effective length, append position (-1: none) -- or nullptr
 };
@@ -209,6 +213,16 @@ struct Cursor {
   int prob, grp, nsc, b, h;   // (request, KV head) of prob are refreshed only when prob changes
 };
 
+// Four rows of a 2D tensor map (box = one row) to consecutive rows in shared memory, completion on an mbarrier.
+__device__ __forceinline__ void tma_gather4(void *dst, const CUtensorMap *tmap, int r0, int r1, int r2, int r3,
+                                            uint64_t *bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, "
+      "%5, %6}], [%7];\n" ::"r"(smem_u32(dst)),
+      "l"(tmap), "r"(0), "r"(r0), "r"(r1), "r"(r2), "r"(r3), "r"(smem_u32(bar))
+      : "memory");
+}
+
 __device__ __forceinline__ uint32_t movm_trans(uint32_t v) {
   uint32_t d;
   asm("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(v));
@@ -233,7 +247,7 @@ __device__ __forceinline__ uint32_t movm_trans(uint32_t v) {
 // the log-sum-exp handle two pages at once (rows 0-3 = page A's heads, rows 4-7 = page B's heads, the two
 // pages separated along K) instead of leaving half of the lanes idle.
 template <int R, int NH, bool PK, bool CR>
-__global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4_kernel(ScanParams p) {
+__global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4_kernel(ScanParams p, const __grid_constant__ CUtensorMap tmap) {
   constexpr int kBlob = i4_stride(R);   // stored bytes of one summary; a stage keeps room for rank-8 blobs
   extern __shared__ __align__(128) uint8_t smem[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -285,7 +299,23 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4_kerne
       set_status(p.status, LOCKS_ERR_BAD_BLOCK);
       block = 0;
     }
-    if (kScanBulk) {
+    if (R == 8 && p.use_gather) {
+      // Summaries are rows of a 2D tensor [block * Hkv + head][832 B]: one gather fetches four of them, so a
+      // group costs two copy instructions instead of eight (about 3 of 115 instructions per summary; the
+      // staging throughput itself does not change).  Slots past the last page repeat the group's first row.
+      int row = block * p.Hkv + h;
+      row = __shfl_sync(0xffffffffu, row, lane < nvalid ? lane : 0);
+      const int r1 = __shfl_sync(0xffffffffu, row, 1), r2 = __shfl_sync(0xffffffffu, row, 2);
+      const int r3 = __shfl_sync(0xffffffffu, row, 3), r4 = __shfl_sync(0xffffffffu, row, 4);
+      const int r5 = __shfl_sync(0xffffffffu, row, 5), r6 = __shfl_sync(0xffffffffu, row, 6);
+      const int r7 = __shfl_sync(0xffffffffu, row, 7);
+      if (lane == 0) {
+        uint8_t *dst = ring + stage * kStageBytes;
+        mbar_expect_tx(&full[stage], (uint32_t)(nvalid > 4 ? 8 : 4) * kBlob);
+        tma_gather4(dst, &tmap, row, r1, r2, r3, &full[stage]);
+        if (nvalid > 4) tma_gather4(dst + 4 * kBlob, &tmap, r4, r5, r6, r7, &full[stage]);
+      }
+    } else if (kScanBulk) {
       if (lane == 0) mbar_expect_tx(&full[stage], (uint32_t)nvalid * kBlob);
       __syncwarp();
       if (lane < nvalid)
@@ -761,6 +791,33 @@ int locks_launch_scan(locks_ctx *c, const void *q, const void *summaries, const 
     }
     const dim3 g(grid), blk(kScanWarps * 32);
     const int gsel = c->G <= 4 ? 0 : (c->G <= 8 ? 1 : 2);
+    // tensor map over the summaries for the gather path (rank 8): rows = (block, KV head), 208 32-bit words each
+    alignas(64) CUtensorMap tmap;
+    memset(&tmap, 0, sizeof(tmap));
+    p.use_gather = 0;
+    if (c->cfg.rank == 8 && LOCKS_SCAN_GATHER) {
+      static PFN_cuTensorMapEncodeTiled encode = nullptr;
+      static bool looked = false;
+      if (!looked) {
+        looked = true;
+        void *fn = nullptr;
+        cudaDriverEntryPointQueryResult qr;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qr) == cudaSuccess &&
+            qr == cudaDriverEntryPointSuccess)
+          encode = reinterpret_cast<PFN_cuTensorMapEncodeTiled>(fn);
+        (void)cudaGetLastError();
+      }
+      if (encode) {
+        const cuuint64_t gdim[2] = {(cuuint64_t)(i4_stride(8) / 4), (cuuint64_t)kv->num_blocks * p.Hkv};
+        const cuuint64_t gstride[1] = {(cuuint64_t)i4_stride(8)};
+        const cuuint32_t box[2] = {(cuuint32_t)(i4_stride(8) / 4), 1u};
+        const cuuint32_t estride[2] = {1u, 1u};
+        if (encode(&tmap, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<void *>(summaries), gdim, gstride, box, estride,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS)
+          p.use_gather = 1;
+      }
+    }
 #define LOCKS_SCAN_LAUNCH(R_, CR_)                                                                                     \
   do {                                                                                                                 \
     static bool attr_done = false;                                                                                     \
@@ -770,9 +827,9 @@ int locks_launch_scan(locks_ctx *c, const void *q, const void *summaries, const 
       cudaFuncSetAttribute(scan_i4_kernel<R_, 2, false, CR_>, cudaFuncAttributeMaxDynamicSharedMemorySize, kScanSmem); \
       attr_done = true;                                                                                                \
     }                                                                                                                  \
-    if (gsel == 0) locks_launch_pdl(scan_i4_kernel<R_, 1, true, CR_>, g, blk, kScanSmem, st, p);                       \
-    else if (gsel == 1) locks_launch_pdl(scan_i4_kernel<R_, 1, false, CR_>, g, blk, kScanSmem, st, p);                 \
-    else locks_launch_pdl(scan_i4_kernel<R_, 2, false, CR_>, g, blk, kScanSmem, st, p);                                \
+    if (gsel == 0) locks_launch_pdl(scan_i4_kernel<R_, 1, true, CR_>, g, blk, kScanSmem, st, p, tmap);                       \
+    else if (gsel == 1) locks_launch_pdl(scan_i4_kernel<R_, 1, false, CR_>, g, blk, kScanSmem, st, p, tmap);                 \
+    else locks_launch_pdl(scan_i4_kernel<R_, 2, false, CR_>, g, blk, kScanSmem, st, p, tmap);                                \
   } while (0)
     if (c->cfg.rank == 8 && p.cta_reduce) LOCKS_SCAN_LAUNCH(8, true);
     else if (c->cfg.rank == 8) LOCKS_SCAN_LAUNCH(8, false);
