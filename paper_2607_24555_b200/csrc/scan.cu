@@ -520,50 +520,94 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4_kerne
 #pragma unroll
     for (int i = 0; i < 2 * NH; ++i) res[i] = 0.f;
 
-    if constexpr (R == 2 && PK) {
-      // ---- rank 2, G <= 4: one MMA #1 chain covers the whole group.  Rows = (page x >> 1, rank x & 1) for pages
-      // 0-3 and, in rows 8-15, pages 4-7; lane (x, t) loads the quarter-t words of that (page, rank).
-      const int pr = x >> 1, lr = x & 1;
-      const uint4 wa4 = *reinterpret_cast<const uint4 *>(sb + pr * kBlob + (lr * 4 + t) * 16);
-      const uint4 wb4 = *reinterpret_cast<const uint4 *>(sb + (4 + pr) * kBlob + (lr * 4 + t) * 16);
-      const uint32_t wa[4] = {wa4.x, wa4.y, wa4.z, wa4.w}, wb[4] = {wb4.x, wb4.y, wb4.z, wb4.w};
-      float c1[4];
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const uint32_t ua = wa[j], ub = wb[j], ua8 = ua >> 8, ub8 = ub >> 8;
-        if (j == 0) mma_f16_z(c1, ua & kM0, ub & kM0, ua & kM1, ub & kM1, qb0[0][0], qb2[0][0]);
-        else mma_f16(c1, ua & kM0, ub & kM0, ua & kM1, ub & kM1, qb0[0][2 * j], qb2[0][2 * j]);
-        mma_f16(c1, ua8 & kM0, ub8 & kM0, ua8 & kM1, ub8 & kM1, qb0[0][2 * j + 1], qb2[0][2 * j + 1]);
-      }
-      // projections of (page, rank) for heads 2t, 2t+1: prj[half][e]
-      const float svA = __half2float(*reinterpret_cast<const __half *>(sb + pr * kBlob + i4_off_sv(R) + 2 * lr));
-      const float svB = __half2float(*reinterpret_cast<const __half *>(sb + (4 + pr) * kBlob + i4_off_sv(R) + 2 * lr));
-      const float prj[2][2] = {{fmaf(c1[0], 16777216.f, -ksum[0]) * svA, fmaf(c1[1], 16777216.f, -ksum[1]) * svA},
-                               {fmaf(c1[2], 16777216.f, -ksum[0]) * svB, fmaf(c1[3], 16777216.f, -ksum[1]) * svB}};
-      // ---- MMA #2, four pages at a time: rows = (page a, head g) = a * 4 + g, k = part * 8 + a * 2 + rank with
-      // part 0 = fp16 hi, part 1 = fp16 lo of the projection (block diagonal: a row meets its own page only),
-      // columns = tokens.  Lane (x, t) feeds page t of the four, head x & 3, if its row x (t < 2) or x + 8
-      // (t >= 2) belongs to that page; both ranks come from the lanes that hold them after MMA #1.
-      const bool mine = (x >> 2) == (t & 1);
-      const int src0 = (2 * t) * 4 + ((x & 3) >> 1), src1 = src0 + 4;   // lanes (rank 0 | rank 1 of page t, head pair)
+    float prj2[2][2] = {{0.f, 0.f}, {0.f, 0.f}};   // small-rank tile: projections of the current MMA #1 chain
+    (void)prj2;
+    if constexpr (R <= 4 && PK) {
+      // ---- ranks 2 and 4, G <= 4.  MMA #1: the 16 rows are (page, rank) pairs, 8 / R pages in rows 0-7 and the
+      // next 8 / R in rows 8-15, so one chain of 8 MMAs projects 16 / R pages (rank 2: the whole group; rank 4:
+      // half of it); lane (x, t) loads the quarter-t words of its (page, rank).  MMA #2 works on four pages at a
+      // time: rows = (page a, head g) = 4 a + g, columns = tokens, k = (page, rank) so that a row meets its own
+      // page only (block diagonal).  Rank 2: k = part * 8 + 2 a + rank with part 0 / 1 = fp16 hi / lo of the
+      // projection, one MMA per token half.  Rank 4: k = 4 a + rank, hi and lo in two MMAs.
+      constexpr int PH = 8 / R;                 // pages per row half of MMA #1
+      const int pr = x / R, lr = x % R;         // this lane's row: page within the half, rank
       const float iv = inv_s[0] * c2;
 #pragma unroll
-      for (int k4 = 0; k4 < 2; ++k4) {   // pages 4 k4 .. 4 k4 + 3
-        const float r00 = __shfl_sync(0xffffffffu, prj[k4][0], src0), r01 = __shfl_sync(0xffffffffu, prj[k4][1], src0);
-        const float r10 = __shfl_sync(0xffffffffu, prj[k4][0], src1), r11 = __shfl_sync(0xffffffffu, prj[k4][1], src1);
-        const float p0 = (x & 1) ? r01 : r00, p1 = (x & 1) ? r11 : r10;   // ranks 0, 1 of (page t, head x & 3)
-        uint32_t hi = pack_f16(p0, p1);
-        const float2 hf = h2f2(hi);
-        uint32_t lo = pack_f16(p0 - hf.x, p1 - hf.y);
-        if (!mine) { hi = 0u; lo = 0u; }
-        const uint32_t a0 = t < 2 ? hi : 0u, a1 = t < 2 ? 0u : hi, a2 = t < 2 ? lo : 0u, a3 = t < 2 ? 0u : lo;
-        // coefficients of page t, token x (and x + 8), ranks 0 and 1; the lo part meets the same values
-        const uint32_t cw = *reinterpret_cast<const uint32_t *>(sb + (4 * k4 + t) * kBlob + i4_off_coef(R) + x * 4);
-        const uint32_t bt0 = f16x2_sub(__byte_perm(cw, 0x64646464u, 0x4140), kSub128);
-        const uint32_t bt8 = f16x2_sub(__byte_perm(cw, 0x64646464u, 0x4342), kSub128);
+      for (int k4 = 0; k4 < 2; ++k4) {          // pages 4 k4 .. 4 k4 + 3
+        float prj[2][2];                        // rank 2: [k4 half][head e]; rank 4: [half of this chain][head e]
+        if (R == 4 || k4 == 0) {
+          const int pa0 = (R == 4 ? 4 * k4 : 0) + pr, pb0 = pa0 + PH;
+          const uint4 wa4 = *reinterpret_cast<const uint4 *>(sb + pa0 * kBlob + (lr * 4 + t) * 16);
+          const uint4 wb4 = *reinterpret_cast<const uint4 *>(sb + pb0 * kBlob + (lr * 4 + t) * 16);
+          const uint32_t wa[4] = {wa4.x, wa4.y, wa4.z, wa4.w}, wb[4] = {wb4.x, wb4.y, wb4.z, wb4.w};
+          float c1[4];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const uint32_t ua = wa[j], ub = wb[j], ua8 = ua >> 8, ub8 = ub >> 8;
+            if (j == 0) mma_f16_z(c1, ua & kM0, ub & kM0, ua & kM1, ub & kM1, qb0[0][0], qb2[0][0]);
+            else mma_f16(c1, ua & kM0, ub & kM0, ua & kM1, ub & kM1, qb0[0][2 * j], qb2[0][2 * j]);
+            mma_f16(c1, ua8 & kM0, ub8 & kM0, ua8 & kM1, ub8 & kM1, qb0[0][2 * j + 1], qb2[0][2 * j + 1]);
+          }
+          const float svA = __half2float(*reinterpret_cast<const __half *>(sb + pa0 * kBlob + i4_off_sv(R) + 2 * lr));
+          const float svB = __half2float(*reinterpret_cast<const __half *>(sb + pb0 * kBlob + i4_off_sv(R) + 2 * lr));
+          prj2[0][0] = fmaf(c1[0], 16777216.f, -ksum[0]) * svA;
+          prj2[0][1] = fmaf(c1[1], 16777216.f, -ksum[1]) * svA;
+          prj2[1][0] = fmaf(c1[2], 16777216.f, -ksum[0]) * svB;
+          prj2[1][1] = fmaf(c1[3], 16777216.f, -ksum[1]) * svB;
+        }
+        prj[0][0] = prj2[0][0]; prj[0][1] = prj2[0][1]; prj[1][0] = prj2[1][0]; prj[1][1] = prj2[1][1];
+        uint32_t a0h, a1h, a2h, a3h, a0l = 0u, a1l = 0u, a2l = 0u, a3l = 0u;
+        uint32_t bt0a, bt0b, bt8a, bt8b;
+        if (R == 2) {
+          // lane (x, t) feeds page t of the four, head x & 3, if its row x (t < 2) or x + 8 (t >= 2) is that page's
+          const bool mine = (x >> 2) == (t & 1);
+          const int src0 = (2 * t) * 4 + ((x & 3) >> 1), src1 = src0 + 4;   // lanes holding rank 0 | 1 of (page t, head pair)
+          const float r00 = __shfl_sync(0xffffffffu, prj[k4][0], src0), r01 = __shfl_sync(0xffffffffu, prj[k4][1], src0);
+          const float r10 = __shfl_sync(0xffffffffu, prj[k4][0], src1), r11 = __shfl_sync(0xffffffffu, prj[k4][1], src1);
+          const float p0 = (x & 1) ? r01 : r00, p1 = (x & 1) ? r11 : r10;   // ranks 0, 1 of (page t, head x & 3)
+          uint32_t hi = pack_f16(p0, p1);
+          const float2 hf = h2f2(hi);
+          uint32_t lo = pack_f16(p0 - hf.x, p1 - hf.y);
+          if (!mine) { hi = 0u; lo = 0u; }
+          a0h = t < 2 ? hi : 0u; a1h = t < 2 ? 0u : hi; a2h = t < 2 ? lo : 0u; a3h = t < 2 ? 0u : lo;
+          // coefficients of page t, token x (and x + 8), ranks 0 and 1; the lo part meets the same values
+          const uint32_t cw = *reinterpret_cast<const uint32_t *>(sb + (4 * k4 + t) * kBlob + i4_off_coef(R) + x * 4);
+          bt0a = bt0b = f16x2_sub(__byte_perm(cw, 0x64646464u, 0x4140), kSub128);
+          bt8a = bt8b = f16x2_sub(__byte_perm(cw, 0x64646464u, 0x4342), kSub128);
+        } else {
+          // k = 2t, 2t+1 is (page t >> 1, ranks 2 (t & 1), + 1) of pages 0-1, k + 8 the same of pages 2-3; rows x are
+          // pages 0-1 (page x >> 2), rows x + 8 pages 2-3: a0 and a3 carry the diagonal blocks, a1 = a2 = 0
+          const bool mine = (x >> 2) == (t >> 1);
+          const int src0 = ((x >> 2) * 4 + 2 * (t & 1)) * 4 + ((x & 3) >> 1), src1 = src0 + 4;
+          float pv[2][2];   // [half][rank of the pair]
+#pragma unroll
+          for (int hf2 = 0; hf2 < 2; ++hf2) {
+            const float r00 = __shfl_sync(0xffffffffu, prj[hf2][0], src0), r01 = __shfl_sync(0xffffffffu, prj[hf2][1], src0);
+            const float r10 = __shfl_sync(0xffffffffu, prj[hf2][0], src1), r11 = __shfl_sync(0xffffffffu, prj[hf2][1], src1);
+            pv[hf2][0] = (x & 1) ? r01 : r00;
+            pv[hf2][1] = (x & 1) ? r11 : r10;
+          }
+          uint32_t hi0 = pack_f16(pv[0][0], pv[0][1]), hi1 = pack_f16(pv[1][0], pv[1][1]);
+          const float2 f0 = h2f2(hi0), f1 = h2f2(hi1);
+          uint32_t lo0 = pack_f16(pv[0][0] - f0.x, pv[0][1] - f0.y), lo1 = pack_f16(pv[1][0] - f1.x, pv[1][1] - f1.y);
+          if (!mine) { hi0 = hi1 = lo0 = lo1 = 0u; }
+          a0h = hi0; a1h = 0u; a2h = 0u; a3h = hi1;
+          a0l = lo0; a3l = lo1;
+          const int wofs = i4_off_coef(R) + (x * 2 + (t & 1)) * 4;   // token x (and x + 8), rank pair t & 1
+          const uint32_t cw0 = *reinterpret_cast<const uint32_t *>(sb + (4 * k4 + (t >> 1)) * kBlob + wofs);
+          const uint32_t cw1 = *reinterpret_cast<const uint32_t *>(sb + (4 * k4 + 2 + (t >> 1)) * kBlob + wofs);
+          bt0a = f16x2_sub(__byte_perm(cw0, 0x64646464u, 0x4140), kSub128);
+          bt0b = f16x2_sub(__byte_perm(cw1, 0x64646464u, 0x4140), kSub128);
+          bt8a = f16x2_sub(__byte_perm(cw0, 0x64646464u, 0x4342), kSub128);
+          bt8b = f16x2_sub(__byte_perm(cw1, 0x64646464u, 0x4342), kSub128);
+        }
         float ca[4], cb[4];   // ca: tokens 2t, 2t+1; cb: tokens 2t+8, 2t+9; [0..1] row x, [2..3] row x + 8
-        mma_f16_z(ca, a0, a1, a2, a3, bt0, bt0);
-        mma_f16_z(cb, a0, a1, a2, a3, bt8, bt8);
+        mma_f16_z(ca, a0h, a1h, a2h, a3h, bt0a, bt0b);
+        mma_f16_z(cb, a0h, a1h, a2h, a3h, bt8a, bt8b);
+        if (R == 4) {
+          mma_f16(ca, a0l, a1l, a2l, a3l, bt0a, bt0b);
+          mma_f16(cb, a0l, a1l, a2l, a3l, bt8a, bt8b);
+        }
 #pragma unroll
         for (int hrow = 0; hrow < 2; ++hrow) {   // row x -> page 4 k4 + (x >> 2), row x + 8 -> two pages further
           const int pg = 4 * k4 + 2 * hrow + (x >> 2);
