@@ -102,8 +102,8 @@ __device__ __forceinline__ uint32_t order_key(float f) {
 
 // K-th largest of the keys sh.key[i*512 + t], i < nslab (invalid elements hold key 0; 1 <= K <= number of
 // valid keys).  Returns (key, how many of the keys equal to it belong to the top K).
-// Radix passes of up to 8 bits from the top; leading bits on which all valid keys agree (page masses share
-// sign and most of the exponent) are skipped after one AND / OR reduction.  A pass costs one barrier: all warps count into
+// Radix passes of up to 8 bits from the top over the keys' offsets from the smallest valid key (one MIN / MAX
+// reduction first).  A pass costs one barrier: all warps count into
 // one 256-bin histogram, then every warp scans it on its own (lane l owns bins 8 (31 - l) .. + 7, so
 // lane order is descending digit order) while the histogram of the next pass -- three rotate -- is
 // already being filled by warps that are ahead.
@@ -111,31 +111,28 @@ __device__ __noinline__ uint2 radix_select(int nslab, int K) {
   SelShared &sh = shared_state();
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   if (tid < 256) sh.hist[tid] = 0;
-  uint32_t all_and = 0xFFFFFFFFu, all_or = 0u;
+  uint32_t kmin = 0xFFFFFFFFu, kmax = 0u;
 #pragma unroll 4
   for (int i = 0; i < nslab; ++i) {
     const uint32_t k = sh.key[i * LOCKS_SEL_THREADS + tid];
-    if (k) { all_and &= k; all_or |= k; }
+    if (k) { kmin = min(kmin, k); kmax = max(kmax, k); }
   }
-  all_and = __reduce_and_sync(0xffffffffu, all_and);
-  all_or = __reduce_or_sync(0xffffffffu, all_or);
-  if (lane == 0) { sh.red[warp] = all_and; sh.red[kNW + warp] = all_or; }
+  kmin = __reduce_min_sync(0xffffffffu, kmin);
+  kmax = __reduce_max_sync(0xffffffffu, kmax);
+  if (lane == 0) { sh.red[warp] = kmin; sh.red[kNW + warp] = kmax; }
   __syncthreads();
-  all_and = sh.red[lane & (kNW - 1)];
-  all_or = sh.red[kNW + (lane & (kNW - 1))];
-  all_and = __reduce_and_sync(0xffffffffu, all_and);
-  all_or = __reduce_or_sync(0xffffffffu, all_or);
-  // Leading bits shared by every valid key (sign, most of the exponent) are skipped, bit by bit: the first
-  // pass then works on the eight most significant bits in which the keys really differ, which spreads them
-  // over the bins (hundreds of atomics on two or three counters would serialise), and the later passes see
-  // only the few keys of the threshold bin.
-  const int common = __clz(all_and ^ all_or);   // 32: all valid keys are equal
-  uint32_t mask = common ? 0xFFFFFFFFu << (32 - common) : 0u;
-  uint32_t prefix = all_or & mask;
+  kmin = __reduce_min_sync(0xffffffffu, sh.red[lane & (kNW - 1)]);
+  kmax = __reduce_max_sync(0xffffffffu, sh.red[kNW + (lane & (kNW - 1))]);
+  // The passes rank the keys' offsets from the smallest valid key: page masses lie within a few units of each
+  // other, so the offsets need far fewer than 32 bits (typically 24: three passes), and the first pass already
+  // works on bits in which the keys differ, which spreads them over the bins (hundreds of atomics on two or
+  // three counters would serialise); the later passes see only the few keys of the threshold bin.
+  const int bits = 32 - __clz(kmax - kmin);   // 0: all valid keys are equal (kmax >= kmin: K >= 1 valid keys)
+  uint32_t mask = 0u, prefix = 0u;            // decided leading bits of the offset of the K-th largest key
   int remaining = K;
   int cur = 0;
 #pragma unroll 1
-  for (int left = 32 - common; left > 0;) {   // bits not yet decided
+  for (int left = bits; left > 0;) {   // bits not yet decided
     const int width = min(8, left), shift = left - width;
     const uint32_t dmask = (1u << width) - 1u;
     left = shift;
@@ -144,8 +141,8 @@ __device__ __noinline__ uint2 radix_select(int nslab, int K) {
     if (tid < 256) sh.hist[nxt * 256 + tid] = 0;   // last read two passes ago
 #pragma unroll 4
     for (int i = 0; i < nslab; ++i) {
-      const uint32_t k = sh.key[i * LOCKS_SEL_THREADS + tid];
-      if (k && (k & mask) == prefix) atomicAdd(&hc[(k >> shift) & dmask], 1);
+      const uint32_t k = sh.key[i * LOCKS_SEL_THREADS + tid], d = k - kmin;
+      if (k && (d & mask) == prefix) atomicAdd(&hc[(d >> shift) & dmask], 1);
     }
     __syncthreads();
     const int base = 8 * (31 - lane);
@@ -173,7 +170,7 @@ __device__ __noinline__ uint2 radix_select(int nslab, int K) {
     mask |= dmask << shift;
     cur = nxt;
   }
-  return make_uint2(prefix, (uint32_t)remaining);
+  return make_uint2(kmin + prefix, (uint32_t)remaining);
 }
 
 enum { kEmitIds = 0, kEmitList = 1, kEmitFinal = 2 };
