@@ -165,6 +165,20 @@ int locks_decode_step_host(locks_ctx *ctx, const void *q_host, const void *k_new
  * *status_host: LOCKS_OK or the first LOCKS_ERR_* a kernel recorded. */
 int locks_poll_status(locks_ctx *ctx, int32_t *status_host, locks_stream stream);
 
+/* How the scan (Eq. 1 over every candidate page of every request) deals the pages of a batch to its warps.
+ * The scores do not depend on it; log Z is summed in a different order (rounding only).
+ *   LOCKS_PARTITION_STRIDED   a fixed share of the warps per (request, KV head): best when the sequences
+ *                             are about equally long;
+ *   LOCKS_PARTITION_BALANCED  equally many pages per warp, whatever the mix of lengths;
+ *   LOCKS_PARTITION_AUTO      (default) every locks_decode_step leaves, in a page-locked word, a suggestion
+ *                             for the lengths it saw; the next call that scans follows it.  A captured CUDA
+ *                             graph keeps the choice made at capture time.
+ * Host-side setting, takes effect from the next call.  LOCKS_ERR_INVALID_ARG for an unknown mode. */
+#define LOCKS_PARTITION_AUTO 0
+#define LOCKS_PARTITION_STRIDED 1
+#define LOCKS_PARTITION_BALANCED 2
+int locks_set_scan_partition(locks_ctx *ctx, int mode);
+
 /* Number of kernels the last call on this context enqueued (for launch accounting). */
 int locks_last_launch_count(const locks_ctx *ctx);
 

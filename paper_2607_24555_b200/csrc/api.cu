@@ -31,7 +31,7 @@ int validate(const locks_config *c) {
 }
 
 struct Layout {
-  size_t status, shat, part, sel_done, cand_val, cand_idx, att_o, att_lse, att_done, ids, cnt, sq, skn, svn, sout, seq_eff, total;
+  size_t status, shat, part, part_cnt, sel_done, cand_val, cand_idx, att_o, att_lse, att_done, ids, cnt, sq, skn, svn, sout, seq_eff, total;
   int G, k, S, max_groups, sel_ept, sel_chunks, sel_kc;
 };
 
@@ -68,6 +68,7 @@ Layout make_layout(const locks_config *c) {
   L.status = take(64);
   L.shat = take(nb * Hq * P * 4);
   L.part = take(nb * Hq * L.max_groups * 8);
+  L.part_cnt = take(nb * Hkv * 4);
   L.sel_done = take(nb * Hkv * 4);
   L.cand_val = take(nb * Hkv * L.sel_chunks * L.sel_kc * 4);
   L.cand_idx = take(nb * Hkv * L.sel_chunks * L.sel_kc * 4);
@@ -127,11 +128,28 @@ int locks_create(const locks_config *cfg, void *workspace, size_t ws_bytes, lock
   for (int i = 0; i < LOCKS_HOST_GRAPHS; ++i) c->hg[i] = locks_host_graph{};
   c->hg_next = 0;
   c->part_slots = L.max_groups;
+  c->part_balanced = 0;
+  c->scan_partition = LOCKS_PARTITION_AUTO;
+  c->hint_host = nullptr; c->hint_dev = nullptr;
+  {   // one page-locked word the device can write and the host can read without synchronising
+    void *hp = nullptr, *dp = nullptr;
+    if (cudaHostAlloc(&hp, 64, cudaHostAllocMapped) == cudaSuccess) {
+      if (cudaHostGetDevicePointer(&dp, hp, 0) == cudaSuccess) {
+        c->hint_host = reinterpret_cast<int32_t *>(hp);
+        c->hint_dev = reinterpret_cast<int32_t *>(dp);
+        *c->hint_host = 0;
+      } else {
+        cudaFreeHost(hp);
+      }
+    }
+    (void)cudaGetLastError();   // without the word the partition simply stays strided
+  }
   c->G = L.G; c->k = L.k; c->S = L.S; c->Pmax = cfg->max_pages_per_seq; c->max_groups = L.max_groups;
   c->sel_ept = L.sel_ept; c->sel_chunks = L.sel_chunks; c->sel_kc = L.sel_kc;
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess ||
       cudaDeviceGetAttribute(&c->num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+    if (c->hint_host) cudaFreeHost(c->hint_host);
     delete c;
     return LOCKS_ERR_CUDA;
   }
@@ -140,6 +158,7 @@ int locks_create(const locks_config *cfg, void *workspace, size_t ws_bytes, lock
   c->status = reinterpret_cast<int32_t *>(ws + L.status);
   c->shat = reinterpret_cast<float *>(ws + L.shat);
   c->part = reinterpret_cast<float2 *>(ws + L.part);
+  c->part_cnt = reinterpret_cast<int32_t *>(ws + L.part_cnt);
   c->sel_done = reinterpret_cast<int32_t *>(ws + L.sel_done);
   c->cand_val = reinterpret_cast<float *>(ws + L.cand_val);
   c->cand_idx = reinterpret_cast<int32_t *>(ws + L.cand_idx);
@@ -156,7 +175,9 @@ int locks_create(const locks_config *cfg, void *workspace, size_t ws_bytes, lock
       cudaMemsetAsync(c->status, 0, 64, 0) != cudaSuccess ||
       cudaMemsetAsync(c->att_done, 0, (size_t)cfg->max_batch * cfg->num_kv_heads * 4, 0) != cudaSuccess ||
       cudaMemsetAsync(c->sel_done, 0, (size_t)cfg->max_batch * cfg->num_kv_heads * 4, 0) != cudaSuccess ||
+      cudaMemsetAsync(c->part_cnt, 0, (size_t)cfg->max_batch * cfg->num_kv_heads * 4, 0) != cudaSuccess ||
       cudaStreamSynchronize(0) != cudaSuccess) {
+    if (c->hint_host) cudaFreeHost(c->hint_host);
     delete c;
     return LOCKS_ERR_CUDA;
   }
@@ -175,7 +196,14 @@ int locks_destroy(locks_ctx *ctx) {
   cudaEventDestroy(ctx->ev_fork);
   cudaEventDestroy(ctx->ev_join);
   cudaStreamDestroy(ctx->side);
+  if (ctx->hint_host) cudaFreeHost(ctx->hint_host);
   delete ctx;
+  return LOCKS_OK;
+}
+
+int locks_set_scan_partition(locks_ctx *ctx, int mode) {
+  if (!ctx || mode < LOCKS_PARTITION_AUTO || mode > LOCKS_PARTITION_BALANCED) return LOCKS_ERR_INVALID_ARG;
+  ctx->scan_partition = mode;
   return LOCKS_OK;
 }
 

@@ -22,6 +22,9 @@ struct BuildParams {
   uint8_t *summ;
   int32_t *status;
   int batch, Hkv, Pmax, num_blocks, r, S, just_filled;
+  // decode step only: where to leave the scan-partition suggestion for these lengths, and the scan's geometry
+  int32_t *hint;
+  int kpages, hint_wpp, hint_rounds, hint_W;
 };
 
 constexpr int kBuildWarps = 4;
@@ -39,6 +42,8 @@ __global__ void __launch_bounds__(kBuildWarps * 32) build_kernel(BuildParams p) 
   extern __shared__ __align__(16) uint8_t smem_raw[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   int b, h, page;
+  if (p.just_filled && p.hint && blockIdx.x == 0 && warp == 0)
+    locks_update_partition_hint(p.hint, p.seq_lens, p.batch, p.Hkv, p.kpages, p.hint_wpp, p.hint_rounds, p.hint_W, lane);
   if (p.just_filled) {
     const int prob = blockIdx.x * kBuildWarps + warp;
     if (prob >= p.batch * p.Hkv) return;
@@ -291,6 +296,11 @@ int locks_launch_build(locks_ctx *c, const locks_kv *kv, int batch, const int32_
   p.summ = reinterpret_cast<uint8_t *>(summaries); p.status = c->status;
   p.batch = batch; p.Hkv = c->cfg.num_kv_heads; p.Pmax = c->Pmax; p.num_blocks = kv->num_blocks;
   p.r = c->cfg.rank; p.S = c->S; p.just_filled = just_filled;
+  p.hint = nullptr; p.kpages = c->k; p.hint_wpp = 1; p.hint_rounds = 1; p.hint_W = 1;
+  if (just_filled && c->hint_dev && c->cfg.summary_fmt == LOCKS_FMT_I4 && c->cfg.q_dtype == LOCKS_BF16) {
+    const locks_scan_geom geo = locks_scan_geometry(c, batch);
+    p.hint = c->hint_dev; p.hint_wpp = geo.wpp; p.hint_rounds = geo.rounds; p.hint_W = geo.W;
+  }
   dim3 grid = just_filled ? dim3((batch * p.Hkv + kBuildWarps - 1) / kBuildWarps)
                           : dim3((c->Pmax + kBuildWarps - 1) / kBuildWarps, p.Hkv, batch);
   const int smem = kBuildWarps * kBuildSmemPerWarp;

@@ -20,6 +20,15 @@
 #ifndef LOCKS_SCAN_GATHER
 #define LOCKS_SCAN_GATHER 1    // rank-8 scan: stage summaries four at a time with tensor-map gathers
 #endif
+#ifndef LOCKS_SCAN_BALANCED
+#define LOCKS_SCAN_BALANCED 1  // tensor scan: deal (problem, group) units to the warps by actual lengths (0: equal warps per problem)
+#endif
+#ifndef LOCKS_SCAN_HINT_LOAD
+#define LOCKS_SCAN_HINT_LOAD 1    // tensor scan: summaries are read with an L2 evict-first policy
+#endif
+#ifndef LOCKS_SCAN_HINT_STORE
+#define LOCKS_SCAN_HINT_STORE 1   // tensor scan: scores are written with an L2 evict-last policy
+#endif
 #ifndef LOCKS_SCAN_BULK
 #define LOCKS_SCAN_BULK 1      // staging of summary blobs in the scan: 1 = cp.async.bulk (TMA) + mbarrier, 0 = 16-byte cp.async
 #endif
@@ -44,6 +53,10 @@ struct locks_ctx {
   int G, k, S, Pmax, max_groups;
   int num_sms;
   int part_slots;          // partial slots per (request, head) the last scan launch may have filled
+  int part_balanced;       // the last scan launch wrote per-problem partial counts to part_cnt instead
+  int scan_partition;      // LOCKS_PARTITION_*: how the tensor scan deals pages to its warps
+  int32_t *hint_host;      // pinned, device-mapped word: partition the device suggests for the current lengths
+  int32_t *hint_dev;       //   (0 none yet, LOCKS_PARTITION_STRIDED, LOCKS_PARTITION_BALANCED)
   int sel_ept;             // pages per thread of a selector CTA (chunk = sel_ept * 512 pages)
   int sel_chunks;          // selector CTAs (chunks) per (request, KV head)
   int sel_kc;              // candidates kept per chunk (k-2)
@@ -53,6 +66,7 @@ struct locks_ctx {
   int32_t *status;         // [4] sticky status, work counters
   float *shat;             // [max_batch][Hq][Pmax]
   float2 *part;            // [max_batch][Hq][max_groups] partial (max, sum exp) over candidate pages
+  int32_t *part_cnt;       // [max_batch][Hkv] partials the scan wrote per head of a problem (balanced partition)
   int32_t *sel_done;       // [max_batch][Hkv] chunk-arrival counters
   float *cand_val;         // [max_batch][Hkv][sel_chunks][sel_kc] chunk lists: 32-bit keys (0 = no entry)
   int32_t *cand_idx;
@@ -85,6 +99,38 @@ struct locks_append {
   int32_t *seq_commit;         // the caller's sequence lengths
   int num_blocks, esz;
 };
+
+// Geometry of a tensor-scan launch: known on the host, used by the launcher and by the partition hint
+struct locks_scan_geom {
+  int grid, W;               // CTAs, warps
+  int wpp, nslots, rounds;   // strided partition: warps per problem, problems in flight, problems per slot
+  int cta_reduce;            // all warps of a CTA share one problem for the whole launch
+};
+locks_scan_geom locks_scan_geometry(const locks_ctx *c, int batch);
+
+// Which partition suits these lengths: iterations of the longest warp, strided = rounds * ceil(max groups / wpp)
+// against balanced = ceil(units / warps); the balanced one has to win by more than its set-up costs.
+// Called by one warp; lane 0 writes *hint.
+__device__ __forceinline__ void locks_update_partition_hint(int32_t *hint, const int32_t *seq_lens, int batch, int Hkv,
+                                                            int k, int wpp, int rounds, int W, int lane) {
+  int sum = 0, mx = 0;
+  for (int b = lane; b < batch; b += 32) {
+    const int P = (seq_lens[b] + LOCKS_B - 1) / LOCKS_B;
+    const int ng = P <= k ? 0 : (P - 1 + LOCKS_GROUP - 1) / LOCKS_GROUP;
+    sum += ng;
+    mx = max(mx, ng);
+  }
+#pragma unroll
+  for (int o = 16; o; o >>= 1) {
+    sum += __shfl_xor_sync(0xffffffffu, sum, o);
+    mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+  }
+  if (lane == 0) {
+    const int strided = rounds * ((mx + wpp - 1) / wpp);
+    const int even = (int)(((int64_t)sum * Hkv + W - 1) / W);
+    *hint = (strided * 16 > even * 17 + 16) ? LOCKS_PARTITION_BALANCED : LOCKS_PARTITION_STRIDED;
+  }
+}
 
 // launchers (each returns LOCKS_OK or LOCKS_ERR_CUDA and adds to ctx->last_launches)
 // seq_inc = 1: lengths are taken one token longer than kv->seq_lens says and published in ctx->seq_eff
@@ -230,6 +276,25 @@ __device__ __forceinline__ void bulk_g2s(void *dst, const void *src, uint32_t by
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n" ::
                    "r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar))
                : "memory");
+}
+// L2 eviction policies: a stream that is read once should not push out what the next kernel reads
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;\n" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_last() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;\n" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ void bulk_g2s_hint(void *dst, const void *src, uint32_t bytes, uint64_t *bar, uint64_t pol) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;\n" ::
+                   "r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)), "l"(pol)
+               : "memory");
+}
+__device__ __forceinline__ void st_f32_hint(float *dst, float v, uint64_t pol) {
+  asm volatile("st.global.L2::cache_hint.f32 [%0], %1, %2;\n" ::"l"(dst), "f"(v), "l"(pol) : "memory");
 }
 __device__ __forceinline__ void fence_barrier_init() {
   asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");

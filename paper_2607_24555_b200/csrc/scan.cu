@@ -31,12 +31,14 @@ struct ScanParams {
   const int32_t *seq_lens;
   float *shat;
   float2 *part;
+  int32_t *part_cnt;   // [batch][Hkv] partials written per head of a problem (balanced partition)
   int32_t *status;
   int batch, Hq, Hkv, G, Pmax, max_groups, num_blocks, k, S, r;
   float sm_scale;
   // decode step with an appended token: lengths count the token that the selector's kernel is about to
   // write (seq_inc = 1); the first CTA publishes them, and the append position, for the step's later kernels
   int cta_reduce;     // every warp of a CTA works on one problem only: one partial per (head, CTA)
+  int wpp, nslots;    // strided partition: warps per problem, problems in flight
   int use_gather;     // rank 8: stage four summaries per tensor-map gather instead of one bulk copy each
   int seq_inc;
   int32_t *seq_eff;   // [2][max_batch]: effective length, append position (-1: none) -- or nullptr
@@ -215,12 +217,19 @@ struct Cursor {
 
 // Four rows of a 2D tensor map (box = one row) to consecutive rows in shared memory, completion on an mbarrier.
 __device__ __forceinline__ void tma_gather4(void *dst, const CUtensorMap *tmap, int r0, int r1, int r2, int r3,
-                                            uint64_t *bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, "
-      "%5, %6}], [%7];\n" ::"r"(smem_u32(dst)),
-      "l"(tmap), "r"(0), "r"(r0), "r"(r1), "r"(r2), "r"(r3), "r"(smem_u32(bar))
-      : "memory");
+                                            uint64_t *bar, uint64_t pol) {
+  if (LOCKS_SCAN_HINT_LOAD)
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes.L2::cache_hint [%0], "
+        "[%1, {%2, %3, %4, %5, %6}], [%7], %8;\n" ::"r"(smem_u32(dst)),
+        "l"(tmap), "r"(0), "r"(r0), "r"(r1), "r"(r2), "r"(r3), "r"(smem_u32(bar)), "l"(pol)
+        : "memory");
+  else
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, "
+        "%5, %6}], [%7];\n" ::"r"(smem_u32(dst)),
+        "l"(tmap), "r"(0), "r"(r0), "r"(r1), "r"(r2), "r"(r3), "r"(smem_u32(bar))
+        : "memory");
 }
 
 __device__ __forceinline__ uint32_t movm_trans(uint32_t v) {
@@ -246,7 +255,7 @@ __device__ __forceinline__ uint32_t movm_trans(uint32_t v) {
 // PK (G <= 4 only): the 8 head columns hold the group twice, so that after MMA#1 the projection, MMA#2 and
 // the log-sum-exp handle two pages at once (rows 0-3 = page A's heads, rows 4-7 = page B's heads, the two
 // pages separated along K) instead of leaving half of the lanes idle.
-template <int R, int NH, bool PK, bool CR>
+template <int R, int NH, bool PK, bool CR, bool BAL>
 __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4_kernel(ScanParams p, const __grid_constant__ CUtensorMap tmap) {
   constexpr int kBlob = i4_stride(R);   // stored bytes of one summary; a stage keeps room for rank-8 blobs
   extern __shared__ __align__(128) uint8_t smem[];
@@ -263,14 +272,86 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4_kerne
   pdl_wait();      // sequence lengths and the previous consumers of the workspace are done
   publish_lengths(p, blockIdx.x == 0, threadIdx.x, kScanWarps * 32);
 
-  // warps stick to one (request, KV head) at a time: `wpp` warps share a problem and stride its groups
+  // Two partitions of the (problem, 8-page group) units over the warps, chosen per launch by the host.
+  // Strided (BAL = false): `wpp` warps share a problem and stride its groups (slot = problem, sub = position
+  // among its warps); best when the sequences are about equally long.  Balanced (BAL = true): every warp owns
+  // an equally long contiguous range of units, whatever the mix of sequence lengths, at the price of a few
+  // hundred instructions of set-up per warp.
+  static_assert(!(CR && BAL), "the CTA-level merge needs the strided partition");
   const int W = gridDim.x * kScanWarps;
   const int wid = blockIdx.x * kScanWarps + warp;
   const int nprob = p.batch * p.Hkv;
-  const int wpp = max(1, W / nprob), nslots = W / wpp;
+  const int wpp = p.wpp, nslots = p.nslots;
   const int slot = wid / wpp, sub = wid - slot * wpp;
-  if (slot >= nslots) return;
+  if (!BAL && slot >= nslots) return;
+  const int gstep = BAL ? 1 : wpp, pstep = BAL ? 1 : nslots, g0 = BAL ? 0 : sub;   // cursor stepping
 
+  auto groups_of = [&](int b) {   // 8-page groups of scored pages of request b
+    const int P = (step_len(p, b) + LOCKS_B - 1) / LOCKS_B;
+    return P <= p.k ? 0 : (P - 1 + LOCKS_GROUP - 1) / LOCKS_GROUP;
+  };
+  int n_units = 0x7fffffff;   // balanced: units this warp owns
+  int pslot_first = 0;        // balanced: partial slot of the first problem this warp touches
+  Cursor cp{slot, sub, 0, 0, 0};
+  if (BAL) {
+    auto scan32 = [&](int v) {   // inclusive prefix sum over the lanes
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int up = __shfl_up_sync(0xffffffffu, v, o);
+        if (lane >= o) v += up;
+      }
+      return v;
+    };
+    // groups per request, 32 requests at a time; the first chunk's totals are kept for the search below
+    const int ng0 = lane < p.batch ? groups_of(lane) : 0;
+    const int incl0 = scan32(ng0);
+    int tot = __shfl_sync(0xffffffffu, incl0, 31);
+    if (p.batch > 32) {
+      int more = 0;
+      for (int b = 32 + lane; b < p.batch; b += 32) more += groups_of(b);
+#pragma unroll
+      for (int o = 16; o; o >>= 1) more += __shfl_xor_sync(0xffffffffu, more, o);
+      tot += more;
+    }
+    // U = q Weff + rem units over the first Weff = min(W, U) warps: the first rem warps own q + 1, the others q
+    const int U = tot * p.Hkv, Weff = min(W, U);
+    if (wid >= Weff) return;
+    const int uq = U / Weff, urem = U - uq * Weff;
+    const int u0 = wid * uq + min(wid, urem);
+    n_units = uq + (wid < urem ? 1 : 0);
+    // the request that holds unit u0 (a request holds Hkv * groups consecutive units)
+    int base = 0, fb = 0, fstart = 0, fng = 1;
+    for (int b0 = 0; b0 < p.batch; b0 += 32) {
+      const int ng = b0 == 0 ? ng0 : ((b0 + lane < p.batch) ? groups_of(b0 + lane) : 0);
+      const int incl = (b0 == 0 ? incl0 : scan32(ng)) * p.Hkv;
+      const int chunk_total = __shfl_sync(0xffffffffu, incl, 31);
+      if (u0 < base + chunk_total) {
+        const int l = __ffs(__ballot_sync(0xffffffffu, base + incl > u0)) - 1;
+        fb = b0 + l;
+        fng = __shfl_sync(0xffffffffu, ng, l);
+        fstart = base + __shfl_sync(0xffffffffu, incl, l) - fng * p.Hkv;
+        break;
+      }
+      base += chunk_total;
+    }
+    const int r = u0 - fstart, hh0 = r / fng;
+    cp.prob = fb * p.Hkv + hh0;
+    cp.grp = r - hh0 * fng;
+    // partials of a problem sit at (warp - first warp that owns one of its units): 0 for every problem this
+    // warp enters at its first group; for the first one, count the warps between its first unit and u0
+    if (cp.grp > 0) {
+      const int us = u0 - cp.grp, big = urem * (uq + 1);
+      const int wf = us < big ? us / (uq + 1) : urem + (us - big) / uq;
+      pslot_first = wid - wf;
+    }
+  }
+
+  // the summaries stream through L2 once; the scores are what the selector reads next
+  const uint64_t pol_stream = l2_policy_evict_first(), pol_keep = l2_policy_evict_last();
+  auto store_score = [&](float *dst, float v) {
+    if (LOCKS_SCAN_HINT_STORE) st_f32_hint(dst, v, pol_keep);
+    else *dst = v;
+  };
   auto enter = [&](Cursor &c) {   // refresh the per-problem fields of the cursor
     c.b = c.prob / p.Hkv;
     c.h = c.prob - c.b * p.Hkv;
@@ -280,10 +361,16 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4_kerne
   };
   auto settle = [&](Cursor &c) {  // move to the next non-empty position at or after (prob, grp)
     while (c.prob < nprob && c.grp * LOCKS_GROUP >= c.nsc) {
-      c.prob += nslots;
-      c.grp = sub;
+      c.prob += pstep;
+      c.grp = g0;
       if (c.prob < nprob) enter(c);
     }
+  };
+  // `more`: the warp owns units past this one (balanced partition; the strided one ends at the last problem)
+  auto advance = [&](Cursor &c, bool more) {
+    c.grp += gstep;
+    if (BAL && !more) c.prob = nprob;
+    else settle(c);
   };
   // the physical block of page (grp*8 + lane) of the producer cursor, fetched one group ahead of use
   auto fetch_block = [&](const Cursor &c) -> int {
@@ -312,15 +399,20 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4_kerne
       if (lane == 0) {
         uint8_t *dst = ring + stage * kStageBytes;
         mbar_expect_tx(&full[stage], (uint32_t)(nvalid > 4 ? 8 : 4) * kBlob);
-        tma_gather4(dst, &tmap, row, r1, r2, r3, &full[stage]);
-        if (nvalid > 4) tma_gather4(dst + 4 * kBlob, &tmap, r4, r5, r6, r7, &full[stage]);
+        tma_gather4(dst, &tmap, row, r1, r2, r3, &full[stage], pol_stream);
+        if (nvalid > 4) tma_gather4(dst + 4 * kBlob, &tmap, r4, r5, r6, r7, &full[stage], pol_stream);
       }
     } else if (kScanBulk) {
       if (lane == 0) mbar_expect_tx(&full[stage], (uint32_t)nvalid * kBlob);
       __syncwarp();
-      if (lane < nvalid)
-        bulk_g2s(ring + stage * kStageBytes + lane * kBlob, p.summ + ((int64_t)block * p.Hkv + h) * kBlob, kBlob,
-                 &full[stage]);
+      if (lane < nvalid) {
+        if (LOCKS_SCAN_HINT_LOAD)
+          bulk_g2s_hint(ring + stage * kStageBytes + lane * kBlob, p.summ + ((int64_t)block * p.Hkv + h) * kBlob, kBlob,
+                        &full[stage], pol_stream);
+        else
+          bulk_g2s(ring + stage * kStageBytes + lane * kBlob, p.summ + ((int64_t)block * p.Hkv + h) * kBlob, kBlob,
+                   &full[stage]);
+      }
     } else {
       // 16-byte chunks of a blob are dealt to the lanes
       uint8_t *dst = ring + stage * kStageBytes;
@@ -335,7 +427,7 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4_kerne
     }
   };
 
-  Cursor cp{slot, sub, 0, 0, 0}, cc;
+  Cursor cc;
   if (cp.prob < nprob) enter(cp);
   settle(cp);
   cc = cp;
@@ -346,8 +438,7 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4_kerne
     if (cp.prob < nprob) {
       issue(s, cp, next_block);
       ++inflight;
-      cp.grp += wpp;
-      settle(cp);
+      advance(cp, inflight < n_units);
       next_block = fetch_block(cp);
     }
   }
@@ -412,7 +503,7 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4_kerne
   float pm[NH], ps[NH];
 #pragma unroll
   for (int hh = 0; hh < NH; ++hh) { pm[hh] = -INFINITY; ps[hh] = 0.f; }
-  int cur_b = 0, cur_h = 0;
+  int cur_b = 0, cur_h = 0, cur_pslot = sub;   // partial slot of this warp in the current problem
   auto accumulate = [&](float &m, float &sacc, float v) {   // online log-sum-exp, one exp per value
     if (v > -INFINITY) {
       const float d = v - m, e = __expf(-fabsf(d));
@@ -420,7 +511,10 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4_kerne
     }
   };
   float2 *red = reinterpret_cast<float2 *>(smem + kScanWarps * (kScanStages * kStageBytes + 64));   // [warp][16]
-  auto flush = [&](bool to_smem) {
+  auto flush = [&](bool to_smem, bool finished) {
+    const int pslot = cur_pslot;
+    // balanced: the warp that finishes a problem's last group knows how many partials it has
+    if (BAL && finished && lane == 0) p.part_cnt[cur_prob] = pslot + 1;
 #pragma unroll
     for (int hh = 0; hh < NH; ++hh) {
       float m = pm[hh], sacc = ps[hh];
@@ -434,7 +528,7 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4_kerne
       const int g = PK ? (x & 3) : x + 8 * hh;
       if (t == 0 && (!PK || x < 4) && g < p.G) {
         if (CR && to_smem) red[warp * 16 + g] = make_float2(m, sacc);
-        else p.part[((int64_t)cur_b * p.Hq + cur_h * p.G + g) * p.max_groups + sub] = make_float2(m, sacc);
+        else p.part[((int64_t)cur_b * p.Hq + cur_h * p.G + g) * p.max_groups + pslot] = make_float2(m, sacc);
       }
       pm[hh] = -INFINITY;
       ps[hh] = 0.f;
@@ -459,10 +553,11 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4_kerne
     --inflight;
     const int b = cc.b, h = cc.h;
     if (cc.prob != cur_prob) {
-      if (cur_prob >= 0) flush(false);
+      if (cur_prob >= 0) flush(false, true);
       cur_prob = cc.prob;
       cur_b = b;
       cur_h = h;
+      cur_pslot = BAL ? (it == 0 ? pslot_first : 0) : sub;
 #pragma unroll
       for (int hh = 0; hh < NH; ++hh) {
         float s8;
@@ -738,8 +833,7 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4_kerne
     if (cp.prob < nprob) {
       issue(stage, cp, next_block);
       ++inflight;
-      cp.grp += wpp;
-      settle(cp);
+      advance(cp, it + 1 + inflight < n_units);
       next_block = fetch_block(cp);
     }
 
@@ -748,7 +842,7 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4_kerne
       const int g = x & 3, page = cc.grp * LOCKS_GROUP + 2 * t + (x >> 2);
       const float v = res[0] * kLn2;
       const bool in = t < LOCKS_GROUP / 2 && page < cc.nsc;
-      if (g < p.G && in) p.shat[((int64_t)b * p.Hq + h * p.G + g) * p.Pmax + page] = v;
+      if (g < p.G && in) store_score(p.shat + ((int64_t)b * p.Hq + h * p.G + g) * p.Pmax + page, v);
       accumulate(pm[0], ps[0], (in && page >= 1) ? v : -INFINITY);
     } else {
     const int page0 = cc.grp * LOCKS_GROUP + 2 * t;
@@ -760,20 +854,19 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4_kerne
       const bool in0 = t < LOCKS_GROUP / 2 && page0 < cc.nsc, in1 = t < LOCKS_GROUP / 2 && page0 + 1 < cc.nsc;
       if (g < p.G) {
         float *dst = p.shat + ((int64_t)b * p.Hq + h * p.G + g) * p.Pmax + page0;
-        if (in0) dst[0] = v0;
-        if (in1) dst[1] = v1;
+        if (in0) store_score(dst, v0);
+        if (in1) store_score(dst + 1, v1);
       }
       accumulate(pm[hh], ps[hh], (in0 && page0 >= 1) ? v0 : -INFINITY);
       accumulate(pm[hh], ps[hh], in1 ? v1 : -INFINITY);
     }
     }
-    cc.grp += wpp;
-    settle(cc);
+    advance(cc, it + 1 < n_units);
     ++it;
   }
   if (CR) {
     // geometry guarantees that all warps of this CTA reach this point and share the problem `slot`
-    flush(true);
+    flush(true, true);
     __syncthreads();
     if (warp == 0 && lane < p.G) {
       float m = -INFINITY, sacc = 0.f;
@@ -787,7 +880,7 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4_kerne
       p.part[((int64_t)pb * p.Hq + ph * p.G + lane) * p.max_groups + sub / kScanWarps] = make_float2(m, sacc);
     }
   } else if (ok && cur_prob >= 0) {
-    flush(false);
+    flush(false, cc.grp * LOCKS_GROUP >= cc.nsc);   // the last unit was the problem's last group
   }
   if (!ok) {
     // a wait ran out: flag it, then give copies still in flight a bounded chance to land before exit
@@ -801,6 +894,24 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4_kerne
 
 }  // namespace
 
+locks_scan_geom locks_scan_geometry(const locks_ctx *c, int batch) {
+  locks_scan_geom g;
+  const int Hkv = c->cfg.num_kv_heads;
+  const int total_groups = batch * Hkv * c->max_groups;
+  g.grid = kScanCtasPerSm * c->num_sms;
+  const int need = (total_groups + kScanWarps - 1) / kScanWarps;
+  if (g.grid > need) g.grid = need < 1 ? 1 : need;
+  g.W = g.grid * kScanWarps;
+  const int nprob = batch * Hkv;
+  g.wpp = g.W / nprob > 1 ? g.W / nprob : 1;
+  g.nslots = g.W / g.wpp;
+  g.rounds = (nprob + g.nslots - 1) / g.nslots;
+  // few problems: every CTA's warps share one problem for the whole launch and none leaves early,
+  // so the CTA merges its warps' partials before writing (the selector reads 8x fewer)
+  g.cta_reduce = (c->cfg.rank == 8 && g.wpp % kScanWarps == 0 && g.nslots == nprob && g.nslots * g.wpp == g.W) ? 1 : 0;
+  return g;
+}
+
 int locks_launch_scan(locks_ctx *c, const void *q, const void *summaries, const locks_kv *kv, int batch,
                       float *shat, int seq_inc, cudaStream_t st) {
   ScanParams p;
@@ -813,26 +924,27 @@ int locks_launch_scan(locks_ctx *c, const void *q, const void *summaries, const 
   p.seq_lens = kv->seq_lens;
   p.shat = shat;
   p.part = c->part;
+  p.part_cnt = c->part_cnt;
   p.status = c->status;
   p.batch = batch; p.Hq = c->cfg.num_q_heads; p.Hkv = c->cfg.num_kv_heads; p.G = c->G;
   p.Pmax = c->Pmax; p.max_groups = c->max_groups; p.num_blocks = kv->num_blocks; p.k = c->k;
   p.S = c->S; p.r = c->cfg.rank; p.sm_scale = c->cfg.sm_scale;
   const bool tensor = c->cfg.summary_fmt == LOCKS_FMT_I4 && c->cfg.q_dtype == LOCKS_BF16;   // ranks 2, 4, 8
   c->part_slots = c->max_groups;   // generic kernel: one partial per 8-page group
+  c->part_balanced = 0;
   if (tensor) {
-    const int total_groups = batch * p.Hkv * p.max_groups;
-    int grid = kScanCtasPerSm * c->num_sms;
-    const int need = (total_groups + kScanWarps - 1) / kScanWarps;
-    if (grid > need) grid = need < 1 ? 1 : need;
-    {   // tensor kernel: one partial per (problem, warp); mirrors the kernel's own partition
-      const int W = grid * kScanWarps, nprob = batch * p.Hkv;
-      const int wpp = W / nprob > 1 ? W / nprob : 1, nslots = W / wpp;
-      c->part_slots = wpp;
-      // few problems: every CTA's warps share one problem for the whole launch and none leaves early,
-      // so the CTA merges its warps' partials before writing (the selector reads 8x fewer)
-      p.cta_reduce = (c->cfg.rank == 8 && wpp % kScanWarps == 0 && nslots == nprob && nslots * wpp == W) ? 1 : 0;
-      if (p.cta_reduce) c->part_slots = wpp / kScanWarps;
-    }
+    const locks_scan_geom geo = locks_scan_geometry(c, batch);
+    const int grid = geo.grid;
+    p.wpp = geo.wpp; p.nslots = geo.nslots; p.cta_reduce = geo.cta_reduce;
+    // strided partition: one partial per (problem, warp), or per (problem, CTA) with the CTA-level merge;
+    // balanced partition: the kernel counts the partials of each problem itself (part_cnt)
+    c->part_slots = geo.cta_reduce ? geo.wpp / kScanWarps : geo.wpp;
+    int mode = c->scan_partition;
+    if (mode == LOCKS_PARTITION_AUTO)
+      mode = (c->hint_host && *reinterpret_cast<volatile int32_t *>(c->hint_host) == LOCKS_PARTITION_BALANCED)
+                 ? LOCKS_PARTITION_BALANCED : LOCKS_PARTITION_STRIDED;
+    const bool balanced = LOCKS_SCAN_BALANCED && !geo.cta_reduce && mode == LOCKS_PARTITION_BALANCED;
+    c->part_balanced = balanced ? 1 : 0;
     const dim3 g(grid), blk(kScanWarps * 32);
     const int gsel = c->G <= 4 ? 0 : (c->G <= 8 ? 1 : 2);
     // tensor map over the summaries for the gather path (rank 8): rows = (block, KV head), 208 32-bit words each
@@ -862,23 +974,26 @@ int locks_launch_scan(locks_ctx *c, const void *q, const void *summaries, const 
           p.use_gather = 1;
       }
     }
-#define LOCKS_SCAN_LAUNCH(R_, CR_)                                                                                     \
+#define LOCKS_SCAN_LAUNCH(R_, CR_, BAL_)                                                                                  \
   do {                                                                                                                 \
     static bool attr_done = false;                                                                                     \
     if (!attr_done) {                                                                                                  \
-      cudaFuncSetAttribute(scan_i4_kernel<R_, 1, true, CR_>, cudaFuncAttributeMaxDynamicSharedMemorySize, kScanSmem);  \
-      cudaFuncSetAttribute(scan_i4_kernel<R_, 1, false, CR_>, cudaFuncAttributeMaxDynamicSharedMemorySize, kScanSmem); \
-      cudaFuncSetAttribute(scan_i4_kernel<R_, 2, false, CR_>, cudaFuncAttributeMaxDynamicSharedMemorySize, kScanSmem); \
+      cudaFuncSetAttribute(scan_i4_kernel<R_, 1, true, CR_, BAL_>, cudaFuncAttributeMaxDynamicSharedMemorySize, kScanSmem);  \
+      cudaFuncSetAttribute(scan_i4_kernel<R_, 1, false, CR_, BAL_>, cudaFuncAttributeMaxDynamicSharedMemorySize, kScanSmem); \
+      cudaFuncSetAttribute(scan_i4_kernel<R_, 2, false, CR_, BAL_>, cudaFuncAttributeMaxDynamicSharedMemorySize, kScanSmem); \
       attr_done = true;                                                                                                \
     }                                                                                                                  \
-    if (gsel == 0) locks_launch_pdl(scan_i4_kernel<R_, 1, true, CR_>, g, blk, kScanSmem, st, p, tmap);                       \
-    else if (gsel == 1) locks_launch_pdl(scan_i4_kernel<R_, 1, false, CR_>, g, blk, kScanSmem, st, p, tmap);                 \
-    else locks_launch_pdl(scan_i4_kernel<R_, 2, false, CR_>, g, blk, kScanSmem, st, p, tmap);                                \
+    if (gsel == 0) locks_launch_pdl(scan_i4_kernel<R_, 1, true, CR_, BAL_>, g, blk, kScanSmem, st, p, tmap);                       \
+    else if (gsel == 1) locks_launch_pdl(scan_i4_kernel<R_, 1, false, CR_, BAL_>, g, blk, kScanSmem, st, p, tmap);                 \
+    else locks_launch_pdl(scan_i4_kernel<R_, 2, false, CR_, BAL_>, g, blk, kScanSmem, st, p, tmap);                                \
   } while (0)
-    if (c->cfg.rank == 8 && p.cta_reduce) LOCKS_SCAN_LAUNCH(8, true);
-    else if (c->cfg.rank == 8) LOCKS_SCAN_LAUNCH(8, false);
-    else if (c->cfg.rank == 4) LOCKS_SCAN_LAUNCH(4, false);
-    else LOCKS_SCAN_LAUNCH(2, false);
+    if (c->cfg.rank == 8 && p.cta_reduce) LOCKS_SCAN_LAUNCH(8, true, false);
+    else if (c->cfg.rank == 8 && balanced) LOCKS_SCAN_LAUNCH(8, false, true);
+    else if (c->cfg.rank == 8) LOCKS_SCAN_LAUNCH(8, false, false);
+    else if (c->cfg.rank == 4 && balanced) LOCKS_SCAN_LAUNCH(4, false, true);
+    else if (c->cfg.rank == 4) LOCKS_SCAN_LAUNCH(4, false, false);
+    else if (balanced) LOCKS_SCAN_LAUNCH(2, false, true);
+    else LOCKS_SCAN_LAUNCH(2, false, false);
 #undef LOCKS_SCAN_LAUNCH
   } else {
     dim3 grid((c->max_groups + 3) / 4, p.Hkv, batch);

@@ -28,6 +28,7 @@ struct SelParams {
   const float *shat;
   const float2 *part;
   const int32_t *seq_lens;
+  const int32_t *part_cnt;   // partials per head of each problem, or nullptr: part_slots for all
   int32_t *ids, *cnt;
   float *logshare;
   uint32_t *cand_key;  // [batch][Hkv][chunks][kc] chunk lists (chunked selection only): keys, 0 = no entry
@@ -445,7 +446,8 @@ __global__ void __launch_bounds__(LOCKS_SEL_THREADS) select_kernel(SelParams p) 
     const float *shat0 = p.shat + ((int64_t)b * p.Hq + h * p.G) * p.Pmax;
     const float2 *part0 = p.part + ((int64_t)b * p.Hq + h * p.G) * p.max_groups;
     float *ls0 = p.logshare ? p.logshare + prob * p.Pmax : nullptr;
-    const int nparts = min(p.part_slots, (P - 1 + LOCKS_GROUP - 1) / LOCKS_GROUP);
+    const int nparts = p.part_cnt ? min(max(p.part_cnt[prob], 0), p.max_groups)
+                                  : min(p.part_slots, (P - 1 + LOCKS_GROUP - 1) / LOCKS_GROUP);
     if (nslab >= 3) chunk_keys<4>(shat0, part0, ls0, p.G, p.Pmax, p.max_groups, nparts, c0, nslab, P);
     else if (nslab == 2) chunk_keys<2>(shat0, part0, ls0, p.G, p.Pmax, p.max_groups, nparts, c0, nslab, P);
     else chunk_keys<1>(shat0, part0, ls0, p.G, p.Pmax, p.max_groups, nparts, c0, nslab, P);
@@ -484,6 +486,7 @@ int locks_launch_select(locks_ctx *c, const float *shat, const locks_kv *kv, int
   p.max_groups = c->max_groups; p.k = c->k; p.chunks = c->sel_chunks; p.kc = c->sel_kc;
   p.chunk_pages = c->sel_ept * LOCKS_SEL_THREADS;
   p.part_slots = c->part_slots;
+  p.part_cnt = c->part_balanced ? c->part_cnt : nullptr;
   if (p.chunk_pages > kMaxKeys || (int64_t)c->sel_chunks * c->sel_kc > kMaxKeys || p.G > 16) return LOCKS_ERR_UNSUPPORTED;
   static bool attr_done = false;
   if (!attr_done) {

@@ -14,6 +14,7 @@ import torch
 
 import locks_synth
 import oracle
+import paper_2607_24555_b200 as locks
 from common import t2np
 
 pytestmark = pytest.mark.gpu
@@ -170,6 +171,69 @@ def test_randomized_shapes(trial):
     ids2, cnt2, lm2, ls2 = gc.gpu_select(torch.from_numpy(summ).cuda())
     assert np.array_equal(ids1, ids2) and np.array_equal(cnt1, cnt2)
     assert gc.status() == 0
+
+
+@pytest.mark.parametrize("Hq,Hkv,rank", [(8, 2, 8), (16, 2, 8), (32, 2, 8), (8, 2, 2), (8, 2, 4), (12, 2, 2)])
+def test_balanced_partition_ragged_batch(Hq, Hkv, rank):
+    """The scan's balanced partition (equal page ranges per warp) on a batch of very different lengths:
+    warps that start inside a problem, warps that span several problems, requests shorter than the
+    budget (no candidates) and a one-page request.  Scores, shares, sets and outputs against the oracle,
+    and the same selection as the strided partition."""
+    from gpu_util import check_select_and_attend
+    lens = [16 * 700 + 5, 40, 16 * 90, 16 * 2300 + 9, 7, 16 * 300 + 1, 16 * 41]
+    w = small_bf16(lens, Hq=Hq, Hkv=Hkv, rank=rank, budget=256, seed=300 + Hq + rank)
+    gc = _gc(w)
+    summ = gc.oracle_summaries()
+    dsumm = torch.from_numpy(summ).cuda()
+    gc.ctx.locks_set_scan_partition(locks.PARTITION_STRIDED)
+    ids_s, cnt_s, lm_s, ls_s = gc.gpu_select(dsumm)
+    gc.ctx.locks_set_scan_partition(locks.PARTITION_BALANCED)
+    check_select_and_attend(gc, summ, out_tol=2e-2)
+    ids_b, cnt_b, lm_b, ls_b = gc.gpu_select(dsumm)
+    assert np.array_equal(cnt_s, cnt_b)
+    for b, T in enumerate(lens):
+        P = -(-T // 16)
+        if P > gc.k:   # same scores bit for bit (the partition only changes who computes them)
+            assert np.array_equal(lm_s[b, :, :P - 1], lm_b[b, :, :P - 1])
+            assert np.abs(ls_s[b, :, 1:P - 1] - ls_b[b, :, 1:P - 1]).max() <= 1e-5
+    assert gc.status() == 0
+
+
+def test_balanced_partition_more_problems_than_warps_per_problem():
+    """Balanced partition with many short problems: most warps cross several problem boundaries."""
+    from gpu_util import check_select_and_attend
+    rng = np.random.default_rng(77)
+    lens = [int(rng.integers(16 * 20, 16 * 60)) for _ in range(48)]
+    w = small_bf16(lens, Hq=8, Hkv=4, rank=8, budget=128, seed=78)
+    gc = _gc(w)
+    gc.ctx.locks_set_scan_partition(locks.PARTITION_BALANCED)
+    check_select_and_attend(gc, gc.oracle_summaries(), out_tol=2e-2)
+
+
+def test_partition_suggestion_follows_lengths():
+    """Decode steps leave a suggestion for the scan's partition: ragged lengths turn the balanced one on
+    for the following calls, and the step's results do not depend on it."""
+    from common import check_page_sets, oracle_cache
+    lens = [16 * 9000, 16 * 150, 16 * 200, 16 * 120, 16 * 180]   # 10 problems, one 50 times longer
+    w = small_bf16([t + 16 for t in lens], Hq=8, Hkv=2, rank=8, budget=256, seed=91)
+    gc = _gc(w)
+    gc.case.seq_lens.copy_(torch.tensor(lens, dtype=torch.int32, device="cuda:0"))
+    summ = gc.ctx.new_summaries(gc.case.num_blocks)
+    gc.ctx.locks_build_summaries(gc.kv, w.n, summ)
+    out = torch.empty(w.n, w.Hq, w.d, dtype=torch.bfloat16, device="cuda:0")
+    ids = torch.empty(w.n, w.Hkv, gc.k, dtype=torch.int32, device="cuda:0")
+    cnt = torch.empty(w.n, w.Hkv, dtype=torch.int32, device="cuda:0")
+    for step in range(3):   # step 0 runs strided (no suggestion yet), the later ones balanced
+        kn, vn, qn = locks_synth.new_token(w, step, device="cuda:0")
+        gc.ctx.locks_decode_step(qn, kn, vn, gc.kv, summ, w.n, out, ids, cnt)
+        torch.cuda.synchronize()
+        assert gc.status() == 0
+        cache = oracle_cache(gc.case)
+        shat = oracle.page_logmass(cache, t2np(qn), w.rank, gc.fmt, summ.cpu().numpy(), gc.sm)
+        oids, ocnt, ols = oracle.select(cache, shat, gc.k)
+        check_page_sets(ids.cpu().numpy(), cnt.cpu().numpy(), oids, ocnt, ols, cache.seq_lens, w.B, gc.k)
+        oout, _ = oracle.attend(cache, t2np(qn), gc.sm, ids.cpu().numpy(), cnt.cpu().numpy())
+        assert np.abs(out.float().cpu().numpy() - oout).max() <= 2e-2, step
 
 
 def test_two_level_select_long_context():
