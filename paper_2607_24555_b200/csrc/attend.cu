@@ -129,6 +129,7 @@ __global__ void __launch_bounds__(LOCKS_ATT_WARPS * 32) attend_bf16_kernel(AttPa
   int blk_cur, nt_cur, blk_nxt = 0, nt_nxt = 0;
   resolve_batch(0, blk_cur, nt_cur);
 
+  const uint64_t pol_stream = l2_policy_evict_first();
   auto issue = [&](int j, int stage) -> int {  // j-th page of this warp; returns its valid tokens
     const int block = __shfl_sync(0xffffffffu, blk_cur, j & 31);
     const int ntok = __shfl_sync(0xffffffffu, nt_cur, j & 31);
@@ -139,7 +140,16 @@ __global__ void __launch_bounds__(LOCKS_ATT_WARPS * 32) attend_bf16_kernel(AttPa
     for (int i = 0; i < 8; ++i) {
       const uint32_t so = sw[i & 3] + 512 * i;
       const bool valid = tok0 + 2 * i < ntok;   // rows past the sequence end are zero-filled
-      if (CONTIG) {   // token rows are 256 bytes apart: immediate offsets
+      if (LOCKS_ATT_HINT_LOAD) {   // K and V stream through L2 once: they should not push out the small
+                                   // tables (lengths, block table, page ids) every kernel of the step re-reads
+        if (CONTIG) {   // token rows are 256 bytes apart: immediate offsets
+          cp_async16_hint(kt + so, kp + i * 512, valid, pol_stream);
+          cp_async16_hint(vt + so, vp + i * 512, valid, pol_stream);
+        } else {
+          cp_async16_hint(kt + so, kp + i * gstep, valid, pol_stream);
+          cp_async16_hint(vt + so, vp + i * gstep, valid, pol_stream);
+        }
+      } else if (CONTIG) {
         cp_async16(kt + so, kp + i * 512, valid);
         cp_async16(vt + so, vp + i * 512, valid);
       } else {

@@ -29,6 +29,9 @@
 #ifndef LOCKS_SCAN_HINT_STORE
 #define LOCKS_SCAN_HINT_STORE 1   // tensor scan: scores are written with an L2 evict-last policy
 #endif
+#ifndef LOCKS_ATT_HINT_LOAD
+#define LOCKS_ATT_HINT_LOAD 1     // sparse attention: K and V tiles are read with an L2 evict-first policy
+#endif
 #ifndef LOCKS_SCAN_BULK
 #define LOCKS_SCAN_BULK 1      // staging of summary blobs in the scan: 1 = cp.async.bulk (TMA) + mbarrier, 0 = 16-byte cp.async
 #endif
@@ -305,6 +308,16 @@ __device__ __forceinline__ void cp_async16(void *dst, const void *src, bool vali
   int sz = valid ? 16 : 0;  // src-size 0 zero-fills the destination
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(smem_u32(dst)), "l"(src), "r"(sz)
                : "memory");
+}
+// With an L2 cache policy.  The policy operand is only ever combined with a full 16-byte copy: the hinted
+// form with a source size below the copy size (the zero-fill idiom) raised "illegal instruction" on sm_100a,
+// so rows to be zero-filled take the plain form.
+__device__ __forceinline__ void cp_async16_hint(void *dst, const void *src, bool valid, uint64_t pol) {
+  if (valid)
+    asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2;\n" ::"r"(smem_u32(dst)), "l"(src), "l"(pol)
+                 : "memory");
+  else
+    cp_async16(dst, src, false);
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
 template <int N> __device__ __forceinline__ void cp_async_wait() {
