@@ -152,6 +152,9 @@ int locks_decode_step(locks_ctx *ctx, const void *q, const void *k_new, const vo
  * the workspace, runs locks_decode_step, copies out back to out_host (and the page ids / counts
  * if page_ids_host / page_count_host are given) and synchronises the stream before returning.
  * The cache, summaries, block table and seq_lens stay on the device.
+ * Host buffers that the device can address (page-locked and mapped, as cudaHostAlloc returns them) are not
+ * copied by the copy engine: one small kernel fetches q / k_new / v_new over the bus and the attention kernel
+ * writes out_host itself, which saves four copy nodes per step; other buffers go through async copies.
  * Repeated calls with the same arguments (a serving loop calls once per layer and step with fixed
  * buffers) are cached: from the third call on, the copies and the step are one CUDA-graph launch.
  * The cache holds 8 argument sets per context, needs page-locked host buffers and a stream that is
