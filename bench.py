@@ -70,12 +70,13 @@ def algorithmic_bytes(w, reserve_tokens=0):
     return scan, attend, dense
 
 
-def config_dict(w, layers, identity):
+def config_dict(w, layers, identity, partition="auto"):
     scan_b, att_b, _ = algorithmic_bytes(w)
     return {"workload": w.name, "batch_per_gpu": w.n, "context": w.seq_lens[0], "q_heads": w.Hq, "kv_heads": w.Hkv,
             "head_dim": w.d, "page": w.B, "rank": w.rank, "budget_tokens": w.budget,
             "summary": f"r{w.rank}i4" if w.fmt == "i4" else f"r{w.rank}f32", "launch": "one CUDA graph per step",
             "block_mapping": "identity" if identity else "seeded random permutation",
+            "scan_partition": partition,
             "l2": f"inputs larger than L2: replays cycle over {layers} independent layers "
                   f"({(scan_b + att_b) / 1e6:.0f} MB touched per step, L2 126 MB)"}
 
@@ -189,7 +190,7 @@ def run_reference(args):
     line = {"impl": "reference", "metric": METRIC, "value": us, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
             "warmup": 1, "ms_per_step": us / 1e3, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
             "dtype": "f64", "data": "synthetic",
-            "config": config_dict(w, args.layers, args.identity_blocks),
+            "config": config_dict(w, args.layers, args.identity_blocks, args.scan_partition),
             "cpu_baseline": {"value": us, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
             "e2e": {"value": us, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line))
@@ -225,6 +226,8 @@ def run_ours(args):
     max_pages = layers[0].block_table.shape[1]
     cfg = make_config(w0.Hq, w0.Hkv, w0.rank, w0.fmt, w0.dtype, w0.n, max_pages, w0.budget)
     ctx = locks.Context(cfg, device=dev)
+    ctx.locks_set_scan_partition({"auto": locks.PARTITION_AUTO, "strided": locks.PARTITION_STRIDED,
+                                  "balanced": locks.PARTITION_BALANCED}[args.scan_partition])
     kvs = [KVView(c.k, c.v, c.strides, c.num_blocks, c.block_table, c.seq_lens) for c in layers]
     summs = [ctx.new_summaries(c.num_blocks) for c in layers]
     t0 = time.perf_counter()
@@ -338,7 +341,7 @@ def run_ours(args):
         "metric": METRIC, "value": step_ms_max * 1e3, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": step_ms_max, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16" if w0.dtype == "bf16" else "f32", "data": "synthetic",
-        "config": config_dict(w0, L, args.identity_blocks),
+        "config": config_dict(w0, L, args.identity_blocks, args.scan_partition),
         "e2e": {"value": e2e_ms_max * 1e3, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": launches_per_step * K,
         "clocks": clocks,
@@ -368,6 +371,8 @@ def main():
     ap.add_argument("--workload", default="cfg1")
     ap.add_argument("--layers", type=int, default=4)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--scan-partition", default="auto", choices=["auto", "strided", "balanced"],
+                    help="how the scan deals pages to its warps (auto: the library follows the lengths)")
     ap.add_argument("--identity-blocks", action="store_true",
                     help="logical page i of a request sits in consecutive physical blocks (default: seeded permutation)")
     args = ap.parse_args()

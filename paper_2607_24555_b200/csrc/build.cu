@@ -110,64 +110,108 @@ __global__ void __launch_bounds__(kBuildWarps * 32) build_kernel(BuildParams p) 
     U[i * 17 + j] = (i == j) ? 1.f : 0.f;
   }
   __syncwarp();
-  // ---- 3. parallel cyclic Jacobi
-  float normA = 0.f;
-  for (int e = lane; e < 256; e += 32) { const float a = A[(e >> 4) * 17 + (e & 15)]; normA += a * a; }
-  normA = warp_sum(normA);
-  for (int sweep = 0; sweep < 12; ++sweep) {
-    float off = 0.f;
-    for (int e = lane; e < 256; e += 32) {
-      const int i = e >> 4, j = e & 15;
-      if (i != j) { const float a = A[i * 17 + j]; off += a * a; }
+  // ---- 3. parallel cyclic Jacobi, matrix held in registers.
+  // "Slot" space: the 8 rotations of a round always act on the slot pairs (2m, 2m+1); between rounds the 16
+  // indices move through the slots by the fixed round-robin permutation `next_slot` (slot 0 stays, the others
+  // go round the circle), so that 15 rounds pair every two indices once.  Lane (m = lane / 4, k = lane % 4) holds
+  // rows 2m, 2m+1 x columns 4k .. 4k+3 of A (two 2x2 blocks) and of U (rows = tokens, columns = slots).  A round
+  // is: rotation angles at the lanes that hold a diagonal block, six shuffles to hand them to the rows and
+  // columns they act on, the block updates in registers, and one pass through shared memory (ping-pong
+  // buffers, one warp barrier) that applies the permutation.
+  {
+    const int m = lane >> 2, k = lane & 3;
+    auto next_slot = [](int x) { return x == 0 ? 0 : (x == 1 ? 2 : (x == 14 ? 15 : ((x & 1) ? x - 2 : x + 2))); };
+    constexpr int kJS = 20;   // row stride of the exchange buffers (16-byte aligned rows)
+    float *buf0 = Ds, *buf1 = Ds + 2 * LOCKS_B * kJS;   // each: A[16][kJS] then U[16][kJS]
+    float a[8], u[8];   // index = 4 * blk + 2 * rowbit + colbit, columns 4k + 2 blk + colbit
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      const int i = 2 * m + ((e >> 1) & 1), j = 4 * k + 2 * (e >> 2) + (e & 1);
+      a[e] = A[i * 17 + j];
+      u[e] = (i == j) ? 1.f : 0.f;
     }
-    off = warp_sum(off);
-    if (off <= 1e-13f * normA || normA == 0.f) break;
-    for (int round = 0; round < 15; ++round) {
-      // round-robin pairing: (15, round), ((round + m) % 15, (round - m + 15) % 15), m = 1..7
-      if (lane < 8) {
-        int pi, qi;
-        if (lane == 0) { pi = round; qi = 15; }
-        else { pi = (round + lane) % 15; qi = (round - lane + 15) % 15; }
-        if (pi > qi) { const int tmp = pi; pi = qi; qi = tmp; }
-        const float apq = A[pi * 17 + qi], app = A[pi * 17 + pi], aqq = A[qi * 17 + qi];
-        float c = 1.f, s = 0.f;
-        if (fabsf(apq) > 1e-30f) {
-          const float theta = (aqq - app) / (2.f * apq);
-          const float tt = copysignf(1.f, theta) / (fabsf(theta) + sqrtf(theta * theta + 1.f));
-          c = rsqrtf(tt * tt + 1.f);
-          s = tt * c;
+    int wr_row[2], wr_col[4];   // where this lane's rows / columns go after a round
+#pragma unroll
+    for (int rb = 0; rb < 2; ++rb) wr_row[rb] = next_slot(2 * m + rb);
+#pragma unroll
+    for (int c4 = 0; c4 < 4; ++c4) wr_col[c4] = next_slot(4 * k + c4);
+    const bool diag_lane = k == (m >> 1);
+    const int dblk = m & 1;             // which of the two blocks is the diagonal one (diag lanes)
+    const int src_row = m * 4 + (m >> 1);           // lane holding the diagonal block of row pair m
+    const int src_c0 = 9 * k, src_c1 = 9 * k + 4;   // ... of column pairs 2k and 2k + 1
+    float normA = 0.f;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) normA += a[e] * a[e];
+    normA = warp_sum(normA);
+    int parity = 0;
+    for (int sweep = 0; sweep < 12; ++sweep) {
+      float off = 0.f;
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        const bool on_diag = diag_lane && (e >> 2) == dblk && (((e >> 1) & 1) == (e & 1));
+        off += on_diag ? 0.f : a[e] * a[e];
+      }
+      off = warp_sum(off);
+      if (off <= 1e-13f * normA || normA == 0.f) break;
+#pragma unroll 1
+      for (int round = 0; round < 15; ++round) {
+        // rotation of the slot pair held as a diagonal block (other lanes compute on whatever they hold; unused)
+        const float app = dblk ? a[4] : a[0], apq = dblk ? a[5] : a[1], aqq = dblk ? a[7] : a[3];
+        float c = 1.f, sn = 0.f;
+        {
+          // tan of the rotation angle: t = 2 apq / (d + sign(d) sqrt(d^2 + 4 apq^2)), d = aqq - app (the smaller
+          // root).  Approximate root and division are enough for the angle; c^2 + s^2 = 1 comes from the last
+          // two lines.  Entries too small to square are left alone.
+          const float d = aqq - app, h = d * d + 4.f * apq * apq;
+          if (h > 1e-37f && h < 1e37f) {
+            const float tt = __fdividef(2.f * apq, d + copysignf(h * rsqrtf(h), d));
+            c = rsqrtf(tt * tt + 1.f);
+            sn = tt * c;
+          }
         }
-        rot[lane] = c; rot[8 + lane] = s;
-        reinterpret_cast<int *>(rot)[16 + lane] = pi;
-        reinterpret_cast<int *>(rot)[24 + lane] = qi;
-      }
-      __syncwarp();
-      // columns: A <- A J, U <- U J   (item = (row i, pair m))
+        const float cr = __shfl_sync(0xffffffffu, c, src_row), sr = __shfl_sync(0xffffffffu, sn, src_row);
+        const float cc[2] = {__shfl_sync(0xffffffffu, c, src_c0), __shfl_sync(0xffffffffu, c, src_c1)};
+        const float sc[2] = {__shfl_sync(0xffffffffu, sn, src_c0), __shfl_sync(0xffffffffu, sn, src_c1)};
+        float *dst = parity ? buf1 : buf0;
 #pragma unroll
-      for (int it = 0; it < 4; ++it) {
-        const int item = lane + 32 * it, i = item >> 3, m = item & 7;
-        const float c = rot[m], s = rot[8 + m];
-        const int pi = reinterpret_cast<int *>(rot)[16 + m], qi = reinterpret_cast<int *>(rot)[24 + m];
-        const float aip = A[i * 17 + pi], aiq = A[i * 17 + qi];
-        A[i * 17 + pi] = c * aip - s * aiq;
-        A[i * 17 + qi] = s * aip + c * aiq;
-        const float uip = U[i * 17 + pi], uiq = U[i * 17 + qi];
-        U[i * 17 + pi] = c * uip - s * uiq;
-        U[i * 17 + qi] = s * uip + c * uiq;
-      }
-      __syncwarp();
-      // rows: A <- J^T A
+        for (int blk = 0; blk < 2; ++blk) {
+          float *x = a + 4 * blk, *y = u + 4 * blk;
+          // columns: [x_ip x_iq] <- [c x_ip - s x_iq, s x_ip + c x_iq]
+          const float t00 = cc[blk] * x[0] - sc[blk] * x[1], t01 = sc[blk] * x[0] + cc[blk] * x[1];
+          const float t10 = cc[blk] * x[2] - sc[blk] * x[3], t11 = sc[blk] * x[2] + cc[blk] * x[3];
+          // rows: [x_pj; x_qj] <- [c x_pj - s x_qj; s x_pj + c x_qj]
+          x[0] = cr * t00 - sr * t10; x[1] = cr * t01 - sr * t11;
+          x[2] = sr * t00 + cr * t10; x[3] = sr * t01 + cr * t11;
+          const float v00 = cc[blk] * y[0] - sc[blk] * y[1], v01 = sc[blk] * y[0] + cc[blk] * y[1];
+          const float v10 = cc[blk] * y[2] - sc[blk] * y[3], v11 = sc[blk] * y[2] + cc[blk] * y[3];
+          y[0] = v00; y[1] = v01; y[2] = v10; y[3] = v11;
+        }
+        // the permutation: A rows and columns, U columns
 #pragma unroll
-      for (int it = 0; it < 4; ++it) {
-        const int item = lane + 32 * it, i = item >> 3, m = item & 7;
-        const float c = rot[m], s = rot[8 + m];
-        const int pi = reinterpret_cast<int *>(rot)[16 + m], qi = reinterpret_cast<int *>(rot)[24 + m];
-        const float api = A[pi * 17 + i], aqi = A[qi * 17 + i];
-        A[pi * 17 + i] = c * api - s * aqi;
-        A[qi * 17 + i] = s * api + c * aqi;
+        for (int e = 0; e < 8; ++e) {
+          const int rb = (e >> 1) & 1, c4 = 2 * (e >> 2) + (e & 1);
+          dst[wr_row[rb] * kJS + wr_col[c4]] = a[e];
+          dst[LOCKS_B * kJS + (2 * m + rb) * kJS + wr_col[c4]] = u[e];
+        }
+        __syncwarp();
+#pragma unroll
+        for (int rb = 0; rb < 2; ++rb) {   // columns 4k .. 4k+3 of a row are one 16-byte read
+          const float4 ra = *reinterpret_cast<const float4 *>(dst + (2 * m + rb) * kJS + 4 * k);
+          const float4 ru = *reinterpret_cast<const float4 *>(dst + LOCKS_B * kJS + (2 * m + rb) * kJS + 4 * k);
+          a[2 * rb] = ra.x; a[2 * rb + 1] = ra.y; a[4 + 2 * rb] = ra.z; a[4 + 2 * rb + 1] = ra.w;
+          u[2 * rb] = ru.x; u[2 * rb + 1] = ru.y; u[4 + 2 * rb] = ru.z; u[4 + 2 * rb + 1] = ru.w;
+        }
+        parity ^= 1;
       }
-      __syncwarp();
     }
+    __syncwarp();
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      const int i = 2 * m + ((e >> 1) & 1), j = 4 * k + 2 * (e >> 2) + (e & 1);
+      A[i * 17 + j] = a[e];
+      U[i * 17 + j] = u[e];
+    }
+    __syncwarp();
   }
   // ---- 4. order the eigenvalues (descending, ties by index), choose r_eff
   float lam = (lane < 16) ? A[lane * 17 + lane] : -INFINITY;

@@ -271,20 +271,31 @@ def test_ties_across_chunks(pages):
 
 
 def test_gpu_i4_build_decoupled_parity():
-    """I4 build: codes agree with the oracle's on >= 99.9 % of entries (|diff| <= 1 elsewhere), the
-    stored scales are the fp16 abs-max scales of the blob's own values, probe scores stay close."""
+    """I4 build: codes agree with the oracle's on >= 99.9 % of entries (|diff| <= 1 elsewhere) after sign
+    alignment, the stored scales are the fp16 abs-max scales of the blob's own values, probe scores stay
+    close.  The sign of a mode (largest-magnitude basis entry positive) is a determinism convention: the score
+    only sees the products of a basis vector with its coefficients, and the rule is decided by a comparison
+    of two magnitudes that fp32 and fp64 can order differently when they are within a code of each other.
+    Such a joint flip of (basis row, coefficient column) is accepted only at a near-tie and must stay rare."""
     gc = _gc(small_bf16([16 * 600], Hq=8, Hkv=2, seed=21))
     w = gc.w
     g_summ = gc.gpu_build().cpu().numpy()
     o_summ = gc.oracle_summaries()
     rng = np.random.default_rng(1)
     bt = gc.cache.block_table[0]
-    tot = diff = 0
+    tot = diff = flips = 0
     worst = 0.0
     for p in range(600):
         for h in range(2):
             gV, gC, gMu, gsV, gsC, gsMu = oracle.unpack_codes(8, g_summ[bt[p], h])
             oV, oC, oMu, osV, osC, osMu = oracle.unpack_codes(8, o_summ[bt[p], h])
+            for l in range(8):
+                if int(np.dot(gV[l], oV[l])) < 0:
+                    top = np.sort(np.abs(oV[l]))[-2:]
+                    assert top[1] - top[0] <= 1, (p, h, l, top)
+                    gV[l] = -gV[l]
+                    gC[:, l] = -gC[:, l]
+                    flips += 1
             for a, b_ in ((gV, oV), (gC, oC), (gMu, oMu)):
                 d = np.abs(a - b_)
                 assert d.max() <= 1
@@ -298,6 +309,7 @@ def test_gpu_i4_build_decoupled_parity():
                 q = rng.standard_normal(128)
                 worst = max(worst, abs(oracle.score(*mg, q, gc.sm) - oracle.score(*mo, q, gc.sm)))
     assert diff / tot <= 1e-3, diff / tot
+    assert flips <= 2, flips   # of 9600 modes
     assert worst <= 5e-3, worst
     assert gc.status() == 0
 
