@@ -214,7 +214,7 @@ int locks_build_summaries(locks_ctx *ctx, const locks_kv *kv, int batch, const i
   if (!summaries || ((uintptr_t)summaries % 16) || ((page_begin == nullptr) != (page_end == nullptr)))
     return LOCKS_ERR_INVALID_ARG;
   ctx->last_launches = 0;
-  return locks_launch_build(ctx, kv, batch, page_begin, page_end, 0, summaries, (cudaStream_t)stream);
+  return locks_launch_build(ctx, kv, batch, page_begin, page_end, 0, summaries, nullptr, nullptr, (cudaStream_t)stream);
 }
 
 int locks_select(locks_ctx *ctx, const void *q, const void *summaries, const locks_kv *kv, int batch,
@@ -278,13 +278,18 @@ int locks_decode_step(locks_ctx *ctx, const void *q, const void *k_new, const vo
   mark(0);
   if ((rc = locks_launch_scan(ctx, q, summaries, kv, batch, ctx->shat, k_new ? 1 : 0, st)) != LOCKS_OK) return rc;
   mark(1);
-  if ((rc = locks_launch_select(ctx, ctx->shat, &kv_step, batch, ids, cnt, nullptr, k_new ? &app : nullptr, st)) != LOCKS_OK)
-    return rc;
-  // the freshly completed page (if any) is summarised beside attention, which does not read its summary
+  // The page that this step's token completes (if any) is summarised on a second stream beside the selector
+  // and attention: its summary is first read by the next step's scan.  The build starts when the scan has
+  // published the lengths; the token itself it takes from k_new, since the selector's kernel is writing it
+  // into the cache at the same time.
   if (cudaEventRecord(ctx->ev_fork, st) != cudaSuccess || cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0) != cudaSuccess)
     return LOCKS_ERR_CUDA;
-  if ((rc = locks_launch_build(ctx, &kv_step, batch, nullptr, nullptr, 1, summaries, ctx->side)) != LOCKS_OK) return rc;
+  if ((rc = locks_launch_build(ctx, &kv_step, batch, nullptr, nullptr, 1, summaries, k_new,
+                               k_new ? ctx->seq_eff + batch : nullptr, ctx->side)) != LOCKS_OK)
+    return rc;
   if (cudaEventRecord(ctx->ev_join, ctx->side) != cudaSuccess) return LOCKS_ERR_CUDA;
+  if ((rc = locks_launch_select(ctx, ctx->shat, &kv_step, batch, ids, cnt, nullptr, k_new ? &app : nullptr, st)) != LOCKS_OK)
+    return rc;
   mark(2);
   if ((rc = locks_launch_attend(ctx, q, &kv_step, batch, ids, cnt, out, nullptr, st)) != LOCKS_OK) return rc;
   mark(3);

@@ -25,6 +25,10 @@ struct BuildParams {
   // decode step only: where to leave the scan-partition suggestion for these lengths, and the scan's geometry
   int32_t *hint;
   int kpages, hint_wpp, hint_rounds, hint_W;
+  // decode step only: the token appended by this step is read from the caller's buffer, not from the cache
+  // (the append runs in another kernel at the same time); append_pos[b] = its position or -1
+  const void *k_new;
+  const int32_t *append_pos;
 };
 
 constexpr int kBuildWarps = 4;
@@ -42,6 +46,7 @@ __global__ void __launch_bounds__(kBuildWarps * 32) build_kernel(BuildParams p) 
   extern __shared__ __align__(16) uint8_t smem_raw[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   int b, h, page;
+  bool last_from_new = false;   // row 15 of the page is this step's token
   if (p.just_filled && p.hint && blockIdx.x == 0 && warp == 0)
     locks_update_partition_hint(p.hint, p.seq_lens, p.batch, p.Hkv, p.kpages, p.hint_wpp, p.hint_rounds, p.hint_W, lane);
   if (p.just_filled) {
@@ -51,6 +56,7 @@ __global__ void __launch_bounds__(kBuildWarps * 32) build_kernel(BuildParams p) 
     const int Tb = p.seq_lens[b];
     if (Tb <= 0 || (Tb % LOCKS_B) != 0) return;
     page = Tb / LOCKS_B - 1;
+    last_from_new = p.k_new && p.append_pos && p.append_pos[b] == Tb - 1;
   } else {
     b = blockIdx.z; h = blockIdx.y;
     const int complete = p.seq_lens[b] / LOCKS_B;
@@ -74,13 +80,14 @@ __global__ void __launch_bounds__(kBuildWarps * 32) build_kernel(BuildParams p) 
 
   // ---- 1. load, centre
   const T *K = reinterpret_cast<const T *>(p.k) + (int64_t)block * p.sb + (int64_t)h * p.sh;
+  const T *Knew = reinterpret_cast<const T *>(p.k_new) + ((int64_t)b * p.Hkv + h) * LOCKS_D;
   float kv[LOCKS_B][4], mu[4] = {0.f, 0.f, 0.f, 0.f};
   float knorm2 = 0.f;
 #pragma unroll
   for (int i = 0; i < LOCKS_B; ++i) {
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
-      kv[i][u] = ldf<T>(K, (int64_t)i * p.st + lane * 4 + u);
+      kv[i][u] = (i == LOCKS_B - 1 && last_from_new) ? ldf<T>(Knew, lane * 4 + u) : ldf<T>(K, (int64_t)i * p.st + lane * 4 + u);
       mu[u] += kv[i][u];
       knorm2 += kv[i][u] * kv[i][u];
     }
@@ -333,13 +340,15 @@ __global__ void __launch_bounds__(kBuildWarps * 32) build_kernel(BuildParams p) 
 }  // namespace
 
 int locks_launch_build(locks_ctx *c, const locks_kv *kv, int batch, const int32_t *pb, const int32_t *pe,
-                       int just_filled, void *summaries, cudaStream_t st) {
+                       int just_filled, void *summaries, const void *k_new, const int32_t *append_pos,
+                       cudaStream_t st) {
   BuildParams p;
   p.k = kv->k; p.sb = kv->stride_block; p.sh = kv->stride_head; p.st = kv->stride_token;
   p.block_table = kv->block_table; p.seq_lens = kv->seq_lens; p.page_begin = pb; p.page_end = pe;
   p.summ = reinterpret_cast<uint8_t *>(summaries); p.status = c->status;
   p.batch = batch; p.Hkv = c->cfg.num_kv_heads; p.Pmax = c->Pmax; p.num_blocks = kv->num_blocks;
   p.r = c->cfg.rank; p.S = c->S; p.just_filled = just_filled;
+  p.k_new = just_filled ? k_new : nullptr; p.append_pos = just_filled ? append_pos : nullptr;
   p.hint = nullptr; p.kpages = c->k; p.hint_wpp = 1; p.hint_rounds = 1; p.hint_W = 1;
   if (just_filled && c->hint_dev && c->cfg.summary_fmt == LOCKS_FMT_I4 && c->cfg.q_dtype == LOCKS_BF16) {
     const locks_scan_geom geo = locks_scan_geometry(c, batch);

@@ -144,7 +144,8 @@ int locks_launch_select(locks_ctx *c, const float *shat, const locks_kv *kv, int
 int locks_launch_attend(locks_ctx *c, const void *q, const locks_kv *kv, int batch, const int32_t *ids,
                         const int32_t *cnt, void *out, float *lse, cudaStream_t st);
 int locks_launch_build(locks_ctx *c, const locks_kv *kv, int batch, const int32_t *pb, const int32_t *pe,
-                       int just_filled, void *summaries, cudaStream_t st);
+                       int just_filled, void *summaries, const void *k_new, const int32_t *append_pos,
+                       cudaStream_t st);
 
 // Launch with programmatic dependent launch allowed: the kernel may be scheduled while its stream
 // predecessor is still draining; it must execute pdl_wait() before touching anything the predecessor
