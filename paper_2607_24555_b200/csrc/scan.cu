@@ -39,7 +39,7 @@ struct ScanParams {
   // write (seq_inc = 1); the first CTA publishes them, and the append position, for the step's later kernels
   int cta_reduce;     // every warp of a CTA works on one problem only: one partial per (head, CTA)
   int wpp, nslots;    // strided partition: warps per problem, problems in flight
-  int use_gather;     // rank 8: stage four summaries per tensor-map gather instead of one bulk copy each
+  int use_gather;     // stage four summaries per tensor-map gather instead of one bulk copy each
   int seq_inc;
   int32_t *seq_eff;   // [2][max_batch]: effective length, append position (-1: none) -- or nullptr
 };
@@ -258,6 +258,10 @@ __device__ __forceinline__ uint32_t movm_trans(uint32_t v) {
 template <int R, int NH, bool PK, bool CR, bool BAL>
 __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4_kernel(ScanParams p, const __grid_constant__ CUtensorMap tmap) {
   constexpr int kBlob = i4_stride(R);   // stored bytes of one summary; a stage keeps room for rank-8 blobs
+  // Summaries 4-7 of a stage start on a 128-byte boundary (the destination of the second tensor-map gather):
+  // 4 x 832 bytes already is one, 4 x 336 and 4 x 496 need 64 bytes of padding
+  constexpr int kHalfPad = (4 * kBlob) % 128 ? 128 - (4 * kBlob) % 128 : 0;
+  auto boff = [](int pg) { return pg * kBlob + (kHalfPad ? (pg >> 2) * kHalfPad : 0); };   // offset of summary pg in a stage
   extern __shared__ __align__(128) uint8_t smem[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int x = lane >> 2, t = lane & 3;
@@ -386,8 +390,8 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4_kerne
       set_status(p.status, LOCKS_ERR_BAD_BLOCK);
       block = 0;
     }
-    if (R == 8 && p.use_gather) {
-      // Summaries are rows of a 2D tensor [block * Hkv + head][832 B]: one gather fetches four of them, so a
+    if (p.use_gather) {
+      // Summaries are rows of a 2D tensor [block * Hkv + head][S bytes]: one gather fetches four of them, so a
       // group costs two copy instructions instead of eight (about 3 of 115 instructions per summary; the
       // staging throughput itself does not change).  Slots past the last page repeat the group's first row.
       int row = block * p.Hkv + h;
@@ -400,17 +404,17 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4_kerne
         uint8_t *dst = ring + stage * kStageBytes;
         mbar_expect_tx(&full[stage], (uint32_t)(nvalid > 4 ? 8 : 4) * kBlob);
         tma_gather4(dst, &tmap, row, r1, r2, r3, &full[stage], pol_stream);
-        if (nvalid > 4) tma_gather4(dst + 4 * kBlob, &tmap, r4, r5, r6, r7, &full[stage], pol_stream);
+        if (nvalid > 4) tma_gather4(dst + boff(4), &tmap, r4, r5, r6, r7, &full[stage], pol_stream);
       }
     } else if (kScanBulk) {
       if (lane == 0) mbar_expect_tx(&full[stage], (uint32_t)nvalid * kBlob);
       __syncwarp();
       if (lane < nvalid) {
         if (LOCKS_SCAN_HINT_LOAD)
-          bulk_g2s_hint(ring + stage * kStageBytes + lane * kBlob, p.summ + ((int64_t)block * p.Hkv + h) * kBlob, kBlob,
+          bulk_g2s_hint(ring + stage * kStageBytes + boff(lane), p.summ + ((int64_t)block * p.Hkv + h) * kBlob, kBlob,
                         &full[stage], pol_stream);
         else
-          bulk_g2s(ring + stage * kStageBytes + lane * kBlob, p.summ + ((int64_t)block * p.Hkv + h) * kBlob, kBlob,
+          bulk_g2s(ring + stage * kStageBytes + boff(lane), p.summ + ((int64_t)block * p.Hkv + h) * kBlob, kBlob,
                    &full[stage]);
       }
     } else {
@@ -421,7 +425,7 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4_kerne
         const int blk = __shfl_sync(0xffffffffu, block, pg);
         const uint8_t *src = p.summ + ((int64_t)blk * p.Hkv + h) * kBlob;
         if (pg < nvalid)
-          for (int c = lane; c < kBlob / 16; c += 32) cp_async16(dst + pg * kBlob + c * 16, src + c * 16, true);
+          for (int c = lane; c < kBlob / 16; c += 32) cp_async16(dst + boff(pg) + c * 16, src + c * 16, true);
       }
       cp_async_commit();
     }
@@ -578,7 +582,7 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4_kerne
 #pragma unroll
     for (int hh = 0; hh < NH; ++hh) cenT[hh][0] = cenT[hh][1] = cenT[hh][2] = cenT[hh][3] = 0.f;
     {
-      const uint4 *mp = reinterpret_cast<const uint4 *>(sb + (x & (LOCKS_GROUP - 1)) * kBlob + i4_off_mu(R) + t * 32);
+      const uint4 *mp = reinterpret_cast<const uint4 *>(sb + boff(x & (LOCKS_GROUP - 1)) + i4_off_mu(R) + t * 32);
       const uint4 m0 = mp[0], m1 = mp[1];
       const uint32_t mw[8] = {m0.x, m0.y, m0.z, m0.w, m1.x, m1.y, m1.z, m1.w};
 #pragma unroll
@@ -593,7 +597,7 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4_kerne
     // scaled at the lane that holds them (page x, heads 2t, 2t+1), then moved to the lanes that finish the pages
     float acen[2 * NH];  // log2-domain centroid term: packed, of this lane's (page, head); else of pages 2t, 2t+1 for head x (+8)
     {
-      const float smu = __half2float(*reinterpret_cast<const __half *>(sb + (x & (LOCKS_GROUP - 1)) * kBlob + i4_off_smu(R)));
+      const float smu = __half2float(*reinterpret_cast<const __half *>(sb + boff(x & (LOCKS_GROUP - 1)) + i4_off_smu(R)));
 #pragma unroll
       for (int hh = 0; hh < NH; ++hh) {
         const float v0 = smu * (c2 * inv2[2 * hh]) * cenT[hh][0], v1 = smu * (c2 * inv2[2 * hh + 1]) * cenT[hh][1];
@@ -632,8 +636,8 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4_kerne
         float prj[2][2];                        // rank 2: [k4 half][head e]; rank 4: [half of this chain][head e]
         if (R == 4 || k4 == 0) {
           const int pa0 = (R == 4 ? 4 * k4 : 0) + pr, pb0 = pa0 + PH;
-          const uint4 wa4 = *reinterpret_cast<const uint4 *>(sb + pa0 * kBlob + (lr * 4 + t) * 16);
-          const uint4 wb4 = *reinterpret_cast<const uint4 *>(sb + pb0 * kBlob + (lr * 4 + t) * 16);
+          const uint4 wa4 = *reinterpret_cast<const uint4 *>(sb + boff(pa0) + (lr * 4 + t) * 16);
+          const uint4 wb4 = *reinterpret_cast<const uint4 *>(sb + boff(pb0) + (lr * 4 + t) * 16);
           const uint32_t wa[4] = {wa4.x, wa4.y, wa4.z, wa4.w}, wb[4] = {wb4.x, wb4.y, wb4.z, wb4.w};
           float c1[4];
 #pragma unroll
@@ -643,8 +647,8 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4_kerne
             else mma_f16(c1, ua & kM0, ub & kM0, ua & kM1, ub & kM1, qb0[0][2 * j], qb2[0][2 * j]);
             mma_f16(c1, ua8 & kM0, ub8 & kM0, ua8 & kM1, ub8 & kM1, qb0[0][2 * j + 1], qb2[0][2 * j + 1]);
           }
-          const float svA = __half2float(*reinterpret_cast<const __half *>(sb + pa0 * kBlob + i4_off_sv(R) + 2 * lr));
-          const float svB = __half2float(*reinterpret_cast<const __half *>(sb + pb0 * kBlob + i4_off_sv(R) + 2 * lr));
+          const float svA = __half2float(*reinterpret_cast<const __half *>(sb + boff(pa0) + i4_off_sv(R) + 2 * lr));
+          const float svB = __half2float(*reinterpret_cast<const __half *>(sb + boff(pb0) + i4_off_sv(R) + 2 * lr));
           prj2[0][0] = fmaf(c1[0], 16777216.f, -ksum[0]) * svA;
           prj2[0][1] = fmaf(c1[1], 16777216.f, -ksum[1]) * svA;
           prj2[1][0] = fmaf(c1[2], 16777216.f, -ksum[0]) * svB;
@@ -666,7 +670,7 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4_kerne
           if (!mine) { hi = 0u; lo = 0u; }
           a0h = t < 2 ? hi : 0u; a1h = t < 2 ? 0u : hi; a2h = t < 2 ? lo : 0u; a3h = t < 2 ? 0u : lo;
           // coefficients of page t, token x (and x + 8), ranks 0 and 1; the lo part meets the same values
-          const uint32_t cw = *reinterpret_cast<const uint32_t *>(sb + (4 * k4 + t) * kBlob + i4_off_coef(R) + x * 4);
+          const uint32_t cw = *reinterpret_cast<const uint32_t *>(sb + boff(4 * k4 + t) + i4_off_coef(R) + x * 4);
           bt0a = bt0b = f16x2_sub(__byte_perm(cw, 0x64646464u, 0x4140), kSub128);
           bt8a = bt8b = f16x2_sub(__byte_perm(cw, 0x64646464u, 0x4342), kSub128);
         } else {
@@ -689,8 +693,8 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4_kerne
           a0h = hi0; a1h = 0u; a2h = 0u; a3h = hi1;
           a0l = lo0; a3l = lo1;
           const int wofs = i4_off_coef(R) + (x * 2 + (t & 1)) * 4;   // token x (and x + 8), rank pair t & 1
-          const uint32_t cw0 = *reinterpret_cast<const uint32_t *>(sb + (4 * k4 + (t >> 1)) * kBlob + wofs);
-          const uint32_t cw1 = *reinterpret_cast<const uint32_t *>(sb + (4 * k4 + 2 + (t >> 1)) * kBlob + wofs);
+          const uint32_t cw0 = *reinterpret_cast<const uint32_t *>(sb + boff(4 * k4 + (t >> 1)) + wofs);
+          const uint32_t cw1 = *reinterpret_cast<const uint32_t *>(sb + boff(4 * k4 + 2 + (t >> 1)) + wofs);
           bt0a = f16x2_sub(__byte_perm(cw0, 0x64646464u, 0x4140), kSub128);
           bt0b = f16x2_sub(__byte_perm(cw1, 0x64646464u, 0x4140), kSub128);
           bt8a = f16x2_sub(__byte_perm(cw0, 0x64646464u, 0x4342), kSub128);
@@ -706,7 +710,7 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4_kerne
 #pragma unroll
         for (int hrow = 0; hrow < 2; ++hrow) {   // row x -> page 4 k4 + (x >> 2), row x + 8 -> two pages further
           const int pg = 4 * k4 + 2 * hrow + (x >> 2);
-          const uint2 scw = *reinterpret_cast<const uint2 *>(sb + pg * kBlob + i4_off_sc(R) + 8 * t);
+          const uint2 scw = *reinterpret_cast<const uint2 *>(sb + boff(pg) + i4_off_sc(R) + 8 * t);
           const float2 s01 = h2f2(scw.x), s89 = h2f2(scw.y);
           const float y0 = ca[2 * hrow] * s01.x, y1 = ca[2 * hrow + 1] * s01.y;
           const float y2 = cb[2 * hrow] * s89.x, y3 = cb[2 * hrow + 1] * s89.y;
@@ -725,7 +729,7 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4_kerne
     } else {
 #pragma unroll
     for (int pp = 0; pp < LOCKS_GROUP / 2; ++pp) {
-      const uint8_t *pbA = sb + (2 * pp) * kBlob, *pbB = pbA + kBlob;
+      const uint8_t *pbA = sb + boff(2 * pp), *pbB = pbA + kBlob;
       // ---- MMA #1: rows = (page A ranks 0-7, page B ranks 0-7), cols = heads, k = this lane quarter's dims
       // lane (x, t) holds rank x, dim quarter t; ranks >= R do not exist (their column scale reads as 0 below)
       const uint4 wa4 = (R == 8 || x < R) ? *reinterpret_cast<const uint4 *>(pbA + lane * 16) : make_uint4(0u, 0u, 0u, 0u);
@@ -947,11 +951,11 @@ int locks_launch_scan(locks_ctx *c, const void *q, const void *summaries, const 
     c->part_balanced = balanced ? 1 : 0;
     const dim3 g(grid), blk(kScanWarps * 32);
     const int gsel = c->G <= 4 ? 0 : (c->G <= 8 ? 1 : 2);
-    // tensor map over the summaries for the gather path (rank 8): rows = (block, KV head), 208 32-bit words each
+    // tensor map over the summaries for the gather path: rows = (block, KV head), S / 4 32-bit words each
     alignas(64) CUtensorMap tmap;
     memset(&tmap, 0, sizeof(tmap));
     p.use_gather = 0;
-    if (c->cfg.rank == 8 && LOCKS_SCAN_GATHER) {
+    if (LOCKS_SCAN_GATHER) {
       static PFN_cuTensorMapEncodeTiled encode = nullptr;
       static bool looked = false;
       if (!looked) {
@@ -964,9 +968,10 @@ int locks_launch_scan(locks_ctx *c, const void *q, const void *summaries, const 
         (void)cudaGetLastError();
       }
       if (encode) {
-        const cuuint64_t gdim[2] = {(cuuint64_t)(i4_stride(8) / 4), (cuuint64_t)kv->num_blocks * p.Hkv};
-        const cuuint64_t gstride[1] = {(cuuint64_t)i4_stride(8)};
-        const cuuint32_t box[2] = {(cuuint32_t)(i4_stride(8) / 4), 1u};
+        const int S = i4_stride(c->cfg.rank);
+        const cuuint64_t gdim[2] = {(cuuint64_t)(S / 4), (cuuint64_t)kv->num_blocks * p.Hkv};
+        const cuuint64_t gstride[1] = {(cuuint64_t)S};
+        const cuuint32_t box[2] = {(cuuint32_t)(S / 4), 1u};
         const cuuint32_t estride[2] = {1u, 1u};
         if (encode(&tmap, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<void *>(summaries), gdim, gstride, box, estride,
                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
