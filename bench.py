@@ -49,6 +49,9 @@ def workload(name: str):
         return locks_synth.config2(rank=int(r[1:]), budget=int(b[1:]))
     if name == "cfg3_512k":
         return locks_synth.config3(T=1 << 19)
+    if name.startswith("cfg3g8_"):        # the paper's stated GLM geometry: 4 KV heads, G = 8
+        T = {"128k": 1 << 17, "512k": 1 << 19, "1m": 1 << 20}[name[7:]]
+        return locks_synth.config3(T=T, Hkv=4)
     if name.startswith("cfg4_b"):
         return locks_synth.config4(batch=int(name[6:]))
     if name == "small":
