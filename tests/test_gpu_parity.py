@@ -477,6 +477,42 @@ def test_decode_step_host_repeated_calls_match_device_steps():
     assert gc_h.status() == 0 and gc_d.status() == 0
 
 
+def test_decode_step_host_pageable_buffers_take_the_copy_path():
+    """Host buffers that are not page-locked cannot be read by the staging kernel or written by the attention
+    kernel: the call falls back to plain copies and returns the same results as with page-locked buffers."""
+    w = small_bf16([16 * 40 + 5, 300], Hq=8, Hkv=2, budget=128, seed=58)
+    w = w.with_(seq_lens=[t + 32 for t in w.seq_lens])
+    res = []
+    for pinned in (True, False):
+        gc = _gc(w)
+        gc.case.seq_lens.copy_(torch.tensor([t - 32 for t in w.seq_lens], dtype=torch.int32, device="cuda:0"))
+        summ = gc.ctx.new_summaries(gc.case.num_blocks)
+        gc.ctx.locks_build_summaries(gc.kv, w.n, summ)
+        mk = (lambda t: t.pin_memory()) if pinned else (lambda t: t)
+        out_host = mk(torch.empty(w.n, w.Hq, w.d, dtype=torch.bfloat16))
+        ids_host = mk(torch.empty(w.n, w.Hkv, gc.k, dtype=torch.int32))
+        cnt_host = mk(torch.empty(w.n, w.Hkv, dtype=torch.int32))
+        got = []
+        for step in range(4):
+            kn, vn, qn = locks_synth.new_token(w, step, device="cuda:0")
+            gc.ctx.locks_decode_step_host(mk(qn.cpu()), mk(kn.cpu()), mk(vn.cpu()), gc.kv, summ, w.n, out_host, ids_host,
+                                          cnt_host)
+            got.append((out_host.clone(), ids_host.clone(), cnt_host.clone()))
+        assert gc.status() == 0
+        res.append(got)
+    for (o1, i1, c1), (o2, i2, c2) in zip(*res):
+        assert torch.equal(o1, o2) and torch.equal(i1, i2) and torch.equal(c1, c2)
+
+
+def test_scan_partition_setter_rejects_unknown_modes():
+    gc = _gc(small_bf16([16 * 20], Hq=8, Hkv=2, budget=128))
+    for mode in (locks.PARTITION_AUTO, locks.PARTITION_STRIDED, locks.PARTITION_BALANCED):
+        gc.ctx.locks_set_scan_partition(mode)
+    for mode in (-1, 3):
+        with pytest.raises(locks.LocksError):
+            gc.ctx.locks_set_scan_partition(mode)
+
+
 def test_bad_block_id_sets_status_without_faulting():
     """Host-injected fault: a block id outside the cache is skipped and reported, nothing traps."""
     gc = _gc(small_bf16([16 * 60], Hq=8, Hkv=2, budget=128, seed=66))
