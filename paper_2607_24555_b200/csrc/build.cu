@@ -4,7 +4,8 @@
 //   1. load the page's 16 keys (lane owns 4 consecutive dims of every key), centroid mu, deviations D
 //   2. Gram M = D D^T (16 x 16) from shared memory
 //   3. eigendecomposition of M by parallel-ordered cyclic Jacobi in fp32 (8 disjoint rotations per
-//      round, 15 rounds per sweep, round-robin pairing), eigenvectors accumulated in U
+//      round, 15 rounds per sweep, round-robin pairing), eigenvectors accumulated in U; both matrices
+//      live in registers, one shared-memory exchange per round
 //   4. rank by eigenvalue, keep r_eff <= min(r, 15) modes above the zero-mode thresholds
 //   5. V = D^T U_r Sigma_r^-1 (lane's 4 dims), C = U_r Sigma_r, sign: largest |V| entry positive
 //   6. store fp32 (F32 format) or quantise: symmetric abs-max, fp16 scale, round-half-even codes

@@ -18,7 +18,7 @@
 #define LOCKS_ATT_MAX_SPLITS 128
 #define LOCKS_ATT_SLOT_BOUND 1024 // upper bound on resident attend CTAs of any supported GPU (148 SMs x 4 on B200)
 #ifndef LOCKS_SCAN_GATHER
-#define LOCKS_SCAN_GATHER 1    // rank-8 scan: stage summaries four at a time with tensor-map gathers
+#define LOCKS_SCAN_GATHER 1    // tensor scan: stage summaries four at a time with tensor-map gathers
 #endif
 #ifndef LOCKS_SCAN_BALANCED
 #define LOCKS_SCAN_BALANCED 1  // tensor scan: deal (problem, group) units to the warps by actual lengths (0: equal warps per problem)
