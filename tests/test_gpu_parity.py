@@ -149,8 +149,8 @@ def test_i4_rank2_group_sizes(Hq, Hkv):
 @pytest.mark.parametrize("trial", range(24))
 def test_randomized_shapes(trial):
     """Seeded random shapes: group size, rank, budget, request count, lengths (with ragged tails and requests
-    shorter than the budget), block layout, carriers.  Twice per case: the second call must reproduce the
-    first (no state left behind in the workspace)."""
+    shorter than the budget), block layout, carriers, scan partition.  Twice per case: the second call must
+    reproduce the first (no state left behind in the workspace)."""
     from gpu_util import check_select_and_attend
     rng = np.random.default_rng(1000 + trial)
     Hkv = int(rng.choice([1, 2, 4]))
@@ -165,6 +165,8 @@ def test_randomized_shapes(trial):
                    layout="NHD" if trial % 4 == 1 else "HND", carriers=int(rng.choice([0, 0, 4])),
                    q_scale=float(rng.choice([1.0, 0.25])))
     gc = _gc(w)
+    if trial % 2:   # odd trials force the scan's balanced page partition (even ones: strided, the default here)
+        gc.ctx.locks_set_scan_partition(locks.PARTITION_BALANCED)
     summ = gc.oracle_summaries()
     check_select_and_attend(gc, summ, out_tol=2e-2)
     ids1, cnt1, lm1, ls1 = gc.gpu_select(torch.from_numpy(summ).cuda())
