@@ -42,21 +42,34 @@ Layout make_layout(const locks_config *c) {
   L.S = c->summary_fmt == LOCKS_FMT_I4 ? i4_stride(c->rank) : f32_stride(c->rank);
   L.max_groups = (c->max_pages_per_seq + LOCKS_GROUP - 1) / LOCKS_GROUP;
   // Pages per thread of a selector CTA (1 .. 16; a CTA ranks sel_ept * 512 pages).  With many (request,
-  // KV head) problems one CTA per problem already fills the GPU, so a context of up to 8192 pages is ranked
-  // in one chunk.  With few problems the smallest chunk whose candidate lists still fit the final round
-  // is taken: the selector is a chain of memory round trips, so many small CTAs finish sooner.
+  // KV head) problems and a context of up to 8192 pages, one CTA ranks a whole problem.  Otherwise a problem is
+  // cut into chunks whose top-(k-2) lists are ranked by the chunk that arrives last, and the chunk size is the
+  // one a small cost model likes best (microseconds, fitted to measurements on B200 at 2 .. 256 problems,
+  // G = 4 .. 16, 8K .. 64K pages): a CTA's chain of round trips costs about 6 plus 1.2 per batch of 16 score
+  // loads per thread beyond the first one and a half, plus 0.15 per 512 pages; the CTAs of a launch run in
+  // waves of one per SM; the final ranking costs 3.3 plus 0.43 per 512 candidates.
   const int per_thread = (c->max_pages_per_seq + LOCKS_SEL_THREADS - 1) / LOCKS_SEL_THREADS;
-  const bool many_problems = (int64_t)c->max_batch * c->num_kv_heads >= 32;
+  const int64_t problems = (int64_t)c->max_batch * c->num_kv_heads;
+  const int kcand = L.k - 2 > 0 ? L.k - 2 : 1;
   L.sel_ept = LOCKS_SEL_MAX_EPT;
-  if (many_problems && per_thread <= LOCKS_SEL_MAX_EPT) {
+  if (problems >= 32 && per_thread <= LOCKS_SEL_MAX_EPT) {
     L.sel_ept = per_thread;
   } else {
+    constexpr int kSms = 148;   // the model's machine; the layout must not depend on the device at hand
+    double best = 1e30;
     for (int ept = 1; ept <= LOCKS_SEL_MAX_EPT; ept *= 2) {
       const int chunks = (c->max_pages_per_seq + ept * LOCKS_SEL_THREADS - 1) / (ept * LOCKS_SEL_THREADS);
-      if (chunks == 1 || (size_t)chunks * (L.k - 2 > 0 ? L.k - 2 : 1) <= (size_t)LOCKS_SEL_MAX_EPT * LOCKS_SEL_THREADS) {
+      if (chunks > 1 && (size_t)chunks * kcand > (size_t)LOCKS_SEL_MAX_EPT * LOCKS_SEL_THREADS) continue;
+      const double batches = (double)ept * L.G / 16.0;
+      const double cta = 6.0 + 1.2 * (batches > 1.5 ? batches - 1.5 : 0.0) + 0.15 * ept;
+      const double waves = (double)((problems * chunks + kSms - 1) / kSms);
+      const double fin = chunks == 1 ? 0.0 : 3.3 + 0.43 * (double)chunks * kcand / LOCKS_SEL_THREADS;
+      const double est = waves * cta + fin;
+      if (est < best) {
+        best = est;
         L.sel_ept = ept;
-        break;
       }
+      if (chunks == 1) break;
     }
   }
   L.sel_chunks = (c->max_pages_per_seq + L.sel_ept * LOCKS_SEL_THREADS - 1) / (L.sel_ept * LOCKS_SEL_THREADS);
