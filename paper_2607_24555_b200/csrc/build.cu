@@ -147,6 +147,24 @@ __global__ void __launch_bounds__(kBuildWarps * 32) build_kernel(BuildParams p) 
     const int dblk = m & 1;             // which of the two blocks is the diagonal one (diag lanes)
     const int src_row = m * 4 + (m >> 1);           // lane holding the diagonal block of row pair m
     const int src_c0 = 9 * k, src_c1 = 9 * k + 4;   // ... of column pairs 2k and 2k + 1
+    // The rotations square matrix entries: bring the matrix to unit scale first (an exact power of two, taken
+    // from its largest entry and undone on the eigenvalues), so that keys of any magnitude are handled alike.
+    float unscale = 1.f;
+    {
+      float amax = 0.f;
+#pragma unroll
+      for (int e = 0; e < 8; ++e) amax = fmaxf(amax, fabsf(a[e]));
+      amax = warp_max(amax);
+      if (amax > 0.f && amax < INFINITY) {
+        int ex;
+        (void)frexpf(amax, &ex);
+        ex = max(-120, min(120, ex));
+        const float sc = ldexpf(1.f, -ex);
+        unscale = ldexpf(1.f, ex);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) a[e] *= sc;
+      }
+    }
     float normA = 0.f;
 #pragma unroll
     for (int e = 0; e < 8; ++e) normA += a[e] * a[e];
@@ -216,7 +234,7 @@ __global__ void __launch_bounds__(kBuildWarps * 32) build_kernel(BuildParams p) 
 #pragma unroll
     for (int e = 0; e < 8; ++e) {
       const int i = 2 * m + ((e >> 1) & 1), j = 4 * k + 2 * (e >> 2) + (e & 1);
-      A[i * 17 + j] = a[e];
+      A[i * 17 + j] = a[e] * unscale;
       U[i * 17 + j] = u[e];
     }
     __syncwarp();

@@ -75,6 +75,27 @@ def test_f32_build_matches_oracle_scores():
     assert gc.status() == 0
 
 
+@pytest.mark.parametrize("log2_scale", [-40, 30])
+def test_f32_build_is_invariant_to_the_scale_of_the_keys(log2_scale):
+    """Keys multiplied by a power of two give the same basis, and centroid and coefficients multiplied by it
+    (every step of the build is homogeneous in the keys; a power of two is exact in fp32): the eigen-solver
+    must not depend on the magnitude of the Gram matrix (2^60 times larger or 2^80 times smaller here)."""
+    s = float(2.0 ** log2_scale)
+    w = locks_synth.config0().with_(seq_lens=[16 * 40])
+    ga, gb = _gc(w), _gc(w)
+    gb.case.k.mul_(s)
+    sa = ga.gpu_build().cpu().numpy()
+    sb = gb.gpu_build().cpu().numpy()
+    bt = ga.cache.block_table[0]
+    for p in range(40):
+        mu_a, V_a, C_a = oracle.unpack(oracle.FMT_F32, w.rank, sa[bt[p], 0])
+        mu_b, V_b, C_b = oracle.unpack(oracle.FMT_F32, w.rank, sb[bt[p], 0])
+        assert np.array_equal(mu_b, mu_a * s)
+        assert np.abs(V_b - V_a).max() < 1e-5
+        assert np.abs(C_b / s - C_a).max() < 1e-5 * max(1.0, np.abs(C_a).max())
+    assert ga.status() == 0 and gb.status() == 0
+
+
 def test_full_rank_gpu_summary_is_exact():
     """r = B = 16 in the F32 format reproduces the exact page log-mass (Prop. 3)."""
     gc = _gc(locks_synth.config0().with_(rank=16, seq_lens=[800], n_dirs=0, carriers=0))
