@@ -267,6 +267,16 @@ def test_two_level_select_long_context():
     assert differed <= 1
 
 
+@pytest.mark.parametrize("lens,Hq,Hkv,rank,budget", [([16 * 3000 + 3, 16 * 700], 8, 2, 8, 4096),
+                                                     ([16 * 9000], 32, 2, 8, 8192),
+                                                     ([16 * 2000, 16 * 2500 + 9, 900], 16, 4, 2, 16384)])
+def test_large_budgets(lens, Hq, Hkv, rank, budget):
+    """Budgets of 256 to 1024 pages: long candidate lists per chunk, many winners to compact, long attention."""
+    from gpu_util import check_select_and_attend
+    gc = _gc(locks_synth.Workload("big-budget", lens, Hq=Hq, Hkv=Hkv, rank=rank, budget=budget, seed=5))
+    check_select_and_attend(gc, gc.oracle_summaries(), out_tol=2e-2)
+
+
 def test_ties_resolve_to_lower_index():
     """All keys identical and a zero query: every candidate ties, the lowest indices win."""
     gc = _gc(small_bf16([16 * 40], Hq=4, Hkv=1, budget=128))
