@@ -947,7 +947,13 @@ int locks_launch_scan(locks_ctx *c, const void *q, const void *summaries, const 
     if (mode == LOCKS_PARTITION_AUTO)
       mode = (c->hint_host && *reinterpret_cast<volatile int32_t *>(c->hint_host) == LOCKS_PARTITION_BALANCED)
                  ? LOCKS_PARTITION_BALANCED : LOCKS_PARTITION_STRIDED;
-    const bool balanced = LOCKS_SCAN_BALANCED && !geo.cta_reduce && mode == LOCKS_PARTITION_BALANCED;
+    // the balanced partition also replaces the CTA-level merge of the few-problem geometry when it is asked for:
+    // a few requests of very different lengths would otherwise leave most of the GPU waiting for the longest
+    const bool balanced = LOCKS_SCAN_BALANCED && mode == LOCKS_PARTITION_BALANCED;
+    if (balanced) {
+      p.cta_reduce = 0;
+      c->part_slots = geo.wpp;
+    }
     c->part_balanced = balanced ? 1 : 0;
     const dim3 g(grid), blk(kScanWarps * 32);
     const int gsel = c->G <= 4 ? 0 : (c->G <= 8 ? 1 : 2);

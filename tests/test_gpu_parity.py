@@ -222,6 +222,16 @@ def test_balanced_partition_ragged_batch(Hq, Hkv, rank):
     assert gc.status() == 0
 
 
+def test_balanced_partition_few_problems_of_very_different_lengths():
+    """Two requests, two KV heads, G = 16 (the geometry that otherwise merges partials per CTA), one request
+    40 times longer than the other: hundreds of log Z partials per head in the balanced partition."""
+    from gpu_util import check_select_and_attend
+    w = locks_synth.Workload("few-ragged", [16 * 6000 + 7, 16 * 150], Hq=32, Hkv=2, budget=512, seed=83)
+    gc = _gc(w)
+    gc.ctx.locks_set_scan_partition(locks.PARTITION_BALANCED)
+    check_select_and_attend(gc, gc.oracle_summaries(), out_tol=2e-2)
+
+
 def test_balanced_partition_more_problems_than_warps_per_problem():
     """Balanced partition with many short problems: most warps cross several problem boundaries."""
     from gpu_util import check_select_and_attend
