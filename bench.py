@@ -52,6 +52,8 @@ def workload(name: str):
     if name.startswith("cfg3g8_"):        # the paper's stated GLM geometry: 4 KV heads, G = 8
         T = {"128k": 1 << 17, "512k": 1 << 19, "1m": 1 << 20}[name[7:]]
         return locks_synth.config3(T=T, Hkv=4)
+    if name == "cfg3_mix":               # two GLM-shaped requests of very different lengths (512K and 32K tokens)
+        return locks_synth.Workload("cfg3_glm_mix_512k_32k", [1 << 19, 1 << 15], Hq=32, Hkv=2, seed=3)
     if name.startswith("cfg4_b"):
         return locks_synth.config4(batch=int(name[6:]))
     if name == "small":
