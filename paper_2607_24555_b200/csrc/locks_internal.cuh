@@ -131,7 +131,7 @@ __device__ __forceinline__ void locks_update_partition_hint(int32_t *hint, const
   if (lane == 0) {
     const int strided = rounds * ((mx + wpp - 1) / wpp);
     const int even = (int)(((int64_t)sum * Hkv + W - 1) / W);
-    *hint = (strided * 16 > even * 17 + 16) ? LOCKS_PARTITION_BALANCED : LOCKS_PARTITION_STRIDED;
+    *hint = (strided * 16 > even * 17 + 8) ? LOCKS_PARTITION_BALANCED : LOCKS_PARTITION_STRIDED;
   }
 }
 

@@ -84,7 +84,7 @@ def test_balanced_partition_invariants(seed):
 
 def test_partition_suggestion_rule():
     """Iterations of the longest warp: strided = rounds * ceil(max groups / wpp), balanced = ceil(U / W); the
-    balanced partition is suggested only when it wins by more than 1/16 plus one iteration."""
+    balanced partition is suggested only when it wins by more than 1/16 plus half an iteration."""
     def suggest(ng, Hkv, W):
         nprob = len(ng) * Hkv
         wpp = max(1, W // nprob)
@@ -92,7 +92,7 @@ def test_partition_suggestion_rule():
         rounds = -(-nprob // nslots)
         strided = rounds * -(-max(ng) // wpp)
         even = -(-sum(ng) * Hkv // W)
-        return strided * 16 > even * 17 + 16
+        return strided * 16 > even * 17 + 8
     W = 296 * 8
     assert not suggest([256] * 8, 8, W)                        # equal lengths (8 x 32K tokens)
     assert not suggest([128] * 32, 8, W)                       # equal lengths (32 x 16K tokens)
