@@ -182,6 +182,12 @@ int locks_poll_status(locks_ctx *ctx, int32_t *status_host, locks_stream stream)
 #define LOCKS_PARTITION_BALANCED 2
 int locks_set_scan_partition(locks_ctx *ctx, int mode);
 
+/* Self-test of the bounded device-side wait every kernel of the library uses for its asynchronous copies: one
+ * warp waits, for at most limit_ms milliseconds (1 .. 1000), on a barrier that nothing ever completes, gives up,
+ * and records LOCKS_ERR_TIMEOUT in the status word, which locks_poll_status() then reports.  The context stays
+ * usable.  Enqueues one small kernel on `stream`. */
+int locks_selftest_wait_timeout(locks_ctx *ctx, int limit_ms, locks_stream stream);
+
 /* Number of kernels the last call on this context enqueued (for launch accounting). */
 int locks_last_launch_count(const locks_ctx *ctx);
 

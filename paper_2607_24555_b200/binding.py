@@ -17,7 +17,7 @@ SYMBOLS = ["locks_summary_bytes", "locks_workspace_bytes", "locks_create", "lock
            "locks_build_summaries", "locks_select", "locks_sparse_attend", "locks_decode_step",
            "locks_decode_step_host", "locks_poll_status", "locks_last_launch_count", "locks_strerror",
            "locks_profile_begin", "locks_profile_end", "locks_profile_read", "locks_sparse_attend_noalloc",
-           "locks_set_scan_partition"]
+           "locks_set_scan_partition", "locks_selftest_wait_timeout"]
 
 
 PARTITION_AUTO, PARTITION_STRIDED, PARTITION_BALANCED = 0, 1, 2   # LOCKS_PARTITION_* of include/locks.h
@@ -78,6 +78,8 @@ def lib():
         L.locks_sparse_attend_noalloc.argtypes = [C.POINTER(Config), vp, C.POINTER(KV), C.c_int, i32p, i32p, vp, vp, vp]
         L.locks_sparse_attend_noalloc.restype = C.c_int
         L.locks_set_scan_partition.argtypes = [vp, C.c_int]
+        L.locks_selftest_wait_timeout.argtypes = [vp, C.c_int, vp]
+        L.locks_selftest_wait_timeout.restype = C.c_int
         L.locks_set_scan_partition.restype = C.c_int
         L.locks_strerror.restype = C.c_char_p
         L.locks_strerror.argtypes = [C.c_int]
@@ -213,6 +215,9 @@ class Context:
         st = C.c_int32(0)
         _check(lib().locks_poll_status(self.handle, C.byref(st), _stream(stream)), "locks_poll_status")
         return int(st.value)
+
+    def locks_selftest_wait_timeout(self, limit_ms: int, stream=None):
+        _check(lib().locks_selftest_wait_timeout(self.handle, int(limit_ms), _stream(stream)), "locks_selftest_wait_timeout")
 
     def locks_set_scan_partition(self, mode: int):
         _check(lib().locks_set_scan_partition(self.handle, int(mode)), "locks_set_scan_partition")

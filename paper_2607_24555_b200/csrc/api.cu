@@ -214,6 +214,24 @@ int locks_destroy(locks_ctx *ctx) {
   return LOCKS_OK;
 }
 
+namespace {
+__global__ void __launch_bounds__(32) wait_timeout_kernel(int32_t *status, uint64_t limit_ns) {
+  __shared__ uint64_t bar;
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    fence_barrier_init();
+  }
+  __syncwarp();
+  if (!mbar_wait(&bar, 0, limit_ns) && threadIdx.x == 0) set_status(status, LOCKS_ERR_TIMEOUT);
+}
+}  // namespace
+
+int locks_selftest_wait_timeout(locks_ctx *ctx, int limit_ms, locks_stream stream) {
+  if (!ctx || limit_ms < 1 || limit_ms > 1000) return LOCKS_ERR_INVALID_ARG;
+  wait_timeout_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(ctx->status, (uint64_t)limit_ms * 1000000ull);
+  return cudaPeekAtLastError() == cudaSuccess ? LOCKS_OK : LOCKS_ERR_CUDA;
+}
+
 int locks_set_scan_partition(locks_ctx *ctx, int mode) {
   if (!ctx || mode < LOCKS_PARTITION_AUTO || mode > LOCKS_PARTITION_BALANCED) return LOCKS_ERR_INVALID_ARG;
   ctx->scan_partition = mode;

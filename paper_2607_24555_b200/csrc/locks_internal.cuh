@@ -35,7 +35,8 @@
 #ifndef LOCKS_SCAN_BULK
 #define LOCKS_SCAN_BULK 1      // staging of summary blobs in the scan: 1 = cp.async.bulk (TMA) + mbarrier, 0 = 16-byte cp.async
 #endif
-#define LOCKS_SPIN_LIMIT (1 << 22)  // bounded mbarrier polling (each poll already waits a while)
+#define LOCKS_SPIN_LIMIT (1 << 22)  // bounded mbarrier polling (each poll already waits a while) ...
+#define LOCKS_WAIT_LIMIT_NS 1000000000ull   // ... and never longer than a second
 
 // One cached CUDA graph of the host-buffer decode step (copies in, step, copies out) for one set of arguments.
 struct locks_host_graph {
@@ -262,8 +263,16 @@ __device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes) {
                : "memory");
 }
 // Bounded wait on a phase parity: true when the phase completed, false when the poll limit ran out.
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity) {
+__device__ __forceinline__ uint64_t global_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+// Waits for the phase `parity` of an mbarrier.  Bounded twice: by a number of polls and by wall time (the
+// clock is read only after a poll has failed).  false = the wait ran out; the caller reports LOCKS_ERR_TIMEOUT.
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, uint64_t limit_ns = LOCKS_WAIT_LIMIT_NS) {
   uint32_t a = smem_u32(bar);
+  uint64_t t0 = 0;
   for (int it = 0; it < LOCKS_SPIN_LIMIT; ++it) {
     uint32_t done;
     asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
@@ -272,6 +281,8 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity) {
                  : "r"(a), "r"(parity)
                  : "memory");
     if (done) return true;
+    if (it == 0) t0 = global_ns();
+    else if (global_ns() - t0 > limit_ns) return false;
   }
   return false;
 }

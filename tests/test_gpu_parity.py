@@ -556,6 +556,24 @@ def test_scan_partition_setter_rejects_unknown_modes():
             gc.ctx.locks_set_scan_partition(mode)
 
 
+def test_bounded_wait_runs_out_and_reports():
+    """Host-visible outcome of a device-side wait that nothing completes: the kernel gives up after its limit,
+    the status word says LOCKS_ERR_TIMEOUT (-5), and the context keeps working."""
+    import time
+    gc = _gc(small_bf16([16 * 40], Hq=8, Hkv=2, budget=128, seed=67))
+    summ = gc.gpu_build()
+    ids0, cnt0, _, _ = gc.gpu_select(summ)
+    t0 = time.perf_counter()
+    gc.ctx.locks_selftest_wait_timeout(50)
+    assert gc.status() == -5                      # polling synchronises and clears
+    assert time.perf_counter() - t0 < 2.0        # 50 ms limit, not the one-second default nor the poll count
+    assert gc.status() == 0
+    ids1, cnt1, _, _ = gc.gpu_select(summ)       # the context is as usable as before
+    assert np.array_equal(ids0, ids1) and np.array_equal(cnt0, cnt1)
+    with pytest.raises(locks.LocksError):
+        gc.ctx.locks_selftest_wait_timeout(0)
+
+
 def test_bad_block_id_sets_status_without_faulting():
     """Host-injected fault: a block id outside the cache is skipped and reported, nothing traps."""
     gc = _gc(small_bf16([16 * 60], Hq=8, Hkv=2, budget=128, seed=66))
