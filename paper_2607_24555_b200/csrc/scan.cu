@@ -509,10 +509,13 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4_kerne
   for (int hh = 0; hh < NH; ++hh) { pm[hh] = -INFINITY; ps[hh] = 0.f; }
   int cur_b = 0, cur_h = 0, cur_pslot = sub;   // partial slot of this warp in the current problem
   auto accumulate = [&](float &m, float &sacc, float v) {   // online log-sum-exp, one exp per value
-    if (v > -INFINITY) {
-      const float d = v - m, e = __expf(-fabsf(d));
-      if (d > 0.f) { sacc = sacc * e + 1.f; m = v; } else sacc += e;
-    }
+    // branch-free: a value of -inf (masked page) adds nothing, whatever m is (also -inf at the start)
+    const bool live = v > -INFINITY;
+    const float d = v - m;                                    // NaN only if both are -inf: not live then
+    const float e = live ? __expf(-fabsf(d)) : 0.f;           // m = -inf, v finite: exp(-inf) = 0
+    const bool up = live && d > 0.f;
+    sacc = up ? fmaf(sacc, e, 1.f) : sacc + e;
+    m = up ? v : m;
   };
   float2 *red = reinterpret_cast<float2 *>(smem + kScanWarps * (kScanStages * kStageBytes + 64));   // [warp][16]
   auto flush = [&](bool to_smem, bool finished) {
