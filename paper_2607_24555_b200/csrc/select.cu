@@ -412,7 +412,7 @@ __device__ __noinline__ void select_finish(int32_t *done, int chunks, int kc, in
   }
 }
 
-__global__ void __launch_bounds__(LOCKS_SEL_THREADS) select_kernel(SelParams p) {
+__global__ void __launch_bounds__(LOCKS_SEL_THREADS, 2) select_kernel(SelParams p) {
   SelShared &sh = shared_state();
   const int chunk = blockIdx.x, h = blockIdx.y, b = blockIdx.z, tid = threadIdx.x;
   pdl_trigger();
