@@ -488,11 +488,18 @@ int locks_launch_select(locks_ctx *c, const float *shat, const locks_kv *kv, int
   p.part_slots = c->part_slots;
   p.part_cnt = c->part_balanced ? c->part_cnt : nullptr;
   if (p.chunk_pages > kMaxKeys || (int64_t)c->sel_chunks * c->sel_kc > kMaxKeys || p.G > 16) return LOCKS_ERR_UNSUPPORTED;
+  // Two CTAs fit on an SM (64 registers per thread).  That halves the waves of a launch with many more CTAs
+  // than SMs, but with up to about 1.5 CTAs per SM the block scheduler stacks pairs on the SMs that drain first
+  // while others idle (measured: +15 us at 192 CTAs); such launches ask for enough shared memory to keep one
+  // CTA per SM.
+  constexpr int kSmemAlone = 116 * 1024;
   static bool attr_done = false;
   if (!attr_done) {
-    cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(SelShared));
+    cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemAlone);
     attr_done = true;
   }
-  locks_launch_pdl(select_kernel, dim3(c->sel_chunks, p.Hkv, batch), dim3(LOCKS_SEL_THREADS), sizeof(SelShared), st, p);
+  const int64_t nctas = (int64_t)c->sel_chunks * p.Hkv * batch;
+  const size_t smem = 2 * nctas <= 3 * (int64_t)c->num_sms ? (size_t)kSmemAlone : sizeof(SelShared);
+  locks_launch_pdl(select_kernel, dim3(c->sel_chunks, p.Hkv, batch), dim3(LOCKS_SEL_THREADS), smem, st, p);
   return locks_check_launch(c);
 }
