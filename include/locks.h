@@ -158,11 +158,20 @@ int locks_decode_step(locks_ctx *ctx, const void *q, const void *k_new, const vo
  * Repeated calls with the same arguments (a serving loop calls once per layer and step with fixed
  * buffers) are cached: from the third call on, the copies and the step are one CUDA-graph launch.
  * The cache holds 8 argument sets per context, needs page-locked host buffers and a stream that is
- * not being captured, and is released by locks_destroy(); other calls take the plain path. */
+ * not being captured, and is released by locks_destroy(); other calls take the plain path.
+ * LIFETIME: a cached graph holds the device's alias of the page-locked host buffers and every device pointer
+ * of the argument set.  Buffers passed to this call must therefore stay allocated and page-locked until
+ * locks_destroy() or locks_host_cache_clear(): a later call with the same addresses replays the graph without
+ * looking at the memory behind them again.  Call locks_host_cache_clear() before freeing or unpinning any of
+ * them if the context lives on. */
 int locks_decode_step_host(locks_ctx *ctx, const void *q_host, const void *k_new_host,
                            const void *v_new_host, locks_kv *kv, void *summaries, int batch,
                            void *out_host, int32_t *page_ids_host, int32_t *page_count_host,
                            locks_stream stream);
+
+/* Drop every cached graph of locks_decode_step_host (see its LIFETIME note).  The next calls take the plain
+ * path and rebuild the cache from the buffers they are given.  Host-side only. */
+int locks_host_cache_clear(locks_ctx *ctx);
 
 /* Copy the sticky device status word to the host and clear it.  Synchronises the stream.
  * *status_host: LOCKS_OK or the first LOCKS_ERR_* a kernel recorded. */
@@ -181,6 +190,13 @@ int locks_poll_status(locks_ctx *ctx, int32_t *status_host, locks_stream stream)
 #define LOCKS_PARTITION_STRIDED 1
 #define LOCKS_PARTITION_BALANCED 2
 int locks_set_scan_partition(locks_ctx *ctx, int mode);
+/* The partition the most recent scan launch of this context used (LOCKS_PARTITION_STRIDED or _BALANCED; 0 before
+ * the first one, or when the scan ran the plain kernel that has no partition).  With LOCKS_PARTITION_AUTO the
+ * choice follows a word the device writes asynchronously, so it can differ from run to run near the switching
+ * point; a captured graph (the host entry point's cached graphs included) keeps the choice made at capture.
+ * Callers that need reproducible log Z rounding or timings pin the mode with locks_set_scan_partition(), which
+ * also drops the host entry point's cached graphs when the mode changes. */
+int locks_last_scan_partition(const locks_ctx *ctx);
 
 /* Self-test of the bounded device-side wait every kernel of the library uses for its asynchronous copies: one
  * warp waits, for at most limit_ms milliseconds (1 .. 1000), on a barrier that nothing ever completes, gives up,

@@ -19,7 +19,7 @@
  *   - Lemma 1(ii): exact page log-mass s_j(q) = log sum_{i in P_j} exp(q.k_i/sqrt(d)) (the
  *     "exact" arm used as a ceiling and in invariants).
  *
- * Readings taken where the paper is silent (all listed in the design notes of the repository):
+ * Readings taken where the paper is silent (these are all of them):
  *   quantiser = symmetric abs-max, scale = fp16(maxabs/qmax), qmax 7 (int4) / 127 (int8),
  *   code = clamp(rint(x/scale)) round-half-even with the rounded scale; zero-mode threshold
  *   lambda_l <= 1e-6 lambda_1 (or <= 1e-10 of the page's summed squared key norms) and never more
@@ -28,8 +28,9 @@
  *   log m_bar_j, ties to the lower page index; returned ids ascending, -1 padded;
  *   P <= k selects every page.
  *
- * Parity status: every function here is pinned by the CPU tests (closed forms, invariants from
- * the paper's propositions, brute force, numpy cross-checks) EXCEPT the size of the score error
+ * Parity status: every function here, the batch-level wrappers' request / head / block indexing
+ * included, is pinned by the CPU tests (closed forms, invariants from the paper's propositions,
+ * brute force, numpy cross-checks) EXCEPT the size of the score error
  * caused by the integer storage, for which the paper derives no bound: "parity unpinned" for
  * that one quantity (the integer pack/unpack itself is pinned by round-trip and byte counts).
  *

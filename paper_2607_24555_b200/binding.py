@@ -17,7 +17,8 @@ SYMBOLS = ["locks_summary_bytes", "locks_workspace_bytes", "locks_create", "lock
            "locks_build_summaries", "locks_select", "locks_sparse_attend", "locks_decode_step",
            "locks_decode_step_host", "locks_poll_status", "locks_last_launch_count", "locks_strerror",
            "locks_profile_begin", "locks_profile_end", "locks_profile_read", "locks_sparse_attend_noalloc",
-           "locks_set_scan_partition", "locks_selftest_wait_timeout"]
+           "locks_set_scan_partition", "locks_selftest_wait_timeout", "locks_last_scan_partition",
+           "locks_host_cache_clear"]
 
 
 PARTITION_AUTO, PARTITION_STRIDED, PARTITION_BALANCED = 0, 1, 2   # LOCKS_PARTITION_* of include/locks.h
@@ -81,6 +82,10 @@ def lib():
         L.locks_selftest_wait_timeout.argtypes = [vp, C.c_int, vp]
         L.locks_selftest_wait_timeout.restype = C.c_int
         L.locks_set_scan_partition.restype = C.c_int
+        L.locks_last_scan_partition.argtypes = [vp]
+        L.locks_last_scan_partition.restype = C.c_int
+        L.locks_host_cache_clear.argtypes = [vp]
+        L.locks_host_cache_clear.restype = C.c_int
         L.locks_strerror.restype = C.c_char_p
         L.locks_strerror.argtypes = [C.c_int]
         for fn in ("locks_create", "locks_destroy", "locks_build_summaries", "locks_select", "locks_sparse_attend",
@@ -221,6 +226,12 @@ class Context:
 
     def locks_set_scan_partition(self, mode: int):
         _check(lib().locks_set_scan_partition(self.handle, int(mode)), "locks_set_scan_partition")
+
+    def locks_last_scan_partition(self) -> int:
+        return int(lib().locks_last_scan_partition(self.handle))
+
+    def locks_host_cache_clear(self):
+        _check(lib().locks_host_cache_clear(self.handle), "locks_host_cache_clear")
 
     def locks_profile_begin(self, max_steps: int):
         _check(lib().locks_profile_begin(self.handle, max_steps), "locks_profile_begin")

@@ -1,4 +1,5 @@
 // C-ABI entry points of liblocks (see include/locks.h for the contract of every call).
+#include <mutex>
 #include <new>
 
 #include "locks_internal.cuh"
@@ -114,6 +115,18 @@ int check_common(const locks_ctx *ctx, const locks_kv *kv, int batch) {
 
 }  // namespace
 
+bool locks_attrs_needed(int family) {
+  static std::mutex mu;
+  static uint64_t done[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64 || family < 0 || family >= 64) return true;
+  std::lock_guard<std::mutex> lock(mu);
+  const uint64_t bit = 1ull << family;
+  if (done[dev] & bit) return false;
+  done[dev] |= bit;
+  return true;
+}
+
 extern "C" {
 
 size_t locks_summary_bytes(const locks_config *cfg) {
@@ -143,6 +156,7 @@ int locks_create(const locks_config *cfg, void *workspace, size_t ws_bytes, lock
   c->part_slots = L.max_groups;
   c->part_balanced = 0;
   c->scan_partition = LOCKS_PARTITION_AUTO;
+  c->last_partition = 0;
   c->hint_host = nullptr; c->hint_dev = nullptr;
   {   // one page-locked word the device can write and the host can read without synchronising
     void *hp = nullptr, *dp = nullptr;
@@ -234,7 +248,20 @@ int locks_selftest_wait_timeout(locks_ctx *ctx, int limit_ms, locks_stream strea
 
 int locks_set_scan_partition(locks_ctx *ctx, int mode) {
   if (!ctx || mode < LOCKS_PARTITION_AUTO || mode > LOCKS_PARTITION_BALANCED) return LOCKS_ERR_INVALID_ARG;
+  if (mode != ctx->scan_partition) (void)locks_host_cache_clear(ctx);   // cached graphs froze the old choice
   ctx->scan_partition = mode;
+  return LOCKS_OK;
+}
+
+int locks_last_scan_partition(const locks_ctx *ctx) { return ctx ? ctx->last_partition : 0; }
+
+int locks_host_cache_clear(locks_ctx *ctx) {
+  if (!ctx) return LOCKS_ERR_INVALID_ARG;
+  for (int i = 0; i < LOCKS_HOST_GRAPHS; ++i) {
+    if (ctx->hg[i].exec) cudaGraphExecDestroy(ctx->hg[i].exec);
+    ctx->hg[i] = locks_host_graph{};
+  }
+  ctx->hg_next = 0;
   return LOCKS_OK;
 }
 

@@ -7,6 +7,7 @@
 // log-sum-exp.  Partial (o, lse) per split are merged by a second small kernel.
 // A NULL page table means "all pages": the same kernel is the dense flash-decode baseline.
 #include <cooperative_groups.h>
+#include <mutex>
 #include "locks_internal.cuh"
 
 namespace {
@@ -96,7 +97,11 @@ __global__ void __launch_bounds__(LOCKS_ATT_WARPS * 32) attend_bf16_kernel(AttPa
   pdl_wait();   // page table from the selector, appended K/V rows, sequence lengths
   const int T = p.seq_lens[b];
   const int P = (T + LOCKS_B - 1) / LOCKS_B;
-  const int npages = p.ids ? p.cnt[prob] : P;
+  int npages = p.ids ? p.cnt[prob] : P;
+  if (p.ids && (npages < 0 || npages > p.kbud)) {   // a count beyond the table's row: use the row, report it
+    if (threadIdx.x == 0) set_status(p.status, LOCKS_ERR_BAD_BLOCK);
+    npages = npages < 0 ? 0 : p.kbud;
+  }
   const int lo = split * p.pages_per_cta;
   const int hi = min(lo + p.pages_per_cta, npages);
 
@@ -438,7 +443,11 @@ __global__ void __launch_bounds__(128) attend_generic_kernel(AttParams p) {
   const int64_t prob = (int64_t)b * p.Hkv + h;
   const int Tn = p.seq_lens[b];
   const int P = (Tn + LOCKS_B - 1) / LOCKS_B;
-  const int npages = p.ids ? p.cnt[prob] : P;
+  int npages = p.ids ? p.cnt[prob] : P;
+  if (p.ids && (npages < 0 || npages > p.kbud)) {
+    if (threadIdx.x == 0) set_status(p.status, LOCKS_ERR_BAD_BLOCK);
+    npages = npages < 0 ? 0 : p.kbud;
+  }
   const int lo = split * p.pages_per_cta, hi = min(lo + p.pages_per_cta, npages);
   const T *K = reinterpret_cast<const T *>(p.k), *V = reinterpret_cast<const T *>(p.v), *Q = reinterpret_cast<const T *>(p.q);
   float qv[4], o[4] = {0.f, 0.f, 0.f, 0.f};
@@ -604,8 +613,7 @@ int locks_launch_attend(locks_ctx *c, const void *q, const locks_kv *kv, int bat
   }
   const bool bf = c->cfg.kv_dtype == LOCKS_BF16;
   if (bf) {
-    static bool attr_done = false;
-    if (!attr_done) {
+    if (locks_attrs_needed(LOCKS_ATTR_ATTEND)) {
       cudaFuncSetAttribute(attend_bf16_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttSmem);
       cudaFuncSetAttribute(attend_bf16_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttSmem);
       cudaFuncSetAttribute(attend_bf16_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttSmem);
@@ -614,7 +622,6 @@ int locks_launch_attend(locks_ctx *c, const void *q, const locks_kv *kv, int bat
       cudaFuncSetAttribute(attend_bf16_kernel<2, true>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
       cudaFuncSetAttribute(attend_bf16_kernel<1, false>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
       cudaFuncSetAttribute(attend_bf16_kernel<2, false>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
-      attr_done = true;
     }
     dim3 grid(p.splits, p.Hkv, batch);
     const bool contig = kv->stride_token == LOCKS_D;
@@ -674,6 +681,7 @@ struct NoAllocDevice {
   bool ready;
 };
 NoAllocDevice g_noalloc_dev[64] = {};
+std::mutex g_noalloc_mu;   // guards the per-device set-up (two host threads may make a device's first call)
 
 }  // namespace
 
@@ -696,6 +704,7 @@ extern "C" int locks_sparse_attend_noalloc(const locks_config *cfg, const void *
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return LOCKS_ERR_CUDA;
   NoAllocDevice &nd = g_noalloc_dev[dev];
+  std::unique_lock<std::mutex> setup_lock(g_noalloc_mu);
   if (!nd.ready) {
     // first call on this device: ask the runtime where the array lives on the CURRENT device
     void *ptr = nullptr;
@@ -708,6 +717,7 @@ extern "C" int locks_sparse_attend_noalloc(const locks_config *cfg, const void *
     nd.scratch = reinterpret_cast<unsigned char *>(ptr);
     nd.ready = true;
   }
+  setup_lock.unlock();
   cudaStream_t st = (cudaStream_t)stream;
   AttParams p;
   p.q = q; p.k = kv->k; p.v = kv->v; p.sb = kv->stride_block; p.sh = kv->stride_head; p.st = kv->stride_token;

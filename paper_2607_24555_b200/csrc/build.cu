@@ -377,13 +377,11 @@ int locks_launch_build(locks_ctx *c, const locks_kv *kv, int batch, const int32_
                           : dim3((c->Pmax + kBuildWarps - 1) / kBuildWarps, p.Hkv, batch);
   const int smem = kBuildWarps * kBuildSmemPerWarp;
   const bool bf = c->cfg.kv_dtype == LOCKS_BF16, i4 = c->cfg.summary_fmt == LOCKS_FMT_I4;
-  static bool attr_done = false;
-  if (!attr_done) {
+  if (locks_attrs_needed(LOCKS_ATTR_BUILD)) {
     cudaFuncSetAttribute(build_kernel<__nv_bfloat16, LOCKS_FMT_I4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     cudaFuncSetAttribute(build_kernel<__nv_bfloat16, LOCKS_FMT_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     cudaFuncSetAttribute(build_kernel<float, LOCKS_FMT_I4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     cudaFuncSetAttribute(build_kernel<float, LOCKS_FMT_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    attr_done = true;
   }
   if (bf && i4) build_kernel<__nv_bfloat16, LOCKS_FMT_I4><<<grid, kBuildWarps * 32, smem, st>>>(p);
   else if (bf) build_kernel<__nv_bfloat16, LOCKS_FMT_F32><<<grid, kBuildWarps * 32, smem, st>>>(p);

@@ -59,6 +59,7 @@ struct locks_ctx {
   int part_slots;          // partial slots per (request, head) the last scan launch may have filled
   int part_balanced;       // the last scan launch wrote per-problem partial counts to part_cnt instead
   int scan_partition;      // LOCKS_PARTITION_*: how the tensor scan deals pages to its warps
+  int last_partition;      // partition the last tensor-scan launch used (0: no such launch yet)
   int32_t *hint_host;      // pinned, device-mapped word: partition the device suggests for the current lengths
   int32_t *hint_dev;       //   (0 none yet, LOCKS_PARTITION_STRIDED, LOCKS_PARTITION_BALANCED)
   int sel_ept;             // pages per thread of a selector CTA (chunk = sel_ept * 512 pages)
@@ -189,10 +190,20 @@ static inline void locks_launch_pdl_cluster(void (*kernel)(KArgs...), dim3 grid,
   (void)cudaLaunchKernelEx(&cfg, kernel, args...);
 }
 
+// A failed launch is reported once: the runtime's sticky-until-read error is cleared, so that the next call
+// on this thread is judged on its own launches.
 static inline int locks_check_launch(locks_ctx *c) {
   c->last_launches++;
-  return cudaPeekAtLastError() == cudaSuccess ? LOCKS_OK : LOCKS_ERR_CUDA;
+  if (cudaPeekAtLastError() == cudaSuccess) return LOCKS_OK;
+  (void)cudaGetLastError();
+  return LOCKS_ERR_CUDA;
 }
+
+// Function attributes (dynamic shared-memory limit, non-portable cluster size) belong to a device, not to the
+// process: true exactly once per (current device, kernel family), so that a process that drives several GPUs
+// sets them on each.  Thread-safe.
+enum { LOCKS_ATTR_SELECT = 0, LOCKS_ATTR_ATTEND = 1, LOCKS_ATTR_BUILD = 2, LOCKS_ATTR_EXACT = 3, LOCKS_ATTR_SCAN = 8 };
+bool locks_attrs_needed(int family);
 
 // ---------------------------------------------------------------- I4 blob geometry (B = 16, d = 128)
 // [basis 64 r][coefficients 16 r][centroid 128][sC 16 x fp16][sV r x fp16][sMu fp16], padded to 16.

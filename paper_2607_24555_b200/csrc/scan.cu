@@ -939,6 +939,7 @@ int locks_launch_scan(locks_ctx *c, const void *q, const void *summaries, const 
   const bool tensor = c->cfg.summary_fmt == LOCKS_FMT_I4 && c->cfg.q_dtype == LOCKS_BF16;   // ranks 2, 4, 8
   c->part_slots = c->max_groups;   // generic kernel: one partial per 8-page group
   c->part_balanced = 0;
+  c->last_partition = 0;
   if (tensor) {
     const locks_scan_geom geo = locks_scan_geometry(c, batch);
     const int grid = geo.grid;
@@ -958,6 +959,7 @@ int locks_launch_scan(locks_ctx *c, const void *q, const void *summaries, const 
       c->part_slots = geo.wpp;
     }
     c->part_balanced = balanced ? 1 : 0;
+    c->last_partition = balanced ? LOCKS_PARTITION_BALANCED : LOCKS_PARTITION_STRIDED;
     const dim3 g(grid), blk(kScanWarps * 32);
     const int gsel = c->G <= 4 ? 0 : (c->G <= 8 ? 1 : 2);
     // tensor map over the summaries for the gather path: rows = (block, KV head), S / 4 32-bit words each
@@ -990,12 +992,10 @@ int locks_launch_scan(locks_ctx *c, const void *q, const void *summaries, const 
     }
 #define LOCKS_SCAN_LAUNCH(R_, CR_, BAL_)                                                                                  \
   do {                                                                                                                 \
-    static bool attr_done = false;                                                                                     \
-    if (!attr_done) {                                                                                                  \
+    if (locks_attrs_needed(LOCKS_ATTR_SCAN + (R_ == 8 ? 0 : (R_ == 4 ? 4 : 8)) + (CR_ ? 2 : 0) + (BAL_ ? 1 : 0))) {     \
       cudaFuncSetAttribute(scan_i4_kernel<R_, 1, true, CR_, BAL_>, cudaFuncAttributeMaxDynamicSharedMemorySize, kScanSmem);  \
       cudaFuncSetAttribute(scan_i4_kernel<R_, 1, false, CR_, BAL_>, cudaFuncAttributeMaxDynamicSharedMemorySize, kScanSmem); \
       cudaFuncSetAttribute(scan_i4_kernel<R_, 2, false, CR_, BAL_>, cudaFuncAttributeMaxDynamicSharedMemorySize, kScanSmem); \
-      attr_done = true;                                                                                                \
     }                                                                                                                  \
     if (gsel == 0) locks_launch_pdl(scan_i4_kernel<R_, 1, true, CR_, BAL_>, g, blk, kScanSmem, st, p, tmap);                       \
     else if (gsel == 1) locks_launch_pdl(scan_i4_kernel<R_, 1, false, CR_, BAL_>, g, blk, kScanSmem, st, p, tmap);                 \

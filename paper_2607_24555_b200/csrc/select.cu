@@ -493,11 +493,8 @@ int locks_launch_select(locks_ctx *c, const float *shat, const locks_kv *kv, int
   // while others idle (measured: +15 us at 192 CTAs); such launches ask for enough shared memory to keep one
   // CTA per SM.
   constexpr int kSmemAlone = 116 * 1024;
-  static bool attr_done = false;
-  if (!attr_done) {
+  if (locks_attrs_needed(LOCKS_ATTR_SELECT))
     cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemAlone);
-    attr_done = true;
-  }
   const int64_t nctas = (int64_t)c->sel_chunks * p.Hkv * batch;
   const size_t smem = 2 * nctas <= 3 * (int64_t)c->num_sms ? (size_t)kSmemAlone : sizeof(SelShared);
   locks_launch_pdl(select_kernel, dim3(c->sel_chunks, p.Hkv, batch), dim3(LOCKS_SEL_THREADS), smem, st, p);

@@ -459,3 +459,133 @@ def test_full_budget_equals_dense_and_pipeline_runs():
     sex = oracle.page_logmass(cache, q, w.rank, fmt_code(w), None, SM, exact=True)
     assert np.nanmax(np.abs(shat - sex)[:, :, :P - 1]) < 0.5
     assert np.all(np.isnan(shat[:, :, P - 1:]))
+
+
+# ------------------------------------------------------------------ batch / head indexing of the wrappers
+
+def ragged_batch_cache(layout="HND", bf16=False, seed=5):
+    """3 requests of different lengths (one with a partial tail page), 2 KV heads x 3 query heads each,
+    physical blocks dealt by a permutation that interleaves the requests, spare blocks in between."""
+    g = np.random.default_rng(seed)
+    B, d, Hkv, Hq = 16, 128, 2, 6
+    lens = [16 * 9 + 5, 16 * 7, 16 * 12 + 1]
+    pages = [-(-t // B) for t in lens]
+    nb = sum(pages) + 4
+    shape = (nb, Hkv, B, d) if layout == "HND" else (nb, B, Hkv, d)
+    k = g.standard_normal(shape).astype(np.float32)
+    v = g.standard_normal(shape).astype(np.float32)
+    if bf16:   # stored as raw bfloat16 bits; `vals` are the values those bits stand for
+        k = (k.view(np.uint32) >> 16).astype(np.uint16)
+        v = (v.view(np.uint32) >> 16).astype(np.uint16)
+    perm = g.permutation(nb)
+    bt = np.full((3, max(pages)), -12345, np.int32)      # slots past a request's pages hold a poison id
+    at = 0
+    for b, P in enumerate(pages):
+        bt[b, :P] = perm[at:at + P]
+        at += P
+    if layout == "HND":
+        strides = {"shape": (nb, Hkv, B, d), "block": Hkv * B * d, "head": B * d, "token": d}
+    else:
+        strides = {"shape": (nb, Hkv, B, d), "block": B * Hkv * d, "head": d, "token": Hkv * d}
+    cache = oracle.Cache(k, v, bt, np.array(lens, np.int32), Hq, strides=strides)
+
+    def vals(a):
+        f = (a.astype(np.uint32) << 16).view(np.float32) if bf16 else a
+        return f.astype(np.float64)
+
+    def page(a, blk, h):   # [B, d] values of (block, head), whatever the layout
+        return vals(a[blk, h]) if layout == "HND" else vals(a[blk, :, h])
+
+    q = g.standard_normal((3, Hq, d)).astype(np.float32)
+    if bf16:
+        q = (q.view(np.uint32) >> 16).astype(np.uint16)
+    return cache, q, vals(q), page, lens, pages
+
+
+@pytest.mark.parametrize("layout,bf16,fmt,r", [("HND", False, oracle.FMT_I4, 8), ("NHD", True, oracle.FMT_I4, 4),
+                                               ("HND", True, oracle.FMT_F32, 3)])
+def test_batch_wrappers_index_requests_heads_and_blocks(layout, bf16, fmt, r):
+    """build_summaries, page_logmass, select, attend and decode_step on a ragged batch of 3 requests, 2 KV heads,
+    G = 3, permuted blocks: every entry equals what the per-page functions (pinned above one by one) give when
+    they are composed with the index arithmetic written out here."""
+    cache, q_raw, q, page, lens, pages = ragged_batch_cache(layout, bf16)
+    B, d, Hkv, Hq, G = 16, 128, 2, 6, 3
+    k = 5
+    summ = oracle.build_summaries(cache, r, fmt)
+    stride = oracle.summary_stride_bytes(fmt, r)
+    assert summ.shape == (cache.num_blocks, Hkv, stride)
+    used = set()
+    shat_ref = np.full((3, Hq, max(pages)), np.nan)
+    sex_ref = np.full((3, Hq, max(pages)), np.nan)
+    for b in range(3):
+        for h in range(Hkv):
+            for p in range(lens[b] // B):                              # complete pages only
+                blk = int(cache.block_table[b, p])
+                used.add((blk, h))
+                mu, V, Cc, _, _ = oracle.build_page(page(cache.k, blk, h), r)
+                assert np.array_equal(summ[blk, h], oracle.pack(fmt, mu, V, Cc)), (b, h, p)
+            for p in range(pages[b] - 1):                              # pages 0 .. P-2 are scored
+                blk = int(cache.block_table[b, p])
+                m = oracle.unpack(fmt, r, summ[blk, h])
+                for gi in range(G):
+                    shat_ref[b, h * G + gi, p] = oracle.score(*m, q[b, h * G + gi], SM)
+                    sex_ref[b, h * G + gi, p] = oracle.exact_lse(page(cache.k, blk, h), q[b, h * G + gi], SM)
+    for blk in range(cache.num_blocks):                                # nothing else was written
+        for h in range(Hkv):
+            if (blk, h) not in used:
+                assert not summ[blk, h].any()
+    shat = oracle.page_logmass(cache, q_raw, r, fmt, summ, SM)
+    sex = oracle.page_logmass(cache, q_raw, r, fmt, None, SM, exact=True)
+    assert np.array_equal(np.isnan(shat), np.isnan(shat_ref)) and np.array_equal(np.isnan(sex), np.isnan(sex_ref))
+    assert np.nanmax(np.abs(shat - shat_ref)) == 0.0 and np.nanmax(np.abs(sex - sex_ref)) == 0.0
+    ids, cnt, ls = oracle.select(cache, shat, k)
+    ids_ref = np.full((3, Hkv, k), -1, np.int32)
+    for b in range(3):
+        for h in range(Hkv):
+            i1, c1, l1 = oracle.select_one(shat[b, h * G:(h + 1) * G], pages[b], k)
+            ids_ref[b, h] = i1
+            assert cnt[b, h] == c1 == k and np.array_equal(ids[b, h], i1)
+            assert np.array_equal(ls[b, h, 1:pages[b] - 1], l1[1:pages[b] - 1])
+            assert np.all(np.isnan(ls[b, h, pages[b] - 1:])) and np.isnan(ls[b, h, 0])
+    # the two heads and the three requests do select different pages here, so a swapped index would show
+    assert len({tuple(ids[b, h]) for b in range(3) for h in range(Hkv)}) == 3 * Hkv
+
+    def attend_ref(b, gq, plist):
+        h = gq // G
+        ks, vs = [], []
+        for p in plist:
+            blk = int(cache.block_table[b, p])
+            n = min(B, lens[b] - p * B)
+            ks.append(page(cache.k, blk, h)[:n]); vs.append(page(cache.v, blk, h)[:n])
+        ks, vs = np.concatenate(ks), np.concatenate(vs)
+        x = ks @ q[b, gq] / math.sqrt(d)
+        wgt = np.exp(x - x.max())
+        return (wgt / wgt.sum()) @ vs, x.max() + math.log(wgt.sum())
+
+    out, lse = oracle.attend(cache, q_raw, SM, ids, cnt)
+    dense, dlse = oracle.attend(cache, q_raw, SM)
+    sids, scnt, sout, slse = oracle.decode_step(cache, q_raw, r, fmt, summ, SM, k)
+    assert np.array_equal(sids, ids) and np.array_equal(scnt, cnt)
+    assert np.array_equal(sout, out) and np.array_equal(slse, lse)
+    for b in range(3):
+        for gq in range(Hq):
+            o, l = attend_ref(b, gq, ids[b, gq // G, :k].tolist())
+            assert np.allclose(out[b, gq], o, atol=1e-12) and abs(lse[b, gq] - l) < 1e-12
+            o, l = attend_ref(b, gq, range(pages[b]))
+            assert np.allclose(dense[b, gq], o, atol=1e-12) and abs(dlse[b, gq] - l) < 1e-12
+
+
+def test_build_summaries_page_ranges_per_request():
+    """page_begin / page_end are per request: only the named complete pages are written."""
+    cache, _, _, page, lens, pages = ragged_batch_cache()
+    r, fmt = 8, oracle.FMT_I4
+    full = oracle.build_summaries(cache, r, fmt)
+    part = oracle.build_summaries(cache, r, fmt, page_begin=[2, 0, 11], page_end=[4, 0, 99])
+    want = {(0, 2), (0, 3), (2, 11)}                                   # request 2 has 12 complete pages: 11 is the last
+    for b in range(3):
+        for p in range(pages[b]):
+            blk = int(cache.block_table[b, p])
+            if (b, p) in want:
+                assert np.array_equal(part[blk], full[blk]) and part[blk].any()
+            else:
+                assert not part[blk].any()

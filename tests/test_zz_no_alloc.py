@@ -1,4 +1,4 @@
-"""The allocation-free sparse-attention entry point against the regular one.
+"""The allocation-free sparse-attention entry point against the regular one and against the oracle.
 
 Some callers of the library cannot allocate device memory (a plugin inside an engine that owns the
 whole device's memory pool, a path that must not synchronise, a fixed memory budget), so they have no
@@ -28,6 +28,9 @@ def test_noalloc_entry_point_matches_workspace_entry_point_twice():
     summ = gc.gpu_build()
     ids, cnt, _, _ = gc.gpu_select(summ)
     ref, ref_lse = gc.gpu_attend(ids, cnt)                      # existing entry point (context + workspace)
+    import oracle
+    from common import t2np
+    ora, ora_lse = oracle.attend(gc.cache, t2np(gc.case.q), gc.sm, ids, cnt)   # and the definition itself
     ids_d = torch.as_tensor(ids, device="cuda:0").contiguous()
     cnt_d = torch.as_tensor(cnt, device="cuda:0").contiguous()
     for call in range(2):                                       # two calls in a row share the built-in array
@@ -38,6 +41,7 @@ def test_noalloc_entry_point_matches_workspace_entry_point_twice():
         got = out.float().cpu().numpy().astype(np.float64)
         assert np.abs(got - ref).max() <= 2e-2, (call, np.abs(got - ref).max())
         assert np.abs(lse.cpu().numpy() - ref_lse).max() <= 1e-3, call
+        assert np.abs(got - ora).max() <= 2e-2 and np.abs(lse.cpu().numpy() - ora_lse).max() <= 1e-3, call
     # dense mode (no page table) through the same entry point
     dref, dref_lse = gc.gpu_attend()
     out = torch.empty(w.n, w.Hq, w.d, dtype=torch.bfloat16, device="cuda:0")
