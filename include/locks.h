@@ -121,6 +121,30 @@ int locks_select(locks_ctx *ctx, const void *q, const void *summaries, const loc
                  int32_t *page_ids, int32_t *page_count, float *page_logmass, float *page_logshare,
                  locks_stream stream);
 
+/* The exact-LSE arm (Lemma 1(ii); the "Oracle" / "exact LSE (ceiling)" rows of the paper's tables): the same
+ * selection as locks_select, but ranked by the exact page log-mass s_j(q_g) = log sum_{i in P_j} exp(q_g.k_i/sqrt(d))
+ * computed from the K pages themselves (reads 4 KB per (page, KV head): a diagnostic, not the hot path).  Same
+ * share-average combine, candidates, tie rule and outputs as locks_select, except that page_logmass (optional,
+ * [batch][Hq][max_pages_per_seq]) receives the exact mass of ALL pages 0..P-1 (the last page over its valid
+ * tokens), which locks_selection_quality needs. */
+int locks_select_exact(locks_ctx *ctx, const void *q, const locks_kv *kv, int batch, int32_t *page_ids,
+                       int32_t *page_count, float *page_logmass, float *page_logshare, locks_stream stream);
+
+/* Selection fidelity of a page table against exact masses (the paper's App. B "microscope" metrics), per
+ * (request, KV head), means over the heads of the group:
+ *   quality[(b*Hkv + h)*4 + 0] = gamma    total attention mass captured:  sum_{j in S} e^{s_j} / sum_{j<P} e^{s_j}
+ *                         + 1] = gamma_c  contested mass: pages 0 and P-1 (always kept) taken out of numerator and
+ *                                         denominator
+ *                         + 2] = recall   overlap of the candidate pages of S with those of the reference table
+ *                         + 3] = needle   of the marked pages the reference table keeps, the fraction S keeps too
+ *   exact_logmass [batch][Hq][max_pages_per_seq] from locks_select_exact; (page_ids, page_count) the table under
+ *   test; (ref_ids, ref_count) the reference (locks_select_exact's); marked_pages [batch][n_marked] logical pages
+ *   (-1 = unused slot) or NULL with n_marked = 0 (needle then reads 1).  An empty denominator reads 1. */
+int locks_selection_quality(locks_ctx *ctx, const float *exact_logmass, const locks_kv *kv, int batch,
+                            const int32_t *page_ids, const int32_t *page_count, const int32_t *ref_ids,
+                            const int32_t *ref_count, const int32_t *marked_pages, int n_marked, float *quality,
+                            locks_stream stream);
+
 /* Stage B, sparse paged attention (Sec. 3 "Decode-time attention"; App. E): for every query head,
  * softmax(q.k_i/sqrt(d))-weighted mean of v_i over the tokens i < T_b of the listed pages
  * (split over CTAs, partial results merged by log-sum-exp).  page_ids == NULL: every page, i.e.

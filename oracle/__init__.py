@@ -234,6 +234,27 @@ def select(cache: Cache, shat, k: int):
     return ids, cnt, logshare
 
 
+def page_exact_mass_all(cache: Cache, q, sm_scale: float):
+    """Exact log-mass of every page 0..P-1 (last page over its valid tokens): [batch, Hq, max_pages]."""
+    q, qd = _q_arg(q)
+    mass = np.full((cache.batch, cache.Hq, cache.max_pages), np.nan)
+    lib().ora_page_exact_mass_all(cache.ref(), C.c_int(cache.batch), _p(q), C.c_int(qd), C.c_double(sm_scale), _p(mass))
+    return mass
+
+
+def selection_quality(s, P: int, A, R, marked=()):
+    """s [G, >=P] exact page log-masses of one KV head; A, R page lists -> (gamma, gamma_c, recall, needle)."""
+    s = _f64(s)
+    G, ld = s.shape
+    A = np.ascontiguousarray(A, dtype=np.int32)
+    R = np.ascontiguousarray(R, dtype=np.int32)
+    M = np.ascontiguousarray(marked, dtype=np.int32)
+    out = np.zeros(4)
+    lib().ora_selection_quality(C.c_int(P), C.c_int(G), _p(s), C.c_int64(ld), _p(A), C.c_int(A.size), _p(R),
+                                C.c_int(R.size), _p(M) if M.size else None, C.c_int(M.size), _p(out))
+    return tuple(float(x) for x in out)
+
+
 def attend(cache: Cache, q, sm_scale: float, page_ids=None, page_count=None):
     q, qd = _q_arg(q)
     out = np.zeros((cache.batch, cache.Hq, cache.d))

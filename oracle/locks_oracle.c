@@ -592,6 +592,72 @@ void ora_attend(const ora_kv *kv, int batch, const void *q, int q_dtype, double 
     }
 }
 
+/* Exact log-mass of EVERY page 0..P-1 (the last page over its valid tokens), Lemma 1(ii):
+ * mass[(b*Hq + g)*max_pages + p].  Other entries are left untouched. */
+void ora_page_exact_mass_all(const ora_kv *kv, int batch, const void *q, int q_dtype, double sm_scale,
+                             double *mass) {
+  int B = kv->B, d = kv->d, G = kv->Hq / kv->Hkv;
+#pragma omp parallel for collapse(2) num_threads(g_threads) schedule(dynamic)
+  for (int b = 0; b < batch; ++b)
+    for (int h = 0; h < kv->Hkv; ++h) {
+      int T = kv->seq_lens[b], P = num_pages(T, B);
+      double *keys = (double *)malloc(sizeof(double) * B * d);
+      double *qd = (double *)malloc(sizeof(double) * d);
+      for (int p = 0; p < P; ++p) {
+        int ntok = T - p * B < B ? T - p * B : B;
+        int block = kv->block_table[(int64_t)b * kv->max_pages + p];
+        load_page_keys(kv, kv->k, block, h, ntok, keys);
+        for (int gi = 0; gi < G; ++gi) {
+          int g = h * G + gi;
+          for (int c = 0; c < d; ++c) qd[c] = load_elem(q, q_dtype, ((int64_t)b * kv->Hq + g) * d + c);
+          mass[((int64_t)b * kv->Hq + g) * kv->max_pages + p] = ora_exact_lse(ntok, d, keys, qd, sm_scale);
+        }
+      }
+      free(keys); free(qd);
+    }
+}
+
+/* Selection fidelity of a page set A against exact page log-masses (App. B, selection-fidelity table), for one
+ * KV head of one request, averaged over its G query heads.  s: G rows (stride ld) of exact log-masses of pages
+ * 0..P-1.  A / R: page lists of the table under test / of the reference ranking.  marked: pages of interest
+ * ("carriers"; entries outside 1..P-2 are ignored).
+ *   out[0] gamma   = sum_{j in A} e^{s_j} / sum_{j<P} e^{s_j}
+ *   out[1] gamma_c = the same with pages 0 and P-1 removed from numerator and denominator
+ *   out[2] recall  = |A n R| / |R| counted over candidate pages 1..P-2
+ *   out[3] needle  = |marked n R n A| / |marked n R|
+ * An empty denominator reads 1. */
+void ora_selection_quality(int P, int G, const double *s, int64_t ld, const int32_t *A, int na,
+                           const int32_t *R, int nr, const int32_t *marked, int nm, double *out) {
+  double gam = 0, gamc = 0;
+  for (int g = 0; g < G; ++g) {
+    const double *sg = s + g * ld;
+    double mx = -INFINITY, z = 0, kept = 0, always;
+    for (int j = 0; j < P; ++j) if (sg[j] > mx) mx = sg[j];
+    for (int j = 0; j < P; ++j) z += exp(sg[j] - mx);
+    for (int i = 0; i < na; ++i) if (A[i] >= 0 && A[i] < P) kept += exp(sg[A[i]] - mx);
+    always = exp(sg[0] - mx) + (P > 1 ? exp(sg[P - 1] - mx) : 0.0);
+    gam += kept / z;
+    gamc += (z - always > 0) ? (kept - always > 0 ? kept - always : 0.0) / (z - always) : 1.0;
+  }
+  out[0] = gam / G;
+  out[1] = gamc / G;
+  int hit = 0, tot = 0, nk = 0, nh = 0;
+  for (int j = 0; j < nr; ++j) {
+    if (R[j] <= 0 || R[j] >= P - 1) continue;
+    ++tot;
+    for (int i = 0; i < na; ++i) if (A[i] == R[j]) { ++hit; break; }
+  }
+  for (int j = 0; j < nm; ++j) {
+    int in_r = 0, in_a = 0;
+    if (marked[j] <= 0 || marked[j] >= P - 1) continue;
+    for (int i = 0; i < nr; ++i) in_r |= R[i] == marked[j];
+    for (int i = 0; i < na; ++i) in_a |= A[i] == marked[j];
+    if (in_r) { ++nk; nh += in_a; }
+  }
+  out[2] = tot ? (double)hit / tot : 1.0;
+  out[3] = nk ? (double)nh / nk : 1.0;
+}
+
 /* One decode step on resident summaries: score -> select -> attend (the timed CPU baseline).
  * shat is caller-provided scratch [batch, Hq, max_pages]. */
 void ora_decode_step(const ora_kv *kv, int batch, const void *q, int q_dtype, int r, int fmt,

@@ -18,7 +18,7 @@ SYMBOLS = ["locks_summary_bytes", "locks_workspace_bytes", "locks_create", "lock
            "locks_decode_step_host", "locks_poll_status", "locks_last_launch_count", "locks_strerror",
            "locks_profile_begin", "locks_profile_end", "locks_profile_read", "locks_sparse_attend_noalloc",
            "locks_set_scan_partition", "locks_selftest_wait_timeout", "locks_last_scan_partition",
-           "locks_host_cache_clear"]
+           "locks_host_cache_clear", "locks_select_exact", "locks_selection_quality"]
 
 
 PARTITION_AUTO, PARTITION_STRIDED, PARTITION_BALANCED = 0, 1, 2   # LOCKS_PARTITION_* of include/locks.h
@@ -86,6 +86,10 @@ def lib():
         L.locks_last_scan_partition.restype = C.c_int
         L.locks_host_cache_clear.argtypes = [vp]
         L.locks_host_cache_clear.restype = C.c_int
+        L.locks_select_exact.argtypes = [vp, vp, C.POINTER(KV), C.c_int, i32p, i32p, vp, vp, vp]
+        L.locks_select_exact.restype = C.c_int
+        L.locks_selection_quality.argtypes = [vp, vp, C.POINTER(KV), C.c_int, i32p, i32p, i32p, i32p, i32p, C.c_int, vp, vp]
+        L.locks_selection_quality.restype = C.c_int
         L.locks_strerror.restype = C.c_char_p
         L.locks_strerror.argtypes = [C.c_int]
         for fn in ("locks_create", "locks_destroy", "locks_build_summaries", "locks_select", "locks_sparse_attend",
@@ -196,6 +200,20 @@ class Context:
         _check(lib().locks_select(self.handle, _ptr(q), _ptr(summaries), C.byref(s), batch, _ptr(page_ids),
                                   _ptr(page_count), _ptr(page_logmass), _ptr(page_logshare), _stream(stream)),
                "locks_select")
+
+    def locks_select_exact(self, q, kv: KVView, batch, page_ids, page_count, page_logmass=None, page_logshare=None,
+                           stream=None):
+        s = kv.struct()
+        _check(lib().locks_select_exact(self.handle, _ptr(q), C.byref(s), batch, _ptr(page_ids), _ptr(page_count),
+                                        _ptr(page_logmass), _ptr(page_logshare), _stream(stream)), "locks_select_exact")
+
+    def locks_selection_quality(self, exact_logmass, kv: KVView, batch, page_ids, page_count, ref_ids, ref_count,
+                                quality, marked_pages=None, stream=None):
+        s = kv.struct()
+        n_marked = 0 if marked_pages is None else int(marked_pages.shape[-1])
+        _check(lib().locks_selection_quality(self.handle, _ptr(exact_logmass), C.byref(s), batch, _ptr(page_ids),
+                                             _ptr(page_count), _ptr(ref_ids), _ptr(ref_count), _ptr(marked_pages),
+                                             n_marked, _ptr(quality), _stream(stream)), "locks_selection_quality")
 
     def locks_sparse_attend(self, q, kv: KVView, batch, page_ids, page_count, out, lse=None, stream=None):
         s = kv.struct()

@@ -289,6 +289,32 @@ int locks_select(locks_ctx *ctx, const void *q, const void *summaries, const loc
   return locks_launch_select(ctx, shat, kv, batch, page_ids, page_count, page_logshare, nullptr, st);
 }
 
+int locks_select_exact(locks_ctx *ctx, const void *q, const locks_kv *kv, int batch, int32_t *page_ids,
+                       int32_t *page_count, float *page_logmass, float *page_logshare, locks_stream stream) {
+  int rc = check_common(ctx, kv, batch);
+  if (rc != LOCKS_OK) return rc;
+  if (!q || !page_ids || !page_count || ((uintptr_t)q % 16)) return LOCKS_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  ctx->last_launches = 0;
+  float *shat = page_logmass ? page_logmass : ctx->shat;
+  if ((rc = locks_launch_exact_scan(ctx, q, kv, batch, shat, st)) != LOCKS_OK) return rc;
+  return locks_launch_select(ctx, shat, kv, batch, page_ids, page_count, page_logshare, nullptr, st);
+}
+
+int locks_selection_quality(locks_ctx *ctx, const float *exact_logmass, const locks_kv *kv, int batch,
+                            const int32_t *page_ids, const int32_t *page_count, const int32_t *ref_ids,
+                            const int32_t *ref_count, const int32_t *marked_pages, int n_marked, float *quality,
+                            locks_stream stream) {
+  int rc = check_common(ctx, kv, batch);
+  if (rc != LOCKS_OK) return rc;
+  if (!exact_logmass || !page_ids || !page_count || !ref_ids || !ref_count || !quality || n_marked < 0 ||
+      (n_marked > 0 && !marked_pages))
+    return LOCKS_ERR_INVALID_ARG;
+  ctx->last_launches = 0;
+  return locks_launch_quality(ctx, exact_logmass, kv, batch, page_ids, page_count, ref_ids, ref_count, marked_pages,
+                              n_marked, quality, (cudaStream_t)stream);
+}
+
 int locks_sparse_attend(locks_ctx *ctx, const void *q, const locks_kv *kv, int batch, const int32_t *page_ids,
                         const int32_t *page_count, void *out, float *lse, locks_stream stream) {
   int rc = check_common(ctx, kv, batch);

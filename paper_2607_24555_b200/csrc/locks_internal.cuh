@@ -149,6 +149,11 @@ int locks_launch_build(locks_ctx *c, const locks_kv *kv, int batch, const int32_
                        int just_filled, void *summaries, const void *k_new, const int32_t *append_pos,
                        cudaStream_t st);
 
+int locks_launch_exact_scan(locks_ctx *c, const void *q, const locks_kv *kv, int batch, float *shat, cudaStream_t st);
+int locks_launch_quality(locks_ctx *c, const float *mass, const locks_kv *kv, int batch, const int32_t *ids_a,
+                         const int32_t *cnt_a, const int32_t *ids_r, const int32_t *cnt_r, const int32_t *marked,
+                         int n_marked, float *out, cudaStream_t st);
+
 // Launch with programmatic dependent launch allowed: the kernel may be scheduled while its stream
 // predecessor is still draining; it must execute pdl_wait() before touching anything the predecessor
 // writes (the wait returns once the predecessor grid has completed and its writes are visible).

@@ -432,11 +432,20 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4_kerne
   };
 
   Cursor cc;
+  // strided partition: the first group's position does not depend on the lengths, so its block ids are fetched
+  // beside the length instead of after it (block-table slots past a sequence's pages are readable, just unused)
+  int spec_block = 0;
+  if (!BAL && slot < nprob && lane < LOCKS_GROUP && sub * LOCKS_GROUP + lane < p.Pmax)
+    spec_block = p.block_table[(int64_t)(slot / p.Hkv) * p.Pmax + sub * LOCKS_GROUP + lane];
   if (cp.prob < nprob) enter(cp);
   settle(cp);
   cc = cp;
   int inflight = 0;
-  int next_block = fetch_block(cp);
+  int next_block;
+  if (!BAL && cp.prob == slot && cp.grp == sub)
+    next_block = (lane < LOCKS_GROUP && sub * LOCKS_GROUP + lane < cp.nsc) ? spec_block : 0;
+  else
+    next_block = fetch_block(cp);
 #pragma unroll
   for (int s = 0; s < kScanStages; ++s) {
     if (cp.prob < nprob) {
@@ -547,18 +556,9 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4_kerne
   while (cc.prob < nprob) {
     const int stage = it % kScanStages;
     const uint32_t parity = (it / kScanStages) & 1;
-    if (kScanBulk) {
-      if (!mbar_wait(&full[stage], parity)) {
-        ok = false;
-        break;
-      }
-    } else {
-      // groups complete in order: all but the newest (kScanStages - 1) committed groups must have landed
-      if (inflight >= kScanStages) cp_async_wait<kScanStages - 1>(); else cp_async_wait<0>();
-      __syncwarp();
-    }
-    --inflight;
     const int b = cc.b, h = cc.h;
+    // a new problem's query is fetched and normalised BEFORE waiting for the group's summaries, so that the
+    // round trip of the query load runs beside the copy instead of after it
     if (cc.prob != cur_prob) {
       if (cur_prob >= 0) flush(false, true);
       cur_prob = cc.prob;
@@ -577,6 +577,17 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4_kerne
         inv2[2 * hh + 1] = __shfl_sync(0xffffffffu, inv_s[hh], (2 * t + 1) * 4);
       }
     }
+    if (kScanBulk) {
+      if (!mbar_wait(&full[stage], parity)) {
+        ok = false;
+        break;
+      }
+    } else {
+      // groups complete in order: all but the newest (kScanStages - 1) committed groups must have landed
+      if (inflight >= kScanStages) cp_async_wait<kScanStages - 1>(); else cp_async_wait<0>();
+      __syncwarp();
+    }
+    --inflight;
 
     const uint8_t *sb = ring + stage * kStageBytes;
     // ---- centroid dots of the 8 pages.  Pages are the MMA rows (rows 8-15 idle) and the query is the B operand,

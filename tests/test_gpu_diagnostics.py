@@ -1,0 +1,92 @@
+"""GPU parity of the diagnostics: the exact-LSE selection arm (Lemma 1(ii)) and the selection-fidelity metrics
+(App. B) against the oracle, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+import locks_synth
+import oracle
+from common import check_page_sets, t2np
+
+pytestmark = pytest.mark.gpu
+
+
+def _gc(w, **kw):
+    from gpu_util import GpuCase
+    return GpuCase(w, **kw)
+
+
+def _exact(gc):
+    w = gc.w
+    ids = torch.full((w.n, w.Hkv, gc.k), -7, dtype=torch.int32, device="cuda:0")
+    cnt = torch.full((w.n, w.Hkv), -7, dtype=torch.int32, device="cuda:0")
+    mass = torch.full((w.n, w.Hq, gc.max_pages), float("nan"), dtype=torch.float32, device="cuda:0")
+    share = torch.full((w.n, w.Hkv, gc.max_pages), float("nan"), dtype=torch.float32, device="cuda:0")
+    gc.ctx.locks_select_exact(gc.case.q, gc.kv, w.n, ids, cnt, mass, share)
+    torch.cuda.synchronize()
+    return ids, cnt, mass, share
+
+
+def _check_exact(gc, tol):
+    w = gc.w
+    ids, cnt, mass, share = _exact(gc)
+    omass = oracle.page_exact_mass_all(gc.cache, t2np(gc.case.q), gc.sm)
+    oids, ocnt, oshare = oracle.select(gc.cache, omass, gc.k)
+    gm, gs = mass.cpu().numpy(), share.cpu().numpy()
+    for b, T in enumerate(gc.cache.seq_lens):
+        P = -(-int(T) // w.B)
+        assert np.abs(gm[b, :, :P] - omass[b, :, :P]).max() <= tol, b         # every page, the partial tail included
+        if P > gc.k:
+            assert np.abs(gs[b, :, 1:P - 1] - oshare[b, :, 1:P - 1]).max() <= tol
+    check_page_sets(ids.cpu().numpy(), cnt.cpu().numpy(), oids, ocnt, oshare, gc.cache.seq_lens, w.B, gc.k)
+    assert gc.status() == 0
+    return ids, cnt, mass, omass, oids, ocnt
+
+
+@pytest.mark.parametrize("Hq,Hkv", [(8, 2), (32, 2), (6, 2), (4, 4)])
+def test_exact_selection_matches_oracle(Hq, Hkv):
+    gc = _gc(locks_synth.Workload("exact", [16 * 700 + 5, 16 * 64, 300, 16 * 65 + 1], Hq=Hq, Hkv=Hkv, budget=256,
+                                  carriers=4, seed=Hq))
+    _check_exact(gc, 1e-3)
+
+
+def test_exact_selection_fp32_config0():
+    gc = _gc(locks_synth.config0())
+    ids, cnt, mass, omass, oids, ocnt = _check_exact(gc, 1e-4)
+    assert np.array_equal(ids.cpu().numpy(), oids)
+    for cp in gc.case.carrier_pages[0]:
+        assert cp in oids[0, 0].tolist()
+
+
+def test_selection_quality_matches_oracle_and_estimator_tracks_the_ceiling():
+    """gamma, gamma_c, recall and needle of the estimated selection against the exact arm: the kernel's numbers
+    equal the oracle's on the same tables, and on locally low-rank keys the rank-8 summary keeps nearly all of
+    the mass the exact ranking keeps (the paper's selection-fidelity table: gamma within a point of the ceiling)."""
+    w = locks_synth.Workload("quality", [16 * 1500 + 3, 16 * 900], Hq=8, Hkv=2, budget=512, carriers=8, q_scale=0.5, seed=12)
+    gc = _gc(w)
+    summ = gc.gpu_build()
+    ids_e, cnt_e, mass, _ = _exact(gc)
+    ids_s, cnt_s, _, _ = gc.gpu_select(summ)
+    ids_s = torch.from_numpy(ids_s).cuda(); cnt_s = torch.from_numpy(cnt_s).cuda()
+    marked = torch.tensor([cp[:8] for cp in gc.case.carrier_pages], dtype=torch.int32, device="cuda:0")
+    qual = torch.full((w.n, w.Hkv, 4), float("nan"), dtype=torch.float32, device="cuda:0")
+    ceil_ = torch.full((w.n, w.Hkv, 4), float("nan"), dtype=torch.float32, device="cuda:0")
+    gc.ctx.locks_selection_quality(mass, gc.kv, w.n, ids_s, cnt_s, ids_e, cnt_e, qual, marked_pages=marked)
+    gc.ctx.locks_selection_quality(mass, gc.kv, w.n, ids_e, cnt_e, ids_e, cnt_e, ceil_, marked_pages=marked)
+    torch.cuda.synchronize()
+    omass = oracle.page_exact_mass_all(gc.cache, t2np(gc.case.q), gc.sm)
+    G = w.Hq // w.Hkv
+    for b in range(w.n):
+        P = -(-w.seq_lens[b] // w.B)
+        for h in range(w.Hkv):
+            A = ids_s[b, h, :int(cnt_s[b, h])].cpu().numpy()
+            R = ids_e[b, h, :int(cnt_e[b, h])].cpu().numpy()
+            want = oracle.selection_quality(omass[b, h * G:(h + 1) * G], P, A, R, marked[b].cpu().numpy())
+            assert np.abs(qual[b, h].cpu().numpy() - np.array(want)).max() <= 2e-3, (b, h, qual[b, h], want)
+            want_c = oracle.selection_quality(omass[b, h * G:(h + 1) * G], P, R, R, marked[b].cpu().numpy())
+            assert np.abs(ceil_[b, h].cpu().numpy() - np.array(want_c)).max() <= 2e-3
+    q_, c_ = qual.cpu().numpy(), ceil_.cpu().numpy()
+    assert np.all(c_[..., 2] == 1.0) and np.all(c_[..., 3] == 1.0)
+    assert np.all(q_[..., 0] >= c_[..., 0] - 0.02)        # total mass within two points of the ceiling
+    assert np.all(q_[..., 3] >= 0.99)                     # carriers the exact ranking keeps are kept
+    assert gc.status() == 0

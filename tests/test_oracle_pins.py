@@ -589,3 +589,42 @@ def test_build_summaries_page_ranges_per_request():
                 assert np.array_equal(part[blk], full[blk]) and part[blk].any()
             else:
                 assert not part[blk].any()
+
+
+# ------------------------------------------------------------------ selection fidelity metrics (App. B)
+
+def test_selection_quality_closed_forms_and_token_level_softmax():
+    """gamma, gamma_c, recall, needle: hand-computable cases, and gamma against the token-level softmax mass of the
+    selected pages computed straight from numpy (the quantity Lemma 1 calls gamma_S)."""
+    P = 6
+    s = np.log(np.array([[1.0, 2.0, 3.0, 4.0, 5.0, 5.0], [6.0, 1.0, 1.0, 1.0, 1.0, 10.0]]))
+    A, R = [0, 2, 3, 5], [0, 3, 4, 5]
+    gam, gamc, rec, ndl = oracle.selection_quality(s, P, A, R, marked=[3, 4, 1, 0, 99])
+    assert abs(gam - 0.5 * ((1 + 3 + 4 + 5) / 20.0 + (6 + 1 + 1 + 10) / 20.0)) < 1e-14
+    assert abs(gamc - 0.5 * ((3 + 4) / 14.0 + (1 + 1) / 4.0)) < 1e-14
+    assert rec == 0.5                      # candidates of R: {3, 4}; A keeps 3
+    assert ndl == 0.5                      # marked candidates R keeps: {3, 4}; A keeps 3 (1 is not in R; 0, 99 ignored)
+    assert oracle.selection_quality(s, P, list(range(P)), R)[:3] == (1.0, 1.0, 1.0)
+    g2 = oracle.selection_quality(s, P, [0, 5], [0, 5])
+    assert g2[1] == 0.0 and g2[2] == 1.0 and g2[3] == 1.0
+    # against the definition at token level on a random cache (partial last page)
+    cache, g = tiny_cache(T=93, Hq=4, Hkv=2)
+    q = g.standard_normal((1, 4, 128)).astype(np.float32)
+    mass = oracle.page_exact_mass_all(cache, q, SM)
+    Pn, Bsz = 6, 16
+    assert np.all(np.isfinite(mass[0, :, :Pn]))
+    sel = [0, 2, 5]
+    for h in range(2):
+        want = 0.0
+        for gq in (2 * h, 2 * h + 1):
+            ks = np.concatenate([cache.k[cache.block_table[0, p], h, :min(Bsz, 93 - p * Bsz)] for p in range(Pn)])
+            x = ks.astype(np.float64) @ q[0, gq].astype(np.float64) / math.sqrt(128)
+            wgt = np.exp(x - x.max()); wgt /= wgt.sum()
+            want += sum(wgt[p * Bsz:min((p + 1) * Bsz, 93)].sum() for p in sel) / 2
+            # a page's exact log-mass is the log of its tokens' summed exponentials
+            assert abs(mass[0, gq, 5] - math.log(np.exp(x[80:93]).sum())) < 1e-12
+        got = oracle.selection_quality(mass[0, 2 * h:2 * h + 2], Pn, sel, sel)[0]
+        assert abs(got - want) < 1e-13
+    # pages 0..P-2 agree with the candidate-only exact arm
+    part = oracle.page_logmass(cache, q, 8, oracle.FMT_F32, None, SM, exact=True)
+    assert np.array_equal(part[0, :, :Pn - 1], mass[0, :, :Pn - 1])
