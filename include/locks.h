@@ -47,6 +47,16 @@ extern "C" {
 #define LOCKS_FMT_F32 0 /* summary stored as fp32 mu, V, C                               */
 #define LOCKS_FMT_I4 1  /* int4 basis, int8 coefficients + centroid, fp16 scales (r8i4)  */
 
+/* How the G query heads of a KV head are combined into one ranking key per page (Sec. 4; ablated in the
+ * paper's App. D "GQA combine" table).  The selection (sink + most recent + top k-2 by key, ties to the lower
+ * page) is the same for all; page_logshare receives the key.
+ *   LOCKS_COMBINE_SHARE_AVG   log mean_g exp(s^_j(q_g) - log Z_g): the paper's rule (Cor. 4)
+ *   LOCKS_COMBINE_GROUP_MAX   max_g s^_j(q_g): the largest raw page log-mass of the group
+ *   LOCKS_COMBINE_GROUP_MASS  log sum_g exp s^_j(q_g): the group's summed, un-normalised page mass */
+#define LOCKS_COMBINE_SHARE_AVG 0
+#define LOCKS_COMBINE_GROUP_MAX 1
+#define LOCKS_COMBINE_GROUP_MASS 2
+
 typedef struct locks_ctx locks_ctx;
 typedef void *locks_stream; /* cudaStream_t */
 
@@ -63,6 +73,7 @@ typedef struct {
   int32_t max_pages_per_seq; /* row length of block_table                                     */
   int32_t budget_tokens;     /* b; k = ceil(b/B) >= 2                                         */
   float sm_scale;            /* logit scale, 1/sqrt(d) in the paper                           */
+  int32_t combine;           /* LOCKS_COMBINE_*: how a group's heads share one page table (0 = the paper's)   */
 } locks_config;
 
 /* Paged KV cache view.  Element (block, kv head, token-in-page, dim) of K lives at

@@ -55,6 +55,7 @@ def lib():
         L.ora_exact_lse.restype = C.c_double
         L.ora_build_page.restype = C.c_int
         L.ora_select_one.restype = C.c_int
+        L.ora_select_one_rule.restype = C.c_int
         L.ora_get_max_threads.restype = C.c_int
         _lib = L
     return _lib
@@ -158,6 +159,20 @@ def select_one(s, P: int, k: int):
     logshare = np.full(max(P, 1), np.nan)
     cnt = lib().ora_select_one(C.c_int(P), C.c_int(G), C.c_int(k), _p(s), C.c_int64(ld), _p(ids), _p(logshare))
     return ids, int(cnt), logshare
+
+
+RULE_SHARE_AVG, RULE_GROUP_MAX, RULE_GROUP_MASS = 0, 1, 2
+
+
+def select_one_rule(s, P: int, k: int, rule: int):
+    """select_one under one of the ablated combine rules -> (ids, count, ranking key [P])."""
+    s = _f64(s)
+    G, ld = s.shape
+    ids = np.full(k, -1, np.int32)
+    key = np.full(max(P, 1), np.nan)
+    cnt = lib().ora_select_one_rule(C.c_int(P), C.c_int(G), C.c_int(k), _p(s), C.c_int64(ld), C.c_int(rule), _p(ids),
+                                    _p(key))
+    return ids, int(cnt), key
 
 
 # ----------------------------------------------------------------------------- batch level

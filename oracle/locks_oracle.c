@@ -533,6 +533,37 @@ int ora_select_one(int P, int G, int k, const double *s, int64_t ld, int32_t *id
   return cnt;
 }
 
+/* The combine rules the paper ablates against its own (App. D, GQA combine table), same selection otherwise:
+ * rule 0 share-average (ora_select_one), rule 1 group-max: key_j = max_g s_j(q_g), rule 2 group-mass:
+ * key_j = log sum_g exp s_j(q_g).  key (optional, length >= P) receives the ranking key of the candidates. */
+int ora_select_one_rule(int P, int G, int k, const double *s, int64_t ld, int rule, int32_t *ids, double *key) {
+  if (rule == 0) return ora_select_one(P, G, k, s, ld, ids, key);
+  if (P <= k) {
+    for (int j = 0; j < k; ++j) ids[j] = j < P ? j : -1;
+    return P;
+  }
+  double *kk = (double *)malloc(sizeof(double) * P);
+  char *taken = (char *)calloc(P, 1);
+  for (int j = 1; j <= P - 2; ++j) {
+    double mx = -INFINITY, z = 0;
+    for (int g = 0; g < G; ++g) if (s[g * ld + j] > mx) mx = s[g * ld + j];
+    for (int g = 0; g < G; ++g) z += exp(s[g * ld + j] - mx);
+    kk[j] = rule == 1 ? mx : mx + log(z);
+    if (key) key[j] = kk[j];
+  }
+  taken[0] = 1; taken[P - 1] = 1;
+  for (int n = 0; n < k - 2; ++n) {
+    int best = -1;
+    for (int j = 1; j <= P - 2; ++j)
+      if (!taken[j] && (best < 0 || kk[j] > kk[best])) best = j;
+    taken[best] = 1;
+  }
+  int cnt = 0;
+  for (int j = 0; j < P; ++j) if (taken[j]) ids[cnt++] = j;
+  free(kk); free(taken);
+  return cnt;
+}
+
 void ora_select(const ora_kv *kv, int batch, int k, const double *shat, int32_t *page_ids,
                 int32_t *page_count, double *logshare) {
   int G = kv->Hq / kv->Hkv;

@@ -32,7 +32,8 @@ class Config(C.Structure):
     _fields_ = [("head_dim", C.c_int32), ("page_size", C.c_int32), ("num_q_heads", C.c_int32),
                 ("num_kv_heads", C.c_int32), ("rank", C.c_int32), ("summary_fmt", C.c_int32),
                 ("kv_dtype", C.c_int32), ("q_dtype", C.c_int32), ("max_batch", C.c_int32),
-                ("max_pages_per_seq", C.c_int32), ("budget_tokens", C.c_int32), ("sm_scale", C.c_float)]
+                ("max_pages_per_seq", C.c_int32), ("budget_tokens", C.c_int32), ("sm_scale", C.c_float),
+                ("combine", C.c_int32)]
 
 
 class KV(C.Structure):
@@ -132,12 +133,16 @@ def _stream(stream) -> int:
     return stream.cuda_stream
 
 
-def make_config(Hq, Hkv, rank, fmt, dtype, max_batch, max_pages, budget, sm_scale=None, d=128, B=16) -> Config:
+COMBINE_SHARE_AVG, COMBINE_GROUP_MAX, COMBINE_GROUP_MASS = 0, 1, 2   # LOCKS_COMBINE_* of include/locks.h
+
+
+def make_config(Hq, Hkv, rank, fmt, dtype, max_batch, max_pages, budget, sm_scale=None, d=128, B=16,
+                combine=COMBINE_SHARE_AVG) -> Config:
     if sm_scale is None:
         sm_scale = d ** -0.5
     dt = BF16 if dtype in ("bf16", torch.bfloat16) else F32
     f = FMT_I4 if fmt == "i4" else FMT_F32
-    return Config(d, B, Hq, Hkv, rank, f, dt, dt, max_batch, max_pages, budget, sm_scale)
+    return Config(d, B, Hq, Hkv, rank, f, dt, dt, max_batch, max_pages, budget, sm_scale, combine)
 
 
 @dataclass

@@ -17,6 +17,7 @@ int validate(const locks_config *c) {
   if (c->budget_tokens <= 0 || k < 2) return LOCKS_ERR_INVALID_ARG;
   if (!(c->sm_scale > 0.f)) return LOCKS_ERR_INVALID_ARG;
   if (c->summary_fmt != LOCKS_FMT_F32 && c->summary_fmt != LOCKS_FMT_I4) return LOCKS_ERR_INVALID_ARG;
+  if (c->combine < LOCKS_COMBINE_SHARE_AVG || c->combine > LOCKS_COMBINE_GROUP_MASS) return LOCKS_ERR_INVALID_ARG;
   if ((c->kv_dtype != LOCKS_F32 && c->kv_dtype != LOCKS_BF16) || (c->q_dtype != LOCKS_F32 && c->q_dtype != LOCKS_BF16))
     return LOCKS_ERR_INVALID_ARG;
   if (c->head_dim != LOCKS_D || c->page_size != LOCKS_B) return LOCKS_ERR_UNSUPPORTED;

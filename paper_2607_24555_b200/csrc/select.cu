@@ -36,6 +36,7 @@ struct SelParams {
   int32_t *sel_done;   // [batch][Hkv] chunk-arrival counters (zero between launches)
   int32_t *status;
   int batch, Hq, Hkv, G, Pmax, max_groups, k, chunks, kc, chunk_pages, part_slots;
+  int combine;       // LOCKS_COMBINE_*
   locks_append app;  // decode step only: the new token's K/V rows, written here beside the ranking
 };
 
@@ -303,9 +304,11 @@ __device__ __noinline__ void group_logz(const float2 *part0, int G, int max_grou
 // (0 for pages that are not candidates).  Scores are fetched in batches of (16 / SB) heads x SB slabs, 16
 // loads in flight per thread, the next batch while the current one is reduced; the first batch is in
 // flight during the log Z reduction.  Per page a running (max, sum) over the heads, log2 domain.
+// combine: share-average (the paper's rule) subtracts log Z_g per head and averages; group-mass sums the raw
+// masses (log Z_g = 0, no 1/G); group-max keeps the largest raw score.
 template <int SB>
 __device__ __noinline__ void chunk_keys(const float *shat0, const float2 *part0, float *logshare0, int G, int Pmax,
-                                        int max_groups, int nparts, int c0, int nslab, int P) {
+                                        int max_groups, int nparts, int c0, int nslab, int P, int combine) {
   constexpr int HB = 16 / SB;
   SelShared &sh = shared_state();
   const int tid = threadIdx.x;
@@ -327,8 +330,13 @@ __device__ __noinline__ void chunk_keys(const float *shat0, const float2 *part0,
         x[u][sl] = (ok[sl] && g0 + u < G) ? r[u * Pmax + sl * LOCKS_SEL_THREADS] : -INFINITY;
   };
   load(0, 0, cur);
-  group_logz(part0, G, max_groups, nparts);
-  const float logG = __logf((float)G);
+  if (combine == LOCKS_COMBINE_SHARE_AVG) {
+    group_logz(part0, G, max_groups, nparts);
+  } else {
+    if (tid < 16) sh.lz2[tid] = 0.f;
+    __syncthreads();
+  }
+  const float logG = combine == LOCKS_COMBINE_SHARE_AVG ? __logf((float)G) : 0.f;
   float m[SB], s[SB];
 #pragma unroll
   for (int sl = 0; sl < SB; ++sl) { m[sl] = -INFINITY; s[sl] = 0.f; }
@@ -359,7 +367,7 @@ __device__ __noinline__ void chunk_keys(const float *shat0, const float2 *part0,
         const int i = i0 + sl, page = c0 + i * LOCKS_SEL_THREADS + tid;
         if (i < nslab) {
           const bool valid = page >= 1 && page <= P - 2;
-          const float val = (m[sl] + lg2f(s[sl])) * kLn2 - logG;
+          const float val = (combine == LOCKS_COMBINE_GROUP_MAX ? m[sl] : m[sl] + lg2f(s[sl])) * kLn2 - logG;
           sh.key[i * LOCKS_SEL_THREADS + tid] = valid ? order_key(val) : 0u;
           if (valid && logshare0) logshare0[page] = val;
         }
@@ -448,9 +456,9 @@ __global__ void __launch_bounds__(LOCKS_SEL_THREADS, 2) select_kernel(SelParams 
     float *ls0 = p.logshare ? p.logshare + prob * p.Pmax : nullptr;
     const int nparts = p.part_cnt ? min(max(p.part_cnt[prob], 0), p.max_groups)
                                   : min(p.part_slots, (P - 1 + LOCKS_GROUP - 1) / LOCKS_GROUP);
-    if (nslab >= 3) chunk_keys<4>(shat0, part0, ls0, p.G, p.Pmax, p.max_groups, nparts, c0, nslab, P);
-    else if (nslab == 2) chunk_keys<2>(shat0, part0, ls0, p.G, p.Pmax, p.max_groups, nparts, c0, nslab, P);
-    else chunk_keys<1>(shat0, part0, ls0, p.G, p.Pmax, p.max_groups, nparts, c0, nslab, P);
+    if (nslab >= 3) chunk_keys<4>(shat0, part0, ls0, p.G, p.Pmax, p.max_groups, nparts, c0, nslab, P, p.combine);
+    else if (nslab == 2) chunk_keys<2>(shat0, part0, ls0, p.G, p.Pmax, p.max_groups, nparts, c0, nslab, P, p.combine);
+    else chunk_keys<1>(shat0, part0, ls0, p.G, p.Pmax, p.max_groups, nparts, c0, nslab, P, p.combine);
   }
   const int cand_in_chunk = min(P - 2, c0 + p.chunk_pages - 1) - max(1, c0) + 1;
   const int K = min(p.k - 2, cand_in_chunk);
@@ -486,6 +494,7 @@ int locks_launch_select(locks_ctx *c, const float *shat, const locks_kv *kv, int
   p.max_groups = c->max_groups; p.k = c->k; p.chunks = c->sel_chunks; p.kc = c->sel_kc;
   p.chunk_pages = c->sel_ept * LOCKS_SEL_THREADS;
   p.part_slots = c->part_slots;
+  p.combine = c->cfg.combine;
   p.part_cnt = c->part_balanced ? c->part_cnt : nullptr;
   if (p.chunk_pages > kMaxKeys || (int64_t)c->sel_chunks * c->sel_kc > kMaxKeys || p.G > 16) return LOCKS_ERR_UNSUPPORTED;
   // Two CTAs fit on an SM (64 registers per thread).  That halves the waves of a launch with many more CTAs

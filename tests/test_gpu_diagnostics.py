@@ -90,3 +90,36 @@ def test_selection_quality_matches_oracle_and_estimator_tracks_the_ceiling():
     assert np.all(q_[..., 0] >= c_[..., 0] - 0.02)        # total mass within two points of the ceiling
     assert np.all(q_[..., 3] >= 0.99)                     # carriers the exact ranking keeps are kept
     assert gc.status() == 0
+
+
+@pytest.mark.parametrize("rule", [1, 2])
+@pytest.mark.parametrize("lens,Hq,Hkv", [([16 * 700 + 5, 16 * 90], 8, 2), ([16 * 9000 + 3], 32, 2)])
+def test_combine_rule_switch_matches_oracle(rule, lens, Hq, Hkv):
+    """Group-max and group-mass combine (the rules the paper ablates its share-average against), single- and
+    multi-chunk selection: ranking keys and page sets against the oracle's statement of each rule."""
+    import paper_2607_24555_b200 as locks
+    from paper_2607_24555_b200.binding import make_config
+    gc = _gc(locks_synth.Workload("combine", lens, Hq=Hq, Hkv=Hkv, budget=256, q_scale=0.5, seed=rule + Hq))
+    w = gc.w
+    cfg = make_config(w.Hq, w.Hkv, w.rank, w.fmt, w.dtype, w.n, gc.max_pages, w.budget, combine=rule)
+    ctx = locks.Context(cfg)
+    summ_np = gc.oracle_summaries()
+    summ = torch.from_numpy(summ_np).cuda()
+    ids = torch.full((w.n, w.Hkv, gc.k), -7, dtype=torch.int32, device="cuda:0")
+    cnt = torch.full((w.n, w.Hkv), -7, dtype=torch.int32, device="cuda:0")
+    key = torch.full((w.n, w.Hkv, gc.max_pages), float("nan"), dtype=torch.float32, device="cuda:0")
+    ctx.locks_select(gc.case.q, summ, gc.kv, w.n, ids, cnt, None, key)
+    torch.cuda.synchronize()
+    assert ctx.locks_poll_status() == 0
+    shat = oracle.page_logmass(gc.cache, t2np(gc.case.q), w.rank, gc.fmt, summ_np, gc.sm)
+    G = w.Hq // w.Hkv
+    oids = np.full((w.n, w.Hkv, gc.k), -1, np.int32)
+    ocnt = np.zeros((w.n, w.Hkv), np.int32)
+    okey = np.full((w.n, w.Hkv, gc.max_pages), np.nan)
+    for b in range(w.n):
+        P = -(-w.seq_lens[b] // w.B)
+        for h in range(w.Hkv):
+            oids[b, h], ocnt[b, h], kk = oracle.select_one_rule(shat[b, h * G:(h + 1) * G], P, gc.k, rule)
+            okey[b, h, :P] = kk[:P]
+            assert np.abs(key[b, h, 1:P - 1].cpu().numpy() - kk[1:P - 1]).max() <= 1e-3
+    check_page_sets(ids.cpu().numpy(), cnt.cpu().numpy(), oids, ocnt, okey, gc.cache.seq_lens, w.B, gc.k)

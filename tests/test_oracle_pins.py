@@ -628,3 +628,24 @@ def test_selection_quality_closed_forms_and_token_level_softmax():
     # pages 0..P-2 agree with the candidate-only exact arm
     part = oracle.page_logmass(cache, q, 8, oracle.FMT_F32, None, SM, exact=True)
     assert np.array_equal(part[0, :, :Pn - 1], mass[0, :, :Pn - 1])
+
+
+def test_combine_rules_differ_where_they_should():
+    """Share-average, group-max and group-mass on a hand-made group of two heads with very different partition
+    functions: head 0 has huge raw masses spread evenly, head 1 small raw masses with one page holding nearly all
+    of its share.  Group-max and group-mass follow head 0's raw scores; the share-average keeps head 1's page."""
+    P, k = 8, 3                                                   # one free slot
+    s = np.zeros((2, P))
+    s[0, 1:7] = [10.0, 10.1, 10.2, 10.05, 10.0, 10.0]             # head 0: flat, page 3 barely the largest
+    s[1, 1:7] = [-5.0, -5.0, -5.0, -5.0, 1.0, -5.0]               # head 1: page 5 carries ~99 % of its mass
+    ids0, c0, key0 = oracle.select_one_rule(s, P, k, oracle.RULE_SHARE_AVG)
+    ids1, c1, key1 = oracle.select_one_rule(s, P, k, oracle.RULE_GROUP_MAX)
+    ids2, c2, key2 = oracle.select_one_rule(s, P, k, oracle.RULE_GROUP_MASS)
+    assert ids0.tolist() == [0, 5, 7] and ids1.tolist() == [0, 3, 7] and ids2.tolist() == [0, 3, 7]
+    assert np.array_equal(ids0, oracle.select_one(s, P, k)[0])
+    assert np.allclose(key1[1:7], s[:, 1:7].max(0)) and np.allclose(key2[1:7], np.log(np.exp(s[:, 1:7]).sum(0)))
+    # one head: every rule ranks by the raw score
+    s1 = np.random.default_rng(3).standard_normal((1, 40))
+    want = sorted([0, 39] + (np.argsort(-s1[0, 1:39])[:6] + 1).tolist())
+    for rule in (0, 1, 2):
+        assert oracle.select_one_rule(s1, 40, 8, rule)[0].tolist() == want
