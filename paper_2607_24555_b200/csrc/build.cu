@@ -32,9 +32,27 @@ struct BuildParams {
   const int32_t *append_pos;
 };
 
+#ifndef LOCKS_BUILD_SWEEPS
+#define LOCKS_BUILD_SWEEPS 12   // upper bound; a page stops as soon as its off-diagonal norm is at rounding level
+#endif
 constexpr int kBuildWarps = 4;
-constexpr int kDStride = LOCKS_D + 4;                            // padded row of D in shared memory
-constexpr int kBuildSmemPerWarp = (LOCKS_B * kDStride + 2 * LOCKS_B * 17 + 64) * 4 + i4_stride(8);
+constexpr int kBuildCtasPerSm = 6;                               // 24 warps per SM: 80 registers, 8.4 KB per warp
+constexpr int kBuildScratch = 2 * 2 * LOCKS_B * LOCKS_B * 4;      // 4096 B: bf16 tile of D, then the exchange buffers
+// Placement of a 16 x 16 matrix in an exchange buffer.  A round writes entry (row, column) with rows and
+// columns permuted (32 lanes x one scalar store: 8 rows x 4 columns) and reads it back row by row (8 rows x 4
+// columns again), 32 instructions per round in all, so bank conflicts are what a round costs.  The placement
+// below makes every one of those instructions conflict-free: bank = 4 f(row) + g(column), where f takes each of
+// its 8 values on two rows that never meet in one instruction (one even, one odd, on either side of the
+// permutation) and g takes each of its 4 values on four columns that never meet either.
+__device__ __forceinline__ int jrow_part(int r) {   // 128 (odd row) + 4 f(r)
+  const int f = (r & 1) ? (r == 15 ? 1 : (r == 1 ? 0 : (r + 1) >> 1)) : (r >> 1);
+  return ((r & 1) << 7) + 4 * f;
+}
+__device__ __forceinline__ int jcol_part(int c) {   // 32 (c mod 4) + g(c)
+  const int g = ((c & 3) == 3) ? (((c + 1) >> 2) & 3) : (c >> 2);
+  return ((c & 3) << 5) + g;
+}
+constexpr int kBuildSmemPerWarp = kBuildScratch + (2 * LOCKS_B * 17 + 64) * 4 + i4_stride(8);
 
 __device__ __forceinline__ float round_code(float x, float scale, float qmax) {
   if (scale == 0.f) return 0.f;
@@ -42,8 +60,25 @@ __device__ __forceinline__ float round_code(float x, float scale, float qmax) {
   return fminf(fmaxf(c, -qmax), qmax);
 }
 
+// packed fp32 pairs (two independent lanes of arithmetic per instruction)
+__device__ __forceinline__ float2 fma2(float2 a, float2 b, float2 c) {
+  float2 d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;"
+      : "=l"(*reinterpret_cast<unsigned long long *>(&d))
+      : "l"(*reinterpret_cast<unsigned long long *>(&a)), "l"(*reinterpret_cast<unsigned long long *>(&b)),
+        "l"(*reinterpret_cast<unsigned long long *>(&c)));
+  return d;
+}
+__device__ __forceinline__ float2 mul2(float2 a, float2 b) {
+  float2 d;
+  asm("mul.rn.f32x2 %0, %1, %2;"
+      : "=l"(*reinterpret_cast<unsigned long long *>(&d))
+      : "l"(*reinterpret_cast<unsigned long long *>(&a)), "l"(*reinterpret_cast<unsigned long long *>(&b)));
+  return d;
+}
+
 template <typename T, int FMT>
-__global__ void __launch_bounds__(kBuildWarps * 32) build_kernel(BuildParams p) {
+__global__ void __launch_bounds__(kBuildWarps * 32, kBuildCtasPerSm) build_kernel(BuildParams p) {
   extern __shared__ __align__(16) uint8_t smem_raw[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   int b, h, page;
@@ -72,52 +107,89 @@ __global__ void __launch_bounds__(kBuildWarps * 32) build_kernel(BuildParams p) 
     if (lane == 0) set_status(p.status, LOCKS_ERR_BAD_BLOCK);
     return;
   }
-  float *Ds = reinterpret_cast<float *>(smem_raw + warp * kBuildSmemPerWarp);   // [16][kDStride]
-  float *A = Ds + LOCKS_B * kDStride;                                             // [16][17]
-  float *U = A + LOCKS_B * 17;                                                    // [16][17]
-  float *rot = U + LOCKS_B * 17;                                                  // c[8], s[8], misc
+  uint8_t *scratch = smem_raw + warp * kBuildSmemPerWarp;                        // D tile, then exchange buffers
+  float *A = reinterpret_cast<float *>(scratch + kBuildScratch);                 // [16][17]
+  float *U = A + LOCKS_B * 17;                                                    // [16][17] (first: the cross product)
+  float *rot = U + LOCKS_B * 17;                                                  // misc
   uint8_t *blob = reinterpret_cast<uint8_t *>(rot + 64);
   const int r = p.r;
 
-  // ---- 1. load, centre
+  // ---- 1. load, centre.  The deviations are needed twice (Gram matrix now, basis after the eigenproblem); they
+  // are not kept in registers in between but fetched again (the page is 4 KB and still in cache).
   const T *K = reinterpret_cast<const T *>(p.k) + (int64_t)block * p.sb + (int64_t)h * p.sh;
   const T *Knew = reinterpret_cast<const T *>(p.k_new) + ((int64_t)b * p.Hkv + h) * LOCKS_D;
-  float kv[LOCKS_B][4], mu[4] = {0.f, 0.f, 0.f, 0.f};
+  float mu[4] = {0.f, 0.f, 0.f, 0.f};
   float knorm2 = 0.f;
+  auto load_keys = [&](float (&kv)[LOCKS_B][4]) {
 #pragma unroll
-  for (int i = 0; i < LOCKS_B; ++i) {
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      kv[i][u] = (i == LOCKS_B - 1 && last_from_new) ? ldf<T>(Knew, lane * 4 + u) : ldf<T>(K, (int64_t)i * p.st + lane * 4 + u);
-      mu[u] += kv[i][u];
-      knorm2 += kv[i][u] * kv[i][u];
+    for (int i = 0; i < LOCKS_B; ++i) {
+      const T *row = (i == LOCKS_B - 1 && last_from_new) ? Knew : K + (int64_t)i * p.st;
+      if (sizeof(T) == 2) {
+        const uint2 w = *reinterpret_cast<const uint2 *>(reinterpret_cast<const uint16_t *>(row) + lane * 4);
+        kv[i][0] = __uint_as_float(w.x << 16); kv[i][1] = __uint_as_float(w.x & 0xFFFF0000u);
+        kv[i][2] = __uint_as_float(w.y << 16); kv[i][3] = __uint_as_float(w.y & 0xFFFF0000u);
+      } else {
+        const float4 w = *reinterpret_cast<const float4 *>(reinterpret_cast<const float *>(row) + lane * 4);
+        kv[i][0] = w.x; kv[i][1] = w.y; kv[i][2] = w.z; kv[i][3] = w.w;
+      }
     }
-  }
-  knorm2 = warp_sum(knorm2);
+  };
+  // ---- 2. Gram matrix M = D D^T on the tensor cores.  D = H + L with H = bf16(D), L = bf16(D - H) (16 significant
+  // bits; the bf16 products are exact and accumulate in fp32): M = (H H^T + L L^T) + H L^T + (H L^T)^T.  The A
+  // operand (tokens x dims) and the B operand (dims x tokens) of an m16n8k16 step are the same registers.
+  {
+    float kv[LOCKS_B][4];
+    load_keys(kv);
 #pragma unroll
-  for (int u = 0; u < 4; ++u) mu[u] *= (1.f / LOCKS_B);
+    for (int i = 0; i < LOCKS_B; ++i)
 #pragma unroll
-  for (int i = 0; i < LOCKS_B; ++i) {
+      for (int u = 0; u < 4; ++u) { mu[u] += kv[i][u]; knorm2 = fmaf(kv[i][u], kv[i][u], knorm2); }
+    knorm2 = warp_sum(knorm2);
 #pragma unroll
-    for (int u = 0; u < 4; ++u) kv[i][u] -= mu[u];
-    *reinterpret_cast<float4 *>(Ds + i * kDStride + lane * 4) = make_float4(kv[i][0], kv[i][1], kv[i][2], kv[i][3]);
-  }
-  __syncwarp();
-  // ---- 2. Gram: lane computes entries e = lane + 32 m -> (i = e / 16, j = e % 16)
-#pragma unroll 1
-  for (int m = 0; m < 8; ++m) {
-    const int e = lane + 32 * m, i = e >> 4, j = e & 15;
-    const float4 *ri = reinterpret_cast<const float4 *>(Ds + i * kDStride);
-    const float4 *rj = reinterpret_cast<const float4 *>(Ds + j * kDStride);
-    float s = 0.f;
-    for (int c = 0; c < LOCKS_D / 4; ++c) {
-      const float4 a = ri[c], bb = rj[c];
-      s += a.x * bb.x + a.y * bb.y + a.z * bb.z + a.w * bb.w;
+    for (int u = 0; u < 4; ++u) mu[u] *= (1.f / LOCKS_B);
+    // lane owns dims 4 lane .. 4 lane + 3: 8 bytes of 16-byte chunk lane / 2 of every token row (256-byte rows,
+    // chunks XOR-swizzled with the token so that ldmatrix reads are conflict-free)
+    uint2 lo_pk[LOCKS_B];
+#pragma unroll
+    for (int i = 0; i < LOCKS_B; ++i) {
+      float dv[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) dv[u] = kv[i][u] - mu[u];
+      const uint32_t h01 = pack_bf16(dv[0], dv[1]), h23 = pack_bf16(dv[2], dv[3]);
+      lo_pk[i].x = pack_bf16(dv[0] - __uint_as_float(h01 << 16), dv[1] - __uint_as_float(h01 & 0xFFFF0000u));
+      lo_pk[i].y = pack_bf16(dv[2] - __uint_as_float(h23 << 16), dv[3] - __uint_as_float(h23 & 0xFFFF0000u));
+      *reinterpret_cast<uint2 *>(scratch + i * 256 + ((((lane >> 1) ^ (i & 7)) << 4) | ((lane & 1) << 3))) = make_uint2(h01, h23);
     }
-    A[i * 17 + j] = s;
-    U[i * 17 + j] = (i == j) ? 1.f : 0.f;
+    __syncwarp();
+    const int mq = lane >> 3, rr = lane & 7, tok = (mq & 1) * 8 + rr;
+    uint32_t Hf[8][4];
+#pragma unroll
+    for (int s = 0; s < 8; ++s) ldsm_x4(Hf[s], scratch + tok * 256 + (((2 * s + (mq >> 1)) ^ (tok & 7)) << 4));
+    __syncwarp();
+#pragma unroll
+    for (int i = 0; i < LOCKS_B; ++i)
+      *reinterpret_cast<uint2 *>(scratch + i * 256 + ((((lane >> 1) ^ (i & 7)) << 4) | ((lane & 1) << 3))) = lo_pk[i];
+    __syncwarp();
+    float X0[4] = {0.f, 0.f, 0.f, 0.f}, X1[4] = {0.f, 0.f, 0.f, 0.f}, Y0[4] = {0.f, 0.f, 0.f, 0.f}, Y1[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int s = 0; s < 8; ++s) {
+      uint32_t Lf[4];
+      ldsm_x4(Lf, scratch + tok * 256 + (((2 * s + (mq >> 1)) ^ (tok & 7)) << 4));
+      mma_bf16(X0, Hf[s][0], Hf[s][1], Hf[s][2], Hf[s][3], Hf[s][0], Hf[s][2]);
+      mma_bf16(X1, Hf[s][0], Hf[s][1], Hf[s][2], Hf[s][3], Hf[s][1], Hf[s][3]);
+      mma_bf16(X0, Lf[0], Lf[1], Lf[2], Lf[3], Lf[0], Lf[2]);
+      mma_bf16(X1, Lf[0], Lf[1], Lf[2], Lf[3], Lf[1], Lf[3]);
+      mma_bf16(Y0, Hf[s][0], Hf[s][1], Hf[s][2], Hf[s][3], Lf[0], Lf[2]);
+      mma_bf16(Y1, Hf[s][0], Hf[s][1], Hf[s][2], Hf[s][3], Lf[1], Lf[3]);
+    }
+    // accumulator (x = lane / 4, t = lane % 4): [0..1] = row x, columns 2t, 2t+1; [2..3] = row x + 8
+    const int x = lane >> 2, t = lane & 3;
+    A[x * 17 + 2 * t] = X0[0]; A[x * 17 + 2 * t + 1] = X0[1]; A[(x + 8) * 17 + 2 * t] = X0[2]; A[(x + 8) * 17 + 2 * t + 1] = X0[3];
+    A[x * 17 + 8 + 2 * t] = X1[0]; A[x * 17 + 9 + 2 * t] = X1[1]; A[(x + 8) * 17 + 8 + 2 * t] = X1[2]; A[(x + 8) * 17 + 9 + 2 * t] = X1[3];
+    U[x * 17 + 2 * t] = Y0[0]; U[x * 17 + 2 * t + 1] = Y0[1]; U[(x + 8) * 17 + 2 * t] = Y0[2]; U[(x + 8) * 17 + 2 * t + 1] = Y0[3];
+    U[x * 17 + 8 + 2 * t] = Y1[0]; U[x * 17 + 9 + 2 * t] = Y1[1]; U[(x + 8) * 17 + 8 + 2 * t] = Y1[2]; U[(x + 8) * 17 + 9 + 2 * t] = Y1[3];
+    __syncwarp();
   }
-  __syncwarp();
   // ---- 3. parallel cyclic Jacobi, matrix held in registers.
   // "Slot" space: the 8 rotations of a round always act on the slot pairs (2m, 2m+1); between rounds the 16
   // indices move through the slots by the fixed round-robin permutation `next_slot` (slot 0 stays, the others
@@ -125,24 +197,32 @@ __global__ void __launch_bounds__(kBuildWarps * 32) build_kernel(BuildParams p) 
   // rows 2m, 2m+1 x columns 4k .. 4k+3 of A (two 2x2 blocks) and of U (rows = tokens, columns = slots).  A round
   // is: rotation angles at the lanes that hold a diagonal block, six shuffles to hand them to the rows and
   // columns they act on, the block updates in registers, and one pass through shared memory (ping-pong
-  // buffers, one warp barrier) that applies the permutation.
+  // buffers, one warp barrier) that applies the permutation.  The two blocks of a lane are updated together:
+  // entry (row bit, column bit) of both blocks forms one packed fp32 pair (.x = columns 4k, 4k+1, .y = columns
+  // 4k+2, 4k+3), the column rotation multiplies by per-block coefficient pairs, the row rotation by the same
+  // coefficient in both halves.
   {
     const int m = lane >> 2, k = lane & 3;
     auto next_slot = [](int x) { return x == 0 ? 0 : (x == 1 ? 2 : (x == 14 ? 15 : ((x & 1) ? x - 2 : x + 2))); };
-    constexpr int kJS = 20;   // row stride of the exchange buffers (16-byte aligned rows)
-    float *buf0 = Ds, *buf1 = Ds + 2 * LOCKS_B * kJS;   // each: A[16][kJS] then U[16][kJS]
-    float a[8], u[8];   // index = 4 * blk + 2 * rowbit + colbit, columns 4k + 2 blk + colbit
+    float *buf0 = reinterpret_cast<float *>(scratch), *buf1 = buf0 + 2 * LOCKS_B * LOCKS_B;   // each: A then U, 256 floats
+    float2 pa[2][2], pu[2][2];   // [row bit][column bit]
 #pragma unroll
-    for (int e = 0; e < 8; ++e) {
-      const int i = 2 * m + ((e >> 1) & 1), j = 4 * k + 2 * (e >> 2) + (e & 1);
-      a[e] = A[i * 17 + j];
-      u[e] = (i == j) ? 1.f : 0.f;
-    }
-    int wr_row[2], wr_col[4];   // where this lane's rows / columns go after a round
+    for (int rb = 0; rb < 2; ++rb)
 #pragma unroll
-    for (int rb = 0; rb < 2; ++rb) wr_row[rb] = next_slot(2 * m + rb);
+      for (int cb = 0; cb < 2; ++cb) {
+        const int i = 2 * m + rb, j0 = 4 * k + cb, j1 = j0 + 2;
+        pa[rb][cb].x = 0.5f * (A[i * 17 + j0] + A[j0 * 17 + i]) + U[i * 17 + j0] + U[j0 * 17 + i];
+        pa[rb][cb].y = 0.5f * (A[i * 17 + j1] + A[j1 * 17 + i]) + U[i * 17 + j1] + U[j1 * 17 + i];
+        pu[rb][cb].x = (i == j0) ? 1.f : 0.f;
+        pu[rb][cb].y = (i == j1) ? 1.f : 0.f;
+      }
+    __syncwarp();
+    // buffer offsets of this lane's entries: where its rows / columns go after a round, and where they are read
+    int wr_row[2], wr_col[4], rd_row[2], rd_col[4];
 #pragma unroll
-    for (int c4 = 0; c4 < 4; ++c4) wr_col[c4] = next_slot(4 * k + c4);
+    for (int rb = 0; rb < 2; ++rb) { wr_row[rb] = jrow_part(next_slot(2 * m + rb)); rd_row[rb] = jrow_part(2 * m + rb); }
+#pragma unroll
+    for (int c4 = 0; c4 < 4; ++c4) { wr_col[c4] = jcol_part(next_slot(4 * k + c4)); rd_col[c4] = jcol_part(4 * k + c4); }
     const bool diag_lane = k == (m >> 1);
     const int dblk = m & 1;             // which of the two blocks is the diagonal one (diag lanes)
     const int src_row = m * 4 + (m >> 1);           // lane holding the diagonal block of row pair m
@@ -153,7 +233,9 @@ __global__ void __launch_bounds__(kBuildWarps * 32) build_kernel(BuildParams p) 
     {
       float amax = 0.f;
 #pragma unroll
-      for (int e = 0; e < 8; ++e) amax = fmaxf(amax, fabsf(a[e]));
+      for (int rb = 0; rb < 2; ++rb)
+#pragma unroll
+        for (int cb = 0; cb < 2; ++cb) amax = fmaxf(amax, fmaxf(fabsf(pa[rb][cb].x), fabsf(pa[rb][cb].y)));
       amax = warp_max(amax);
       if (amax > 0.f && amax < INFINITY) {
         int ex;
@@ -162,81 +244,97 @@ __global__ void __launch_bounds__(kBuildWarps * 32) build_kernel(BuildParams p) 
         const float sc = ldexpf(1.f, -ex);
         unscale = ldexpf(1.f, ex);
 #pragma unroll
-        for (int e = 0; e < 8; ++e) a[e] *= sc;
+        for (int rb = 0; rb < 2; ++rb)
+#pragma unroll
+          for (int cb = 0; cb < 2; ++cb) { pa[rb][cb].x *= sc; pa[rb][cb].y *= sc; }
       }
     }
     float normA = 0.f;
 #pragma unroll
-    for (int e = 0; e < 8; ++e) normA += a[e] * a[e];
+    for (int rb = 0; rb < 2; ++rb)
+#pragma unroll
+      for (int cb = 0; cb < 2; ++cb) normA += pa[rb][cb].x * pa[rb][cb].x + pa[rb][cb].y * pa[rb][cb].y;
     normA = warp_sum(normA);
     int parity = 0;
-    for (int sweep = 0; sweep < 12; ++sweep) {
+    for (int sweep = 0; sweep < LOCKS_BUILD_SWEEPS; ++sweep) {
       float off = 0.f;
 #pragma unroll
-      for (int e = 0; e < 8; ++e) {
-        const bool on_diag = diag_lane && (e >> 2) == dblk && (((e >> 1) & 1) == (e & 1));
-        off += on_diag ? 0.f : a[e] * a[e];
-      }
+      for (int rb = 0; rb < 2; ++rb)
+#pragma unroll
+        for (int cb = 0; cb < 2; ++cb) {
+          const bool dg = diag_lane && rb == cb;   // diagonal entries of the diagonal block do not count
+          off += (dg && dblk == 0) ? 0.f : pa[rb][cb].x * pa[rb][cb].x;
+          off += (dg && dblk == 1) ? 0.f : pa[rb][cb].y * pa[rb][cb].y;
+        }
       off = warp_sum(off);
       if (off <= 1e-13f * normA || normA == 0.f) break;
 #pragma unroll 1
       for (int round = 0; round < 15; ++round) {
         // rotation of the slot pair held as a diagonal block (other lanes compute on whatever they hold; unused)
-        const float app = dblk ? a[4] : a[0], apq = dblk ? a[5] : a[1], aqq = dblk ? a[7] : a[3];
+        const float app = dblk ? pa[0][0].y : pa[0][0].x, apq = dblk ? pa[0][1].y : pa[0][1].x;
+        const float aqq = dblk ? pa[1][1].y : pa[1][1].x;
         float c = 1.f, sn = 0.f;
         {
           // tan of the rotation angle: t = 2 apq / (d + sign(d) sqrt(d^2 + 4 apq^2)), d = aqq - app (the smaller
           // root).  Approximate root and division are enough for the angle; c^2 + s^2 = 1 comes from the last
           // two lines.  Entries too small to square are left alone.
-          const float d = aqq - app, h = d * d + 4.f * apq * apq;
-          if (h > 1e-37f && h < 1e37f) {
-            const float tt = __fdividef(2.f * apq, d + copysignf(h * rsqrtf(h), d));
+          const float d = aqq - app, hh = d * d + 4.f * apq * apq;
+          if (hh > 1e-37f && hh < 1e37f) {
+            const float tt = __fdividef(2.f * apq, d + copysignf(hh * rsqrtf(hh), d));
             c = rsqrtf(tt * tt + 1.f);
             sn = tt * c;
           }
         }
         const float cr = __shfl_sync(0xffffffffu, c, src_row), sr = __shfl_sync(0xffffffffu, sn, src_row);
-        const float cc[2] = {__shfl_sync(0xffffffffu, c, src_c0), __shfl_sync(0xffffffffu, c, src_c1)};
-        const float sc[2] = {__shfl_sync(0xffffffffu, sn, src_c0), __shfl_sync(0xffffffffu, sn, src_c1)};
+        const float2 Cc = make_float2(__shfl_sync(0xffffffffu, c, src_c0), __shfl_sync(0xffffffffu, c, src_c1));
+        const float2 Sc = make_float2(__shfl_sync(0xffffffffu, sn, src_c0), __shfl_sync(0xffffffffu, sn, src_c1));
+        const float2 nSc = make_float2(-Sc.x, -Sc.y), Cr = make_float2(cr, cr), Sr = make_float2(sr, sr), nSr = make_float2(-sr, -sr);
         float *dst = parity ? buf1 : buf0;
+        // columns: [x_ip x_iq] <- [c x_ip - s x_iq, s x_ip + c x_iq]; rows: [x_pj; x_qj] <- [c x_pj - s x_qj; s x_pj + c x_qj]
+        float2 ta[2][2];
 #pragma unroll
-        for (int blk = 0; blk < 2; ++blk) {
-          float *x = a + 4 * blk, *y = u + 4 * blk;
-          // columns: [x_ip x_iq] <- [c x_ip - s x_iq, s x_ip + c x_iq]
-          const float t00 = cc[blk] * x[0] - sc[blk] * x[1], t01 = sc[blk] * x[0] + cc[blk] * x[1];
-          const float t10 = cc[blk] * x[2] - sc[blk] * x[3], t11 = sc[blk] * x[2] + cc[blk] * x[3];
-          // rows: [x_pj; x_qj] <- [c x_pj - s x_qj; s x_pj + c x_qj]
-          x[0] = cr * t00 - sr * t10; x[1] = cr * t01 - sr * t11;
-          x[2] = sr * t00 + cr * t10; x[3] = sr * t01 + cr * t11;
-          const float v00 = cc[blk] * y[0] - sc[blk] * y[1], v01 = sc[blk] * y[0] + cc[blk] * y[1];
-          const float v10 = cc[blk] * y[2] - sc[blk] * y[3], v11 = sc[blk] * y[2] + cc[blk] * y[3];
-          y[0] = v00; y[1] = v01; y[2] = v10; y[3] = v11;
+        for (int rb = 0; rb < 2; ++rb) {
+          ta[rb][0] = fma2(Cc, pa[rb][0], mul2(nSc, pa[rb][1]));
+          ta[rb][1] = fma2(Sc, pa[rb][0], mul2(Cc, pa[rb][1]));
+          const float2 u0 = fma2(Cc, pu[rb][0], mul2(nSc, pu[rb][1]));
+          const float2 u1 = fma2(Sc, pu[rb][0], mul2(Cc, pu[rb][1]));
+          pu[rb][0] = u0; pu[rb][1] = u1;
+        }
+#pragma unroll
+        for (int cb = 0; cb < 2; ++cb) {
+          pa[0][cb] = fma2(Cr, ta[0][cb], mul2(nSr, ta[1][cb]));
+          pa[1][cb] = fma2(Sr, ta[0][cb], mul2(Cr, ta[1][cb]));
         }
         // the permutation: A rows and columns, U columns
 #pragma unroll
-        for (int e = 0; e < 8; ++e) {
-          const int rb = (e >> 1) & 1, c4 = 2 * (e >> 2) + (e & 1);
-          dst[wr_row[rb] * kJS + wr_col[c4]] = a[e];
-          dst[LOCKS_B * kJS + (2 * m + rb) * kJS + wr_col[c4]] = u[e];
-        }
+        for (int rb = 0; rb < 2; ++rb)
+#pragma unroll
+          for (int cb = 0; cb < 2; ++cb) {
+            dst[wr_row[rb] + wr_col[cb]] = pa[rb][cb].x;
+            dst[wr_row[rb] + wr_col[2 + cb]] = pa[rb][cb].y;
+            dst[LOCKS_B * LOCKS_B + rd_row[rb] + wr_col[cb]] = pu[rb][cb].x;
+            dst[LOCKS_B * LOCKS_B + rd_row[rb] + wr_col[2 + cb]] = pu[rb][cb].y;
+          }
         __syncwarp();
 #pragma unroll
-        for (int rb = 0; rb < 2; ++rb) {   // columns 4k .. 4k+3 of a row are one 16-byte read
-          const float4 ra = *reinterpret_cast<const float4 *>(dst + (2 * m + rb) * kJS + 4 * k);
-          const float4 ru = *reinterpret_cast<const float4 *>(dst + LOCKS_B * kJS + (2 * m + rb) * kJS + 4 * k);
-          a[2 * rb] = ra.x; a[2 * rb + 1] = ra.y; a[4 + 2 * rb] = ra.z; a[4 + 2 * rb + 1] = ra.w;
-          u[2 * rb] = ru.x; u[2 * rb + 1] = ru.y; u[4 + 2 * rb] = ru.z; u[4 + 2 * rb + 1] = ru.w;
-        }
+        for (int rb = 0; rb < 2; ++rb)
+#pragma unroll
+          for (int cb = 0; cb < 2; ++cb) {
+            pa[rb][cb] = make_float2(dst[rd_row[rb] + rd_col[cb]], dst[rd_row[rb] + rd_col[2 + cb]]);
+            pu[rb][cb] = make_float2(dst[LOCKS_B * LOCKS_B + rd_row[rb] + rd_col[cb]], dst[LOCKS_B * LOCKS_B + rd_row[rb] + rd_col[2 + cb]]);
+          }
         parity ^= 1;
       }
     }
     __syncwarp();
 #pragma unroll
-    for (int e = 0; e < 8; ++e) {
-      const int i = 2 * m + ((e >> 1) & 1), j = 4 * k + 2 * (e >> 2) + (e & 1);
-      A[i * 17 + j] = a[e] * unscale;
-      U[i * 17 + j] = u[e];
-    }
+    for (int rb = 0; rb < 2; ++rb)
+#pragma unroll
+      for (int cb = 0; cb < 2; ++cb) {
+        const int i = 2 * m + rb, j0 = 4 * k + cb, j1 = j0 + 2;
+        A[i * 17 + j0] = pa[rb][cb].x * unscale; A[i * 17 + j1] = pa[rb][cb].y * unscale;
+        U[i * 17 + j0] = pu[rb][cb].x; U[i * 17 + j1] = pu[rb][cb].y;
+      }
     __syncwarp();
   }
   // ---- 4. order the eigenvalues (descending, ties by index), choose r_eff
@@ -261,55 +359,60 @@ __global__ void __launch_bounds__(kBuildWarps * 32) build_kernel(BuildParams p) 
     __syncwarp();
   }
   float *fout = reinterpret_cast<float *>(p.summ + ((int64_t)block * p.Hkv + h) * p.S);
-  float csign[16];
+  uint32_t sign_bits = 0u;   // bit l: mode l was flipped
+  {
+    float kv[LOCKS_B][4];
+    load_keys(kv);
+#pragma unroll
+    for (int i = 0; i < LOCKS_B; ++i)
+#pragma unroll
+      for (int u = 0; u < 4; ++u) kv[i][u] -= mu[u];
 #pragma unroll 1
-  for (int l = 0; l < r; ++l) {
-    float v[4] = {0.f, 0.f, 0.f, 0.f};
-    float sgn = 1.f;
-    if (l < r_eff) {
-      const int col = reinterpret_cast<int *>(rot)[32 + l];
-      const float inv = rsqrtf(rot[48 + l]);
+    for (int l = 0; l < r; ++l) {
+      float v[4] = {0.f, 0.f, 0.f, 0.f};
+      float best = 0.f;   // largest magnitude of the mode's basis vector
+      if (l < r_eff) {
+        const int col = reinterpret_cast<int *>(rot)[32 + l];
+        const float inv = rsqrtf(rot[48 + l]);
 #pragma unroll
-      for (int i = 0; i < LOCKS_B; ++i) {
-        const float u = U[i * 17 + col];
+        for (int i = 0; i < LOCKS_B; ++i) {
+          const float u = U[i * 17 + col];
 #pragma unroll
-        for (int c = 0; c < 4; ++c) v[c] += kv[i][c] * u;
+          for (int c = 0; c < 4; ++c) v[c] = fmaf(kv[i][c], u, v[c]);
+        }
+#pragma unroll
+        for (int c = 0; c < 4; ++c) v[c] *= inv;
+        // sign: entry of largest magnitude (lowest dim on ties) positive.  Magnitudes order like their bit
+        // patterns; the lowest lane that holds the maximum owns the lowest such dim.
+        best = fabsf(v[0]); float bv = v[0];
+#pragma unroll
+        for (int c = 1; c < 4; ++c) if (fabsf(v[c]) > best) { best = fabsf(v[c]); bv = v[c]; }
+        const uint32_t mxb = __reduce_max_sync(0xffffffffu, __float_as_uint(best));
+        const uint32_t who = __ballot_sync(0xffffffffu, __float_as_uint(best) == mxb);
+        bv = __shfl_sync(0xffffffffu, bv, __ffs(who) - 1);
+        best = __uint_as_float(mxb);
+        if (bv < 0.f) {
+          sign_bits |= 1u << l;
+#pragma unroll
+          for (int c = 0; c < 4; ++c) v[c] = -v[c];
+        }
       }
+      if (FMT == LOCKS_FMT_F32) {
+        *reinterpret_cast<float4 *>(fout + LOCKS_D + l * LOCKS_D + lane * 4) = make_float4(v[0], v[1], v[2], v[3]);
+      } else {
+        const __half sh = __float2half_rn(best / 7.f);
+        const float sc = __half2float(sh);
+        if (lane == 0) *reinterpret_cast<__half *>(blob + i4_off_sv(r) + 2 * l) = sh;
+        // lane = 8 t + s owns dims 32 t + 4 s + {0,1,2,3} = (half, e) in {0,1}^2 of k-step s
+        const int t = lane >> 3, s = lane & 7, i0 = (s & 1) << 1;
+        uint32_t n[4];
 #pragma unroll
-      for (int c = 0; c < 4; ++c) v[c] *= inv;
-      // sign: entry of largest magnitude (lowest dim on ties) positive
-      float best = fabsf(v[0]); int bi = lane * 4; float bv = v[0];
-#pragma unroll
-      for (int c = 1; c < 4; ++c) if (fabsf(v[c]) > best) { best = fabsf(v[c]); bi = lane * 4 + c; bv = v[c]; }
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) {
-        const float ob = __shfl_xor_sync(0xffffffffu, best, o);
-        const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
-        const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
-        if (ob > best || (ob == best && oi < bi)) { best = ob; bi = oi; bv = ov; }
+        for (int c = 0; c < 4; ++c) n[c] = (uint32_t)((int)round_code(v[c], sc, 7.f) + 8);
+        // dim offset c = 2*half + e -> nibble i0 + half + 4 e
+        uint32_t pw = (n[0] << (4 * i0)) | (n[1] << (4 * (i0 + 4))) | (n[2] << (4 * (i0 + 1))) | (n[3] << (4 * (i0 + 5)));
+        pw |= __shfl_xor_sync(0xffffffffu, pw, 1);
+        if ((s & 1) == 0) *reinterpret_cast<uint32_t *>(blob + (l * 4 + t) * 16 + (s >> 1) * 4) = pw;
       }
-      if (bv < 0.f) sgn = -1.f;
-#pragma unroll
-      for (int c = 0; c < 4; ++c) v[c] *= sgn;
-    }
-    csign[l & 15] = sgn;
-    if (FMT == LOCKS_FMT_F32) {
-      *reinterpret_cast<float4 *>(fout + LOCKS_D + l * LOCKS_D + lane * 4) = make_float4(v[0], v[1], v[2], v[3]);
-    } else {
-      float mx = fmaxf(fmaxf(fabsf(v[0]), fabsf(v[1])), fmaxf(fabsf(v[2]), fabsf(v[3])));
-      mx = warp_max(mx);
-      const __half sh = __float2half_rn(mx / 7.f);
-      const float sc = __half2float(sh);
-      if (lane == 0) *reinterpret_cast<__half *>(blob + i4_off_sv(r) + 2 * l) = sh;
-      // lane = 8 t + s owns dims 32 t + 4 s + {0,1,2,3} = (half, e) in {0,1}^2 of k-step s
-      const int t = lane >> 3, s = lane & 7, i0 = (s & 1) << 1;
-      uint32_t n[4];
-#pragma unroll
-      for (int c = 0; c < 4; ++c) n[c] = (uint32_t)((int)round_code(v[c], sc, 7.f) + 8);
-      // dim offset c = 2*half + e -> nibble i0 + half + 4 e
-      uint32_t pw = (n[0] << (4 * i0)) | (n[1] << (4 * (i0 + 4))) | (n[2] << (4 * (i0 + 1))) | (n[3] << (4 * (i0 + 5)));
-      pw |= __shfl_xor_sync(0xffffffffu, pw, 1);
-      if ((s & 1) == 0) *reinterpret_cast<uint32_t *>(blob + (l * 4 + t) * 16 + (s >> 1) * 4) = pw;
     }
   }
   // coefficients: lane i < 16 owns token i
@@ -318,7 +421,10 @@ __global__ void __launch_bounds__(kBuildWarps * 32) build_kernel(BuildParams p) 
     float mx = 0.f;
     for (int l = 0; l < r; ++l) {
       float c = 0.f;
-      if (l < r_eff) c = sqrtf(rot[48 + l]) * U[lane * 17 + reinterpret_cast<int *>(rot)[32 + l]] * csign[l & 15];
+      if (l < r_eff) {
+        c = sqrtf(rot[48 + l]) * U[lane * 17 + reinterpret_cast<int *>(rot)[32 + l]];
+        if ((sign_bits >> l) & 1u) c = -c;
+      }
       cf[l & 15] = c;
       mx = fmaxf(mx, fabsf(c));
     }
@@ -340,7 +446,7 @@ __global__ void __launch_bounds__(kBuildWarps * 32) build_kernel(BuildParams p) 
     *reinterpret_cast<float4 *>(fout + lane * 4) = make_float4(mu[0], mu[1], mu[2], mu[3]);
   } else {
     float mx = fmaxf(fmaxf(fabsf(mu[0]), fabsf(mu[1])), fmaxf(fabsf(mu[2]), fabsf(mu[3])));
-    mx = warp_max(mx);
+    mx = __uint_as_float(__reduce_max_sync(0xffffffffu, __float_as_uint(mx)));
     const __half sh = __float2half_rn(mx / 127.f);
     const float sc = __half2float(sh);
     if (lane == 0) *reinterpret_cast<__half *>(blob + i4_off_smu(r)) = sh;
