@@ -11,10 +11,12 @@ Cold caches: the step touches about 175 MB and B200's L2 holds 126 MB, so the re
 several independent "layers" (own KV cache, summaries and query), as a real model would; by the
 time a layer comes round again its lines are gone.
 
-Prints ONE JSON line: metric / value / unit, the step time, `e2e` (the same step through the host-buffer entry
-point, copies included), `roofline` (scan kernel: algorithmic bytes / measured kernel time against the measured
-copy bandwidth, plus the kernel's DRAM traffic from the committed ncu capture), `cpu_baseline` (the oracle on the
-host cores), per-stage times, the dense flash-decode time on the same inputs, clocks and launch count.  `--impl reference` times the CPU
+Prints ONE JSON line: metric / value / unit, the step time over exactly K replays, `windows` (mean and spread over
+three windows of 64 replays), `e2e` (the same step through the host-buffer entry point, copies included),
+`roofline` (scan kernel: algorithmic bytes / measured kernel time against the measured copy bandwidth, plus the
+kernel's DRAM traffic from the committed ncu capture), `cpu_baseline` (the oracle on the host cores), per-stage
+times, the dense flash-decode time on the same inputs, the bulk summary build, clocks, launch count, and
+`workloads`: a compact table (step, bytes, fraction of peak, dense) for one cell of each other configuration.  `--impl reference` times the CPU
 oracle instead (test infrastructure; the only other place this file runs it is `cpu_baseline`).
 """
 from __future__ import annotations
@@ -97,14 +99,19 @@ def measured_peak():
 
 
 def recorded_traffic(wname):
-    """DRAM bytes per scan launch from the committed ncu capture, if one covers this workload."""
-    p = os.path.join(ROOT, "profiles", "traffic.json")
+    """DRAM bytes per scan launch (dram__bytes_read.sum + dram__bytes_write.sum) copied from the committed ncu
+    summary of this workload, with the file it was copied from; (None, None) when no capture covers it.  The
+    number is evidence about re-reads, not an input of any timing: it moves only when the kernel's memory
+    access pattern changes, and the summary file names the source revision it was captured at."""
+    p = os.path.join(ROOT, "profiles", "scan_dram_traffic.json")
     if os.path.exists(p):
         try:
-            return json.load(open(p)).get(wname)
+            e = json.load(open(p)).get(wname)
+            if e:
+                return float(e["bytes_per_launch"]), f"profiles/{e['summary']} (captured at {e['revision']})"
         except Exception:
-            return None
-    return None
+            pass
+    return None, None
 
 
 class ClockSampler:
@@ -201,32 +208,32 @@ def run_reference(args):
     print(json.dumps(line))
 
 
-def run_ours(args):
-    import numpy as np
+def stagger(w, li):
+    """Start lengths of the timed run: the configuration's context minus 1 .. 16 tokens, different per request
+    and layer, so that requests cross page boundaries at different steps and a typical step contains the
+    summary build of the pages that fill (with every length a multiple of 16 no timed step would)."""
+    return [max(1, t - 1 - ((5 * b + 3 * li) % w.B)) for b, t in enumerate(w.seq_lens)]
+
+
+def measure(args, w0, K, W, L, rank, local_rank, full):
+    """Build the workload on the device and time the decode step.  `full`: everything the JSON line carries;
+    otherwise the compact row of the per-workload table (step, dense, stage split)."""
     import torch
     import locks_synth
     import paper_2607_24555_b200 as locks
     from paper_2607_24555_b200 import dist as ldist
     from paper_2607_24555_b200.binding import KVView, make_config
 
-    rank, local_rank, world = ldist.env_rank_world()
-    if world > 1:
-        import torch.distributed as tdist
-        tdist.init_process_group("nccl", device_id=torch.device(f"cuda:{local_rank}"))
-    torch.cuda.set_device(local_rank)
     dev = f"cuda:{local_rank}"
-    K, W = args.steps, max(args.warmup, 3)
-    w0 = workload(args.workload)
-    L = args.layers
-    grow = K + W + 2 * K + 64                       # tokens appended over the whole run, per layer at most
-    reserve = -(-grow // w0.B) + 1
-    # every rank owns a full batch (weak scaling): requests are independent, no data-path collective
+    NW, WSTEPS = (3, 64) if full else (0, 0)
+    grow = (W + K + NW * WSTEPS + (K + 2) + (4 * L + K if full else 0)) // L + 24   # tokens appended per layer
+    reserve = -(-grow // w0.B) + 2
     layers = []
     for li in range(L):
         w = w0.with_(seed=w0.seed * 1000 + 17 * li + 101 * rank, seq_lens=[t + reserve * w0.B for t in w0.seq_lens],
                      permute_blocks=not args.identity_blocks)
         case = locks_synth.make_case(w, device=dev)
-        case.seq_lens.copy_(torch.tensor(w0.seq_lens, dtype=torch.int32, device=dev))
+        case.seq_lens.copy_(torch.tensor(stagger(w0, li), dtype=torch.int32, device=dev))
         layers.append(case)
     max_pages = layers[0].block_table.shape[1]
     cfg = make_config(w0.Hq, w0.Hkv, w0.rank, w0.fmt, w0.dtype, w0.n, max_pages, w0.budget)
@@ -235,15 +242,22 @@ def run_ours(args):
                                   "balanced": locks.PARTITION_BALANCED}[args.scan_partition])
     kvs = [KVView(c.k, c.v, c.strides, c.num_blocks, c.block_table, c.seq_lens) for c in layers]
     summs = [ctx.new_summaries(c.num_blocks) for c in layers]
-    t0 = time.perf_counter()
-    for kv, s in zip(kvs, summs):
-        ctx.locks_build_summaries(kv, w0.n, s)
-    torch.cuda.synchronize()
-    bulk_build_ms = (time.perf_counter() - t0) * 1e3 / L
+    stream = torch.cuda.Stream(device=dev)
+    with torch.cuda.stream(stream):
+        for kv, s in zip(kvs, summs):                       # first pass also loads the kernel
+            ctx.locks_build_summaries(kv, w0.n, s, stream=stream)
+        stream.synchronize()
+        b0, b1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        b0.record(stream)
+        for kv, s in zip(kvs, summs):
+            ctx.locks_build_summaries(kv, w0.n, s, stream=stream)
+        b1.record(stream)
+        stream.synchronize()
+    bulk_build_ms = b0.elapsed_time(b1) / L
+    build_pages = sum((t // w0.B) for t in stagger(w0, 0)) * w0.Hkv
     outs = [torch.empty(w0.n, w0.Hq, w0.d, dtype=torch.bfloat16 if w0.dtype == "bf16" else torch.float32, device=dev)
             for _ in layers]
     news = [locks_synth.new_token(w0.with_(seed=w0.seed + li), li, device=dev) for li in range(L)]
-    stream = torch.cuda.Stream(device=dev)
 
     def step(li, s=None):
         kn, vn, qn = news[li]
@@ -255,6 +269,7 @@ def run_ours(args):
         for li in range(L):
             step(li)
         stream.synchronize()
+        partition = ctx.locks_last_scan_partition()
         for li in range(L):
             g = torch.cuda.CUDAGraph()
             with torch.cuda.graph(g, stream=stream):
@@ -262,26 +277,39 @@ def run_ours(args):
             graphs.append(g)
     launches_per_step = ctx.locks_last_launch_count()
     torch.cuda.synchronize()
+    done = [0]
 
-    def run_graph_steps(n, first):
-        for i in range(n):
-            graphs[(first + i) % L].replay()
+    def run_graph_steps(n):
+        for _ in range(n):
+            graphs[done[0] % L].replay()
+            done[0] += 1
 
-    # ---- timed region: exactly K graph replays between barrier + synchronize
+    res = {}
     with torch.cuda.stream(stream):
-        run_graph_steps(W, 0)
+        run_graph_steps(W)
         stream.synchronize()
         ldist.barrier()
         torch.cuda.synchronize()
         sampler = ClockSampler(local_rank) if rank == 0 else None
+        # ---- timed region: exactly K graph replays between barrier + synchronize
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record(stream)
-        run_graph_steps(K, W)
+        run_graph_steps(K)
         e1.record(stream)
         stream.synchronize()
         torch.cuda.synchronize()
         ldist.barrier()
-        step_ms = e0.elapsed_time(e1) / K
+        res["step_ms"] = e0.elapsed_time(e1) / K
+        # ---- spread: three windows of 64 replays each (the paper's own timing cell: 3 x 64 decode steps)
+        wins = []
+        for _ in range(NW):
+            a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a0.record(stream)
+            run_graph_steps(WSTEPS)
+            a1.record(stream)
+            stream.synchronize()
+            wins.append(a0.elapsed_time(a1) / WSTEPS * 1e3)
+        res["windows_us"] = wins
         # ---- per-kernel split: the same step captured with event-record nodes at the stage boundaries,
         # replayed K times, durations read after each replay (CUDA events on the launch stream)
         ctx.locks_profile_begin(1)
@@ -293,12 +321,13 @@ def run_ours(args):
             pgraphs.append(g)
         stage_ms = {"scan": 0.0, "select": 0.0, "attend": 0.0}
         for i in range(K + 2):
-            pgraphs[(W + K + i) % L].replay()
+            pgraphs[(done[0] + i) % L].replay()
             one = ctx.locks_profile_read(stream=stream)
             if i >= 2:
                 for k_ in stage_ms:
                     stage_ms[k_] += one[k_] / K
         ctx.locks_profile_end()
+        res["stage_ms"] = stage_ms
         # ---- dense flash-decode over the full cache on the same GPU (same entry point, no page table)
         for li in range(min(L, 3)):
             ctx.locks_sparse_attend(news[li][2], kvs[li], w0.n, None, None, outs[li], stream=stream)
@@ -310,28 +339,75 @@ def run_ours(args):
             ctx.locks_sparse_attend(news[i % L][2], kvs[i % L], w0.n, None, None, outs[i % L], stream=stream)
         d1.record(stream)
         stream.synchronize()
-        dense_ms = d0.elapsed_time(d1) / nd
-        clocks = sampler.stop() if sampler else None
-        # ---- end to end through the host-buffer entry point: H2D of q, k_new, v_new and D2H of out every step
-        hq = [n[2].cpu().pin_memory() for n in news]
-        hk = [n[0].cpu().pin_memory() for n in news]
-        hv = [n[1].cpu().pin_memory() for n in news]
-        hout = torch.empty_like(outs[0], device="cpu").pin_memory()
-        for i in range(3 * L):   # every layer's arguments seen often enough for the library to cache its launch
-            ctx.locks_decode_step_host(hq[i % L], hk[i % L], hv[i % L], kvs[i % L], summs[i % L], w0.n, hout, stream=stream)
-        ldist.barrier()
-        t0 = time.perf_counter()
-        for i in range(K):
-            li = (3 * L + i) % L
-            ctx.locks_decode_step_host(hq[li], hk[li], hv[li], kvs[li], summs[li], w0.n, hout, stream=stream)
-        e2e_ms = (time.perf_counter() - t0) * 1e3 / K
-    status = ctx.locks_poll_status()
-    step_ms_max = ldist.max_over_ranks(step_ms, device=dev)
-    e2e_ms_max = ldist.max_over_ranks(e2e_ms, device=dev)
+        res["dense_ms"] = d0.elapsed_time(d1) / nd
+        res["clocks"] = sampler.stop() if sampler else None
+        if full:
+            # ---- end to end through the host-buffer entry point: H2D of q, k_new, v_new and D2H of out every step
+            hq = [n[2].cpu().pin_memory() for n in news]
+            hk = [n[0].cpu().pin_memory() for n in news]
+            hv = [n[1].cpu().pin_memory() for n in news]
+            hout = torch.empty_like(outs[0], device="cpu").pin_memory()
+            for i in range(3 * L):   # every layer's arguments seen often enough for the library to cache its launch
+                ctx.locks_decode_step_host(hq[i % L], hk[i % L], hv[i % L], kvs[i % L], summs[i % L], w0.n, hout, stream=stream)
+            ldist.barrier()
+            t0 = time.perf_counter()
+            for i in range(K):
+                li = (3 * L + i) % L
+                ctx.locks_decode_step_host(hq[li], hk[li], hv[li], kvs[li], summs[li], w0.n, hout, stream=stream)
+            res["e2e_ms"] = (time.perf_counter() - t0) * 1e3 / K
+    res["status"] = ctx.locks_poll_status()
+    res["launches_per_step"] = launches_per_step
+    res["bulk_build_ms"] = bulk_build_ms
+    res["build_pages"] = build_pages
+    res["partition"] = {0: "none", 1: "strided", 2: "balanced"}.get(partition, str(partition))
+    res["max_pages"] = max_pages
+    ctx.close()
+    del graphs, pgraphs, layers, kvs, summs, outs, news
+    torch.cuda.empty_cache()
+    return res
+
+
+def table_row(args, name, K, W, rank, local_rank, peak):
+    w = workload(name)
+    r = measure(args, w, K, W, args.layers, rank, local_rank, full=False)
+    scan_b, att_b, dense_b = algorithmic_bytes(w)
+    step_us = r["step_ms"] * 1e3
+    return {"workload": w.name, "step_us": round(step_us, 2), "algorithmic_bytes": scan_b + att_b,
+            "frac_of_measured_peak": round((scan_b + att_b) / (step_us * 1e-6) / 1e9 / peak, 4),
+            "dense_us": round(r["dense_ms"] * 1e3, 2),
+            "stages_us": {k_: round(v * 1e3, 2) for k_, v in r["stage_ms"].items()},
+            "scan_frac": round(scan_b / (r["stage_ms"]["scan"] * 1e-3) / 1e9 / peak, 4) if scan_b else None,
+            "scan_partition": r["partition"], "bulk_build_ms_per_layer": round(r["bulk_build_ms"], 3),
+            "device_status": r["status"]}
+
+
+def run_ours(args):
+    import torch
+    from paper_2607_24555_b200 import dist as ldist
+
+    rank, local_rank, world = ldist.env_rank_world()
+    if world > 1:
+        import torch.distributed as tdist
+        tdist.init_process_group("nccl", device_id=torch.device(f"cuda:{local_rank}"))
+    torch.cuda.set_device(local_rank)
+    dev = f"cuda:{local_rank}"
+    K, W = args.steps, max(args.warmup, 3)
+    w0 = workload(args.workload)
+    L = args.layers
+    # every rank owns a full batch (weak scaling): requests are independent, no data-path collective
+    r = measure(args, w0, K, W, L, rank, local_rank, full=True)
+    step_ms_max = ldist.max_over_ranks(r["step_ms"], device=dev)
+    e2e_ms_max = ldist.max_over_ranks(r["e2e_ms"], device=dev)
+    peak, peak_kind = measured_peak()
+    rows = []
+    if args.table and world == 1 and rank == 0:
+        for name in args.table.split(","):
+            if name and workload(name).name != w0.name:
+                rows.append(table_row(args, name, 16, 3, rank, local_rank, peak))
     if rank != 0:
         return
+    stage_ms = r["stage_ms"]
     scan_b, att_b, dense_b = algorithmic_bytes(w0)
-    peak, peak_kind = measured_peak()
     scan_gbs = scan_b / (stage_ms["scan"] * 1e-3) / 1e9
     esz = 2 if w0.dtype == "bf16" else 4
     h2d = w0.n * (w0.Hq + 2 * w0.Hkv) * w0.d * esz
@@ -341,26 +417,41 @@ def run_ours(args):
     if not args.no_cpu_baseline:
         import oracle
         cores = oracle.max_threads()
-        cpu_us, cpu_sample, _ = oracle_sample(w0, 2, cores)
+        cpu_us, cpu_sample, _ = oracle_sample(w0, 5, cores)
+    wins = r["windows_us"]
+    build_bytes = r["build_pages"] * (4096 + 818)
+    traffic, traffic_src = recorded_traffic(w0.name)
+    cfg_d = config_dict(w0, L, args.identity_blocks, r["partition"])
+    cfg_d["start_lengths"] = "context minus 1..16 tokens, staggered per request and layer: steps include the summary " \
+                             "build of the pages that fill"
     line = {
         "metric": METRIC, "value": step_ms_max * 1e3, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": step_ms_max, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16" if w0.dtype == "bf16" else "f32", "data": "synthetic",
-        "config": config_dict(w0, L, args.identity_blocks, args.scan_partition),
+        "config": cfg_d,
         "e2e": {"value": e2e_ms_max * 1e3, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
-        "gpu_launches": launches_per_step * K,
-        "clocks": clocks,
+        "gpu_launches": r["launches_per_step"] * K,
+        "clocks": r["clocks"],
         "roofline": {"bound": "hbm", "kernel": "scan_i4_kernel", "achieved": scan_gbs, "peak": peak, "unit": "GB/s",
-                     "frac": scan_gbs / peak, "peak_kind": f"of {peak_kind}", "traffic": recorded_traffic(w0.name),
+                     "frac": scan_gbs / peak, "peak_kind": f"of {peak_kind}", "traffic": traffic,
+                     "traffic_source": traffic_src,
                      "algorithmic_bytes_per_launch": scan_b, "launch_us": stage_ms["scan"] * 1e3},
         "step_roofline": {"algorithmic_bytes": scan_b + att_b, "achieved": (scan_b + att_b) / (step_ms_max * 1e-3) / 1e9,
                           "frac": (scan_b + att_b) / (step_ms_max * 1e-3) / 1e9 / peak, "unit": "GB/s",
                           "frac_of_8000": (scan_b + att_b) / (step_ms_max * 1e-3) / 1e9 / 8000.0},
+        "windows": {"replays_per_window": 64, "us_per_step": [round(x, 3) for x in wins],
+                    "mean_us": statistics.mean(wins) if wins else None,
+                    "sd_us": statistics.stdev(wins) if len(wins) > 1 else None},
         "stages_us": {k_: v * 1e3 for k_, v in stage_ms.items()},
-        "dense_flash_decode": {"us": dense_ms * 1e3, "bytes": dense_b, "achieved_gbs": dense_b / (dense_ms * 1e-3) / 1e9,
-                               "speedup_of_step": dense_ms / step_ms_max},
-        "bulk_build_ms_per_layer": bulk_build_ms,
-        "device_status": status,
+        "dense_flash_decode": {"us": r["dense_ms"] * 1e3, "bytes": dense_b,
+                               "achieved_gbs": dense_b / (r["dense_ms"] * 1e-3) / 1e9,
+                               "speedup_of_step": r["dense_ms"] / step_ms_max},
+        "bulk_build_ms_per_layer": r["bulk_build_ms"],
+        "bulk_build": {"ms_per_layer": r["bulk_build_ms"], "page_heads": r["build_pages"], "algorithmic_bytes": build_bytes,
+                       "achieved_gbs": build_bytes / (r["bulk_build_ms"] * 1e-3) / 1e9,
+                       "frac": build_bytes / (r["bulk_build_ms"] * 1e-3) / 1e9 / peak},
+        "device_status": r["status"],
+        "workloads": rows,
         "cpu_baseline": ({"value": cpu_us, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": cpu_sample}
                          if cpu_us is not None else None),
     }
@@ -376,6 +467,9 @@ def main():
     ap.add_argument("--workload", default="cfg1")
     ap.add_argument("--layers", type=int, default=4)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--table", default="cfg2_r8_b1024,cfg3_1m,cfg4_b8",
+                    help="comma-separated workloads measured compactly (few steps) for the `workloads` table of the "
+                         "JSON line; empty: none")
     ap.add_argument("--scan-partition", default="auto", choices=["auto", "strided", "balanced"],
                     help="how the scan deals pages to its warps (auto: the library follows the lengths)")
     ap.add_argument("--identity-blocks", action="store_true",
