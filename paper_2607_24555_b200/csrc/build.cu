@@ -32,12 +32,18 @@ struct BuildParams {
   const int32_t *append_pos;
 };
 
+#ifndef LOCKS_BUILD_OFF_TOL
+#define LOCKS_BUILD_OFF_TOL 1e-13f   // squared off-diagonal norm over squared norm at which the sweeps stop
+#endif
 #ifndef LOCKS_BUILD_SWEEPS
 #define LOCKS_BUILD_SWEEPS 12   // upper bound; a page stops as soon as its off-diagonal norm is at rounding level
 #endif
-constexpr int kBuildWarps = 4;
-constexpr int kBuildCtasPerSm = 6;                               // 24 warps per SM: 80 registers, 8.4 KB per warp
-constexpr int kBuildScratch = 2 * 2 * LOCKS_B * LOCKS_B * 4;      // 4096 B: bf16 tile of D, then the exchange buffers
+constexpr int kBuildWarps = 3;
+constexpr int kBuildCtasPerSm = 6;                               // 18 warps per SM (bf16 keys: 11.3 KB per warp)
+constexpr int kBuildScratch = 2 * 2 * LOCKS_B * LOCKS_B * 4;      // 4096 B: bf16 half-tiles of D (hi | lo), then the exchange buffers
+template <typename T> __host__ __device__ constexpr int build_smem_per_warp() {      // raw key tile + scratch + A, U + misc + blob
+  return LOCKS_B * LOCKS_D * (int)sizeof(T) + kBuildScratch + (2 * LOCKS_B * 17 + 64) * 4 + i4_stride(8);
+}
 // Placement of a 16 x 16 matrix in an exchange buffer.  A round writes entry (row, column) with rows and
 // columns permuted (32 lanes x one scalar store: 8 rows x 4 columns) and reads it back row by row (8 rows x 4
 // columns again), 32 instructions per round in all, so bank conflicts are what a round costs.  The placement
@@ -52,12 +58,12 @@ __device__ __forceinline__ int jcol_part(int c) {   // 32 (c mod 4) + g(c)
   const int g = ((c & 3) == 3) ? (((c + 1) >> 2) & 3) : (c >> 2);
   return ((c & 3) << 5) + g;
 }
-constexpr int kBuildSmemPerWarp = kBuildScratch + (2 * LOCKS_B * 17 + 64) * 4 + i4_stride(8);
 
-__device__ __forceinline__ float round_code(float x, float scale, float qmax) {
-  if (scale == 0.f) return 0.f;
-  float c = rintf(__fdiv_rn(x, scale));
-  return fminf(fmaxf(c, -qmax), qmax);
+// code = clamp(rint(x / scale)); `inv` = 1 / scale correctly rounded (0 for a zero scale: all codes 0).  The
+// product differs from the quotient by at most an ulp, which matters only within an ulp of a rounding boundary.
+__device__ __forceinline__ float inv_scale(float scale) { return scale == 0.f ? 0.f : __frcp_rn(scale); }
+__device__ __forceinline__ float round_code(float x, float inv, float qmax) {
+  return fminf(fmaxf(rintf(x * inv), -qmax), qmax);
 }
 
 // packed fp32 pairs (two independent lanes of arithmetic per instruction)
@@ -107,80 +113,99 @@ __global__ void __launch_bounds__(kBuildWarps * 32, kBuildCtasPerSm) build_kerne
     if (lane == 0) set_status(p.status, LOCKS_ERR_BAD_BLOCK);
     return;
   }
-  uint8_t *scratch = smem_raw + warp * kBuildSmemPerWarp;                        // D tile, then exchange buffers
+  // Loops over the 16 keys stay rolled: a warp runs through this code once per page, and when a page fills inside
+  // a decode step the code is cold, so its length in instructions is part of the latency.  The page's keys are
+  // staged in shared memory once and every phase reads them from there.
+  constexpr int kRawBytes = LOCKS_B * LOCKS_D * (int)sizeof(T);
+  constexpr int kRowBytes = LOCKS_D * (int)sizeof(T);
+  uint8_t *raw = smem_raw + warp * build_smem_per_warp<T>();                      // [16][128] keys as stored
+  uint8_t *scratch = raw + kRawBytes;                                             // D half-tiles, then exchange buffers
   float *A = reinterpret_cast<float *>(scratch + kBuildScratch);                 // [16][17]
   float *U = A + LOCKS_B * 17;                                                    // [16][17] (first: the cross product)
   float *rot = U + LOCKS_B * 17;                                                  // misc
   uint8_t *blob = reinterpret_cast<uint8_t *>(rot + 64);
+  float *mus = reinterpret_cast<float *>(blob);                                   // centroid, until the blob is assembled
   const int r = p.r;
 
-  // ---- 1. load, centre.  The deviations are needed twice (Gram matrix now, basis after the eigenproblem); they
-  // are not kept in registers in between but fetched again (the page is 4 KB and still in cache).
-  const T *K = reinterpret_cast<const T *>(p.k) + (int64_t)block * p.sb + (int64_t)h * p.sh;
-  const T *Knew = reinterpret_cast<const T *>(p.k_new) + ((int64_t)b * p.Hkv + h) * LOCKS_D;
-  float mu[4] = {0.f, 0.f, 0.f, 0.f};
-  float knorm2 = 0.f;
-  auto load_keys = [&](float (&kv)[LOCKS_B][4]) {
-#pragma unroll
-    for (int i = 0; i < LOCKS_B; ++i) {
-      const T *row = (i == LOCKS_B - 1 && last_from_new) ? Knew : K + (int64_t)i * p.st;
-      if (sizeof(T) == 2) {
-        const uint2 w = *reinterpret_cast<const uint2 *>(reinterpret_cast<const uint16_t *>(row) + lane * 4);
-        kv[i][0] = __uint_as_float(w.x << 16); kv[i][1] = __uint_as_float(w.x & 0xFFFF0000u);
-        kv[i][2] = __uint_as_float(w.y << 16); kv[i][3] = __uint_as_float(w.y & 0xFFFF0000u);
-      } else {
-        const float4 w = *reinterpret_cast<const float4 *>(reinterpret_cast<const float *>(row) + lane * 4);
-        kv[i][0] = w.x; kv[i][1] = w.y; kv[i][2] = w.z; kv[i][3] = w.w;
-      }
+  // ---- 1. stage the keys, centroid
+  {
+    const uint8_t *K = reinterpret_cast<const uint8_t *>(p.k) + ((int64_t)block * p.sb + (int64_t)h * p.sh) * (int64_t)sizeof(T);
+    const uint8_t *Knew = reinterpret_cast<const uint8_t *>(p.k_new) + ((int64_t)b * p.Hkv + h) * kRowBytes;
+    constexpr int kCpr = kRowBytes / 16;   // 16-byte chunks per row
+#pragma unroll 4
+    for (int c = lane; c < LOCKS_B * kCpr; c += 32) {
+      const int row = c / kCpr, ch = c - row * kCpr;
+      const uint8_t *src = (row == LOCKS_B - 1 && last_from_new) ? Knew : K + (int64_t)row * p.st * (int64_t)sizeof(T);
+      cp_async16(raw + c * 16, src + ch * 16, true);
+    }
+    cp_async_commit();
+    cp_async_wait<0>();
+    __syncwarp();
+  }
+  auto key4 = [&](int row, int d0, float (&v)[4]) {   // keys (row, d0 .. d0 + 3) as fp32
+    if (sizeof(T) == 2) {
+      const uint2 w = *reinterpret_cast<const uint2 *>(raw + row * kRowBytes + d0 * 2);
+      v[0] = __uint_as_float(w.x << 16); v[1] = __uint_as_float(w.x & 0xFFFF0000u);
+      v[2] = __uint_as_float(w.y << 16); v[3] = __uint_as_float(w.y & 0xFFFF0000u);
+    } else {
+      const float4 w = *reinterpret_cast<const float4 *>(raw + row * kRowBytes + d0 * 4);
+      v[0] = w.x; v[1] = w.y; v[2] = w.z; v[3] = w.w;
     }
   };
+  float mu[4] = {0.f, 0.f, 0.f, 0.f};   // of this lane's dims 4 lane .. 4 lane + 3
+  float knorm2 = 0.f;
+#pragma unroll 4
+  for (int i = 0; i < LOCKS_B; ++i) {
+    float v[4];
+    key4(i, 4 * lane, v);
+#pragma unroll
+    for (int u = 0; u < 4; ++u) { mu[u] += v[u]; knorm2 = fmaf(v[u], v[u], knorm2); }
+  }
+  knorm2 = warp_sum(knorm2);
+#pragma unroll
+  for (int u = 0; u < 4; ++u) mu[u] *= (1.f / LOCKS_B);
+  *reinterpret_cast<float4 *>(mus + 4 * lane) = make_float4(mu[0], mu[1], mu[2], mu[3]);
+  __syncwarp();
   // ---- 2. Gram matrix M = D D^T on the tensor cores.  D = H + L with H = bf16(D), L = bf16(D - H) (16 significant
   // bits; the bf16 products are exact and accumulate in fp32): M = (H H^T + L L^T) + H L^T + (H L^T)^T.  The A
   // operand (tokens x dims) and the B operand (dims x tokens) of an m16n8k16 step are the same registers.
+  // Two passes over 64 dims each: the half-tiles of H and L (16 rows x 128 bytes, 16-byte chunks XOR-swizzled with
+  // the row so that ldmatrix reads are conflict-free) share the 4 KB of scratch.
   {
-    float kv[LOCKS_B][4];
-    load_keys(kv);
-#pragma unroll
-    for (int i = 0; i < LOCKS_B; ++i)
-#pragma unroll
-      for (int u = 0; u < 4; ++u) { mu[u] += kv[i][u]; knorm2 = fmaf(kv[i][u], kv[i][u], knorm2); }
-    knorm2 = warp_sum(knorm2);
-#pragma unroll
-    for (int u = 0; u < 4; ++u) mu[u] *= (1.f / LOCKS_B);
-    // lane owns dims 4 lane .. 4 lane + 3: 8 bytes of 16-byte chunk lane / 2 of every token row (256-byte rows,
-    // chunks XOR-swizzled with the token so that ldmatrix reads are conflict-free)
-    uint2 lo_pk[LOCKS_B];
-#pragma unroll
-    for (int i = 0; i < LOCKS_B; ++i) {
-      float dv[4];
-#pragma unroll
-      for (int u = 0; u < 4; ++u) dv[u] = kv[i][u] - mu[u];
-      const uint32_t h01 = pack_bf16(dv[0], dv[1]), h23 = pack_bf16(dv[2], dv[3]);
-      lo_pk[i].x = pack_bf16(dv[0] - __uint_as_float(h01 << 16), dv[1] - __uint_as_float(h01 & 0xFFFF0000u));
-      lo_pk[i].y = pack_bf16(dv[2] - __uint_as_float(h23 << 16), dv[3] - __uint_as_float(h23 & 0xFFFF0000u));
-      *reinterpret_cast<uint2 *>(scratch + i * 256 + ((((lane >> 1) ^ (i & 7)) << 4) | ((lane & 1) << 3))) = make_uint2(h01, h23);
-    }
-    __syncwarp();
-    const int mq = lane >> 3, rr = lane & 7, tok = (mq & 1) * 8 + rr;
-    uint32_t Hf[8][4];
-#pragma unroll
-    for (int s = 0; s < 8; ++s) ldsm_x4(Hf[s], scratch + tok * 256 + (((2 * s + (mq >> 1)) ^ (tok & 7)) << 4));
-    __syncwarp();
-#pragma unroll
-    for (int i = 0; i < LOCKS_B; ++i)
-      *reinterpret_cast<uint2 *>(scratch + i * 256 + ((((lane >> 1) ^ (i & 7)) << 4) | ((lane & 1) << 3))) = lo_pk[i];
-    __syncwarp();
     float X0[4] = {0.f, 0.f, 0.f, 0.f}, X1[4] = {0.f, 0.f, 0.f, 0.f}, Y0[4] = {0.f, 0.f, 0.f, 0.f}, Y1[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-    for (int s = 0; s < 8; ++s) {
-      uint32_t Lf[4];
-      ldsm_x4(Lf, scratch + tok * 256 + (((2 * s + (mq >> 1)) ^ (tok & 7)) << 4));
-      mma_bf16(X0, Hf[s][0], Hf[s][1], Hf[s][2], Hf[s][3], Hf[s][0], Hf[s][2]);
-      mma_bf16(X1, Hf[s][0], Hf[s][1], Hf[s][2], Hf[s][3], Hf[s][1], Hf[s][3]);
-      mma_bf16(X0, Lf[0], Lf[1], Lf[2], Lf[3], Lf[0], Lf[2]);
-      mma_bf16(X1, Lf[0], Lf[1], Lf[2], Lf[3], Lf[1], Lf[3]);
-      mma_bf16(Y0, Hf[s][0], Hf[s][1], Hf[s][2], Hf[s][3], Lf[0], Lf[2]);
-      mma_bf16(Y1, Hf[s][0], Hf[s][1], Hf[s][2], Hf[s][3], Lf[1], Lf[3]);
+    const int rh = lane >> 4, c16 = lane & 15;                      // writer: rows 8 rh .. 8 rh + 7, dims 4 c16 .. + 3 of the half
+    const int mq = lane >> 3, rr = lane & 7, tok = (mq & 1) * 8 + rr;   // reader (ldmatrix address lanes)
+#pragma unroll 1
+    for (int hf = 0; hf < 2; ++hf) {
+      const float4 m4 = *reinterpret_cast<const float4 *>(mus + 64 * hf + 4 * c16);
+#pragma unroll 2
+      for (int i = 0; i < 8; ++i) {
+        const int row = 8 * rh + i;
+        float v[4];
+        key4(row, 64 * hf + 4 * c16, v);
+        v[0] -= m4.x; v[1] -= m4.y; v[2] -= m4.z; v[3] -= m4.w;
+        const uint32_t h01 = pack_bf16(v[0], v[1]), h23 = pack_bf16(v[2], v[3]);
+        const uint32_t l01 = pack_bf16(v[0] - __uint_as_float(h01 << 16), v[1] - __uint_as_float(h01 & 0xFFFF0000u));
+        const uint32_t l23 = pack_bf16(v[2] - __uint_as_float(h23 << 16), v[3] - __uint_as_float(h23 & 0xFFFF0000u));
+        uint8_t *dst = scratch + row * 128 + ((((c16 >> 1) ^ (row & 7)) << 4) | ((c16 & 1) << 3));
+        *reinterpret_cast<uint2 *>(dst) = make_uint2(h01, h23);
+        *reinterpret_cast<uint2 *>(dst + 2048) = make_uint2(l01, l23);
+      }
+      __syncwarp();
+#pragma unroll 1
+      for (int s4 = 0; s4 < 4; ++s4) {
+        uint32_t Hf[4], Lf[4];
+        const uint8_t *src = scratch + tok * 128 + (((2 * s4 + (mq >> 1)) ^ (tok & 7)) << 4);
+        ldsm_x4(Hf, src);
+        ldsm_x4(Lf, src + 2048);
+        mma_bf16(X0, Hf[0], Hf[1], Hf[2], Hf[3], Hf[0], Hf[2]);
+        mma_bf16(X1, Hf[0], Hf[1], Hf[2], Hf[3], Hf[1], Hf[3]);
+        mma_bf16(X0, Lf[0], Lf[1], Lf[2], Lf[3], Lf[0], Lf[2]);
+        mma_bf16(X1, Lf[0], Lf[1], Lf[2], Lf[3], Lf[1], Lf[3]);
+        mma_bf16(Y0, Hf[0], Hf[1], Hf[2], Hf[3], Lf[0], Lf[2]);
+        mma_bf16(Y1, Hf[0], Hf[1], Hf[2], Hf[3], Lf[1], Lf[3]);
+      }
+      __syncwarp();
     }
     // accumulator (x = lane / 4, t = lane % 4): [0..1] = row x, columns 2t, 2t+1; [2..3] = row x + 8
     const int x = lane >> 2, t = lane & 3;
@@ -267,7 +292,7 @@ __global__ void __launch_bounds__(kBuildWarps * 32, kBuildCtasPerSm) build_kerne
           off += (dg && dblk == 1) ? 0.f : pa[rb][cb].y * pa[rb][cb].y;
         }
       off = warp_sum(off);
-      if (off <= 1e-13f * normA || normA == 0.f) break;
+      if (off <= LOCKS_BUILD_OFF_TOL * normA || normA == 0.f) break;
 #pragma unroll 1
       for (int round = 0; round < 15; ++round) {
         // rotation of the slot pair held as a diagonal block (other lanes compute on whatever they hold; unused)
@@ -275,14 +300,18 @@ __global__ void __launch_bounds__(kBuildWarps * 32, kBuildCtasPerSm) build_kerne
         const float aqq = dblk ? pa[1][1].y : pa[1][1].x;
         float c = 1.f, sn = 0.f;
         {
-          // tan of the rotation angle: t = 2 apq / (d + sign(d) sqrt(d^2 + 4 apq^2)), d = aqq - app (the smaller
-          // root).  Approximate root and division are enough for the angle; c^2 + s^2 = 1 comes from the last
-          // two lines.  Entries too small to square are left alone.
+          // The rotation that annihilates apq, smaller angle: with d = aqq - app and h = d^2 + 4 apq^2,
+          // cos 2t = |d| / sqrt(h) and sin 2t = 2 apq sign(d) / sqrt(h), so c = sqrt((1 + cos 2t) / 2) and
+          // s = sin 2t / (2 c): two reciprocal square roots in a row (approximate ones are enough for the angle;
+          // c^2 + s^2 = 1 holds to their rounding).  Entries too small to square are left alone.
           const float d = aqq - app, hh = d * d + 4.f * apq * apq;
           if (hh > 1e-37f && hh < 1e37f) {
-            const float tt = __fdividef(2.f * apq, d + copysignf(hh * rsqrtf(hh), d));
-            c = rsqrtf(tt * tt + 1.f);
-            sn = tt * c;
+            const float rs = rsqrtf(hh);
+            const float x = fmaf(0.5f * fabsf(d), rs, 0.5f);
+            const float r2 = rsqrtf(x);
+            c = x * r2;
+            sn = copysignf(apq * rs * r2, apq * d);
+            if (d == 0.f) sn = copysignf(fabsf(sn), apq);
           }
         }
         const float cr = __shfl_sync(0xffffffffu, c, src_row), sr = __shfl_sync(0xffffffffu, sn, src_row);
@@ -361,12 +390,6 @@ __global__ void __launch_bounds__(kBuildWarps * 32, kBuildCtasPerSm) build_kerne
   float *fout = reinterpret_cast<float *>(p.summ + ((int64_t)block * p.Hkv + h) * p.S);
   uint32_t sign_bits = 0u;   // bit l: mode l was flipped
   {
-    float kv[LOCKS_B][4];
-    load_keys(kv);
-#pragma unroll
-    for (int i = 0; i < LOCKS_B; ++i)
-#pragma unroll
-      for (int u = 0; u < 4; ++u) kv[i][u] -= mu[u];
 #pragma unroll 1
     for (int l = 0; l < r; ++l) {
       float v[4] = {0.f, 0.f, 0.f, 0.f};
@@ -377,8 +400,10 @@ __global__ void __launch_bounds__(kBuildWarps * 32, kBuildCtasPerSm) build_kerne
 #pragma unroll
         for (int i = 0; i < LOCKS_B; ++i) {
           const float u = U[i * 17 + col];
+          float kd[4];
+          key4(i, 4 * lane, kd);
 #pragma unroll
-          for (int c = 0; c < 4; ++c) v[c] = fmaf(kv[i][c], u, v[c]);
+          for (int c = 0; c < 4; ++c) v[c] = fmaf(kd[c] - mu[c], u, v[c]);
         }
 #pragma unroll
         for (int c = 0; c < 4; ++c) v[c] *= inv;
@@ -401,7 +426,7 @@ __global__ void __launch_bounds__(kBuildWarps * 32, kBuildCtasPerSm) build_kerne
         *reinterpret_cast<float4 *>(fout + LOCKS_D + l * LOCKS_D + lane * 4) = make_float4(v[0], v[1], v[2], v[3]);
       } else {
         const __half sh = __float2half_rn(best / 7.f);
-        const float sc = __half2float(sh);
+        const float sc = inv_scale(__half2float(sh));
         if (lane == 0) *reinterpret_cast<__half *>(blob + i4_off_sv(r) + 2 * l) = sh;
         // lane = 8 t + s owns dims 32 t + 4 s + {0,1,2,3} = (half, e) in {0,1}^2 of k-step s
         const int t = lane >> 3, s = lane & 7, i0 = (s & 1) << 1;
@@ -432,7 +457,7 @@ __global__ void __launch_bounds__(kBuildWarps * 32, kBuildCtasPerSm) build_kerne
       for (int l = 0; l < r; ++l) fout[LOCKS_D + r * LOCKS_D + lane * r + l] = cf[l & 15];
     } else {
       const __half sh = __float2half_rn(mx / 127.f);
-      const float sc = __half2float(sh);
+      const float sc = inv_scale(__half2float(sh));
       const int tpos = ((lane & 7) >> 1) * 4 + (lane >> 3) * 2 + (lane & 1);
       *reinterpret_cast<__half *>(blob + i4_off_sc(r) + 2 * tpos) = sh;
       const int xx = lane & 7, hi = lane >> 3;
@@ -448,7 +473,7 @@ __global__ void __launch_bounds__(kBuildWarps * 32, kBuildCtasPerSm) build_kerne
     float mx = fmaxf(fmaxf(fabsf(mu[0]), fabsf(mu[1])), fmaxf(fabsf(mu[2]), fabsf(mu[3])));
     mx = __uint_as_float(__reduce_max_sync(0xffffffffu, __float_as_uint(mx)));
     const __half sh = __float2half_rn(mx / 127.f);
-    const float sc = __half2float(sh);
+    const float sc = inv_scale(__half2float(sh));
     if (lane == 0) *reinterpret_cast<__half *>(blob + i4_off_smu(r)) = sh;
     uint32_t bytes[4];
 #pragma unroll
@@ -481,13 +506,14 @@ int locks_launch_build(locks_ctx *c, const locks_kv *kv, int batch, const int32_
   }
   dim3 grid = just_filled ? dim3((batch * p.Hkv + kBuildWarps - 1) / kBuildWarps)
                           : dim3((c->Pmax + kBuildWarps - 1) / kBuildWarps, p.Hkv, batch);
-  const int smem = kBuildWarps * kBuildSmemPerWarp;
   const bool bf = c->cfg.kv_dtype == LOCKS_BF16, i4 = c->cfg.summary_fmt == LOCKS_FMT_I4;
+  const int smem_bf = kBuildWarps * build_smem_per_warp<__nv_bfloat16>(), smem_f32 = kBuildWarps * build_smem_per_warp<float>();
+  const int smem = bf ? smem_bf : smem_f32;
   if (locks_attrs_needed(LOCKS_ATTR_BUILD)) {
-    cudaFuncSetAttribute(build_kernel<__nv_bfloat16, LOCKS_FMT_I4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    cudaFuncSetAttribute(build_kernel<__nv_bfloat16, LOCKS_FMT_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    cudaFuncSetAttribute(build_kernel<float, LOCKS_FMT_I4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    cudaFuncSetAttribute(build_kernel<float, LOCKS_FMT_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    cudaFuncSetAttribute(build_kernel<__nv_bfloat16, LOCKS_FMT_I4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bf);
+    cudaFuncSetAttribute(build_kernel<__nv_bfloat16, LOCKS_FMT_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bf);
+    cudaFuncSetAttribute(build_kernel<float, LOCKS_FMT_I4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_f32);
+    cudaFuncSetAttribute(build_kernel<float, LOCKS_FMT_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_f32);
   }
   if (bf && i4) build_kernel<__nv_bfloat16, LOCKS_FMT_I4><<<grid, kBuildWarps * 32, smem, st>>>(p);
   else if (bf) build_kernel<__nv_bfloat16, LOCKS_FMT_F32><<<grid, kBuildWarps * 32, smem, st>>>(p);
