@@ -141,6 +141,25 @@ int locks_select(locks_ctx *ctx, const void *q, const void *summaries, const loc
 int locks_select_exact(locks_ctx *ctx, const void *q, const locks_kv *kv, int batch, int32_t *page_ids,
                        int32_t *page_count, float *page_logmass, float *page_logshare, locks_stream stream);
 
+/* Rival page scorers the paper measures the summary against (App. B selection-fidelity table; Sec. 2 / App. A),
+ * run through the SAME combine and selection as locks_select, for diagnostics:
+ *   LOCKS_SCORER_CENTROID  q.mu_j/sqrt(d) + log B: the centroid term of Eq. 1 alone (from the stored summary);
+ *   LOCKS_SCORER_MOMENT    the rank-r moment core, Eq. 3: q.mu_j/sqrt(d) + log B + (1/(2 B d)) sum_{l<=r} sigma_l^2
+ *                          (v_l.q)^2, i.e. the second-cumulant truncation of the page mass, computed from the
+ *                          stored summary as (1/(2B)) sum_i z_i^2 with z_i the reconstructed within-page logits;
+ *   LOCKS_SCORER_ENVELOPE  the min/max envelope (Quest), Lemma 2: sum_c max(q_c u_jc, q_c l_jc)/sqrt(d) with the
+ *                          per-dimension key extremes u, l of the page, computed from the K pages (`summaries`
+ *                          may be NULL).
+ * page_score (optional) [batch][Hq][max_pages_per_seq]: the rival's score of pages 0..P-2 (envelope: 0..P-1);
+ * page_logshare (optional): its ranking key.  Plain fp32 kernels: a measuring device, not a fast path. */
+#define LOCKS_SCORER_SUMMARY 0
+#define LOCKS_SCORER_CENTROID 1
+#define LOCKS_SCORER_MOMENT 2
+#define LOCKS_SCORER_ENVELOPE 3
+int locks_select_rival(locks_ctx *ctx, int scorer, const void *q, const void *summaries, const locks_kv *kv, int batch,
+                       int32_t *page_ids, int32_t *page_count, float *page_score, float *page_logshare,
+                       locks_stream stream);
+
 /* Selection fidelity of a page table against exact masses (the paper's App. B "microscope" metrics), per
  * (request, KV head), means over the heads of the group:
  *   quality[(b*Hkv + h)*4 + 0] = gamma    total attention mass captured:  sum_{j in S} e^{s_j} / sum_{j<P} e^{s_j}

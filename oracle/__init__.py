@@ -53,6 +53,8 @@ def lib():
         L.ora_summary_stride_bytes.restype = C.c_int64
         L.ora_score.restype = C.c_double
         L.ora_exact_lse.restype = C.c_double
+        L.ora_rival_score.restype = C.c_double
+        L.ora_envelope_score.restype = C.c_double
         L.ora_build_page.restype = C.c_int
         L.ora_select_one.restype = C.c_int
         L.ora_select_one_rule.restype = C.c_int
@@ -151,6 +153,24 @@ def exact_lse(keys, q, sm_scale: float) -> float:
     return float(lib().ora_exact_lse(C.c_int(n), C.c_int(d), _p(keys), _p(q), C.c_double(sm_scale)))
 
 
+SCORER_CENTROID, SCORER_MOMENT, SCORER_ENVELOPE = 1, 2, 3
+
+
+def rival_score(scorer: int, mu, V, Cc, q, sm_scale: float) -> float:
+    """Centroid-only (1) or rank-r moment-core (2) score of one page from its summary."""
+    mu, V, Cc, q = _f64(mu), _f64(V), _f64(Cc), _f64(q)
+    r, d = V.shape
+    B = Cc.shape[0]
+    return float(lib().ora_rival_score(C.c_int(scorer), C.c_int(B), C.c_int(d), C.c_int(r), _p(mu), _p(V), _p(Cc), _p(q),
+                                       C.c_double(sm_scale)))
+
+
+def envelope_score(keys, q, sm_scale: float) -> float:
+    keys, q = _f64(keys), _f64(q)
+    n, d = keys.shape
+    return float(lib().ora_envelope_score(C.c_int(n), C.c_int(d), _p(keys), _p(q), C.c_double(sm_scale)))
+
+
 def select_one(s, P: int, k: int):
     """s [G, >=P] page scores of one KV head -> (ids [k] ascending/-1 padded, count, log m_bar [P])."""
     s = _f64(s)
@@ -238,6 +258,16 @@ def page_logmass(cache: Cache, q, r: int, fmt: int, summaries, sm_scale: float, 
     lib().ora_page_logmass(cache.ref(), C.c_int(cache.batch), _p(q), C.c_int(qd), C.c_int(r), C.c_int(fmt),
                            _p(summ), C.c_double(sm_scale), C.c_int(1 if exact else 0), _p(shat))
     return shat
+
+
+def rival_logmass(cache: Cache, q, r: int, fmt: int, summaries, sm_scale: float, scorer: int):
+    """Rival scores of every page: [batch, Hq, max_pages] (NaN where a scorer has no value)."""
+    q, qd = _q_arg(q)
+    out = np.full((cache.batch, cache.Hq, cache.max_pages), np.nan)
+    summ = np.ascontiguousarray(summaries, dtype=np.uint8) if summaries is not None else None
+    lib().ora_rival_logmass(cache.ref(), C.c_int(cache.batch), _p(q), C.c_int(qd), C.c_int(r), C.c_int(fmt), _p(summ),
+                            C.c_double(sm_scale), C.c_int(scorer), _p(out))
+    return out
 
 
 def select(cache: Cache, shat, k: int):

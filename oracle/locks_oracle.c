@@ -399,6 +399,50 @@ double ora_score(int B, int d, int r, const double *mu, const double *V, const d
   return mx + log(z);
 }
 
+/* Rival page scores the paper measures the summary against (App. A / App. B), from the same summary:
+ *   scorer 1, centroid only:  q.mu/sqrt(d) + log B
+ *   scorer 2, rank-r moment core (Eq. 3): q.mu/sqrt(d) + log B + (1/(2 B d)) sum_{l<=r} sigma_l^2 (v_l.q)^2.
+ *             With z_i = (V^T q).c_i / sqrt(d) the reconstructed within-page logits, sum_i z_i^2 equals
+ *             (1/d) sum_l sigma_l^2 (v_l.q)^2 because the columns of C = U_r Sigma_r are orthogonal with squared
+ *             norms sigma_l^2; the score is evaluated in that form, (1/(2B)) sum_i z_i^2, so that it is defined
+ *             by the stored (possibly quantised) values alone. */
+double ora_rival_score(int scorer, int B, int d, int r, const double *mu, const double *V, const double *C,
+                       const double *q, double sm_scale) {
+  double a = 0;
+  for (int c = 0; c < d; ++c) a += mu[c] * q[c];
+  double s = sm_scale * a + log((double)B);
+  if (scorer == 2) {
+    double *p = (double *)malloc(sizeof(double) * r);
+    for (int l = 0; l < r; ++l) {
+      p[l] = 0;
+      for (int c = 0; c < d; ++c) p[l] += V[l * d + c] * q[c];
+    }
+    double z2 = 0;
+    for (int i = 0; i < B; ++i) {
+      double z = 0;
+      for (int l = 0; l < r; ++l) z += p[l] * C[i * r + l];
+      z2 += (sm_scale * z) * (sm_scale * z);
+    }
+    s += z2 / (2.0 * B);
+    free(p);
+  }
+  return s;
+}
+
+/* The min/max envelope score (Lemma 2): sum_c max(q_c u_c, q_c l_c) * sm_scale over the first ntok keys. */
+double ora_envelope_score(int ntok, int d, const double *keys, const double *q, double sm_scale) {
+  double e = 0;
+  for (int c = 0; c < d; ++c) {
+    double u = -INFINITY, l = INFINITY;
+    for (int i = 0; i < ntok; ++i) {
+      if (keys[i * d + c] > u) u = keys[i * d + c];
+      if (keys[i * d + c] < l) l = keys[i * d + c];
+    }
+    e += (q[c] * u > q[c] * l) ? q[c] * u : q[c] * l;
+  }
+  return sm_scale * e;
+}
+
 /* exact page log-mass of Lemma 1(ii) over the first ntok keys (rows of keys, ntok x d) */
 double ora_exact_lse(int ntok, int d, const double *keys, const double *q, double sm_scale) {
   double mx = -INFINITY, logit[1024];
@@ -489,6 +533,39 @@ void ora_page_logmass(const ora_kv *kv, int batch, const void *q, int q_dtype, i
           shat[((int64_t)b * kv->Hq + g) * kv->max_pages + p] =
               exact ? ora_exact_lse(B, d, keys, qd, sm_scale)
                     : ora_score(B, d, r, mu, V, C, qd, sm_scale);
+        }
+      }
+      free(keys); free(mu); free(V); free(C); free(qd);
+    }
+}
+
+/* Rival scores of every page (scorer 1, 2: pages 0..P-2 from the summaries; scorer 3, envelope: pages 0..P-1 from
+ * the keys): out[(b*Hq + g)*max_pages + p]. */
+void ora_rival_logmass(const ora_kv *kv, int batch, const void *q, int q_dtype, int r, int fmt,
+                       const uint8_t *summaries, double sm_scale, int scorer, double *out) {
+  int B = kv->B, d = kv->d, G = kv->Hq / kv->Hkv;
+  int64_t stride = ora_summary_stride_bytes(fmt, r, B, d);
+#pragma omp parallel for collapse(2) num_threads(g_threads) schedule(dynamic)
+  for (int b = 0; b < batch; ++b)
+    for (int h = 0; h < kv->Hkv; ++h) {
+      int T = kv->seq_lens[b], P = num_pages(T, B);
+      double *keys = (double *)malloc(sizeof(double) * B * d);
+      double *mu = (double *)malloc(sizeof(double) * d);
+      double *V = (double *)malloc(sizeof(double) * r * d);
+      double *C = (double *)malloc(sizeof(double) * B * r);
+      double *qd = (double *)malloc(sizeof(double) * d);
+      int last = scorer == 3 ? P : P - 1;
+      for (int p = 0; p < last; ++p) {
+        int block = kv->block_table[(int64_t)b * kv->max_pages + p];
+        int ntok = T - p * B < B ? T - p * B : B;
+        if (scorer == 3) load_page_keys(kv, kv->k, block, h, ntok, keys);
+        else ora_unpack(fmt, r, B, d, summaries + ((int64_t)block * kv->Hkv + h) * stride, mu, V, C);
+        for (int gi = 0; gi < G; ++gi) {
+          int g = h * G + gi;
+          for (int c = 0; c < d; ++c) qd[c] = load_elem(q, q_dtype, ((int64_t)b * kv->Hq + g) * d + c);
+          out[((int64_t)b * kv->Hq + g) * kv->max_pages + p] =
+              scorer == 3 ? ora_envelope_score(ntok, d, keys, qd, sm_scale)
+                          : ora_rival_score(scorer, B, d, r, mu, V, C, qd, sm_scale);
         }
       }
       free(keys); free(mu); free(V); free(C); free(qd);

@@ -18,10 +18,12 @@ SYMBOLS = ["locks_summary_bytes", "locks_workspace_bytes", "locks_create", "lock
            "locks_decode_step_host", "locks_poll_status", "locks_last_launch_count", "locks_strerror",
            "locks_profile_begin", "locks_profile_end", "locks_profile_read", "locks_sparse_attend_noalloc",
            "locks_set_scan_partition", "locks_selftest_wait_timeout", "locks_last_scan_partition",
-           "locks_host_cache_clear", "locks_select_exact", "locks_selection_quality"]
+           "locks_host_cache_clear", "locks_select_exact", "locks_selection_quality",
+           "locks_select_rival"]
 
 
 PARTITION_AUTO, PARTITION_STRIDED, PARTITION_BALANCED = 0, 1, 2   # LOCKS_PARTITION_* of include/locks.h
+SCORER_SUMMARY, SCORER_CENTROID, SCORER_MOMENT, SCORER_ENVELOPE = 0, 1, 2, 3   # LOCKS_SCORER_*
 
 
 class LocksError(RuntimeError):
@@ -87,6 +89,8 @@ def lib():
         L.locks_last_scan_partition.restype = C.c_int
         L.locks_host_cache_clear.argtypes = [vp]
         L.locks_host_cache_clear.restype = C.c_int
+        L.locks_select_rival.argtypes = [vp, C.c_int, vp, vp, C.POINTER(KV), C.c_int, i32p, i32p, vp, vp, vp]
+        L.locks_select_rival.restype = C.c_int
         L.locks_select_exact.argtypes = [vp, vp, C.POINTER(KV), C.c_int, i32p, i32p, vp, vp, vp]
         L.locks_select_exact.restype = C.c_int
         L.locks_selection_quality.argtypes = [vp, vp, C.POINTER(KV), C.c_int, i32p, i32p, i32p, i32p, i32p, C.c_int, vp, vp]
@@ -211,6 +215,13 @@ class Context:
         s = kv.struct()
         _check(lib().locks_select_exact(self.handle, _ptr(q), C.byref(s), batch, _ptr(page_ids), _ptr(page_count),
                                         _ptr(page_logmass), _ptr(page_logshare), _stream(stream)), "locks_select_exact")
+
+    def locks_select_rival(self, scorer, q, summaries, kv: KVView, batch, page_ids, page_count, page_score=None,
+                           page_logshare=None, stream=None):
+        s = kv.struct()
+        _check(lib().locks_select_rival(self.handle, int(scorer), _ptr(q), _ptr(summaries), C.byref(s), batch,
+                                        _ptr(page_ids), _ptr(page_count), _ptr(page_score), _ptr(page_logshare),
+                                        _stream(stream)), "locks_select_rival")
 
     def locks_selection_quality(self, exact_logmass, kv: KVView, batch, page_ids, page_count, ref_ids, ref_count,
                                 quality, marked_pages=None, stream=None):

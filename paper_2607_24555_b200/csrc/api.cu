@@ -158,6 +158,7 @@ int locks_create(const locks_config *cfg, void *workspace, size_t ws_bytes, lock
   c->part_balanced = 0;
   c->scan_partition = LOCKS_PARTITION_AUTO;
   c->last_partition = 0;
+  c->scorer = LOCKS_SCORER_SUMMARY;
   c->hint_host = nullptr; c->hint_dev = nullptr;
   {   // one page-locked word the device can write and the host can read without synchronising
     void *hp = nullptr, *dp = nullptr;
@@ -298,7 +299,30 @@ int locks_select_exact(locks_ctx *ctx, const void *q, const locks_kv *kv, int ba
   cudaStream_t st = (cudaStream_t)stream;
   ctx->last_launches = 0;
   float *shat = page_logmass ? page_logmass : ctx->shat;
-  if ((rc = locks_launch_exact_scan(ctx, q, kv, batch, shat, st)) != LOCKS_OK) return rc;
+  if ((rc = locks_launch_exact_scan(ctx, q, kv, batch, shat, 0, st)) != LOCKS_OK) return rc;
+  return locks_launch_select(ctx, shat, kv, batch, page_ids, page_count, page_logshare, nullptr, st);
+}
+
+int locks_select_rival(locks_ctx *ctx, int scorer, const void *q, const void *summaries, const locks_kv *kv, int batch,
+                       int32_t *page_ids, int32_t *page_count, float *page_score, float *page_logshare,
+                       locks_stream stream) {
+  int rc = check_common(ctx, kv, batch);
+  if (rc != LOCKS_OK) return rc;
+  if (!q || !page_ids || !page_count || ((uintptr_t)q % 16)) return LOCKS_ERR_INVALID_ARG;
+  if (scorer != LOCKS_SCORER_CENTROID && scorer != LOCKS_SCORER_MOMENT && scorer != LOCKS_SCORER_ENVELOPE)
+    return LOCKS_ERR_INVALID_ARG;
+  if (scorer != LOCKS_SCORER_ENVELOPE && (!summaries || ((uintptr_t)summaries % 16))) return LOCKS_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  ctx->last_launches = 0;
+  float *shat = page_score ? page_score : ctx->shat;
+  if (scorer == LOCKS_SCORER_ENVELOPE) {
+    rc = locks_launch_exact_scan(ctx, q, kv, batch, shat, 1, st);
+  } else {
+    ctx->scorer = scorer;
+    rc = locks_launch_scan(ctx, q, summaries, kv, batch, shat, 0, st);
+    ctx->scorer = LOCKS_SCORER_SUMMARY;
+  }
+  if (rc != LOCKS_OK) return rc;
   return locks_launch_select(ctx, shat, kv, batch, page_ids, page_count, page_logshare, nullptr, st);
 }
 

@@ -184,7 +184,9 @@ __global__ void __launch_bounds__(kExWarps * 32) exact_bf16_kernel(ExactParams p
 }
 
 // Plain fp32 arithmetic for any element type: one warp per page, a lane owns four dims.
-template <typename T>
+// ENV: instead of the exact log-mass, the min/max envelope score (the bound Quest ranks by, Lemma 2 of the paper):
+//   e_j(q) = sum_c max(q_c u_c, q_c l_c) / sqrt(d),  u_c / l_c = largest / smallest key entry of the page in dim c.
+template <typename T, bool ENV>
 __global__ void __launch_bounds__(kExWarps * 32) exact_generic_kernel(ExactParams p) {
   __shared__ float2 red[kExWarps][16];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -207,14 +209,29 @@ __global__ void __launch_bounds__(kExWarps * 32) exact_generic_kernel(ExactParam
       }
       const int ntok = min(LOCKS_B, Tn - page * LOCKS_B);
       const int64_t base = (int64_t)block * p.sb + (int64_t)h * p.sh;
-      float m = -INFINITY, s = 0.f;
-      for (int i = 0; i < ntok; ++i) {
-        float d = 0.f;
+      float v;
+      if (ENV) {
+        float hi[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY}, lo[4] = {INFINITY, INFINITY, INFINITY, INFINITY};
+        for (int i = 0; i < ntok; ++i)
 #pragma unroll
-        for (int u = 0; u < 4; ++u) d += qv[u] * ldf<T>(K, base + (int64_t)i * p.st + lane * 4 + u);
-        lse_push(m, s, warp_sum(d) * p.sm_scale);
+          for (int u = 0; u < 4; ++u) {
+            const float kk = ldf<T>(K, base + (int64_t)i * p.st + lane * 4 + u);
+            hi[u] = fmaxf(hi[u], kk); lo[u] = fminf(lo[u], kk);
+          }
+        float e = 0.f;
+#pragma unroll
+        for (int u = 0; u < 4; ++u) e += fmaxf(qv[u] * hi[u], qv[u] * lo[u]);
+        v = warp_sum(e) * p.sm_scale;
+      } else {
+        float m = -INFINITY, s = 0.f;
+        for (int i = 0; i < ntok; ++i) {
+          float d = 0.f;
+#pragma unroll
+          for (int u = 0; u < 4; ++u) d += qv[u] * ldf<T>(K, base + (int64_t)i * p.st + lane * 4 + u);
+          lse_push(m, s, warp_sum(d) * p.sm_scale);
+        }
+        v = m + logf(s);
       }
-      const float v = m + logf(s);
       if (lane == 0) {
         p.shat[((int64_t)b * p.Hq + h * p.G + g) * p.Pmax + page] = v;
         if (page >= 1 && page <= P - 2) lse_push(pm, ps, v);
@@ -313,7 +330,8 @@ __global__ void __launch_bounds__(128) quality_kernel(QualityParams p) {
 
 }  // namespace
 
-int locks_launch_exact_scan(locks_ctx *c, const void *q, const locks_kv *kv, int batch, float *shat, cudaStream_t st) {
+int locks_launch_exact_scan(locks_ctx *c, const void *q, const locks_kv *kv, int batch, float *shat, int envelope,
+                            cudaStream_t st) {
   ExactParams p;
   p.q = q; p.k = kv->k; p.sb = kv->stride_block; p.sh = kv->stride_head; p.st = kv->stride_token;
   p.block_table = kv->block_table; p.seq_lens = kv->seq_lens; p.shat = shat; p.part = c->part; p.status = c->status;
@@ -324,7 +342,10 @@ int locks_launch_exact_scan(locks_ctx *c, const void *q, const locks_kv *kv, int
   c->part_balanced = 0;
   c->last_partition = 0;
   dim3 grid(chunks, p.Hkv, batch);
-  if (c->cfg.kv_dtype == LOCKS_BF16) {
+  if (envelope) {
+    if (c->cfg.kv_dtype == LOCKS_BF16) locks_launch_pdl(exact_generic_kernel<__nv_bfloat16, true>, grid, dim3(kExWarps * 32), 0, st, p);
+    else locks_launch_pdl(exact_generic_kernel<float, true>, grid, dim3(kExWarps * 32), 0, st, p);
+  } else if (c->cfg.kv_dtype == LOCKS_BF16) {
     if (locks_attrs_needed(LOCKS_ATTR_EXACT)) {
       cudaFuncSetAttribute(exact_bf16_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kExSmem);
       cudaFuncSetAttribute(exact_bf16_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kExSmem);
@@ -332,7 +353,7 @@ int locks_launch_exact_scan(locks_ctx *c, const void *q, const locks_kv *kv, int
     if (c->G <= 8) locks_launch_pdl(exact_bf16_kernel<1>, grid, dim3(kExWarps * 32), kExSmem, st, p);
     else locks_launch_pdl(exact_bf16_kernel<2>, grid, dim3(kExWarps * 32), kExSmem, st, p);
   } else {
-    locks_launch_pdl(exact_generic_kernel<float>, grid, dim3(kExWarps * 32), 0, st, p);
+    locks_launch_pdl(exact_generic_kernel<float, false>, grid, dim3(kExWarps * 32), 0, st, p);
   }
   return locks_check_launch(c);
 }

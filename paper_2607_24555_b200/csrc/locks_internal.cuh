@@ -60,6 +60,7 @@ struct locks_ctx {
   int part_balanced;       // the last scan launch wrote per-problem partial counts to part_cnt instead
   int scan_partition;      // LOCKS_PARTITION_*: how the tensor scan deals pages to its warps
   int last_partition;      // partition the last tensor-scan launch used (0: no such launch yet)
+  int scorer;              // LOCKS_SCORER_*: what the next scan launch computes per page (diagnostics switch it)
   int32_t *hint_host;      // pinned, device-mapped word: partition the device suggests for the current lengths
   int32_t *hint_dev;       //   (0 none yet, LOCKS_PARTITION_STRIDED, LOCKS_PARTITION_BALANCED)
   int sel_ept;             // pages per thread of a selector CTA (chunk = sel_ept * 512 pages)
@@ -149,7 +150,9 @@ int locks_launch_build(locks_ctx *c, const locks_kv *kv, int batch, const int32_
                        int just_filled, void *summaries, const void *k_new, const int32_t *append_pos,
                        cudaStream_t st);
 
-int locks_launch_exact_scan(locks_ctx *c, const void *q, const locks_kv *kv, int batch, float *shat, cudaStream_t st);
+// envelope = 0: exact page log-mass; 1: the min/max envelope bound of the page's largest logit
+int locks_launch_exact_scan(locks_ctx *c, const void *q, const locks_kv *kv, int batch, float *shat, int envelope,
+                            cudaStream_t st);
 int locks_launch_quality(locks_ctx *c, const float *mass, const locks_kv *kv, int batch, const int32_t *ids_a,
                          const int32_t *cnt_a, const int32_t *ids_r, const int32_t *cnt_r, const int32_t *marked,
                          int n_marked, float *out, cudaStream_t st);

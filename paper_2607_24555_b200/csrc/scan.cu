@@ -41,6 +41,7 @@ struct ScanParams {
   int wpp, nslots;    // strided partition: warps per problem, problems in flight
   int use_gather;     // stage four summaries per tensor-map gather instead of one bulk copy each
   int seq_inc;
+  int scorer;         // generic kernel only: LOCKS_SCORER_* (the summary's own score, or a rival functional of it)
   int32_t *seq_eff;   // [2][max_batch]: effective length, append position (-1: none) -- or nullptr
 };
 
@@ -149,9 +150,17 @@ __global__ void __launch_bounds__(128) scan_generic_kernel(ScanParams p) {
         }
         logit = p.sm_scale * (a + s);
       }
-      const float mx = warp_max(logit);
-      const float z = warp_sum(lane < LOCKS_B ? expf(logit - mx) : 0.f);
-      const float sh = mx + logf(z);
+      float sh;
+      if (p.scorer == LOCKS_SCORER_CENTROID) {          // the centroid term alone: q.mu / sqrt(d) + log B
+        sh = p.sm_scale * a + logf((float)LOCKS_B);
+      } else if (p.scorer == LOCKS_SCORER_MOMENT) {     // second-cumulant truncation of the mass (moment core)
+        const float zi = lane < LOCKS_B ? logit - p.sm_scale * a : 0.f;
+        sh = p.sm_scale * a + logf((float)LOCKS_B) + warp_sum(zi * zi) * (0.5f / LOCKS_B);
+      } else {
+        const float mx = warp_max(logit);
+        const float z = warp_sum(lane < LOCKS_B ? expf(logit - mx) : 0.f);
+        sh = mx + logf(z);
+      }
       if (lane == 0) {
         p.shat[((int64_t)b * p.Hq + hq) * p.Pmax + page] = sh;
         if (page >= 1) {  // candidates only
@@ -947,7 +956,9 @@ int locks_launch_scan(locks_ctx *c, const void *q, const void *summaries, const 
   p.batch = batch; p.Hq = c->cfg.num_q_heads; p.Hkv = c->cfg.num_kv_heads; p.G = c->G;
   p.Pmax = c->Pmax; p.max_groups = c->max_groups; p.num_blocks = kv->num_blocks; p.k = c->k;
   p.S = c->S; p.r = c->cfg.rank; p.sm_scale = c->cfg.sm_scale;
-  const bool tensor = c->cfg.summary_fmt == LOCKS_FMT_I4 && c->cfg.q_dtype == LOCKS_BF16;   // ranks 2, 4, 8
+  p.scorer = c->scorer;
+  const bool tensor = c->cfg.summary_fmt == LOCKS_FMT_I4 && c->cfg.q_dtype == LOCKS_BF16 &&
+                      c->scorer == LOCKS_SCORER_SUMMARY;   // ranks 2, 4, 8
   c->part_slots = c->max_groups;   // generic kernel: one partial per 8-page group
   c->part_balanced = 0;
   c->last_partition = 0;

@@ -123,3 +123,34 @@ def test_combine_rule_switch_matches_oracle(rule, lens, Hq, Hkv):
             okey[b, h, :P] = kk[:P]
             assert np.abs(key[b, h, 1:P - 1].cpu().numpy() - kk[1:P - 1]).max() <= 1e-3
     check_page_sets(ids.cpu().numpy(), cnt.cpu().numpy(), oids, ocnt, okey, gc.cache.seq_lens, w.B, gc.k)
+
+
+@pytest.mark.parametrize("scorer", [1, 2, 3])
+@pytest.mark.parametrize("fmt,dtype,Hq,Hkv", [("i4", "bf16", 8, 2), ("f32", "f32", 4, 1), ("i4", "bf16", 32, 2)])
+def test_rival_scorers_match_oracle(scorer, fmt, dtype, Hq, Hkv):
+    """Centroid-only, moment-core and envelope scores, and the selections they lead to, against the oracle."""
+    import paper_2607_24555_b200 as locks
+    w = locks_synth.Workload("rival", [16 * 300 + 5, 16 * 70], Hq=Hq, Hkv=Hkv, budget=256, fmt=fmt, dtype=dtype,
+                             carriers=4, q_scale=0.5, seed=scorer + Hq)
+    gc = _gc(w)
+    summ_np = gc.oracle_summaries()
+    summ = torch.from_numpy(summ_np).cuda()
+    ids = torch.full((w.n, w.Hkv, gc.k), -7, dtype=torch.int32, device="cuda:0")
+    cnt = torch.full((w.n, w.Hkv), -7, dtype=torch.int32, device="cuda:0")
+    score = torch.full((w.n, w.Hq, gc.max_pages), float("nan"), dtype=torch.float32, device="cuda:0")
+    key = torch.full((w.n, w.Hkv, gc.max_pages), float("nan"), dtype=torch.float32, device="cuda:0")
+    gc.ctx.locks_select_rival(scorer, gc.case.q, summ, gc.kv, w.n, ids, cnt, score, key)
+    torch.cuda.synchronize()
+    assert gc.status() == 0
+    oscore = oracle.rival_logmass(gc.cache, t2np(gc.case.q), w.rank, gc.fmt, summ_np, gc.sm, scorer)
+    oids, ocnt, okey = oracle.select(gc.cache, oscore, gc.k)
+    tol = 1e-3 if dtype == "bf16" else 2e-4
+    for b, T in enumerate(w.seq_lens):
+        P = -(-T // w.B)
+        assert np.abs(score[b, :, :P - 1].cpu().numpy() - oscore[b, :, :P - 1]).max() <= tol
+        assert np.abs(key[b, :, 1:P - 1].cpu().numpy() - okey[b, :, 1:P - 1]).max() <= tol
+    check_page_sets(ids.cpu().numpy(), cnt.cpu().numpy(), oids, ocnt, okey, gc.cache.seq_lens, w.B, gc.k)
+    # the context still runs the summary's own scorer afterwards
+    ids2, cnt2, lm, _ = gc.gpu_select(summ)
+    shat = oracle.page_logmass(gc.cache, t2np(gc.case.q), w.rank, gc.fmt, summ_np, gc.sm)
+    assert np.nanmax(np.abs(lm[0, :, :10] - shat[0, :, :10])) <= 1e-3

@@ -649,3 +649,41 @@ def test_combine_rules_differ_where_they_should():
     want = sorted([0, 39] + (np.argsort(-s1[0, 1:39])[:6] + 1).tolist())
     for rule in (0, 1, 2):
         assert oracle.select_one_rule(s1, 40, 8, rule)[0].tolist() == want
+
+
+# ------------------------------------------------------------------ rival scorers (App. A / B)
+
+def test_rival_scorers_against_the_paper_s_statements():
+    """Moment core: s - log B = s^q + R_cum + R_rank with |R_cum| <= L^3 / 3 and 0 <= R_rank <= sigma_{r+1}^2 |q|^2 /
+    (2 B d) (Prop. 4), on random pages and queries, unquantised summaries.  Centroid: the score of a summary
+    whose coefficients vanish.  Envelope: an upper bound of every logit of the page, tight for a page of one
+    repeated key (Lemma 2)."""
+    rng = np.random.default_rng(11)
+    B, d = 16, 128
+    for trial in range(30):
+        r = int(rng.integers(1, 15))
+        keys = low_rank_page(int(rng.integers(2, 9)), noise=0.3, seed=100 + trial) * float(rng.choice([0.2, 1.0]))
+        q = rng.standard_normal(d) * float(rng.choice([0.3, 1.0]))
+        mu, V, Cc, lam, r_eff = oracle.build_page(keys, r)
+        s_exact = oracle.exact_lse(keys, q, SM)
+        s_mom = oracle.rival_score(oracle.SCORER_MOMENT, mu, V, Cc, q, SM)
+        s_cen = oracle.rival_score(oracle.SCORER_CENTROID, mu, V, Cc, q, SM)
+        z = (keys - keys.mean(0)) @ q * SM                         # centred per-key logits
+        kappa2 = float((z ** 2).mean())
+        a = float(keys.mean(0) @ q) * SM
+        assert abs(s_cen - (a + math.log(B))) < 1e-12
+        assert abs(s_cen - oracle.score(mu, V, np.zeros_like(Cc), q, SM)) < 1e-12
+        r_rank = 0.5 * kappa2 - (s_mom - s_cen)                    # what the rank truncation leaves out
+        assert -1e-12 <= r_rank <= lam[r] * (q @ q) / (2 * B * d) + 1e-12 if r < B else abs(r_rank) < 1e-12
+        r_cum = s_exact - math.log(B) - a - 0.5 * kappa2
+        assert abs(r_cum) <= np.abs(z).max() ** 3 / 3 + 1e-12
+        env = oracle.envelope_score(keys, q, SM)
+        assert env >= (keys @ q * SM).max() - 1e-12
+    one = np.tile(rng.standard_normal(d), (B, 1))
+    q = rng.standard_normal(d)
+    assert abs(oracle.envelope_score(one, q, SM) - float(one[0] @ q) * SM) < 1e-12
+    # full rank: the moment core is a + log B + kappa_2 / 2 exactly
+    keys = rng.standard_normal((B, d))
+    mu, V, Cc, lam, _ = oracle.build_page(keys, 15)
+    z = (keys - keys.mean(0)) @ q * SM
+    assert abs(oracle.rival_score(oracle.SCORER_MOMENT, mu, V, Cc, q, SM) - (float(keys.mean(0) @ q) * SM + math.log(B) + 0.5 * float((z ** 2).mean()))) < 1e-10
