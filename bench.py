@@ -458,6 +458,62 @@ def run_ours(args):
     print(json.dumps(line))
 
 
+def run_diagnostics(args):
+    """Selection fidelity on the synthetic workloads (the paper's App. B metrics): for the summary's own score, the
+    exact-LSE arm and the rival scorers, all under the same share-average selection, measured against exact page
+    masses by the library's own kernels.  Prints one JSON line."""
+    import torch
+    import locks_synth
+    import paper_2607_24555_b200 as locks
+    from paper_2607_24555_b200.binding import KVView, make_config
+    dev = "cuda:0"
+    rows = []
+    cells = [("cfg0_tiny", locks_synth.config0()), ("cfg1_llama_8x32k", locks_synth.config1().with_(carriers=16)),
+             ("cfg2_qwen_32x16k_r8_b1024", locks_synth.config2(rank=8, budget=1024)),
+             ("cfg2_qwen_32x16k_r2_b256", locks_synth.config2(rank=2, budget=256)),
+             ("cfg1_soft_queries", locks_synth.config1().with_(q_scale=0.25, carriers=0))]
+    for name, w in cells:
+        case = locks_synth.make_case(w, device=dev)
+        max_pages = case.block_table.shape[1]
+        ctx = locks.Context(make_config(w.Hq, w.Hkv, w.rank, w.fmt, w.dtype, w.n, max_pages, w.budget), device=dev)
+        kv = KVView(case.k, case.v, case.strides, case.num_blocks, case.block_table, case.seq_lens)
+        summ = ctx.new_summaries(case.num_blocks)
+        ctx.locks_build_summaries(kv, w.n, summ)
+        mk = lambda: (torch.zeros(w.n, w.Hkv, w.k, dtype=torch.int32, device=dev), torch.zeros(w.n, w.Hkv, dtype=torch.int32, device=dev))
+        ids_e, cnt_e = mk()
+        mass = torch.zeros(w.n, w.Hq, max_pages, dtype=torch.float32, device=dev)
+        ctx.locks_select_exact(case.q, kv, w.n, ids_e, cnt_e, mass)
+        ncar = max((len(c) for c in case.carrier_pages), default=0)
+        marked = None
+        if ncar:
+            marked = torch.full((w.n, ncar), -1, dtype=torch.int32, device=dev)
+            for b, cps in enumerate(case.carrier_pages):
+                marked[b, :len(cps)] = torch.tensor(cps, dtype=torch.int32, device=dev)
+        row = {"workload": name, "budget_tokens": w.budget, "rank": w.rank, "carriers_per_request": ncar, "scorers": {}}
+        arms = [("exact_lse", None), ("locks_summary", 0), ("moment_core", locks.SCORER_MOMENT),
+                ("centroid_only", locks.SCORER_CENTROID), ("envelope_quest", locks.SCORER_ENVELOPE)]
+        for label, sc in arms:
+            ids, cnt = mk()
+            if sc is None:
+                ids, cnt = ids_e, cnt_e
+            elif sc == 0:
+                ctx.locks_select(case.q, summ, kv, w.n, ids, cnt)
+            else:
+                ctx.locks_select_rival(sc, case.q, summ, kv, w.n, ids, cnt)
+            qual = torch.zeros(w.n, w.Hkv, 4, dtype=torch.float32, device=dev)
+            ctx.locks_selection_quality(mass, kv, w.n, ids, cnt, ids_e, cnt_e, qual, marked_pages=marked)
+            torch.cuda.synchronize()
+            m = qual.mean(dim=(0, 1)).tolist()
+            row["scorers"][label] = {"gamma": round(m[0], 4), "gamma_c": round(m[1], 4), "recall": round(m[2], 4),
+                                     "needle": round(m[3], 4) if ncar else None}
+        rows.append(row)
+        ctx.close()
+        del case, summ, mass
+        torch.cuda.empty_cache()
+    print(json.dumps({"diagnostics": "selection fidelity against exact page masses (App. B metrics), synthetic keys",
+                      "rows": rows}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -474,7 +530,12 @@ def main():
                     help="how the scan deals pages to its warps (auto: the library follows the lengths)")
     ap.add_argument("--identity-blocks", action="store_true",
                     help="logical page i of a request sits in consecutive physical blocks (default: seeded permutation)")
+    ap.add_argument("--diagnostics", action="store_true",
+                    help="print the selection-fidelity table (gamma, gamma_c, recall, needle per scorer) instead of timing")
     args = ap.parse_args()
+    if args.diagnostics:
+        run_diagnostics(args)
+        return
     if args.impl == "reference":
         run_reference(args)
     else:
