@@ -117,6 +117,18 @@ int locks_destroy(locks_ctx *ctx);
 int locks_build_summaries(locks_ctx *ctx, const locks_kv *kv, int batch, const int32_t *page_begin,
                           const int32_t *page_end, void *summaries, locks_stream stream);
 
+/* KV-cache quantisation stacked on the selector (Sec. 5 "KV-cache quantization under extreme sparsity"; App. C,
+ * KIVI x LOCKS grid): fake-quantise (quantise, then dequantise in the cache's own element type, in place) every
+ * COMPLETE page p with page_begin[b] <= p < page_end[b] (NULL, NULL: all complete pages) of every request and KV
+ * head.  KIVI's grouping, page-aligned as in the paper's protocol: keys per channel over the 16 tokens of the page,
+ * values per token over groups of 32 consecutive dimensions; asymmetric uniform grid of 2^bits levels between a
+ * group's minimum and maximum (bits 1..8; the paper measures 4 and 2).  The partial last page is left untouched
+ * (the paper keeps it unquantised inside the always-attended window).  The two arms of the paper's grid are call
+ * orders: "post" = locks_build_summaries, then this; "pre" = this, then locks_build_summaries.  Attention and
+ * scoring then run unchanged on the quantised values. */
+int locks_fake_quantize_pages(locks_ctx *ctx, const locks_kv *kv, int batch, const int32_t *page_begin,
+                              const int32_t *page_end, int bits, locks_stream stream);
+
 /* Stage A, "score-then-select" (Sec. 4 "Score (every step)", Eq. 1; share-average combine;
  * App. E): for every request and query head, s^_j(q_g) for all pages j <= P-2 from the resident
  * summaries; shares normalised over the candidates 1..P-2; m_bar_j = mean over the group; per KV

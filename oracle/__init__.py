@@ -245,6 +245,13 @@ def build_summaries(cache: Cache, r: int, fmt: int, summaries=None, page_begin=N
     return summaries
 
 
+def fake_quantize_pages(cache: Cache, bits: int, page_begin=None, page_end=None):
+    """KIVI-style fake quantisation of the complete pages of `cache`, IN PLACE (cache.k / cache.v are overwritten)."""
+    pb = np.ascontiguousarray(page_begin, dtype=np.int32) if page_begin is not None else None
+    pe = np.ascontiguousarray(page_end, dtype=np.int32) if page_end is not None else None
+    lib().ora_fake_quantize_pages(cache.ref(), C.c_int(cache.batch), _p(pb), _p(pe), C.c_int(int(bits)))
+
+
 def _q_arg(q):
     q = np.ascontiguousarray(q)
     return q, _dtype_code(q)

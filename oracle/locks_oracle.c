@@ -539,6 +539,62 @@ void ora_page_logmass(const ora_kv *kv, int batch, const void *q, int q_dtype, i
     }
 }
 
+/* KIVI-style fake quantisation of complete pages, in place (Sec. 5; App. C protocol): keys per channel over the
+ * page's B tokens, values per token over groups of 32 dims; asymmetric uniform grid of 2^bits levels between the
+ * group's minimum and maximum, x^ = min + s rint((x - min)/s), s = (max - min)/(2^bits - 1); a constant group is
+ * kept.  The result is stored back in the cache's element type (round to nearest even for bf16).  k, v must be
+ * writable.  Only fp32 and bf16 caches. */
+static void store_elem(void *base, int dtype, int64_t idx, double x) {
+  if (dtype == ORA_F32) { ((float *)base)[idx] = (float)x; return; }
+  float f = (float)x;
+  uint32_t u; memcpy(&u, &f, 4);
+  uint32_t r = u + 0x7FFFu + ((u >> 16) & 1u);   /* round to nearest even on the dropped 16 bits */
+  ((uint16_t *)base)[idx] = (uint16_t)(r >> 16);
+}
+static double requant(double x, double lo, double hi, int levels) {
+  double s = (hi - lo) / levels;
+  if (!(s > 0)) return x;
+  return lo + s * rint((x - lo) / s);
+}
+void ora_fake_quantize_pages(const ora_kv *kv, int batch, const int32_t *page_begin, const int32_t *page_end, int bits) {
+  int B = kv->B, d = kv->d, levels = (1 << bits) - 1;
+  for (int b = 0; b < batch; ++b)
+    for (int h = 0; h < kv->Hkv; ++h) {
+      int complete = kv->seq_lens[b] / B;
+      int p0 = page_begin ? page_begin[b] : 0, p1 = page_end ? page_end[b] : complete;
+      if (p1 > complete) p1 = complete;
+      for (int p = p0; p < p1; ++p) {
+        int block = kv->block_table[(int64_t)b * kv->max_pages + p];
+        int64_t base = (int64_t)block * kv->stride_block + (int64_t)h * kv->stride_head;
+        for (int c = 0; c < d; ++c) { /* keys: one group per channel */
+          double lo = INFINITY, hi = -INFINITY;
+          for (int i = 0; i < B; ++i) {
+            double x = load_elem(kv->k, kv->dtype, base + (int64_t)i * kv->stride_token + c);
+            if (x < lo) lo = x;
+            if (x > hi) hi = x;
+          }
+          for (int i = 0; i < B; ++i) {
+            int64_t at = base + (int64_t)i * kv->stride_token + c;
+            store_elem((void *)kv->k, kv->dtype, at, requant(load_elem(kv->k, kv->dtype, at), lo, hi, levels));
+          }
+        }
+        for (int i = 0; i < B; ++i) /* values: groups of 32 dims of one token */
+          for (int g0 = 0; g0 < d; g0 += 32) {
+            double lo = INFINITY, hi = -INFINITY;
+            for (int c = g0; c < g0 + 32 && c < d; ++c) {
+              double x = load_elem(kv->v, kv->dtype, base + (int64_t)i * kv->stride_token + c);
+              if (x < lo) lo = x;
+              if (x > hi) hi = x;
+            }
+            for (int c = g0; c < g0 + 32 && c < d; ++c) {
+              int64_t at = base + (int64_t)i * kv->stride_token + c;
+              store_elem((void *)kv->v, kv->dtype, at, requant(load_elem(kv->v, kv->dtype, at), lo, hi, levels));
+            }
+          }
+      }
+    }
+}
+
 /* Rival scores of every page (scorer 1, 2: pages 0..P-2 from the summaries; scorer 3, envelope: pages 0..P-1 from
  * the keys): out[(b*Hq + g)*max_pages + p]. */
 void ora_rival_logmass(const ora_kv *kv, int batch, const void *q, int q_dtype, int r, int fmt,

@@ -19,7 +19,7 @@ SYMBOLS = ["locks_summary_bytes", "locks_workspace_bytes", "locks_create", "lock
            "locks_profile_begin", "locks_profile_end", "locks_profile_read", "locks_sparse_attend_noalloc",
            "locks_set_scan_partition", "locks_selftest_wait_timeout", "locks_last_scan_partition",
            "locks_host_cache_clear", "locks_select_exact", "locks_selection_quality",
-           "locks_select_rival"]
+           "locks_select_rival", "locks_fake_quantize_pages"]
 
 
 PARTITION_AUTO, PARTITION_STRIDED, PARTITION_BALANCED = 0, 1, 2   # LOCKS_PARTITION_* of include/locks.h
@@ -91,6 +91,8 @@ def lib():
         L.locks_host_cache_clear.restype = C.c_int
         L.locks_select_rival.argtypes = [vp, C.c_int, vp, vp, C.POINTER(KV), C.c_int, i32p, i32p, vp, vp, vp]
         L.locks_select_rival.restype = C.c_int
+        L.locks_fake_quantize_pages.argtypes = [vp, C.POINTER(KV), C.c_int, i32p, i32p, C.c_int, vp]
+        L.locks_fake_quantize_pages.restype = C.c_int
         L.locks_select_exact.argtypes = [vp, vp, C.POINTER(KV), C.c_int, i32p, i32p, vp, vp, vp]
         L.locks_select_exact.restype = C.c_int
         L.locks_selection_quality.argtypes = [vp, vp, C.POINTER(KV), C.c_int, i32p, i32p, i32p, i32p, i32p, C.c_int, vp, vp]
@@ -202,6 +204,11 @@ class Context:
         s = kv.struct()
         _check(lib().locks_build_summaries(self.handle, C.byref(s), batch, _ptr(page_begin), _ptr(page_end),
                                            _ptr(summaries), _stream(stream)), "locks_build_summaries")
+
+    def locks_fake_quantize_pages(self, kv: KVView, batch, bits, page_begin=None, page_end=None, stream=None):
+        s = kv.struct()
+        _check(lib().locks_fake_quantize_pages(self.handle, C.byref(s), batch, _ptr(page_begin), _ptr(page_end), int(bits),
+                                               _stream(stream)), "locks_fake_quantize_pages")
 
     def locks_select(self, q, summaries, kv: KVView, batch, page_ids, page_count, page_logmass=None,
                      page_logshare=None, stream=None):

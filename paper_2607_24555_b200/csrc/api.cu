@@ -277,6 +277,15 @@ int locks_build_summaries(locks_ctx *ctx, const locks_kv *kv, int batch, const i
   return locks_launch_build(ctx, kv, batch, page_begin, page_end, 0, summaries, nullptr, nullptr, (cudaStream_t)stream);
 }
 
+int locks_fake_quantize_pages(locks_ctx *ctx, const locks_kv *kv, int batch, const int32_t *page_begin,
+                              const int32_t *page_end, int bits, locks_stream stream) {
+  int rc = check_common(ctx, kv, batch);
+  if (rc != LOCKS_OK) return rc;
+  if (bits < 1 || bits > 8 || ((page_begin == nullptr) != (page_end == nullptr))) return LOCKS_ERR_INVALID_ARG;
+  ctx->last_launches = 0;
+  return locks_launch_fake_quant(ctx, kv, batch, page_begin, page_end, bits, (cudaStream_t)stream);
+}
+
 int locks_select(locks_ctx *ctx, const void *q, const void *summaries, const locks_kv *kv, int batch,
                  int32_t *page_ids, int32_t *page_count, float *page_logmass, float *page_logshare,
                  locks_stream stream) {

@@ -157,6 +157,9 @@ int locks_launch_quality(locks_ctx *c, const float *mass, const locks_kv *kv, in
                          const int32_t *cnt_a, const int32_t *ids_r, const int32_t *cnt_r, const int32_t *marked,
                          int n_marked, float *out, cudaStream_t st);
 
+int locks_launch_fake_quant(locks_ctx *c, const locks_kv *kv, int batch, const int32_t *pb, const int32_t *pe, int bits,
+                            cudaStream_t st);
+
 // Launch with programmatic dependent launch allowed: the kernel may be scheduled while its stream
 // predecessor is still draining; it must execute pdl_wait() before touching anything the predecessor
 // writes (the wait returns once the predecessor grid has completed and its writes are visible).

@@ -154,3 +154,35 @@ def test_rival_scorers_match_oracle(scorer, fmt, dtype, Hq, Hkv):
     ids2, cnt2, lm, _ = gc.gpu_select(summ)
     shat = oracle.page_logmass(gc.cache, t2np(gc.case.q), w.rank, gc.fmt, summ_np, gc.sm)
     assert np.nanmax(np.abs(lm[0, :, :10] - shat[0, :, :10])) <= 1e-3
+
+
+@pytest.mark.parametrize("bits,dtype,arm", [(4, "bf16", "post"), (2, "bf16", "pre"), (4, "f32", "pre")])
+def test_fake_quantised_cache_composition(bits, dtype, arm):
+    """KIVI-style fake quantisation of the complete pages on the GPU against the oracle's, then the paper's two
+    compositions: "post" (summaries from the original keys, attention on quantised KV) and "pre" (summaries from
+    the quantised keys): page masses, sets and outputs against the oracle on the quantised cache."""
+    from common import oracle_cache
+    from gpu_util import check_select_and_attend, upload
+    fmt = "i4" if dtype == "bf16" else "f32"
+    w = locks_synth.Workload("kivi", [16 * 200 + 7, 16 * 90], Hq=8, Hkv=2, budget=256, dtype=dtype, fmt=fmt, q_scale=0.5,
+                             layout="NHD" if bits == 2 else "HND", seed=bits)
+    gc = _gc(w)
+    ref = oracle_cache(gc.case)                                       # CPU copy of the original values
+    summ_before = gc.gpu_build() if arm == "post" else None
+    gc.ctx.locks_fake_quantize_pages(gc.kv, w.n, bits)
+    torch.cuda.synchronize()
+    assert gc.status() == 0
+    oracle.fake_quantize_pages(ref, bits)
+    got = oracle_cache(gc.case)
+
+    def vals(a):
+        return ((a.astype(np.uint32) << 16).view(np.float32) if a.dtype == np.uint16 else a).astype(np.float64)
+
+    for a, b_ in ((got.k, ref.k), (got.v, ref.v)):
+        d = np.abs(vals(a) - vals(b_))
+        # fp32 against fp64 arithmetic: an entry within rounding of a grid midpoint may land on the neighbouring level
+        assert (d > 1e-6 * np.abs(vals(b_)).max() + 2.0 ** -8 * np.abs(vals(b_)) * (a.dtype == np.uint16)).mean() <= 2e-3
+        assert d.max() <= (vals(b_).max() - vals(b_).min()) / (2 ** bits - 1)
+    gc.cache = got                                                    # from here on: the GPU's quantised cache
+    summ = summ_before if arm == "post" else gc.gpu_build()
+    check_select_and_attend(gc, summ.cpu().numpy(), out_tol=2e-2 if dtype == "bf16" else 1e-4)

@@ -687,3 +687,54 @@ def test_rival_scorers_against_the_paper_s_statements():
     mu, V, Cc, lam, _ = oracle.build_page(keys, 15)
     z = (keys - keys.mean(0)) @ q * SM
     assert abs(oracle.rival_score(oracle.SCORER_MOMENT, mu, V, Cc, q, SM) - (float(keys.mean(0) @ q) * SM + math.log(B) + 0.5 * float((z ** 2).mean()))) < 1e-10
+
+
+# ------------------------------------------------------------------ KV-cache fake quantisation (Sec. 5, KIVI grid)
+
+@pytest.mark.parametrize("bits,bf16", [(4, True), (2, True), (4, False), (8, False)])
+def test_fake_quantisation_groups_levels_and_bounds(bits, bf16):
+    """Keys: per channel over the page's 16 tokens; values: per token over groups of 32 dims.  Every group keeps its
+    minimum and maximum, takes at most 2^bits distinct values, moves no entry by more than half a step (plus the
+    storage rounding), and nothing outside the complete pages changes."""
+    cache, _, _, page, lens, pages = ragged_batch_cache("HND", bf16, seed=9)
+    k0, v0 = cache.k.copy(), cache.v.copy()
+
+    def vals(a):
+        return ((a.astype(np.uint32) << 16).view(np.float32) if bf16 else a).astype(np.float64)
+
+    oracle.fake_quantize_pages(cache, bits)
+    ulp = 2.0 ** -8 if bf16 else 2.0 ** -23
+    touched = set()
+    for b in range(3):
+        for p in range(lens[b] // 16):
+            blk = int(cache.block_table[b, p])
+            touched.add(blk)
+            for h in range(2):
+                K0, K1 = vals(k0[blk, h]), vals(cache.k[blk, h])          # [16, 128]
+                lo, hi = K0.min(0), K0.max(0)
+                step = (hi - lo) / (2 ** bits - 1)
+                assert np.array_equal(K1.min(0), lo) and np.allclose(K1.max(0), hi, rtol=ulp, atol=0)
+                assert np.all(np.abs(K1 - K0) <= step / 2 + np.maximum(np.abs(K0), np.abs(K1)) * ulp + 1e-12)
+                assert max(len(np.unique(K1[:, c])) for c in range(128)) <= 2 ** bits
+                V0, V1 = vals(v0[blk, h]).reshape(16, 4, 32), vals(cache.v[blk, h]).reshape(16, 4, 32)
+                lo, hi = V0.min(-1, keepdims=True), V0.max(-1, keepdims=True)
+                step = (hi - lo) / (2 ** bits - 1)
+                assert np.array_equal(V1.min(-1, keepdims=True), lo)
+                assert np.all(np.abs(V1 - V0) <= step / 2 + np.maximum(np.abs(V0), np.abs(V1)) * ulp + 1e-12)
+                assert max(len(np.unique(V1[i, g])) for i in range(16) for g in range(4)) <= 2 ** bits
+    for blk in range(cache.num_blocks):
+        if blk not in touched:
+            assert np.array_equal(cache.k[blk], k0[blk]) and np.array_equal(cache.v[blk], v0[blk])
+    # a constant group is kept as it is; a two-valued group is a fixed point at any width
+    c2, _ = tiny_cache(T=32)
+    c2.k[:] = 1.25
+    c2.v[:] = np.where(np.arange(128) % 2 == 0, -3.0, 5.0).astype(np.float32)
+    kk, vv = c2.k.copy(), c2.v.copy()
+    oracle.fake_quantize_pages(c2, 2)
+    assert np.array_equal(c2.k, kk) and np.array_equal(c2.v, vv)
+    # page ranges are per request
+    c3, _, _, _, _, _ = ragged_batch_cache("HND", False, seed=9)
+    before = c3.k.copy()
+    oracle.fake_quantize_pages(c3, 4, page_begin=[1, 0, 0], page_end=[2, 0, 0])
+    changed = {blk for blk in range(c3.num_blocks) if not np.array_equal(c3.k[blk], before[blk])}
+    assert changed == {int(c3.block_table[0, 1])}
