@@ -117,6 +117,38 @@ int locks_destroy(locks_ctx *ctx);
 int locks_build_summaries(locks_ctx *ctx, const locks_kv *kv, int batch, const int32_t *page_begin,
                           const int32_t *page_end, void *summaries, locks_stream stream);
 
+/* ---- Page-sharded decode -------------------------------------------------------------------------------------
+ * One long request (the GLM-shaped 128K..1M case) whose pages are dealt to several GPUs in page order.  The path
+ * itself has no exchange step (every (request, KV head) owns its pages); sharding ONE sequence adds three small
+ * ones, which the caller runs with its own collective (torch.distributed / NCCL all-gather of a few KB):
+ *   (1) the per-head partition functions log Z_g of the shards, (2) each shard's top-(k-2) candidates (key, page),
+ *   (3) each shard's attention partial (out, lse).
+ * A shard is presented to the library as an ordinary sequence: [sink or a dummy page] + its candidate pages + [the
+ * request's last page or a dummy page], so that "pages 1 .. P-2 are the candidates" holds shard by shard.
+ *
+ * locks_scan: Eq. 1 over the shard's pages (as locks_select does), plus head_logz [batch][Hq] = log sum over the
+ * shard's candidate pages of exp s^_j(q_g) (-inf if it has none).  page_logmass optional (else kept in the
+ * workspace for locks_select_scored). */
+int locks_scan(locks_ctx *ctx, const void *q, const void *summaries, const locks_kv *kv, int batch, float *page_logmass,
+               float *head_logz, locks_stream stream);
+/* The selection of locks_select on scores that are already there, with the partition functions given from
+ * outside: head_logz_parts [nparts][batch][Hq] (every shard's locks_scan output, gathered); log Z_g = log sum of
+ * their exponentials.  page_logmass NULL: the scores the last locks_scan of this context left in the workspace.
+ * Outputs as locks_select (the shard's own table and keys); needs more than k pages in the shard. */
+int locks_select_scored(locks_ctx *ctx, const float *page_logmass, const float *head_logz_parts, int nparts,
+                        const locks_kv *kv, int batch, int32_t *page_ids, int32_t *page_count, float *page_logshare,
+                        locks_stream stream);
+/* Global top-(k-2) of the shards' candidate lists: cand_key / cand_page [nparts][batch][Hkv][k-2] (ranking key and
+ * GLOBAL logical page of each shard's winners, in page order, shards in page order; page -1 = empty slot) ->
+ * page_ids [batch][Hkv][k-2] global pages ascending, -1 padded; page_count [batch][Hkv].  Ties to the lower page. */
+int locks_merge_selection(locks_ctx *ctx, const float *cand_key, const int32_t *cand_page, int nparts, int batch,
+                          int32_t *page_ids, int32_t *page_count, locks_stream stream);
+/* Merge of the shards' attention partials (each locks_sparse_attend output normalised over the shard's own pages,
+ * with its lse): part_out [nparts][batch][Hq][d] (q dtype), part_lse [nparts][batch][Hq] (-inf: the shard attended
+ * nothing) -> out [batch][Hq][d], lse optional. */
+int locks_merge_attention(locks_ctx *ctx, const void *part_out, const float *part_lse, int nparts, int batch, void *out,
+                          float *lse, locks_stream stream);
+
 /* KV-cache quantisation stacked on the selector (Sec. 5 "KV-cache quantization under extreme sparsity"; App. C,
  * KIVI x LOCKS grid): fake-quantise (quantise, then dequantise in the cache's own element type, in place) every
  * COMPLETE page p with page_begin[b] <= p < page_end[b] (NULL, NULL: all complete pages) of every request and KV

@@ -19,7 +19,8 @@ SYMBOLS = ["locks_summary_bytes", "locks_workspace_bytes", "locks_create", "lock
            "locks_profile_begin", "locks_profile_end", "locks_profile_read", "locks_sparse_attend_noalloc",
            "locks_set_scan_partition", "locks_selftest_wait_timeout", "locks_last_scan_partition",
            "locks_host_cache_clear", "locks_select_exact", "locks_selection_quality",
-           "locks_select_rival", "locks_fake_quantize_pages"]
+           "locks_select_rival", "locks_fake_quantize_pages", "locks_scan",
+           "locks_select_scored", "locks_merge_selection", "locks_merge_attention"]
 
 
 PARTITION_AUTO, PARTITION_STRIDED, PARTITION_BALANCED = 0, 1, 2   # LOCKS_PARTITION_* of include/locks.h
@@ -93,6 +94,12 @@ def lib():
         L.locks_select_rival.restype = C.c_int
         L.locks_fake_quantize_pages.argtypes = [vp, C.POINTER(KV), C.c_int, i32p, i32p, C.c_int, vp]
         L.locks_fake_quantize_pages.restype = C.c_int
+        L.locks_scan.argtypes = [vp, vp, vp, C.POINTER(KV), C.c_int, vp, vp, vp]
+        L.locks_select_scored.argtypes = [vp, vp, vp, C.c_int, C.POINTER(KV), C.c_int, i32p, i32p, vp, vp]
+        L.locks_merge_selection.argtypes = [vp, vp, i32p, C.c_int, C.c_int, i32p, i32p, vp]
+        L.locks_merge_attention.argtypes = [vp, vp, vp, C.c_int, C.c_int, vp, vp, vp]
+        for fn in ("locks_scan", "locks_select_scored", "locks_merge_selection", "locks_merge_attention"):
+            getattr(L, fn).restype = C.c_int
         L.locks_select_exact.argtypes = [vp, vp, C.POINTER(KV), C.c_int, i32p, i32p, vp, vp, vp]
         L.locks_select_exact.restype = C.c_int
         L.locks_selection_quality.argtypes = [vp, vp, C.POINTER(KV), C.c_int, i32p, i32p, i32p, i32p, i32p, C.c_int, vp, vp]
@@ -209,6 +216,26 @@ class Context:
         s = kv.struct()
         _check(lib().locks_fake_quantize_pages(self.handle, C.byref(s), batch, _ptr(page_begin), _ptr(page_end), int(bits),
                                                _stream(stream)), "locks_fake_quantize_pages")
+
+    def locks_scan(self, q, summaries, kv: KVView, batch, head_logz, page_logmass=None, stream=None):
+        s = kv.struct()
+        _check(lib().locks_scan(self.handle, _ptr(q), _ptr(summaries), C.byref(s), batch, _ptr(page_logmass), _ptr(head_logz),
+                                _stream(stream)), "locks_scan")
+
+    def locks_select_scored(self, head_logz_parts, kv: KVView, batch, page_ids, page_count, page_logshare=None,
+                            page_logmass=None, stream=None):
+        s = kv.struct()
+        _check(lib().locks_select_scored(self.handle, _ptr(page_logmass), _ptr(head_logz_parts), int(head_logz_parts.shape[0]),
+                                         C.byref(s), batch, _ptr(page_ids), _ptr(page_count), _ptr(page_logshare),
+                                         _stream(stream)), "locks_select_scored")
+
+    def locks_merge_selection(self, cand_key, cand_page, batch, page_ids, page_count, stream=None):
+        _check(lib().locks_merge_selection(self.handle, _ptr(cand_key), _ptr(cand_page), int(cand_key.shape[0]), batch,
+                                           _ptr(page_ids), _ptr(page_count), _stream(stream)), "locks_merge_selection")
+
+    def locks_merge_attention(self, part_out, part_lse, batch, out, lse=None, stream=None):
+        _check(lib().locks_merge_attention(self.handle, _ptr(part_out), _ptr(part_lse), int(part_out.shape[0]), batch,
+                                           _ptr(out), _ptr(lse), _stream(stream)), "locks_merge_attention")
 
     def locks_select(self, q, summaries, kv: KVView, batch, page_ids, page_count, page_logmass=None,
                      page_logshare=None, stream=None):

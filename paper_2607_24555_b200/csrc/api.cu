@@ -277,6 +277,48 @@ int locks_build_summaries(locks_ctx *ctx, const locks_kv *kv, int batch, const i
   return locks_launch_build(ctx, kv, batch, page_begin, page_end, 0, summaries, nullptr, nullptr, (cudaStream_t)stream);
 }
 
+// ---- page-sharded decode: one long request whose pages are dealt to several GPUs (three small exchanges) ------
+
+int locks_scan(locks_ctx *ctx, const void *q, const void *summaries, const locks_kv *kv, int batch, float *page_logmass,
+               float *head_logz, locks_stream stream) {
+  int rc = check_common(ctx, kv, batch);
+  if (rc != LOCKS_OK) return rc;
+  if (!q || !summaries || !head_logz || ((uintptr_t)summaries % 16) || ((uintptr_t)q % 16)) return LOCKS_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  ctx->last_launches = 0;
+  if ((rc = locks_launch_scan(ctx, q, summaries, kv, batch, page_logmass ? page_logmass : ctx->shat, 0, st)) != LOCKS_OK) return rc;
+  return locks_launch_head_logz(ctx, kv, batch, head_logz, st);
+}
+
+int locks_select_scored(locks_ctx *ctx, const float *page_logmass, const float *head_logz_parts, int nparts,
+                        const locks_kv *kv, int batch, int32_t *page_ids, int32_t *page_count, float *page_logshare,
+                        locks_stream stream) {
+  int rc = check_common(ctx, kv, batch);
+  if (rc != LOCKS_OK) return rc;
+  if (!head_logz_parts || !page_ids || !page_count || nparts < 1) return LOCKS_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  ctx->last_launches = 0;
+  if ((rc = locks_launch_ext_partials(ctx, head_logz_parts, nparts, batch, st)) != LOCKS_OK) return rc;
+  return locks_launch_select(ctx, page_logmass ? page_logmass : ctx->shat, kv, batch, page_ids, page_count, page_logshare,
+                             nullptr, st);
+}
+
+int locks_merge_selection(locks_ctx *ctx, const float *cand_key, const int32_t *cand_page, int nparts, int batch,
+                          int32_t *page_ids, int32_t *page_count, locks_stream stream) {
+  if (!ctx || !cand_key || !cand_page || !page_ids || !page_count || nparts < 1 || batch < 1 || batch > ctx->cfg.max_batch)
+    return LOCKS_ERR_INVALID_ARG;
+  ctx->last_launches = 0;
+  return locks_launch_merge_selection(ctx, cand_key, cand_page, nparts, batch, page_ids, page_count, (cudaStream_t)stream);
+}
+
+int locks_merge_attention(locks_ctx *ctx, const void *part_out, const float *part_lse, int nparts, int batch, void *out,
+                          float *lse, locks_stream stream) {
+  if (!ctx || !part_out || !part_lse || !out || nparts < 1 || batch < 1 || batch > ctx->cfg.max_batch)
+    return LOCKS_ERR_INVALID_ARG;
+  ctx->last_launches = 0;
+  return locks_launch_merge_shards(ctx, part_out, part_lse, nparts, batch, out, lse, (cudaStream_t)stream);
+}
+
 int locks_fake_quantize_pages(locks_ctx *ctx, const locks_kv *kv, int batch, const int32_t *page_begin,
                               const int32_t *page_end, int bits, locks_stream stream) {
   int rc = check_common(ctx, kv, batch);

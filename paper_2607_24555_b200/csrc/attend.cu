@@ -548,7 +548,42 @@ __global__ void __launch_bounds__(128) attend_merge_kernel(const float *part_o, 
   }
 }
 
+// Merge of the attention partials of several shards of one sequence (each normalised over its own pages, with
+// its natural-log lse): out = sum_r w_r o_r, w_r = exp(lse_r - LSE), LSE = log sum_r exp(lse_r).
+template <typename T>
+__global__ void __launch_bounds__(LOCKS_D) merge_shards_kernel(const T *part_out, const float *part_lse, int nparts, int rows,
+                                                              T *out, float *lse) {
+  const int row = blockIdx.x, dim = threadIdx.x;
+  float M = -INFINITY;
+  for (int r = 0; r < nparts; ++r) M = fmaxf(M, part_lse[(int64_t)r * rows + row]);
+  float L = 0.f, acc = 0.f;
+  if (M > -INFINITY) {
+    for (int r = 0; r < nparts; ++r) {
+      const float l = part_lse[(int64_t)r * rows + row];
+      if (l == -INFINITY) continue;
+      const float w = __expf(l - M);
+      L += w;
+      acc += w * ldf<T>(part_out, ((int64_t)r * rows + row) * LOCKS_D + dim);
+    }
+    acc /= L;
+  }
+  stf<T>(out, (int64_t)row * LOCKS_D + dim, acc);
+  if (lse && dim == 0) lse[row] = M > -INFINITY ? M + __logf(L) : -INFINITY;
+}
+
 }  // namespace
+
+int locks_launch_merge_shards(locks_ctx *c, const void *part_out, const float *part_lse, int nparts, int batch, void *out,
+                              float *lse, cudaStream_t st) {
+  const int rows = batch * c->cfg.num_q_heads;
+  if (c->cfg.q_dtype == LOCKS_BF16)
+    merge_shards_kernel<__nv_bfloat16><<<rows, LOCKS_D, 0, st>>>(reinterpret_cast<const __nv_bfloat16 *>(part_out), part_lse, nparts,
+                                                                rows, reinterpret_cast<__nv_bfloat16 *>(out), lse);
+  else
+    merge_shards_kernel<float><<<rows, LOCKS_D, 0, st>>>(reinterpret_cast<const float *>(part_out), part_lse, nparts, rows,
+                                                        reinterpret_cast<float *>(out), lse);
+  return locks_check_launch(c);
+}
 
 int locks_launch_attend(locks_ctx *c, const void *q, const locks_kv *kv, int batch, const int32_t *ids,
                         const int32_t *cnt, void *out, float *lse, cudaStream_t st) {

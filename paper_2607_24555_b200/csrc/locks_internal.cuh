@@ -157,6 +157,12 @@ int locks_launch_quality(locks_ctx *c, const float *mass, const locks_kv *kv, in
                          const int32_t *cnt_a, const int32_t *ids_r, const int32_t *cnt_r, const int32_t *marked,
                          int n_marked, float *out, cudaStream_t st);
 
+int locks_launch_head_logz(locks_ctx *c, const locks_kv *kv, int batch, float *logz, cudaStream_t st);
+int locks_launch_ext_partials(locks_ctx *c, const float *logz_parts, int nparts, int batch, cudaStream_t st);
+int locks_launch_merge_selection(locks_ctx *c, const float *cand_key, const int32_t *cand_page, int nparts, int batch,
+                                 int32_t *ids, int32_t *cnt, cudaStream_t st);
+int locks_launch_merge_shards(locks_ctx *c, const void *part_out, const float *part_lse, int nparts, int batch, void *out,
+                              float *lse, cudaStream_t st);
 int locks_launch_fake_quant(locks_ctx *c, const locks_kv *kv, int batch, const int32_t *pb, const int32_t *pe, int bits,
                             cudaStream_t st);
 

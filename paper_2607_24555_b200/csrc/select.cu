@@ -480,7 +480,117 @@ __global__ void __launch_bounds__(LOCKS_SEL_THREADS, 2) select_kernel(SelParams 
   }
 }
 
+// ---- page-sharded selection (one long request whose pages are dealt to several GPUs) -----------------------
+// log Z_g of the pages one shard scanned, from the scan's partials: one warp per (request, query head)
+__global__ void __launch_bounds__(32) head_logz_kernel(const float2 *part, const int32_t *part_cnt, const int32_t *seq_lens,
+                                                       float *logz, int Hq, int Hkv, int max_groups, int part_slots, int k) {
+  const int hq = blockIdx.x, b = blockIdx.y, lane = threadIdx.x;
+  pdl_wait();
+  const int P = (seq_lens[b] + LOCKS_B - 1) / LOCKS_B;
+  const int64_t prob = (int64_t)b * Hkv + hq / (Hq / Hkv);
+  int nparts = part_cnt ? min(max(part_cnt[prob], 0), max_groups) : min(part_slots, (P - 1 + LOCKS_GROUP - 1) / LOCKS_GROUP);
+  if (P <= k) nparts = 0;
+  const float2 *pp = part + ((int64_t)b * Hq + hq) * max_groups;
+  float m = -INFINITY, s = 0.f;
+  for (int i = lane; i < nparts; i += 32) {
+    const float2 x = pp[i];
+    const float nm = fmaxf(m, x.x);
+    if (nm > -INFINITY) { s = s * __expf(m - nm) + x.y * __expf(x.x - nm); m = nm; }
+  }
+  const float M = warp_max(m);
+  s = warp_sum(M > -INFINITY ? s * __expf(m - M) : 0.f);
+  if (lane == 0) logz[(int64_t)b * Hq + hq] = M > -INFINITY ? M + __logf(s) : -INFINITY;
+}
+
+// the shards' log Z values as the selector's partials: slot r of head g holds (log Z_g of shard r, 1)
+__global__ void __launch_bounds__(128) ext_partials_kernel(const float *logz_parts, int nparts, float2 *part, int32_t *part_cnt,
+                                                           int batch, int Hq, int Hkv, int max_groups) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < batch * Hkv) part_cnt[i] = nparts;
+  if (i >= batch * Hq) return;
+  for (int r = 0; r < nparts; ++r) {
+    const float v = logz_parts[(int64_t)r * batch * Hq + i];
+    part[(int64_t)i * max_groups + r] = make_float2(v, v > -INFINITY ? 1.f : 0.f);
+  }
+}
+
+// Global top-(k-2) of the shards' candidate lists (each in page order, shards in page order, so that list order
+// is page order and the lower-page tie rule carries over): one CTA per (request, KV head).
+__global__ void __launch_bounds__(LOCKS_SEL_THREADS) merge_selection_kernel(const float *cand_key, const int32_t *cand_page, int nparts,
+                                                                           int batch, int Hkv, int kc, int32_t *ids, int32_t *cnt) {
+  SelShared &sh = shared_state();
+  const int h = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
+  const int64_t prob = (int64_t)b * Hkv + h, nprob = (int64_t)batch * Hkv;
+  const int N = nparts * kc, nslab = (N + LOCKS_SEL_THREADS - 1) / LOCKS_SEL_THREADS;
+  int32_t *out = ids + prob * kc;
+  __shared__ int s_valid;
+  if (tid == 0) s_valid = 0;
+  __syncthreads();
+  int mine = 0;
+  for (int i = 0; i < nslab; ++i) {
+    const int e = i * LOCKS_SEL_THREADS + tid;
+    uint32_t key = 0u;
+    if (e < N) {
+      const int r = e / kc, j = e - r * kc;
+      const int64_t at = ((int64_t)r * nprob + prob) * kc + j;
+      if (cand_page[at] >= 0) { key = order_key(cand_key[at]); ++mine; }
+    }
+    sh.key[e] = key;
+  }
+  for (int j = tid; j < kc; j += LOCKS_SEL_THREADS) out[j] = -1;
+  if (mine) atomicAdd(&s_valid, mine);
+  __syncthreads();
+  const int K = min(kc, s_valid);
+  if (K > 0) {
+    const uint2 r = radix_select(nslab, K);
+    compact_emit(nslab, r.x, (int)r.y, K, kEmitIds, 0, out - 1, nullptr, nullptr);   // out[pos] = winning entry, in list order
+    __syncthreads();
+    int page[(kMaxWin + LOCKS_SEL_THREADS - 1) / LOCKS_SEL_THREADS];
+#pragma unroll
+    for (int u = 0; u < (kMaxWin + LOCKS_SEL_THREADS - 1) / LOCKS_SEL_THREADS; ++u) {
+      const int j = tid + u * LOCKS_SEL_THREADS;
+      page[u] = -1;
+      if (j < K) {
+        const int e = out[j], rr = e / kc, jj = e - rr * kc;
+        page[u] = cand_page[((int64_t)rr * nprob + prob) * kc + jj];
+      }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int u = 0; u < (kMaxWin + LOCKS_SEL_THREADS - 1) / LOCKS_SEL_THREADS; ++u)
+      if (tid + u * LOCKS_SEL_THREADS < K) out[tid + u * LOCKS_SEL_THREADS] = page[u];
+  }
+  if (tid == 0) cnt[prob] = K;
+}
+
 }  // namespace
+
+int locks_launch_head_logz(locks_ctx *c, const locks_kv *kv, int batch, float *logz, cudaStream_t st) {
+  locks_launch_pdl(head_logz_kernel, dim3(c->cfg.num_q_heads, batch), dim3(32), 0, st, (const float2 *)c->part,
+                   (const int32_t *)(c->part_balanced ? c->part_cnt : nullptr), (const int32_t *)kv->seq_lens, logz,
+                   c->cfg.num_q_heads, c->cfg.num_kv_heads, c->max_groups, c->part_slots, c->k);
+  return locks_check_launch(c);
+}
+
+int locks_launch_ext_partials(locks_ctx *c, const float *logz_parts, int nparts, int batch, cudaStream_t st) {
+  if (nparts < 1 || nparts > c->max_groups) return LOCKS_ERR_INVALID_ARG;
+  const int n = batch * c->cfg.num_q_heads;
+  ext_partials_kernel<<<(n + 127) / 128, 128, 0, st>>>(logz_parts, nparts, c->part, c->part_cnt, batch, c->cfg.num_q_heads,
+                                                       c->cfg.num_kv_heads, c->max_groups);
+  c->part_slots = nparts;
+  c->part_balanced = 1;   // the selector takes the count from part_cnt
+  return locks_check_launch(c);
+}
+
+int locks_launch_merge_selection(locks_ctx *c, const float *cand_key, const int32_t *cand_page, int nparts, int batch,
+                                 int32_t *ids, int32_t *cnt, cudaStream_t st) {
+  if (nparts < 1 || (int64_t)nparts * c->sel_kc > kMaxKeys) return LOCKS_ERR_UNSUPPORTED;
+  if (locks_attrs_needed(LOCKS_ATTR_SELECT))
+    cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 116 * 1024);
+  merge_selection_kernel<<<dim3(c->cfg.num_kv_heads, batch), LOCKS_SEL_THREADS, sizeof(SelShared), st>>>(
+      cand_key, cand_page, nparts, batch, c->cfg.num_kv_heads, c->sel_kc, ids, cnt);
+  return locks_check_launch(c);
+}
 
 int locks_launch_select(locks_ctx *c, const float *shat, const locks_kv *kv, int batch, int32_t *ids,
                         int32_t *cnt, float *logshare, const locks_append *app, cudaStream_t st) {
