@@ -46,6 +46,10 @@ extern "C" {
 
 #define LOCKS_FMT_F32 0 /* summary stored as fp32 mu, V, C                               */
 #define LOCKS_FMT_I4 1  /* int4 basis, int8 coefficients + centroid, fp16 scales (r8i4)  */
+#define LOCKS_FMT_I8 2  /* int8 basis, int8 coefficients + centroid: the "int8 basis" arm of the paper's rank x
+                           precision ablation (App. B); plain fp32-arithmetic kernels                    */
+#define LOCKS_FMT_BF16 3 /* bf16 basis, int8 coefficients + centroid: the paper's "r8fp" control (Sec. 4
+                           robustness paragraph, App. B); plain fp32-arithmetic kernels                  */
 
 /* How the G query heads of a KV head are combined into one ranking key per page (Sec. 4; ablated in the
  * paper's App. D "GQA combine" table).  The selection (sink + most recent + top k-2 by key, ties to the lower
@@ -65,7 +69,7 @@ typedef struct {
   int32_t page_size;         /* B; 16                                                         */
   int32_t num_q_heads;       /* Hq                                                            */
   int32_t num_kv_heads;      /* Hkv, Hq % Hkv == 0, G = Hq/Hkv <= 16                          */
-  int32_t rank;              /* r: I4 format 2|4|8, F32 format 1..16                          */
+  int32_t rank;              /* r: I4 format 2|4|8, other formats 1..16                       */
   int32_t summary_fmt;       /* LOCKS_FMT_*                                                   */
   int32_t kv_dtype;          /* LOCKS_F32 | LOCKS_BF16 (K, V, k_new, v_new)                   */
   int32_t q_dtype;           /* LOCKS_F32 | LOCKS_BF16 (q and out); must equal kv_dtype       */
@@ -92,7 +96,10 @@ typedef struct {
 /* Bytes of one stored summary, per (physical block, KV head), padded to a multiple of 16.
  * I4 format: 82 r + 162 payload bytes at B=16, d=128 (818 / 490 / 326 at r = 8 / 4 / 2: the
  * paper's stored-payload table, App. C.1), i.e. d r/2 int4 basis + B r int8 coefficients + d int8
- * centroid + (r + B + 1) fp16 scales (Sec. 4 "Build").  F32 format: 4 (d + r d + B r).
+ * centroid + (r + B + 1) fp16 scales (Sec. 4 "Build").  F32 format: 4 (d + r d + B r).  I8 format: d r + B r + d +
+ * 2 (r + B + 1).  BF16 format: 2 d r + B r + d + 2 (B + 1).  The last two are plain row-major:
+ * [basis r x d][coefficients B x r][centroid d][coefficient scales B][basis scales r (I8 only)][centroid scale],
+ * integer codes stored offset-binary (byte = code + 128).
  * The summaries buffer is [num_blocks][Hkv][locks_summary_bytes]. 0 on an invalid config. */
 size_t locks_summary_bytes(const locks_config *cfg);
 

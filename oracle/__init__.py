@@ -18,7 +18,7 @@ _SRC = os.path.join(_HERE, "locks_oracle.c")
 _LIB = os.path.join(_HERE, "liblocks_oracle.so")
 
 F32, BF16, F64 = 0, 1, 2
-FMT_F32, FMT_I4 = 0, 1
+FMT_F32, FMT_I4, FMT_I8, FMT_BF16 = 0, 1, 2, 3
 
 _lib = None
 

@@ -50,6 +50,8 @@
 
 #define ORA_FMT_F32 0
 #define ORA_FMT_I4 1
+#define ORA_FMT_I8 2   /* int8 basis, int8 coefficients + centroid: the "int8 basis" arm of the paper's precision ablation */
+#define ORA_FMT_BF16 3 /* bf16 basis, int8 coefficients + centroid: the paper's "r8fp" control */
 
 typedef struct {
   const void *k, *v;        /* paged cache, element (block, head, token, dim) at
@@ -229,6 +231,10 @@ int ora_build_page(const double *keys, int B, int d, int r, double *mu, double *
 /* Bytes of one stored summary (what the paper's payload table counts) and its padded stride. */
 int64_t ora_summary_payload_bytes(int fmt, int r, int B, int d) {
   if (fmt == ORA_FMT_F32) return 4 * ((int64_t)d + (int64_t)r * d + (int64_t)B * r);
+  /* int8 basis d*r, int8 coefficients B*r, int8 centroid d, fp16 scales r + B + 1 */
+  if (fmt == ORA_FMT_I8) return (int64_t)d * r + (int64_t)B * r + d + 2 * ((int64_t)r + B + 1);
+  /* bf16 basis 2*d*r (no basis scales), int8 coefficients and centroid, fp16 scales B + 1 */
+  if (fmt == ORA_FMT_BF16) return 2 * (int64_t)d * r + (int64_t)B * r + d + 2 * ((int64_t)B + 1);
   /* int4 basis d*r/2, int8 coefficients B*r, int8 centroid d, fp16 scales: r + B + 1 */
   return (int64_t)d * r / 2 + (int64_t)B * r + d + 2 * ((int64_t)r + B + 1);
 }
@@ -289,6 +295,36 @@ void ora_pack(int fmt, int r, int B, int d, const double *mu, const double *V, c
       for (int l = 0; l < r; ++l) f[d + r * d + i * r + l] = (float)C[i * r + l];
     return;
   }
+  if (fmt == ORA_FMT_I8 || fmt == ORA_FMT_BF16) {
+    /* plain row-major layout: [basis r x d][coefficients B x r][centroid d][sC B][sV r (int8 basis only)][sMu];
+       integer codes offset-binary (byte = code + 128), bf16 by round-to-nearest-even */
+    int wide = fmt == ORA_FMT_BF16 ? 2 : 1;
+    int oc = wide * d * r, om = oc + B * r, osc = om + d, osv = osc + 2 * B, osmu = osv + (fmt == ORA_FMT_I8 ? 2 * r : 0);
+    uint16_t hb;
+    for (int l = 0; l < r; ++l) {
+      if (fmt == ORA_FMT_I8) {
+        double sc = quant_scale(V + l * d, d, 1, 127, &hb);
+        memcpy(blob + osv + 2 * l, &hb, 2);
+        for (int c = 0; c < d; ++c) blob[l * d + c] = (uint8_t)(quant_code(V[l * d + c], sc, 127) + 128);
+      } else {
+        for (int c = 0; c < d; ++c) {
+          float f = (float)V[l * d + c];
+          uint32_t u; memcpy(&u, &f, 4);
+          uint16_t b16 = (uint16_t)((u + 0x7FFFu + ((u >> 16) & 1u)) >> 16);
+          memcpy(blob + 2 * (l * d + c), &b16, 2);
+        }
+      }
+    }
+    for (int i = 0; i < B; ++i) {
+      double sc = quant_scale(C + i * r, r, 1, 127, &hb);
+      memcpy(blob + osc + 2 * i, &hb, 2);
+      for (int l = 0; l < r; ++l) blob[oc + i * r + l] = (uint8_t)(quant_code(C[i * r + l], sc, 127) + 128);
+    }
+    double sc = quant_scale(mu, d, 1, 127, &hb);
+    memcpy(blob + osmu, &hb, 2);
+    for (int c = 0; c < d; ++c) blob[om + c] = (uint8_t)(quant_code(mu[c], sc, 127) + 128);
+    return;
+  }
   int off_coef = d * r / 2, off_mu = off_coef + B * r, off_sc = off_mu + d;
   int off_sv = off_sc + 2 * B, off_smu = off_sv + 2 * r;
   uint16_t bits;
@@ -325,6 +361,32 @@ void ora_unpack(int fmt, int r, int B, int d, const uint8_t *blob, double *mu, d
       for (int c = 0; c < d; ++c) V[l * d + c] = f[d + l * d + c];
     for (int i = 0; i < B; ++i)
       for (int l = 0; l < r; ++l) C[i * r + l] = f[d + r * d + i * r + l];
+    return;
+  }
+  if (fmt == ORA_FMT_I8 || fmt == ORA_FMT_BF16) {
+    int wide = fmt == ORA_FMT_BF16 ? 2 : 1;
+    int oc = wide * d * r, om = oc + B * r, osc = om + d, osv = osc + 2 * B, osmu = osv + (fmt == ORA_FMT_I8 ? 2 * r : 0);
+    uint16_t hb;
+    for (int l = 0; l < r; ++l) {
+      double sc = 1;
+      if (fmt == ORA_FMT_I8) { memcpy(&hb, blob + osv + 2 * l, 2); sc = half_to_double(hb); }
+      for (int c = 0; c < d; ++c) {
+        if (fmt == ORA_FMT_I8) V[l * d + c] = sc * ((int)blob[l * d + c] - 128);
+        else {
+          uint16_t b16; memcpy(&b16, blob + 2 * (l * d + c), 2);
+          uint32_t u = (uint32_t)b16 << 16; float f; memcpy(&f, &u, 4);
+          V[l * d + c] = f;
+        }
+      }
+    }
+    for (int i = 0; i < B; ++i) {
+      memcpy(&hb, blob + osc + 2 * i, 2);
+      double sc = half_to_double(hb);
+      for (int l = 0; l < r; ++l) C[i * r + l] = sc * ((int)blob[oc + i * r + l] - 128);
+    }
+    memcpy(&hb, blob + osmu, 2);
+    double sc = half_to_double(hb);
+    for (int c = 0; c < d; ++c) mu[c] = sc * ((int)blob[om + c] - 128);
     return;
   }
   int off_coef = d * r / 2, off_mu = off_coef + B * r, off_sc = off_mu + d;

@@ -11,7 +11,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "liblocks.so")
 
 F32, BF16 = 0, 1
-FMT_F32, FMT_I4 = 0, 1
+FMT_F32, FMT_I4, FMT_I8, FMT_BF16 = 0, 1, 2, 3
 
 SYMBOLS = ["locks_summary_bytes", "locks_workspace_bytes", "locks_create", "locks_destroy",
            "locks_build_summaries", "locks_select", "locks_sparse_attend", "locks_decode_step",
@@ -154,7 +154,7 @@ def make_config(Hq, Hkv, rank, fmt, dtype, max_batch, max_pages, budget, sm_scal
     if sm_scale is None:
         sm_scale = d ** -0.5
     dt = BF16 if dtype in ("bf16", torch.bfloat16) else F32
-    f = FMT_I4 if fmt == "i4" else FMT_F32
+    f = {"i4": FMT_I4, "f32": FMT_F32, "i8": FMT_I8, "bf16": FMT_BF16}[fmt]
     return Config(d, B, Hq, Hkv, rank, f, dt, dt, max_batch, max_pages, budget, sm_scale, combine)
 
 

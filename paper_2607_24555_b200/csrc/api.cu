@@ -16,7 +16,7 @@ int validate(const locks_config *c) {
   const int k = (c->budget_tokens + c->page_size - 1) / c->page_size;
   if (c->budget_tokens <= 0 || k < 2) return LOCKS_ERR_INVALID_ARG;
   if (!(c->sm_scale > 0.f)) return LOCKS_ERR_INVALID_ARG;
-  if (c->summary_fmt != LOCKS_FMT_F32 && c->summary_fmt != LOCKS_FMT_I4) return LOCKS_ERR_INVALID_ARG;
+  if (c->summary_fmt < LOCKS_FMT_F32 || c->summary_fmt > LOCKS_FMT_BF16) return LOCKS_ERR_INVALID_ARG;
   if (c->combine < LOCKS_COMBINE_SHARE_AVG || c->combine > LOCKS_COMBINE_GROUP_MASS) return LOCKS_ERR_INVALID_ARG;
   if ((c->kv_dtype != LOCKS_F32 && c->kv_dtype != LOCKS_BF16) || (c->q_dtype != LOCKS_F32 && c->q_dtype != LOCKS_BF16))
     return LOCKS_ERR_INVALID_ARG;
@@ -24,7 +24,7 @@ int validate(const locks_config *c) {
   if (c->num_q_heads / c->num_kv_heads > 16) return LOCKS_ERR_UNSUPPORTED;
   if (c->kv_dtype != c->q_dtype) return LOCKS_ERR_UNSUPPORTED;
   if (c->summary_fmt == LOCKS_FMT_I4 && c->rank != 2 && c->rank != 4 && c->rank != 8) return LOCKS_ERR_UNSUPPORTED;
-  if (c->summary_fmt == LOCKS_FMT_F32 && c->rank > 16) return LOCKS_ERR_UNSUPPORTED;
+  if (c->summary_fmt != LOCKS_FMT_I4 && c->rank > 16) return LOCKS_ERR_UNSUPPORTED;
   const int chunk_max = LOCKS_SEL_THREADS * LOCKS_SEL_MAX_EPT;
   const int chunks = (c->max_pages_per_seq + chunk_max - 1) / chunk_max;
   if (chunks > 1 && (size_t)chunks * (k - 2) > 16 * LOCKS_SEL_THREADS) return LOCKS_ERR_UNSUPPORTED;
@@ -41,7 +41,7 @@ Layout make_layout(const locks_config *c) {
   Layout L;
   L.G = c->num_q_heads / c->num_kv_heads;
   L.k = (c->budget_tokens + c->page_size - 1) / c->page_size;
-  L.S = c->summary_fmt == LOCKS_FMT_I4 ? i4_stride(c->rank) : f32_stride(c->rank);
+  L.S = locks_fmt_stride(c->summary_fmt, c->rank);
   L.max_groups = (c->max_pages_per_seq + LOCKS_GROUP - 1) / LOCKS_GROUP;
   // Pages per thread of a selector CTA (1 .. 16; a CTA ranks sel_ept * 512 pages).  With many (request,
   // KV head) problems and a context of up to 8192 pages, one CTA ranks a whole problem.  Otherwise a problem is

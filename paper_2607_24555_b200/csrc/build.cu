@@ -387,7 +387,8 @@ __global__ void __launch_bounds__(kBuildWarps * 32, kBuildCtasPerSm) build_kerne
     for (int e = lane; e < i4_stride(8) / 4; e += 32) reinterpret_cast<uint32_t *>(blob)[e] = 0u;
     __syncwarp();
   }
-  float *fout = reinterpret_cast<float *>(p.summ + ((int64_t)block * p.Hkv + h) * p.S);
+  uint8_t *gout = p.summ + ((int64_t)block * p.Hkv + h) * p.S;
+  float *fout = reinterpret_cast<float *>(gout);
   uint32_t sign_bits = 0u;   // bit l: mode l was flipped
   {
 #pragma unroll 1
@@ -424,6 +425,16 @@ __global__ void __launch_bounds__(kBuildWarps * 32, kBuildCtasPerSm) build_kerne
       }
       if (FMT == LOCKS_FMT_F32) {
         *reinterpret_cast<float4 *>(fout + LOCKS_D + l * LOCKS_D + lane * 4) = make_float4(v[0], v[1], v[2], v[3]);
+      } else if (FMT == LOCKS_FMT_BF16) {   // row-major bf16 basis, straight to global memory
+        *reinterpret_cast<uint2 *>(gout + 2 * (l * LOCKS_D + lane * 4)) = make_uint2(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]));
+      } else if (FMT == LOCKS_FMT_I8) {     // row-major int8 basis, one scale per mode
+        const __half sh = __float2half_rn(best / 127.f);
+        const float sc = inv_scale(__half2float(sh));
+        if (lane == 0) *reinterpret_cast<__half *>(gout + wb_off_sv(r, 1) + 2 * l) = sh;
+        uint32_t w = 0u;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) w |= (uint32_t)((int)round_code(v[c], sc, 127.f) + 128) << (8 * c);
+        *reinterpret_cast<uint32_t *>(gout + l * LOCKS_D + lane * 4) = w;
       } else {
         const __half sh = __float2half_rn(best / 7.f);
         const float sc = inv_scale(__half2float(sh));
@@ -455,6 +466,12 @@ __global__ void __launch_bounds__(kBuildWarps * 32, kBuildCtasPerSm) build_kerne
     }
     if (FMT == LOCKS_FMT_F32) {
       for (int l = 0; l < r; ++l) fout[LOCKS_D + r * LOCKS_D + lane * r + l] = cf[l & 15];
+    } else if (FMT == LOCKS_FMT_I8 || FMT == LOCKS_FMT_BF16) {
+      constexpr int W = FMT == LOCKS_FMT_BF16 ? 2 : 1;
+      const __half sh = __float2half_rn(mx / 127.f);
+      const float sc = inv_scale(__half2float(sh));
+      *reinterpret_cast<__half *>(gout + wb_off_sc(r, W) + 2 * lane) = sh;
+      for (int l = 0; l < r; ++l) gout[wb_off_coef(r, W) + lane * r + l] = (uint8_t)((int)round_code(cf[l & 15], sc, 127.f) + 128);
     } else {
       const __half sh = __float2half_rn(mx / 127.f);
       const float sc = inv_scale(__half2float(sh));
@@ -469,6 +486,19 @@ __global__ void __launch_bounds__(kBuildWarps * 32, kBuildCtasPerSm) build_kerne
   // centroid
   if (FMT == LOCKS_FMT_F32) {
     *reinterpret_cast<float4 *>(fout + lane * 4) = make_float4(mu[0], mu[1], mu[2], mu[3]);
+  } else if (FMT == LOCKS_FMT_I8 || FMT == LOCKS_FMT_BF16) {
+    constexpr int W = FMT == LOCKS_FMT_BF16 ? 2 : 1;
+    float mx = fmaxf(fmaxf(fabsf(mu[0]), fabsf(mu[1])), fmaxf(fabsf(mu[2]), fabsf(mu[3])));
+    mx = __uint_as_float(__reduce_max_sync(0xffffffffu, __float_as_uint(mx)));
+    const __half sh = __float2half_rn(mx / 127.f);
+    const float sc = inv_scale(__half2float(sh));
+    if (lane == 0) *reinterpret_cast<__half *>(gout + wb_off_smu(r, W)) = sh;
+    uint32_t w = 0u;
+#pragma unroll
+    for (int c = 0; c < 4; ++c) w |= (uint32_t)((int)round_code(mu[c], sc, 127.f) + 128) << (8 * c);
+    *reinterpret_cast<uint32_t *>(gout + wb_off_mu(r, W) + lane * 4) = w;
+    // bytes between the payload and the 16-byte padded stride stay zero (the buffer is the caller's; clear them)
+    for (int e = wb_off_smu(r, W) + 2 + lane; e < p.S; e += 32) gout[e] = 0;
   } else {
     float mx = fmaxf(fmaxf(fabsf(mu[0]), fabsf(mu[1])), fmaxf(fabsf(mu[2]), fabsf(mu[3])));
     mx = __uint_as_float(__reduce_max_sync(0xffffffffu, __float_as_uint(mx)));
@@ -506,18 +536,24 @@ int locks_launch_build(locks_ctx *c, const locks_kv *kv, int batch, const int32_
   }
   dim3 grid = just_filled ? dim3((batch * p.Hkv + kBuildWarps - 1) / kBuildWarps)
                           : dim3((c->Pmax + kBuildWarps - 1) / kBuildWarps, p.Hkv, batch);
-  const bool bf = c->cfg.kv_dtype == LOCKS_BF16, i4 = c->cfg.summary_fmt == LOCKS_FMT_I4;
+  const bool bf = c->cfg.kv_dtype == LOCKS_BF16;
   const int smem_bf = kBuildWarps * build_smem_per_warp<__nv_bfloat16>(), smem_f32 = kBuildWarps * build_smem_per_warp<float>();
   const int smem = bf ? smem_bf : smem_f32;
-  if (locks_attrs_needed(LOCKS_ATTR_BUILD)) {
-    cudaFuncSetAttribute(build_kernel<__nv_bfloat16, LOCKS_FMT_I4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bf);
-    cudaFuncSetAttribute(build_kernel<__nv_bfloat16, LOCKS_FMT_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bf);
-    cudaFuncSetAttribute(build_kernel<float, LOCKS_FMT_I4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_f32);
-    cudaFuncSetAttribute(build_kernel<float, LOCKS_FMT_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_f32);
+#define LOCKS_BUILD_CASE(F_)                                                                                                \
+  do {                                                                                                                     \
+    if (locks_attrs_needed(LOCKS_ATTR_BUILD + F_)) {                                                                       \
+      cudaFuncSetAttribute(build_kernel<__nv_bfloat16, F_>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bf);       \
+      cudaFuncSetAttribute(build_kernel<float, F_>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_f32);               \
+    }                                                                                                                      \
+    if (bf) build_kernel<__nv_bfloat16, F_><<<grid, kBuildWarps * 32, smem, st>>>(p);                                     \
+    else build_kernel<float, F_><<<grid, kBuildWarps * 32, smem, st>>>(p);                                                 \
+  } while (0)
+  switch (c->cfg.summary_fmt) {
+    case LOCKS_FMT_I4: LOCKS_BUILD_CASE(LOCKS_FMT_I4); break;
+    case LOCKS_FMT_I8: LOCKS_BUILD_CASE(LOCKS_FMT_I8); break;
+    case LOCKS_FMT_BF16: LOCKS_BUILD_CASE(LOCKS_FMT_BF16); break;
+    default: LOCKS_BUILD_CASE(LOCKS_FMT_F32); break;
   }
-  if (bf && i4) build_kernel<__nv_bfloat16, LOCKS_FMT_I4><<<grid, kBuildWarps * 32, smem, st>>>(p);
-  else if (bf) build_kernel<__nv_bfloat16, LOCKS_FMT_F32><<<grid, kBuildWarps * 32, smem, st>>>(p);
-  else if (i4) build_kernel<float, LOCKS_FMT_I4><<<grid, kBuildWarps * 32, smem, st>>>(p);
-  else build_kernel<float, LOCKS_FMT_F32><<<grid, kBuildWarps * 32, smem, st>>>(p);
+#undef LOCKS_BUILD_CASE
   return locks_check_launch(c);
 }

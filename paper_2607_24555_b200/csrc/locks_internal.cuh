@@ -219,7 +219,7 @@ static inline int locks_check_launch(locks_ctx *c) {
 // Function attributes (dynamic shared-memory limit, non-portable cluster size) belong to a device, not to the
 // process: true exactly once per (current device, kernel family), so that a process that drives several GPUs
 // sets them on each.  Thread-safe.
-enum { LOCKS_ATTR_SELECT = 0, LOCKS_ATTR_ATTEND = 1, LOCKS_ATTR_BUILD = 2, LOCKS_ATTR_EXACT = 3, LOCKS_ATTR_SCAN = 8 };
+enum { LOCKS_ATTR_SELECT = 0, LOCKS_ATTR_ATTEND = 1, LOCKS_ATTR_EXACT = 3, LOCKS_ATTR_BUILD = 4 /* + format */, LOCKS_ATTR_SCAN = 8 };
 bool locks_attrs_needed(int family);
 
 // ---------------------------------------------------------------- I4 blob geometry (B = 16, d = 128)
@@ -231,6 +231,17 @@ __host__ __device__ constexpr int i4_off_sv(int r) { return 80 * r + 160; }
 __host__ __device__ constexpr int i4_off_smu(int r) { return 82 * r + 160; }
 __host__ __device__ constexpr int i4_stride(int r) { return (82 * r + 162 + 15) / 16 * 16; }
 __host__ __device__ constexpr int f32_stride(int r) { return 4 * (LOCKS_D + r * LOCKS_D + LOCKS_B * r); }
+// Row-major formats with an int8 (wide = 1) or bf16 (wide = 2) basis:
+// [basis r x d][coefficients B x r][centroid d][sC B x fp16][sV r x fp16 (int8 basis only)][sMu fp16], padded to 16.
+__host__ __device__ constexpr int wb_off_coef(int r, int wide) { return wide * LOCKS_D * r; }
+__host__ __device__ constexpr int wb_off_mu(int r, int wide) { return wide * LOCKS_D * r + LOCKS_B * r; }
+__host__ __device__ constexpr int wb_off_sc(int r, int wide) { return wb_off_mu(r, wide) + LOCKS_D; }
+__host__ __device__ constexpr int wb_off_sv(int r, int wide) { return wb_off_sc(r, wide) + 2 * LOCKS_B; }
+__host__ __device__ constexpr int wb_off_smu(int r, int wide) { return wb_off_sv(r, wide) + (wide == 1 ? 2 * r : 0); }
+__host__ __device__ constexpr int wb_stride(int r, int wide) { return (wb_off_smu(r, wide) + 2 + 15) / 16 * 16; }
+__host__ __device__ constexpr int locks_fmt_stride(int fmt, int r) {
+  return fmt == LOCKS_FMT_I4 ? i4_stride(r) : fmt == LOCKS_FMT_F32 ? f32_stride(r) : wb_stride(r, fmt == LOCKS_FMT_BF16 ? 2 : 1);
+}
 
 #ifdef __CUDACC__
 

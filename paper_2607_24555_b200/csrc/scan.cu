@@ -124,6 +124,25 @@ __global__ void __launch_bounds__(128) scan_generic_kernel(ScanParams p) {
           for (int u = 0; u < 4; ++u) s += f[LOCKS_D + l * LOCKS_D + lane * 4 + u] * qv[u];
           proj[l] = warp_sum(s);
         }
+      } else if (FMT == LOCKS_FMT_I8 || FMT == LOCKS_FMT_BF16) {
+        constexpr int W = FMT == LOCKS_FMT_BF16 ? 2 : 1;
+        const float smu = __half2float(*reinterpret_cast<const __half *>(blob + wb_off_smu(r, W)));
+#pragma unroll
+        for (int u = 0; u < 4; ++u) a += (float)((int)blob[wb_off_mu(r, W) + lane * 4 + u] - 128) * qv[u];
+        a *= smu;
+        for (int l = 0; l < r; ++l) {
+          float s = 0.f;
+          if (FMT == LOCKS_FMT_I8) {
+#pragma unroll
+            for (int u = 0; u < 4; ++u) s += (float)((int)blob[l * LOCKS_D + lane * 4 + u] - 128) * qv[u];
+            s *= __half2float(*reinterpret_cast<const __half *>(blob + wb_off_sv(r, W) + 2 * l));
+          } else {
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+              s += __bfloat162float(reinterpret_cast<const __nv_bfloat16 *>(blob)[l * LOCKS_D + lane * 4 + u]) * qv[u];
+          }
+          proj[l] = warp_sum(s);
+        }
       } else {
         const float smu = __half2float(*reinterpret_cast<const __half *>(blob + i4_off_smu(r)));
 #pragma unroll
@@ -144,6 +163,10 @@ __global__ void __launch_bounds__(128) scan_generic_kernel(ScanParams p) {
         if (FMT == LOCKS_FMT_F32) {
           const float *f = reinterpret_cast<const float *>(blob) + LOCKS_D + r * LOCKS_D + lane * r;
           for (int l = 0; l < r; ++l) s += proj[l] * f[l];
+        } else if (FMT == LOCKS_FMT_I8 || FMT == LOCKS_FMT_BF16) {
+          constexpr int W = FMT == LOCKS_FMT_BF16 ? 2 : 1;
+          for (int l = 0; l < r; ++l) s += proj[l] * (float)((int)blob[wb_off_coef(r, W) + lane * r + l] - 128);
+          s *= __half2float(*reinterpret_cast<const __half *>(blob + wb_off_sc(r, W) + 2 * lane));
         } else {
           for (int l = 0; l < r; ++l) s += proj[l] * i4_coef_val(blob, r, lane, l);
           s *= i4_sc_val(blob, r, lane);
@@ -1037,6 +1060,12 @@ int locks_launch_scan(locks_ctx *c, const void *q, const void *summaries, const 
     if (c->cfg.summary_fmt == LOCKS_FMT_F32) {
       if (qbf) locks_launch_pdl(scan_generic_kernel<LOCKS_FMT_F32, __nv_bfloat16>, grid, dim3(128), 0, st, p);
       else locks_launch_pdl(scan_generic_kernel<LOCKS_FMT_F32, float>, grid, dim3(128), 0, st, p);
+    } else if (c->cfg.summary_fmt == LOCKS_FMT_I8) {
+      if (qbf) locks_launch_pdl(scan_generic_kernel<LOCKS_FMT_I8, __nv_bfloat16>, grid, dim3(128), 0, st, p);
+      else locks_launch_pdl(scan_generic_kernel<LOCKS_FMT_I8, float>, grid, dim3(128), 0, st, p);
+    } else if (c->cfg.summary_fmt == LOCKS_FMT_BF16) {
+      if (qbf) locks_launch_pdl(scan_generic_kernel<LOCKS_FMT_BF16, __nv_bfloat16>, grid, dim3(128), 0, st, p);
+      else locks_launch_pdl(scan_generic_kernel<LOCKS_FMT_BF16, float>, grid, dim3(128), 0, st, p);
     } else {
       if (qbf) locks_launch_pdl(scan_generic_kernel<LOCKS_FMT_I4, __nv_bfloat16>, grid, dim3(128), 0, st, p);
       else locks_launch_pdl(scan_generic_kernel<LOCKS_FMT_I4, float>, grid, dim3(128), 0, st, p);

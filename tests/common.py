@@ -48,7 +48,7 @@ def oracle_cache(case) -> oracle.Cache:
 
 
 def fmt_code(w) -> int:
-    return oracle.FMT_I4 if w.fmt == "i4" else oracle.FMT_F32
+    return {"i4": oracle.FMT_I4, "f32": oracle.FMT_F32, "i8": oracle.FMT_I8, "bf16": oracle.FMT_BF16}[w.fmt]
 
 
 def check_page_sets(ids_gpu, cnt_gpu, ids_ora, cnt_ora, logshare_ora, seq_lens, B, k, band=2e-3):

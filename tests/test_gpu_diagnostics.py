@@ -186,3 +186,34 @@ def test_fake_quantised_cache_composition(bits, dtype, arm):
     gc.cache = got                                                    # from here on: the GPU's quantised cache
     summ = summ_before if arm == "post" else gc.gpu_build()
     check_select_and_attend(gc, summ.cpu().numpy(), out_tol=2e-2 if dtype == "bf16" else 1e-4)
+
+
+@pytest.mark.parametrize("fmt,rank,dtype", [("i8", 8, "bf16"), ("bf16", 8, "bf16"), ("i8", 5, "f32"), ("bf16", 3, "f32")])
+def test_wide_basis_formats(fmt, rank, dtype):
+    """Int8-basis and bf16-basis ("r8fp") summaries (the precision arms of the paper's ablation): select + attend on
+    oracle-built blobs, then the GPU build against the oracle's build through probe scores, stored scales and the
+    basis itself (after aligning the sign convention of each mode)."""
+    from gpu_util import check_select_and_attend
+    w = locks_synth.Workload("widefmt", [16 * 300 + 3, 16 * 80], Hq=8, Hkv=2, budget=256, rank=rank, fmt=fmt, dtype=dtype,
+                             q_scale=0.5, seed=rank)
+    gc = _gc(w)
+    o_summ = gc.oracle_summaries()
+    check_select_and_attend(gc, o_summ, out_tol=2e-2 if dtype == "bf16" else 1e-4)
+    g_summ = gc.gpu_build().cpu().numpy()
+    assert g_summ.shape == o_summ.shape
+    rng = np.random.default_rng(2)
+    bt = gc.cache.block_table[0]
+    worst = 0.0
+    for p in range(0, 300, 7):
+        for h in range(2):
+            mg = oracle.unpack(gc.fmt, rank, g_summ[bt[p], h])
+            mo = oracle.unpack(gc.fmt, rank, o_summ[bt[p], h])
+            for l in range(rank):
+                if float(np.dot(mg[1][l], mo[1][l])) < 0:
+                    mg[1][l] *= -1; mg[2][:, l] *= -1
+            assert np.abs(mg[0] - mo[0]).max() <= np.abs(mo[0]).max() / 127 + 1e-6            # centroid within one code
+            assert np.abs(mg[1] - mo[1]).max() <= 0.02                                        # basis entries (|v| <= 1)
+            q = rng.standard_normal(128)
+            worst = max(worst, abs(oracle.score(*mg, q, gc.sm) - oracle.score(*mo, q, gc.sm)))
+    assert worst <= 5e-3, worst
+    assert gc.status() == 0

@@ -738,3 +738,41 @@ def test_fake_quantisation_groups_levels_and_bounds(bits, bf16):
     oracle.fake_quantize_pages(c3, 4, page_begin=[1, 0, 0], page_end=[2, 0, 0])
     changed = {blk for blk in range(c3.num_blocks) if not np.array_equal(c3.k[blk], before[blk])}
     assert changed == {int(c3.block_table[0, 1])}
+
+
+# ------------------------------------------------------------------ int8-basis and bf16-basis formats (App. B ablation)
+
+@pytest.mark.parametrize("fmt,r", [(oracle.FMT_I8, 8), (oracle.FMT_I8, 3), (oracle.FMT_BF16, 8), (oracle.FMT_BF16, 5)])
+def test_wide_basis_formats_roundtrip_and_sizes(fmt, r):
+    """The int8-basis and the bf16-basis ("r8fp") summaries: payload arithmetic, quantiser identities against numpy,
+    and the ordering of the three basis precisions on the same page (the score error shrinks with the basis width,
+    as in the paper's rank x precision ablation)."""
+    B, d = 16, 128
+    want = (d * r + B * r + d + 2 * (r + B + 1)) if fmt == oracle.FMT_I8 else (2 * d * r + B * r + d + 2 * (B + 1))
+    assert oracle.summary_payload_bytes(fmt, r) == want
+    assert oracle.summary_stride_bytes(fmt, r) == (want + 15) // 16 * 16
+    keys = low_rank_page(6, noise=0.1, seed=41)
+    mu, V, Cc, lam, r_eff = oracle.build_page(keys, r)
+    blob = oracle.pack(fmt, mu, V, Cc)
+    mu2, V2, C2 = oracle.unpack(fmt, r, blob)
+    if fmt == oracle.FMT_I8:
+        sV = np.float16(np.abs(V).max(1) / 127).astype(np.float64)
+        codes = np.clip(np.rint(V / sV[:, None]), -127, 127)
+        assert np.array_equal(V2, codes * sV[:, None])
+    else:
+        import torch
+        assert np.array_equal(V2, torch.from_numpy(V).to(torch.float32).to(torch.bfloat16).to(torch.float64).numpy())
+    sC = np.float16(np.abs(Cc).max(1) / 127).astype(np.float64)
+    assert np.array_equal(C2, np.clip(np.rint(Cc / np.where(sC > 0, sC, 1)[:, None]), -127, 127) * sC[:, None])
+    sMu = float(np.float16(np.abs(mu).max() / 127))
+    assert np.array_equal(mu2, np.clip(np.rint(mu / sMu), -127, 127) * sMu)
+    # every byte of the payload is used, padding stays zero
+    assert not blob[want:].any()
+    if r == 8:
+        rng = np.random.default_rng(5)
+        errs = {}
+        for f in (oracle.FMT_I4, oracle.FMT_I8, oracle.FMT_BF16):
+            m = oracle.unpack(f, r, oracle.pack(f, mu, V, Cc))
+            errs[f] = np.mean([abs(oracle.score(*m, q, SM) - oracle.score(mu, V, Cc, q, SM))
+                               for q in rng.standard_normal((40, d))])
+        assert errs[oracle.FMT_I4] > errs[oracle.FMT_I8] and errs[oracle.FMT_I4] > errs[oracle.FMT_BF16]
