@@ -137,6 +137,19 @@ def test_carriers_and_nhd_layout():
     assert differed <= 1
 
 
+@pytest.mark.parametrize("Hq,Hkv,rank,qs", [(8, 2, 8, 6.0), (32, 2, 8, 6.0), (8, 2, 2, 8.0), (12, 2, 4, 8.0), (8, 2, 8, 0.0)])
+def test_extreme_logits_take_the_safe_log_sum_exp(Hq, Hkv, rank, qs):
+    """Queries scaled up until within-page logit deviations exceed what 2^x holds in fp32 without subtracting a
+    maximum (hundreds of log2 units), and a zero query: the scan's page masses must still match the oracle."""
+    from gpu_util import check_select_and_attend
+    gc = _gc(small_bf16([16 * 300 + 5, 16 * 90], Hq=Hq, Hkv=Hkv, rank=rank, budget=256, q_scale=qs, carriers=4, seed=int(qs) + Hq))
+    summ = gc.oracle_summaries()
+    shat = oracle.page_logmass(gc.cache, t2np(gc.case.q), rank, gc.fmt, summ, gc.sm)
+    if qs > 0:
+        assert np.nanmax(shat) - np.nanmedian(shat) > 100          # logits far beyond the fp32 exponent range in log2
+    check_select_and_attend(gc, summ, out_tol=2e-2, mass_tol=1e-3 * max(1.0, float(np.nanmax(np.abs(shat))) / 50))
+
+
 def test_tail_slots_are_never_read_as_data():
     """Cache slots past the sequence end hold NaN: outputs must not change."""
     from gpu_util import check_select_and_attend
