@@ -124,6 +124,16 @@ int locks_destroy(locks_ctx *ctx);
 int locks_build_summaries(locks_ctx *ctx, const locks_kv *kv, int batch, const int32_t *page_begin,
                           const int32_t *page_end, void *summaries, locks_stream stream);
 
+/* The same build for several layers of a model in ONE launch (Sec. 4 "Build": the pass at the prefill-decode
+ * boundary summarises the whole prompt, every layer of it).  All layers share kv's geometry (strides, block table,
+ * lengths, page ranges); layer l reads its keys from k_layers[l] (kv->k is ignored) and writes summaries_layers[l].
+ * k_layers and summaries_layers are DEVICE arrays of num_layers device pointers (the caller's; read by the kernel,
+ * so they must stay valid until the launch has run); 1 <= num_layers, batch * num_layers <= 65535.  Each summary is
+ * byte-identical to what locks_build_summaries writes for that layer alone. */
+int locks_build_summaries_layers(locks_ctx *ctx, const locks_kv *kv, const void *const *k_layers,
+                                 void *const *summaries_layers, int num_layers, int batch, const int32_t *page_begin,
+                                 const int32_t *page_end, locks_stream stream);
+
 /* ---- Page-sharded decode -------------------------------------------------------------------------------------
  * One long request (the GLM-shaped 128K..1M case) whose pages are dealt to several GPUs in page order.  The path
  * itself has no exchange step (every (request, KV head) owns its pages); sharding ONE sequence adds three small

@@ -20,7 +20,8 @@ SYMBOLS = ["locks_summary_bytes", "locks_workspace_bytes", "locks_create", "lock
            "locks_set_scan_partition", "locks_selftest_wait_timeout", "locks_last_scan_partition",
            "locks_host_cache_clear", "locks_select_exact", "locks_selection_quality",
            "locks_select_rival", "locks_fake_quantize_pages", "locks_scan",
-           "locks_select_scored", "locks_merge_selection", "locks_merge_attention"]
+           "locks_select_scored", "locks_merge_selection", "locks_merge_attention",
+           "locks_build_summaries_layers"]
 
 
 PARTITION_AUTO, PARTITION_STRIDED, PARTITION_BALANCED = 0, 1, 2   # LOCKS_PARTITION_* of include/locks.h
@@ -69,6 +70,8 @@ def lib():
         L.locks_destroy.argtypes = [vp]
         L.locks_build_summaries.argtypes = [vp, C.POINTER(KV), C.c_int, i32p, i32p, vp, vp]
         L.locks_select.argtypes = [vp, vp, vp, C.POINTER(KV), C.c_int, i32p, i32p, vp, vp, vp]
+        L.locks_build_summaries_layers.argtypes = [vp, C.POINTER(KV), vp, vp, C.c_int, C.c_int, i32p, i32p, vp]
+        L.locks_build_summaries_layers.restype = C.c_int
         L.locks_sparse_attend.argtypes = [vp, vp, C.POINTER(KV), C.c_int, i32p, i32p, vp, vp, vp]
         L.locks_decode_step.argtypes = [vp, vp, vp, vp, C.POINTER(KV), vp, C.c_int, vp, i32p, i32p, vp]
         L.locks_decode_step_host.argtypes = [vp, vp, vp, vp, C.POINTER(KV), vp, C.c_int, vp, i32p, i32p, vp]
@@ -211,6 +214,20 @@ class Context:
         s = kv.struct()
         _check(lib().locks_build_summaries(self.handle, C.byref(s), batch, _ptr(page_begin), _ptr(page_end),
                                            _ptr(summaries), _stream(stream)), "locks_build_summaries")
+
+    def locks_build_summaries_layers(self, kv: KVView, k_layers, summaries_layers, batch, page_begin=None, page_end=None,
+                                     stream=None):
+        """k_layers / summaries_layers: lists of tensors (one per layer).  Returns the two device pointer arrays, which
+        the caller keeps alive until the launch has run."""
+        import torch
+        dev = summaries_layers[0].device
+        kp = torch.tensor([t.data_ptr() for t in k_layers], dtype=torch.int64, device=dev)
+        sp = torch.tensor([t.data_ptr() for t in summaries_layers], dtype=torch.int64, device=dev)
+        s = kv.struct()
+        _check(lib().locks_build_summaries_layers(self.handle, C.byref(s), _ptr(kp), _ptr(sp), len(k_layers), batch,
+                                                  _ptr(page_begin), _ptr(page_end), _stream(stream)),
+               "locks_build_summaries_layers")
+        return kp, sp
 
     def locks_fake_quantize_pages(self, kv: KVView, batch, bits, page_begin=None, page_end=None, stream=None):
         s = kv.struct()

@@ -277,6 +277,22 @@ int locks_build_summaries(locks_ctx *ctx, const locks_kv *kv, int batch, const i
   return locks_launch_build(ctx, kv, batch, page_begin, page_end, 0, summaries, nullptr, nullptr, (cudaStream_t)stream);
 }
 
+int locks_build_summaries_layers(locks_ctx *ctx, const locks_kv *kv, const void *const *k_layers,
+                                 void *const *summaries_layers, int num_layers, int batch, const int32_t *page_begin,
+                                 const int32_t *page_end, locks_stream stream) {
+  if (!kv || !k_layers || !summaries_layers || num_layers < 1) return LOCKS_ERR_INVALID_ARG;
+  locks_kv kv0 = *kv;
+  // kv->k and kv->v are not read by this call: a placeholder passes the common checks
+  kv0.k = reinterpret_cast<void *>(uintptr_t(256));
+  kv0.v = kv0.k;
+  int rc = check_common(ctx, &kv0, batch);
+  if (rc != LOCKS_OK) return rc;
+  if ((int64_t)batch * num_layers > 65535 || ((page_begin == nullptr) != (page_end == nullptr))) return LOCKS_ERR_INVALID_ARG;
+  ctx->last_launches = 0;
+  return locks_launch_build(ctx, &kv0, batch, page_begin, page_end, 0, nullptr, nullptr, nullptr, (cudaStream_t)stream,
+                            k_layers, summaries_layers, num_layers);
+}
+
 // ---- page-sharded decode: one long request whose pages are dealt to several GPUs (three small exchanges) ------
 
 int locks_scan(locks_ctx *ctx, const void *q, const void *summaries, const locks_kv *kv, int batch, float *page_logmass,

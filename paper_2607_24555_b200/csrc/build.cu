@@ -32,6 +32,9 @@ struct BuildParams {
   // (the append runs in another kernel at the same time); append_pos[b] = its position or -1
   const void *k_new;
   const int32_t *append_pos;
+  // bulk build of several layers in one launch: per-layer key caches and summary buffers (device arrays), or null
+  const void *const *k_layers;
+  void *const *summ_layers;
 };
 
 #ifndef LOCKS_BUILD_COS_TOL
@@ -412,7 +415,7 @@ __global__ void __launch_bounds__(kBuildWarps * 32, kBuildCtasPerSm) build_kerne
         }
       }
     } else {
-      it_b = blockIdx.z; it_h = blockIdx.y;
+      it_b = blockIdx.z % p.batch; it_h = blockIdx.y;
       const int complete = p.seq_lens[it_b] / LOCKS_B;
       const int p0 = p.page_begin ? p.page_begin[it_b] : 0;
       const int p1 = min(p.page_end ? p.page_end[it_b] : complete, complete);
@@ -431,6 +434,9 @@ __global__ void __launch_bounds__(kBuildWarps * 32, kBuildCtasPerSm) build_kerne
   const uint32_t live = __ballot_sync(0xffffffffu, it_block >= 0);
   if (!live) return;
 
+  const int layer = STEP ? 0 : blockIdx.z / p.batch;
+  const void *kbase = p.k_layers ? p.k_layers[layer] : p.k;
+  uint8_t *sbase = p.summ_layers ? reinterpret_cast<uint8_t *>(p.summ_layers[layer]) : p.summ;
   uint8_t *scratch = smem_raw + warp * kBuildSmemPerWarp;                        // D half-tiles; phase 3: the blob
   float *mat = reinterpret_cast<float *>(scratch + kBuildScratch);              // [8][16][16] Gram; then [8][16][8] pairs (u, u) of U_r
   float *kn_s = mat + kBuildItems * LOCKS_B * LOCKS_B;                          // [8] squared norm of the page's keys
@@ -442,7 +448,7 @@ __global__ void __launch_bounds__(kBuildWarps * 32, kBuildCtasPerSm) build_kerne
   auto load_item = [&](int s, float (&v)[LOCKS_B][4]) {
     const int b = __shfl_sync(0xffffffffu, it_b, s), h = __shfl_sync(0xffffffffu, it_h, s);
     const int block = __shfl_sync(0xffffffffu, it_block, s), nw = __shfl_sync(0xffffffffu, it_new, s);
-    const T *K = reinterpret_cast<const T *>(p.k) + ((int64_t)block * p.sb + (int64_t)h * p.sh) + 4 * lane;
+    const T *K = reinterpret_cast<const T *>(kbase) + ((int64_t)block * p.sb + (int64_t)h * p.sh) + 4 * lane;
     const T *Knew = reinterpret_cast<const T *>(p.k_new) + ((int64_t)b * p.Hkv + h) * LOCKS_D + 4 * lane;
 #pragma unroll
     for (int i = 0; i < LOCKS_B; ++i) {
@@ -584,7 +590,7 @@ __global__ void __launch_bounds__(kBuildWarps * 32, kBuildCtasPerSm) build_kerne
       for (int e = lane; e < i4_stride(8) / 4; e += 32) reinterpret_cast<uint32_t *>(blob)[e] = 0u;
       __syncwarp();
     }
-    uint8_t *gout = p.summ + ((int64_t)block * p.Hkv + h) * p.S;
+    uint8_t *gout = sbase + ((int64_t)block * p.Hkv + h) * p.S;
     float *fout = reinterpret_cast<float *>(gout);
     uint32_t sign_bits = 0u;   // bit l: mode l was flipped
 #pragma unroll 1
@@ -725,13 +731,14 @@ __global__ void __launch_bounds__(kBuildWarps * 32, kBuildCtasPerSm) build_kerne
 
 int locks_launch_build(locks_ctx *c, const locks_kv *kv, int batch, const int32_t *pb, const int32_t *pe,
                        int just_filled, void *summaries, const void *k_new, const int32_t *append_pos,
-                       cudaStream_t st) {
+                       cudaStream_t st, const void *const *k_layers, void *const *summ_layers, int num_layers) {
   BuildParams p;
   p.k = kv->k; p.sb = kv->stride_block; p.sh = kv->stride_head; p.st = kv->stride_token;
   p.block_table = kv->block_table; p.seq_lens = kv->seq_lens; p.page_begin = pb; p.page_end = pe;
   p.summ = reinterpret_cast<uint8_t *>(summaries); p.status = c->status;
   p.batch = batch; p.Hkv = c->cfg.num_kv_heads; p.Pmax = c->Pmax; p.num_blocks = kv->num_blocks;
   p.r = c->cfg.rank; p.S = c->S; p.just_filled = just_filled;
+  p.k_layers = just_filled ? nullptr : k_layers; p.summ_layers = just_filled ? nullptr : summ_layers;
   p.k_new = just_filled ? k_new : nullptr; p.append_pos = just_filled ? append_pos : nullptr;
   p.hint = nullptr; p.kpages = c->k; p.hint_wpp = 1; p.hint_rounds = 1; p.hint_W = 1;
   if (just_filled && c->hint_dev && c->cfg.summary_fmt == LOCKS_FMT_I4 && c->cfg.q_dtype == LOCKS_BF16) {
@@ -740,7 +747,7 @@ int locks_launch_build(locks_ctx *c, const locks_kv *kv, int batch, const int32_
   }
   constexpr int kPer = kBuildWarps * kBuildItems;   // items per CTA (bulk)
   dim3 grid = just_filled ? dim3((batch * p.Hkv + kBuildWarps - 1) / kBuildWarps)
-                          : dim3((c->Pmax + kPer - 1) / kPer, p.Hkv, batch);
+                          : dim3((c->Pmax + kPer - 1) / kPer, p.Hkv, batch * (k_layers ? num_layers : 1));
   const bool bf = c->cfg.kv_dtype == LOCKS_BF16;
   const int smem = kBuildWarps * kBuildSmemPerWarp;
 #define LOCKS_BUILD_CASE(F_)                                                                                                \

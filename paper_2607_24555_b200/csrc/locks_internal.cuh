@@ -148,7 +148,8 @@ int locks_launch_attend(locks_ctx *c, const void *q, const locks_kv *kv, int bat
                         const int32_t *cnt, void *out, float *lse, cudaStream_t st);
 int locks_launch_build(locks_ctx *c, const locks_kv *kv, int batch, const int32_t *pb, const int32_t *pe,
                        int just_filled, void *summaries, const void *k_new, const int32_t *append_pos,
-                       cudaStream_t st);
+                       cudaStream_t st, const void *const *k_layers = nullptr, void *const *summ_layers = nullptr,
+                       int num_layers = 1);
 
 // envelope = 0: exact page log-mass; 1: the min/max envelope bound of the page's largest logit
 int locks_launch_exact_scan(locks_ctx *c, const void *q, const locks_kv *kv, int batch, float *shat, int envelope,

@@ -371,6 +371,72 @@ def test_gpu_i4_build_decoupled_parity(rank):
     assert gc.status() == 0
 
 
+def test_multi_layer_build_in_one_launch():
+    """locks_build_summaries_layers: three layers with different keys (same block table and lengths) in one launch.
+    Every layer's blobs equal, byte for byte, what the single-layer call writes for that layer, and one layer's codes
+    are checked against the oracle's build of that layer's keys (sign-aligned code agreement, as in the decoupled
+    test); pages outside the requested range and the blocks of other layers are not touched."""
+    gc = _gc(small_bf16([16 * 70 + 3, 16 * 33], Hq=8, Hkv=2, seed=91))
+    w = gc.w
+    g = torch.Generator(device="cuda:0").manual_seed(5)
+    k_layers = [gc.case.k] + [(gc.case.k.float() * s + torch.randn(gc.case.k.shape, generator=g, device="cuda:0") * 0.5)
+                              .to(gc.case.k.dtype) for s in (0.5, -1.25)]
+    singles = []
+    from paper_2607_24555_b200.binding import KVView
+    for kl in k_layers:
+        kv = KVView(kl, gc.case.v, gc.case.strides, gc.case.num_blocks, gc.case.block_table, gc.case.seq_lens)
+        summ = gc.ctx.new_summaries(gc.case.num_blocks)
+        summ.fill_(0x5A)
+        gc.ctx.locks_build_summaries(kv, w.n, summ)
+        singles.append(summ)
+    multi = [gc.ctx.new_summaries(gc.case.num_blocks) for _ in k_layers]
+    for m in multi:
+        m.fill_(0x5A)
+    keep = gc.ctx.locks_build_summaries_layers(gc.kv, k_layers, multi, w.n)
+    torch.cuda.synchronize()
+    assert keep is not None and gc.status() == 0
+    for l in range(len(k_layers)):
+        assert torch.equal(multi[l], singles[l]), l
+    # layer 2 against the oracle's build of the same keys
+    import copy
+    from common import oracle_cache
+    case2 = copy.copy(gc.case)
+    case2.k = k_layers[2]
+    o_summ = oracle.build_summaries(oracle_cache(case2), w.rank, gc.fmt)
+    g_summ = multi[2].cpu().numpy()
+    tot = diff = 0
+    for b in range(w.n):
+        bt = gc.cache.block_table[b]
+        for p in range(w.seq_lens[b] // 16):
+            for h in range(w.Hkv):
+                gV, gC, gMu, _, _, _ = oracle.unpack_codes(w.rank, g_summ[bt[p], h])
+                oV, oC, oMu, _, _, _ = oracle.unpack_codes(w.rank, o_summ[bt[p], h])
+                for l in range(w.rank):
+                    if int(np.dot(gV[l], oV[l])) < 0:
+                        gV[l] = -gV[l]; gC[:, l] = -gC[:, l]
+                for a_, b_ in ((gV, oV), (gC, oC), (gMu, oMu)):
+                    d = np.abs(a_ - b_)
+                    assert d.max() <= 1
+                    tot += d.size; diff += int((d > 0).sum())
+    assert diff / tot <= 1e-3, diff / tot
+    # a page range: only pages 2..4 of every request are rebuilt
+    pb = torch.full((w.n,), 2, dtype=torch.int32, device="cuda:0")
+    pe = torch.full((w.n,), 5, dtype=torch.int32, device="cuda:0")
+    part = [torch.full_like(m, 0x5A) for m in multi]
+    keep2 = gc.ctx.locks_build_summaries_layers(gc.kv, k_layers, part, w.n, pb, pe)
+    torch.cuda.synchronize()
+    assert keep2 is not None
+    bt_all = gc.case.block_table.cpu().numpy()
+    touched = sorted({int(bt_all[b, p]) for b in range(w.n) for p in range(2, 5)})
+    for l in range(len(k_layers)):
+        pl, ml = part[l].cpu().numpy(), multi[l].cpu().numpy()
+        for blk in range(gc.case.num_blocks):
+            if blk in touched:
+                assert np.array_equal(pl[blk], ml[blk]), (l, blk)
+            else:
+                assert (pl[blk] == 0x5A).all(), (l, blk)
+
+
 def test_decode_step_matches_stepwise_oracle():
     """locks_decode_step with appends across page boundaries; summaries of freshly filled pages
     are built on the device and handed to the oracle (identical bytes) for the next steps."""
