@@ -66,7 +66,7 @@ typedef void *locks_stream; /* cudaStream_t */
 
 typedef struct {
   int32_t head_dim;          /* d; 128                                                        */
-  int32_t page_size;         /* B; 16                                                         */
+  int32_t page_size;         /* B; 16, or 32 | 64 (App. D "Page size": F32 / I8 / BF16 formats) */
   int32_t num_q_heads;       /* Hq                                                            */
   int32_t num_kv_heads;      /* Hkv, Hq % Hkv == 0, G = Hq/Hkv <= 16                          */
   int32_t rank;              /* r: I4 format 2|4|8, other formats 1..16                       */
@@ -110,8 +110,11 @@ size_t locks_workspace_bytes(const locks_config *cfg);
 /* Validate the configuration, record it and the workspace pointer, zero the status word (one
  * small async memset on the default stream followed by a synchronise).  The context is a small
  * host object; *out must be released with locks_destroy().  Errors: INVALID_ARG (bad field, NULL),
- * UNSUPPORTED (shape the kernels do not cover: d != 128, B != 16, G > 16, mixed dtypes, I4 rank
- * not in {2,4,8}), WORKSPACE (ws_bytes too small or misaligned). */
+ * UNSUPPORTED (shape the kernels do not cover: d != 128, B not in {16, 32, 64}, B != 16 with the I4 format (its
+ * blob is laid out for 16 tokens), G > 16, mixed dtypes, I4 rank not in {2,4,8}), WORKSPACE (ws_bytes too small or
+ * misaligned).  Pages of 32 and 64 tokens run build, select, attend and the decode step on plain fp32 kernels (no
+ * tensor-core path); the diagnostics, the KV fake quantiser, the page-sharded calls, the multi-layer build and the
+ * allocation-free attention entry point return UNSUPPORTED for them. */
 int locks_create(const locks_config *cfg, void *workspace, size_t ws_bytes, locks_ctx **out);
 int locks_destroy(locks_ctx *ctx);
 

@@ -20,7 +20,10 @@ int validate(const locks_config *c) {
   if (c->combine < LOCKS_COMBINE_SHARE_AVG || c->combine > LOCKS_COMBINE_GROUP_MASS) return LOCKS_ERR_INVALID_ARG;
   if ((c->kv_dtype != LOCKS_F32 && c->kv_dtype != LOCKS_BF16) || (c->q_dtype != LOCKS_F32 && c->q_dtype != LOCKS_BF16))
     return LOCKS_ERR_INVALID_ARG;
-  if (c->head_dim != LOCKS_D || c->page_size != LOCKS_B) return LOCKS_ERR_UNSUPPORTED;
+  if (c->head_dim != LOCKS_D) return LOCKS_ERR_UNSUPPORTED;
+  // pages of 32 and 64 tokens (App. D "Page size") run on the plain fp32 kernels with the row-major summary formats
+  if (c->page_size != LOCKS_B && !((c->page_size == 32 || c->page_size == 64) && c->summary_fmt != LOCKS_FMT_I4))
+    return LOCKS_ERR_UNSUPPORTED;
   if (c->num_q_heads / c->num_kv_heads > 16) return LOCKS_ERR_UNSUPPORTED;
   if (c->kv_dtype != c->q_dtype) return LOCKS_ERR_UNSUPPORTED;
   if (c->summary_fmt == LOCKS_FMT_I4 && c->rank != 2 && c->rank != 4 && c->rank != 8) return LOCKS_ERR_UNSUPPORTED;
@@ -41,7 +44,7 @@ Layout make_layout(const locks_config *c) {
   Layout L;
   L.G = c->num_q_heads / c->num_kv_heads;
   L.k = (c->budget_tokens + c->page_size - 1) / c->page_size;
-  L.S = locks_fmt_stride(c->summary_fmt, c->rank);
+  L.S = locks_fmt_stride(c->summary_fmt, c->rank, c->page_size);
   L.max_groups = (c->max_pages_per_seq + LOCKS_GROUP - 1) / LOCKS_GROUP;
   // Pages per thread of a selector CTA (1 .. 16; a CTA ranks sel_ept * 512 pages).  With many (request,
   // KV head) problems and a context of up to 8192 pages, one CTA ranks a whole problem.  Otherwise a problem is
@@ -174,6 +177,7 @@ int locks_create(const locks_config *cfg, void *workspace, size_t ws_bytes, lock
     (void)cudaGetLastError();   // without the word the partition simply stays strided
   }
   c->G = L.G; c->k = L.k; c->S = L.S; c->Pmax = cfg->max_pages_per_seq; c->max_groups = L.max_groups;
+  c->B = cfg->page_size;
   c->sel_ept = L.sel_ept; c->sel_chunks = L.sel_chunks; c->sel_kc = L.sel_kc;
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess ||
@@ -280,6 +284,7 @@ int locks_build_summaries(locks_ctx *ctx, const locks_kv *kv, int batch, const i
 int locks_build_summaries_layers(locks_ctx *ctx, const locks_kv *kv, const void *const *k_layers,
                                  void *const *summaries_layers, int num_layers, int batch, const int32_t *page_begin,
                                  const int32_t *page_end, locks_stream stream) {
+  if (ctx && ctx->B != LOCKS_B) return LOCKS_ERR_UNSUPPORTED;   // 16-token pages only
   if (!kv || !k_layers || !summaries_layers || num_layers < 1) return LOCKS_ERR_INVALID_ARG;
   locks_kv kv0 = *kv;
   // kv->k and kv->v are not read by this call: a placeholder passes the common checks
@@ -297,6 +302,7 @@ int locks_build_summaries_layers(locks_ctx *ctx, const locks_kv *kv, const void 
 
 int locks_scan(locks_ctx *ctx, const void *q, const void *summaries, const locks_kv *kv, int batch, float *page_logmass,
                float *head_logz, locks_stream stream) {
+  if (ctx && ctx->B != LOCKS_B) return LOCKS_ERR_UNSUPPORTED;   // 16-token pages only
   int rc = check_common(ctx, kv, batch);
   if (rc != LOCKS_OK) return rc;
   if (!q || !summaries || !head_logz || ((uintptr_t)summaries % 16) || ((uintptr_t)q % 16)) return LOCKS_ERR_INVALID_ARG;
@@ -309,6 +315,7 @@ int locks_scan(locks_ctx *ctx, const void *q, const void *summaries, const locks
 int locks_select_scored(locks_ctx *ctx, const float *page_logmass, const float *head_logz_parts, int nparts,
                         const locks_kv *kv, int batch, int32_t *page_ids, int32_t *page_count, float *page_logshare,
                         locks_stream stream) {
+  if (ctx && ctx->B != LOCKS_B) return LOCKS_ERR_UNSUPPORTED;   // 16-token pages only
   int rc = check_common(ctx, kv, batch);
   if (rc != LOCKS_OK) return rc;
   if (!head_logz_parts || !page_ids || !page_count || nparts < 1) return LOCKS_ERR_INVALID_ARG;
@@ -321,6 +328,7 @@ int locks_select_scored(locks_ctx *ctx, const float *page_logmass, const float *
 
 int locks_merge_selection(locks_ctx *ctx, const float *cand_key, const int32_t *cand_page, int nparts, int batch,
                           int32_t *page_ids, int32_t *page_count, locks_stream stream) {
+  if (ctx && ctx->B != LOCKS_B) return LOCKS_ERR_UNSUPPORTED;   // 16-token pages only
   if (!ctx || !cand_key || !cand_page || !page_ids || !page_count || nparts < 1 || batch < 1 || batch > ctx->cfg.max_batch)
     return LOCKS_ERR_INVALID_ARG;
   ctx->last_launches = 0;
@@ -337,6 +345,7 @@ int locks_merge_attention(locks_ctx *ctx, const void *part_out, const float *par
 
 int locks_fake_quantize_pages(locks_ctx *ctx, const locks_kv *kv, int batch, const int32_t *page_begin,
                               const int32_t *page_end, int bits, locks_stream stream) {
+  if (ctx && ctx->B != LOCKS_B) return LOCKS_ERR_UNSUPPORTED;   // 16-token pages only
   int rc = check_common(ctx, kv, batch);
   if (rc != LOCKS_OK) return rc;
   if (bits < 1 || bits > 8 || ((page_begin == nullptr) != (page_end == nullptr))) return LOCKS_ERR_INVALID_ARG;
@@ -360,6 +369,7 @@ int locks_select(locks_ctx *ctx, const void *q, const void *summaries, const loc
 
 int locks_select_exact(locks_ctx *ctx, const void *q, const locks_kv *kv, int batch, int32_t *page_ids,
                        int32_t *page_count, float *page_logmass, float *page_logshare, locks_stream stream) {
+  if (ctx && ctx->B != LOCKS_B) return LOCKS_ERR_UNSUPPORTED;   // 16-token pages only
   int rc = check_common(ctx, kv, batch);
   if (rc != LOCKS_OK) return rc;
   if (!q || !page_ids || !page_count || ((uintptr_t)q % 16)) return LOCKS_ERR_INVALID_ARG;
@@ -373,6 +383,7 @@ int locks_select_exact(locks_ctx *ctx, const void *q, const locks_kv *kv, int ba
 int locks_select_rival(locks_ctx *ctx, int scorer, const void *q, const void *summaries, const locks_kv *kv, int batch,
                        int32_t *page_ids, int32_t *page_count, float *page_score, float *page_logshare,
                        locks_stream stream) {
+  if (ctx && ctx->B != LOCKS_B) return LOCKS_ERR_UNSUPPORTED;   // 16-token pages only
   int rc = check_common(ctx, kv, batch);
   if (rc != LOCKS_OK) return rc;
   if (!q || !page_ids || !page_count || ((uintptr_t)q % 16)) return LOCKS_ERR_INVALID_ARG;
@@ -397,6 +408,7 @@ int locks_selection_quality(locks_ctx *ctx, const float *exact_logmass, const lo
                             const int32_t *page_ids, const int32_t *page_count, const int32_t *ref_ids,
                             const int32_t *ref_count, const int32_t *marked_pages, int n_marked, float *quality,
                             locks_stream stream) {
+  if (ctx && ctx->B != LOCKS_B) return LOCKS_ERR_UNSUPPORTED;   // 16-token pages only
   int rc = check_common(ctx, kv, batch);
   if (rc != LOCKS_OK) return rc;
   if (!exact_logmass || !page_ids || !page_count || !ref_ids || !ref_count || !quality || n_marked < 0 ||

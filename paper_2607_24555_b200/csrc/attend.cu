@@ -28,6 +28,7 @@ struct AttParams {
   int32_t *status;
   int32_t *done;   // [batch*Hkv] split-arrival counters (zero between launches)
   int batch, Hq, Hkv, G, Pmax, kbud, num_blocks, splits, pages_per_cta;
+  int B;             // tokens per page (the bf16 kernels: 16 only)
   int fused_merge;   // 1: the last CTA of a problem merges its splits; 0: a separate merge kernel follows
   int cluster;       // 1: the splits of a problem form one thread-block cluster and merge through its shared memory
   float sm_scale;
@@ -51,7 +52,7 @@ __device__ __forceinline__ bool resolve_page(const AttParams &p, int b, int64_t 
   if (page < 0 || page >= p.Pmax) { set_status(p.status, LOCKS_ERR_BAD_BLOCK); return false; }
   block = p.block_table[(int64_t)b * p.Pmax + page];
   if (block < 0 || block >= p.num_blocks) { set_status(p.status, LOCKS_ERR_BAD_BLOCK); return false; }
-  ntok = min(LOCKS_B, T - page * LOCKS_B);
+  ntok = min(p.B, T - page * p.B);
   return ntok > 0;
 }
 
@@ -442,7 +443,7 @@ __global__ void __launch_bounds__(128) attend_generic_kernel(AttParams p) {
   pdl_wait();
   const int64_t prob = (int64_t)b * p.Hkv + h;
   const int Tn = p.seq_lens[b];
-  const int P = (Tn + LOCKS_B - 1) / LOCKS_B;
+  const int P = (Tn + p.B - 1) / p.B;
   int npages = p.ids ? p.cnt[prob] : P;
   if (p.ids && (npages < 0 || npages > p.kbud)) {
     if (threadIdx.x == 0) set_status(p.status, LOCKS_ERR_BAD_BLOCK);
@@ -592,7 +593,7 @@ int locks_launch_attend(locks_ctx *c, const void *q, const locks_kv *kv, int bat
   p.block_table = kv->block_table; p.seq_lens = kv->seq_lens; p.ids = ids; p.cnt = cnt;
   p.part_o = c->att_o; p.part_lse = c->att_lse; p.out = out; p.lse = lse; p.status = c->status;
   p.batch = batch; p.Hq = c->cfg.num_q_heads; p.Hkv = c->cfg.num_kv_heads; p.G = c->G; p.Pmax = c->Pmax;
-  p.kbud = c->k; p.num_blocks = kv->num_blocks; p.sm_scale = c->cfg.sm_scale;
+  p.kbud = c->k; p.num_blocks = kv->num_blocks; p.sm_scale = c->cfg.sm_scale; p.B = c->B;
   const bool dense = ids == nullptr;
   // one wave: as many splits per problem as resident CTA slots allow, at least one page per warp
   const int npages = dense ? c->Pmax : c->k;
@@ -635,7 +636,7 @@ int locks_launch_attend(locks_ctx *c, const void *q, const locks_kv *kv, int bat
     }
     (void)cudaGetLastError();   // a refused probe is not an error of this call
   }
-  if (c->cfg.kv_dtype == LOCKS_BF16 && splits >= 2 && c->att_cluster_max >= 2) {
+  if (c->cfg.kv_dtype == LOCKS_BF16 && c->B == LOCKS_B && splits >= 2 && c->att_cluster_max >= 2) {
     int cs = 2;
     while (cs * 2 <= splits && cs * 2 <= c->att_cluster_max) cs *= 2;
     const int ppc = (npages + cs - 1) / cs;
@@ -646,7 +647,7 @@ int locks_launch_attend(locks_ctx *c, const void *q, const locks_kv *kv, int bat
       p.fused_merge = 1;   // no merge launch follows
     }
   }
-  const bool bf = c->cfg.kv_dtype == LOCKS_BF16;
+  const bool bf = c->cfg.kv_dtype == LOCKS_BF16 && c->B == LOCKS_B;   // tensor-core kernel: bf16 cache, 16-token pages
   if (bf) {
     if (locks_attrs_needed(LOCKS_ATTR_ATTEND)) {
       cudaFuncSetAttribute(attend_bf16_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kAttSmem);
@@ -678,12 +679,13 @@ int locks_launch_attend(locks_ctx *c, const void *q, const locks_kv *kv, int bat
     }
   } else {
     dim3 grid(p.splits, p.Hq, batch);
-    locks_launch_pdl(attend_generic_kernel<float>, grid, dim3(128), 0, st, p);
+    if (c->cfg.kv_dtype == LOCKS_BF16) locks_launch_pdl(attend_generic_kernel<__nv_bfloat16>, grid, dim3(128), 0, st, p);
+    else locks_launch_pdl(attend_generic_kernel<float>, grid, dim3(128), 0, st, p);
   }
   int rc = locks_check_launch(c);
   if (rc != LOCKS_OK || p.splits == 1 || (bf && p.fused_merge)) return rc;
   dim3 mg(p.Hq, batch);
-  if (bf) locks_launch_pdl(attend_merge_kernel<__nv_bfloat16>, mg, dim3(128), 0, st, (const float *)c->att_o,
+  if (c->cfg.kv_dtype == LOCKS_BF16) locks_launch_pdl(attend_merge_kernel<__nv_bfloat16>, mg, dim3(128), 0, st, (const float *)c->att_o,
                            (const float *)c->att_lse, p.splits, reinterpret_cast<__nv_bfloat16 *>(out), lse, p.Hq);
   else locks_launch_pdl(attend_merge_kernel<float>, mg, dim3(128), 0, st, (const float *)c->att_o,
                         (const float *)c->att_lse, p.splits, reinterpret_cast<float *>(out), lse, p.Hq);
@@ -763,7 +765,7 @@ extern "C" int locks_sparse_attend_noalloc(const locks_config *cfg, const void *
   p.status = reinterpret_cast<int32_t *>(nd.scratch + kNoAllocO + kNoAllocLse + kNoAllocDone);
   p.out = out; p.lse = lse;
   p.batch = batch; p.Hq = cfg->num_q_heads; p.Hkv = cfg->num_kv_heads; p.G = G; p.Pmax = cfg->max_pages_per_seq;
-  p.kbud = (cfg->budget_tokens + LOCKS_B - 1) / LOCKS_B; p.num_blocks = kv->num_blocks; p.sm_scale = cfg->sm_scale;
+  p.kbud = (cfg->budget_tokens + LOCKS_B - 1) / LOCKS_B; p.num_blocks = kv->num_blocks; p.sm_scale = cfg->sm_scale; p.B = LOCKS_B;
   const int npages = page_ids ? p.kbud : p.Pmax;
   int splits = nd.num_sms * LOCKS_ATT_CTAS_PER_SM / (batch * p.Hkv);
   const int most = (npages + LOCKS_ATT_WARPS - 1) / LOCKS_ATT_WARPS;

@@ -727,6 +727,248 @@ __global__ void __launch_bounds__(kBuildWarps * 32, kBuildCtasPerSm) build_kerne
   }
 }
 
+// ------------------------------------------------------------------------------------------------
+// Pages of 32 and 64 tokens (App. D "Page size"): one warp per (page, KV head), everything in fp32 from shared
+// memory, the row-major summary formats only.  The same method as above (centre, Gram, one-sided Jacobi by
+// odd-even transposition, rank, project, quantise), written for brevity rather than speed: lane m rotates the
+// column pair m of a step.
+// ------------------------------------------------------------------------------------------------
+constexpr int kWideDStride = LOCKS_D + 4;   // floats per staged key row (16-byte aligned rows, no bank conflicts)
+__host__ __device__ constexpr int build_wide_smem(int B) {
+  return (B * kWideDStride + B * (B + 1) + 2 * B + 32) * 4;   // keys, W (column-major, padded), norms, order, misc
+}
+
+template <typename T, int FMT>
+__global__ void __launch_bounds__(32) build_wide_kernel(BuildParams p, int B, int step) {
+  extern __shared__ __align__(16) uint8_t smem_raw[];
+  const int lane = threadIdx.x;
+  int b, h, page, last_from_new = 0;
+  if (step) {
+    const int prob = blockIdx.x;
+    if (prob >= p.batch * p.Hkv) return;
+    b = prob / p.Hkv; h = prob - b * p.Hkv;
+    const int Tb = p.seq_lens[b];
+    if (Tb <= 0 || (Tb % B) != 0) return;
+    page = Tb / B - 1;
+    last_from_new = (p.k_new && p.append_pos && p.append_pos[b] == Tb - 1) ? 1 : 0;
+  } else {
+    b = blockIdx.z; h = blockIdx.y;
+    const int complete = p.seq_lens[b] / B;
+    const int p0 = p.page_begin ? p.page_begin[b] : 0;
+    const int p1 = min(p.page_end ? p.page_end[b] : complete, complete);
+    page = p0 + blockIdx.x;
+    if (page < 0 || page >= p1) return;
+  }
+  if (page >= p.Pmax) return;
+  const int block = p.block_table[(int64_t)b * p.Pmax + page];
+  if (block < 0 || block >= p.num_blocks) {
+    if (lane == 0) set_status(p.status, LOCKS_ERR_BAD_BLOCK);
+    return;
+  }
+  float *Ds = reinterpret_cast<float *>(smem_raw);   // [B][kWideDStride] deviations
+  float *W = Ds + B * kWideDStride;                  // [B columns][B + 1]
+  float *nr = W + B * (B + 1);                       // [B] squared column norms
+  int *order = reinterpret_cast<int *>(nr + B);      // [B] column of rank l
+  const int WS = B + 1, r = p.r;
+  // ---- keys, centroid, deviations
+  float mu[4] = {0.f, 0.f, 0.f, 0.f}, knorm2 = 0.f;
+  {
+    const T *K = reinterpret_cast<const T *>(p.k) + ((int64_t)block * p.sb + (int64_t)h * p.sh) + 4 * lane;
+    const T *Knew = reinterpret_cast<const T *>(p.k_new) + ((int64_t)b * p.Hkv + h) * LOCKS_D + 4 * lane;
+    for (int i = 0; i < B; ++i) {
+      const T *src = (i == B - 1 && last_from_new) ? Knew : K + (int64_t)i * p.st;
+      float v[4];
+#pragma unroll
+      for (int c = 0; c < 4; ++c) v[c] = ldf<T>(src, c);
+#pragma unroll
+      for (int c = 0; c < 4; ++c) { mu[c] += v[c]; knorm2 = fmaf(v[c], v[c], knorm2); }
+      *reinterpret_cast<float4 *>(Ds + i * kWideDStride + 4 * lane) = make_float4(v[0], v[1], v[2], v[3]);
+    }
+    knorm2 = warp_sum(knorm2);
+#pragma unroll
+    for (int c = 0; c < 4; ++c) mu[c] /= (float)B;
+    for (int i = 0; i < B; ++i) {
+      float4 *d4 = reinterpret_cast<float4 *>(Ds + i * kWideDStride + 4 * lane);
+      float4 v = *d4;
+      v.x -= mu[0]; v.y -= mu[1]; v.z -= mu[2]; v.w -= mu[3];
+      *d4 = v;
+    }
+    __syncwarp();
+  }
+  // ---- Gram matrix: lane j (and j + 32) computes column j of M, row by row
+  float amax = 0.f;
+  for (int jj = lane; jj < B; jj += 32) {
+    for (int i = 0; i < B; ++i) {
+      const float4 *di = reinterpret_cast<const float4 *>(Ds + i * kWideDStride);
+      const float4 *dj = reinterpret_cast<const float4 *>(Ds + jj * kWideDStride);
+      float acc = 0.f;
+#pragma unroll 8
+      for (int c = 0; c < LOCKS_D / 4; ++c) {
+        const float4 x = di[c], y = dj[c];
+        acc = fmaf(x.x, y.x, fmaf(x.y, y.y, fmaf(x.z, y.z, fmaf(x.w, y.w, acc))));
+      }
+      W[jj * WS + i] = acc;
+      amax = fmaxf(amax, fabsf(acc));
+    }
+  }
+  amax = warp_max(amax);
+  // unit scale (an exact power of two, undone on the eigenvalues)
+  float unscale = 1.f;
+  if (amax > 0.f && amax < INFINITY) {
+    int ex;
+    (void)frexpf(amax, &ex);
+    ex = max(-120, min(120, ex));
+    const float sc = ldexpf(1.f, -ex);
+    unscale = ldexpf(1.f, ex);
+    for (int jj = lane; jj < B; jj += 32)
+      for (int i = 0; i < B; ++i) W[jj * WS + i] *= sc;
+  }
+  __syncwarp();
+  // ---- one-sided Jacobi, odd-even transposition, rotate then swap
+  const float tol2 = LOCKS_BUILD_COS_TOL * LOCKS_BUILD_COS_TOL;
+  for (int sweep = 0; sweep < 2 * LOCKS_BUILD_SWEEPS; ++sweep) {
+    float nm = 0.f;
+    for (int jj = lane; jj < B; jj += 32) {
+      float a = 0.f;
+      for (int i = 0; i < B; ++i) a = fmaf(W[jj * WS + i], W[jj * WS + i], a);
+      nr[jj] = a;
+      nm = fmaxf(nm, a);
+    }
+    const float floor_n = 1e-11f * warp_max(nm);
+    __syncwarp();
+    int bad = 0;
+    for (int st = 0; st < B; ++st) {
+      const int pc = 2 * lane + (st & 1), qc = pc + 1;   // the pair of this lane
+      if (qc < B) {
+        float *wp = W + pc * WS, *wq = W + qc * WS;
+        const float a = nr[pc], bq = nr[qc];
+        float g = 0.f;
+        for (int i = 0; i < B; ++i) g = fmaf(wp[i], wq[i], g);
+        bad |= (int)(g * g > tol2 * a * bq) & (int)(fminf(a, bq) > floor_n);
+        float c, sn;
+        jacobi_angle(a, bq, g, c, sn);
+        for (int i = 0; i < B; ++i) {
+          const float x = wp[i], y = wq[i];
+          wp[i] = fmaf(sn, x, c * y);    // q' takes p's place
+          wq[i] = fmaf(c, x, -sn * y);   // p' takes q's place
+        }
+        nr[pc] = fmaxf(fmaf(sn * sn, a, fmaf(c * c, bq, 2.f * c * sn * g)), 0.f);
+        nr[qc] = fmaxf(fmaf(c * c, a, fmaf(sn * sn, bq, -2.f * c * sn * g)), 0.f);
+      }
+      __syncwarp();
+    }
+    if (!__any_sync(0xffffffffu, bad != 0)) break;
+  }
+  // ---- exact norms, ranking (descending, ties to the lower position)
+  for (int jj = lane; jj < B; jj += 32) {
+    float a = 0.f;
+    for (int i = 0; i < B; ++i) a = fmaf(W[jj * WS + i], W[jj * WS + i], a);
+    nr[jj] = a;
+  }
+  __syncwarp();
+  for (int jj = lane; jj < B; jj += 32) {
+    const float mine = nr[jj];
+    int rk = 0;
+    for (int o = 0; o < B; ++o) rk += (nr[o] > mine) || (nr[o] == mine && o < jj);
+    order[rk] = jj;
+  }
+  __syncwarp();
+  const float lam0 = sqrtf(nr[order[0]]) * unscale;
+  int r_eff = 0;
+  const int rmax = min(r, B - 1);
+  for (int l = 0; l < rmax; ++l) {
+    const float ll = sqrtf(nr[order[l]]) * unscale;
+    if (lam0 > 0.f && ll > 1e-6f * lam0 && ll > 1e-10f * knorm2) r_eff = l + 1; else break;
+  }
+  uint8_t *gout = p.summ + ((int64_t)block * p.Hkv + h) * p.S;
+  float *fout = reinterpret_cast<float *>(gout);
+  constexpr int WD = FMT == LOCKS_FMT_BF16 ? 2 : 1;
+  uint32_t sign_bits = 0u;
+  for (int l = 0; l < r; ++l) {
+    float v[4] = {0.f, 0.f, 0.f, 0.f}, best = 0.f;
+    if (l < r_eff) {
+      const int col = order[l];
+      const float n2 = nr[col], lam = sqrtf(n2) * unscale;
+      const float inv = rsqrtf(n2) * rsqrtf(lam);   // unit eigenvector entries, then 1 / sigma
+      for (int i = 0; i < B; ++i) {
+        const float u = W[col * WS + i];
+        const float4 d4 = *reinterpret_cast<const float4 *>(Ds + i * kWideDStride + 4 * lane);
+        v[0] = fmaf(d4.x, u, v[0]); v[1] = fmaf(d4.y, u, v[1]); v[2] = fmaf(d4.z, u, v[2]); v[3] = fmaf(d4.w, u, v[3]);
+      }
+#pragma unroll
+      for (int c = 0; c < 4; ++c) v[c] *= inv;
+      best = fabsf(v[0]); float bv = v[0];
+#pragma unroll
+      for (int c = 1; c < 4; ++c) if (fabsf(v[c]) > best) { best = fabsf(v[c]); bv = v[c]; }
+      const uint32_t mxb = __reduce_max_sync(0xffffffffu, __float_as_uint(best));
+      const uint32_t who = __ballot_sync(0xffffffffu, __float_as_uint(best) == mxb);
+      bv = __shfl_sync(0xffffffffu, bv, __ffs(who) - 1);
+      best = __uint_as_float(mxb);
+      if (bv < 0.f) {
+        sign_bits |= 1u << l;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) v[c] = -v[c];
+      }
+    }
+    if (FMT == LOCKS_FMT_F32) {
+      *reinterpret_cast<float4 *>(fout + LOCKS_D + l * LOCKS_D + lane * 4) = make_float4(v[0], v[1], v[2], v[3]);
+    } else if (FMT == LOCKS_FMT_BF16) {
+      *reinterpret_cast<uint2 *>(gout + 2 * (l * LOCKS_D + lane * 4)) = make_uint2(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]));
+    } else {
+      const __half sh = __float2half_rn(best / 127.f);
+      const float sc = inv_scale(__half2float(sh));
+      if (lane == 0) *reinterpret_cast<__half *>(gout + wb_off_sv(r, 1, B) + 2 * l) = sh;
+      uint32_t wd = 0u;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) wd |= (uint32_t)((int)round_code(v[c], sc, 127.f) + 128) << (8 * c);
+      *reinterpret_cast<uint32_t *>(gout + l * LOCKS_D + lane * 4) = wd;
+    }
+  }
+  // coefficients: lane owns tokens lane and lane + 32
+  for (int tok = lane; tok < B; tok += 32) {
+    float mx = 0.f;
+    for (int l = 0; l < r; ++l) {
+      float c = 0.f;
+      if (l < r_eff) {
+        const int col = order[l];
+        c = W[col * WS + tok] * rsqrtf(nr[col]) * sqrtf(sqrtf(nr[col]) * unscale);
+        if ((sign_bits >> l) & 1u) c = -c;
+      }
+      mx = fmaxf(mx, fabsf(c));
+      if (FMT == LOCKS_FMT_F32) fout[LOCKS_D + r * LOCKS_D + tok * r + l] = c;
+    }
+    if (FMT != LOCKS_FMT_F32) {
+      const __half sh = __float2half_rn(mx / 127.f);
+      const float sc = inv_scale(__half2float(sh));
+      *reinterpret_cast<__half *>(gout + wb_off_sc(r, WD, B) + 2 * tok) = sh;
+      for (int l = 0; l < r; ++l) {
+        float c = 0.f;
+        if (l < r_eff) {
+          const int col = order[l];
+          c = W[col * WS + tok] * rsqrtf(nr[col]) * sqrtf(sqrtf(nr[col]) * unscale);
+          if ((sign_bits >> l) & 1u) c = -c;
+        }
+        gout[wb_off_coef(r, WD) + tok * r + l] = (uint8_t)((int)round_code(c, sc, 127.f) + 128);
+      }
+    }
+  }
+  // centroid
+  if (FMT == LOCKS_FMT_F32) {
+    *reinterpret_cast<float4 *>(fout + lane * 4) = make_float4(mu[0], mu[1], mu[2], mu[3]);
+  } else {
+    float mx = fmaxf(fmaxf(fabsf(mu[0]), fabsf(mu[1])), fmaxf(fabsf(mu[2]), fabsf(mu[3])));
+    mx = __uint_as_float(__reduce_max_sync(0xffffffffu, __float_as_uint(mx)));
+    const __half sh = __float2half_rn(mx / 127.f);
+    const float sc = inv_scale(__half2float(sh));
+    if (lane == 0) *reinterpret_cast<__half *>(gout + wb_off_smu(r, WD, B)) = sh;
+    uint32_t wd = 0u;
+#pragma unroll
+    for (int c = 0; c < 4; ++c) wd |= (uint32_t)((int)round_code(mu[c], sc, 127.f) + 128) << (8 * c);
+    *reinterpret_cast<uint32_t *>(gout + wb_off_mu(r, WD, B) + lane * 4) = wd;
+    for (int e = wb_off_smu(r, WD, B) + 2 + lane; e < p.S; e += 32) gout[e] = 0;
+  }
+}
+
 }  // namespace
 
 int locks_launch_build(locks_ctx *c, const locks_kv *kv, int batch, const int32_t *pb, const int32_t *pe,
@@ -744,6 +986,28 @@ int locks_launch_build(locks_ctx *c, const locks_kv *kv, int batch, const int32_
   if (just_filled && c->hint_dev && c->cfg.summary_fmt == LOCKS_FMT_I4 && c->cfg.q_dtype == LOCKS_BF16) {
     const locks_scan_geom geo = locks_scan_geometry(c, batch);
     p.hint = c->hint_dev; p.hint_wpp = geo.wpp; p.hint_rounds = geo.rounds; p.hint_W = geo.W;
+  }
+  if (c->B != LOCKS_B) {   // pages of 32 / 64 tokens: the plain kernel (row-major formats; one layer per launch)
+    if (k_layers || c->cfg.summary_fmt == LOCKS_FMT_I4) return LOCKS_ERR_UNSUPPORTED;
+    const int B = c->B, smem = build_wide_smem(B);
+    const dim3 grid = just_filled ? dim3(batch * p.Hkv) : dim3(c->Pmax, p.Hkv, batch);
+    const bool bf16kv = c->cfg.kv_dtype == LOCKS_BF16;
+#define LOCKS_WIDE_CASE(F_)                                                                                              \
+  do {                                                                                                                  \
+    if (locks_attrs_needed(LOCKS_ATTR_BUILD_WIDE + F_)) {                                                                \
+      cudaFuncSetAttribute(build_wide_kernel<__nv_bfloat16, F_>, cudaFuncAttributeMaxDynamicSharedMemorySize, build_wide_smem(64)); \
+      cudaFuncSetAttribute(build_wide_kernel<float, F_>, cudaFuncAttributeMaxDynamicSharedMemorySize, build_wide_smem(64));         \
+    }                                                                                                                   \
+    if (bf16kv) build_wide_kernel<__nv_bfloat16, F_><<<grid, 32, smem, st>>>(p, B, just_filled);                        \
+    else build_wide_kernel<float, F_><<<grid, 32, smem, st>>>(p, B, just_filled);                                       \
+  } while (0)
+    switch (c->cfg.summary_fmt) {
+      case LOCKS_FMT_I8: LOCKS_WIDE_CASE(LOCKS_FMT_I8); break;
+      case LOCKS_FMT_BF16: LOCKS_WIDE_CASE(LOCKS_FMT_BF16); break;
+      default: LOCKS_WIDE_CASE(LOCKS_FMT_F32); break;
+    }
+#undef LOCKS_WIDE_CASE
+    return locks_check_launch(c);
   }
   constexpr int kPer = kBuildWarps * kBuildItems;   // items per CTA (bulk)
   dim3 grid = just_filled ? dim3((batch * p.Hkv + kBuildWarps - 1) / kBuildWarps)

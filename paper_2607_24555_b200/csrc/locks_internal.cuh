@@ -8,7 +8,8 @@
 #include "locks.h"
 
 #define LOCKS_D 128          // head dimension the kernels are written for
-#define LOCKS_B 16           // tokens per page
+#define LOCKS_B 16           // tokens per page of the main (tensor-core) paths; pages of 32 and 64 tokens
+                             // (cfg.page_size) go through the plain fp32 kernels, which take the size at run time
 #define LOCKS_GROUP 8        // pages scored together by one warp in the scan (one ring stage, one partial)
 #define LOCKS_SEL_THREADS 512
 #define LOCKS_SEL_MAX_EPT 16 // pages per thread a selector CTA ranks at most (512 threads: 8192 pages or list entries)
@@ -55,6 +56,7 @@ struct locks_host_graph {
 struct locks_ctx {
   locks_config cfg;
   int G, k, S, Pmax, max_groups;
+  int B;                   // tokens per page (cfg.page_size): 16, or 32 / 64 on the plain kernels
   int num_sms;
   int part_slots;          // partial slots per (request, head) the last scan launch may have filled
   int part_balanced;       // the last scan launch wrote per-problem partial counts to part_cnt instead
@@ -121,7 +123,7 @@ __device__ __forceinline__ void locks_update_partition_hint(int32_t *hint, const
                                                             int k, int wpp, int rounds, int W, int lane) {
   int sum = 0, mx = 0;
   for (int b = lane; b < batch; b += 32) {
-    const int P = (seq_lens[b] + LOCKS_B - 1) / LOCKS_B;
+    const int P = (seq_lens[b] + LOCKS_B - 1) / LOCKS_B;   // (the hint serves the tensor scan: 16-token pages)
     const int ng = P <= k ? 0 : (P - 1 + LOCKS_GROUP - 1) / LOCKS_GROUP;
     sum += ng;
     mx = max(mx, ng);
@@ -220,7 +222,8 @@ static inline int locks_check_launch(locks_ctx *c) {
 // Function attributes (dynamic shared-memory limit, non-portable cluster size) belong to a device, not to the
 // process: true exactly once per (current device, kernel family), so that a process that drives several GPUs
 // sets them on each.  Thread-safe.
-enum { LOCKS_ATTR_SELECT = 0, LOCKS_ATTR_ATTEND = 1, LOCKS_ATTR_EXACT = 3, LOCKS_ATTR_BUILD = 4 /* + format */, LOCKS_ATTR_SCAN = 8 };
+enum { LOCKS_ATTR_SELECT = 0, LOCKS_ATTR_ATTEND = 1, LOCKS_ATTR_EXACT = 3, LOCKS_ATTR_BUILD = 4 /* + format */, LOCKS_ATTR_SCAN = 8,
+       LOCKS_ATTR_BUILD_WIDE = 24 /* + format */ };
 bool locks_attrs_needed(int family);
 
 // ---------------------------------------------------------------- I4 blob geometry (B = 16, d = 128)
@@ -231,17 +234,17 @@ __host__ __device__ constexpr int i4_off_sc(int r) { return 80 * r + 128; }
 __host__ __device__ constexpr int i4_off_sv(int r) { return 80 * r + 160; }
 __host__ __device__ constexpr int i4_off_smu(int r) { return 82 * r + 160; }
 __host__ __device__ constexpr int i4_stride(int r) { return (82 * r + 162 + 15) / 16 * 16; }
-__host__ __device__ constexpr int f32_stride(int r) { return 4 * (LOCKS_D + r * LOCKS_D + LOCKS_B * r); }
+__host__ __device__ constexpr int f32_stride(int r, int B = LOCKS_B) { return 4 * (LOCKS_D + r * LOCKS_D + B * r); }
 // Row-major formats with an int8 (wide = 1) or bf16 (wide = 2) basis:
 // [basis r x d][coefficients B x r][centroid d][sC B x fp16][sV r x fp16 (int8 basis only)][sMu fp16], padded to 16.
 __host__ __device__ constexpr int wb_off_coef(int r, int wide) { return wide * LOCKS_D * r; }
-__host__ __device__ constexpr int wb_off_mu(int r, int wide) { return wide * LOCKS_D * r + LOCKS_B * r; }
-__host__ __device__ constexpr int wb_off_sc(int r, int wide) { return wb_off_mu(r, wide) + LOCKS_D; }
-__host__ __device__ constexpr int wb_off_sv(int r, int wide) { return wb_off_sc(r, wide) + 2 * LOCKS_B; }
-__host__ __device__ constexpr int wb_off_smu(int r, int wide) { return wb_off_sv(r, wide) + (wide == 1 ? 2 * r : 0); }
-__host__ __device__ constexpr int wb_stride(int r, int wide) { return (wb_off_smu(r, wide) + 2 + 15) / 16 * 16; }
-__host__ __device__ constexpr int locks_fmt_stride(int fmt, int r) {
-  return fmt == LOCKS_FMT_I4 ? i4_stride(r) : fmt == LOCKS_FMT_F32 ? f32_stride(r) : wb_stride(r, fmt == LOCKS_FMT_BF16 ? 2 : 1);
+__host__ __device__ constexpr int wb_off_mu(int r, int wide, int B = LOCKS_B) { return wide * LOCKS_D * r + B * r; }
+__host__ __device__ constexpr int wb_off_sc(int r, int wide, int B = LOCKS_B) { return wb_off_mu(r, wide, B) + LOCKS_D; }
+__host__ __device__ constexpr int wb_off_sv(int r, int wide, int B = LOCKS_B) { return wb_off_sc(r, wide, B) + 2 * B; }
+__host__ __device__ constexpr int wb_off_smu(int r, int wide, int B = LOCKS_B) { return wb_off_sv(r, wide, B) + (wide == 1 ? 2 * r : 0); }
+__host__ __device__ constexpr int wb_stride(int r, int wide, int B = LOCKS_B) { return (wb_off_smu(r, wide, B) + 2 + 15) / 16 * 16; }
+__host__ __device__ constexpr int locks_fmt_stride(int fmt, int r, int B = LOCKS_B) {
+  return fmt == LOCKS_FMT_I4 ? i4_stride(r) : fmt == LOCKS_FMT_F32 ? f32_stride(r, B) : wb_stride(r, fmt == LOCKS_FMT_BF16 ? 2 : 1, B);
 }
 
 #ifdef __CUDACC__

@@ -34,6 +34,7 @@ struct ScanParams {
   int32_t *part_cnt;   // [batch][Hkv] partials written per head of a problem (balanced partition)
   int32_t *status;
   int batch, Hq, Hkv, G, Pmax, max_groups, num_blocks, k, S, r;
+  int B;   // tokens per page
   float sm_scale;
   // decode step with an appended token: lengths count the token that the selector's kernel is about to
   // write (seq_inc = 1); the first CTA publishes them, and the append position, for the step's later kernels
@@ -47,14 +48,14 @@ struct ScanParams {
 
 // Length of request b as this step sees it.  A sequence that has no room for the token keeps its length.
 __device__ __forceinline__ int step_len(const ScanParams &p, int b) {
-  return min(p.seq_lens[b] + p.seq_inc, p.Pmax * LOCKS_B);
+  return min(p.seq_lens[b] + p.seq_inc, p.Pmax * p.B);
 }
 
 __device__ __forceinline__ void publish_lengths(const ScanParams &p, bool first_cta, int tid, int nthreads) {
   if (!first_cta || !p.seq_eff) return;
   for (int b = tid; b < p.batch; b += nthreads) {
     const int T0 = p.seq_lens[b], T1 = T0 + p.seq_inc;
-    const bool room = T1 <= p.Pmax * LOCKS_B;
+    const bool room = T1 <= p.Pmax * p.B;
     if (!room) set_status(p.status, LOCKS_ERR_BAD_BLOCK);
     p.seq_eff[b] = room ? T1 : T0;
     p.seq_eff[p.batch + b] = (room && p.seq_inc) ? T0 : -1;
@@ -91,7 +92,8 @@ __global__ void __launch_bounds__(128) scan_generic_kernel(ScanParams p) {
   pdl_wait();
   publish_lengths(p, (blockIdx.x | blockIdx.y | blockIdx.z) == 0, threadIdx.x, 128);
   const int T = step_len(p, b);
-  const int P = (T + LOCKS_B - 1) / LOCKS_B;
+  const int B = p.B;                  // 16, 32 or 64 tokens per page: lane i holds tokens i and i + 32
+  const int P = (T + B - 1) / B;
   if (P <= p.k) return;               // every page is kept: nothing to rank
   const int nsc = P - 1;              // pages 0 .. P-2 are scored
   if (grp * LOCKS_GROUP >= nsc) return;
@@ -126,16 +128,16 @@ __global__ void __launch_bounds__(128) scan_generic_kernel(ScanParams p) {
         }
       } else if (FMT == LOCKS_FMT_I8 || FMT == LOCKS_FMT_BF16) {
         constexpr int W = FMT == LOCKS_FMT_BF16 ? 2 : 1;
-        const float smu = __half2float(*reinterpret_cast<const __half *>(blob + wb_off_smu(r, W)));
+        const float smu = __half2float(*reinterpret_cast<const __half *>(blob + wb_off_smu(r, W, B)));
 #pragma unroll
-        for (int u = 0; u < 4; ++u) a += (float)((int)blob[wb_off_mu(r, W) + lane * 4 + u] - 128) * qv[u];
+        for (int u = 0; u < 4; ++u) a += (float)((int)blob[wb_off_mu(r, W, B) + lane * 4 + u] - 128) * qv[u];
         a *= smu;
         for (int l = 0; l < r; ++l) {
           float s = 0.f;
           if (FMT == LOCKS_FMT_I8) {
 #pragma unroll
             for (int u = 0; u < 4; ++u) s += (float)((int)blob[l * LOCKS_D + lane * 4 + u] - 128) * qv[u];
-            s *= __half2float(*reinterpret_cast<const __half *>(blob + wb_off_sv(r, W) + 2 * l));
+            s *= __half2float(*reinterpret_cast<const __half *>(blob + wb_off_sv(r, W, B) + 2 * l));
           } else {
 #pragma unroll
             for (int u = 0; u < 4; ++u)
@@ -157,32 +159,41 @@ __global__ void __launch_bounds__(128) scan_generic_kernel(ScanParams p) {
         }
       }
       a = warp_sum(a);
-      float logit = -INFINITY;
-      if (lane < LOCKS_B) {
+      float logit[2] = {-INFINITY, -INFINITY};   // tokens lane and lane + 32
+#pragma unroll
+      for (int half = 0; half < 2; ++half) {
+        const int tok = lane + 32 * half;
+        if (tok >= B) continue;
         float s = 0.f;
         if (FMT == LOCKS_FMT_F32) {
-          const float *f = reinterpret_cast<const float *>(blob) + LOCKS_D + r * LOCKS_D + lane * r;
+          const float *f = reinterpret_cast<const float *>(blob) + LOCKS_D + r * LOCKS_D + tok * r;
           for (int l = 0; l < r; ++l) s += proj[l] * f[l];
         } else if (FMT == LOCKS_FMT_I8 || FMT == LOCKS_FMT_BF16) {
           constexpr int W = FMT == LOCKS_FMT_BF16 ? 2 : 1;
-          for (int l = 0; l < r; ++l) s += proj[l] * (float)((int)blob[wb_off_coef(r, W) + lane * r + l] - 128);
-          s *= __half2float(*reinterpret_cast<const __half *>(blob + wb_off_sc(r, W) + 2 * lane));
+          for (int l = 0; l < r; ++l) s += proj[l] * (float)((int)blob[wb_off_coef(r, W) + tok * r + l] - 128);
+          s *= __half2float(*reinterpret_cast<const __half *>(blob + wb_off_sc(r, W, B) + 2 * tok));
         } else {
-          for (int l = 0; l < r; ++l) s += proj[l] * i4_coef_val(blob, r, lane, l);
-          s *= i4_sc_val(blob, r, lane);
+          for (int l = 0; l < r; ++l) s += proj[l] * i4_coef_val(blob, r, tok, l);
+          s *= i4_sc_val(blob, r, tok);
         }
-        logit = p.sm_scale * (a + s);
+        logit[half] = p.sm_scale * (a + s);
       }
       float sh;
       if (p.scorer == LOCKS_SCORER_CENTROID) {          // the centroid term alone: q.mu / sqrt(d) + log B
-        sh = p.sm_scale * a + logf((float)LOCKS_B);
+        sh = p.sm_scale * a + logf((float)B);
       } else if (p.scorer == LOCKS_SCORER_MOMENT) {     // second-cumulant truncation of the mass (moment core)
-        const float zi = lane < LOCKS_B ? logit - p.sm_scale * a : 0.f;
-        sh = p.sm_scale * a + logf((float)LOCKS_B) + warp_sum(zi * zi) * (0.5f / LOCKS_B);
+        float z2 = 0.f;
+#pragma unroll
+        for (int half = 0; half < 2; ++half)
+          if (lane + 32 * half < B) { const float zi = logit[half] - p.sm_scale * a; z2 = fmaf(zi, zi, z2); }
+        sh = p.sm_scale * a + logf((float)B) + warp_sum(z2) * (0.5f / B);
       } else {
-        const float mx = warp_max(logit);
-        const float z = warp_sum(lane < LOCKS_B ? expf(logit - mx) : 0.f);
-        sh = mx + logf(z);
+        const float mx = warp_max(fmaxf(logit[0], logit[1]));
+        float e = 0.f;
+#pragma unroll
+        for (int half = 0; half < 2; ++half)
+          if (lane + 32 * half < B) e += expf(logit[half] - mx);
+        sh = mx + logf(warp_sum(e));
       }
       if (lane == 0) {
         p.shat[((int64_t)b * p.Hq + hq) * p.Pmax + page] = sh;
@@ -978,10 +989,10 @@ int locks_launch_scan(locks_ctx *c, const void *q, const void *summaries, const 
   p.status = c->status;
   p.batch = batch; p.Hq = c->cfg.num_q_heads; p.Hkv = c->cfg.num_kv_heads; p.G = c->G;
   p.Pmax = c->Pmax; p.max_groups = c->max_groups; p.num_blocks = kv->num_blocks; p.k = c->k;
-  p.S = c->S; p.r = c->cfg.rank; p.sm_scale = c->cfg.sm_scale;
+  p.S = c->S; p.r = c->cfg.rank; p.sm_scale = c->cfg.sm_scale; p.B = c->B;
   p.scorer = c->scorer;
   const bool tensor = c->cfg.summary_fmt == LOCKS_FMT_I4 && c->cfg.q_dtype == LOCKS_BF16 &&
-                      c->scorer == LOCKS_SCORER_SUMMARY;   // ranks 2, 4, 8
+                      c->scorer == LOCKS_SCORER_SUMMARY && c->B == LOCKS_B;   // ranks 2, 4, 8
   c->part_slots = c->max_groups;   // generic kernel: one partial per 8-page group
   c->part_balanced = 0;
   c->last_partition = 0;

@@ -37,6 +37,7 @@ struct SelParams {
   int32_t *status;
   int batch, Hq, Hkv, G, Pmax, max_groups, k, chunks, kc, chunk_pages, part_slots;
   int combine;       // LOCKS_COMBINE_*
+  int Bshift;        // log2 of the page size (4, 5 or 6)
   locks_append app;  // decode step only: the new token's K/V rows, written here beside the ranking
 };
 
@@ -46,11 +47,11 @@ struct SelParams {
 // the scan (complete before this kernel passes its wait) and the end of the step: the step's other
 // kernels take lengths from the published copy.
 __device__ __forceinline__ void append_token(const locks_append &a, int batch, int Hkv, int Pmax, int b, int h,
-                                             int lane, int T, int32_t *status) {
+                                             int lane, int T, int32_t *status, int Bshift) {
   if (h == 0 && lane == 0) a.seq_commit[b] = T;
   const int at = a.seq_eff[batch + b];
   if (at < 0) return;
-  const int page = at / LOCKS_B, slot = at % LOCKS_B;
+  const int page = at >> Bshift, slot = at & ((1 << Bshift) - 1);
   const int block = a.block_table[(int64_t)b * Pmax + page];
   if (block < 0 || block >= a.num_blocks) {
     if (lane == 0) set_status(status, LOCKS_ERR_BAD_BLOCK);
@@ -427,8 +428,8 @@ __global__ void __launch_bounds__(LOCKS_SEL_THREADS, 2) select_kernel(SelParams 
   pdl_wait();   // the scan's scores and partials
   const int T = p.seq_lens[b];
   if (p.app.k_new && chunk == 0 && tid >= LOCKS_SEL_THREADS - 32)
-    append_token(p.app, p.batch, p.Hkv, p.Pmax, b, h, tid & 31, T, p.status);
-  const int P = (T + LOCKS_B - 1) / LOCKS_B;
+    append_token(p.app, p.batch, p.Hkv, p.Pmax, b, h, tid & 31, T, p.status, p.Bshift);
+  const int P = (T + (1 << p.Bshift) - 1) >> p.Bshift;
   const int64_t prob = (int64_t)b * p.Hkv + h;
   int32_t *ids = p.ids + prob * p.k;
   if (P <= p.k) {  // every page is kept
@@ -605,6 +606,7 @@ int locks_launch_select(locks_ctx *c, const float *shat, const locks_kv *kv, int
   p.chunk_pages = c->sel_ept * LOCKS_SEL_THREADS;
   p.part_slots = c->part_slots;
   p.combine = c->cfg.combine;
+  p.Bshift = c->B == 64 ? 6 : (c->B == 32 ? 5 : 4);
   p.part_cnt = c->part_balanced ? c->part_cnt : nullptr;
   if (p.chunk_pages > kMaxKeys || (int64_t)c->sel_chunks * c->sel_kc > kMaxKeys || p.G > 16) return LOCKS_ERR_UNSUPPORTED;
   // Two CTAs fit on an SM (64 registers per thread).  That halves the waves of a launch with many more CTAs

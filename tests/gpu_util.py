@@ -22,7 +22,7 @@ class GpuCase:
         self.case = locks_synth.make_case(w, device="cuda:0")
         self.max_pages = self.case.block_table.shape[1]
         self.sm = 1.0 / math.sqrt(w.d)
-        self.cfg = make_config(w.Hq, w.Hkv, w.rank, w.fmt, w.dtype, max_batch or w.n, self.max_pages, w.budget)
+        self.cfg = make_config(w.Hq, w.Hkv, w.rank, w.fmt, w.dtype, max_batch or w.n, self.max_pages, w.budget, B=w.B)
         self.ctx = locks.Context(self.cfg)
         self.kv = KVView(self.case.k, self.case.v, self.case.strides, self.case.num_blocks, self.case.block_table,
                          self.case.seq_lens)

@@ -1,0 +1,107 @@
+"""Pages of 32 and 64 tokens (the paper's App. D "Page size" ablation) on the plain fp32 kernels: build, scan,
+selection, attention and the decode step against the oracle, which takes the page size as an argument."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import locks_synth
+import oracle
+from common import t2np
+
+pytestmark = pytest.mark.gpu
+
+
+def _gc(w, **kw):
+    from gpu_util import GpuCase
+    return GpuCase(w, **kw)
+
+
+def _w(B, fmt, dtype, lens, **kw):
+    return locks_synth.Workload(f"b{B}", list(lens), Hq=8, Hkv=2, B=B, rank=8, fmt=fmt, dtype=dtype, budget=8 * B, **kw)
+
+
+@pytest.mark.parametrize("B,fmt,dtype", [(32, "f32", "f32"), (64, "f32", "f32"), (32, "i8", "bf16"), (64, "bf16", "bf16"),
+                                         (64, "i8", "f32")])
+def test_wide_page_build_select_attend(B, fmt, dtype):
+    """Summaries built on the GPU score like the oracle's own; selection and attention on identical bytes."""
+    from gpu_util import check_select_and_attend
+    gc = _gc(_w(B, fmt, dtype, [B * 40 + 5, B * 23, B * 9 + B - 1], seed=B + len(fmt)))
+    w = gc.w
+    assert gc.k == 8
+    g_summ = gc.gpu_build().cpu().numpy()
+    o_summ = gc.oracle_summaries()
+    assert g_summ.shape == o_summ.shape and g_summ.shape[-1] == oracle.summary_stride_bytes(gc.fmt, w.rank, B, w.d)
+    rng = np.random.default_rng(B)
+    worst = 0.0
+    for b in range(w.n):
+        bt = gc.cache.block_table[b]
+        for p in range(w.seq_lens[b] // B):
+            for h in range(w.Hkv):
+                mg = oracle.unpack(gc.fmt, w.rank, g_summ[bt[p], h], B, w.d)
+                mo = oracle.unpack(gc.fmt, w.rank, o_summ[bt[p], h], B, w.d)
+                assert np.abs(mg[0] - mo[0]).max() <= 2e-2 * max(1.0, np.abs(mo[0]).max())        # centroid (one code)
+                assert np.abs(mg[1] @ mg[1].T - np.eye(w.rank)).max() < (1e-3 if fmt == "f32" else 0.1)
+                for _ in range(2):
+                    q = rng.standard_normal(w.d)
+                    worst = max(worst, abs(oracle.score(*mg, q, gc.sm) - oracle.score(*mo, q, gc.sm)))
+    assert worst <= (1e-3 if fmt == "f32" else 3e-2), worst
+    # the partial last page of request 0 and 2 was not built
+    assert gc.status() == 0
+    check_select_and_attend(gc, o_summ, out_tol=1e-4 if dtype == "f32" else 2e-2)
+    out, lse = gc.gpu_attend()                                            # dense mode
+    oout, olse = oracle.attend(gc.cache, t2np(gc.case.q), gc.sm)
+    assert np.abs(out - oout).max() <= (1e-4 if dtype == "f32" else 2e-2) and np.abs(lse - olse).max() <= 1e-3
+
+
+@pytest.mark.parametrize("B", [32, 64])
+def test_wide_page_decode_step_crosses_page_boundaries(B):
+    """locks_decode_step with appends across page boundaries at B = 32 / 64; summaries of freshly filled pages come
+    from the device and are handed to the oracle (identical bytes) for the next steps."""
+    from common import check_page_sets, oracle_cache
+    w = _w(B, "f32", "f32", [B * 12 - 3, B * 11 + B - 2], seed=7 * B)
+    reserve = 2
+    w = w.with_(seq_lens=[t + B * reserve for t in w.seq_lens])
+    gc = _gc(w)
+    start = torch.tensor([t - B * reserve for t in w.seq_lens], dtype=torch.int32, device="cuda:0")
+    gc.case.seq_lens.copy_(start)
+    summ = gc.ctx.new_summaries(gc.case.num_blocks)
+    gc.ctx.locks_build_summaries(gc.kv, w.n, summ)
+    out = torch.empty(w.n, w.Hq, w.d, dtype=torch.float32, device="cuda:0")
+    ids = torch.empty(w.n, w.Hkv, gc.k, dtype=torch.int32, device="cuda:0")
+    cnt = torch.empty(w.n, w.Hkv, dtype=torch.int32, device="cuda:0")
+    for step in range(B + 6):
+        kn, vn, qn = locks_synth.new_token(w, step, device="cuda:0")
+        gc.ctx.locks_decode_step(qn, kn, vn, gc.kv, summ, w.n, out, ids, cnt)
+        torch.cuda.synchronize()
+        assert gc.status() == 0
+        assert gc.case.seq_lens.cpu().tolist() == [int(s) + step + 1 for s in start.cpu()]
+        cache = oracle_cache(gc.case)
+        summ_np = summ.cpu().numpy()
+        shat = oracle.page_logmass(cache, t2np(qn), w.rank, gc.fmt, summ_np, gc.sm)
+        oids, ocnt, ols = oracle.select(cache, shat, gc.k)
+        check_page_sets(ids.cpu().numpy(), cnt.cpu().numpy(), oids, ocnt, ols, cache.seq_lens, B, gc.k)
+        oout, _ = oracle.attend(cache, t2np(qn), gc.sm, ids.cpu().numpy(), cnt.cpu().numpy())
+        assert np.abs(out.cpu().numpy().astype(np.float64) - oout).max() <= 1e-4, step
+        # a page that filled at this step: its device-built summary scores like the oracle's build of the same keys
+        for b in range(w.n):
+            T = int(cache.seq_lens[b])
+            if T % B == 0:
+                o_summ = oracle.build_summaries(cache, w.rank, gc.fmt)
+                blk = cache.block_table[b][T // B - 1]
+                rng = np.random.default_rng(step)
+                for h in range(w.Hkv):
+                    mg = oracle.unpack(gc.fmt, w.rank, summ_np[blk, h], B, w.d)
+                    mo = oracle.unpack(gc.fmt, w.rank, o_summ[blk, h], B, w.d)
+                    q = rng.standard_normal(w.d)
+                    assert abs(oracle.score(*mg, q, gc.sm) - oracle.score(*mo, q, gc.sm)) <= 1e-3
+
+
+def test_wide_pages_refuse_what_they_do_not_cover():
+    import paper_2607_24555_b200 as locks
+    from paper_2607_24555_b200.binding import make_config
+    with pytest.raises(locks.LocksError):
+        locks.Context(make_config(8, 2, 8, "i4", "bf16", 1, 64, 256, B=32))      # the int4 blob is laid out for 16 tokens
+    with pytest.raises(locks.LocksError):
+        locks.Context(make_config(8, 2, 8, "f32", "f32", 1, 64, 256, B=48))
