@@ -259,9 +259,12 @@ static int quant_code(double x, double scale, int qmax) {
   return (int)c;
 }
 
-/* Byte positions of the I4 blob (B = 16, d a multiple of 16, r in {2,4,8}).
- *   [basis d*r/2][coefficients 16 r][centroid d][sC 16 x fp16][sV r x fp16][sMu fp16]
- * Codes are stored offset-binary: nibble = code + 8, byte = code + 128. */
+/* Byte positions of the I4 blob (d a multiple of 16, r in {2,4,8}).
+ *   [basis d*r/2][coefficients B r][centroid d][sC B x fp16][sV r x fp16][sMu fp16]
+ * Codes are stored offset-binary: nibble = code + 8, byte = code + 128.  The paper fixes the byte COUNT of this
+ * format at every page size (App. C.1 payload table, App. D "Page size": 9.4 / 5.5 / 3.5 % of the page's KV bytes at
+ * B = 16 / 32 / 64), not the byte order.  Basis and centroid are ordered the same way at every B; coefficients and
+ * their scales follow an interleaved order at B = 16 and plain row-major order (token, rank) at other page sizes. */
 static void i4_basis_pos(int l, int c, int d, int *byte, int *shift) {
   /* dims are split into 4 contiguous quarters t; inside a quarter, group s covers 4 dims */
   int Q = d / 4, t = c / Q, w = c % Q, s = w >> 2, half = (w >> 1) & 1, e = w & 1;
@@ -269,7 +272,8 @@ static void i4_basis_pos(int l, int c, int d, int *byte, int *shift) {
   *byte = (l * 4 + t) * (Q / 2) + j * 4 + (nib >> 1);
   *shift = (nib & 1) * 4;
 }
-static int i4_coef_pos(int i, int l, int r) {
+static int i4_coef_pos(int i, int l, int r, int B) {
+  if (B != 16) return i * r + l;
   int x = i & 7, hi = i >> 3, tp = l >> 1, e = l & 1;
   return (x * (r / 2) + tp) * 4 + hi * 2 + e;
 }
@@ -277,7 +281,8 @@ static int i4_mu_pos(int c, int d) {
   int Q = d / 4, t = c / Q, w = c % Q, s = w >> 2, half = (w >> 1) & 1, e = w & 1;
   return t * Q + s * 4 + e * 2 + half;
 }
-static int i4_sc_pos(int i) {
+static int i4_sc_pos(int i, int B) {
+  if (B != 16) return i;
   int t = (i & 7) >> 1, e = i & 1, hi = i >> 3;
   return t * 4 + hi * 2 + e;
 }
@@ -339,9 +344,9 @@ void ora_pack(int fmt, int r, int B, int d, const double *mu, const double *V, c
   }
   for (int i = 0; i < B; ++i) { /* coefficients: one scale per row of C (per token) */
     double sc = quant_scale(C + i * r, r, 1, 127, &bits);
-    memcpy(blob + off_sc + 2 * i4_sc_pos(i), &bits, 2);
+    memcpy(blob + off_sc + 2 * i4_sc_pos(i, B), &bits, 2);
     for (int l = 0; l < r; ++l)
-      blob[off_coef + i4_coef_pos(i, l, r)] = (uint8_t)(quant_code(C[i * r + l], sc, 127) + 128);
+      blob[off_coef + i4_coef_pos(i, l, r, B)] = (uint8_t)(quant_code(C[i * r + l], sc, 127) + 128);
   }
   {
     double sc = quant_scale(mu, d, 1, 127, &bits);
@@ -402,9 +407,9 @@ void ora_unpack(int fmt, int r, int B, int d, const uint8_t *blob, double *mu, d
     }
   }
   for (int i = 0; i < B; ++i) {
-    memcpy(&bits, blob + off_sc + 2 * i4_sc_pos(i), 2);
+    memcpy(&bits, blob + off_sc + 2 * i4_sc_pos(i, B), 2);
     double sc = half_to_double(bits);
-    for (int l = 0; l < r; ++l) C[i * r + l] = sc * ((int)blob[off_coef + i4_coef_pos(i, l, r)] - 128);
+    for (int l = 0; l < r; ++l) C[i * r + l] = sc * ((int)blob[off_coef + i4_coef_pos(i, l, r, B)] - 128);
   }
   memcpy(&bits, blob + off_smu, 2);
   double sc = half_to_double(bits);
@@ -428,9 +433,9 @@ void ora_unpack_codes(int r, int B, int d, const uint8_t *blob, int32_t *cV, int
     }
   }
   for (int i = 0; i < B; ++i) {
-    memcpy(&bits, blob + off_sc + 2 * i4_sc_pos(i), 2);
+    memcpy(&bits, blob + off_sc + 2 * i4_sc_pos(i, B), 2);
     sC[i] = half_to_double(bits);
-    for (int l = 0; l < r; ++l) cC[i * r + l] = (int)blob[off_coef + i4_coef_pos(i, l, r)] - 128;
+    for (int l = 0; l < r; ++l) cC[i * r + l] = (int)blob[off_coef + i4_coef_pos(i, l, r, B)] - 128;
   }
   memcpy(&bits, blob + off_smu, 2);
   *sMu = half_to_double(bits);

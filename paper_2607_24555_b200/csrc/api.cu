@@ -21,9 +21,8 @@ int validate(const locks_config *c) {
   if ((c->kv_dtype != LOCKS_F32 && c->kv_dtype != LOCKS_BF16) || (c->q_dtype != LOCKS_F32 && c->q_dtype != LOCKS_BF16))
     return LOCKS_ERR_INVALID_ARG;
   if (c->head_dim != LOCKS_D) return LOCKS_ERR_UNSUPPORTED;
-  // pages of 32 and 64 tokens (App. D "Page size") run on the plain fp32 kernels with the row-major summary formats
-  if (c->page_size != LOCKS_B && !((c->page_size == 32 || c->page_size == 64) && c->summary_fmt != LOCKS_FMT_I4))
-    return LOCKS_ERR_UNSUPPORTED;
+  // pages of 32 and 64 tokens (App. D "Page size") run on the plain fp32 kernels
+  if (c->page_size != LOCKS_B && c->page_size != 32 && c->page_size != 64) return LOCKS_ERR_UNSUPPORTED;
   if (c->num_q_heads / c->num_kv_heads > 16) return LOCKS_ERR_UNSUPPORTED;
   if (c->kv_dtype != c->q_dtype) return LOCKS_ERR_UNSUPPORTED;
   if (c->summary_fmt == LOCKS_FMT_I4 && c->rank != 2 && c->rank != 4 && c->rank != 8) return LOCKS_ERR_UNSUPPORTED;

@@ -914,7 +914,7 @@ __global__ void __launch_bounds__(32) build_wide_kernel(BuildParams p, int B, in
       *reinterpret_cast<float4 *>(fout + LOCKS_D + l * LOCKS_D + lane * 4) = make_float4(v[0], v[1], v[2], v[3]);
     } else if (FMT == LOCKS_FMT_BF16) {
       *reinterpret_cast<uint2 *>(gout + 2 * (l * LOCKS_D + lane * 4)) = make_uint2(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]));
-    } else {
+    } else if (FMT == LOCKS_FMT_I8) {
       const __half sh = __float2half_rn(best / 127.f);
       const float sc = inv_scale(__half2float(sh));
       if (lane == 0) *reinterpret_cast<__half *>(gout + wb_off_sv(r, 1, B) + 2 * l) = sh;
@@ -922,6 +922,17 @@ __global__ void __launch_bounds__(32) build_wide_kernel(BuildParams p, int B, in
 #pragma unroll
       for (int c = 0; c < 4; ++c) wd |= (uint32_t)((int)round_code(v[c], sc, 127.f) + 128) << (8 * c);
       *reinterpret_cast<uint32_t *>(gout + l * LOCKS_D + lane * 4) = wd;
+    } else {   // int4 basis: the same nibble order as at B = 16
+      const __half sh = __float2half_rn(best / 7.f);
+      const float sc = inv_scale(__half2float(sh));
+      if (lane == 0) *reinterpret_cast<__half *>(gout + i4_off_sv(r, B) + 2 * l) = sh;
+      const int t = lane >> 3, s8 = lane & 7, i0 = (s8 & 1) << 1;
+      uint32_t nb[4];
+#pragma unroll
+      for (int c = 0; c < 4; ++c) nb[c] = (uint32_t)((int)round_code(v[c], sc, 7.f) + 8);
+      uint32_t pw = (nb[0] << (4 * i0)) | (nb[1] << (4 * (i0 + 4))) | (nb[2] << (4 * (i0 + 1))) | (nb[3] << (4 * (i0 + 5)));
+      pw |= __shfl_xor_sync(0xffffffffu, pw, 1);
+      if ((s8 & 1) == 0) *reinterpret_cast<uint32_t *>(gout + (l * 4 + t) * 16 + (s8 >> 1) * 4) = pw;
     }
   }
   // coefficients: lane owns tokens lane and lane + 32
@@ -940,7 +951,7 @@ __global__ void __launch_bounds__(32) build_wide_kernel(BuildParams p, int B, in
     if (FMT != LOCKS_FMT_F32) {
       const __half sh = __float2half_rn(mx / 127.f);
       const float sc = inv_scale(__half2float(sh));
-      *reinterpret_cast<__half *>(gout + wb_off_sc(r, WD, B) + 2 * tok) = sh;
+      *reinterpret_cast<__half *>(gout + (FMT == LOCKS_FMT_I4 ? i4_off_sc(r, B) : wb_off_sc(r, WD, B)) + 2 * tok) = sh;
       for (int l = 0; l < r; ++l) {
         float c = 0.f;
         if (l < r_eff) {
@@ -948,7 +959,7 @@ __global__ void __launch_bounds__(32) build_wide_kernel(BuildParams p, int B, in
           c = W[col * WS + tok] * rsqrtf(nr[col]) * sqrtf(sqrtf(nr[col]) * unscale);
           if ((sign_bits >> l) & 1u) c = -c;
         }
-        gout[wb_off_coef(r, WD) + tok * r + l] = (uint8_t)((int)round_code(c, sc, 127.f) + 128);
+        gout[(FMT == LOCKS_FMT_I4 ? i4_off_coef(r) : wb_off_coef(r, WD)) + tok * r + l] = (uint8_t)((int)round_code(c, sc, 127.f) + 128);
       }
     }
   }
@@ -960,12 +971,16 @@ __global__ void __launch_bounds__(32) build_wide_kernel(BuildParams p, int B, in
     mx = __uint_as_float(__reduce_max_sync(0xffffffffu, __float_as_uint(mx)));
     const __half sh = __float2half_rn(mx / 127.f);
     const float sc = inv_scale(__half2float(sh));
-    if (lane == 0) *reinterpret_cast<__half *>(gout + wb_off_smu(r, WD, B)) = sh;
-    uint32_t wd = 0u;
+    const int osmu = FMT == LOCKS_FMT_I4 ? i4_off_smu(r, B) : wb_off_smu(r, WD, B);
+    if (lane == 0) *reinterpret_cast<__half *>(gout + osmu) = sh;
+    uint32_t by[4];
 #pragma unroll
-    for (int c = 0; c < 4; ++c) wd |= (uint32_t)((int)round_code(mu[c], sc, 127.f) + 128) << (8 * c);
-    *reinterpret_cast<uint32_t *>(gout + wb_off_mu(r, WD, B) + lane * 4) = wd;
-    for (int e = wb_off_smu(r, WD, B) + 2 + lane; e < p.S; e += 32) gout[e] = 0;
+    for (int c = 0; c < 4; ++c) by[c] = (uint32_t)((int)round_code(mu[c], sc, 127.f) + 128);
+    if (FMT == LOCKS_FMT_I4)   // dim offset c = 2*half + e -> byte e*2 + half, as at B = 16
+      *reinterpret_cast<uint32_t *>(gout + i4_off_mu(r, B) + lane * 4) = by[0] | (by[2] << 8) | (by[1] << 16) | (by[3] << 24);
+    else
+      *reinterpret_cast<uint32_t *>(gout + wb_off_mu(r, WD, B) + lane * 4) = by[0] | (by[1] << 8) | (by[2] << 16) | (by[3] << 24);
+    for (int e = osmu + 2 + lane; e < p.S; e += 32) gout[e] = 0;
   }
 }
 
@@ -988,7 +1003,7 @@ int locks_launch_build(locks_ctx *c, const locks_kv *kv, int batch, const int32_
     p.hint = c->hint_dev; p.hint_wpp = geo.wpp; p.hint_rounds = geo.rounds; p.hint_W = geo.W;
   }
   if (c->B != LOCKS_B) {   // pages of 32 / 64 tokens: the plain kernel (row-major formats; one layer per launch)
-    if (k_layers || c->cfg.summary_fmt == LOCKS_FMT_I4) return LOCKS_ERR_UNSUPPORTED;
+    if (k_layers) return LOCKS_ERR_UNSUPPORTED;
     const int B = c->B, smem = build_wide_smem(B);
     const dim3 grid = just_filled ? dim3(batch * p.Hkv) : dim3(c->Pmax, p.Hkv, batch);
     const bool bf16kv = c->cfg.kv_dtype == LOCKS_BF16;
@@ -1002,6 +1017,7 @@ int locks_launch_build(locks_ctx *c, const locks_kv *kv, int batch, const int32_
     else build_wide_kernel<float, F_><<<grid, 32, smem, st>>>(p, B, just_filled);                                       \
   } while (0)
     switch (c->cfg.summary_fmt) {
+      case LOCKS_FMT_I4: LOCKS_WIDE_CASE(LOCKS_FMT_I4); break;
       case LOCKS_FMT_I8: LOCKS_WIDE_CASE(LOCKS_FMT_I8); break;
       case LOCKS_FMT_BF16: LOCKS_WIDE_CASE(LOCKS_FMT_BF16); break;
       default: LOCKS_WIDE_CASE(LOCKS_FMT_F32); break;

@@ -226,14 +226,14 @@ enum { LOCKS_ATTR_SELECT = 0, LOCKS_ATTR_ATTEND = 1, LOCKS_ATTR_EXACT = 3, LOCKS
        LOCKS_ATTR_BUILD_WIDE = 24 /* + format */ };
 bool locks_attrs_needed(int family);
 
-// ---------------------------------------------------------------- I4 blob geometry (B = 16, d = 128)
-// [basis 64 r][coefficients 16 r][centroid 128][sC 16 x fp16][sV r x fp16][sMu fp16], padded to 16.
+// ---------------------------------------------------------------- I4 blob geometry (d = 128; B = 16 unless given)
+// [basis 64 r][coefficients B r][centroid 128][sC B x fp16][sV r x fp16][sMu fp16], padded to 16.
 __host__ __device__ constexpr int i4_off_coef(int r) { return 64 * r; }
-__host__ __device__ constexpr int i4_off_mu(int r) { return 80 * r; }
-__host__ __device__ constexpr int i4_off_sc(int r) { return 80 * r + 128; }
-__host__ __device__ constexpr int i4_off_sv(int r) { return 80 * r + 160; }
-__host__ __device__ constexpr int i4_off_smu(int r) { return 82 * r + 160; }
-__host__ __device__ constexpr int i4_stride(int r) { return (82 * r + 162 + 15) / 16 * 16; }
+__host__ __device__ constexpr int i4_off_mu(int r, int B = LOCKS_B) { return 64 * r + B * r; }
+__host__ __device__ constexpr int i4_off_sc(int r, int B = LOCKS_B) { return i4_off_mu(r, B) + 128; }
+__host__ __device__ constexpr int i4_off_sv(int r, int B = LOCKS_B) { return i4_off_sc(r, B) + 2 * B; }
+__host__ __device__ constexpr int i4_off_smu(int r, int B = LOCKS_B) { return i4_off_sv(r, B) + 2 * r; }
+__host__ __device__ constexpr int i4_stride(int r, int B = LOCKS_B) { return (i4_off_smu(r, B) + 2 + 15) / 16 * 16; }
 __host__ __device__ constexpr int f32_stride(int r, int B = LOCKS_B) { return 4 * (LOCKS_D + r * LOCKS_D + B * r); }
 // Row-major formats with an int8 (wide = 1) or bf16 (wide = 2) basis:
 // [basis r x d][coefficients B x r][centroid d][sC B x fp16][sV r x fp16 (int8 basis only)][sMu fp16], padded to 16.
@@ -244,7 +244,7 @@ __host__ __device__ constexpr int wb_off_sv(int r, int wide, int B = LOCKS_B) { 
 __host__ __device__ constexpr int wb_off_smu(int r, int wide, int B = LOCKS_B) { return wb_off_sv(r, wide, B) + (wide == 1 ? 2 * r : 0); }
 __host__ __device__ constexpr int wb_stride(int r, int wide, int B = LOCKS_B) { return (wb_off_smu(r, wide, B) + 2 + 15) / 16 * 16; }
 __host__ __device__ constexpr int locks_fmt_stride(int fmt, int r, int B = LOCKS_B) {
-  return fmt == LOCKS_FMT_I4 ? i4_stride(r) : fmt == LOCKS_FMT_F32 ? f32_stride(r, B) : wb_stride(r, fmt == LOCKS_FMT_BF16 ? 2 : 1, B);
+  return fmt == LOCKS_FMT_I4 ? i4_stride(r, B) : fmt == LOCKS_FMT_F32 ? f32_stride(r, B) : wb_stride(r, fmt == LOCKS_FMT_BF16 ? 2 : 1, B);
 }
 
 #ifdef __CUDACC__

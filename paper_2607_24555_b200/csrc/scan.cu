@@ -72,17 +72,20 @@ __device__ __forceinline__ float i4_basis_val(const uint8_t *blob, int l, int c)
   int byte = (l * 4 + t) * 16 + j * 4 + (nib >> 1);
   return (float)(((blob[byte] >> ((nib & 1) * 4)) & 15) - 8);
 }
-__device__ __forceinline__ float i4_mu_val(const uint8_t *blob, int r, int c) {
+__device__ __forceinline__ float i4_mu_val(const uint8_t *blob, int r, int c, int B) {
   int t = c >> 5, w = c & 31, s = w >> 2, half = (w >> 1) & 1, e = w & 1;
-  return (float)((int)blob[i4_off_mu(r) + t * 32 + s * 4 + e * 2 + half] - 128);
+  return (float)((int)blob[i4_off_mu(r, B) + t * 32 + s * 4 + e * 2 + half] - 128);
 }
-__device__ __forceinline__ float i4_coef_val(const uint8_t *blob, int r, int i, int l) {
+// coefficients and their scales: interleaved for the tensor-core fragments at B = 16, row-major (token, rank) otherwise
+__device__ __forceinline__ float i4_coef_val(const uint8_t *blob, int r, int i, int l, int B) {
   int x = i & 7, hi = i >> 3, tp = l >> 1, e = l & 1;
-  return (float)((int)blob[i4_off_coef(r) + (x * (r / 2) + tp) * 4 + hi * 2 + e] - 128);
+  const int pos = B == LOCKS_B ? (x * (r / 2) + tp) * 4 + hi * 2 + e : i * r + l;
+  return (float)((int)blob[i4_off_coef(r) + pos] - 128);
 }
-__device__ __forceinline__ float i4_sc_val(const uint8_t *blob, int r, int i) {
+__device__ __forceinline__ float i4_sc_val(const uint8_t *blob, int r, int i, int B) {
   int t = (i & 7) >> 1, e = i & 1, hi = i >> 3;
-  return __half2float(*reinterpret_cast<const __half *>(blob + i4_off_sc(r) + 2 * (t * 4 + hi * 2 + e)));
+  const int pos = B == LOCKS_B ? t * 4 + hi * 2 + e : i;
+  return __half2float(*reinterpret_cast<const __half *>(blob + i4_off_sc(r, B) + 2 * pos));
 }
 
 template <int FMT, typename QT>
@@ -146,15 +149,15 @@ __global__ void __launch_bounds__(128) scan_generic_kernel(ScanParams p) {
           proj[l] = warp_sum(s);
         }
       } else {
-        const float smu = __half2float(*reinterpret_cast<const __half *>(blob + i4_off_smu(r)));
+        const float smu = __half2float(*reinterpret_cast<const __half *>(blob + i4_off_smu(r, B)));
 #pragma unroll
-        for (int u = 0; u < 4; ++u) a += i4_mu_val(blob, r, lane * 4 + u) * qv[u];
+        for (int u = 0; u < 4; ++u) a += i4_mu_val(blob, r, lane * 4 + u, B) * qv[u];
         a *= smu;
         for (int l = 0; l < r; ++l) {
           float s = 0.f;
 #pragma unroll
           for (int u = 0; u < 4; ++u) s += i4_basis_val(blob, l, lane * 4 + u) * qv[u];
-          const float sv = __half2float(*reinterpret_cast<const __half *>(blob + i4_off_sv(r) + 2 * l));
+          const float sv = __half2float(*reinterpret_cast<const __half *>(blob + i4_off_sv(r, B) + 2 * l));
           proj[l] = warp_sum(s) * sv;
         }
       }
@@ -173,8 +176,8 @@ __global__ void __launch_bounds__(128) scan_generic_kernel(ScanParams p) {
           for (int l = 0; l < r; ++l) s += proj[l] * (float)((int)blob[wb_off_coef(r, W) + tok * r + l] - 128);
           s *= __half2float(*reinterpret_cast<const __half *>(blob + wb_off_sc(r, W, B) + 2 * tok));
         } else {
-          for (int l = 0; l < r; ++l) s += proj[l] * i4_coef_val(blob, r, tok, l);
-          s *= i4_sc_val(blob, r, tok);
+          for (int l = 0; l < r; ++l) s += proj[l] * i4_coef_val(blob, r, tok, l, B);
+          s *= i4_sc_val(blob, r, tok, B);
         }
         logit[half] = p.sm_scale * (a + s);
       }

@@ -23,7 +23,7 @@ def _w(B, fmt, dtype, lens, **kw):
 
 
 @pytest.mark.parametrize("B,fmt,dtype", [(32, "f32", "f32"), (64, "f32", "f32"), (32, "i8", "bf16"), (64, "bf16", "bf16"),
-                                         (64, "i8", "f32")])
+                                         (64, "i8", "f32"), (32, "i4", "bf16"), (64, "i4", "bf16")])
 def test_wide_page_build_select_attend(B, fmt, dtype):
     """Summaries built on the GPU score like the oracle's own; selection and attention on identical bytes."""
     from gpu_util import check_select_and_attend
@@ -42,11 +42,29 @@ def test_wide_page_build_select_attend(B, fmt, dtype):
                 mg = oracle.unpack(gc.fmt, w.rank, g_summ[bt[p], h], B, w.d)
                 mo = oracle.unpack(gc.fmt, w.rank, o_summ[bt[p], h], B, w.d)
                 assert np.abs(mg[0] - mo[0]).max() <= 2e-2 * max(1.0, np.abs(mo[0]).max())        # centroid (one code)
-                assert np.abs(mg[1] @ mg[1].T - np.eye(w.rank)).max() < (1e-3 if fmt == "f32" else 0.1)
+                assert np.abs(mg[1] @ mg[1].T - np.eye(w.rank)).max() < (1e-3 if fmt == "f32" else 0.25 if fmt == "i4" else 0.1)
                 for _ in range(2):
                     q = rng.standard_normal(w.d)
                     worst = max(worst, abs(oracle.score(*mg, q, gc.sm) - oracle.score(*mo, q, gc.sm)))
-    assert worst <= (1e-3 if fmt == "f32" else 3e-2), worst
+    assert worst <= (1e-3 if fmt == "f32" else 0.15 if fmt == "i4" else 3e-2), worst   # one int4 / int8 code of a near-boundary entry
+    if fmt == "i4":   # integer codes agree with the oracle's after sign alignment (as at B = 16)
+        tot = diff = 0
+        for b in range(w.n):
+            bt = gc.cache.block_table[b]
+            for p in range(w.seq_lens[b] // B):
+                for h in range(w.Hkv):
+                    gV, gC, gMu, gsV, gsC, gsMu = oracle.unpack_codes(w.rank, g_summ[bt[p], h], B)
+                    oV, oC, oMu, osV, osC, osMu = oracle.unpack_codes(w.rank, o_summ[bt[p], h], B)
+                    for l in range(w.rank):
+                        if int(np.dot(gV[l], oV[l])) < 0:
+                            gV[l] = -gV[l]; gC[:, l] = -gC[:, l]
+                    for a_, b_ in ((gV, oV), (gC, oC), (gMu, oMu)):
+                        d = np.abs(a_ - b_)
+                        tot += d.size; diff += int((d > 0).sum())
+                        assert d.max() <= 1
+                    assert np.all(np.abs(gsV - osV) <= np.spacing(np.float16(osV)).astype(np.float64))
+                    assert np.all(np.abs(gsC - osC) <= np.spacing(np.float16(osC)).astype(np.float64))
+        assert diff / tot <= 2e-3, diff / tot
     # the partial last page of request 0 and 2 was not built
     assert gc.status() == 0
     check_select_and_attend(gc, o_summ, out_tol=1e-4 if dtype == "f32" else 2e-2)
@@ -101,7 +119,5 @@ def test_wide_page_decode_step_crosses_page_boundaries(B):
 def test_wide_pages_refuse_what_they_do_not_cover():
     import paper_2607_24555_b200 as locks
     from paper_2607_24555_b200.binding import make_config
-    with pytest.raises(locks.LocksError):
-        locks.Context(make_config(8, 2, 8, "i4", "bf16", 1, 64, 256, B=32))      # the int4 blob is laid out for 16 tokens
     with pytest.raises(locks.LocksError):
         locks.Context(make_config(8, 2, 8, "f32", "f32", 1, 64, 256, B=48))

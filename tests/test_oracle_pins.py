@@ -217,22 +217,28 @@ def test_half_conversion_matches_numpy():
             assert oracle.half_to_double(bits) == float(ref)
 
 
+@pytest.mark.parametrize("B", [16, 32, 64])
 @pytest.mark.parametrize("r", [2, 4, 8])
-def test_i4_pack_roundtrip_and_quantiser(r):
-    keys = low_rank_page(6, noise=0.2, seed=40 + r) + 3.0
+def test_i4_pack_roundtrip_and_quantiser(r, B):
+    """(B = 32, 64: the page sizes of the paper's App. D ablation; same quantiser, coefficients stored row-major.)"""
+    g = np.random.default_rng(40 + r + B)
+    keys = (low_rank_page(6, noise=0.2, seed=40 + r) + 3.0) if B == 16 else \
+        (g.standard_normal((B, 6)) @ g.standard_normal((6, 128)) * 2.0 + 0.2 * g.standard_normal((B, 128)) + 3.0)
     mu, V, C, _, _ = oracle.build_page(keys, r)
+    assert C.shape == (B, r)
     blob = oracle.pack(oracle.FMT_I4, mu, V, C)
-    assert blob.size == oracle.summary_stride_bytes(oracle.FMT_I4, r)
-    assert np.all(blob[oracle.summary_payload_bytes(oracle.FMT_I4, r):] == 0)
-    cV, cC, cMu, sV, sC, sMu = oracle.unpack_codes(r, blob)
-    mu2, V2, C2 = oracle.unpack(oracle.FMT_I4, r, blob)
+    assert blob.size == oracle.summary_stride_bytes(oracle.FMT_I4, r, B)
+    assert oracle.summary_payload_bytes(oracle.FMT_I4, r, B) == 128 * r // 2 + B * r + 128 + 2 * (r + B + 1)
+    assert np.all(blob[oracle.summary_payload_bytes(oracle.FMT_I4, r, B):] == 0)
+    cV, cC, cMu, sV, sC, sMu = oracle.unpack_codes(r, blob, B)
+    mu2, V2, C2 = oracle.unpack(oracle.FMT_I4, r, blob, B)
     assert np.abs(cV).max() <= 7 and np.abs(cC).max() <= 127 and np.abs(cMu).max() <= 127
     for l in range(r):   # one fp16 scale per basis column, abs-max symmetric, round-half-even codes
         assert sV[l] == float(np.float16(np.abs(V[l]).max() / 7))
         assert np.array_equal(cV[l], np.clip(np.rint(V[l] / sV[l]), -7, 7))
         assert np.allclose(V2[l], cV[l] * sV[l], rtol=0, atol=0)
         assert np.abs(V2[l] - V[l]).max() <= 0.5 * sV[l] * (1 + 1e-3) + 1e-12
-    for i in range(16):  # one scale per coefficient row
+    for i in range(B):  # one scale per coefficient row
         assert sC[i] == float(np.float16(np.abs(C[i]).max() / 127))
         assert np.array_equal(cC[i], np.clip(np.rint(C[i] / sC[i]), -127, 127))
         assert np.array_equal(C2[i], cC[i] * sC[i])
@@ -241,11 +247,11 @@ def test_i4_pack_roundtrip_and_quantiser(r):
     assert np.array_equal(mu2, cMu * sMu)
 
 
-@pytest.mark.parametrize("r", [2, 4, 8])
-def test_i4_layout_is_a_bijection(r):
+@pytest.mark.parametrize("r,B", [(2, 16), (4, 16), (8, 16), (8, 32), (4, 64)])
+def test_i4_layout_is_a_bijection(r, B):
     """Every payload byte/nibble is owned by exactly one entry: flipping one entry changes exactly
     one nibble (basis) or one byte (coefficients, centroid) and nothing else."""
-    V = np.zeros((r, 128)); C = np.zeros((16, r)); mu = np.zeros(128)
+    V = np.zeros((r, 128)); C = np.zeros((B, r)); mu = np.zeros(128)
     V[:, 0] = 7.0; C[:, 0] = 127.0; mu[0] = 127.0       # fixes every scale at 1.0
     base = oracle.pack(oracle.FMT_I4, mu, V, C)
     seen = set()
@@ -258,7 +264,7 @@ def test_i4_layout_is_a_bijection(r):
             key = (int(diff[0]), "lo" if b < 16 else "hi")
             assert key not in seen
             seen.add(key)
-    for i in range(16):
+    for i in range(B):
         for l in range(1, r):
             C2 = C.copy(); C2[i, l] = 5.0
             diff = np.nonzero(oracle.pack(oracle.FMT_I4, mu, V, C2) != base)[0]
