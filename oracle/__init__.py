@@ -286,6 +286,16 @@ def select(cache: Cache, shat, k: int):
     return ids, cnt, logshare
 
 
+def select_per_head(cache: Cache, shat, k: int):
+    """Per-head arm of the combine ablation: ids [batch, Hq, k], count [batch, Hq], log share [batch, Hq, max_pages]."""
+    shat = _f64(shat)
+    ids = np.full((cache.batch, cache.Hq, k), -1, np.int32)
+    cnt = np.zeros((cache.batch, cache.Hq), np.int32)
+    logshare = np.full((cache.batch, cache.Hq, cache.max_pages), np.nan)
+    lib().ora_select_per_head(cache.ref(), C.c_int(cache.batch), C.c_int(k), _p(shat), _p(ids), _p(cnt), _p(logshare))
+    return ids, cnt, logshare
+
+
 def page_exact_mass_all(cache: Cache, q, sm_scale: float):
     """Exact log-mass of every page 0..P-1 (last page over its valid tokens): [batch, Hq, max_pages]."""
     q, qd = _q_arg(q)
@@ -307,7 +317,8 @@ def selection_quality(s, P: int, A, R, marked=()):
     return tuple(float(x) for x in out)
 
 
-def attend(cache: Cache, q, sm_scale: float, page_ids=None, page_count=None):
+def attend(cache: Cache, q, sm_scale: float, page_ids=None, page_count=None, per_head: bool = False):
+    """per_head: page_ids [batch, Hq, k] / page_count [batch, Hq] (one table per query head) instead of per KV head."""
     q, qd = _q_arg(q)
     out = np.zeros((cache.batch, cache.Hq, cache.d))
     lse = np.zeros((cache.batch, cache.Hq))
@@ -316,8 +327,9 @@ def attend(cache: Cache, q, sm_scale: float, page_ids=None, page_count=None):
         page_ids = np.ascontiguousarray(page_ids, dtype=np.int32)
         page_count = np.ascontiguousarray(page_count, dtype=np.int32)
         k = page_ids.shape[-1]
-    lib().ora_attend(cache.ref(), C.c_int(cache.batch), _p(q), C.c_int(qd), C.c_double(sm_scale), C.c_int(k),
-                     _p(page_ids), _p(page_count), _p(out), _p(lse))
+    fn = lib().ora_attend_per_head if (per_head and page_ids is not None) else lib().ora_attend
+    fn(cache.ref(), C.c_int(cache.batch), _p(q), C.c_int(qd), C.c_double(sm_scale), C.c_int(k),
+       _p(page_ids), _p(page_count), _p(out), _p(lse))
     return out, lse
 
 

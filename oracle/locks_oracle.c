@@ -777,17 +777,32 @@ void ora_select(const ora_kv *kv, int batch, int k, const double *shat, int32_t 
                                         logshare ? logshare + prob * kv->max_pages : NULL);
     }
 }
+/* Per-head arm: every query head ranks the pages by its own share and keeps its own k pages (a group of one):
+ * page_ids [batch][Hq][k], page_count [batch][Hq], logshare [batch][Hq][max_pages] = log share of the head. */
+void ora_select_per_head(const ora_kv *kv, int batch, int k, const double *shat, int32_t *page_ids,
+                         int32_t *page_count, double *logshare) {
+#pragma omp parallel for collapse(2) num_threads(g_threads) schedule(dynamic)
+  for (int b = 0; b < batch; ++b)
+    for (int g = 0; g < kv->Hq; ++g) {
+      int P = num_pages(kv->seq_lens[b], kv->B);
+      int64_t row = (int64_t)b * kv->Hq + g;
+      page_count[row] = ora_select_one(P, 1, k, shat + row * kv->max_pages, kv->max_pages, page_ids + row * k,
+                                       logshare ? logshare + row * kv->max_pages : NULL);
+    }
+}
 
 /* Softmax attention of every query head over the tokens (< T) of the listed pages.
  * page_ids == NULL: every page (dense attention).  out[(b*Hq+g)*d + c], lse[b*Hq+g]. */
-void ora_attend(const ora_kv *kv, int batch, const void *q, int q_dtype, double sm_scale, int k,
-                const int32_t *page_ids, const int32_t *page_count, double *out, double *lse) {
+/* per_head = 0: one page table per (request, KV head), shared by the group's query heads (the method);
+ * per_head = 1: one page table per (request, query head) (the per-head arm of App. D's combine table). */
+static void attend_impl(const ora_kv *kv, int batch, const void *q, int q_dtype, double sm_scale, int k,
+                        const int32_t *page_ids, const int32_t *page_count, double *out, double *lse, int per_head) {
   int B = kv->B, d = kv->d, G = kv->Hq / kv->Hkv;
 #pragma omp parallel for collapse(2) num_threads(g_threads) schedule(dynamic)
   for (int b = 0; b < batch; ++b)
     for (int g = 0; g < kv->Hq; ++g) {
       int h = g / G, T = kv->seq_lens[b], P = num_pages(T, B);
-      int64_t prob = (int64_t)b * kv->Hkv + h;
+      int64_t prob = per_head ? (int64_t)b * kv->Hq + g : (int64_t)b * kv->Hkv + h;
       int npages = page_ids ? page_count[prob] : P;
       double *qd = (double *)malloc(sizeof(double) * d);
       double *x = (double *)malloc(sizeof(double) * (size_t)npages * B);
@@ -821,6 +836,15 @@ void ora_attend(const ora_kv *kv, int batch, const void *q, int q_dtype, double 
       if (lse) lse[(int64_t)b * kv->Hq + g] = mx + log(z);
       free(qd); free(x); free(tokpage); free(tokslot);
     }
+}
+void ora_attend(const ora_kv *kv, int batch, const void *q, int q_dtype, double sm_scale, int k,
+                const int32_t *page_ids, const int32_t *page_count, double *out, double *lse) {
+  attend_impl(kv, batch, q, q_dtype, sm_scale, k, page_ids, page_count, out, lse, 0);
+}
+/* Per-head arm (App. D, GQA combine table, "per-head" row): page_ids [batch][Hq][k], page_count [batch][Hq]. */
+void ora_attend_per_head(const ora_kv *kv, int batch, const void *q, int q_dtype, double sm_scale, int k,
+                         const int32_t *page_ids, const int32_t *page_count, double *out, double *lse) {
+  attend_impl(kv, batch, q, q_dtype, sm_scale, k, page_ids, page_count, out, lse, 1);
 }
 
 /* Exact log-mass of EVERY page 0..P-1 (the last page over its valid tokens), Lemma 1(ii):

@@ -581,6 +581,48 @@ def test_batch_wrappers_index_requests_heads_and_blocks(layout, bf16, fmt, r):
             assert np.allclose(dense[b, gq], o, atol=1e-12) and abs(dlse[b, gq] - l) < 1e-12
 
 
+def test_per_head_arm_selects_and_attends_head_by_head():
+    """The per-head arm of the combine ablation (App. D): every query head keeps the pages of its own largest shares
+    and attends them.  select_per_head equals select_one on a group of one, head by head; attend with per-head tables
+    equals a numpy softmax over exactly that head's pages, and equals the grouped call when the heads of a group are
+    handed the same table; heads of one group do end up with different pages here."""
+    cache, q_raw, q, page, lens, pages = ragged_batch_cache("NHD", True, seed=9)
+    B, d, Hkv, Hq, G, k, r, fmt = 16, 128, 2, 6, 3, 5, 8, oracle.FMT_I4
+    summ = oracle.build_summaries(cache, r, fmt)
+    shat = oracle.page_logmass(cache, q_raw, r, fmt, summ, SM)
+    ids, cnt, ls = oracle.select_per_head(cache, shat, k)
+    assert ids.shape == (3, Hq, k) and cnt.shape == (3, Hq) and ls.shape == (3, Hq, max(pages))
+    for b in range(3):
+        for gq in range(Hq):
+            i1, c1, l1 = oracle.select_one(shat[b, gq:gq + 1], pages[b], k)
+            assert cnt[b, gq] == c1 and np.array_equal(ids[b, gq], i1)
+            assert np.array_equal(ls[b, gq, 1:pages[b] - 1], l1[1:pages[b] - 1])
+            # a group of one: the key is the head's own log share
+            cand = shat[b, gq, 1:pages[b] - 1]
+            assert np.allclose(l1[1:pages[b] - 1], cand - (cand.max() + np.log(np.exp(cand - cand.max()).sum())), atol=1e-12)
+    assert any(len({tuple(ids[b, h * G + gi]) for gi in range(G)}) > 1 for b in range(3) for h in range(Hkv))
+    out, lse = oracle.attend(cache, q_raw, SM, ids, cnt, per_head=True)
+    for b in range(3):
+        for gq in range(Hq):
+            h = gq // G
+            ks, vs = [], []
+            for pg in ids[b, gq, :cnt[b, gq]]:
+                blk = int(cache.block_table[b, pg])
+                n = min(B, lens[b] - pg * B)
+                ks.append(page(cache.k, blk, h)[:n]); vs.append(page(cache.v, blk, h)[:n])
+            ks, vs = np.concatenate(ks), np.concatenate(vs)
+            x = ks @ q[b, gq] / math.sqrt(d)
+            wgt = np.exp(x - x.max())
+            assert np.allclose(out[b, gq], (wgt / wgt.sum()) @ vs, atol=1e-12)
+            assert abs(lse[b, gq] - (x.max() + math.log(wgt.sum()))) < 1e-12
+    gids, gcnt, _ = oracle.select(cache, shat, k)
+    rep_ids = np.repeat(gids, G, axis=1)
+    rep_cnt = np.repeat(gcnt, G, axis=1)
+    o1, l1 = oracle.attend(cache, q_raw, SM, gids, gcnt)
+    o2, l2 = oracle.attend(cache, q_raw, SM, rep_ids, rep_cnt, per_head=True)
+    assert np.array_equal(o1, o2) and np.array_equal(l1, l2)
+
+
 def test_build_summaries_page_ranges_per_request():
     """page_begin / page_end are per request: only the named complete pages are written."""
     cache, _, _, page, lens, pages = ragged_batch_cache()
