@@ -56,10 +56,16 @@ extern "C" {
  * page) is the same for all; page_logshare receives the key.
  *   LOCKS_COMBINE_SHARE_AVG   log mean_g exp(s^_j(q_g) - log Z_g): the paper's rule (Cor. 4)
  *   LOCKS_COMBINE_GROUP_MAX   max_g s^_j(q_g): the largest raw page log-mass of the group
- *   LOCKS_COMBINE_GROUP_MASS  log sum_g exp s^_j(q_g): the group's summed, un-normalised page mass */
+ *   LOCKS_COMBINE_GROUP_MASS  log sum_g exp s^_j(q_g): the group's summed, un-normalised page mass
+ *   LOCKS_COMBINE_PER_HEAD    no combine: every query head ranks by its own share and keeps its own k pages (the
+ *                             per-head arm of that table: up to G times the attention traffic).  page_ids is then
+ *                             [batch][Hq][k], page_count [batch][Hq], page_logshare [batch][Hq][max_pages_per_seq] in
+ *                             locks_select and locks_sparse_attend; locks_decode_step and the diagnostics that take a
+ *                             page table per KV head return UNSUPPORTED. */
 #define LOCKS_COMBINE_SHARE_AVG 0
 #define LOCKS_COMBINE_GROUP_MAX 1
 #define LOCKS_COMBINE_GROUP_MASS 2
+#define LOCKS_COMBINE_PER_HEAD 3
 
 typedef struct locks_ctx locks_ctx;
 typedef void *locks_stream; /* cudaStream_t */

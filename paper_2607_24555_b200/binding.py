@@ -149,7 +149,7 @@ def _stream(stream) -> int:
     return stream.cuda_stream
 
 
-COMBINE_SHARE_AVG, COMBINE_GROUP_MAX, COMBINE_GROUP_MASS = 0, 1, 2   # LOCKS_COMBINE_* of include/locks.h
+COMBINE_SHARE_AVG, COMBINE_GROUP_MAX, COMBINE_GROUP_MASS, COMBINE_PER_HEAD = 0, 1, 2, 3   # LOCKS_COMBINE_* of include/locks.h
 
 
 def make_config(Hq, Hkv, rank, fmt, dtype, max_batch, max_pages, budget, sm_scale=None, d=128, B=16,

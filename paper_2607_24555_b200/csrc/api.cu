@@ -17,7 +17,7 @@ int validate(const locks_config *c) {
   if (c->budget_tokens <= 0 || k < 2) return LOCKS_ERR_INVALID_ARG;
   if (!(c->sm_scale > 0.f)) return LOCKS_ERR_INVALID_ARG;
   if (c->summary_fmt < LOCKS_FMT_F32 || c->summary_fmt > LOCKS_FMT_BF16) return LOCKS_ERR_INVALID_ARG;
-  if (c->combine < LOCKS_COMBINE_SHARE_AVG || c->combine > LOCKS_COMBINE_GROUP_MASS) return LOCKS_ERR_INVALID_ARG;
+  if (c->combine < LOCKS_COMBINE_SHARE_AVG || c->combine > LOCKS_COMBINE_PER_HEAD) return LOCKS_ERR_INVALID_ARG;
   if ((c->kv_dtype != LOCKS_F32 && c->kv_dtype != LOCKS_BF16) || (c->q_dtype != LOCKS_F32 && c->q_dtype != LOCKS_BF16))
     return LOCKS_ERR_INVALID_ARG;
   if (c->head_dim != LOCKS_D) return LOCKS_ERR_UNSUPPORTED;
@@ -53,7 +53,8 @@ Layout make_layout(const locks_config *c) {
   // loads per thread beyond the first one and a half, plus 0.15 per 512 pages; the CTAs of a launch run in
   // waves of one per SM; the final ranking costs 3.3 plus 0.43 per 512 candidates.
   const int per_thread = (c->max_pages_per_seq + LOCKS_SEL_THREADS - 1) / LOCKS_SEL_THREADS;
-  const int64_t problems = (int64_t)c->max_batch * c->num_kv_heads;
+  // (per-head arm: one ranking per query head)
+  const int64_t problems = (int64_t)c->max_batch * (c->combine == LOCKS_COMBINE_PER_HEAD ? c->num_q_heads : c->num_kv_heads);
   const int kcand = L.k - 2 > 0 ? L.k - 2 : 1;
   L.sel_ept = LOCKS_SEL_MAX_EPT;
   if (problems >= 32 && per_thread <= LOCKS_SEL_MAX_EPT) {
@@ -86,16 +87,17 @@ Layout make_layout(const locks_config *c) {
   L.shat = take(nb * Hq * P * 4);
   L.part = take(nb * Hq * L.max_groups * 8);
   L.part_cnt = take(nb * Hkv * 4);
-  L.sel_done = take(nb * Hkv * 4);
-  L.cand_val = take(nb * Hkv * L.sel_chunks * L.sel_kc * 4);
-  L.cand_idx = take(nb * Hkv * L.sel_chunks * L.sel_kc * 4);
+  const size_t Hsel = c->combine == LOCKS_COMBINE_PER_HEAD ? Hq : Hkv;   // rankings per request
+  L.sel_done = take(nb * Hq * 4);
+  L.cand_val = take(nb * Hsel * L.sel_chunks * L.sel_kc * 4);
+  L.cand_idx = take(nb * Hsel * L.sel_chunks * L.sel_kc * 4);
   // split-K partial rows: batch * Hq * splits with splits <= slots / (batch * Hkv) (+1 rounding) and <= 128
   const size_t att_rows = (size_t)L.G * LOCKS_ATT_SLOT_BOUND + 2 * nb * Hq;
   L.att_o = take(att_rows * LOCKS_D * 4);
   L.att_lse = take(att_rows * 4);
-  L.att_done = take(nb * Hkv * 4);
-  L.ids = take(nb * Hkv * L.k * 4);
-  L.cnt = take(nb * Hkv * 4);
+  L.att_done = take(nb * Hq * 4);
+  L.ids = take(nb * Hsel * L.k * 4);
+  L.cnt = take(nb * Hsel * 4);
   L.sq = take(nb * Hq * LOCKS_D * esz);
   L.skn = take(nb * Hkv * LOCKS_D * esz);
   L.svn = take(nb * Hkv * LOCKS_D * esz);
@@ -205,8 +207,8 @@ int locks_create(const locks_config *cfg, void *workspace, size_t ws_bytes, lock
       cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
       cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) != cudaSuccess ||
       cudaMemsetAsync(c->status, 0, 64, 0) != cudaSuccess ||
-      cudaMemsetAsync(c->att_done, 0, (size_t)cfg->max_batch * cfg->num_kv_heads * 4, 0) != cudaSuccess ||
-      cudaMemsetAsync(c->sel_done, 0, (size_t)cfg->max_batch * cfg->num_kv_heads * 4, 0) != cudaSuccess ||
+      cudaMemsetAsync(c->att_done, 0, (size_t)cfg->max_batch * cfg->num_q_heads * 4, 0) != cudaSuccess ||
+      cudaMemsetAsync(c->sel_done, 0, (size_t)cfg->max_batch * cfg->num_q_heads * 4, 0) != cudaSuccess ||
       cudaMemsetAsync(c->part_cnt, 0, (size_t)cfg->max_batch * cfg->num_kv_heads * 4, 0) != cudaSuccess ||
       cudaStreamSynchronize(0) != cudaSuccess) {
     if (c->hint_host) cudaFreeHost(c->hint_host);
@@ -314,6 +316,7 @@ int locks_scan(locks_ctx *ctx, const void *q, const void *summaries, const locks
 int locks_select_scored(locks_ctx *ctx, const float *page_logmass, const float *head_logz_parts, int nparts,
                         const locks_kv *kv, int batch, int32_t *page_ids, int32_t *page_count, float *page_logshare,
                         locks_stream stream) {
+  if (ctx && ctx->cfg.combine == LOCKS_COMBINE_PER_HEAD) return LOCKS_ERR_UNSUPPORTED;   // one page table per KV head only
   if (ctx && ctx->B != LOCKS_B) return LOCKS_ERR_UNSUPPORTED;   // 16-token pages only
   int rc = check_common(ctx, kv, batch);
   if (rc != LOCKS_OK) return rc;
@@ -327,6 +330,7 @@ int locks_select_scored(locks_ctx *ctx, const float *page_logmass, const float *
 
 int locks_merge_selection(locks_ctx *ctx, const float *cand_key, const int32_t *cand_page, int nparts, int batch,
                           int32_t *page_ids, int32_t *page_count, locks_stream stream) {
+  if (ctx && ctx->cfg.combine == LOCKS_COMBINE_PER_HEAD) return LOCKS_ERR_UNSUPPORTED;   // one page table per KV head only
   if (ctx && ctx->B != LOCKS_B) return LOCKS_ERR_UNSUPPORTED;   // 16-token pages only
   if (!ctx || !cand_key || !cand_page || !page_ids || !page_count || nparts < 1 || batch < 1 || batch > ctx->cfg.max_batch)
     return LOCKS_ERR_INVALID_ARG;
@@ -368,6 +372,7 @@ int locks_select(locks_ctx *ctx, const void *q, const void *summaries, const loc
 
 int locks_select_exact(locks_ctx *ctx, const void *q, const locks_kv *kv, int batch, int32_t *page_ids,
                        int32_t *page_count, float *page_logmass, float *page_logshare, locks_stream stream) {
+  if (ctx && ctx->cfg.combine == LOCKS_COMBINE_PER_HEAD) return LOCKS_ERR_UNSUPPORTED;   // one page table per KV head only
   if (ctx && ctx->B != LOCKS_B) return LOCKS_ERR_UNSUPPORTED;   // 16-token pages only
   int rc = check_common(ctx, kv, batch);
   if (rc != LOCKS_OK) return rc;
@@ -382,6 +387,7 @@ int locks_select_exact(locks_ctx *ctx, const void *q, const locks_kv *kv, int ba
 int locks_select_rival(locks_ctx *ctx, int scorer, const void *q, const void *summaries, const locks_kv *kv, int batch,
                        int32_t *page_ids, int32_t *page_count, float *page_score, float *page_logshare,
                        locks_stream stream) {
+  if (ctx && ctx->cfg.combine == LOCKS_COMBINE_PER_HEAD) return LOCKS_ERR_UNSUPPORTED;   // one page table per KV head only
   if (ctx && ctx->B != LOCKS_B) return LOCKS_ERR_UNSUPPORTED;   // 16-token pages only
   int rc = check_common(ctx, kv, batch);
   if (rc != LOCKS_OK) return rc;
@@ -407,6 +413,7 @@ int locks_selection_quality(locks_ctx *ctx, const float *exact_logmass, const lo
                             const int32_t *page_ids, const int32_t *page_count, const int32_t *ref_ids,
                             const int32_t *ref_count, const int32_t *marked_pages, int n_marked, float *quality,
                             locks_stream stream) {
+  if (ctx && ctx->cfg.combine == LOCKS_COMBINE_PER_HEAD) return LOCKS_ERR_UNSUPPORTED;   // one page table per KV head only
   if (ctx && ctx->B != LOCKS_B) return LOCKS_ERR_UNSUPPORTED;   // 16-token pages only
   int rc = check_common(ctx, kv, batch);
   if (rc != LOCKS_OK) return rc;
@@ -431,6 +438,7 @@ int locks_sparse_attend(locks_ctx *ctx, const void *q, const locks_kv *kv, int b
 int locks_decode_step(locks_ctx *ctx, const void *q, const void *k_new, const void *v_new, locks_kv *kv,
                       void *summaries, int batch, void *out, int32_t *page_ids, int32_t *page_count,
                       locks_stream stream) {
+  if (ctx && ctx->cfg.combine == LOCKS_COMBINE_PER_HEAD) return LOCKS_ERR_UNSUPPORTED;   // one page table per KV head only
   int rc = check_common(ctx, kv, batch);
   if (rc != LOCKS_OK) return rc;
   if (!q || !summaries || !out || ((k_new == nullptr) != (v_new == nullptr)) || ((uintptr_t)summaries % 16) ||

@@ -29,6 +29,7 @@ struct AttParams {
   int32_t *done;   // [batch*Hkv] split-arrival counters (zero between launches)
   int batch, Hq, Hkv, G, Pmax, kbud, num_blocks, splits, pages_per_cta;
   int B;             // tokens per page (the bf16 kernels: 16 only)
+  int kvdiv;         // the KV head of problem h is h / kvdiv (1; per-head page tables: G, with G = 1 and Hkv = Hq here)
   int fused_merge;   // 1: the last CTA of a problem merges its splits; 0: a separate merge kernel follows
   int cluster;       // 1: the splits of a problem form one thread-block cluster and merge through its shared memory
   float sm_scale;
@@ -74,6 +75,7 @@ __global__ void __launch_bounds__(LOCKS_ATT_WARPS * 32) attend_bf16_kernel(AttPa
   const int x = lane >> 2, t = lane & 3;
   const int split = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
   const int64_t prob = (int64_t)b * p.Hkv + h;
+  const int hkv = h / p.kvdiv;   // head of the cache this problem reads
   uint8_t *ring = smem + warp * kAttStages * kAttStage;
   const uint8_t *Kb = reinterpret_cast<const uint8_t *>(p.k);
   const uint8_t *Vb = reinterpret_cast<const uint8_t *>(p.v);
@@ -140,7 +142,7 @@ __global__ void __launch_bounds__(LOCKS_ATT_WARPS * 32) attend_bf16_kernel(AttPa
     const int block = __shfl_sync(0xffffffffu, blk_cur, j & 31);
     const int ntok = __shfl_sync(0xffffffffu, nt_cur, j & 31);
     uint8_t *kt = ring + stage * kAttStage, *vt = kt + kTile;
-    const int64_t base = ((int64_t)block * p.sb + (int64_t)h * p.sh) * 2 + goff0;
+    const int64_t base = ((int64_t)block * p.sb + (int64_t)hkv * p.sh) * 2 + goff0;
     const uint8_t *kp = Kb + base, *vp = Vb + base;
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
@@ -459,7 +461,7 @@ __global__ void __launch_bounds__(128) attend_generic_kernel(AttParams p) {
   for (int idx = lo + warp; idx < hi; idx += 4) {
     int block, ntok;
     if (!resolve_page(p, b, prob, idx, Tn, block, ntok)) continue;
-    const int64_t base = (int64_t)block * p.sb + (int64_t)h * p.sh;
+    const int64_t base = (int64_t)block * p.sb + (int64_t)(h / p.kvdiv) * p.sh;
     for (int i = 0; i < ntok; ++i) {
       float s = 0.f;
 #pragma unroll
@@ -593,7 +595,10 @@ int locks_launch_attend(locks_ctx *c, const void *q, const locks_kv *kv, int bat
   p.block_table = kv->block_table; p.seq_lens = kv->seq_lens; p.ids = ids; p.cnt = cnt;
   p.part_o = c->att_o; p.part_lse = c->att_lse; p.out = out; p.lse = lse; p.status = c->status;
   p.batch = batch; p.Hq = c->cfg.num_q_heads; p.Hkv = c->cfg.num_kv_heads; p.G = c->G; p.Pmax = c->Pmax;
-  p.kbud = c->k; p.num_blocks = kv->num_blocks; p.sm_scale = c->cfg.sm_scale; p.B = c->B;
+  p.kbud = c->k; p.num_blocks = kv->num_blocks; p.sm_scale = c->cfg.sm_scale; p.B = c->B; p.kvdiv = 1;
+  if (c->cfg.combine == LOCKS_COMBINE_PER_HEAD && ids) {   // one page table per query head: groups of one
+    p.kvdiv = p.G; p.Hkv = p.Hq; p.G = 1;
+  }
   const bool dense = ids == nullptr;
   // one wave: as many splits per problem as resident CTA slots allow, at least one page per warp
   const int npages = dense ? c->Pmax : c->k;
@@ -612,7 +617,7 @@ int locks_launch_attend(locks_ctx *c, const void *q, const locks_kv *kv, int bat
   p.done = c->att_done;
   // a single CTA merging many splits of many heads is a serial tail: beyond 64 (head, split) pairs use the
   // parallel merge kernel instead
-  p.fused_merge = (c->G * p.splits <= 64) ? 1 : 0;
+  p.fused_merge = (p.G * p.splits <= 64) ? 1 : 0;
   // Preferred: the splits of a problem as one thread-block cluster (2, 4, 8 or 16 CTAs) that merges through
   // distributed shared memory, as long as a CTA then has at most 8 pages per warp to stream.
   p.cluster = 0;
@@ -663,14 +668,14 @@ int locks_launch_attend(locks_ctx *c, const void *q, const locks_kv *kv, int bat
     const bool contig = kv->stride_token == LOCKS_D;
     const dim3 blk(LOCKS_ATT_WARPS * 32);
     if (p.cluster) {
-      if (c->G <= 8) {
+      if (p.G <= 8) {
         if (contig) locks_launch_pdl_cluster(attend_bf16_kernel<1, true>, grid, blk, kAttSmem, p.splits, st, p);
         else locks_launch_pdl_cluster(attend_bf16_kernel<1, false>, grid, blk, kAttSmem, p.splits, st, p);
       } else {
         if (contig) locks_launch_pdl_cluster(attend_bf16_kernel<2, true>, grid, blk, kAttSmem, p.splits, st, p);
         else locks_launch_pdl_cluster(attend_bf16_kernel<2, false>, grid, blk, kAttSmem, p.splits, st, p);
       }
-    } else if (c->G <= 8) {
+    } else if (p.G <= 8) {
       if (contig) locks_launch_pdl(attend_bf16_kernel<1, true>, grid, blk, kAttSmem, st, p);
       else locks_launch_pdl(attend_bf16_kernel<1, false>, grid, blk, kAttSmem, st, p);
     } else {
@@ -765,7 +770,7 @@ extern "C" int locks_sparse_attend_noalloc(const locks_config *cfg, const void *
   p.status = reinterpret_cast<int32_t *>(nd.scratch + kNoAllocO + kNoAllocLse + kNoAllocDone);
   p.out = out; p.lse = lse;
   p.batch = batch; p.Hq = cfg->num_q_heads; p.Hkv = cfg->num_kv_heads; p.G = G; p.Pmax = cfg->max_pages_per_seq;
-  p.kbud = (cfg->budget_tokens + LOCKS_B - 1) / LOCKS_B; p.num_blocks = kv->num_blocks; p.sm_scale = cfg->sm_scale; p.B = LOCKS_B;
+  p.kbud = (cfg->budget_tokens + LOCKS_B - 1) / LOCKS_B; p.num_blocks = kv->num_blocks; p.sm_scale = cfg->sm_scale; p.B = LOCKS_B; p.kvdiv = 1;
   const int npages = page_ids ? p.kbud : p.Pmax;
   int splits = nd.num_sms * LOCKS_ATT_CTAS_PER_SM / (batch * p.Hkv);
   const int most = (npages + LOCKS_ATT_WARPS - 1) / LOCKS_ATT_WARPS;

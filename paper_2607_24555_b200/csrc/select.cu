@@ -29,6 +29,7 @@ struct SelParams {
   const float2 *part;
   const int32_t *seq_lens;
   const int32_t *part_cnt;   // partials per head of each problem, or nullptr: part_slots for all
+  int pc_div;                // rankings per entry of part_cnt (1; per-head arm: G)
   int32_t *ids, *cnt;
   float *logshare;
   uint32_t *cand_key;  // [batch][Hkv][chunks][kc] chunk lists (chunked selection only): keys, 0 = no entry
@@ -455,7 +456,7 @@ __global__ void __launch_bounds__(LOCKS_SEL_THREADS, 2) select_kernel(SelParams 
     const float *shat0 = p.shat + ((int64_t)b * p.Hq + h * p.G) * p.Pmax;
     const float2 *part0 = p.part + ((int64_t)b * p.Hq + h * p.G) * p.max_groups;
     float *ls0 = p.logshare ? p.logshare + prob * p.Pmax : nullptr;
-    const int nparts = p.part_cnt ? min(max(p.part_cnt[prob], 0), p.max_groups)
+    const int nparts = p.part_cnt ? min(max(p.part_cnt[prob / p.pc_div], 0), p.max_groups)
                                   : min(p.part_slots, (P - 1 + LOCKS_GROUP - 1) / LOCKS_GROUP);
     if (nslab >= 3) chunk_keys<4>(shat0, part0, ls0, p.G, p.Pmax, p.max_groups, nparts, c0, nslab, P, p.combine);
     else if (nslab == 2) chunk_keys<2>(shat0, part0, ls0, p.G, p.Pmax, p.max_groups, nparts, c0, nslab, P, p.combine);
@@ -606,6 +607,11 @@ int locks_launch_select(locks_ctx *c, const float *shat, const locks_kv *kv, int
   p.chunk_pages = c->sel_ept * LOCKS_SEL_THREADS;
   p.part_slots = c->part_slots;
   p.combine = c->cfg.combine;
+  p.pc_div = 1;
+  if (p.combine == LOCKS_COMBINE_PER_HEAD) {   // every query head is a group of one with a page table of its own
+    if (app) return LOCKS_ERR_UNSUPPORTED;
+    p.pc_div = p.G; p.Hkv = p.Hq; p.G = 1; p.combine = LOCKS_COMBINE_SHARE_AVG;
+  }
   p.Bshift = c->B == 64 ? 6 : (c->B == 32 ? 5 : 4);
   p.part_cnt = c->part_balanced ? c->part_cnt : nullptr;
   if (p.chunk_pages > kMaxKeys || (int64_t)c->sel_chunks * c->sel_kc > kMaxKeys || p.G > 16) return LOCKS_ERR_UNSUPPORTED;

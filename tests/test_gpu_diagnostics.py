@@ -125,6 +125,61 @@ def test_combine_rule_switch_matches_oracle(rule, lens, Hq, Hkv):
     check_page_sets(ids.cpu().numpy(), cnt.cpu().numpy(), oids, ocnt, okey, gc.cache.seq_lens, w.B, gc.k)
 
 
+@pytest.mark.parametrize("lens,Hq,Hkv,dtype,fmt,part", [([16 * 700 + 5, 16 * 90, 16 * 300], 8, 2, "bf16", "i4", 1),
+                                                        ([16 * 9000 + 3], 32, 2, "bf16", "i4", 1),
+                                                        ([16 * 500 + 9, 16 * 64], 4, 1, "f32", "f32", 1),
+                                                        ([16 * 2000 + 5, 16 * 90, 16 * 700, 16 * 31], 8, 2, "bf16", "i4", 2)])
+def test_per_head_arm_matches_oracle(lens, Hq, Hkv, dtype, fmt, part):
+    """The per-head arm of the paper's combine ablation: every query head ranks by its own share, keeps its own k
+    pages and attends them (one page table per query head).  Keys, page sets and attention outputs against the
+    oracle; single- and multi-chunk selection, both scan partitions, the tensor-core and the plain attention kernels;
+    calls that need one table per KV head refuse the configuration."""
+    import paper_2607_24555_b200 as locks
+    from paper_2607_24555_b200.binding import make_config
+    gc = _gc(locks_synth.Workload("perhead", lens, Hq=Hq, Hkv=Hkv, budget=256, q_scale=0.5, dtype=dtype, fmt=fmt, seed=Hq + len(lens)))
+    w = gc.w
+    cfg = make_config(w.Hq, w.Hkv, w.rank, w.fmt, w.dtype, w.n, gc.max_pages, w.budget, combine=locks.COMBINE_PER_HEAD)
+    ctx = locks.Context(cfg)
+    ctx.locks_set_scan_partition(part)
+    summ_np = gc.oracle_summaries()
+    summ = torch.from_numpy(summ_np).cuda()
+    ids = torch.full((w.n, w.Hq, gc.k), -7, dtype=torch.int32, device="cuda:0")
+    cnt = torch.full((w.n, w.Hq), -7, dtype=torch.int32, device="cuda:0")
+    key = torch.full((w.n, w.Hq, gc.max_pages), float("nan"), dtype=torch.float32, device="cuda:0")
+    ctx.locks_select(gc.case.q, summ, gc.kv, w.n, ids, cnt, None, key)
+    torch.cuda.synchronize()
+    assert ctx.locks_poll_status() == 0
+    qn = t2np(gc.case.q)
+    shat = oracle.page_logmass(gc.cache, qn, w.rank, gc.fmt, summ_np, gc.sm)
+    oids, ocnt, okey = oracle.select_per_head(gc.cache, shat, gc.k)
+    for b in range(w.n):
+        P = -(-w.seq_lens[b] // w.B)
+        if P > gc.k:
+            assert np.abs(key[b, :, 1:P - 1].cpu().numpy() - okey[b, :, 1:P - 1]).max() <= 1e-3
+    # the tie-aware set check treats every (request, query head) as a problem: a view with Hq "KV heads"
+    check_page_sets(ids.cpu().numpy(), cnt.cpu().numpy(), oids, ocnt, okey, gc.cache.seq_lens, w.B, gc.k)
+    if w.Hq > w.Hkv:
+        G = w.Hq // w.Hkv
+        assert any(len({tuple(r) for r in ids[b, h * G:(h + 1) * G].cpu().tolist()}) > 1 for b in range(w.n) for h in range(w.Hkv))
+    out = torch.full((w.n, w.Hq, w.d), float("nan"), dtype=gc.case.q.dtype, device="cuda:0")
+    lse = torch.full((w.n, w.Hq), float("nan"), dtype=torch.float32, device="cuda:0")
+    ctx.locks_sparse_attend(gc.case.q, gc.kv, w.n, ids, cnt, out, lse)
+    torch.cuda.synchronize()
+    assert ctx.locks_poll_status() == 0
+    oout, olse = oracle.attend(gc.cache, qn, gc.sm, ids.cpu().numpy(), cnt.cpu().numpy(), per_head=True)
+    assert np.abs(out.float().cpu().numpy() - oout).max() <= (2e-2 if dtype == "bf16" else 1e-4)
+    assert np.abs(lse.cpu().numpy() - olse).max() <= 1e-3
+    # dense mode is unchanged by the rule
+    dout = torch.empty_like(out)
+    ctx.locks_sparse_attend(gc.case.q, gc.kv, w.n, None, None, dout)
+    torch.cuda.synchronize()
+    dref, _ = oracle.attend(gc.cache, qn, gc.sm)
+    assert np.abs(dout.float().cpu().numpy() - dref).max() <= (2e-2 if dtype == "bf16" else 1e-4)
+    kn, vn, q1 = locks_synth.new_token(w, 0, device="cuda:0")
+    with pytest.raises(locks.LocksError):
+        ctx.locks_decode_step(q1, kn, vn, gc.kv, summ, w.n, out, ids, cnt)
+
+
 @pytest.mark.parametrize("scorer", [1, 2, 3])
 @pytest.mark.parametrize("fmt,dtype,Hq,Hkv", [("i4", "bf16", 8, 2), ("f32", "f32", 4, 1), ("i4", "bf16", 32, 2)])
 def test_rival_scorers_match_oracle(scorer, fmt, dtype, Hq, Hkv):
