@@ -100,7 +100,8 @@ typedef struct {
 } locks_kv;
 
 /* Bytes of one stored summary, per (physical block, KV head), padded to a multiple of 16.
- * I4 format: 82 r + 162 payload bytes at B=16, d=128 (978 / 1298 at r = 8, B = 32 / 64; 818 / 490 / 326 at r = 8 / 4 / 2: the
+ * I4 format: 82 r + 162 payload bytes at B=16, d=128 (978 / 1298 at r = 8, B = 32 / 64;
+ * 818 / 490 / 326 at r = 8 / 4 / 2: the
  * paper's stored-payload table, App. C.1), i.e. d r/2 int4 basis + B r int8 coefficients + d int8
  * centroid + (r + B + 1) fp16 scales (Sec. 4 "Build").  F32 format: 4 (d + r d + B r).  I8 format: d r + B r + d +
  * 2 (r + B + 1).  BF16 format: 2 d r + B r + d + 2 (B + 1).  The last two are plain row-major:
@@ -117,9 +118,10 @@ size_t locks_workspace_bytes(const locks_config *cfg);
  * small async memset on the default stream followed by a synchronise).  The context is a small
  * host object; *out must be released with locks_destroy().  Errors: INVALID_ARG (bad field, NULL),
  * UNSUPPORTED (shape the kernels do not cover: d != 128, B not in {16, 32, 64}, G > 16, mixed dtypes, I4 rank not
- * in {2,4,8}), WORKSPACE (ws_bytes too small or misaligned).  Pages of 32 and 64 tokens run build, select, attend and the decode step on plain fp32 kernels (no
- * tensor-core path); the diagnostics, the KV fake quantiser, the page-sharded calls, the multi-layer build and the
- * allocation-free attention entry point return UNSUPPORTED for them. */
+ * in {2,4,8}), WORKSPACE (ws_bytes too small or misaligned).  Pages of 32 and 64 tokens run build, select, attend
+ * and the decode step on plain fp32 kernels (no tensor-core path); the diagnostics, the KV fake quantiser, the
+ * page-sharded calls, the multi-layer build and the allocation-free attention entry point return UNSUPPORTED for
+ * them. */
 int locks_create(const locks_config *cfg, void *workspace, size_t ws_bytes, locks_ctx **out);
 int locks_destroy(locks_ctx *ctx);
 
