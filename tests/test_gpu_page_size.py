@@ -121,3 +121,10 @@ def test_wide_pages_refuse_what_they_do_not_cover():
     from paper_2607_24555_b200.binding import make_config
     with pytest.raises(locks.LocksError):
         locks.Context(make_config(8, 2, 8, "f32", "f32", 1, 64, 256, B=48))
+    # calls that exist for 16-token pages only say so instead of running
+    gc = _gc(_w(32, "i4", "bf16", [32 * 12 + 3]))
+    with pytest.raises(locks.LocksError):
+        gc.ctx.locks_fake_quantize_pages(gc.kv, 1, 4)
+    with pytest.raises(locks.LocksError):
+        gc.ctx.locks_build_summaries_layers(gc.kv, [gc.case.k], [gc.ctx.new_summaries(gc.case.num_blocks)], 1)
+    assert gc.status() == 0
