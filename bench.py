@@ -15,7 +15,8 @@ Prints ONE JSON line: metric / value / unit, the step time over exactly K replay
 three windows of 64 replays), `e2e` (the same step through the host-buffer entry point, copies included),
 `roofline` (scan kernel: algorithmic bytes / measured kernel time against the measured copy bandwidth, plus the
 kernel's DRAM traffic from the committed ncu capture), `cpu_baseline` (the oracle on the host cores), per-stage
-times, the dense flash-decode time on the same inputs, the bulk summary build, clocks, launch count, and
+times, the dense flash-decode time on the same inputs, the bulk summary build, `multi_layer_graph` (for information:
+the same steps with all layers in one graph), clocks, launch count, and
 `workloads`: a compact table (step, bytes, fraction of peak, dense) for one cell of each other configuration.  `--impl reference` times the CPU
 oracle instead (test infrastructure; the only other place this file runs it is `cpu_baseline`).
 """
@@ -226,7 +227,7 @@ def measure(args, w0, K, W, L, rank, local_rank, full):
 
     dev = f"cuda:{local_rank}"
     NW, WSTEPS = (3, 64) if (full and not args.no_windows) else (0, 0)
-    grow = (W + K + NW * WSTEPS + (K + 2) + (4 * L + K if full else 0)) // L + 24   # tokens appended per layer
+    grow = (W + K + NW * WSTEPS + (K + 2) + (4 * L + 3 * K if full else 0)) // L + 24   # tokens appended per layer
     reserve = -(-grow // w0.B) + 2
     layers = []
     for li in range(L):
@@ -346,6 +347,24 @@ def measure(args, w0, K, W, L, rank, local_rank, full):
         res["dense_ms"] = d0.elapsed_time(d1) / nd
         res["clocks"] = sampler.stop() if sampler else None
         if full:
+            # ---- for information: the same steps with all L layers captured in ONE graph, as a caller that batches a
+            # model's layers would launch them (the launch gap is paid once per L steps and the next scan is
+            # scheduled while the attention drains); not the headline, which keeps one graph per step
+            mg = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(mg, stream=stream):
+                for li in range(L):
+                    step(li)
+            reps = max(2, K // L)
+            mg.replay()
+            stream.synchronize()
+            m0, m1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            m0.record(stream)
+            for _ in range(reps):
+                mg.replay()
+            m1.record(stream)
+            stream.synchronize()
+            res["multi_layer_graph_us"] = m0.elapsed_time(m1) / (reps * L) * 1e3
+            del mg
             # ---- end to end through the host-buffer entry point: H2D of q, k_new, v_new and D2H of out every step
             hq = [n[2].cpu().pin_memory() for n in news]
             hk = [n[0].cpu().pin_memory() for n in news]
@@ -444,6 +463,7 @@ def run_ours(args):
         "step_roofline": {"algorithmic_bytes": scan_b + att_b, "achieved": (scan_b + att_b) / (step_ms_max * 1e-3) / 1e9,
                           "frac": (scan_b + att_b) / (step_ms_max * 1e-3) / 1e9 / peak, "unit": "GB/s",
                           "frac_of_8000": (scan_b + att_b) / (step_ms_max * 1e-3) / 1e9 / 8000.0},
+        "multi_layer_graph": {"layers_per_graph": L, "us_per_step": r.get("multi_layer_graph_us")},
         "windows": {"replays_per_window": 64, "us_per_step": [round(x, 3) for x in wins],
                     "mean_us": statistics.mean(wins) if wins else None,
                     "sd_us": statistics.stdev(wins) if len(wins) > 1 else None},
