@@ -531,6 +531,28 @@ def run_diagnostics(args):
             m = qual.mean(dim=(0, 1)).tolist()
             row["scorers"][label] = {"gamma": round(m[0], 4), "gamma_c": round(m[1], 4), "recall": round(m[2], 4),
                                      "needle": round(m[3], 4) if ncar else None}
+        # ---- the combine rules of the paper's GQA ablation (App. D) on the summary's scores: mass kept by each rule's
+        # page tables (mean over the query heads); the per-head arm keeps one table per query head
+        row["combine_rules"] = {}
+        if w.G > 1:
+            for label, rule in (("share_average", locks.COMBINE_SHARE_AVG), ("group_max", locks.COMBINE_GROUP_MAX),
+                                ("group_mass", locks.COMBINE_GROUP_MASS), ("per_head", locks.COMBINE_PER_HEAD)):
+                per_head = rule == locks.COMBINE_PER_HEAD
+                c2 = locks.Context(make_config(w.Hq, w.Hkv, w.rank, w.fmt, w.dtype, w.n, max_pages, w.budget, combine=rule), device=dev)
+                H = w.Hq if per_head else w.Hkv
+                ids = torch.zeros(w.n, H, w.k, dtype=torch.int32, device=dev)
+                cnt = torch.zeros(w.n, H, dtype=torch.int32, device=dev)
+                c2.locks_select(case.q, summ, kv, w.n, ids, cnt)
+                # the metrics kernel of a context whose groups are single heads reads a table per query head
+                cq = locks.Context(make_config(w.Hq, w.Hq, w.rank, w.fmt, w.dtype, w.n, max_pages, w.budget), device=dev) if per_head else ctx
+                qual = torch.zeros(w.n, H, 4, dtype=torch.float32, device=dev)
+                cq.locks_selection_quality(mass, kv, w.n, ids, cnt, ids, cnt, qual, marked_pages=marked)
+                torch.cuda.synchronize()
+                m = qual.mean(dim=(0, 1)).tolist()
+                row["combine_rules"][label] = {"gamma": round(m[0], 4), "gamma_c": round(m[1], 4)}
+                if per_head:
+                    cq.close()
+                c2.close()
         rows.append(row)
         ctx.close()
         del case, summ, mass
