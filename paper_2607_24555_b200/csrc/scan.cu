@@ -259,6 +259,7 @@ __device__ __forceinline__ void mma_f16_z(float (&d)[4], uint32_t a0, uint32_t a
 
 struct Cursor {
   int prob, grp, nsc, b, h;   // (request, KV head) of prob are refreshed only when prob changes
+  const int32_t *bt;          // block-table row of request b
 };
 
 // Four rows of a 2D tensor map (box = one row) to consecutive rows in shared memory, completion on an mbarrier.
@@ -342,7 +343,7 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4_kerne
   };
   int n_units = 0x7fffffff;   // balanced: units this warp owns
   int pslot_first = 0;        // balanced: partial slot of the first problem this warp touches
-  Cursor cp{slot, sub, 0, 0, 0};
+  Cursor cp{slot, sub, 0, 0, 0, p.block_table};
   if (BAL) {
     auto scan32 = [&](int v) {   // inclusive prefix sum over the lanes
 #pragma unroll
@@ -408,6 +409,7 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4_kerne
     const int T = step_len(p, c.b);
     const int P = (T + LOCKS_B - 1) / LOCKS_B;
     c.nsc = (P <= p.k) ? 0 : P - 1;
+    c.bt = p.block_table + (int64_t)c.b * p.Pmax;
   };
   auto settle = [&](Cursor &c) {  // move to the next non-empty position at or after (prob, grp)
     while (c.prob < nprob && c.grp * LOCKS_GROUP >= c.nsc) {
@@ -427,7 +429,7 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4_kerne
     if (c.prob >= nprob) return 0;
     const int page = c.grp * LOCKS_GROUP + lane;
     if (lane >= LOCKS_GROUP || page >= c.nsc) return 0;
-    return p.block_table[(int64_t)c.b * p.Pmax + page];
+    return c.bt[page];
   };
   auto issue = [&](int stage, const Cursor &c, int block) {
     const int h = c.h;
@@ -563,6 +565,9 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4_kerne
 #pragma unroll
   for (int hh = 0; hh < NH; ++hh) { pm[hh] = -INFINITY; ps[hh] = 0.f; }
   int cur_b = 0, cur_h = 0, cur_pslot = sub;   // partial slot of this warp in the current problem
+  float *srow[NH];                              // score row(s) of this lane's head(s) of the current problem
+#pragma unroll
+  for (int hh = 0; hh < NH; ++hh) srow[hh] = p.shat;
   auto accumulate = [&](float &m, float &sacc, float v) {   // online log-sum-exp, one exp per value
     // branch-free: a value of -inf (masked page) adds nothing, whatever m is (also -inf at the start)
     const bool live = v > -INFINITY;
@@ -611,6 +616,9 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4_kerne
       cur_b = b;
       cur_h = h;
       cur_pslot = BAL ? (it == 0 ? pslot_first : 0) : sub;
+#pragma unroll
+      for (int hh = 0; hh < NH; ++hh)
+        srow[hh] = p.shat + ((int64_t)b * p.Hq + h * p.G + (PK ? (x & 3) : x + 8 * hh)) * p.Pmax;
 #pragma unroll
       for (int hh = 0; hh < NH; ++hh) {
         float s8;
@@ -906,7 +914,7 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4_kerne
       const int g = x & 3, page = cc.grp * LOCKS_GROUP + 2 * t + (x >> 2);
       const float v = res[0] * kLn2;
       const bool in = t < LOCKS_GROUP / 2 && page < cc.nsc;
-      if (g < p.G && in) store_score(p.shat + ((int64_t)b * p.Hq + h * p.G + g) * p.Pmax + page, v);
+      if (g < p.G && in) store_score(srow[0] + page, v);
       accumulate(pm[0], ps[0], (in && page >= 1) ? v : -INFINITY);
     } else {
     const int page0 = cc.grp * LOCKS_GROUP + 2 * t;
@@ -917,7 +925,7 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4_kerne
       const float v1 = (res[2 * hh + 1] + acen[2 * hh + 1]) * kLn2;
       const bool in0 = t < LOCKS_GROUP / 2 && page0 < cc.nsc, in1 = t < LOCKS_GROUP / 2 && page0 + 1 < cc.nsc;
       if (g < p.G) {
-        float *dst = p.shat + ((int64_t)b * p.Hq + h * p.G + g) * p.Pmax + page0;
+        float *dst = srow[hh] + page0;
         if (in0) store_score(dst, v0);
         if (in1) store_score(dst + 1, v1);
       }
