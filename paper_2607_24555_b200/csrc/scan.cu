@@ -513,8 +513,8 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4_kerne
 
   // query of the current problem: qb0/qb2 = this lane's dims of head x (tile 0) / head x + 8 (tile 1)
   uint32_t qb0[NH][8], qb2[NH][8];
-  float inv_s[NH], ksum[2 * NH];   // 1/scale of head x (+8); 8 * sum_c q'[c] of heads 2t, 2t+1 (+8)
-  float inv2[2 * NH];              // 1/scale of heads 2t, 2t+1 (+8)
+  float inv_s[NH], ksum[2 * NH];   // c2 / scale of head x (+8); 8 * sum_c q'[c] of heads 2t, 2t+1 (+8)
+  float inv2[2 * NH];              // c2 / scale of heads 2t, 2t+1 (+8)
   int cur_prob = -1;
   const __nv_bfloat16 *q = reinterpret_cast<const __nv_bfloat16 *>(p.q);
   const float c2 = p.sm_scale * kLog2e;
@@ -627,6 +627,7 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4_kerne
         // lane (x, t) owns head gx; the column fragment needs the heads of columns 2t, 2t+1
         ksum[2 * hh] = __shfl_sync(0xffffffffu, s8, (2 * t) * 4);
         ksum[2 * hh + 1] = __shfl_sync(0xffffffffu, s8, (2 * t + 1) * 4);
+        inv_s[hh] *= c2;   // from here on: the factor that turns a scaled dot product into a log2-domain logit
         inv2[2 * hh] = __shfl_sync(0xffffffffu, inv_s[hh], (2 * t) * 4);
         inv2[2 * hh + 1] = __shfl_sync(0xffffffffu, inv_s[hh], (2 * t + 1) * 4);
       }
@@ -668,7 +669,7 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4_kerne
       const float smu = __half2float(*reinterpret_cast<const __half *>(sb + boff(x & (LOCKS_GROUP - 1)) + i4_off_smu(R)));
 #pragma unroll
       for (int hh = 0; hh < NH; ++hh) {
-        const float v0 = smu * (c2 * inv2[2 * hh]) * cenT[hh][0], v1 = smu * (c2 * inv2[2 * hh + 1]) * cenT[hh][1];
+        const float v0 = smu * inv2[2 * hh] * cenT[hh][0], v1 = smu * inv2[2 * hh + 1] * cenT[hh][1];
         if (PK) {   // lane (x, t) finishes page 2t + (x >> 2), head x & 3: held by lane (that page, (x & 3) >> 1)
           const int src = (2 * t + (x >> 2)) * 4 + ((x & 3) >> 1);
           const float a0 = __shfl_sync(0xffffffffu, v0, src), a1 = __shfl_sync(0xffffffffu, v1, src);
@@ -698,7 +699,7 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4_kerne
       // projection, one MMA per token half.  Rank 4: k = 4 a + rank, hi and lo in two MMAs.
       constexpr int PH = 8 / R;                 // pages per row half of MMA #1
       const int pr = x / R, lr = x % R;         // this lane's row: page within the half, rank
-      const float iv = inv_s[0] * c2;
+      const float iv = inv_s[0];
 #pragma unroll
       for (int k4 = 0; k4 < 2; ++k4) {          // pages 4 k4 .. 4 k4 + 3
         float prj[2][2];                        // rank 2: [k4 half][head e]; rank 4: [half of this chain][head e]
@@ -842,7 +843,7 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4_kerne
         mma_f16(cb, lA, 0u, lB, 0u, a1, b1);
         const uint2 scw = *reinterpret_cast<const uint2 *>((ra ? pbA : pbB) + i4_off_sc(R) + 8 * t);
         const float2 s01 = h2f2(scw.x), s89 = h2f2(scw.y);
-        const float iv = inv_s[0] * c2;
+        const float iv = inv_s[0];
         const float y0 = ca[0] * s01.x, y1 = ca[1] * s01.y, y2 = cb[0] * s89.x, y3 = cb[1] * s89.y;
         float my = fmaxf(fmaxf(y0, y1), fmaxf(y2, y3));
         my = fmaxf(my, __shfl_xor_sync(0xffffffffu, my, 1));
@@ -883,7 +884,7 @@ __global__ void __launch_bounds__(kScanWarps * 32, kScanCtasPerSm) scan_i4_kerne
         const float2 s01 = h2f2(scw.x), s89 = h2f2(scw.y);
 #pragma unroll
         for (int hh = 0; hh < NH; ++hh) {
-          const float iv = inv_s[hh] * c2;   // logits (log2 domain) are y * iv, iv > 0
+          const float iv = inv_s[hh];   // logits (log2 domain) are y * iv, iv > 0
           const float y0 = ca[2 * hh] * s01.x, y1 = ca[2 * hh + 1] * s01.y;
           const float y2 = cb[2 * hh] * s89.x, y3 = cb[2 * hh + 1] * s89.y;
           float my = fmaxf(fmaxf(y0, y1), fmaxf(y2, y3));
