@@ -35,6 +35,16 @@ def test_size_helpers_and_validation_need_no_gpu():
     assert locks.locks_workspace_bytes(make_config(32, 2, 8, "i4", "bf16", 1, 65536, 2048)) > 0
     assert locks.locks_workspace_bytes(make_config(34, 2, 8, "i4", "bf16", 1, 64, 256)) == 0    # G = 17
     assert locks.locks_workspace_bytes(make_config(8, 2, 8, "i4", "bf16", 1, 64, 256, d=64)) == 0
+    # page sizes of the paper's App. D ablation: 978 / 1298 payload bytes at r = 8 int4, padded to 16
+    assert locks.locks_summary_bytes(make_config(32, 8, 8, "i4", "bf16", 8, 2048, 2048, B=32)) == 992
+    assert locks.locks_summary_bytes(make_config(32, 8, 8, "i4", "bf16", 8, 2048, 2048, B=64)) == 1312
+    assert locks.locks_summary_bytes(make_config(4, 1, 8, "f32", "f32", 1, 256, 256, B=32)) == 4 * (128 + 8 * 128 + 32 * 8)
+    assert locks.locks_workspace_bytes(make_config(8, 2, 8, "i4", "bf16", 1, 64, 256, B=48)) == 0
+    # the per-head arm ranks and attends one page table per query head: its workspace is the larger one
+    grouped = locks.locks_workspace_bytes(make_config(32, 2, 8, "i4", "bf16", 1, 65536, 2048))
+    per_head = locks.locks_workspace_bytes(make_config(32, 2, 8, "i4", "bf16", 1, 65536, 2048, combine=locks.COMBINE_PER_HEAD))
+    assert per_head > grouped
+    assert locks.locks_workspace_bytes(make_config(32, 2, 8, "i4", "bf16", 1, 65536, 2048, combine=4)) == 0
     assert locks.locks_strerror(-6).startswith("page or block")
     assert locks.locks_strerror(0) == "ok"
 
